@@ -1,0 +1,323 @@
+"""Seeded synthetic workloads for the integer-only inference path of HAWQ-V3.
+
+This module only *draws inputs*: tensors, weights, INT32 biases, dyadic pairs and the layer
+tables of ResNet-shaped networks.  It contains none of the inference arithmetic (no convolution,
+no requantization, no pooling), and it imports neither the CUDA binding nor the CPU oracle; both
+consume what it produces, so generator details can never create a parity difference.
+
+Value ranges follow the paper's quantizers (Section 3 "Uniform Quantization", Appendix A/B):
+weights symmetric in [-(2^(k-1)-1), 2^(k-1)-1] per output channel, post-ReLU activations unsigned in
+[0, 2^k-1] with zero point 0, bias in INT32 at scale S_h*S_w (Appendix D), every rescaling a
+dyadic number b/2^c (Eq. 4 and the DN(.) definition).  Real-valued scales appear only here,
+offline, exactly as in the paper, where DN(.) is evaluated once from statically known scales
+(Section 3.3); the integer pipeline itself never sees them.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "rng", "dyadic_from_scale", "pack4", "unpack4", "conv_case", "config1_case",
+    "resnet_table", "table_cost", "out_hw", "SWEEP_LAYERS",
+]
+
+
+def rng(seed: int, *stream: int) -> np.random.Generator:
+    """Counter-based generator keyed by (seed, stream ids): the same key gives the same numbers."""
+    return np.random.Generator(np.random.Philox(key=np.random.SeedSequence([seed, *stream]).generate_state(2, np.uint64)))
+
+
+# --------------------------------------------------------------------------------------------
+# DN(.): real scale -> dyadic pair (offline; Section 3.1, equation after Eq. 4)
+# --------------------------------------------------------------------------------------------
+def dyadic_from_scale(s):
+    """Return int32 arrays (b, c) with b / 2^c ~= s, 2^30 <= b < 2^31 and 1 <= c <= 62.
+
+    The paper defines DN only by its result.  Reading used here: normalise s = m * 2^e with
+    m in [0.5, 1), take b = round_half_up(m * 2^31), c = 31 - e (and renormalise if b hits 2^31).
+    The error is at most 2^-(c+1).  Scales so small that c would pass 62 keep c = 62 and a
+    smaller b; scales of 2^30 and above are rejected.
+    """
+    s = np.atleast_1d(np.asarray(s, dtype=np.float64))
+    if np.any(~np.isfinite(s)) or np.any(s <= 0):
+        raise ValueError("scale must be finite and positive")
+    m, e = np.frexp(s)
+    b = np.floor(m * float(2 ** 31) + 0.5).astype(np.int64)
+    c = 31 - e.astype(np.int64)
+    carry = b == 2 ** 31
+    b[carry] = 2 ** 30
+    c[carry] -= 1
+    if np.any(c < 1):
+        raise ValueError("scale too large for a dyadic pair with c >= 1")
+    deep = c > 62
+    if np.any(deep):
+        sh = c[deep] - 62
+        b[deep] = (b[deep] + (1 << (sh - 1))) >> sh
+        c[deep] = 62
+    return b.astype(np.int32), c.astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------------
+# 4-bit packing (two per byte along the channel axis, even element in the low nibble)
+# --------------------------------------------------------------------------------------------
+def pack4(a: np.ndarray) -> np.ndarray:
+    """Pack integers in [-8, 15] (last axis even) into bytes, element 2j -> bits 3:0 of byte j."""
+    a = np.asarray(a)
+    if a.shape[-1] % 2:
+        raise ValueError("last axis must be even to pack 4-bit values")
+    u = (a.astype(np.int16) & 0xF).astype(np.uint8)
+    return (u[..., 0::2] | (u[..., 1::2] << 4)).astype(np.uint8)
+
+
+def unpack4(p: np.ndarray, signed: bool) -> np.ndarray:
+    """Inverse of pack4, returning int8 (signed) or uint8 values."""
+    p = np.asarray(p, dtype=np.uint8)
+    out = np.empty(p.shape[:-1] + (p.shape[-1] * 2,), dtype=np.int16)
+    out[..., 0::2] = p & 0xF
+    out[..., 1::2] = p >> 4
+    if signed:
+        out = np.where(out >= 8, out - 16, out)
+        return out.astype(np.int8)
+    return out.astype(np.uint8)
+
+
+def out_hw(h: int, w: int, k: int, stride: int, pad: int) -> tuple[int, int]:
+    return (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
+
+
+# --------------------------------------------------------------------------------------------
+# Single-layer cases (configs 1 and 5)
+# --------------------------------------------------------------------------------------------
+def conv_case(seed: int, n: int, h: int, w: int, cin: int, cout: int, k: int, stride: int = 1,
+              pad: int = 0, bits: int = 8, out_bits: int = 8, residual: bool = False,
+              res_bits: int = 8, relu: bool = True, in_signed: bool = False,
+              c_range: tuple[int, int] = (36, 44), out_signed: bool | None = None) -> dict:
+    """One fused conv layer with the value distributions of the single-layer benchmark config.
+
+    Activations uniform over the full unsigned (or signed) range, weights uniform symmetric,
+    bias uniform in [-2^15, 2^15], b uniform in [2^30, 2^31), c uniform in c_range, residual rescale
+    (when asked for) with c in [28, 34] so that both roundings and both signs of `c - 32` occur.
+    4-bit tensors are returned packed (last axis halved); `*_bits` say how to read them.
+    """
+    g = rng(seed, n, h, w, cin, cout, k, stride, pad, bits)
+    amax = (1 << bits) - 1
+    if in_signed:
+        x = g.integers(-(1 << (bits - 1)), 1 << (bits - 1), size=(n, h, w, cin), dtype=np.int64)
+    else:
+        x = g.integers(0, amax + 1, size=(n, h, w, cin), dtype=np.int64)
+    wmax = (1 << (bits - 1)) - 1
+    wt = g.integers(-wmax, wmax + 1, size=(cout, k, k, cin), dtype=np.int64)
+    bias = g.integers(-(1 << 15), (1 << 15) + 1, size=cout, dtype=np.int64).astype(np.int32)
+    b = g.integers(1 << 30, 1 << 31, size=cout, dtype=np.int64).astype(np.int32)
+    if bits == 4:
+        # 4-bit accumulators are ~2^9 times smaller; keep a comparable spread of outputs
+        c_lo, c_hi = c_range[0] - 8, c_range[1] - 8
+    else:
+        c_lo, c_hi = c_range
+    c = g.integers(c_lo, c_hi + 1, size=cout, dtype=np.int64).astype(np.int32)
+    ho, wo = out_hw(h, w, k, stride, pad)
+    if out_signed is None:
+        out_signed = not relu
+    if out_bits == 32:
+        qmin, qmax, out_signed = -(1 << 31), (1 << 31) - 1, True
+    elif out_signed:
+        qmin, qmax = -(1 << (out_bits - 1)), (1 << (out_bits - 1)) - 1
+    else:
+        qmin, qmax = 0, (1 << out_bits) - 1
+    case = dict(
+        n=n, h=h, w=w, cin=cin, cout=cout, kh=k, kw=k, stride=stride, pad=pad, bits=bits,
+        in_signed=int(in_signed), ho=ho, wo=wo,
+        x=(pack4(x) if bits == 4 else x.astype(np.int8 if in_signed else np.uint8)),
+        wgt=(pack4(wt) if bits == 4 else wt.astype(np.int8)),
+        bias=bias, b=b, c=c, relu=int(relu), qmin=qmin, qmax=qmax,
+        out_bits=out_bits, out_signed=int(out_signed),
+        res=None, res_bits=0, res_signed=0, rb=None, rc=None,
+    )
+    if residual:
+        if res_bits == 32:
+            r = g.integers(-(1 << 20), 1 << 20, size=(n, ho, wo, cout), dtype=np.int64).astype(np.int32)
+            rc = g.integers(40, 47, size=cout, dtype=np.int64).astype(np.int32)
+            case["res_signed"] = 1
+        else:
+            r = g.integers(0, 256, size=(n, ho, wo, cout), dtype=np.int64).astype(np.uint8)
+            rc = g.integers(28, 35, size=cout, dtype=np.int64).astype(np.int32)
+        case.update(res=r, res_bits=res_bits,
+                    rb=g.integers(1 << 30, 1 << 31, size=cout, dtype=np.int64).astype(np.int32), rc=rc)
+    return case
+
+
+def config1_case() -> dict:
+    """Benchmark config 1: batch 1, 56x56x64 -> 64, 3x3, stride 1, pad 1, seed 0, c in [36, 44]."""
+    return conv_case(0, 1, 56, 56, 64, 64, 3, stride=1, pad=1, bits=8, relu=True)
+
+
+# ResNet-50 layer shapes used by the conv/GEMM sweep (H=W, Cin, Cout, k, stride, has residual)
+SWEEP_LAYERS = [
+    (56, 64, 64, 1, 1, False), (56, 64, 64, 3, 1, False), (56, 64, 256, 1, 1, True),
+    (56, 256, 64, 1, 1, False), (28, 128, 128, 3, 1, False), (28, 128, 512, 1, 1, True),
+    (28, 512, 128, 1, 1, False), (14, 256, 256, 3, 1, False), (14, 256, 1024, 1, 1, True),
+    (14, 1024, 256, 1, 1, False), (7, 512, 512, 3, 1, False), (7, 512, 2048, 1, 1, True),
+    (7, 2048, 512, 1, 1, False),
+]
+
+
+# --------------------------------------------------------------------------------------------
+# Network tables (configs 2-4)
+# --------------------------------------------------------------------------------------------
+def _draw_scale(g: np.random.Generator) -> float:
+    """Activation scale, log-uniform in [2^-6, 2^-2): octave uniform in {-6..-3}, mantissa in [1,2)."""
+    e = int(g.integers(-6, -2))
+    return float(2.0 ** e * (1.0 + g.random()))
+
+
+def _draw_weights(g: np.random.Generator, cout: int, k: int, cin: int, bits: int):
+    """Real weights N(0, sqrt(2/fan_in)) quantized symmetrically per output channel (Appendix A)."""
+    fan_in = k * k * cin
+    wr = g.standard_normal(size=(cout, k, k, cin)) * np.sqrt(2.0 / fan_in)
+    wmax = (1 << (bits - 1)) - 1
+    s_w = np.abs(wr).reshape(cout, -1).max(axis=1) / wmax
+    q = np.floor(wr / s_w[:, None, None, None] + 0.5)
+    q = np.clip(q, -wmax, wmax).astype(np.int64)
+    return q, s_w
+
+
+class _Builder:
+    def __init__(self, seed: int):
+        self.g = rng(seed, 7)
+        self.layers: list[dict] = []
+        self.scale: dict[int, float] = {}
+        self.shape: dict[int, tuple[int, int, int]] = {}   # h, w, c of each tensor id
+        self.bits: dict[int, int] = {}
+
+    def _emit(self, layer: dict, scale: float, hwc, bits: int) -> int:
+        self.layers.append(layer)
+        tid = len(self.layers) - 1
+        self.scale[tid], self.shape[tid], self.bits[tid] = scale, hwc, bits
+        return tid
+
+    def conv(self, src: int, cout: int, k: int, stride: int, pad: int, bits: int, *, relu: bool,
+             out_bits: int, out_signed: bool = False, res: int = -1, op: str = "conv") -> int:
+        g = self.g
+        h, w, cin = self.shape[src]
+        assert self.bits[src] == bits, "conv input must already have the conv's bit-width"
+        q, s_w = _draw_weights(g, cout, k, cin, bits)
+        bias = g.integers(-(1 << 15), (1 << 15) + 1, size=cout, dtype=np.int64).astype(np.int32)
+        ho, wo = out_hw(h, w, k, stride, pad)
+        s_in = self.scale[src]
+        layer = dict(op=op, in0=src, in1=res, kh=k, kw=k, stride=stride, pad=pad, cin=cin, cout=cout,
+                     bits=bits, wgt=(pack4(q) if bits == 4 else q.astype(np.int8)), bias=bias,
+                     relu=int(relu), out_bits=out_bits, out_signed=int(out_signed),
+                     b=None, c=None, rb=None, rc=None, qmin=0, qmax=0,
+                     macs=ho * wo * cout * k * k * cin, params=cout * k * k * cin)
+        if out_bits == 32:                      # raw INT32 logits: bias added, no requantization
+            layer.update(qmin=-(1 << 31), qmax=(1 << 31) - 1, out_signed=1)
+            return self._emit(layer, s_in * float(s_w.mean()), (ho, wo, cout), 32)
+        s_out = _draw_scale(g)
+        layer["b"], layer["c"] = dyadic_from_scale(s_w * s_in / s_out)
+        if res >= 0:
+            rb, rc = dyadic_from_scale(self.scale[res] / s_out)
+            layer["rb"] = np.full(cout, rb[0], np.int32)
+            layer["rc"] = np.full(cout, rc[0], np.int32)
+        if out_signed:
+            layer.update(qmin=-(1 << (out_bits - 1)), qmax=(1 << (out_bits - 1)) - 1)
+        else:
+            layer.update(qmin=0, qmax=(1 << out_bits) - 1)
+        return self._emit(layer, s_out, (ho, wo, cout), out_bits)
+
+    def requant(self, src: int, out_bits: int) -> int:
+        """Unsigned stream tensor -> lower-bit unsigned copy (Fig. 2: quantize the input once)."""
+        h, w, c = self.shape[src]
+        s_out = _draw_scale(self.g) * (255.0 / 15.0 if out_bits == 4 else 1.0)
+        b, cc = dyadic_from_scale(self.scale[src] / s_out)
+        layer = dict(op="requant", in0=src, in1=-1, cout=c, b=np.full(c, b[0], np.int32),
+                     c=np.full(c, cc[0], np.int32), rb=None, rc=None, relu=0, qmin=0,
+                     qmax=(1 << out_bits) - 1, out_bits=out_bits, out_signed=0, macs=0, params=0)
+        return self._emit(layer, s_out, (h, w, c), out_bits)
+
+    def maxpool(self, src: int, k: int, stride: int, pad: int) -> int:
+        h, w, c = self.shape[src]
+        ho, wo = out_hw(h, w, k, stride, pad)
+        layer = dict(op="maxpool", in0=src, in1=-1, pool_k=k, pool_stride=stride, pool_pad=pad, cout=c,
+                     out_bits=8, out_signed=0, relu=0, qmin=0, qmax=255, macs=0, params=0)
+        return self._emit(layer, self.scale[src], (ho, wo, c), 8)
+
+    def avgpool(self, src: int) -> int:
+        h, w, c = self.shape[src]
+        s_out = _draw_scale(self.g)
+        b, cc = dyadic_from_scale(self.scale[src] / (h * w * s_out))   # 1/(h*w) folded in: no division
+        layer = dict(op="avgpool", in0=src, in1=-1, cout=c, b=np.full(c, b[0], np.int32),
+                     c=np.full(c, cc[0], np.int32), out_bits=8, out_signed=0, relu=0, qmin=0, qmax=255,
+                     macs=0, params=0)
+        return self._emit(layer, s_out, (1, 1, c), 8)
+
+
+def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: bool = False,
+                 image_hw: int = 224, classes: int = 1000, width: int = 64) -> dict:
+    """Layer table of an ImageNet-shaped ResNet-18 or ResNet-50 with integer parameters.
+
+    Tensor id -1 is the uint8 input image (n, image_hw, image_hw, 3); layer i produces tensor i.
+    Dataflow (Fig. 2, fused form): every block output is stored as a uint8 stream tensor; the last
+    conv of a block carries the residual add in its epilogue (both branches dyadically rescaled,
+    each rounded, then added); a down-sampling shortcut is a 1x1 conv whose signed 8-bit output
+    is the residual operand.  With mixed=True the convs of the last two stages run at 4 bit: the
+    block input is requantized once to uint4 and shared by conv1 and the shortcut conv, and
+    convs inside the block write uint4 directly.  First conv and classifier stay 8-bit
+    (Appendix H).  ResNet-50 puts the stride on the first 1x1 of a down-sampling bottleneck unless
+    stride_on_3x3 is set; only that placement reproduces the paper's BOPS column (Table 1b).
+    """
+    if depth not in (18, 50):
+        raise ValueError("depth must be 18 or 50")
+    bd = _Builder(seed)
+    bd.scale[-1], bd.shape[-1], bd.bits[-1] = _draw_scale(bd.g), (image_hw, image_hw, 3), 8
+    x = bd.conv(-1, width, 7, 2, 3, 8, relu=True, out_bits=8)
+    x = bd.maxpool(x, 3, 2, 1)
+    blocks = [2, 2, 2, 2] if depth == 18 else [3, 4, 6, 3]
+    expansion = 1 if depth == 18 else 4
+    for stage, nblk in enumerate(blocks):
+        planes = width << stage
+        wb = 4 if (mixed and stage >= 2) else 8
+        for blk in range(nblk):
+            stride = 2 if (blk == 0 and stage > 0) else 1
+            cin = bd.shape[x][2]
+            need_ds = stride != 1 or cin != planes * expansion
+            xin = bd.requant(x, 4) if wb == 4 else x
+            if depth == 18:
+                y = bd.conv(xin, planes, 3, stride, 1, wb, relu=True, out_bits=wb)
+                shortcut = bd.conv(xin, planes, 1, stride, 0, wb, relu=False, out_bits=8,
+                                   out_signed=True) if need_ds else x
+                x = bd.conv(y, planes, 3, 1, 1, wb, relu=True, out_bits=8, res=shortcut)
+            else:
+                s1, s2 = (1, stride) if stride_on_3x3 else (stride, 1)
+                y = bd.conv(xin, planes, 1, s1, 0, wb, relu=True, out_bits=wb)
+                y = bd.conv(y, planes, 3, s2, 1, wb, relu=True, out_bits=wb)
+                shortcut = bd.conv(xin, planes * 4, 1, stride, 0, wb, relu=False, out_bits=8,
+                                   out_signed=True) if need_ds else x
+                x = bd.conv(y, planes * 4, 1, 1, 0, wb, relu=True, out_bits=8, res=shortcut)
+    x = bd.avgpool(x)
+    x = bd.conv(x, classes, 1, 1, 0, 8, relu=False, out_bits=32, op="linear")
+    return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=depth,
+                shapes=[bd.shape[i] for i in range(len(bd.layers))],
+                bits=[bd.bits[i] for i in range(len(bd.layers))])
+
+
+def table_cost(table: dict, force_bits: int | None = None) -> dict:
+    """MACs, parameters, BOPS (= b_w * b_a * MACs, Section 3.4) and weight bytes of a table.
+
+    force_bits=4 evaluates the uniform 4-bit variant with first and last layer kept at 8 bit.
+    """
+    convs = [l for l in table["layers"] if l["op"] in ("conv", "linear")]
+    macs = params = bops = size_bits = 0
+    for i, l in enumerate(convs):
+        bits = l["bits"]
+        if force_bits is not None:
+            bits = 8 if (i == 0 or i == len(convs) - 1) else force_bits
+        macs += l["macs"]
+        params += l["params"]
+        bops += bits * bits * l["macs"]
+        size_bits += bits * l["params"]
+    return dict(macs=macs, params=params, bops=bops, weight_bytes=size_bits // 8)
+
+
+def random_images(seed: int, n: int, hw: int = 224) -> np.ndarray:
+    """uint8 images uniform in [0, 255], NHWC with 3 channels."""
+    return rng(seed, 99, n, hw).integers(0, 256, size=(n, hw, hw, 3), dtype=np.int64).astype(np.uint8)
