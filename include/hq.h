@@ -1,0 +1,175 @@
+/*
+ * hq.h - C ABI of the B200 (sm_100a) library for HAWQ-V3 integer-only inference.
+ *
+ * Every entry point works on DEVICE memory unless its comment says otherwise.  The caller owns
+ * all tensors, weights, biases and dyadic arrays and keeps them alive until the work queued on
+ * `stream` has finished.  The library allocates only inside hq_handle / hq_network objects and
+ * frees that memory in the matching destroy call.  Calls are asynchronous on `stream` (a
+ * cudaStream_t passed as void*; NULL = the legacy default stream).  Argument and launch errors
+ * come back synchronously as hq_status; a device-side wait that ran out of its bounded budget is
+ * reported by hq_sync().  Nothing aborts, throws or prints.  There is no CPU fallback: a shape
+ * the kernels cannot run returns HQ_ERR_UNSUPPORTED.
+ *
+ * Conventions
+ *   - activations are dense NHWC; weights are [cout][kh][kw][cin], signed;
+ *   - bits == 4 tensors hold two values per byte along the channel axis: channel 2j in bits 3:0
+ *     of byte j, channel 2j+1 in bits 7:4, signed values in two's complement; c must be even;
+ *   - activations have zero point 0, so spatial padding is the integer 0;
+ *   - `data` pointers are 16-byte aligned, otherwise HQ_ERR_ALIGNMENT;
+ *   - input and output of a call must not overlap.
+ *
+ * Integer semantics (identical for all entry points), with Int(.) = round-half-up:
+ *   dn(q, b, c) = (q * b + 2^(c-1)) >> c      64-bit product, arithmetic shift, 1 <= c <= 62,
+ *                                             0 <= b < 2^31: the dyadic number b / 2^c applied
+ *                                             to an INT32 value (Eq. 4 and the DN(.) definition).
+ */
+#ifndef HQ_H_
+#define HQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hq_handle hq_handle;   /* opaque: device, status word, workspace */
+typedef struct hq_network hq_network; /* opaque: a planned layer table */
+
+typedef enum {
+  HQ_OK = 0,
+  HQ_ERR_INVALID_ARG = 1,  /* null pointer, bad dimension, bits/sign/clamp combination */
+  HQ_ERR_UNSUPPORTED = 2,  /* valid request no kernel covers */
+  HQ_ERR_ALIGNMENT = 3,    /* a data pointer is not 16-byte aligned */
+  HQ_ERR_RANGE = 4,        /* reserved: accumulator + bias left INT32 (the CPU oracle reports it) */
+  HQ_ERR_WORKSPACE = 5,    /* device allocation failed */
+  HQ_ERR_CUDA = 6,         /* a CUDA runtime or driver call failed */
+  HQ_ERR_TIMEOUT = 7       /* a bounded device-side wait expired; outputs are not valid */
+} hq_status;
+
+typedef struct {  /* activation tensor, dense NHWC */
+  void* data;     /* device pointer, caller-owned */
+  int32_t n, h, w, c; /* logical extents; bits == 4 needs c even */
+  int32_t bits;       /* 4, 8 or 32 */
+  int32_t is_signed;  /* 0: values in [0, 2^bits-1]; 1: two's complement (always 1 for 32) */
+} hq_tensor;
+
+typedef struct {    /* per-channel dyadic pairs b / 2^c, two device arrays of the channel count */
+  const int32_t* b; /* 0 <= b < 2^31 */
+  const int32_t* c; /* 1 <= c <= 62 */
+} hq_dyadic;
+
+typedef struct {
+  int32_t kh, kw, stride, pad, cin, cout;
+  int32_t w_bits;      /* 8 or 4; must equal the input tensor's bits (Section 3.4: b_w == b_a) */
+  const void* w;       /* [cout][kh][kw][cin] signed, 4-bit packed along cin */
+  const int32_t* bias; /* [cout] INT32 at scale S_h * S_w[oc] (Appendix D); NULL means 0 */
+  hq_dyadic requant;   /* DN(S_w[oc] S_h / S_a); ignored when the output has bits == 32 */
+  const hq_tensor* residual; /* NULL, or a tensor with the output's n,h,w,c and bits 8 or 32 */
+  hq_dyadic res_rescale;     /* DN(S_r / S_a) as arrays of length cout; used with residual */
+  int32_t relu;              /* applied after the residual add */
+  int32_t qmin, qmax;        /* clamp bounds, inside the output type's range */
+} hq_conv_desc;
+
+typedef enum {
+  HQ_OP_CONV = 0,    /* hq_conv2d; in1 = residual tensor id or -1 */
+  HQ_OP_LINEAR = 1,  /* hq_linear on the flattened input */
+  HQ_OP_MAXPOOL = 2, /* hq_maxpool */
+  HQ_OP_AVGPOOL = 3, /* hq_avgpool_requant with `rescale0` */
+  HQ_OP_ADD = 4,     /* hq_residual_add(in0 by rescale0, in1 by rescale1) */
+  HQ_OP_REQUANT = 5  /* hq_residual_add with no second operand */
+} hq_op;
+
+typedef struct {       /* one row of the per-layer table; layer i produces tensor id i */
+  int32_t op;          /* hq_op */
+  int32_t in0, in1;    /* tensor ids: -1 = the network input image (in0) / none (in1) */
+  hq_conv_desc conv;   /* CONV / LINEAR: geometry, bit-width, device pointers; .residual ignored */
+  hq_dyadic rescale0;  /* AVGPOOL / ADD / REQUANT: pair applied to in0 */
+  hq_dyadic rescale1;  /* ADD: pair applied to in1 */
+  int32_t pool_k, pool_stride, pool_pad; /* MAXPOOL */
+  int32_t out_bits, out_signed;          /* type of the produced tensor */
+  int32_t relu, qmin, qmax;              /* AVGPOOL / ADD / REQUANT (CONV uses conv.*) */
+} hq_layer;
+
+/* Create / destroy the per-device context.  `device` is a CUDA ordinal.  Host call. */
+hq_status hq_create(int32_t device, hq_handle** out);
+hq_status hq_destroy(hq_handle* h);
+
+/* Wait for `stream` and report HQ_ERR_TIMEOUT if any kernel launched through `h` gave up a
+ * bounded wait since the last hq_sync (the status word is cleared). */
+hq_status hq_sync(hq_handle* h, void* stream);
+
+/*
+ * Quantized convolution with the fused integer epilogue (Section 3.1, Eq. 3-4; Section 3.2 /
+ * Appendix D for the bias; Section 3.3 and Appendix G for the residual):
+ *   acc = sum_{r,s,ci} in[n, oh*stride+r-pad, ow*stride+s-pad, ci] * w[oc,r,s,ci]   (INT32)
+ *   t   = acc + bias[oc]
+ *   out->bits == 32 :  out = t
+ *   otherwise       :  y = dn(t, b[oc], c[oc]);  if residual: y += dn(res, rb[oc], rc[oc]);
+ *                      if relu: y = max(y, 0);  out = clamp(y, qmin, qmax), stored at out->bits.
+ * in: bits 8 or 4 (== w_bits), signed or unsigned.  out: n, h, w, c must equal the convolution's
+ * output extents.  The tensor-core path needs cin*bits/8 to be a multiple of 32 bytes (16 for the
+ * first-layer path); other shapes run on the CUDA-core path.  Accumulator overflow beyond INT32
+ * is undefined (cannot happen for K = kh*kw*cin <= 66311 with 8-bit operands).
+ */
+hq_status hq_conv2d(hq_handle* h, const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
+
+/* Fully connected layer = hq_conv2d with kh = kw = 1 on an (n,1,1,c) tensor (Eq. 3 as a matrix
+ * product).  `desc` must have kh = kw = stride = 1, pad = 0, residual = NULL. */
+hq_status hq_linear(hq_handle* h, const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
+
+/*
+ * Integer residual add on stored tensors (Section 3.3): per element of channel ch
+ *   y = dn(main, mb[ch], mc[ch]) + (res ? dn(res, rb[ch], rc[ch]) : 0); ReLU; clamp; store.
+ * Each branch is rounded on its own and then added (Appendix G).  main/res: bits 4, 8 or 32;
+ * out: bits 4 or 8.  res == NULL gives a plain dyadic requantization.
+ */
+hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic main_rescale,
+                          const hq_tensor* res, hq_dyadic res_rescale,
+                          int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
+
+/*
+ * Global average pooling on wide integers with no division (Appendix E; Section 1 on avoiding
+ * integer division): sum over the h*w pixels in INT32, then clamp(dn(sum, b[ch], c[ch])), the
+ * factor 1/(h*w) being part of b / 2^c.  in: (n,h,w,c) bits 4/8/32; out: (n,1,1,c) bits 4/8.
+ */
+hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic rescale,
+                             int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
+
+/* k x k max pooling of an 8-bit tensor; window taps outside the image are ignored (ResNet stem;
+ * an integer max commutes with the monotone requantization of Eq. 4).  pad < k. */
+hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,
+                     hq_tensor* out, void* stream);
+
+/*
+ * Plan a network from its per-layer table (bit-widths, geometry, dyadic pairs, residual wiring;
+ * Fig. 2 dataflow in fused form, first and last layer 8-bit per Appendix H).  `table` is a HOST
+ * array; the pointers inside it are DEVICE pointers that must outlive the network.  Activation
+ * buffers for `batch` images of image_h x image_w x image_c (8-bit) are allocated here.
+ */
+hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layers, int32_t batch,
+                            int32_t image_h, int32_t image_w, int32_t image_c, int32_t image_signed,
+                            hq_network** out);
+
+/*
+ * Run the table on `images` (device, NHWC 8-bit, the planned batch) and write the last layer's
+ * output to `logits` (device; its n,c,bits must match the last layer).  `layer_taps` is NULL or
+ * a HOST array of n_layers device pointers (NULL entries allowed) that receive a copy of each
+ * layer's output in its stored format.
+ */
+hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* logits,
+                         void* const* layer_taps, void* stream);
+
+/* Bytes of layer i's stored output and the number of kernels one hq_run_network launches. */
+hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* bytes);
+hq_status hq_network_launch_count(const hq_network* net, int32_t* launches);
+hq_status hq_network_destroy(hq_network* net);
+
+/* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail. */
+hq_status hq_set_conv_path(hq_handle* h, int32_t path);
+
+const char* hq_status_string(hq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HQ_H_ */

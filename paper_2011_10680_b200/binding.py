@@ -1,0 +1,271 @@
+"""Thin ctypes binding over libhq.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams; every step of the inference path runs inside the
+library's CUDA kernels.  There is no CPU fallback: if the shared library is missing or the device
+is not a B200-class GPU, loading or hq_create fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhq.so")
+
+HQ_OK, HQ_ERR_INVALID_ARG, HQ_ERR_UNSUPPORTED, HQ_ERR_ALIGNMENT = 0, 1, 2, 3
+HQ_ERR_RANGE, HQ_ERR_WORKSPACE, HQ_ERR_CUDA, HQ_ERR_TIMEOUT = 4, 5, 6, 7
+HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant": 5}
+
+EXPORTS = [
+    "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
+    "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
+    "hq_network_destroy", "hq_set_conv_path", "hq_status_string",
+]
+
+
+class HqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+        self.code = code
+
+
+class hq_tensor(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("n", C.c_int32), ("h", C.c_int32), ("w", C.c_int32), ("c", C.c_int32),
+                ("bits", C.c_int32), ("is_signed", C.c_int32)]
+
+
+class hq_dyadic(C.Structure):
+    _fields_ = [("b", C.c_void_p), ("c", C.c_void_p)]
+
+
+class hq_conv_desc(C.Structure):
+    _fields_ = [("kh", C.c_int32), ("kw", C.c_int32), ("stride", C.c_int32), ("pad", C.c_int32),
+                ("cin", C.c_int32), ("cout", C.c_int32), ("w_bits", C.c_int32), ("w", C.c_void_p),
+                ("bias", C.c_void_p), ("requant", hq_dyadic), ("residual", C.POINTER(hq_tensor)),
+                ("res_rescale", hq_dyadic), ("relu", C.c_int32), ("qmin", C.c_int32), ("qmax", C.c_int32)]
+
+
+class hq_layer(C.Structure):
+    _fields_ = [("op", C.c_int32), ("in0", C.c_int32), ("in1", C.c_int32), ("conv", hq_conv_desc),
+                ("rescale0", hq_dyadic), ("rescale1", hq_dyadic), ("pool_k", C.c_int32),
+                ("pool_stride", C.c_int32), ("pool_pad", C.c_int32), ("out_bits", C.c_int32),
+                ("out_signed", C.c_int32), ("relu", C.c_int32), ("qmin", C.c_int32), ("qmax", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libhq.so (must have been built in-tree; see build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build the CUDA library first (python -m paper_2011_10680_b200.build)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32 = C.c_void_p, C.c_int32
+        TP, DP, LP = C.POINTER(hq_tensor), C.POINTER(hq_conv_desc), C.POINTER(hq_layer)
+        L.hq_create.argtypes = [i32, C.POINTER(vp)]
+        L.hq_destroy.argtypes = [vp]
+        L.hq_sync.argtypes = [vp, vp]
+        L.hq_conv2d.argtypes = [vp, TP, DP, TP, vp]
+        L.hq_linear.argtypes = [vp, TP, DP, TP, vp]
+        L.hq_residual_add.argtypes = [vp, TP, hq_dyadic, TP, hq_dyadic, i32, i32, i32, TP, vp]
+        L.hq_avgpool_requant.argtypes = [vp, TP, hq_dyadic, i32, i32, TP, vp]
+        L.hq_maxpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
+        L.hq_network_create.argtypes = [vp, LP, i32, i32, i32, i32, i32, i32, C.POINTER(vp)]
+        L.hq_run_network.argtypes = [vp, TP, TP, C.POINTER(vp), vp]
+        L.hq_network_layer_bytes.argtypes = [vp, i32, C.POINTER(C.c_int64)]
+        L.hq_network_launch_count.argtypes = [vp, C.POINTER(i32)]
+        L.hq_network_destroy.argtypes = [vp]
+        L.hq_set_conv_path.argtypes = [vp, i32]
+        L.hq_status_string.argtypes = [i32]
+        L.hq_status_string.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "hq_status_string":
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().hq_status_string(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != HQ_OK:
+        raise HqError(code, where)
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def tensor_of(t, c: int, bits: int, is_signed: int) -> hq_tensor:
+    """Describe a torch CUDA tensor of shape (n, h, w, c_stored) as an hq_tensor with logical channels c."""
+    n, h, w = t.shape[0], t.shape[1], t.shape[2]
+    return hq_tensor(t.data_ptr(), n, h, w, c, bits, is_signed)
+
+
+def _dy(b, c) -> hq_dyadic:
+    return hq_dyadic(b.data_ptr() if b is not None else None, c.data_ptr() if c is not None else None)
+
+
+def to_device(a):
+    """numpy array -> CUDA tensor with the same bytes (int8/uint8/int32)."""
+    import torch
+    if a is None:
+        return None
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def alloc_out(n, h, w, c, bits, signed):
+    import torch
+    if bits == 32:
+        return torch.empty((n, h, w, c), dtype=torch.int32, device="cuda")
+    if bits == 8:
+        return torch.empty((n, h, w, c), dtype=torch.int8 if signed else torch.uint8, device="cuda")
+    return torch.empty((n, h, w, c // 2), dtype=torch.uint8, device="cuda")
+
+
+class Handle:
+    """Owns an hq_handle for one device."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        _check(lib().hq_create(device, C.byref(self._h)), "hq_create")
+
+    def close(self):
+        if self._h:
+            lib().hq_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_conv_path(self, path: int):
+        _check(lib().hq_set_conv_path(self._h, path), "hq_set_conv_path")
+
+    def sync(self):
+        _check(lib().hq_sync(self._h, _stream()), "hq_sync")
+
+    # ---- one call per C entry point --------------------------------------------------------
+    def conv2d(self, x, in_bits, in_signed, cin, wgt, cout, kh, kw, stride, pad, bias, b, c, out, out_bits, out_signed,
+               res=None, res_bits=0, res_signed=0, rb=None, rc=None, relu=1, qmin=0, qmax=255, linear=False):
+        tin = tensor_of(x, cin, in_bits, in_signed)
+        tout = tensor_of(out, cout, out_bits, out_signed)
+        tres = tensor_of(res, cout, res_bits, res_signed) if res is not None else None
+        d = hq_conv_desc(kh, kw, stride, pad, cin, cout, in_bits, wgt.data_ptr(),
+                         bias.data_ptr() if bias is not None else None, _dy(b, c),
+                         C.pointer(tres) if tres is not None else None, _dy(rb, rc), relu, qmin, qmax)
+        fn = lib().hq_linear if linear else lib().hq_conv2d
+        return fn(self._h, C.byref(tin), C.byref(d), C.byref(tout), _stream())
+
+    def residual_add(self, main, main_bits, main_signed, mb, mc, res, res_bits, res_signed, rb, rc, ch,
+                     relu, qmin, qmax, out, out_bits, out_signed):
+        tm = tensor_of(main, ch, main_bits, main_signed)
+        to = tensor_of(out, ch, out_bits, out_signed)
+        tr = tensor_of(res, ch, res_bits, res_signed) if res is not None else None
+        return lib().hq_residual_add(self._h, C.byref(tm), _dy(mb, mc), C.byref(tr) if tr is not None else None,
+                                     _dy(rb, rc), relu, qmin, qmax, C.byref(to), _stream())
+
+    def avgpool_requant(self, x, ch, in_bits, in_signed, b, c, qmin, qmax, out, out_bits, out_signed):
+        ti = tensor_of(x, ch, in_bits, in_signed)
+        to = tensor_of(out, ch, out_bits, out_signed)
+        return lib().hq_avgpool_requant(self._h, C.byref(ti), _dy(b, c), qmin, qmax, C.byref(to), _stream())
+
+    def maxpool(self, x, ch, signed, k, stride, pad, out):
+        ti = tensor_of(x, ch, 8, signed)
+        to = tensor_of(out, ch, 8, signed)
+        return lib().hq_maxpool(self._h, C.byref(ti), k, stride, pad, C.byref(to), _stream())
+
+    # ---- convenience for the dict-shaped single-layer cases of the workload generator -------
+    def conv_case(self, case: dict, dev: dict | None = None):
+        """Upload (or reuse `dev`) a generated conv case, run hq_conv2d, return (status, out tensor)."""
+        dev = dev if dev is not None else upload_case(case)
+        out = alloc_out(case["n"], case["ho"], case["wo"], case["cout"], case["out_bits"], case["out_signed"])
+        st = self.conv2d(dev["x"], case["bits"], case["in_signed"], case["cin"], dev["wgt"], case["cout"], case["kh"],
+                         case["kw"], case["stride"], case["pad"], dev["bias"], dev["b"], dev["c"], out,
+                         case["out_bits"], case["out_signed"], dev["res"], case["res_bits"], case["res_signed"],
+                         dev["rb"], dev["rc"], case["relu"], case["qmin"], case["qmax"])
+        return st, out
+
+
+def upload_case(case: dict) -> dict:
+    return {k: to_device(case[k]) for k in ("x", "wgt", "bias", "b", "c", "res", "rb", "rc")}
+
+
+class Network:
+    """hq_network built from a generated layer table; keeps the device copies of all parameters alive."""
+
+    def __init__(self, handle: Handle, table: dict, batch: int, image_signed: int = 0):
+        self.handle, self.table, self.batch = handle, table, batch
+        self._keep = []
+        layers = table["layers"]
+        arr = (hq_layer * len(layers))()
+        for i, l in enumerate(layers):
+            e = arr[i]
+            e.op, e.in0, e.in1 = HQ_OP[l["op"]], l["in0"], l["in1"]
+            e.out_bits, e.out_signed = l["out_bits"], l["out_signed"]
+            e.relu, e.qmin, e.qmax = l["relu"], l["qmin"], l["qmax"]
+            if l["op"] in ("conv", "linear"):
+                dv = {k: to_device(l[k]) for k in ("wgt", "bias", "b", "c", "rb", "rc")}
+                self._keep.append(dv)
+                e.conv = hq_conv_desc(l["kh"], l["kw"], l["stride"], l["pad"], l["cin"], l["cout"], l["bits"],
+                                      dv["wgt"].data_ptr(),
+                                      dv["bias"].data_ptr() if dv["bias"] is not None else None, _dy(dv["b"], dv["c"]), None,
+                                      _dy(dv["rb"], dv["rc"]), l["relu"], l["qmin"], l["qmax"])
+            elif l["op"] == "maxpool":
+                e.pool_k, e.pool_stride, e.pool_pad = l["pool_k"], l["pool_stride"], l["pool_pad"]
+            else:
+                dv = {k: to_device(l.get(k)) for k in ("b", "c", "rb", "rc")}
+                self._keep.append(dv)
+                e.rescale0 = _dy(dv["b"], dv["c"])
+                e.rescale1 = _dy(dv["rb"], dv["rc"])
+        self._arr = arr
+        self._net = C.c_void_p()
+        hw = table["image_hw"]
+        _check(lib().hq_network_create(handle._h, arr, len(layers), batch, hw, hw, 3, image_signed,
+                                       C.byref(self._net)), "hq_network_create")
+        last = layers[-1]
+        self.logits_shape = (batch, 1, 1, last["cout"])
+
+    def layer_bytes(self, i: int) -> int:
+        v = C.c_int64()
+        _check(lib().hq_network_layer_bytes(self._net, i, C.byref(v)), "hq_network_layer_bytes")
+        return v.value
+
+    def launch_count(self) -> int:
+        v = C.c_int32()
+        _check(lib().hq_network_launch_count(self._net, C.byref(v)), "hq_network_launch_count")
+        return v.value
+
+    def run(self, images, logits, taps=None):
+        """images: uint8 CUDA tensor (batch, H, W, 3); logits: int32 CUDA tensor; taps: list of CUDA tensors or None."""
+        ti = tensor_of(images, images.shape[3], 8, 0)
+        last = self.table["layers"][-1]
+        tl = hq_tensor(logits.data_ptr(), self.batch, 1, 1, last["cout"], last["out_bits"], last["out_signed"])
+        tap_arr = None
+        if taps is not None:
+            tap_arr = (C.c_void_p * len(taps))(*[t.data_ptr() if t is not None else None for t in taps])
+        return lib().hq_run_network(self._net, C.byref(ti), C.byref(tl), tap_arr, _stream())
+
+    def alloc_taps(self):
+        import torch
+        return [torch.empty(self.layer_bytes(i), dtype=torch.uint8, device="cuda") for i in range(len(self.table["layers"]))]
+
+    def close(self):
+        if self._net:
+            lib().hq_network_destroy(self._net)
+            self._net = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

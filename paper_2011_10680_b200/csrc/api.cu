@@ -1,0 +1,387 @@
+// C ABI of libhq.so: argument validation, dispatch to the kernels, and the table-driven network
+// runner.  Host code only; every step of the inference path runs in the kernels of the other
+// translation units.
+#include <new>
+#include <vector>
+
+#include "hq_internal.cuh"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool type_range_ok(int bits, int is_signed, int qmin, int qmax) {
+  long long lo, hi;
+  if (bits == 32) { lo = -(1LL << 31); hi = (1LL << 31) - 1; }
+  else if (is_signed) { lo = -(1LL << (bits - 1)); hi = (1LL << (bits - 1)) - 1; }
+  else { lo = 0; hi = (1LL << bits) - 1; }
+  return qmin <= qmax && qmin >= lo && qmax <= hi;
+}
+
+inline hq_status check_tensor(const hq_tensor* t, bool allow4, bool allow8, bool allow32) {
+  if (!t || !t->data) return HQ_ERR_INVALID_ARG;
+  if (t->n < 0 || t->h < 1 || t->w < 1 || t->c < 1) return HQ_ERR_INVALID_ARG;
+  if (!((t->bits == 4 && allow4) || (t->bits == 8 && allow8) || (t->bits == 32 && allow32))) return HQ_ERR_INVALID_ARG;
+  if (t->bits == 4 && (t->c & 1)) return HQ_ERR_INVALID_ARG;
+  if (!aligned16(t->data)) return HQ_ERR_ALIGNMENT;
+  return HQ_OK;
+}
+
+inline long long tensor_bytes(int n, int h, int w, int c, int bits) {
+  return (long long)n * h * w * c * bits / 8;
+}
+
+hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream) {
+  if (!h || !d) return HQ_ERR_INVALID_ARG;
+  hq_status st = check_tensor(in, true, true, false);
+  if (st != HQ_OK) return st;
+  st = check_tensor(out, true, true, true);
+  if (st != HQ_OK) return st;
+  if (d->kh < 1 || d->kw < 1 || d->stride < 1 || d->pad < 0 || d->cin < 1 || d->cout < 1) return HQ_ERR_INVALID_ARG;
+  if (d->cin != in->c || d->w_bits != in->bits || !d->w) return HQ_ERR_INVALID_ARG;
+  if (in->h + 2 * d->pad < d->kh || in->w + 2 * d->pad < d->kw) return HQ_ERR_INVALID_ARG;
+  const int ho = (in->h + 2 * d->pad - d->kh) / d->stride + 1;
+  const int wo = (in->w + 2 * d->pad - d->kw) / d->stride + 1;
+  if (out->n != in->n || out->h != ho || out->w != wo || out->c != d->cout) return HQ_ERR_INVALID_ARG;
+  if (!aligned16(d->w)) return HQ_ERR_ALIGNMENT;
+  if (out->bits == 32) {
+    if (d->residual) return HQ_ERR_INVALID_ARG;
+  } else {
+    if (!d->requant.b || !d->requant.c) return HQ_ERR_INVALID_ARG;
+    if (!type_range_ok(out->bits, out->is_signed, d->qmin, d->qmax)) return HQ_ERR_INVALID_ARG;
+    if (d->residual) {
+      const hq_tensor* r = d->residual;
+      st = check_tensor(r, false, true, true);
+      if (st != HQ_OK) return st;
+      if (r->n != out->n || r->h != out->h || r->w != out->w || r->c != out->c) return HQ_ERR_INVALID_ARG;
+      if (!d->res_rescale.b || !d->res_rescale.c) return HQ_ERR_INVALID_ARG;
+    }
+  }
+  ConvArgs a{};
+  a.in = in->data; a.n = in->n; a.h = in->h; a.w = in->w; a.cin = in->c; a.in_bits = in->bits; a.in_signed = in->is_signed;
+  a.wgt = d->w; a.cout = d->cout; a.kh = d->kh; a.kw = d->kw; a.stride = d->stride; a.pad = d->pad;
+  a.bias = d->bias; a.b = d->requant.b; a.c = d->requant.c;
+  if (d->residual && out->bits != 32) {
+    a.res = d->residual->data; a.res_bits = d->residual->bits; a.res_signed = d->residual->is_signed;
+    a.rb = d->res_rescale.b; a.rc = d->res_rescale.c;
+  }
+  a.relu = d->relu; a.qmin = d->qmin; a.qmax = d->qmax;
+  a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool tc_ok = hq_conv_tc_supported(a);
+  if (h->conv_path == 2 && !tc_ok) return HQ_ERR_UNSUPPORTED;
+  if (h->conv_path != 1 && tc_ok) return hq_launch_conv_tc(h, a, s);
+  return hq_launch_conv_cuda_core(a, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+struct hq_network {
+  hq_handle* h;
+  std::vector<hq_layer> layers;
+  std::vector<hq_tensor> outs;       // planned output tensor of every layer (data owned by the network)
+  std::vector<long long> bytes;
+  int32_t batch, image_h, image_w, image_c, image_signed;
+  int32_t launches;
+  // graph cache
+  cudaGraphExec_t graph_exec;
+  const void* graph_images;
+  void* graph_logits;
+};
+
+extern "C" {
+
+const char* hq_status_string(hq_status s) {
+  switch (s) {
+    case HQ_OK: return "HQ_OK";
+    case HQ_ERR_INVALID_ARG: return "HQ_ERR_INVALID_ARG";
+    case HQ_ERR_UNSUPPORTED: return "HQ_ERR_UNSUPPORTED";
+    case HQ_ERR_ALIGNMENT: return "HQ_ERR_ALIGNMENT";
+    case HQ_ERR_RANGE: return "HQ_ERR_RANGE";
+    case HQ_ERR_WORKSPACE: return "HQ_ERR_WORKSPACE";
+    case HQ_ERR_CUDA: return "HQ_ERR_CUDA";
+    case HQ_ERR_TIMEOUT: return "HQ_ERR_TIMEOUT";
+  }
+  return "HQ_ERR_UNKNOWN";
+}
+
+hq_status hq_create(int32_t device, hq_handle** out) {
+  if (!out) return HQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess) return HQ_ERR_CUDA;
+  if (device < 0 || device >= count) return HQ_ERR_INVALID_ARG;
+  if (cudaSetDevice(device) != cudaSuccess) return HQ_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return HQ_ERR_CUDA;
+  if (prop.major != 10) return HQ_ERR_UNSUPPORTED;       // kernels are built for sm_100a only
+  hq_handle* h = new (std::nothrow) hq_handle();
+  if (!h) return HQ_ERR_WORKSPACE;
+  h->device = device;
+  h->conv_path = 0;
+  h->sm_count = prop.multiProcessorCount;
+  h->workspace = nullptr;
+  h->workspace_bytes = 0;
+  if (!hq_conv_tc_init()) { delete h; return HQ_ERR_CUDA; }
+  if (cudaMalloc(&h->dev_status, sizeof(uint32_t)) != cudaSuccess) { delete h; return HQ_ERR_WORKSPACE; }
+  if (cudaMemset(h->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) { cudaFree(h->dev_status); delete h; return HQ_ERR_CUDA; }
+  *out = h;
+  return HQ_OK;
+}
+
+hq_status hq_destroy(hq_handle* h) {
+  if (!h) return HQ_ERR_INVALID_ARG;
+  cudaFree(h->dev_status);
+  if (h->workspace) cudaFree(h->workspace);
+  delete h;
+  return HQ_OK;
+}
+
+hq_status hq_set_conv_path(hq_handle* h, int32_t path) {
+  if (!h || path < 0 || path > 2) return HQ_ERR_INVALID_ARG;
+  h->conv_path = path;
+  return HQ_OK;
+}
+
+hq_status hq_sync(hq_handle* h, void* stream) {
+  if (!h) return HQ_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HQ_ERR_CUDA;
+  uint32_t word = 0;
+  if (cudaMemcpy(&word, h->dev_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return HQ_ERR_CUDA;
+  if (word != 0) {
+    cudaMemset(h->dev_status, 0, sizeof(uint32_t));
+    return HQ_ERR_TIMEOUT;
+  }
+  return HQ_OK;
+}
+
+hq_status hq_conv2d(hq_handle* h, const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream) {
+  return conv_common(h, in, desc, out, stream);
+}
+
+hq_status hq_linear(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream) {
+  if (!in || !d || !out) return HQ_ERR_INVALID_ARG;
+  if (d->kh != 1 || d->kw != 1 || d->stride != 1 || d->pad != 0 || d->residual) return HQ_ERR_INVALID_ARG;
+  if (in->h != 1 || in->w != 1) return HQ_ERR_INVALID_ARG;
+  return conv_common(h, in, d, out, stream);
+}
+
+hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, const hq_tensor* res, hq_dyadic rr,
+                          int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream) {
+  if (!h) return HQ_ERR_INVALID_ARG;
+  hq_status st = check_tensor(main_t, true, true, true);
+  if (st != HQ_OK) return st;
+  st = check_tensor(out, true, true, false);
+  if (st != HQ_OK) return st;
+  if (out->n != main_t->n || out->h != main_t->h || out->w != main_t->w || out->c != main_t->c) return HQ_ERR_INVALID_ARG;
+  if (!mr.b || !mr.c) return HQ_ERR_INVALID_ARG;
+  if (!type_range_ok(out->bits, out->is_signed, qmin, qmax)) return HQ_ERR_INVALID_ARG;
+  EltArgs a{};
+  if (res) {
+    st = check_tensor(res, true, true, true);
+    if (st != HQ_OK) return st;
+    if (res->n != out->n || res->h != out->h || res->w != out->w || res->c != out->c) return HQ_ERR_INVALID_ARG;
+    if (!rr.b || !rr.c) return HQ_ERR_INVALID_ARG;
+    a.res = res->data; a.res_bits = res->bits; a.res_signed = res->is_signed; a.rb = rr.b; a.rc = rr.c;
+  }
+  a.main_t = main_t->data; a.main_bits = main_t->bits; a.main_signed = main_t->is_signed; a.mb = mr.b; a.mc = mr.c;
+  a.pixels = (long long)out->n * out->h * out->w; a.ch = out->c;
+  a.relu = relu; a.qmin = qmin; a.qmax = qmax; a.out = out->data; a.out_bits = out->bits;
+  return hq_launch_residual_add(a, h->sm_count, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic r, int32_t qmin, int32_t qmax,
+                             hq_tensor* out, void* stream) {
+  if (!h) return HQ_ERR_INVALID_ARG;
+  hq_status st = check_tensor(in, true, true, true);
+  if (st != HQ_OK) return st;
+  st = check_tensor(out, true, true, false);
+  if (st != HQ_OK) return st;
+  if (out->n != in->n || out->h != 1 || out->w != 1 || out->c != in->c) return HQ_ERR_INVALID_ARG;
+  if (!r.b || !r.c) return HQ_ERR_INVALID_ARG;
+  if (!type_range_ok(out->bits, out->is_signed, qmin, qmax)) return HQ_ERR_INVALID_ARG;
+  if ((long long)in->h * in->w > (1LL << 23)) return HQ_ERR_UNSUPPORTED;   // INT32 sum of 8-bit values
+  return hq_launch_avgpool(in->data, in->n, in->h, in->w, in->c, in->bits, in->is_signed, r.b, r.c, qmin, qmax,
+                           out->data, out->bits, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad, hq_tensor* out,
+                     void* stream) {
+  if (!h) return HQ_ERR_INVALID_ARG;
+  hq_status st = check_tensor(in, false, true, false);
+  if (st != HQ_OK) return st;
+  st = check_tensor(out, false, true, false);
+  if (st != HQ_OK) return st;
+  if (k < 1 || stride < 1 || pad < 0 || pad >= k) return HQ_ERR_INVALID_ARG;
+  if (in->h + 2 * pad < k || in->w + 2 * pad < k) return HQ_ERR_INVALID_ARG;
+  const int ho = (in->h + 2 * pad - k) / stride + 1, wo = (in->w + 2 * pad - k) / stride + 1;
+  if (out->n != in->n || out->h != ho || out->w != wo || out->c != in->c || out->is_signed != in->is_signed)
+    return HQ_ERR_INVALID_ARG;
+  return hq_launch_maxpool(in->data, in->n, in->h, in->w, in->c, in->is_signed, k, stride, pad, out->data, ho, wo,
+                           (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layers, int32_t batch,
+                            int32_t image_h, int32_t image_w, int32_t image_c, int32_t image_signed,
+                            hq_network** out) {
+  if (!h || !table || !out || n_layers < 1 || batch < 1 || image_h < 1 || image_w < 1 || image_c < 1)
+    return HQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  hq_network* net = new (std::nothrow) hq_network();
+  if (!net) return HQ_ERR_WORKSPACE;
+  net->h = h; net->batch = batch;
+  net->image_h = image_h; net->image_w = image_w; net->image_c = image_c; net->image_signed = image_signed;
+  net->graph_exec = nullptr; net->graph_images = nullptr; net->graph_logits = nullptr;
+  net->layers.assign(table, table + n_layers);
+  net->outs.resize(n_layers);
+  net->bytes.resize(n_layers);
+  net->launches = n_layers;
+  hq_status st = HQ_OK;
+  auto shape_of = [&](int id, hq_tensor* t) -> bool {
+    if (id == -1) { *t = hq_tensor{nullptr, batch, image_h, image_w, image_c, 8, image_signed}; return true; }
+    if (id < 0) return false;
+    *t = net->outs[id];
+    return true;
+  };
+  for (int i = 0; i < n_layers && st == HQ_OK; ++i) {
+    const hq_layer& l = net->layers[i];
+    hq_tensor in{}, o{};
+    if (l.in0 >= i || l.in1 >= i || !shape_of(l.in0, &in)) { st = HQ_ERR_INVALID_ARG; break; }
+    o.n = batch; o.bits = l.out_bits; o.is_signed = l.out_signed;
+    switch (l.op) {
+      case HQ_OP_CONV: {
+        const hq_conv_desc& d = l.conv;
+        if (d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0 || in.h + 2 * d.pad < d.kh || in.w + 2 * d.pad < d.kw) {
+          st = HQ_ERR_INVALID_ARG; break;
+        }
+        o.h = (in.h + 2 * d.pad - d.kh) / d.stride + 1; o.w = (in.w + 2 * d.pad - d.kw) / d.stride + 1; o.c = d.cout;
+        break;
+      }
+      case HQ_OP_LINEAR:
+        if (l.conv.cin != in.h * in.w * in.c) { st = HQ_ERR_INVALID_ARG; break; }
+        o.h = 1; o.w = 1; o.c = l.conv.cout;
+        break;
+      case HQ_OP_MAXPOOL:
+        if (l.pool_k < 1 || l.pool_stride < 1 || l.pool_pad < 0 || in.h + 2 * l.pool_pad < l.pool_k ||
+            in.w + 2 * l.pool_pad < l.pool_k) { st = HQ_ERR_INVALID_ARG; break; }
+        o.h = (in.h + 2 * l.pool_pad - l.pool_k) / l.pool_stride + 1;
+        o.w = (in.w + 2 * l.pool_pad - l.pool_k) / l.pool_stride + 1; o.c = in.c;
+        break;
+      case HQ_OP_AVGPOOL: o.h = 1; o.w = 1; o.c = in.c; break;
+      case HQ_OP_ADD: case HQ_OP_REQUANT: o.h = in.h; o.w = in.w; o.c = in.c; break;
+      default: st = HQ_ERR_INVALID_ARG; break;
+    }
+    if (st != HQ_OK) break;
+    if (!(o.bits == 4 || o.bits == 8 || o.bits == 32) || o.c < 1 || (o.bits == 4 && (o.c & 1))) { st = HQ_ERR_INVALID_ARG; break; }
+    net->bytes[i] = tensor_bytes(o.n, o.h, o.w, o.c, o.bits);
+    void* buf = nullptr;
+    if (cudaMalloc(&buf, (size_t)net->bytes[i] + 256) != cudaSuccess) { st = HQ_ERR_WORKSPACE; break; }
+    o.data = buf;
+    net->outs[i] = o;
+  }
+  if (st != HQ_OK) { hq_network_destroy(net); return st; }
+  *out = net;
+  return HQ_OK;
+}
+
+static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor* logits, void* const* taps,
+                            cudaStream_t s) {
+  hq_handle* h = net->h;
+  const int n_layers = (int)net->layers.size();
+  for (int i = 0; i < n_layers; ++i) {
+    const hq_layer& l = net->layers[i];
+    hq_tensor in = (l.in0 == -1) ? *images : net->outs[l.in0];
+    hq_tensor o = net->outs[i];
+    if (i == n_layers - 1) o.data = logits->data;
+    hq_status st = HQ_OK;
+    switch (l.op) {
+      case HQ_OP_CONV: case HQ_OP_LINEAR: {
+        hq_conv_desc d = l.conv;
+        hq_tensor res{};
+        d.residual = nullptr;
+        if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
+        if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
+        else st = hq_conv2d(h, &in, &d, &o, s);
+        break;
+      }
+      case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
+      case HQ_OP_AVGPOOL: st = hq_avgpool_requant(h, &in, l.rescale0, l.qmin, l.qmax, &o, s); break;
+      case HQ_OP_ADD: {
+        if (l.in1 < 0) return HQ_ERR_INVALID_ARG;
+        hq_tensor res = net->outs[l.in1];
+        st = hq_residual_add(h, &in, l.rescale0, &res, l.rescale1, l.relu, l.qmin, l.qmax, &o, s);
+        break;
+      }
+      case HQ_OP_REQUANT: {
+        hq_dyadic none{nullptr, nullptr};
+        st = hq_residual_add(h, &in, l.rescale0, nullptr, none, l.relu, l.qmin, l.qmax, &o, s);
+        break;
+      }
+      default: return HQ_ERR_INVALID_ARG;
+    }
+    if (st != HQ_OK) return st;
+    if (taps && taps[i]) {
+      if (cudaMemcpyAsync(taps[i], o.data, (size_t)net->bytes[i], cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return HQ_ERR_CUDA;
+    }
+  }
+  return HQ_OK;
+}
+
+hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* logits, void* const* layer_taps,
+                         void* stream) {
+  if (!net || !images || !logits || !images->data || !logits->data) return HQ_ERR_INVALID_ARG;
+  if (images->n != net->batch || images->h != net->image_h || images->w != net->image_w ||
+      images->c != net->image_c || images->bits != 8 || images->is_signed != net->image_signed)
+    return HQ_ERR_INVALID_ARG;
+  const hq_tensor& last = net->outs.back();
+  if (logits->n != last.n || logits->h != last.h || logits->w != last.w || logits->c != last.c ||
+      logits->bits != last.bits) return HQ_ERR_INVALID_ARG;
+  if (!aligned16(images->data) || !aligned16(logits->data)) return HQ_ERR_ALIGNMENT;
+  cudaStream_t s = (cudaStream_t)stream;
+
+  // Inside a caller's capture, or when taps are requested: plain launches.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) return HQ_ERR_CUDA;
+  if (cap != cudaStreamCaptureStatusNone || layer_taps || s == nullptr) return run_layers(net, images, logits, layer_taps, s);
+
+  // Otherwise replay a CUDA graph of the whole table (captured once per (images, logits) pair).
+  if (!net->graph_exec || net->graph_images != images->data || net->graph_logits != logits->data) {
+    if (net->graph_exec) { cudaGraphExecDestroy(net->graph_exec); net->graph_exec = nullptr; }
+    if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return HQ_ERR_CUDA;
+    const hq_status st = run_layers(net, images, logits, nullptr, s);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(s, &graph);
+    if (st != HQ_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+    if (e != cudaSuccess || !graph) return HQ_ERR_CUDA;
+    const cudaError_t e2 = cudaGraphInstantiate(&net->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e2 != cudaSuccess) { net->graph_exec = nullptr; return HQ_ERR_CUDA; }
+    net->graph_images = images->data; net->graph_logits = logits->data;
+  }
+  return cudaGraphLaunch(net->graph_exec, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* bytes) {
+  if (!net || !bytes || layer < 0 || layer >= (int)net->layers.size()) return HQ_ERR_INVALID_ARG;
+  *bytes = net->bytes[layer];
+  return HQ_OK;
+}
+
+hq_status hq_network_launch_count(const hq_network* net, int32_t* launches) {
+  if (!net || !launches) return HQ_ERR_INVALID_ARG;
+  *launches = net->launches;
+  return HQ_OK;
+}
+
+hq_status hq_network_destroy(hq_network* net) {
+  if (!net) return HQ_ERR_INVALID_ARG;
+  if (net->graph_exec) cudaGraphExecDestroy(net->graph_exec);
+  for (auto& t : net->outs) if (t.data) cudaFree(t.data);
+  delete net;
+  return HQ_OK;
+}
+
+}  // extern "C"

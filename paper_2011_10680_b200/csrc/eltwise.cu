@@ -1,0 +1,290 @@
+// Memory-bound kernels of the integer-only pipeline: residual add / requantization on stored
+// tensors (Section 3.3), global average pooling on wide integers (Appendix E) and the stem's max
+// pooling.  Each streams its operands once with 16-byte accesses; the arithmetic is the dyadic
+// multiply-shift of Eq. 4 in 64-bit integers.  No floating point anywhere.
+#include "hq_internal.cuh"
+
+namespace {
+
+// ---- 16-element group load/store for 4-, 8- and 32-bit dense tensors -----------------------
+template <int BITS>
+__device__ __forceinline__ void load16(const void* base, long long elem, int is_signed, int (&v)[16]) {
+  if constexpr (BITS == 32) {
+    const int4* p = (const int4*)((const int*)base + elem);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      int4 t = __ldg(p + i);
+      v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
+    }
+  } else if constexpr (BITS == 8) {
+    const uint4 t = __ldg((const uint4*)((const unsigned char*)base + elem));
+    const unsigned w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const unsigned byte = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+      v[i] = is_signed ? (int)(signed char)byte : (int)byte;
+    }
+  } else {
+    const uint2 t = __ldg((const uint2*)((const unsigned char*)base + (elem >> 1)));
+    const unsigned w[2] = {t.x, t.y};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      int nib = (int)((w[i >> 3] >> (4 * (i & 7))) & 0xFu);
+      if (is_signed && (nib & 8)) nib -= 16;
+      v[i] = nib;
+    }
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void store16(void* base, long long elem, const int (&v)[16]) {
+  if constexpr (BITS == 8) {
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      w[i] = (unsigned)(v[4 * i] & 0xFF) | ((unsigned)(v[4 * i + 1] & 0xFF) << 8) |
+             ((unsigned)(v[4 * i + 2] & 0xFF) << 16) | ((unsigned)(v[4 * i + 3] & 0xFF) << 24);
+    *(uint4*)((unsigned char*)base + elem) = make_uint4(w[0], w[1], w[2], w[3]);
+  } else {
+    unsigned w[2] = {0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) w[i >> 3] |= (unsigned)(v[i] & 0xF) << (4 * (i & 7));
+    *(uint2*)((unsigned char*)base + (elem >> 1)) = make_uint2(w[0], w[1]);
+  }
+}
+
+// Each thread owns one group of 16 channels for the whole launch (its dyadic pairs stay in
+// registers) and walks the pixels with a grid stride.
+template <int MB, int RB, int OB>
+__global__ void __launch_bounds__(256) residual_add_vec_kernel(EltArgs a, int groups, int pix_per_block) {
+  const int g = threadIdx.x % groups;
+  const int pl = threadIdx.x / groups;
+  if (pl >= pix_per_block) return;
+  const int ch0 = g * 16;
+  int mb[16], mc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { mb[i] = __ldg(a.mb + ch0 + i); mc[i] = __ldg(a.mc + ch0 + i); }
+  int rb[16], rc[16];
+  if constexpr (RB != 0) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { rb[i] = __ldg(a.rb + ch0 + i); rc[i] = __ldg(a.rc + ch0 + i); }
+  }
+  const long long step = (long long)gridDim.x * pix_per_block;
+  for (long long p = (long long)blockIdx.x * pix_per_block + pl; p < a.pixels; p += step) {
+    const long long e = p * a.ch + ch0;
+    int m[16], o[16];
+    load16<MB>(a.main_t, e, a.main_signed, m);
+    if constexpr (RB != 0) {
+      int r[16];
+      load16<RB>(a.res, e, a.res_signed, r);
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        o[i] = hq_clamp_ll(hq_dn(m[i], mb[i], mc[i]) + hq_dn(r[i], rb[i], rc[i]), a.relu, a.qmin, a.qmax);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[i] = hq_clamp_ll(hq_dn(m[i], mb[i], mc[i]), a.relu, a.qmin, a.qmax);
+    }
+    store16<OB>(a.out, e, o);
+  }
+}
+
+// Any channel count: one thread per output byte (one element at 8 bit, two at 4 bit).
+__global__ void residual_add_scalar_kernel(EltArgs a) {
+  const int per = (a.out_bits == 4) ? 2 : 1;
+  const long long total = a.pixels * a.ch / per;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    int q[2] = {0, 0};
+    for (int j = 0; j < per; ++j) {
+      const long long e = i * per + j;
+      const int ch = (int)(e % a.ch);
+      long long y = hq_dn(hq_load_elem(a.main_t, e, a.main_bits, a.main_signed), a.mb[ch], a.mc[ch]);
+      if (a.res) y += hq_dn(hq_load_elem(a.res, e, a.res_bits, a.res_signed), a.rb[ch], a.rc[ch]);
+      q[j] = hq_clamp_ll(y, a.relu, a.qmin, a.qmax);
+    }
+    if (a.out_bits == 4) ((unsigned char*)a.out)[i] = (unsigned char)((q[0] & 0xF) | ((q[1] & 0xF) << 4));
+    else ((unsigned char*)a.out)[i] = (unsigned char)(q[0] & 0xFF);
+  }
+}
+
+template <int MB, int RB>
+cudaError_t launch_vec_out(const EltArgs& a, int groups, int ppb, int grid, cudaStream_t s) {
+  if (a.out_bits == 8) residual_add_vec_kernel<MB, RB, 8><<<grid, 256, 0, s>>>(a, groups, ppb);
+  else residual_add_vec_kernel<MB, RB, 4><<<grid, 256, 0, s>>>(a, groups, ppb);
+  return cudaGetLastError();
+}
+
+template <int MB>
+cudaError_t launch_vec_res(const EltArgs& a, int groups, int ppb, int grid, cudaStream_t s) {
+  if (!a.res) return launch_vec_out<MB, 0>(a, groups, ppb, grid, s);
+  switch (a.res_bits) {
+    case 4: return launch_vec_out<MB, 4>(a, groups, ppb, grid, s);
+    case 8: return launch_vec_out<MB, 8>(a, groups, ppb, grid, s);
+    default: return launch_vec_out<MB, 32>(a, groups, ppb, grid, s);
+  }
+}
+
+// ---- global average pooling -----------------------------------------------------------------
+// One thread per (image, 4 channels): 8-bit input read as 32-bit words, coalesced across threads.
+__global__ void avgpool_vec4_kernel(const unsigned* __restrict__ in, int n, int hw, int ch, int is_signed,
+                                    const int32_t* __restrict__ b, const int32_t* __restrict__ c,
+                                    int qmin, int qmax, unsigned* __restrict__ out) {
+  const int cg = ch >> 2;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * cg) return;
+  const int img = i / cg, g = i - img * cg;
+  const unsigned* p = in + (long long)img * hw * cg + g;
+  int s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+  for (int k = 0; k < hw; ++k) {
+    const unsigned v = __ldg(p + (long long)k * cg);
+    if (is_signed) {
+      s0 += (int)(signed char)(v & 0xFF); s1 += (int)(signed char)((v >> 8) & 0xFF);
+      s2 += (int)(signed char)((v >> 16) & 0xFF); s3 += (int)(signed char)(v >> 24);
+    } else {
+      s0 += (int)(v & 0xFF); s1 += (int)((v >> 8) & 0xFF); s2 += (int)((v >> 16) & 0xFF); s3 += (int)(v >> 24);
+    }
+  }
+  const int sums[4] = {s0, s1, s2, s3};
+  unsigned w = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int q = hq_clamp_ll(hq_dn(sums[j], b[4 * g + j], c[4 * g + j]), 0, qmin, qmax);
+    w |= (unsigned)(q & 0xFF) << (8 * j);
+  }
+  out[i] = w;
+}
+
+__global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int in_bits, int in_signed,
+                                      const int32_t* b, const int32_t* c, int qmin, int qmax,
+                                      void* out, int out_bits) {
+  const int per = (out_bits == 4) ? 2 : 1;
+  const int total = n * ch / per;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int q[2] = {0, 0};
+  for (int j = 0; j < per; ++j) {
+    const int e = i * per + j;
+    const int img = e / ch, k = e - img * ch;
+    long long sum = 0;
+    for (int px = 0; px < hw; ++px)
+      sum += hq_load_elem(in, ((long long)img * hw + px) * ch + k, in_bits, in_signed);
+    q[j] = hq_clamp_ll(hq_dn((int)sum, b[k], c[k]), 0, qmin, qmax);
+  }
+  if (out_bits == 4) ((unsigned char*)out)[i] = (unsigned char)((q[0] & 0xF) | ((q[1] & 0xF) << 4));
+  else ((unsigned char*)out)[i] = (unsigned char)(q[0] & 0xFF);
+}
+
+// ---- max pooling ----------------------------------------------------------------------------
+template <bool SIGNED>
+__global__ void maxpool_vec16_kernel(const uint4* __restrict__ in, int n, int h, int w, int cg,
+                                     int k, int stride, int pad, uint4* __restrict__ out, int ho, int wo) {
+  const long long total = (long long)n * ho * wo * cg;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int g = (int)(i % cg);
+    long long t = i / cg;
+    const int ow = (int)(t % wo); t /= wo;
+    const int oh = (int)(t % ho);
+    const int img = (int)(t / ho);
+    const unsigned init = SIGNED ? 0x80808080u : 0u;
+    uint4 m = make_uint4(init, init, init, init);
+    for (int r = 0; r < k; ++r) {
+      const int ih = oh * stride + r - pad;
+      if (ih < 0 || ih >= h) continue;
+      for (int s = 0; s < k; ++s) {
+        const int iw = ow * stride + s - pad;
+        if (iw < 0 || iw >= w) continue;
+        const uint4 v = __ldg(in + (((long long)img * h + ih) * w + iw) * cg + g);
+        if (SIGNED) { m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y); m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w); }
+        else        { m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w); }
+      }
+    }
+    out[i] = m;
+  }
+}
+
+__global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int ch, int is_signed,
+                                      int k, int stride, int pad, void* out, int ho, int wo) {
+  const long long total = (long long)n * ho * wo * ch;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int cc = (int)(i % ch);
+    long long t = i / ch;
+    const int ow = (int)(t % wo); t /= wo;
+    const int oh = (int)(t % ho);
+    const int img = (int)(t / ho);
+    int best = is_signed ? -128 : 0;
+    for (int r = 0; r < k; ++r) {
+      const int ih = oh * stride + r - pad;
+      if (ih < 0 || ih >= h) continue;
+      for (int s = 0; s < k; ++s) {
+        const int iw = ow * stride + s - pad;
+        if (iw < 0 || iw >= w) continue;
+        const int v = hq_load_elem(in, (((long long)img * h + ih) * w + iw) * ch + cc, 8, is_signed);
+        best = v > best ? v : best;
+      }
+    }
+    ((unsigned char*)out)[i] = (unsigned char)(best & 0xFF);
+  }
+}
+
+}  // namespace
+
+cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s) {
+  if (a.pixels == 0) return cudaSuccess;
+  const int groups = a.ch / 16;
+  if (a.ch % 16 == 0 && groups <= 256) {
+    const int ppb = 256 / groups;
+    long long blocks = (a.pixels + ppb - 1) / ppb;
+    const long long cap = (long long)sm_count * 8;
+    const int grid = (int)(blocks < cap ? blocks : cap);
+    switch (a.main_bits) {
+      case 4: return launch_vec_res<4>(a, groups, ppb, grid, s);
+      case 8: return launch_vec_res<8>(a, groups, ppb, grid, s);
+      default: return launch_vec_res<32>(a, groups, ppb, grid, s);
+    }
+  }
+  const long long total = a.pixels * a.ch / (a.out_bits == 4 ? 2 : 1);
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)sm_count * 16;
+  residual_add_scalar_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int in_bits, int in_signed,
+                              const int32_t* b, const int32_t* c, int qmin, int qmax,
+                              void* out, int out_bits, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  if (in_bits == 8 && out_bits == 8 && ch % 4 == 0) {
+    const int total = n * (ch / 4);
+    avgpool_vec4_kernel<<<(total + 127) / 128, 128, 0, s>>>((const unsigned*)in, n, h * w, ch, in_signed,
+                                                             b, c, qmin, qmax, (unsigned*)out);
+  } else {
+    const int total = n * ch / (out_bits == 4 ? 2 : 1);
+    avgpool_scalar_kernel<<<(total + 127) / 128, 128, 0, s>>>(in, n, h * w, ch, in_bits, in_signed, b, c,
+                                                               qmin, qmax, out, out_bits);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int is_signed,
+                              int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  if (ch % 16 == 0) {
+    const long long total = (long long)n * ho * wo * (ch / 16);
+    long long blocks = (total + 255) / 256;
+    if (blocks > (1 << 20)) blocks = 1 << 20;
+    if (is_signed)
+      maxpool_vec16_kernel<true><<<(int)blocks, 256, 0, s>>>((const uint4*)in, n, h, w, ch / 16, k, stride, pad,
+                                                              (uint4*)out, ho, wo);
+    else
+      maxpool_vec16_kernel<false><<<(int)blocks, 256, 0, s>>>((const uint4*)in, n, h, w, ch / 16, k, stride, pad,
+                                                               (uint4*)out, ho, wo);
+  } else {
+    const long long total = (long long)n * ho * wo * ch;
+    long long blocks = (total + 255) / 256;
+    if (blocks > (1 << 20)) blocks = 1 << 20;
+    maxpool_scalar_kernel<<<(int)blocks, 256, 0, s>>>(in, n, h, w, ch, is_signed, k, stride, pad, out, ho, wo);
+  }
+  return cudaGetLastError();
+}

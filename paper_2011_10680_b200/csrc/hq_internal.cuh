@@ -1,0 +1,78 @@
+// Internal declarations shared by the translation units of libhq.so (CUDA side only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/hq.h"
+
+// Device-side status word values (written by a kernel that gave up a bounded wait).
+enum : uint32_t {
+  HQ_DEV_OK = 0,
+  HQ_DEV_TIMEOUT_PRODUCER = 1,   // TMA producer waited too long for a free stage
+  HQ_DEV_TIMEOUT_MMA = 2,        // MMA issuer waited too long for operands or a free accumulator
+  HQ_DEV_TIMEOUT_EPILOGUE = 3,   // epilogue waited too long for a finished accumulator
+  HQ_DEV_TIMEOUT_DRAIN = 4       // teardown waited too long for work in flight
+};
+
+struct hq_handle {
+  int32_t device;
+  int32_t conv_path;          // 0 auto, 1 CUDA cores only, 2 tensor cores or fail
+  int32_t sm_count;
+  uint32_t* dev_status;       // one word in device memory, sticky until hq_sync
+  void* workspace;            // scratch owned by the handle (grown on demand, never inside a capture)
+  size_t workspace_bytes;
+};
+
+// ------------------------------------------------------------------------------------------
+// Dyadic arithmetic (Eq. 4): dn(q, b, c) = (q*b + 2^(c-1)) >> c, 64-bit product, arithmetic shift.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ long long hq_dn(int q, int b, int c) {
+  return ((long long)q * (long long)b + (1LL << (c - 1))) >> c;
+}
+
+// Element access for dense tensors with 4, 8 or 32 bits per element (even element = low nibble).
+__device__ __forceinline__ int hq_load_elem(const void* base, long long idx, int bits, int is_signed) {
+  if (bits == 32) return ((const int*)base)[idx];
+  if (bits == 8) return is_signed ? (int)((const signed char*)base)[idx] : (int)((const unsigned char*)base)[idx];
+  const unsigned byte = ((const unsigned char*)base)[idx >> 1];
+  int v = (idx & 1) ? (int)(byte >> 4) : (int)(byte & 0xF);
+  if (is_signed && (v & 8)) v -= 16;
+  return v;
+}
+
+__device__ __forceinline__ int hq_clamp_ll(long long y, int relu, int qmin, int qmax) {
+  if (relu && y < 0) y = 0;
+  if (y < (long long)qmin) y = qmin;
+  if (y > (long long)qmax) y = qmax;
+  return (int)y;
+}
+
+// Launchers implemented in the other translation units.  All return a cudaError_t from the launch.
+struct ConvArgs {
+  const void* in; int32_t n, h, w, cin, in_bits, in_signed;
+  const void* wgt; int32_t cout, kh, kw, stride, pad;
+  const int32_t* bias; const int32_t* b; const int32_t* c;
+  const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
+  int32_t relu, qmin, qmax;
+  void* out; int32_t ho, wo, out_bits, out_signed;
+};
+
+struct EltArgs {
+  const void* main_t; int32_t main_bits, main_signed; const int32_t* mb; const int32_t* mc;
+  const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
+  long long pixels; int32_t ch; int32_t relu, qmin, qmax;
+  void* out; int32_t out_bits;
+};
+
+cudaError_t hq_launch_conv_cuda_core(const ConvArgs& a, cudaStream_t s);
+bool hq_conv_tc_init();
+bool hq_conv_tc_supported(const ConvArgs& a);
+// Tensor-core path; returns HQ_OK, HQ_ERR_UNSUPPORTED or HQ_ERR_CUDA.
+hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
+cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s);
+cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int in_bits, int in_signed,
+                              const int32_t* b, const int32_t* c, int qmin, int qmax,
+                              void* out, int out_bits, cudaStream_t s);
+cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int is_signed,
+                              int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s);

@@ -1,0 +1,267 @@
+"""Parity of the CUDA library with the CPU oracle, element by element and bit-exact, through the C ABI."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_2011_10680_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hq():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    h = binding.Handle(0)
+    yield h
+    h.close()
+
+
+def oracle():
+    from oracle import hqref
+    return hqref
+
+
+def host(t, like: np.ndarray) -> np.ndarray:
+    return t.cpu().numpy().view(like.dtype).reshape(like.shape)
+
+
+def run_conv_and_compare(hq, case, path):
+    from paper_2011_10680_b200 import binding
+    hq.set_conv_path(path)
+    try:
+        st, out = hq.conv_case(case)
+        assert st == binding.HQ_OK, binding.status_string(st)
+        hq.sync()
+    finally:
+        hq.set_conv_path(0)
+    ref = oracle().conv_case(case)
+    got = host(out, ref)
+    if not np.array_equal(got, ref):
+        bad = np.argwhere(got != ref)
+        raise AssertionError(f"{len(bad)} of {ref.size} outputs differ; first at {bad[0]}: got {got[tuple(bad[0])]} want {ref[tuple(bad[0])]}")
+
+
+# ------------------------------------------------------------------ CUDA-core conv path --------
+CORE_CASES = [
+    # n, h, w, cin, cout, k, stride, pad, bits, out_bits, residual, res_bits, relu
+    (2, 9, 11, 3, 8, 7, 2, 3, 8, 8, False, 8, True),        # stem-like, odd channels
+    (1, 8, 8, 16, 12, 3, 1, 1, 8, 8, True, 8, True),
+    (2, 7, 6, 8, 10, 3, 2, 1, 8, 32, False, 8, False),
+    (1, 6, 6, 8, 8, 1, 1, 0, 4, 4, False, 8, True),
+    (2, 5, 7, 16, 6, 3, 1, 1, 4, 8, True, 32, True),
+    (1, 6, 6, 6, 4, 3, 1, 1, 4, 8, False, 8, False),         # 4-bit, cin not a multiple of 8
+]
+
+
+@pytest.mark.parametrize("cfg", CORE_CASES)
+def test_conv_cuda_core_path(hq, cfg):
+    n, h, w, cin, cout, k, stride, pad, bits, out_bits, residual, res_bits, relu = cfg
+    case = inputs.conv_case(101, n, h, w, cin, cout, k, stride, pad, bits=bits, out_bits=out_bits,
+                            residual=residual, res_bits=res_bits, relu=relu, c_range=(38, 44))
+    run_conv_and_compare(hq, case, path=1)
+
+
+def test_conv_cuda_core_signed_input(hq):
+    case = inputs.conv_case(102, 1, 6, 6, 8, 8, 3, 1, 1, in_signed=True, c_range=(38, 44))
+    run_conv_and_compare(hq, case, path=1)
+
+
+# ------------------------------------------------------------------ tensor-core conv path ------
+TC_CASES = [
+    # n, h, w, cin, cout, k, stride, pad, out_bits, residual, res_bits, relu
+    (1, 56, 56, 64, 64, 3, 1, 1, 8, False, 8, True),         # benchmark config 1 geometry (ragged last M tile)
+    (2, 16, 16, 128, 128, 1, 1, 0, 8, False, 8, True),       # 1x1, 128-byte K blocks, 4 M tiles
+    (2, 14, 14, 256, 64, 3, 1, 1, 8, False, 8, True),        # several K chunks per tap
+    (3, 15, 13, 64, 96, 3, 2, 1, 8, False, 8, True),         # stride 2, odd extents, N not a multiple of the tile
+    (2, 28, 28, 64, 128, 1, 2, 0, 8, False, 8, False),       # strided 1x1 (shortcut conv), signed output
+    (2, 14, 14, 64, 256, 1, 1, 0, 8, True, 8, True),         # residual, N = 256
+    (1, 14, 14, 128, 512, 1, 1, 0, 8, True, 32, True),       # INT32 residual, two N tiles
+    (2, 10, 10, 32, 72, 3, 1, 1, 32, False, 8, False),       # 32-byte K blocks, INT32 output, N tail
+    (1, 9, 9, 96, 40, 5, 1, 2, 8, False, 8, True),           # 5x5, cin = 3 x 32
+    (2, 12, 12, 64, 64, 3, 1, 1, 4, False, 8, True),         # uint4 output
+    (1, 7, 7, 512, 1000, 1, 1, 0, 32, False, 8, False),      # classifier-like N = 1000
+]
+
+
+@pytest.mark.parametrize("cfg", TC_CASES)
+def test_conv_tensor_core_path(hq, cfg):
+    n, h, w, cin, cout, k, stride, pad, out_bits, residual, res_bits, relu = cfg
+    kk = k * k * cin
+    lo = 36 + int(np.log2(kk)) // 2
+    case = inputs.conv_case(201, n, h, w, cin, cout, k, stride, pad, bits=8, out_bits=out_bits, residual=residual,
+                            res_bits=res_bits, relu=relu, c_range=(lo, lo + 4) if out_bits != 4 else (lo + 4, lo + 8))
+    run_conv_and_compare(hq, case, path=2)
+
+
+def test_conv_tensor_core_config1_exact_distribution(hq):
+    run_conv_and_compare(hq, inputs.config1_case(), path=2)
+
+
+def test_conv_tensor_core_signed_input_and_small_c(hq):
+    case = inputs.conv_case(203, 1, 12, 12, 64, 64, 3, 1, 1, in_signed=True, relu=False, c_range=(41, 45))
+    run_conv_and_compare(hq, case, path=2)
+    # shifts below 32 and very large shifts both take the general 64-bit path
+    case = inputs.conv_case(204, 1, 12, 12, 64, 64, 1, 1, 0, relu=True, c_range=(20, 62))
+    run_conv_and_compare(hq, case, path=2)
+
+
+def test_linear_matches_oracle_and_conv(hq):
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(7, 1)
+    x = g.integers(0, 256, size=(8, 1, 1, 512), dtype=np.int64).astype(np.uint8)
+    w = g.integers(-127, 128, size=(1000, 1, 1, 512), dtype=np.int64).astype(np.int8)
+    bias = g.integers(-(1 << 15), 1 << 15, size=1000, dtype=np.int64).astype(np.int32)
+    ref = oracle().linear(x.reshape(8, 512), 512, 8, 0, w, 1000, bias, None, None, 0, -(1 << 31), (1 << 31) - 1, 32, 1)
+    out = binding.alloc_out(8, 1, 1, 1000, 32, 1)
+    st = hq.conv2d(binding.to_device(x), 8, 0, 512, binding.to_device(w), 1000, 1, 1, 1, 0, binding.to_device(bias),
+                   None, None, out, 32, 1, relu=0, qmin=-(1 << 31), qmax=(1 << 31) - 1, linear=True)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
+# ------------------------------------------------------------------ memory-bound kernels -------
+@pytest.mark.parametrize("main_bits,res_bits,out_bits,ch", [
+    (32, 8, 8, 64), (8, 8, 8, 256), (8, 0, 4, 64), (32, 32, 8, 48), (4, 8, 8, 32), (8, 8, 8, 10), (32, 0, 4, 6),
+])
+def test_residual_add(hq, main_bits, res_bits, out_bits, ch):
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(301, main_bits, res_bits, out_bits, ch)
+    shape = (3, 7, 9, ch)
+
+    def draw(bits):
+        if bits == 32:
+            return g.integers(-(1 << 22), 1 << 22, size=shape, dtype=np.int64).astype(np.int32), 1
+        if bits == 8:
+            return g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8), 0
+        return inputs.pack4(g.integers(0, 16, size=shape, dtype=np.int64)), 0
+
+    main, main_signed = draw(main_bits)
+    mb = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+    mc = g.integers(45, 50, size=ch).astype(np.int32) if main_bits == 32 else g.integers(29, 34, size=ch).astype(np.int32)
+    res = rb = rc = None
+    res_signed = 0
+    if res_bits:
+        res, res_signed = draw(res_bits)
+        rb = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+        rc = g.integers(45, 50, size=ch).astype(np.int32) if res_bits == 32 else g.integers(29, 34, size=ch).astype(np.int32)
+    qmax = 255 if out_bits == 8 else 15
+    ref = oracle().residual_add(main, main_bits, main_signed, mb, mc, res, res_bits, res_signed, rb, rc, ch, 1, 0, qmax,
+                                out_bits, 0)
+    out = binding.alloc_out(*shape[:3], ch, out_bits, 0)
+    st = hq.residual_add(binding.to_device(main), main_bits, main_signed, binding.to_device(mb), binding.to_device(mc),
+                         binding.to_device(res), res_bits, res_signed, binding.to_device(rb), binding.to_device(rc),
+                         ch, 1, 0, qmax, out, out_bits, 0)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
+@pytest.mark.parametrize("n,hw,ch,in_bits", [(4, 7, 64, 8), (2, 7, 2048, 8), (3, 5, 6, 8), (2, 4, 16, 32), (2, 3, 8, 4)])
+def test_avgpool_requant(hq, n, hw, ch, in_bits):
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(302, n, hw, ch, in_bits)
+    if in_bits == 8:
+        x = g.integers(0, 256, size=(n, hw, hw, ch), dtype=np.int64).astype(np.uint8)
+    elif in_bits == 32:
+        x = g.integers(-(1 << 16), 1 << 16, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+    else:
+        x = inputs.pack4(g.integers(0, 16, size=(n, hw, hw, ch), dtype=np.int64))
+    scale = np.exp(g.uniform(np.log(0.2), np.log(2.0), size=ch)) / (hw * hw) / (256.0 if in_bits == 32 else 1.0)
+    b, c = inputs.dyadic_from_scale(scale)
+    ref = oracle().avgpool_requant(x, ch, in_bits, int(in_bits == 32), b, c, 0, 255)
+    out = binding.alloc_out(n, 1, 1, ch, 8, 0)
+    st = hq.avgpool_requant(binding.to_device(x), ch, in_bits, int(in_bits == 32), binding.to_device(b),
+                            binding.to_device(c), 0, 255, out, 8, 0)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
+@pytest.mark.parametrize("n,h,w,ch", [(2, 112, 112, 64), (3, 9, 11, 16), (2, 8, 7, 5)])
+def test_maxpool(hq, n, h, w, ch):
+    from paper_2011_10680_b200 import binding
+    x = inputs.rng(303, n, h, w, ch).integers(0, 256, size=(n, h, w, ch), dtype=np.int64).astype(np.uint8)
+    ref = oracle().maxpool(x, 3, 2, 1)
+    out = binding.alloc_out(n, ref.shape[1], ref.shape[2], ch, 8, 0)
+    st = hq.maxpool(binding.to_device(x), ch, 0, 3, 2, 1, out)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
+# ------------------------------------------------------------------ argument errors ------------
+def test_invalid_arguments_return_codes_not_crashes(hq):
+    from paper_2011_10680_b200 import binding
+    case = inputs.conv_case(401, 1, 8, 8, 32, 32, 3, 1, 1)
+    dev = binding.upload_case(case)
+    out = binding.alloc_out(1, 8, 8, 32, 8, 0)
+    args = dict(res=None, relu=1, qmin=0, qmax=255)
+    ok = hq.conv2d(dev["x"], 8, 0, 32, dev["wgt"], 32, 3, 3, 1, 1, dev["bias"], dev["b"], dev["c"], out, 8, 0, **args)
+    assert ok == binding.HQ_OK
+    bad_shape = binding.alloc_out(1, 7, 8, 32, 8, 0)
+    assert hq.conv2d(dev["x"], 8, 0, 32, dev["wgt"], 32, 3, 3, 1, 1, dev["bias"], dev["b"], dev["c"], bad_shape, 8, 0,
+                     **args) == binding.HQ_ERR_INVALID_ARG
+    assert hq.conv2d(dev["x"], 8, 0, 32, dev["wgt"], 32, 3, 3, 1, 1, dev["bias"], None, None, out, 8, 0,
+                     **args) == binding.HQ_ERR_INVALID_ARG
+    assert hq.conv2d(dev["x"], 8, 0, 32, dev["wgt"], 32, 3, 3, 1, 1, dev["bias"], dev["b"], dev["c"], out, 8, 0,
+                     res=None, relu=1, qmin=0, qmax=256) == binding.HQ_ERR_INVALID_ARG
+    off = dev["x"].view(-1)[1:1 + 4 * 4 * 32].view(1, 4, 4, 32)      # data pointer is 1 byte past alignment
+    assert hq.maxpool(off, 32, 0, 3, 2, 1, binding.alloc_out(1, 2, 2, 32, 8, 0)) == binding.HQ_ERR_ALIGNMENT
+    hq.set_conv_path(2)
+    try:
+        c3 = inputs.conv_case(402, 1, 6, 6, 3, 8, 3, 1, 1)
+        st, _ = hq.conv_case(c3)
+        assert st == binding.HQ_ERR_UNSUPPORTED          # no silent fallback when tensor cores are demanded
+    finally:
+        hq.set_conv_path(0)
+    hq.sync()
+
+
+# ------------------------------------------------------------------ networks -------------------
+def run_network_and_compare(hq, table, batch, seed):
+    from oracle.network import run_network
+    from paper_2011_10680_b200 import binding
+    images = inputs.random_images(seed, batch, table["image_hw"])
+    ref = run_network(table, images)
+    net = binding.Network(hq, table, batch)
+    try:
+        d_img = binding.to_device(images)
+        logits = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+        taps = net.alloc_taps()
+        assert net.run(d_img, logits, taps) == binding.HQ_OK
+        hq.sync()
+        for i, (t, r) in enumerate(zip(taps, ref)):
+            got = t.cpu().numpy().view(r.dtype).reshape(r.shape)
+            assert np.array_equal(got, r), f"layer {i} ({table['layers'][i]['op']}) differs in {(got != r).sum()} of {r.size}"
+        assert np.array_equal(host(logits, ref[-1]), ref[-1])
+        # graph replay path (no taps) must give the same logits, twice in a row
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for _ in range(2):
+                logits.zero_()
+                assert net.run(d_img, logits, None) == binding.HQ_OK
+                hq.sync()
+                assert np.array_equal(host(logits, ref[-1]), ref[-1])
+    finally:
+        net.close()
+    return ref
+
+
+def test_reduced_resnet18_and_resnet50_every_layer(hq):
+    for depth, mixed in ((18, False), (50, False), (50, True)):
+        t = inputs.resnet_table(depth, seed=5, image_hw=64, classes=24, width=32, mixed=mixed)
+        run_network_and_compare(hq, t, batch=3, seed=depth)
+
+
+def test_resnet18_imagenet_shape_batch8_every_layer(hq):
+    """Benchmark config 2: ResNet-18, 224x224x3, 1000 classes, batch 8, all layers INT8."""
+    t = inputs.resnet_table(18, seed=2)
+    ref = run_network_and_compare(hq, t, batch=8, seed=2)
+    sat = [float(np.mean((r == 0) | (r == 255))) for r, l in zip(ref, t["layers"]) if l["op"] == "conv" and l["out_bits"] == 8]
+    assert min(sat) < 0.9, "every layer is saturated: the workload would not exercise the requantization"
