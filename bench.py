@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the integer-only inference hot path: images/s of a table-driven ResNet run.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path (every layer of the table) over one batch of synthetic
+images.  `value` is measured with the batch resident in HBM; `e2e` includes the copy of the
+step's images from pinned host memory and the read-back of its logits.  Under torchrun every rank
+runs the same batch size on its own GPU (independent images, no collective on the data path:
+weak scaling); the time is the maximum over ranks.  `--impl reference` times the CPU oracle.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2011_10680_b200 import inputs
+
+WORKLOADS = {
+    # name: (depth, mixed, batch, seed)
+    "resnet50_int8_b256": (50, False, 256, 3),
+    "resnet50_int4_8_mixed_b256": (50, True, 256, 4),
+    "resnet18_int8_b8": (18, False, 8, 2),
+}
+METRIC = "int-only ResNet-50 images/s @bs256; fused conv INT TOPS vs tcgen05 i8 peak"
+NOMINAL_I8_TOPS = 4500.0
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return d["hbm_gbs"], d["bf16_tflops_sustained"], "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS * 1400.0 / 1590.0, "fallback"
+
+
+def layer_work(table, batch):
+    """Algorithmic ops and bytes of every layer: what the method itself must move, inputs read once."""
+    shapes, bits = table["shapes"], table["bits"]
+    hw_in = {-1: (table["image_hw"], table["image_hw"], 3, 8)}
+    for i in range(len(table["layers"])):
+        hw_in[i] = (*shapes[i], bits[i])
+    rows = []
+    for i, l in enumerate(table["layers"]):
+        h, w, c, b_in = hw_in[l["in0"]]
+        ho, wo, co = shapes[i]
+        out_bytes = batch * ho * wo * co * l["out_bits"] // 8
+        ops = 0
+        if l["op"] in ("conv", "linear"):
+            k = l["kh"] * l["kw"] * l["cin"]
+            m = batch * ho * wo
+            ops = 2 * m * co * k
+            if l["kh"] == 1 and l["stride"] > 1:
+                in_bytes = m * l["cin"] * b_in // 8          # only the sampled pixels
+            else:
+                in_bytes = batch * h * w * c * b_in // 8
+            byt = in_bytes + co * k * l["bits"] // 8 + out_bytes + 13 * co
+            if l["in1"] >= 0:
+                byt += batch * ho * wo * co * hw_in[l["in1"]][3] // 8
+        else:
+            byt = batch * h * w * c * b_in // 8 + out_bytes
+            if l["in1"] >= 0:
+                byt += out_bytes
+        rows.append(dict(layer=i, op=l["op"], ops=ops, bytes=byt))
+    return rows
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle sampling while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line)
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax = float(f[1])
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def run_reference(args, rank):
+    """The CPU oracle as it stands, on a bounded sample of the same workload per step."""
+    if rank != 0:
+        return
+    from oracle import hqref
+    from oracle.network import run_network
+    depth, mixed, batch, seed = WORKLOADS[args.workload]
+    table = inputs.resnet_table(depth, seed, mixed=mixed)
+    t0 = time.perf_counter()
+    run_network(table, inputs.random_images(seed, 1))
+    t1 = time.perf_counter() - t0
+    total_steps = args.steps + args.warmup
+    sample = int(max(1, min(batch, 90.0 / max(t1, 1e-3) / total_steps)))
+    images = inputs.random_images(seed, sample)
+    for _ in range(args.warmup):
+        run_network(table, images)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run_network(table, images)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    cores = hqref.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8" if not mixed else "int4/int8", "data": "synthetic",
+        "config": {"workload": args.workload, "global_batch": batch, "sample_images_per_step": sample,
+                   "note": "CPU oracle (int64, 7-loop conv, OpenMP over rows) on the first images of the batch"},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} of {batch} images per step"},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50_int8_b256", choices=sorted(WORKLOADS))
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers-out", default=None, help="write the per-layer table (JSON) to this file")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2011_10680_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    depth, mixed, batch, seed = WORKLOADS[args.workload]
+    batch = args.batch or batch
+    table = inputs.resnet_table(depth, seed, mixed=mixed)
+    hq = binding.Handle(local_rank)
+    net = binding.Network(hq, table, batch)
+    images_h = torch.from_numpy(inputs.random_images(seed + 1000 * rank, batch)).pin_memory()
+    images_d = images_h.cuda()
+    logits_d = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.Stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---------------- device-resident throughput -------------------------------------------
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            assert net.run(images_d, logits_d) == binding.HQ_OK
+        hq.sync()
+        sampler = ClockSampler(local_rank)
+        barrier()
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.25)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            net.run(images_d, logits_d)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop() if rank == 0 else None
+        hq.sync()
+
+        # ---------------- end to end: pinned host images in, logits out, double-buffered ----
+        copy_stream = torch.cuda.Stream()
+        img_bufs = [torch.empty_like(images_d) for _ in range(2)]
+        log_bufs = [torch.empty_like(logits_d) for _ in range(2)]
+        logits_h = [torch.empty(net.logits_shape, dtype=torch.int32).pin_memory() for _ in range(2)]
+        ready = [torch.cuda.Event() for _ in range(2)]
+        done = [torch.cuda.Event() for _ in range(2)]
+
+        def e2e_steps(k):
+            for i in range(k):
+                j = i & 1
+                with torch.cuda.stream(copy_stream):
+                    copy_stream.wait_event(done[j])              # buffer j free again
+                    img_bufs[j].copy_(images_h, non_blocking=True)
+                    ready[j].record(copy_stream)
+                stream.wait_event(ready[j])
+                net.run(img_bufs[j], log_bufs[j])
+                logits_h[j].copy_(log_bufs[j], non_blocking=True)
+                done[j].record(stream)
+
+        e2e_steps(max(args.warmup, 4))
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        e2e_steps(args.steps)
+        f1.record(stream)
+        copy_stream.synchronize()
+        barrier()
+        ms_e2e = f0.elapsed_time(f1)
+        hq.sync()
+        assert torch.equal(logits_h[0], logits_d.cpu()) and torch.equal(logits_h[1], logits_d.cpu())
+
+        # ---------------- per-layer device times (CUDA events around each layer) -------------
+        reps = 3
+        layer_ns = np.zeros(len(table["layers"]))
+        for _ in range(reps):
+            layer_ns += np.array(net.time_layers(images_d, logits_d), dtype=np.float64)
+        layer_ns /= reps
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+
+    if rank == 0:
+        hbm_peak, bf16_peak, peak_kind = measured_peaks()
+        work = layer_work(table, batch)
+        rows, tc_bytes, tc_ops, tc_ns = [], 0, 0, 0.0
+        for wk, ns, l in zip(work, layer_ns, table["layers"]):
+            on_tc = l["op"] in ("conv", "linear") and l["bits"] == 8 and l["cin"] % 32 == 0
+            if on_tc:
+                tc_bytes += wk["bytes"]; tc_ops += wk["ops"]; tc_ns += ns
+            rows.append({**wk, "us": ns / 1e3, "tensor_core": on_tc, "gbs": wk["bytes"] / max(ns, 1),
+                         "tops": wk["ops"] / max(ns, 1) / 1e3})
+        if args.layers_out:
+            json.dump(rows, open(args.layers_out, "w"), indent=1)
+        n_conv_tc = sum(1 for r in rows if r["tensor_core"])
+        achieved = tc_bytes / max(tc_ns, 1)                      # bytes per ns = GB/s
+        total_ops = sum(r["ops"] for r in rows)
+        value = world * batch * args.steps / (ms / 1e3)
+        line = {
+            "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8" if not mixed else "int4/int8", "data": "synthetic",
+            "config": {"workload": args.workload + (f" (batch overridden to {batch})" if args.batch else ""),
+                       "global_batch": world * batch, "image": "224x224x3 uint8",
+                       "parallelism": f"dp{world}" if world > 1 else "single",
+                       "l2": "activations per step (GBs) exceed the 126 MB L2; no explicit flush",
+                       "launch": "CUDA graph replay of the whole layer table"},
+            "int_tops": total_ops * args.steps / (ms / 1e3) / 1e12 * world,
+            "e2e": {"value": world * batch * args.steps / (ms_e2e / 1e3), "unit": "images/s",
+                    "h2d_bytes_per_step": int(images_h.numel()), "d2h_bytes_per_step": int(logits_d.numel() * 4),
+                    "note": "pinned host images -> device -> hq_run_network -> logits to pinned host, two buffers"},
+            "gpu_launches": net.launch_count() * args.steps,
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                         "frac": achieved / hbm_peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                         "kernel": "conv_tc_kernel", "launches_per_step": n_conv_tc,
+                         "avg_launch_us": tc_ns / 1e3 / max(n_conv_tc, 1),
+                         "algorithmic_bytes_per_step": tc_bytes,
+                         "tensor_tops": tc_ops / max(tc_ns, 1) / 1e3,
+                         "tensor_frac_of_nominal_4500": tc_ops / max(tc_ns, 1) / 1e3 / NOMINAL_I8_TOPS,
+                         "tensor_frac_of_2x_measured_bf16": tc_ops / max(tc_ns, 1) / 1e3 / (2 * bf16_peak),
+                         "share_of_step": tc_ns / max(layer_ns.sum(), 1)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            from oracle import hqref
+            from oracle.network import run_network
+            one = inputs.random_images(seed, 1)
+            t0 = time.perf_counter(); run_network(table, one); t1 = time.perf_counter() - t0
+            sample = int(max(1, min(batch, 15.0 / max(t1, 1e-3))))
+            imgs = inputs.random_images(seed, sample)
+            t0 = time.perf_counter(); ref = run_network(table, imgs); dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": sample / dt, "unit": "images/s", "cores": hqref.num_threads(),
+                                    "kind": "oracle", "sample": f"first {sample} of {batch} images, one pass"}
+        print(json.dumps(line), flush=True)
+    net.close()
+    hq.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -159,6 +159,12 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
 hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* logits,
                          void* const* layer_taps, void* stream);
 
+/* Measurement aid: run the table once with plain launches and a CUDA event pair around every
+ * layer, wait for the stream, and write each layer's device time in nanoseconds to the HOST
+ * array ns[n_layers]. */
+hq_status hq_network_time_layers(hq_network* net, const hq_tensor* images, hq_tensor* logits, int64_t* ns,
+                                 void* stream);
+
 /* Bytes of layer i's stored output and the number of kernels one hq_run_network launches. */
 hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* bytes);
 hq_status hq_network_launch_count(const hq_network* net, int32_t* launches);

@@ -21,7 +21,7 @@ HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant"
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
-    "hq_network_destroy", "hq_set_conv_path", "hq_status_string",
+    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers",
 ]
 
 
@@ -76,6 +76,7 @@ def lib():
         L.hq_maxpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
         L.hq_network_create.argtypes = [vp, LP, i32, i32, i32, i32, i32, i32, C.POINTER(vp)]
         L.hq_run_network.argtypes = [vp, TP, TP, C.POINTER(vp), vp]
+        L.hq_network_time_layers.argtypes = [vp, TP, TP, C.POINTER(C.c_int64), vp]
         L.hq_network_layer_bytes.argtypes = [vp, i32, C.POINTER(C.c_int64)]
         L.hq_network_launch_count.argtypes = [vp, C.POINTER(i32)]
         L.hq_network_destroy.argtypes = [vp]
@@ -254,6 +255,15 @@ class Network:
         if taps is not None:
             tap_arr = (C.c_void_p * len(taps))(*[t.data_ptr() if t is not None else None for t in taps])
         return lib().hq_run_network(self._net, C.byref(ti), C.byref(tl), tap_arr, _stream())
+
+    def time_layers(self, images, logits):
+        """Per-layer device time in nanoseconds (CUDA events around each layer, plain launches)."""
+        ti = tensor_of(images, images.shape[3], 8, 0)
+        last = self.table["layers"][-1]
+        tl = hq_tensor(logits.data_ptr(), self.batch, 1, 1, last["cout"], last["out_bits"], last["out_signed"])
+        ns = (C.c_int64 * len(self.table["layers"]))()
+        _check(lib().hq_network_time_layers(self._net, C.byref(ti), C.byref(tl), ns, _stream()), "hq_network_time_layers")
+        return list(ns)
 
     def alloc_taps(self):
         import torch

@@ -84,10 +84,10 @@ struct hq_network {
   std::vector<long long> bytes;
   int32_t batch, image_h, image_w, image_c, image_signed;
   int32_t launches;
-  // graph cache
-  cudaGraphExec_t graph_exec;
-  const void* graph_images;
-  void* graph_logits;
+  // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
+  // that double-buffered callers do not re-capture every step
+  struct CachedGraph { cudaGraphExec_t exec; const void* images; void* logits; };
+  std::vector<CachedGraph> graphs;
 };
 
 extern "C" {
@@ -233,7 +233,6 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   if (!net) return HQ_ERR_WORKSPACE;
   net->h = h; net->batch = batch;
   net->image_h = image_h; net->image_w = image_w; net->image_c = image_c; net->image_signed = image_signed;
-  net->graph_exec = nullptr; net->graph_images = nullptr; net->graph_logits = nullptr;
   net->layers.assign(table, table + n_layers);
   net->outs.resize(n_layers);
   net->bytes.resize(n_layers);
@@ -287,10 +286,11 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
 }
 
 static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor* logits, void* const* taps,
-                            cudaStream_t s) {
+                            cudaStream_t s, cudaEvent_t* marks = nullptr) {
   hq_handle* h = net->h;
   const int n_layers = (int)net->layers.size();
   for (int i = 0; i < n_layers; ++i) {
+    if (marks && cudaEventRecord(marks[i], s) != cudaSuccess) return HQ_ERR_CUDA;
     const hq_layer& l = net->layers[i];
     hq_tensor in = (l.in0 == -1) ? *images : net->outs[l.in0];
     hq_tensor o = net->outs[i];
@@ -327,7 +327,27 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         return HQ_ERR_CUDA;
     }
   }
+  if (marks && cudaEventRecord(marks[n_layers], s) != cudaSuccess) return HQ_ERR_CUDA;
   return HQ_OK;
+}
+
+hq_status hq_network_time_layers(hq_network* net, const hq_tensor* images, hq_tensor* logits, int64_t* ns,
+                                 void* stream) {
+  if (!net || !images || !logits || !ns || !images->data || !logits->data) return HQ_ERR_INVALID_ARG;
+  const int n_layers = (int)net->layers.size();
+  std::vector<cudaEvent_t> marks(n_layers + 1, nullptr);
+  hq_status st = HQ_OK;
+  for (auto& e : marks) if (cudaEventCreate(&e) != cudaSuccess) st = HQ_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (st == HQ_OK) st = run_layers(net, images, logits, nullptr, s, marks.data());
+  if (st == HQ_OK && cudaStreamSynchronize(s) != cudaSuccess) st = HQ_ERR_CUDA;
+  for (int i = 0; i < n_layers && st == HQ_OK; ++i) {
+    float ms = 0;   // timing only: not part of the integer pipeline
+    if (cudaEventElapsedTime(&ms, marks[i], marks[i + 1]) != cudaSuccess) st = HQ_ERR_CUDA;
+    ns[i] = (int64_t)(ms * 1.0e6f);
+  }
+  for (auto& e : marks) if (e) cudaEventDestroy(e);
+  return st;
 }
 
 hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* logits, void* const* layer_taps,
@@ -348,20 +368,25 @@ hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* lo
   if (cap != cudaStreamCaptureStatusNone || layer_taps || s == nullptr) return run_layers(net, images, logits, layer_taps, s);
 
   // Otherwise replay a CUDA graph of the whole table (captured once per (images, logits) pair).
-  if (!net->graph_exec || net->graph_images != images->data || net->graph_logits != logits->data) {
-    if (net->graph_exec) { cudaGraphExecDestroy(net->graph_exec); net->graph_exec = nullptr; }
-    if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return HQ_ERR_CUDA;
-    const hq_status st = run_layers(net, images, logits, nullptr, s);
-    cudaGraph_t graph = nullptr;
-    const cudaError_t e = cudaStreamEndCapture(s, &graph);
-    if (st != HQ_OK) { if (graph) cudaGraphDestroy(graph); return st; }
-    if (e != cudaSuccess || !graph) return HQ_ERR_CUDA;
-    const cudaError_t e2 = cudaGraphInstantiate(&net->graph_exec, graph, 0);
-    cudaGraphDestroy(graph);
-    if (e2 != cudaSuccess) { net->graph_exec = nullptr; return HQ_ERR_CUDA; }
-    net->graph_images = images->data; net->graph_logits = logits->data;
+  for (const auto& g : net->graphs)
+    if (g.images == images->data && g.logits == logits->data)
+      return cudaGraphLaunch(g.exec, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+  if (net->graphs.size() >= 4) {
+    cudaGraphExecDestroy(net->graphs.front().exec);
+    net->graphs.erase(net->graphs.begin());
   }
-  return cudaGraphLaunch(net->graph_exec, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+  if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return HQ_ERR_CUDA;
+  const hq_status st = run_layers(net, images, logits, nullptr, s);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(s, &graph);
+  if (st != HQ_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+  if (e != cudaSuccess || !graph) return HQ_ERR_CUDA;
+  cudaGraphExec_t exec = nullptr;
+  const cudaError_t e2 = cudaGraphInstantiate(&exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e2 != cudaSuccess || !exec) return HQ_ERR_CUDA;
+  net->graphs.push_back({exec, images->data, logits->data});
+  return cudaGraphLaunch(exec, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* bytes) {
@@ -378,7 +403,7 @@ hq_status hq_network_launch_count(const hq_network* net, int32_t* launches) {
 
 hq_status hq_network_destroy(hq_network* net) {
   if (!net) return HQ_ERR_INVALID_ARG;
-  if (net->graph_exec) cudaGraphExecDestroy(net->graph_exec);
+  for (auto& g : net->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& t : net->outs) if (t.data) cudaFree(t.data);
   delete net;
   return HQ_OK;
