@@ -31,7 +31,10 @@ inline long long tensor_bytes(int n, int h, int w, int c, int bits) {
   return (long long)n * h * w * c * bits / 8;
 }
 
-hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream) {
+// `scratch` / `scratch_bytes`: buffer for the lowered first-layer path owned by the caller (a
+// network); NULL means use (and if needed grow) the handle's own buffer.
+hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream,
+                      void* scratch = nullptr, size_t scratch_bytes = 0) {
   if (!h || !d) return HQ_ERR_INVALID_ARG;
   hq_status st = check_tensor(in, true, true, false);
   if (st != HQ_OK) return st;
@@ -71,10 +74,28 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   const bool tc_ok = hq_conv_tc_supported(a);
   if (h->conv_path == 2 && !tc_ok) return HQ_ERR_UNSUPPORTED;
   if (h->conv_path != 1 && tc_ok) return hq_launch_conv_tc(h, a, s);
+  if (h->conv_path != 1 && hq_conv_lowering_applies(a)) {
+    // thin first layers: patch matrix in the handle's scratch buffer, then the tensor-core kernel
+    const size_t need = hq_conv_lowering_bytes(a);
+    if (scratch && scratch_bytes >= need) return hq_launch_conv_lowered(h, a, scratch, s);
+    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_lowered(h, a, h->workspace, s);
+  }
   return hq_launch_conv_cuda_core(a, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 }  // namespace
+
+hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s) {
+  if (bytes <= h->workspace_bytes) return HQ_OK;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return HQ_ERR_WORKSPACE;
+  // the old buffer may still be read by queued work
+  if (cudaDeviceSynchronize() != cudaSuccess) return HQ_ERR_CUDA;
+  if (h->workspace) { cudaFree(h->workspace); h->workspace = nullptr; h->workspace_bytes = 0; }
+  if (cudaMalloc(&h->workspace, bytes) != cudaSuccess) { cudaGetLastError(); return HQ_ERR_WORKSPACE; }
+  h->workspace_bytes = bytes;
+  return HQ_OK;
+}
 
 // ------------------------------------------------------------------------------------------------
 struct hq_network {
@@ -84,6 +105,8 @@ struct hq_network {
   std::vector<long long> bytes;
   int32_t batch, image_h, image_w, image_c, image_signed;
   int32_t launches;
+  void* scratch;                     // patch matrix of the lowered first layer (owned)
+  size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
   // that double-buffered callers do not re-capture every step
   struct CachedGraph { cudaGraphExec_t exec; const void* images; void* logits; };
@@ -233,6 +256,7 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   if (!net) return HQ_ERR_WORKSPACE;
   net->h = h; net->batch = batch;
   net->image_h = image_h; net->image_w = image_w; net->image_c = image_c; net->image_signed = image_signed;
+  net->scratch = nullptr; net->scratch_bytes = 0;
   net->layers.assign(table, table + n_layers);
   net->outs.resize(n_layers);
   net->bytes.resize(n_layers);
@@ -256,6 +280,16 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
           st = HQ_ERR_INVALID_ARG; break;
         }
         o.h = (in.h + 2 * d.pad - d.kh) / d.stride + 1; o.w = (in.w + 2 * d.pad - d.kw) / d.stride + 1; o.c = d.cout;
+        {
+          ConvArgs a{};
+          a.n = batch; a.h = in.h; a.w = in.w; a.cin = in.c; a.in_bits = in.bits; a.cout = d.cout; a.kh = d.kh; a.kw = d.kw;
+          a.stride = d.stride; a.pad = d.pad; a.ho = o.h; a.wo = o.w; a.out_bits = o.bits;
+          if (!hq_conv_tc_supported(a) && hq_conv_lowering_applies(a)) {
+            const size_t need = hq_conv_lowering_bytes(a);
+            if (need > net->scratch_bytes) net->scratch_bytes = need;
+            net->launches += 2;                 // weight padding + patch matrix kernels
+          }
+        }
         break;
       }
       case HQ_OP_LINEAR:
@@ -280,6 +314,12 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     o.data = buf;
     net->outs[i] = o;
   }
+  if (st == HQ_OK && net->scratch_bytes) {
+    const size_t want = net->scratch_bytes;
+    net->scratch_bytes = 0;
+    if (cudaMalloc(&net->scratch, want) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; }
+    else net->scratch_bytes = want;
+  }
   if (st != HQ_OK) { hq_network_destroy(net); return st; }
   *out = net;
   return HQ_OK;
@@ -303,7 +343,7 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         d.residual = nullptr;
         if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
         if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
-        else st = hq_conv2d(h, &in, &d, &o, s);
+        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes);
         break;
       }
       case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
@@ -405,6 +445,7 @@ hq_status hq_network_destroy(hq_network* net) {
   if (!net) return HQ_ERR_INVALID_ARG;
   for (auto& g : net->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& t : net->outs) if (t.data) cudaFree(t.data);
+  if (net->scratch) cudaFree(net->scratch);
   delete net;
   return HQ_OK;
 }

@@ -26,8 +26,9 @@ namespace {
 
 constexpr int kTileM = 128;
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;
-constexpr int kEpilogueThreads = 128;
+constexpr int kEpilogueWarps = 8;
+constexpr int kEpilogueThreads = kEpilogueWarps * 32;
+constexpr int kThreads = 64 + kEpilogueThreads;               // producer warp + MMA warp + epilogue warps
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;   // 2 s per wait
 
 struct TcParams {
@@ -40,6 +41,12 @@ struct TcParams {
   int32_t m_tiles, n_tiles, stages;
   int32_t a_signed;
   uint32_t tmem_cols;
+  // epilogue
+  int32_t staged_out;    // 1: outputs leave through a swizzled shared-memory tile and TMA stores
+  int32_t staged_res;    // 1: the 8-bit residual tile arrives through TMA loads
+  int32_t out_ib, out_boxes;   // bytes per row of one store box, boxes per tile
+  int32_t res_ib, res_boxes;
+  uint32_t out_stage_off, res_stage_off;   // offsets from the 1024-aligned dynamic base
   const int32_t* bias; const int32_t* b; const int32_t* c;
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   int32_t relu, qmin, qmax;
@@ -47,18 +54,24 @@ struct TcParams {
   uint32_t* status;
 };
 
+struct __align__(16) MainConst { int32_t b; int32_t sh; long long r0; };      // r0 = bias*b + 2^(c-1); sh = c or c-32
+struct __align__(16) ResConst { int32_t rb; int32_t pre; int32_t sh; int32_t pad_; };
+
 struct SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
   unsigned long long tfull[2];
   unsigned long long tempty[2];
+  unsigned long long rfull[2];
+  unsigned long long rempty[2];
   unsigned long long drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
-  volatile uint32_t epi_ok;   // the epilogue's wait result, taken by one thread for all four warps
-  long long r0[256];      // bias*b + 2^(c-1) per channel of the current N tile
-  long long rr0[256];     // 2^(rc-1)
-  int32_t sb[256], sc[256], srb[256], src[256], sbias[256];
+  volatile uint32_t epi_ok;   // the epilogue's wait result, taken by one thread for all its warps
+  MainConst mc[256];
+  ResConst rcst[256];
+  long long rr0[256];         // 2^(rc+pre-1)
+  int32_t sbias[256];
 };
 
 // ---------------------------------------------------------------- PTX wrappers ---------------
@@ -167,8 +180,47 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t bkb) {
 }
 
 // ---------------------------------------------------------------- the kernel -----------------
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory"); }
+__device__ __forceinline__ uint32_t epi_bar_and(uint32_t v) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(v), "n"(kEpilogueThreads) : "memory");
+  return r;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, unsigned x, unsigned y, unsigned z, unsigned w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+// Byte address inside a TMA box of `ib`-byte rows stored with the matching 32/64/128-byte swizzle
+// (16-byte chunk index XOR address bits 7..9, masked to the span); box base is 1024-aligned.
+__device__ __forceinline__ uint32_t swz(uint32_t base, uint32_t row, uint32_t off, uint32_t ib) {
+  const uint32_t a = base + row * ib + off;
+  return a ^ (((a >> 7) & ((ib >> 4) - 1u)) << 4);
+}
+__device__ __forceinline__ unsigned pack4_bytes(int a, int b, int c, int d) {
+  return __byte_perm(__byte_perm((unsigned)a, (unsigned)b, 0x0040), __byte_perm((unsigned)c, (unsigned)d, 0x0040), 0x5410);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
+               const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ SharedCtl ctl;
 
@@ -177,12 +229,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t a_bytes = kTileM * p.bkb;
   const uint32_t b_bytes = p.bn * p.bkb;
   const uint32_t stage_bytes = a_bytes + b_bytes;
+  const uint32_t out_stage = tiles + p.out_stage_off;
+  const uint32_t res_stage = tiles + p.res_stage_off;
+  const uint32_t res_tile_bytes = kTileM * p.bn;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&ctl.full[s]), 1); mbar_init(smem_u32(&ctl.empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), kEpilogueThreads); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), kEpilogueThreads);
+      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), kEpilogueThreads);
+    }
     mbar_init(smem_u32(&ctl.drain), 1);
     ctl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -196,11 +254,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
         const int m0 = m_tile * kTileM;
+        if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
+          const uint32_t rb = tcount & 1u, rph = (tcount >> 1) & 1u;
+          if (!mbar_wait(smem_u32(&ctl.rempty[rb]), rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&ctl.rfull[rb]);
+          mbar_expect_tx(bar, res_tile_bytes);
+          for (int bx = 0; bx < p.res_boxes; ++bx)
+            tma_load_2d(res_stage + rb * res_tile_bytes + bx * (kTileM * p.res_ib), &map_res, bar,
+                        n_tile * p.bn + bx * p.res_ib, m0);
+        }
         const int img = m0 / p.howo, rem = m0 - img * p.howo;
         const int oh = rem / p.wo, ow = rem - oh * p.wo;
         const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad;
@@ -216,7 +283,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tma_load_2d(a_dst + a_bytes, &map_b, bar, tap * p.cin_bytes + chunk * p.bkb, n_tile * p.bn);
         }
       }
-      // Drain: every stage this thread filled must have landed before the CTA may exit.
+      // Drain: every copy this thread started must have landed before the CTA may exit.
       const uint32_t issued = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
       for (uint32_t j = 0; j < issued; ++j) {
         const uint32_t k = it - 1 - j;
@@ -224,6 +291,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const unsigned long long t0 = global_ns();
         while (!mbar_try_wait(smem_u32(&ctl.full[s]), ph)) {
           if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
+        }
+      }
+      if (p.staged_res) {
+        const uint32_t tiles_done = tcount < 2u ? tcount : 2u;
+        for (uint32_t j = 0; j < tiles_done; ++j) {
+          const uint32_t k = tcount - 1 - j;
+          const unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(smem_u32(&ctl.rfull[k & 1u]), (k >> 1) & 1u)) {
+            if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
+          }
         }
       }
     }
@@ -262,49 +339,168 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read
-    const int et = threadIdx.x - 64;              // 0..127
+    const int half = (warp - 2) >> 2;             // which half of the tile's columns this warp owns
+    const int et = threadIdx.x - 64;              // 0..255
     const int row = q * 32 + lane;
+    const int cols_per_warp = p.bn >> 1;
+    const int lo = p.relu ? (p.qmin > 0 ? p.qmin : 0) : p.qmin, hi = p.qmax;
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
       const int n0 = n_tile * p.bn;
       const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
-      // per-channel constants of this N tile
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+      // The previous tile's stores must have read the staging tile before it is overwritten.
+      if (p.staged_out && et == 0) tma_store_wait_read();
+      epi_bar();
+      // per-channel constants of this N tile; `fast` = every live channel allows 32-bit results
+      uint32_t fast = 1;
       for (int j = et; j < p.bn; j += kEpilogueThreads) {
         const int ch = n0 + j;
         const bool live = ch < p.N;
         const int bias = (live && p.bias) ? p.bias[ch] : 0;
         ctl.sbias[j] = bias;
         if (p.out_bits != 32) {
-          const int bb = live ? p.b[ch] : 0, cc = live ? p.c[ch] : 1;
-          ctl.sb[j] = bb; ctl.sc[j] = cc;
-          ctl.r0[j] = (long long)bias * (long long)bb + (1LL << (cc - 1));
+          const int bb = live ? p.b[ch] : 0, cc = live ? p.c[ch] : 32;
+          if (cc < 32) fast = 0;
+          ctl.mc[j].b = bb;
+          ctl.mc[j].r0 = (long long)bias * (long long)bb + (1LL << (cc - 1));
           if (p.res) {
-            const int rcc = live ? p.rc[ch] : 1;
-            ctl.srb[j] = live ? p.rb[ch] : 0; ctl.src[j] = rcc;
+            const int rcc = live ? p.rc[ch] : 32;
+            const int pre = rcc < 32 ? 32 - rcc : 0;
+            if (rcc < 9 || p.res_bits != 8) fast = 0;
+            ctl.rcst[j].rb = live ? p.rb[ch] : 0;
+            ctl.rcst[j].pre = pre;
+            ctl.rcst[j].sh = rcc;              // patched below once the tile's mode is known
             ctl.rr0[j] = 1LL << (rcc - 1);
+          }
+          ctl.mc[j].sh = cc;
+        }
+      }
+      fast = epi_bar_and(fast);
+      if (p.out_bits != 32 && fast) {           // fast tiles shift the high word: store c - 32 and pre-shifted forms
+        for (int j = et; j < p.bn; j += kEpilogueThreads) {
+          ctl.mc[j].sh -= 32;
+          if (p.res) {
+            const int pre = ctl.rcst[j].pre, rcc = ctl.rcst[j].sh;
+            ctl.rcst[j].sh = rcc + pre - 32;
+            ctl.rr0[j] = 1LL << (rcc + pre - 1);
           }
         }
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
-
-      // One thread takes the bounded wait and shares the verdict, so that all four warps leave
-      // (or stay in) the loop together and nobody is left behind at the named barrier.
-      if (et == 0)
-        ctl.epi_ok = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+      // One thread takes the bounded waits and shares the verdict, so that all warps leave (or
+      // stay in) the loop together and nobody is left behind at the named barrier.
+      if (et == 0) {
+        bool w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE);
+        if (w && p.staged_res) w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE);
+        ctl.epi_ok = w ? 1u : 0u;
+      }
+      epi_bar();
       if (!ctl.epi_ok) { ok = false; break; }
       for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.tfull[as]), aph); ++tries) {}
+      if (p.staged_res)
+        for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.rfull[as]), aph); ++tries) {}
       tc_fence_after();
       const long long m = (long long)m_tile * kTileM + row;
       const bool row_live = m < p.M;
-      for (int c0 = 0; c0 < p.bn; c0 += 32) {
+      const uint32_t res_tile = res_stage + as * res_tile_bytes;
+
+      for (int cc0 = 0; cc0 < cols_per_warp; cc0 += 32) {
+        const int c0 = half * cols_per_warp + cc0;          // first column (within the tile) of this chunk
         int v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * p.bn + c0, v);
+
+        if (p.staged_out) {
+          // ---------------- staged path: math in registers, packed bytes to the swizzled tile
+          int y[32];
+          if (fast) {
+            if (p.res) {
+              unsigned rw[8];
+              if (p.staged_res) {
+                const uint32_t bx = (uint32_t)c0 / (uint32_t)p.res_ib, off = (uint32_t)c0 % (uint32_t)p.res_ib;
+                const uint32_t bbase = res_tile + bx * (kTileM * p.res_ib);
+                const uint4 t0 = ld_shared_v4(swz(bbase, row, off, p.res_ib));
+                const uint4 t1 = ld_shared_v4(swz(bbase, row, off + 16, p.res_ib));
+                rw[0] = t0.x; rw[1] = t0.y; rw[2] = t0.z; rw[3] = t0.w; rw[4] = t1.x; rw[5] = t1.y; rw[6] = t1.z; rw[7] = t1.w;
+              } else {
+                const long long o = m * p.N + n0 + c0;
+                if (row_live && n0 + c0 + 32 <= p.N && ((o & 15) == 0)) {
+                  const uint4 t0 = __ldg((const uint4*)((const unsigned char*)p.res + o));
+                  const uint4 t1 = __ldg((const uint4*)((const unsigned char*)p.res + o) + 1);
+                  rw[0] = t0.x; rw[1] = t0.y; rw[2] = t0.z; rw[3] = t0.w; rw[4] = t1.x; rw[5] = t1.y; rw[6] = t1.z; rw[7] = t1.w;
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) rw[j] = 0;
+                  if (row_live)
+                    for (int j = 0; j < 32 && n0 + c0 + j < p.N; ++j)
+                      rw[j >> 2] |= (unsigned)((const unsigned char*)p.res)[o + j] << (8 * (j & 3));
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const MainConst k1 = ctl.mc[c0 + j];
+                const ResConst k2 = ctl.rcst[c0 + j];
+                const unsigned byte = (rw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+                const int r = p.res_signed ? (int)(signed char)byte : (int)byte;
+                const long long t1 = (long long)v[j] * (long long)k1.b + k1.r0;
+                const long long t2 = (long long)(r << k2.pre) * (long long)k2.rb + ctl.rr0[c0 + j];
+                const int s = ((int)(t1 >> 32) >> k1.sh) + ((int)(t2 >> 32) >> k2.sh);
+                y[j] = min(max(s, lo), hi);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const MainConst k1 = ctl.mc[c0 + j];
+                const long long t1 = (long long)v[j] * (long long)k1.b + k1.r0;
+                y[j] = min(max((int)(t1 >> 32) >> k1.sh, lo), hi);
+              }
+            }
+          } else {
+            // general tile: full 64-bit results (any 1 <= c <= 62, INT32 residual operands)
+            const long long o = m * p.N + n0 + c0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const MainConst k1 = ctl.mc[c0 + j];
+              long long s = ((long long)v[j] * (long long)k1.b + k1.r0) >> k1.sh;
+              if (p.res) {
+                int r = 0;
+                if (p.staged_res) {
+                  const uint32_t bx = (uint32_t)(c0 + j) / (uint32_t)p.res_ib, off = (uint32_t)(c0 + j) % (uint32_t)p.res_ib;
+                  const uint32_t a = swz(res_tile + bx * (kTileM * p.res_ib), row, off & ~15u, p.res_ib) + (off & 15u);
+                  unsigned byte;
+                  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(byte) : "r"(a));
+                  r = p.res_signed ? (int)(signed char)byte : (int)byte;
+                } else if (row_live && n0 + c0 + j < p.N) {
+                  r = hq_load_elem(p.res, o + j, p.res_bits, p.res_signed);
+                }
+                const ResConst k2 = ctl.rcst[c0 + j];
+                s += ((long long)r * (long long)k2.rb + ctl.rr0[c0 + j]) >> k2.sh;
+              }
+              y[j] = hq_clamp_ll(s, p.relu, p.qmin, p.qmax);
+            }
+          }
+          if (p.out_bits == 8) {
+            const uint32_t off = (uint32_t)c0 % (uint32_t)p.out_ib, bx = (uint32_t)c0 / (uint32_t)p.out_ib;
+            const uint32_t bbase = out_stage + bx * (kTileM * p.out_ib);
+            st_shared_v4(swz(bbase, row, off, p.out_ib), pack4_bytes(y[0], y[1], y[2], y[3]), pack4_bytes(y[4], y[5], y[6], y[7]),
+                         pack4_bytes(y[8], y[9], y[10], y[11]), pack4_bytes(y[12], y[13], y[14], y[15]));
+            st_shared_v4(swz(bbase, row, off + 16, p.out_ib), pack4_bytes(y[16], y[17], y[18], y[19]),
+                         pack4_bytes(y[20], y[21], y[22], y[23]), pack4_bytes(y[24], y[25], y[26], y[27]),
+                         pack4_bytes(y[28], y[29], y[30], y[31]));
+          } else {   // 4-bit: 32 columns = 16 bytes
+            unsigned w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int j = 0; j < 32; ++j) w[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
+            const uint32_t byte0 = (uint32_t)c0 >> 1;
+            const uint32_t off = byte0 % (uint32_t)p.out_ib, bx = byte0 / (uint32_t)p.out_ib;
+            st_shared_v4(swz(out_stage + bx * (kTileM * p.out_ib), row, off, p.out_ib), w[0], w[1], w[2], w[3]);
+          }
+          continue;
+        }
+
+        // ---------------- direct path: INT32 outputs, odd channel counts
         if (!row_live || n0 + c0 >= p.N) continue;
         const int ncols = (p.N - (n0 + c0)) < 32 ? (p.N - (n0 + c0)) : 32;
         const long long o = m * p.N + n0 + c0;         // element index of the first column
@@ -316,75 +512,51 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               *(int4*)(dst + j) = make_int4(v[j] + ctl.sbias[c0 + j], v[j + 1] + ctl.sbias[c0 + j + 1],
                                             v[j + 2] + ctl.sbias[c0 + j + 2], v[j + 3] + ctl.sbias[c0 + j + 3]);
           } else {
-            for (int j = 0; j < ncols; ++j) dst[j] = v[j] + ctl.sbias[c0 + j];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (j < ncols) dst[j] = v[j] + ctl.sbias[c0 + j];
           }
           continue;
         }
         int y[32];
-        if (p.res) {
-          int r[32];
-          if (p.res_bits == 8) {
-            const unsigned char* rp = (const unsigned char*)p.res + o;
-            if (ncols == 32 && ((o & 15) == 0)) {
-              const uint4 t0 = __ldg((const uint4*)rp), t1 = __ldg((const uint4*)rp + 1);
-              const unsigned w[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+        const int sh_add = fast ? 32 : 0;               // undo the fast-tile form of the shifts
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const unsigned byte = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-                r[j] = p.res_signed ? (int)(signed char)byte : (int)byte;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                r[j] = (j < ncols) ? (p.res_signed ? (int)(signed char)rp[j] : (int)rp[j]) : 0;
-            }
-          } else {
-            const int* rp = (const int*)p.res + o;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] = (j < ncols) ? __ldg(rp + j) : 0;
+        for (int j = 0; j < 32; ++j) {
+          const MainConst k1 = ctl.mc[c0 + j];
+          long long s = ((long long)v[j] * (long long)k1.b + k1.r0) >> (k1.sh + sh_add);
+          if (p.res) {
+            const ResConst k2 = ctl.rcst[c0 + j];
+            const int r = (j < ncols) ? hq_load_elem(p.res, o + j, p.res_bits, p.res_signed) : 0;
+            s += ((long long)(fast ? (r << k2.pre) : r) * (long long)k2.rb + ctl.rr0[c0 + j]) >> (k2.sh + sh_add);
           }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const long long ym = ((long long)v[j] * (long long)ctl.sb[c0 + j] + ctl.r0[c0 + j]) >> ctl.sc[c0 + j];
-            const long long yr = ((long long)r[j] * (long long)ctl.srb[c0 + j] + ctl.rr0[c0 + j]) >> ctl.src[c0 + j];
-            y[j] = hq_clamp_ll(ym + yr, p.relu, p.qmin, p.qmax);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const long long ym = ((long long)v[j] * (long long)ctl.sb[c0 + j] + ctl.r0[c0 + j]) >> ctl.sc[c0 + j];
-            y[j] = hq_clamp_ll(ym, p.relu, p.qmin, p.qmax);
-          }
+          y[j] = hq_clamp_ll(s, p.relu, p.qmin, p.qmax);
         }
         if (p.out_bits == 8) {
           unsigned char* dst = (unsigned char*)p.out + o;
-          if (ncols == 32 && ((o & 15) == 0)) {
-            unsigned w[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              w[j] = (unsigned)(y[4 * j] & 0xFF) | ((unsigned)(y[4 * j + 1] & 0xFF) << 8) |
-                     ((unsigned)(y[4 * j + 2] & 0xFF) << 16) | ((unsigned)(y[4 * j + 3] & 0xFF) << 24);
-            *(uint4*)dst = make_uint4(w[0], w[1], w[2], w[3]);
-            *((uint4*)dst + 1) = make_uint4(w[4], w[5], w[6], w[7]);
-          } else {
-            for (int j = 0; j < ncols; ++j) dst[j] = (unsigned char)(y[j] & 0xFF);
-          }
+          for (int j = 0; j < 32; ++j) if (j < ncols) dst[j] = (unsigned char)(y[j] & 0xFF);
         } else {   // 4-bit output, two per byte; N is even so a pair never straddles the tile edge
           unsigned char* dst = (unsigned char*)p.out + (o >> 1);
-          if (ncols == 32 && ((o & 31) == 0)) {
-            unsigned w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) w[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
-            *(uint4*)dst = make_uint4(w[0], w[1], w[2], w[3]);
-          } else {
-            for (int j = 0; j < ncols; j += 2)
-              dst[j >> 1] = (unsigned char)((y[j] & 0xF) | ((y[j + 1] & 0xF) << 4));
-          }
+          for (int j = 0; j < 32; j += 2)
+            if (j < ncols) dst[j >> 1] = (unsigned char)((y[j] & 0xF) | ((y[j + 1] & 0xF) << 4));
         }
       }
+      // accumulator (and residual tile) are no longer needed: hand them back
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl.tempty[as]));
+      if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
+      if (p.staged_out) {
+        fence_async_smem();                    // make this thread's tile writes visible to the TMA engine
+        epi_bar();
+        if (et == 0) {
+          const int ob = p.out_bits;
+          for (int bx = 0; bx < p.out_boxes; ++bx)
+            tma_store_2d(&map_out, out_stage + bx * (kTileM * p.out_ib), (n0 * ob >> 3) + bx * p.out_ib, m_tile * kTileM);
+          tma_store_commit();
+        }
+      }
     }
+    if (p.staged_out && et == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -426,7 +598,7 @@ bool load_driver_entry_points() {
   return true;
 }
 
-int pick_bn(int n_out, int m_tiles, int sm_count) {
+int pick_bn(int n_out, int m_tiles, int sm_count, bool staged_res) {
   // candidate N tiles; prefer the one that wastes the fewest SM-waves, ties to the larger tile
   const int cands[3] = {256, 128, 64};
   int best = 64;
@@ -434,6 +606,7 @@ int pick_bn(int n_out, int m_tiles, int sm_count) {
   for (int i = 0; i < 3; ++i) {
     const int bn = cands[i];
     if (bn > 64 && bn / 2 >= n_out) continue;            // mostly empty tile
+    if (bn == 256 && staged_res) continue;               // two residual tiles of 256 columns do not fit
     const int n_tiles = (n_out + bn - 1) / bn;
     const long long tiles = (long long)m_tiles * n_tiles;
     const long long waves = (tiles + sm_count - 1) / sm_count;
@@ -449,7 +622,7 @@ int pick_bn(int n_out, int m_tiles, int sm_count) {
 // tensor-map encoders and the kernel's dynamic shared-memory limit.
 bool hq_conv_tc_init() {
   if (!load_driver_entry_points()) return false;
-  return cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 215 * 1024) == cudaSuccess;
+  return cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess;
 }
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
@@ -462,6 +635,26 @@ bool hq_conv_tc_supported(const ConvArgs& a) {
   if (a.res && !(a.res_bits == 8 || a.res_bits == 32)) return false;
   return true;
 }
+
+namespace {
+
+CUtensorMapSwizzle swizzle_for(int row_bytes) {
+  return row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                                        : CU_TENSOR_MAP_SWIZZLE_32B;
+}
+
+// 2-D byte map over a dense [rows][row_bytes] tensor with a box of `ib` bytes x 128 rows.
+bool encode_rows_map(CUtensorMap* map, const void* base, long long rows, long long row_bytes, int ib) {
+  const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)ib, (cuuint32_t)kTileM};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(ib), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
 
 hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream) {
   if (!hq_conv_tc_supported(a)) return HQ_ERR_UNSUPPORTED;
@@ -477,25 +670,42 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.cchunks = a.cin / p.bkb;
   p.k_blocks = a.kh * a.kw * p.cchunks;
   p.m_tiles = (int32_t)((M + kTileM - 1) / kTileM);
-  p.bn = pick_bn(a.cout, p.m_tiles, h->sm_count);
+  // outputs and 8-bit residuals whose rows are 16-byte multiples travel through TMA
+  const long long out_row_bytes = (long long)a.cout * a.out_bits / 8;
+  p.staged_out = (a.out_bits != 32 && out_row_bytes % 16 == 0) ? 1 : 0;
+  p.staged_res = (p.staged_out && a.res && a.res_bits == 8 && a.cout % 16 == 0) ? 1 : 0;
+  p.bn = pick_bn(a.cout, p.m_tiles, h->sm_count, p.staged_res != 0);
   p.n_tiles = (a.cout + p.bn - 1) / p.bn;
   p.a_signed = a.in_signed;
   p.tmem_cols = (uint32_t)(2 * p.bn);
   const int stage_bytes = (kTileM + p.bn) * p.bkb;
-  const int smem_budget = 200 * 1024;
-  int stages = smem_budget / stage_bytes;
+  int out_tile_bytes = 0, res_tile_bytes = 0;
+  if (p.staged_out) {
+    const int tile_row_bytes = p.bn * a.out_bits / 8;
+    p.out_ib = tile_row_bytes < 128 ? tile_row_bytes : 128;
+    p.out_boxes = tile_row_bytes / p.out_ib;
+    out_tile_bytes = kTileM * tile_row_bytes;
+  }
+  if (p.staged_res) {
+    p.res_ib = p.bn < 128 ? p.bn : 128;
+    p.res_boxes = p.bn / p.res_ib;
+    res_tile_bytes = kTileM * p.bn;
+  }
+  const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
+  int stages = (smem_budget - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return HQ_ERR_UNSUPPORTED;
   p.stages = stages;
+  p.out_stage_off = (uint32_t)(stages * stage_bytes);             // all pieces are multiples of 1024 bytes
+  p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.relu = a.relu; p.qmin = a.qmin; p.qmax = a.qmax;
   p.out = a.out; p.out_bits = a.out_bits;
   p.status = h->dev_status;
 
-  const CUtensorMapSwizzle swz = (p.bkb == 128) ? CU_TENSOR_MAP_SWIZZLE_128B
-                               : (p.bkb == 64) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-  alignas(64) CUtensorMap map_a, map_b;
+  const CUtensorMapSwizzle swz = swizzle_for(p.bkb);
+  alignas(64) CUtensorMap map_a, map_b, map_out, map_res;
   {
     // activations: (C, W, H, N) with byte strides; base pixels range over
     // [-pad, W + pad - (kw-1)) so that the hardware's pixel walk equals the output raster
@@ -525,12 +735,15 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return HQ_ERR_CUDA;
   }
+  map_out = map_b; map_res = map_b;                    // valid placeholders when a path is not staged
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, M, out_row_bytes, p.out_ib)) return HQ_ERR_CUDA;
+  if (p.staged_res && !encode_rows_map(&map_res, a.res, M, a.cout, p.res_ib)) return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + 2 * res_tile_bytes + 1024;
   const long long total_tiles = (long long)p.m_tiles * p.n_tiles;
   const int grid = (int)(total_tiles < h->sm_count ? total_tiles : h->sm_count);
   // keep one CTA per SM (tensor-memory allocation assumes it): never request less than 120 KiB
   const size_t smem = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
-  conv_tc_kernel<<<grid, kThreads, smem, stream>>>(map_a, map_b, p);
+  conv_tc_kernel<<<grid, kThreads, smem, stream>>>(map_a, map_b, map_out, map_res, p);
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }

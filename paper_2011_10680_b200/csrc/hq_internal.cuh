@@ -70,6 +70,12 @@ bool hq_conv_tc_init();
 bool hq_conv_tc_supported(const ConvArgs& a);
 // Tensor-core path; returns HQ_OK, HQ_ERR_UNSUPPORTED or HQ_ERR_CUDA.
 hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
+// Lowered path for thin first layers: patch matrix + padded weights in scratch, then the tensor-core kernel.
+bool hq_conv_lowering_applies(const ConvArgs& a);
+size_t hq_conv_lowering_bytes(const ConvArgs& a);
+hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
+// Grow the handle's scratch buffer (not allowed while `s` is capturing).
+hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s);
 cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s);
 cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int in_bits, int in_signed,
                               const int32_t* b, const int32_t* c, int qmin, int qmax,

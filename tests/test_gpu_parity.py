@@ -85,6 +85,11 @@ TC_CASES = [
     (1, 9, 9, 96, 40, 5, 1, 2, 8, False, 8, True),           # 5x5, cin = 3 x 32
     (2, 12, 12, 64, 64, 3, 1, 1, 4, False, 8, True),         # uint4 output
     (1, 7, 7, 512, 1000, 1, 1, 0, 32, False, 8, False),      # classifier-like N = 1000
+    (2, 9, 9, 64, 40, 3, 1, 1, 8, True, 8, True),            # N = 40: rows not 16-byte multiples, direct stores
+    (2, 13, 13, 64, 96, 1, 1, 0, 8, True, 8, True),          # residual tile clipped in N by the TMA box
+    (1, 20, 20, 128, 256, 3, 1, 1, 8, True, 8, True),        # residual + 3x3 + two N tiles of 128
+    (3, 8, 8, 64, 64, 1, 1, 0, 4, True, 8, True),            # uint4 output with residual
+    (2, 16, 16, 32, 128, 1, 1, 0, 4, False, 8, True),        # uint4 output, 64-byte store boxes
 ]
 
 
@@ -108,6 +113,30 @@ def test_conv_tensor_core_signed_input_and_small_c(hq):
     # shifts below 32 and very large shifts both take the general 64-bit path
     case = inputs.conv_case(204, 1, 12, 12, 64, 64, 1, 1, 0, relu=True, c_range=(20, 62))
     run_conv_and_compare(hq, case, path=2)
+
+
+def test_conv_tensor_core_general_tiles_with_residual(hq):
+    # residual shifts below 9 and main shifts below 32 force the 64-bit tile path, staged and direct
+    for cout in (64, 40):
+        case = inputs.conv_case(205, 2, 10, 10, 64, cout, 1, 1, 0, residual=True, c_range=(30, 44))
+        case["rc"][::3] = 5
+        run_conv_and_compare(hq, case, path=2)
+
+
+LOWERED_CASES = [
+    # n, h, w, cin, cout, k, stride, pad
+    (2, 32, 32, 3, 64, 7, 2, 3),
+    (1, 17, 19, 3, 32, 7, 2, 3),
+    (2, 9, 9, 5, 16, 3, 1, 1),
+    (1, 12, 12, 16, 48, 3, 2, 1),
+]
+
+
+@pytest.mark.parametrize("cfg", LOWERED_CASES)
+def test_conv_lowered_first_layer_path(hq, cfg):
+    n, h, w, cin, cout, k, stride, pad = cfg
+    case = inputs.conv_case(206, n, h, w, cin, cout, k, stride, pad, c_range=(38, 42))
+    run_conv_and_compare(hq, case, path=0)     # automatic choice: patch matrix + tensor-core kernel
 
 
 def test_linear_matches_oracle_and_conv(hq):
