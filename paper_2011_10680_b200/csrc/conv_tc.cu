@@ -233,13 +233,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t res_stage = tiles + p.res_stage_off;
   const uint32_t res_tile_bytes = kTileM * p.bn;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  // Tile schedule: the grid is a multiple of n_tiles, so a CTA keeps one N tile for its whole life
+  // (its per-channel constants and weight rows never change) and strides over the M tiles.
+  const int n_tile_cta = blockIdx.x % p.n_tiles;
+  const int m_tile0 = blockIdx.x / p.n_tiles;
+  const int m_step = gridDim.x / p.n_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&ctl.full[s]), 1); mbar_init(smem_u32(&ctl.empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), kEpilogueThreads);
-      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), kEpilogueThreads);
+      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), kEpilogueWarps);
+      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), kEpilogueWarps);
     }
     mbar_init(smem_u32(&ctl.drain), 1);
     ctl.abort_flag = 0;
@@ -256,8 +260,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
+      for (int m_tile = m_tile0; m_tile < p.m_tiles && ok; m_tile += m_step, ++tcount) {
+        const int n_tile = n_tile_cta;
         const int m0 = m_tile * kTileM;
         if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
           const uint32_t rb = tcount & 1u, rph = (tcount >> 1) & 1u;
@@ -312,7 +316,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                              ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int m_tile = m_tile0; m_tile < p.m_tiles && ok; m_tile += m_step, ++tcount) {
         const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctl.tempty[as]), aph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         tc_fence_after();
@@ -340,65 +344,65 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..9)
+    // Each warp owns 32 accumulator rows (its TMEM lane quarter) and one half of the tile's
+    // columns, and runs on its own: private staging box, private TMA store, no CTA-wide barrier
+    // per tile.  The CTA's N tile never changes, so the per-channel constants are staged once.
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;             // which half of the tile's columns this warp owns
+    const int ew = warp - 2;                      // 0..7
+    const int half = ew >> 2;                     // which half of the tile's columns this warp owns
     const int et = threadIdx.x - 64;              // 0..255
     const int row = q * 32 + lane;
     const int cols_per_warp = p.bn >> 1;
     const int lo = p.relu ? (p.qmin > 0 ? p.qmin : 0) : p.qmin, hi = p.qmax;
-    uint32_t tcount = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
-      const int n0 = n_tile * p.bn;
-      const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
-      // The previous tile's stores must have read the staging tile before it is overwritten.
-      if (p.staged_out && et == 0) tma_store_wait_read();
-      epi_bar();
-      // per-channel constants of this N tile; `fast` = every live channel allows 32-bit results
-      uint32_t fast = 1;
+    const int n0 = n_tile_cta * p.bn;
+    uint32_t fast = 1;
+    for (int j = et; j < p.bn; j += kEpilogueThreads) {
+      const int ch = n0 + j;
+      const bool live = ch < p.N;
+      const int bias = (live && p.bias) ? p.bias[ch] : 0;
+      ctl.sbias[j] = bias;
+      if (p.out_bits != 32) {
+        const int bb = live ? p.b[ch] : 0, cc = live ? p.c[ch] : 32;
+        if (cc < 32) fast = 0;
+        ctl.mc[j].b = bb;
+        ctl.mc[j].sh = cc;
+        ctl.mc[j].r0 = (long long)bias * (long long)bb + (1LL << (cc - 1));
+        if (p.res) {
+          const int rcc = live ? p.rc[ch] : 32;
+          if (rcc < 9 || p.res_bits != 8) fast = 0;
+          ctl.rcst[j].rb = live ? p.rb[ch] : 0;
+          ctl.rcst[j].pre = rcc < 32 ? 32 - rcc : 0;
+          ctl.rcst[j].sh = rcc;
+          ctl.rr0[j] = 1LL << (rcc - 1);
+        }
+      }
+    }
+    fast = epi_bar_and(fast);                    // every live channel allows 32-bit intermediate results
+    if (p.out_bits != 32 && fast) {              // fast CTAs shift the high word: store c - 32 and pre-shifted forms
       for (int j = et; j < p.bn; j += kEpilogueThreads) {
-        const int ch = n0 + j;
-        const bool live = ch < p.N;
-        const int bias = (live && p.bias) ? p.bias[ch] : 0;
-        ctl.sbias[j] = bias;
-        if (p.out_bits != 32) {
-          const int bb = live ? p.b[ch] : 0, cc = live ? p.c[ch] : 32;
-          if (cc < 32) fast = 0;
-          ctl.mc[j].b = bb;
-          ctl.mc[j].r0 = (long long)bias * (long long)bb + (1LL << (cc - 1));
-          if (p.res) {
-            const int rcc = live ? p.rc[ch] : 32;
-            const int pre = rcc < 32 ? 32 - rcc : 0;
-            if (rcc < 9 || p.res_bits != 8) fast = 0;
-            ctl.rcst[j].rb = live ? p.rb[ch] : 0;
-            ctl.rcst[j].pre = pre;
-            ctl.rcst[j].sh = rcc;              // patched below once the tile's mode is known
-            ctl.rr0[j] = 1LL << (rcc - 1);
-          }
-          ctl.mc[j].sh = cc;
+        ctl.mc[j].sh -= 32;
+        if (p.res) {
+          const int pre = ctl.rcst[j].pre, rcc = ctl.rcst[j].sh;
+          ctl.rcst[j].sh = rcc + pre - 32;
+          ctl.rr0[j] = 1LL << (rcc + pre - 1);
         }
       }
-      fast = epi_bar_and(fast);
-      if (p.out_bits != 32 && fast) {           // fast tiles shift the high word: store c - 32 and pre-shifted forms
-        for (int j = et; j < p.bn; j += kEpilogueThreads) {
-          ctl.mc[j].sh -= 32;
-          if (p.res) {
-            const int pre = ctl.rcst[j].pre, rcc = ctl.rcst[j].sh;
-            ctl.rcst[j].sh = rcc + pre - 32;
-            ctl.rr0[j] = 1LL << (rcc + pre - 1);
-          }
-        }
+    }
+    epi_bar();
+
+    const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(32 * p.out_ib);
+    uint32_t tcount = 0;
+    for (int m_tile = m_tile0; m_tile < p.m_tiles; m_tile += m_step, ++tcount) {
+      const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
+      uint32_t w = 1;
+      if (lane == 0) {
+        if (p.staged_out) tma_store_wait_read();    // the previous store has read this warp's staging box
+        w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+        if (w && p.staged_res)
+          w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
       }
-      // One thread takes the bounded waits and shares the verdict, so that all warps leave (or
-      // stay in) the loop together and nobody is left behind at the named barrier.
-      if (et == 0) {
-        bool w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE);
-        if (w && p.staged_res) w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE);
-        ctl.epi_ok = w ? 1u : 0u;
-      }
-      epi_bar();
-      if (!ctl.epi_ok) { ok = false; break; }
+      w = __shfl_sync(0xffffffffu, w, 0);
+      if (!w) break;
       for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.tfull[as]), aph); ++tries) {}
       if (p.staged_res)
         for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.rfull[as]), aph); ++tries) {}
@@ -413,7 +417,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * p.bn + c0, v);
 
         if (p.staged_out) {
-          // ---------------- staged path: math in registers, packed bytes to the swizzled tile
+          // ---------------- staged path: math in registers, packed bytes to the swizzled box
           int y[32];
           if (fast) {
             if (p.res) {
@@ -458,7 +462,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               }
             }
           } else {
-            // general tile: full 64-bit results (any 1 <= c <= 62, INT32 residual operands)
+            // general CTA: full 64-bit results (any 1 <= c <= 62, INT32 residual operands)
             const long long o = m * p.N + n0 + c0;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -482,20 +486,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
           if (p.out_bits == 8) {
-            const uint32_t off = (uint32_t)c0 % (uint32_t)p.out_ib, bx = (uint32_t)c0 / (uint32_t)p.out_ib;
-            const uint32_t bbase = out_stage + bx * (kTileM * p.out_ib);
-            st_shared_v4(swz(bbase, row, off, p.out_ib), pack4_bytes(y[0], y[1], y[2], y[3]), pack4_bytes(y[4], y[5], y[6], y[7]),
+            const uint32_t off = (uint32_t)cc0;                 // one box per warp: its column half
+            st_shared_v4(swz(my_stage, lane, off, p.out_ib), pack4_bytes(y[0], y[1], y[2], y[3]), pack4_bytes(y[4], y[5], y[6], y[7]),
                          pack4_bytes(y[8], y[9], y[10], y[11]), pack4_bytes(y[12], y[13], y[14], y[15]));
-            st_shared_v4(swz(bbase, row, off + 16, p.out_ib), pack4_bytes(y[16], y[17], y[18], y[19]),
+            st_shared_v4(swz(my_stage, lane, off + 16, p.out_ib), pack4_bytes(y[16], y[17], y[18], y[19]),
                          pack4_bytes(y[20], y[21], y[22], y[23]), pack4_bytes(y[24], y[25], y[26], y[27]),
                          pack4_bytes(y[28], y[29], y[30], y[31]));
           } else {   // 4-bit: 32 columns = 16 bytes
-            unsigned w[4] = {0u, 0u, 0u, 0u};
+            unsigned wd[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) w[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
-            const uint32_t byte0 = (uint32_t)c0 >> 1;
-            const uint32_t off = byte0 % (uint32_t)p.out_ib, bx = byte0 / (uint32_t)p.out_ib;
-            st_shared_v4(swz(out_stage + bx * (kTileM * p.out_ib), row, off, p.out_ib), w[0], w[1], w[2], w[3]);
+            for (int j = 0; j < 32; ++j) wd[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
+            st_shared_v4(swz(my_stage, lane, (uint32_t)cc0 >> 1, p.out_ib), wd[0], wd[1], wd[2], wd[3]);
           }
           continue;
         }
@@ -518,7 +519,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           continue;
         }
         int y[32];
-        const int sh_add = fast ? 32 : 0;               // undo the fast-tile form of the shifts
+        const int sh_add = fast ? 32 : 0;               // undo the fast form of the shifts
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const MainConst k1 = ctl.mc[c0 + j];
@@ -541,22 +542,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (j < ncols) dst[j >> 1] = (unsigned char)((y[j] & 0xF) | ((y[j + 1] & 0xF) << 4));
         }
       }
-      // accumulator (and residual tile) are no longer needed: hand them back
+      // accumulator rows (and the residual tile) are no longer needed by this warp: hand them back
       tc_fence_before();
-      mbar_arrive(smem_u32(&ctl.tempty[as]));
-      if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
-      if (p.staged_out) {
-        fence_async_smem();                    // make this thread's tile writes visible to the TMA engine
-        epi_bar();
-        if (et == 0) {
-          const int ob = p.out_bits;
-          for (int bx = 0; bx < p.out_boxes; ++bx)
-            tma_store_2d(&map_out, out_stage + bx * (kTileM * p.out_ib), (n0 * ob >> 3) + bx * p.out_ib, m_tile * kTileM);
+      if (p.staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(smem_u32(&ctl.tempty[as]));
+        if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
+        if (p.staged_out) {
+          tma_store_2d(&map_out, my_stage, ((n0 + half * cols_per_warp) * p.out_bits >> 3), m_tile * kTileM + q * 32);
           tma_store_commit();
         }
       }
     }
-    if (p.staged_out && et == 0) tma_store_wait_all();
+    if (p.staged_out && lane == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -640,14 +639,14 @@ namespace {
 
 CUtensorMapSwizzle swizzle_for(int row_bytes) {
   return row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                                                        : CU_TENSOR_MAP_SWIZZLE_32B;
+       : row_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
 }
 
-// 2-D byte map over a dense [rows][row_bytes] tensor with a box of `ib` bytes x 128 rows.
-bool encode_rows_map(CUtensorMap* map, const void* base, long long rows, long long row_bytes, int ib) {
+// 2-D byte map over a dense [rows][row_bytes] tensor with a box of `ib` bytes x `box_rows` rows.
+bool encode_rows_map(CUtensorMap* map, const void* base, long long rows, long long row_bytes, int ib, int box_rows) {
   const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)ib, (cuuint32_t)kTileM};
+  const cuuint32_t box[2] = {(cuuint32_t)ib, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(ib), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -681,10 +680,11 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const int stage_bytes = (kTileM + p.bn) * p.bkb;
   int out_tile_bytes = 0, res_tile_bytes = 0;
   if (p.staged_out) {
-    const int tile_row_bytes = p.bn * a.out_bits / 8;
-    p.out_ib = tile_row_bytes < 128 ? tile_row_bytes : 128;
-    p.out_boxes = tile_row_bytes / p.out_ib;
-    out_tile_bytes = kTileM * tile_row_bytes;
+    // one store box per epilogue warp: 32 rows x (half the tile's columns), at most 128 bytes wide
+    p.out_ib = (p.bn / 2) * a.out_bits / 8;
+    p.out_boxes = 1;
+    out_tile_bytes = kTileM * p.bn * a.out_bits / 8;
+    if (out_tile_bytes < 8 * 1024) out_tile_bytes = 8 * 1024;     // keep the next region 1024-aligned
   }
   if (p.staged_res) {
     p.res_ib = p.bn < 128 ? p.bn : 128;
@@ -736,12 +736,14 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     if (r != CUDA_SUCCESS) return HQ_ERR_CUDA;
   }
   map_out = map_b; map_res = map_b;                    // valid placeholders when a path is not staged
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, M, out_row_bytes, p.out_ib)) return HQ_ERR_CUDA;
-  if (p.staged_res && !encode_rows_map(&map_res, a.res, M, a.cout, p.res_ib)) return HQ_ERR_CUDA;
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, M, out_row_bytes, p.out_ib, 32)) return HQ_ERR_CUDA;
+  if (p.staged_res && !encode_rows_map(&map_res, a.res, M, a.cout, p.res_ib, kTileM)) return HQ_ERR_CUDA;
 
   const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + 2 * res_tile_bytes + 1024;
+  if (p.n_tiles > h->sm_count) return HQ_ERR_UNSUPPORTED;
   const long long total_tiles = (long long)p.m_tiles * p.n_tiles;
-  const int grid = (int)(total_tiles < h->sm_count ? total_tiles : h->sm_count);
+  // a multiple of n_tiles, so that every CTA keeps one N tile
+  const int grid = (int)(total_tiles <= h->sm_count ? total_tiles : (h->sm_count / p.n_tiles) * p.n_tiles);
   // keep one CTA per SM (tensor-memory allocation assumes it): never request less than 120 KiB
   const size_t smem = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
   conv_tc_kernel<<<grid, kThreads, smem, stream>>>(map_a, map_b, map_out, map_res, p);

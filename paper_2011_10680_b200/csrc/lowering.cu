@@ -7,34 +7,47 @@
 
 namespace {
 
+// One block builds the patch rows of `wseg` consecutive output pixels of one output row.  The kh
+// input rows those pixels touch are first copied into shared memory (zero outside the image), so
+// that every output byte is one shared-memory read: for a fixed filter row the (kw, cin) taps of a
+// pixel are contiguous in NHWC, hence patch byte k = r*(kw*cin) + t sits at window byte
+// (ow_local*stride*cin + t) of window row r.
 __global__ void __launch_bounds__(256) patch_matrix_kernel(const unsigned char* __restrict__ in, int n, int h, int w,
                                                            int cin, int kh, int kw, int stride, int pad, int ho, int wo,
-                                                           int K, int Kp, uint4* __restrict__ out) {
-  const int cpr = Kp >> 4;                                   // 16-byte chunks per output row
-  const long long total = (long long)n * ho * wo * cpr;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-       i += (long long)gridDim.x * blockDim.x) {
-    const int j = (int)(i % cpr);
-    long long m = i / cpr;
-    const int ow = (int)(m % wo); m /= wo;
-    const int oh = (int)(m % ho);
-    const int img = (int)(m / ho);
+                                                           int K, int Kp, int wseg, int segs, int win_bytes,
+                                                           uint4* __restrict__ out) {
+  extern __shared__ unsigned char win[];                     // [kh][win_bytes]
+  const int seg = blockIdx.x % segs;
+  const int oh = (blockIdx.x / segs) % ho;
+  const int img = blockIdx.x / (segs * ho);
+  const int ow0 = seg * wseg;
+  const int npix = (wo - ow0) < wseg ? (wo - ow0) : wseg;
+  const int col0 = (ow0 * stride - pad) * cin;                // byte offset of the window inside an input row
+  const int row_bytes = w * cin;
+  for (int i = threadIdx.x; i < kh * win_bytes; i += blockDim.x) {
+    const int r = i / win_bytes, b = i - r * win_bytes;
+    const int ih = oh * stride + r - pad, col = col0 + b;
+    unsigned char v = 0;
+    if (ih >= 0 && ih < h && col >= 0 && col < row_bytes) v = __ldg(in + ((long long)img * h + ih) * row_bytes + col);
+    win[i] = v;
+  }
+  __syncthreads();
+  const int cpr = Kp >> 4, kwc = kw * cin;
+  uint4* dst = out + (((long long)img * ho + oh) * wo + ow0) * cpr;
+  for (int i = threadIdx.x; i < npix * cpr; i += blockDim.x) {
+    const int px = i / cpr, j = i - px * cpr;
     int k = j << 4;
-    int tap = k / cin, ci = k - tap * cin;
-    int r = tap / kw, s = tap - r * kw;
+    int r = k / kwc, t = k - r * kwc;
+    const unsigned char* src = win + px * stride * cin;
     unsigned word[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-    for (int t = 0; t < 16; ++t, ++k) {
+    for (int e = 0; e < 16; ++e, ++k) {
       if (k < K) {
-        const int ih = oh * stride + r - pad, iw = ow * stride + s - pad;
-        if (ih >= 0 && ih < h && iw >= 0 && iw < w) {
-          const unsigned v = __ldg(in + (((long long)img * h + ih) * w + iw) * cin + ci);
-          word[t >> 2] |= v << (8 * (t & 3));
-        }
-        if (++ci == cin) { ci = 0; if (++s == kw) { s = 0; ++r; } }
+        word[e >> 2] |= (unsigned)src[r * win_bytes + t] << (8 * (e & 3));
+        if (++t == kwc) { t = 0; ++r; }
       }
     }
-    out[i] = make_uint4(word[0], word[1], word[2], word[3]);
+    dst[i] = make_uint4(word[0], word[1], word[2], word[3]);
   }
 }
 
@@ -55,6 +68,8 @@ bool hq_conv_lowering_applies(const ConvArgs& a) {
   if (a.in_bits != 8) return false;
   const long long K = (long long)a.kh * a.kw * a.cin;
   if (K > 4096) return false;                                // meant for thin first layers
+  const int wseg = a.wo < 64 ? a.wo : 64;
+  if ((long long)a.kh * ((wseg - 1) * a.stride + a.kw) * a.cin > 48 * 1024) return false;   // window must fit shared memory
   ConvArgs t = a;
   t.cin = (int)((K + 31) / 32 * 32); t.kh = t.kw = 1; t.stride = 1; t.pad = 0; t.h = a.ho; t.w = a.wo;
   return hq_conv_tc_supported(t);
@@ -80,12 +95,16 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
   }
   {
-    const long long total = m * (Kp >> 4);
-    long long blocks = (total + 255) / 256;
-    const long long cap = (long long)h->sm_count * 32;
-    patch_matrix_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>(
-        (const unsigned char*)a.in, a.n, a.h, a.w, a.cin, a.kh, a.kw, a.stride, a.pad, a.ho, a.wo, K, Kp,
-        (uint4*)patches);
+    int wseg = a.wo < 64 ? a.wo : 64;
+    const int win_bytes = ((wseg - 1) * a.stride + a.kw) * a.cin;
+    const int segs = (a.wo + wseg - 1) / wseg;
+    const size_t smem = (size_t)a.kh * win_bytes;
+    if (smem > 48 * 1024) return HQ_ERR_UNSUPPORTED;
+    const long long blocks = (long long)a.n * a.ho * segs;
+    if (blocks >= (1ll << 31)) return HQ_ERR_UNSUPPORTED;
+    patch_matrix_kernel<<<(int)blocks, 256, smem, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, a.cin, a.kh, a.kw,
+                                                       a.stride, a.pad, a.ho, a.wo, K, Kp, wseg, segs, win_bytes,
+                                                       (uint4*)patches);
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
   }
   ConvArgs t = a;
