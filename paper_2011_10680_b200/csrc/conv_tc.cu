@@ -19,6 +19,7 @@
 // handle's status word, raises a CTA-wide abort flag and every role leaves its loop, drains what
 // it has in flight (again bounded), and the CTA frees its tensor memory and returns.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "hq_internal.cuh"
 
@@ -40,22 +41,34 @@ struct TcParams {
   int32_t bn;            // N tile: 64, 128 or 256
   int32_t m_tiles, n_tiles, stages;
   int32_t a_signed;
+  int32_t a_tiled;       // 1: A is a dense [M][cin] matrix (1x1, stride 1, no padding) fetched by a tiled map
   uint32_t tmem_cols;
   // epilogue
   int32_t staged_out;    // 1: outputs leave through a swizzled shared-memory tile and TMA stores
   int32_t staged_res;    // 1: the 8-bit residual tile arrives through TMA loads
+  int32_t sat_pack;      // 1: clamp bounds equal the 8-bit output type's range (saturating pack does the clamp)
+  int32_t out_signed;
+  int32_t store_direct;  // 1 (with staged_out): packed results go straight to global memory, 32 bytes per lane
   int32_t out_ib, out_boxes;   // bytes per row of one store box, boxes per tile
-  int32_t res_ib, res_boxes;
+  int32_t res_ib, res_boxes, res_ib_log2;
   uint32_t out_stage_off, res_stage_off;   // offsets from the 1024-aligned dynamic base
   const int32_t* bias; const int32_t* b; const int32_t* c;
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   int32_t relu, qmin, qmax;
   void* out; int32_t out_bits;
   uint32_t* status;
+  long long* trace;
 };
 
+// Optional timeline instrumentation (compiled only with -DHQ_TC_TRACE; not part of the product build).
+#ifdef HQ_TC_TRACE
+#define HQ_TRACE(role, idx) do { if (p.trace && blockIdx.x == 0 && (idx) < 2048) p.trace[(role) * 2048 + (idx)] = clock64(); } while (0)
+#else
+#define HQ_TRACE(role, idx) do { } while (0)
+#endif
+
 struct __align__(16) MainConst { int32_t b; int32_t sh; long long r0; };      // r0 = bias*b + 2^(c-1); sh = c or c-32
-struct __align__(16) ResConst { int32_t rb; int32_t pre; int32_t sh; int32_t pad_; };
+struct __align__(16) ResConst { int32_t rb; int32_t h; int32_t sh; int32_t pad_; };   // fast: h = 2^(rc-9), sh = rc-8
 
 struct SharedCtl {
   unsigned long long full[kMaxStages];
@@ -133,6 +146,17 @@ __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap*
       ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
 }
 
+// True in exactly one lane of a converged warp; tells the compiler the guarded region is
+// single-lane, which lets it keep TMA / MMA operands in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -185,7 +209,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
                ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory"); }
@@ -215,6 +239,56 @@ __device__ __forceinline__ uint32_t swz(uint32_t base, uint32_t row, uint32_t of
 }
 __device__ __forceinline__ unsigned pack4_bytes(int a, int b, int c, int d) {
   return __byte_perm(__byte_perm((unsigned)a, (unsigned)b, 0x0040), __byte_perm((unsigned)c, (unsigned)d, 0x0040), 0x5410);
+}
+
+// cvt.pack.sat: two INT32 values saturated to 8 bits into the low half-word, `upper` into the high one.
+template <bool SIGNED>
+__device__ __forceinline__ unsigned pack2_sat(int hi_byte, int lo_byte, unsigned upper) {
+  unsigned d;
+  if (SIGNED) asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi_byte), "r"(lo_byte), "r"(upper));
+  else        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi_byte), "r"(lo_byte), "r"(upper));
+  return d;
+}
+
+// Requantization of 32 accumulator columns of one row on the 32-bit fast path (Eq. 4; Section 3.3):
+//   main      y  = hi32(acc*b + bias*b + 2^(c-1)) >> (c-32)                         (needs c >= 32)
+//   residual  y += (hi32((r << 24) * rb) + 2^(rc-9)) >> (rc-8)                      (needs 9 <= rc)
+// The residual form is exact: (r<<24)*rb >> 32 = floor(r*rb / 2^8), the rounding constant 2^(rc-1) is
+// a multiple of 2^8, and the dropped low 8 bits of r*rb cannot carry across a multiple of 2^(rc-8).
+// SAT: the clamp bounds are the 8-bit type's own range, so the saturating pack does ReLU and clamp.
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED>
+__device__ __forceinline__ void requant32_fast(const int (&v)[32], const unsigned (&rw)[8], const SharedCtl& ctl,
+                                               int c0, int lo, int hi, int (&y)[32]) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+#if defined(HQ_EXP) && HQ_EXP == 1
+    const MainConst k1 = ctl.mc[c0];
+#else
+    const MainConst k1 = ctl.mc[c0 + j];
+#endif
+#if defined(HQ_EXP) && HQ_EXP == 2
+    int s = v[j] + k1.b;
+#else
+    const long long t1 = (long long)v[j] * (long long)k1.b + k1.r0;
+    int s = (int)(t1 >> 32) >> k1.sh;
+#endif
+    if (RES) {
+      const ResConst k2 = ctl.rcst[c0 + j];
+      const unsigned top = __byte_perm(rw[j >> 2], 0u, 0x0444u | ((unsigned)(j & 3) << 12));   // byte -> bits 31:24
+      if (RSIGNED) s += (__mulhi((int)top, k2.rb) + k2.h) >> k2.sh;
+      else s += (int)((__umulhi(top, (unsigned)k2.rb) + (unsigned)k2.h) >> k2.sh);
+    }
+    y[j] = SAT ? s : min(max(s, lo), hi);
+  }
+}
+
+template <bool SAT, bool OSIGNED>
+__device__ __forceinline__ void pack32_bytes(const int (&y)[32], unsigned (&wd)[8]) {
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    if (SAT) wd[g] = pack2_sat<OSIGNED>(y[4 * g + 1], y[4 * g], pack2_sat<OSIGNED>(y[4 * g + 3], y[4 * g + 2], 0u));
+    else wd[g] = pack4_bytes(y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -257,11 +331,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0, tcount = 0;
+    if (elect_one()) {
+      // No division or modulo in this loop: one thread runs it and every dependent instruction
+      // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
+      uint32_t it = 0, tcount = 0, s = 0, ph = 0;
       bool ok = true;
+      const int n_tile = n_tile_cta;
+      // (image, row, column) of the tile's first output pixel, advanced by a fixed step per tile
+      const int ho = p.howo / p.wo;
+      int img = (m_tile0 * kTileM) / p.howo;
+      int oh = ((m_tile0 * kTileM) - img * p.howo) / p.wo;
+      int ow = (m_tile0 * kTileM) - img * p.howo - oh * p.wo;
+      const int step = m_step * kTileM;
+      const int d_img = step / p.howo, d_oh = (step - d_img * p.howo) / p.wo, d_ow = step - d_img * p.howo - d_oh * p.wo;
       for (int m_tile = m_tile0; m_tile < p.m_tiles && ok; m_tile += m_step, ++tcount) {
-        const int n_tile = n_tile_cta;
         const int m0 = m_tile * kTileM;
         if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
           const uint32_t rb = tcount & 1u, rph = (tcount >> 1) & 1u;
@@ -272,19 +355,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tma_load_2d(res_stage + rb * res_tile_bytes + bx * (kTileM * p.res_ib), &map_res, bar,
                         n_tile * p.bn + bx * p.res_ib, m0);
         }
-        const int img = m0 / p.howo, rem = m0 - img * p.howo;
-        const int oh = rem / p.wo, ow = rem - oh * p.wo;
-        const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad;
+        const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad, img_now = img;
+        ow += d_ow; if (ow >= p.wo) { ow -= p.wo; ++oh; }
+        oh += d_oh; if (oh >= ho) { oh -= ho; ++img; }
+        img += d_img;
+        int chunk = 0, tap_s = 0, tap_r = 0;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+          HQ_TRACE(8, it);
           if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-          const int tap = kb / p.cchunks, chunk = kb - tap * p.cchunks;
-          const int r = tap / p.kw, sx = tap - r * p.kw;
+          HQ_TRACE(0, it);
           const uint32_t bar = smem_u32(&ctl.full[s]);
           const uint32_t a_dst = tiles + s * stage_bytes;
           mbar_expect_tx(bar, stage_bytes);
-          tma_load_im2col(a_dst, &map_a, bar, chunk * p.bkb, cw, chh, img, (uint16_t)sx, (uint16_t)r);
-          tma_load_2d(a_dst + a_bytes, &map_b, bar, tap * p.cin_bytes + chunk * p.bkb, n_tile * p.bn);
+          HQ_TRACE(5, it);
+          if (p.a_tiled) tma_load_2d(a_dst, &map_a, bar, chunk * p.bkb, m0);
+          else tma_load_im2col(a_dst, &map_a, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
+          HQ_TRACE(6, it);
+          tma_load_2d(a_dst + a_bytes, &map_b, bar, kb * p.bkb, n_tile * p.bn);
+          HQ_TRACE(7, it);
+          if (++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
       }
       // Drain: every copy this thread started must have landed before the CTA may exit.
@@ -310,30 +400,33 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (elect_one()) {
       // instruction descriptor: D = S32, A = u8/s8, B = s8, both K-major, N = bn, M = 128
       const uint32_t idesc = (2u << 4) | ((uint32_t)(p.a_signed ? 1 : 0) << 7) | (1u << 10) |
                              ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-      uint32_t it = 0, tcount = 0;
+      uint32_t it = 0, tcount = 0, s = 0, ph = 0;
       bool ok = true;
+      const uint64_t desc_hi = smem_desc(0, p.bkb);           // everything but the start address
+      const int ksteps = p.bkb >> 5;
       for (int m_tile = m_tile0; m_tile < p.m_tiles && ok; m_tile += m_step, ++tcount) {
         const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctl.tempty[as]), aph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * p.bn;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
           if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
           tc_fence_after();
+          HQ_TRACE(1, it);
           const uint32_t a_addr = tiles + s * stage_bytes;
-          const uint32_t b_addr = a_addr + a_bytes;
-          const int ksteps = p.bkb >> 5;
-          for (int k = 0; k < ksteps; ++k)
-            mma_i8(d_tmem, smem_desc(a_addr + 32u * k, p.bkb), smem_desc(b_addr + 32u * k, p.bkb), idesc,
-                   (kb | k) ? 1u : 0u);
+          uint64_t adesc = desc_hi | (uint64_t)((a_addr >> 4) & 0x3FFF);
+          uint64_t bdesc = desc_hi | (uint64_t)(((a_addr + a_bytes) >> 4) & 0x3FFF);
+          for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
+            mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
           mma_commit(smem_u32(&ctl.empty[s]));     // frees the stage when these MMAs have read it
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
         if (ok) mma_commit(smem_u32(&ctl.tfull[as]));
+        HQ_TRACE(2, tcount);
       }
       // Drain: all issued MMAs must have completed before tensor memory is freed.
       mma_commit(smem_u32(&ctl.drain));
@@ -355,7 +448,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int cols_per_warp = p.bn >> 1;
     const int lo = p.relu ? (p.qmin > 0 ? p.qmin : 0) : p.qmin, hi = p.qmax;
     const int n0 = n_tile_cta * p.bn;
-    uint32_t fast = 1;
+    uint32_t fast = p.staged_out ? 1u : 0u;      // the direct-store path always uses the 64-bit form
     for (int j = et; j < p.bn; j += kEpilogueThreads) {
       const int ch = n0 + j;
       const bool live = ch < p.N;
@@ -371,59 +464,61 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int rcc = live ? p.rc[ch] : 32;
           if (rcc < 9 || p.res_bits != 8) fast = 0;
           ctl.rcst[j].rb = live ? p.rb[ch] : 0;
-          ctl.rcst[j].pre = rcc < 32 ? 32 - rcc : 0;
           ctl.rcst[j].sh = rcc;
           ctl.rr0[j] = 1LL << (rcc - 1);
         }
       }
     }
     fast = epi_bar_and(fast);                    // every live channel allows 32-bit intermediate results
-    if (p.out_bits != 32 && fast) {              // fast CTAs shift the high word: store c - 32 and pre-shifted forms
+    if (p.out_bits != 32 && fast) {              // fast CTAs: shifts of the high word, residual in its 8-bit form
       for (int j = et; j < p.bn; j += kEpilogueThreads) {
         ctl.mc[j].sh -= 32;
         if (p.res) {
-          const int pre = ctl.rcst[j].pre, rcc = ctl.rcst[j].sh;
-          ctl.rcst[j].sh = rcc + pre - 32;
-          ctl.rr0[j] = 1LL << (rcc + pre - 1);
+          const int rcc = ctl.rcst[j].sh;
+          if (rcc >= 40) { ctl.rcst[j].rb = 0; ctl.rcst[j].h = 0; ctl.rcst[j].sh = 1; }   // |r*rb| < 2^39: rounds to 0
+          else { ctl.rcst[j].h = 1 << (rcc - 9); ctl.rcst[j].sh = rcc - 8; }
         }
       }
     }
     epi_bar();
 
-    const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(32 * p.out_ib);
+    // two private staging boxes per warp, used alternately, so a store may still be reading one
+    // while the next tile's results are written to the other
+    const uint32_t my_stage0 = out_stage + (uint32_t)ew * (uint32_t)(64 * p.out_ib);
+    const bool use_tma_store = p.staged_out && !p.store_direct;
     uint32_t tcount = 0;
     for (int m_tile = m_tile0; m_tile < p.m_tiles; m_tile += m_step, ++tcount) {
       const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
       uint32_t w = 1;
       if (lane == 0) {
-        if (p.staged_out) tma_store_wait_read();    // the previous store has read this warp's staging box
+        if (use_tma_store) tma_store_wait_read1();  // the store before the previous one has read its staging box
         w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
         if (w && p.staged_res)
           w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
       }
       w = __shfl_sync(0xffffffffu, w, 0);
       if (!w) break;
-      for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.tfull[as]), aph); ++tries) {}
-      if (p.staged_res)
-        for (int tries = 0; tries < 1024 && !mbar_try_wait(smem_u32(&ctl.rfull[as]), aph); ++tries) {}
-      tc_fence_after();
+      if (ew == 0 && lane == 0) HQ_TRACE(3, tcount);
+      tc_fence_after();                            // lane 0 observed the barriers; the shuffle ordered the warp
       const long long m = (long long)m_tile * kTileM + row;
       const bool row_live = m < p.M;
       const uint32_t res_tile = res_stage + as * res_tile_bytes;
+      const uint32_t my_stage = my_stage0 + as * (uint32_t)(32 * p.out_ib);
 
       for (int cc0 = 0; cc0 < cols_per_warp; cc0 += 32) {
         const int c0 = half * cols_per_warp + cc0;          // first column (within the tile) of this chunk
         int v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * p.bn + c0, v);
+        if (ew == 0 && lane == 0 && cc0 == 0) HQ_TRACE(9, tcount);
 
         if (p.staged_out) {
           // ---------------- staged path: math in registers, packed bytes to the swizzled box
           int y[32];
           if (fast) {
+            unsigned rw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
             if (p.res) {
-              unsigned rw[8];
               if (p.staged_res) {
-                const uint32_t bx = (uint32_t)c0 / (uint32_t)p.res_ib, off = (uint32_t)c0 % (uint32_t)p.res_ib;
+                const uint32_t bx = (uint32_t)c0 >> p.res_ib_log2, off = (uint32_t)c0 & (uint32_t)(p.res_ib - 1);
                 const uint32_t bbase = res_tile + bx * (kTileM * p.res_ib);
                 const uint4 t0 = ld_shared_v4(swz(bbase, row, off, p.res_ib));
                 const uint4 t1 = ld_shared_v4(swz(bbase, row, off + 16, p.res_ib));
@@ -434,32 +529,22 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   const uint4 t0 = __ldg((const uint4*)((const unsigned char*)p.res + o));
                   const uint4 t1 = __ldg((const uint4*)((const unsigned char*)p.res + o) + 1);
                   rw[0] = t0.x; rw[1] = t0.y; rw[2] = t0.z; rw[3] = t0.w; rw[4] = t1.x; rw[5] = t1.y; rw[6] = t1.z; rw[7] = t1.w;
-                } else {
-#pragma unroll
-                  for (int j = 0; j < 8; ++j) rw[j] = 0;
-                  if (row_live)
-                    for (int j = 0; j < 32 && n0 + c0 + j < p.N; ++j)
-                      rw[j >> 2] |= (unsigned)((const unsigned char*)p.res)[o + j] << (8 * (j & 3));
+                } else if (row_live) {
+                  for (int j = 0; j < 32 && n0 + c0 + j < p.N; ++j)
+                    rw[j >> 2] |= (unsigned)((const unsigned char*)p.res)[o + j] << (8 * (j & 3));
                 }
               }
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const MainConst k1 = ctl.mc[c0 + j];
-                const ResConst k2 = ctl.rcst[c0 + j];
-                const unsigned byte = (rw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-                const int r = p.res_signed ? (int)(signed char)byte : (int)byte;
-                const long long t1 = (long long)v[j] * (long long)k1.b + k1.r0;
-                const long long t2 = (long long)(r << k2.pre) * (long long)k2.rb + ctl.rr0[c0 + j];
-                const int s = ((int)(t1 >> 32) >> k1.sh) + ((int)(t2 >> 32) >> k2.sh);
-                y[j] = min(max(s, lo), hi);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const MainConst k1 = ctl.mc[c0 + j];
-                const long long t1 = (long long)v[j] * (long long)k1.b + k1.r0;
-                y[j] = min(max((int)(t1 >> 32) >> k1.sh, lo), hi);
-              }
+            }
+            // uniform dispatch to the specialised instruction sequences
+            const int variant = (p.res ? 4 : 0) | (p.res_signed ? 2 : 0) | (p.sat_pack ? 1 : 0);
+            switch (variant) {
+              case 0: requant32_fast<false, false, false, false>(v, rw, ctl, c0, lo, hi, y); break;
+              case 1: case 3: requant32_fast<false, false, true, false>(v, rw, ctl, c0, lo, hi, y); break;
+              case 2: requant32_fast<false, false, false, false>(v, rw, ctl, c0, lo, hi, y); break;
+              case 4: requant32_fast<true, false, false, false>(v, rw, ctl, c0, lo, hi, y); break;
+              case 5: requant32_fast<true, false, true, false>(v, rw, ctl, c0, lo, hi, y); break;
+              case 6: requant32_fast<true, true, false, false>(v, rw, ctl, c0, lo, hi, y); break;
+              default: requant32_fast<true, true, true, false>(v, rw, ctl, c0, lo, hi, y); break;
             }
           } else {
             // general CTA: full 64-bit results (any 1 <= c <= 62, INT32 residual operands)
@@ -471,7 +556,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (p.res) {
                 int r = 0;
                 if (p.staged_res) {
-                  const uint32_t bx = (uint32_t)(c0 + j) / (uint32_t)p.res_ib, off = (uint32_t)(c0 + j) % (uint32_t)p.res_ib;
+                  const uint32_t bx = (uint32_t)(c0 + j) >> p.res_ib_log2, off = (uint32_t)(c0 + j) & (uint32_t)(p.res_ib - 1);
                   const uint32_t a = swz(res_tile + bx * (kTileM * p.res_ib), row, off & ~15u, p.res_ib) + (off & 15u);
                   unsigned byte;
                   asm volatile("ld.shared.u8 %0, [%1];" : "=r"(byte) : "r"(a));
@@ -485,19 +570,51 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               y[j] = hq_clamp_ll(s, p.relu, p.qmin, p.qmax);
             }
           }
+          if (ew == 0 && lane == 0 && cc0 == 0) HQ_TRACE(10, tcount + (y[0] & 0));
+          unsigned wd[8];
           if (p.out_bits == 8) {
-            const uint32_t off = (uint32_t)cc0;                 // one box per warp: its column half
-            st_shared_v4(swz(my_stage, lane, off, p.out_ib), pack4_bytes(y[0], y[1], y[2], y[3]), pack4_bytes(y[4], y[5], y[6], y[7]),
-                         pack4_bytes(y[8], y[9], y[10], y[11]), pack4_bytes(y[12], y[13], y[14], y[15]));
-            st_shared_v4(swz(my_stage, lane, off + 16, p.out_ib), pack4_bytes(y[16], y[17], y[18], y[19]),
-                         pack4_bytes(y[20], y[21], y[22], y[23]), pack4_bytes(y[24], y[25], y[26], y[27]),
-                         pack4_bytes(y[28], y[29], y[30], y[31]));
-          } else {   // 4-bit: 32 columns = 16 bytes
-            unsigned wd[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int j = 0; j < 32; ++j) wd[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
-            st_shared_v4(swz(my_stage, lane, (uint32_t)cc0 >> 1, p.out_ib), wd[0], wd[1], wd[2], wd[3]);
+            if (fast && p.sat_pack) { if (p.out_signed) pack32_bytes<true, true>(y, wd); else pack32_bytes<true, false>(y, wd); }
+            else pack32_bytes<false, false>(y, wd);
           }
+          if (p.store_direct) {
+            // packed results straight to global memory: 32 contiguous bytes (16 at 4 bit) per lane
+            const long long o = m * p.N + n0 + c0;
+            if (row_live && n0 + c0 < p.N) {
+              const bool whole = n0 + c0 + 32 <= p.N;
+              if (p.out_bits == 8) {
+                unsigned char* dst = (unsigned char*)p.out + o;
+                if (whole) {
+                  *(uint4*)dst = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                  *((uint4*)dst + 1) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) if (n0 + c0 + j < p.N) dst[j] = (unsigned char)((wd[j >> 2] >> (8 * (j & 3))) & 0xFF);
+                }
+              } else {
+                unsigned char* dst = (unsigned char*)p.out + (o >> 1);
+                if (whole) {
+                  unsigned nb[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) nb[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
+                  *(uint4*)dst = make_uint4(nb[0], nb[1], nb[2], nb[3]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; j += 2)
+                    if (n0 + c0 + j < p.N) dst[j >> 1] = (unsigned char)((y[j] & 0xF) | ((y[j + 1] & 0xF) << 4));
+                }
+              }
+            }
+          } else if (p.out_bits == 8) {
+            const uint32_t off = (uint32_t)cc0;                 // one box per warp: its column half
+            st_shared_v4(swz(my_stage, lane, off, p.out_ib), wd[0], wd[1], wd[2], wd[3]);
+            st_shared_v4(swz(my_stage, lane, off + 16, p.out_ib), wd[4], wd[5], wd[6], wd[7]);
+          } else {   // 4-bit: 32 columns = 16 bytes
+            unsigned nb[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int j = 0; j < 32; ++j) nb[j >> 3] |= (unsigned)(y[j] & 0xF) << (4 * (j & 7));
+            st_shared_v4(swz(my_stage, lane, (uint32_t)cc0 >> 1, p.out_ib), nb[0], nb[1], nb[2], nb[3]);
+          }
+          if (ew == 0 && lane == 0 && cc0 == 0) HQ_TRACE(11, tcount);
           continue;
         }
 
@@ -519,15 +636,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           continue;
         }
         int y[32];
-        const int sh_add = fast ? 32 : 0;               // undo the fast form of the shifts
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const MainConst k1 = ctl.mc[c0 + j];
-          long long s = ((long long)v[j] * (long long)k1.b + k1.r0) >> (k1.sh + sh_add);
+          long long s = ((long long)v[j] * (long long)k1.b + k1.r0) >> k1.sh;
           if (p.res) {
             const ResConst k2 = ctl.rcst[c0 + j];
             const int r = (j < ncols) ? hq_load_elem(p.res, o + j, p.res_bits, p.res_signed) : 0;
-            s += ((long long)(fast ? (r << k2.pre) : r) * (long long)k2.rb + ctl.rr0[c0 + j]) >> (k2.sh + sh_add);
+            s += ((long long)r * (long long)k2.rb + ctl.rr0[c0 + j]) >> k2.sh;
           }
           y[j] = hq_clamp_ll(s, p.relu, p.qmin, p.qmax);
         }
@@ -544,18 +660,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       // accumulator rows (and the residual tile) are no longer needed by this warp: hand them back
       tc_fence_before();
-      if (p.staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
+      if (use_tma_store) fence_async_smem();       // make this lane's box writes visible to the TMA engine
       __syncwarp();
+      if (ew == 0 && lane == 0) HQ_TRACE(4, tcount);
       if (lane == 0) {
         mbar_arrive(smem_u32(&ctl.tempty[as]));
         if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
-        if (p.staged_out) {
+        if (use_tma_store) {
           tma_store_2d(&map_out, my_stage, ((n0 + half * cols_per_warp) * p.out_bits >> 3), m_tile * kTileM + q * 32);
           tma_store_commit();
         }
       }
     }
-    if (p.staged_out && lane == 0) tma_store_wait_all();
+    if (use_tma_store && lane == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -579,6 +696,10 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
 int g_driver_version = 0;
+int g_store_direct = 0;
+#ifdef HQ_TC_TRACE
+long long* g_trace_buf = nullptr;
+#endif      // experiment switch (environment variable HQ_TC_STORE=direct)
 
 bool load_driver_entry_points() {
   if (g_encode_tiled && g_encode_im2col) return true;
@@ -594,6 +715,8 @@ bool load_driver_entry_points() {
     return false;
   g_encode_im2col = (EncodeIm2colFn)fn;
   cudaDriverGetVersion(&g_driver_version);
+  const char* e = getenv("HQ_TC_STORE");
+  g_store_direct = (e && e[0] == 'd') ? 1 : 0;
   return true;
 }
 
@@ -683,12 +806,14 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // one store box per epilogue warp: 32 rows x (half the tile's columns), at most 128 bytes wide
     p.out_ib = (p.bn / 2) * a.out_bits / 8;
     p.out_boxes = 1;
-    out_tile_bytes = kTileM * p.bn * a.out_bits / 8;
-    if (out_tile_bytes < 8 * 1024) out_tile_bytes = 8 * 1024;     // keep the next region 1024-aligned
+    p.store_direct = g_store_direct;
+    out_tile_bytes = p.store_direct ? 0 : 2 * kTileM * p.bn * a.out_bits / 8;       // two boxes per warp
+    if (!p.store_direct && out_tile_bytes < 8 * 1024) out_tile_bytes = 8 * 1024;    // keep the next region 1024-aligned
   }
   if (p.staged_res) {
     p.res_ib = p.bn < 128 ? p.bn : 128;
     p.res_boxes = p.bn / p.res_ib;
+    p.res_ib_log2 = p.res_ib == 128 ? 7 : 6;
     res_tile_bytes = kTileM * p.bn;
   }
   const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
@@ -701,12 +826,35 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.relu = a.relu; p.qmin = a.qmin; p.qmax = a.qmax;
-  p.out = a.out; p.out_bits = a.out_bits;
+  p.out = a.out; p.out_bits = a.out_bits; p.out_signed = a.out_signed;
+  {
+    const int lo = a.relu ? (a.qmin > 0 ? a.qmin : 0) : a.qmin;
+    p.sat_pack = (a.out_bits == 8 && ((!a.out_signed && lo == 0 && a.qmax == 255) ||
+                                      (a.out_signed && lo == -128 && a.qmax == 127))) ? 1 : 0;
+  }
   p.status = h->dev_status;
+#ifdef HQ_TC_TRACE
+  {
+    static long long* buf = nullptr;
+    if (!buf) { cudaMalloc(&buf, 12 * 2048 * sizeof(long long)); }
+    cudaMemsetAsync(buf, 0, 12 * 2048 * sizeof(long long), stream);
+    p.trace = buf;
+    g_trace_buf = buf;
+  }
+#endif
 
   const CUtensorMapSwizzle swz = swizzle_for(p.bkb);
   alignas(64) CUtensorMap map_a, map_b, map_out, map_res;
-  {
+  p.a_tiled = (a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0) ? 1 : 0;
+  if (p.a_tiled) {
+    const cuuint64_t dims[2] = {(cuuint64_t)a.cin, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.cin};
+    const cuuint32_t box[2] = {(cuuint32_t)p.bkb, (cuuint32_t)kTileM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (g_encode_tiled(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(a.in), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
+  } else {
     // activations: (C, W, H, N) with byte strides; base pixels range over
     // [-pad, W + pad - (kw-1)) so that the hardware's pixel walk equals the output raster
     const cuuint64_t dims[4] = {(cuuint64_t)a.cin, (cuuint64_t)a.w, (cuuint64_t)a.h, (cuuint64_t)a.n};
@@ -749,3 +897,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   conv_tc_kernel<<<grid, kThreads, smem, stream>>>(map_a, map_b, map_out, map_res, p);
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
+
+#ifdef HQ_TC_TRACE
+extern "C" int hq_debug_trace_read(long long* host) {
+  if (!g_trace_buf) return 1;
+  return cudaMemcpy(host, g_trace_buf, 12 * 2048 * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : 2;
+}
+#endif

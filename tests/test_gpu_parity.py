@@ -123,6 +123,23 @@ def test_conv_tensor_core_general_tiles_with_residual(hq):
         run_conv_and_compare(hq, case, path=2)
 
 
+def test_conv_tensor_core_clamp_variants(hq):
+    # clamp bounds inside the type's range (explicit min/max instead of the saturating pack), signed
+    # residual operand, signed output with residual
+    case = inputs.conv_case(207, 2, 12, 12, 64, 128, 1, 1, 0, residual=True, c_range=(39, 43))
+    case["qmin"], case["qmax"] = 3, 200
+    run_conv_and_compare(hq, case, path=2)
+    case = inputs.conv_case(208, 2, 12, 12, 64, 128, 1, 1, 0, residual=True, relu=False, c_range=(39, 43))
+    case["res"] = case["res"].view(np.int8)
+    case["res_signed"] = 1
+    case["rc"][:] = np.arange(128) % 36 + 9          # every residual shift from 9 to 44
+    run_conv_and_compare(hq, case, path=2)
+    case = inputs.conv_case(209, 1, 12, 12, 64, 64, 3, 1, 1, residual=True, relu=True, c_range=(39, 43))
+    case["rc"][:] = np.arange(64) % 36 + 9
+    case["c"][:] = np.arange(64) % 30 + 32            # main shifts from 32 to 61
+    run_conv_and_compare(hq, case, path=2)
+
+
 LOWERED_CASES = [
     # n, h, w, cin, cout, k, stride, pad
     (2, 32, 32, 3, 64, 7, 2, 3),
