@@ -823,16 +823,20 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const long long out_row_bytes = (long long)a.cout * a.out_bits / 8;
   p.staged_out = (a.out_bits != 32 && out_row_bytes % 16 == 0) ? 1 : 0;
   p.staged_res = (p.staged_out && a.res && a.res_bits == 8 && a.cout % 16 == 0) ? 1 : 0;
-  p.pt = pick_pt(P, p.c_tiles, h->sm_count, p.staged_res ? 128 : 256);
+  const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
+  // staging: 8 warps x 128 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 x [pt][128]
+  const int out_tile_bytes = p.staged_out ? kEpilogueWarps * kTileC * 32 : 0;
+  int stages = 0, stage_bytes = 0, res_tile_bytes = 0;
+  for (int cap = 256; cap >= 64; cap >>= 1) {          // largest pixel tile that leaves room for >= 3 stages
+    p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
+    stage_bytes = (kTileC + p.pt) * p.bkb;
+    res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
+    stages = (smem_budget - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
+    if (stages >= 3 || p.pt == 64) break;
+  }
   p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
   p.x_signed = a.in_signed;
   p.tmem_cols = (uint32_t)(2 * p.pt);
-  const int stage_bytes = (kTileC + p.pt) * p.bkb;
-  // staging: 8 warps x 128 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 x [pt][128]
-  const int out_tile_bytes = p.staged_out ? kEpilogueWarps * kTileC * 32 : 0;
-  const int res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-  const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
-  int stages = (smem_budget - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return HQ_ERR_UNSUPPORTED;
   p.stages = stages;
