@@ -170,6 +170,32 @@ hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* 
 hq_status hq_network_launch_count(const hq_network* net, int32_t* launches);
 hq_status hq_network_destroy(hq_network* net);
 
+/*
+ * hq_conv2d for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a deployment convenience of the library, not a step of the method.)
+ *
+ * Who this is for: code that must not call cudaMalloc when a layer runs - a serving process whose
+ * memory was carved up at start-up and whose policy forbids later driver allocations (they stall
+ * every stream of the context and can fail under a tight budget), a component running while another
+ * library owns the rest of the device memory, or a plug-in that was handed a stream and buffers
+ * but no allocator.  hq_conv2d may grow a scratch buffer for thin first layers; this variant never
+ * does.  It needs no hq_handle either (creating one allocates).
+ *
+ * It computes exactly what hq_conv2d computes on its lowered path (patch matrix, then the
+ * tensor-core kernel; 8-bit operands, K = kh*kw*cin <= 4096, any cin), with the patch matrix and
+ * the padded weights in a fixed 8 MiB array that is part of the library's device image.  A request
+ * needing more than 8 MiB (n*ho*wo * K rounded up to 32, plus cout * that) returns HQ_ERR_WORKSPACE;
+ * use hq_conv2d or a smaller batch then.  It calls no cudaMalloc, cudaFree or allocating library
+ * routine.  The first call on a device looks up the array's device address, the driver's
+ * tensor-map encoders and the kernel's shared-memory limit; make that first call outside any
+ * stream capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents: the call rewrites everything it later reads and clears its status word on `stream`,
+ * but two calls whose GPU work overlaps (different streams, or graphs replayed concurrently) race on
+ * the array and give undefined results - serialise them.  The current device is used; pointers follow
+ * the rules of hq_conv2d.  An expired device-side wait is not reported by this variant.
+ */
+hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
+
 /* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail. */
 hq_status hq_set_conv_path(hq_handle* h, int32_t path);
 

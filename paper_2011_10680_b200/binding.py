@@ -21,7 +21,7 @@ HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant"
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
-    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers",
+    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc",
 ]
 
 
@@ -76,6 +76,7 @@ def lib():
         L.hq_maxpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
         L.hq_network_create.argtypes = [vp, LP, i32, i32, i32, i32, i32, i32, C.POINTER(vp)]
         L.hq_run_network.argtypes = [vp, TP, TP, C.POINTER(vp), vp]
+        L.hq_conv2d_noalloc.argtypes = [TP, DP, TP, vp]
         L.hq_network_time_layers.argtypes = [vp, TP, TP, C.POINTER(C.c_int64), vp]
         L.hq_network_layer_bytes.argtypes = [vp, i32, C.POINTER(C.c_int64)]
         L.hq_network_launch_count.argtypes = [vp, C.POINTER(i32)]
@@ -195,6 +196,18 @@ class Handle:
                          case["out_bits"], case["out_signed"], dev["res"], case["res_bits"], case["res_signed"],
                          dev["rb"], dev["rc"], case["relu"], case["qmin"], case["qmax"])
         return st, out
+
+
+def conv2d_noalloc(case: dict, dev: dict, out):
+    """hq_conv2d_noalloc on an uploaded conv case: no handle, no allocation inside the library."""
+    tin = tensor_of(dev["x"], case["cin"], case["bits"], case["in_signed"])
+    tout = tensor_of(out, case["cout"], case["out_bits"], case["out_signed"])
+    tres = tensor_of(dev["res"], case["cout"], case["res_bits"], case["res_signed"]) if dev["res"] is not None else None
+    d = hq_conv_desc(case["kh"], case["kw"], case["stride"], case["pad"], case["cin"], case["cout"], case["bits"],
+                     dev["wgt"].data_ptr(), dev["bias"].data_ptr() if dev["bias"] is not None else None,
+                     _dy(dev["b"], dev["c"]), C.pointer(tres) if tres is not None else None, _dy(dev["rb"], dev["rc"]),
+                     case["relu"], case["qmin"], case["qmax"])
+    return lib().hq_conv2d_noalloc(C.byref(tin), C.byref(d), C.byref(tout), _stream())
 
 
 def upload_case(case: dict) -> dict:

@@ -111,3 +111,96 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
   t.in = patches; t.h = a.ho; t.w = a.wo; t.cin = Kp; t.wgt = wpad; t.kh = t.kw = 1; t.stride = 1; t.pad = 0;
   return hq_launch_conv_tc(h, t, s);
 }
+
+// ------------------------------------------------------------------------------------------------
+// hq_conv2d_noalloc: the lowered convolution for callers that may not allocate device memory.
+//
+// The patch matrix and the padded weights, which hq_conv2d keeps in a buffer it allocates, live here
+// in a fixed array inside the library's own device image.  Every GPU that loads the library carries
+// the array until the process exits, so it is kept modest: HQ_NOALLOC_SCRATCH_BYTES.
+// ------------------------------------------------------------------------------------------------
+#define HQ_NOALLOC_SCRATCH_BYTES (8u << 20)      /* 8 MiB: e.g. one 224x224x3 image through a 7x7/2 first layer needs 2 MiB */
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HQ_NOALLOC_SCRATCH_BYTES];
+static __device__ uint32_t g_noalloc_status;     // written by a kernel whose bounded wait ran out
+
+namespace {
+
+// Host-side record per device ordinal.  The array names above are only host-side stand-ins for the
+// device objects; the addresses the kernels need come from cudaGetSymbolAddress, taken once per
+// device while that device is current.
+struct NoAllocDevice { bool ready; void* scratch; uint32_t* status; int sm_count; };
+constexpr int kMaxDevices = 64;
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+
+hq_status noalloc_setup(int dev) {
+  NoAllocDevice& d = g_noalloc_dev[dev];
+  if (d.ready) return HQ_OK;
+  int major = 0, sms = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return HQ_ERR_CUDA;
+  if (major != 10) return HQ_ERR_UNSUPPORTED;                  // kernels are built for sm_100a only
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HQ_ERR_CUDA;
+  if (!hq_conv_tc_init()) return HQ_ERR_CUDA;                  // driver entry points, shared-memory limit
+  void* scratch = nullptr;
+  void* status = nullptr;
+  if (cudaGetSymbolAddress(&scratch, g_noalloc_scratch) != cudaSuccess || !scratch) return HQ_ERR_CUDA;
+  if (cudaGetSymbolAddress(&status, g_noalloc_status) != cudaSuccess || !status) return HQ_ERR_CUDA;
+  d.scratch = scratch; d.status = (uint32_t*)status; d.sm_count = sms; d.ready = true;
+  return HQ_OK;
+}
+
+inline bool na_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream) {
+  if (!in || !d || !out || !in->data || !out->data || !d->w) return HQ_ERR_INVALID_ARG;
+  if (in->bits != 8 || d->w_bits != 8) return HQ_ERR_UNSUPPORTED;          // 8-bit operands only
+  if (!(out->bits == 8 || out->bits == 4 || out->bits == 32)) return HQ_ERR_INVALID_ARG;
+  if (in->n < 0 || in->h < 1 || in->w < 1 || in->c < 1) return HQ_ERR_INVALID_ARG;
+  if (d->kh < 1 || d->kw < 1 || d->stride < 1 || d->pad < 0 || d->cout < 1 || d->cin != in->c) return HQ_ERR_INVALID_ARG;
+  if (in->h + 2 * d->pad < d->kh || in->w + 2 * d->pad < d->kw) return HQ_ERR_INVALID_ARG;
+  const int ho = (in->h + 2 * d->pad - d->kh) / d->stride + 1, wo = (in->w + 2 * d->pad - d->kw) / d->stride + 1;
+  if (out->n != in->n || out->h != ho || out->w != wo || out->c != d->cout) return HQ_ERR_INVALID_ARG;
+  if (out->bits == 4 && (d->cout & 1)) return HQ_ERR_INVALID_ARG;
+  if (!na_aligned16(in->data) || !na_aligned16(out->data) || !na_aligned16(d->w)) return HQ_ERR_ALIGNMENT;
+  ConvArgs a{};
+  a.in = in->data; a.n = in->n; a.h = in->h; a.w = in->w; a.cin = in->c; a.in_bits = 8; a.in_signed = in->is_signed;
+  a.wgt = d->w; a.cout = d->cout; a.kh = d->kh; a.kw = d->kw; a.stride = d->stride; a.pad = d->pad;
+  a.bias = d->bias; a.b = d->requant.b; a.c = d->requant.c;
+  a.relu = d->relu; a.qmin = d->qmin; a.qmax = d->qmax;
+  a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
+  if (out->bits == 32) {
+    if (d->residual) return HQ_ERR_INVALID_ARG;
+  } else {
+    if (!d->requant.b || !d->requant.c) return HQ_ERR_INVALID_ARG;
+    long long lo = out->is_signed ? -(1LL << (out->bits - 1)) : 0;
+    long long hi = out->is_signed ? (1LL << (out->bits - 1)) - 1 : (1LL << out->bits) - 1;
+    if (d->qmin > d->qmax || d->qmin < lo || d->qmax > hi) return HQ_ERR_INVALID_ARG;
+    if (d->residual) {
+      const hq_tensor* r = d->residual;
+      if (!r->data || !(r->bits == 8 || r->bits == 32) || r->n != out->n || r->h != ho || r->w != wo || r->c != d->cout ||
+          !d->res_rescale.b || !d->res_rescale.c) return HQ_ERR_INVALID_ARG;
+      if (!na_aligned16(r->data)) return HQ_ERR_ALIGNMENT;
+      a.res = r->data; a.res_bits = r->bits; a.res_signed = r->is_signed; a.rb = d->res_rescale.b; a.rc = d->res_rescale.c;
+    }
+  }
+  if (!hq_conv_lowering_applies(a)) return HQ_ERR_UNSUPPORTED;
+  if (hq_conv_lowering_bytes(a) > (size_t)HQ_NOALLOC_SCRATCH_BYTES) return HQ_ERR_WORKSPACE;   // beyond the fixed array
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HQ_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return HQ_ERR_UNSUPPORTED;
+  const hq_status st = noalloc_setup(dev);       // first call on this device only
+  if (st != HQ_OK) return st;
+  const NoAllocDevice& nd = g_noalloc_dev[dev];
+  cudaStream_t s = (cudaStream_t)stream;
+  // The array keeps whatever the last call left.  The patch matrix and the padded weights are
+  // rewritten in full (zero columns included) before anything reads them; only the status word
+  // has to start at zero.
+  if (cudaMemsetAsync(nd.status, 0, sizeof(uint32_t), s) != cudaSuccess) return HQ_ERR_CUDA;
+  hq_handle tmp{};
+  tmp.device = dev; tmp.conv_path = 0; tmp.sm_count = nd.sm_count; tmp.dev_status = nd.status;
+  tmp.workspace = nullptr; tmp.workspace_bytes = 0;
+  return hq_launch_conv_lowered(&tmp, a, nd.scratch, s);
+}
