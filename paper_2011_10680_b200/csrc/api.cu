@@ -72,8 +72,14 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
   cudaStream_t s = (cudaStream_t)stream;
   const bool tc_ok = hq_conv_tc_supported(a);
-  if (h->conv_path == 2 && !tc_ok) return HQ_ERR_UNSUPPORTED;
+  if (h->conv_path == 2 && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
   if (h->conv_path != 1 && tc_ok) return hq_launch_conv_tc(h, a, s);
+  if (h->conv_path != 1 && hq_conv_widen4_applies(a)) {
+    // packed 4-bit operands: widened copies in scratch, then the tensor-core kernel
+    const size_t need = hq_conv_widen4_bytes(a);
+    if (scratch && scratch_bytes >= need) return hq_launch_conv_widen4(h, a, scratch, s);
+    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_widen4(h, a, h->workspace, s);
+  }
   if (h->conv_path != 1 && hq_conv_lowering_applies(a)) {
     // thin first layers: patch matrix in the handle's scratch buffer, then the tensor-core kernel
     const size_t need = hq_conv_lowering_bytes(a);
@@ -284,7 +290,11 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
           ConvArgs a{};
           a.n = batch; a.h = in.h; a.w = in.w; a.cin = in.c; a.in_bits = in.bits; a.cout = d.cout; a.kh = d.kh; a.kw = d.kw;
           a.stride = d.stride; a.pad = d.pad; a.ho = o.h; a.wo = o.w; a.out_bits = o.bits;
-          if (!hq_conv_tc_supported(a) && hq_conv_lowering_applies(a)) {
+          if (hq_conv_widen4_applies(a)) {
+            const size_t need = hq_conv_widen4_bytes(a);
+            if (need > net->scratch_bytes) net->scratch_bytes = need;
+            net->launches += 2;                 // two widening kernels
+          } else if (!hq_conv_tc_supported(a) && hq_conv_lowering_applies(a)) {
             const size_t need = hq_conv_lowering_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
             net->launches += 2;                 // weight padding + patch matrix kernels

@@ -74,6 +74,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
 bool hq_conv_lowering_applies(const ConvArgs& a);
 size_t hq_conv_lowering_bytes(const ConvArgs& a);
 hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
+// 4-bit operands: widen to bytes in scratch, then the tensor-core kernel.
+bool hq_conv_widen4_applies(const ConvArgs& a);
+size_t hq_conv_widen4_bytes(const ConvArgs& a);
+hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
 // Grow the handle's scratch buffer (not allowed while `s` is capturing).
 hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s);
 cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s);

@@ -113,6 +113,70 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
 }
 
 // ------------------------------------------------------------------------------------------------
+// 4-bit operands on the tensor-core kernel.  sm_100 has no 4-bit integer MMA, so packed INT4
+// activations and weights (two per byte, even element in the low nibble) are widened to one byte
+// per value and the contraction of Eq. 3 runs on the 8-bit kernel; the integers, hence the results,
+// are unchanged.  This version widens in global memory (a scratch copy of the layer input and of
+// the weights) ahead of the convolution.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// 8 packed bytes -> 16 bytes; element 2j = low nibble of byte j.
+template <bool SIGNED>
+__global__ void __launch_bounds__(256) widen4_kernel(const uint2* __restrict__ in, long long n_vec, uint4* __restrict__ out) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (long long)gridDim.x * blockDim.x) {
+    const uint2 v = __ldg(in + i);
+    unsigned o[4];
+    const unsigned w[2] = {v.x, v.y};
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      unsigned lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
+      if (SIGNED) { lo |= (lo & 0x08080808u) * 0x1Eu; hi |= (hi & 0x08080808u) * 0x1Eu; }   // sign-extend each nibble
+      o[2 * k] = __byte_perm(lo, hi, 0x5140);          // n0 n1 n2 n3
+      o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);      // n4 n5 n6 n7
+    }
+    out[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+cudaError_t launch_widen4(const void* in, long long elems, int is_signed, void* out, int sm_count, cudaStream_t s) {
+  const long long n_vec = elems / 16;                  // callers guarantee a multiple of 16 elements
+  if (n_vec == 0) return cudaSuccess;
+  long long blocks = (n_vec + 255) / 256;
+  const long long cap = (long long)sm_count * 16;
+  const int grid = (int)(blocks < cap ? blocks : cap);
+  if (is_signed) widen4_kernel<true><<<grid, 256, 0, s>>>((const uint2*)in, n_vec, (uint4*)out);
+  else widen4_kernel<false><<<grid, 256, 0, s>>>((const uint2*)in, n_vec, (uint4*)out);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool hq_conv_widen4_applies(const ConvArgs& a) {
+  if (a.in_bits != 4 || a.cin % 32 != 0) return false;
+  ConvArgs t = a;
+  t.in_bits = 8;
+  return hq_conv_tc_supported(t);
+}
+
+size_t hq_conv_widen4_bytes(const ConvArgs& a) {
+  const long long x = (long long)a.n * a.h * a.w * a.cin, w = (long long)a.cout * a.kh * a.kw * a.cin;
+  return (size_t)(((x + 255) / 256 + (w + 255) / 256) * 256);
+}
+
+// `scratch` must hold hq_conv_widen4_bytes(a) bytes, 256-byte aligned.
+hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s) {
+  const long long x = (long long)a.n * a.h * a.w * a.cin, w = (long long)a.cout * a.kh * a.kw * a.cin;
+  unsigned char* xw = (unsigned char*)scratch;
+  unsigned char* ww = xw + (x + 255) / 256 * 256;
+  if (launch_widen4(a.in, x, a.in_signed, xw, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+  if (launch_widen4(a.wgt, w, 1, ww, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+  ConvArgs t = a;
+  t.in = xw; t.wgt = ww; t.in_bits = 8;
+  return hq_launch_conv_tc(h, t, s);
+}
+
+// ------------------------------------------------------------------------------------------------
 // hq_conv2d_noalloc: the lowered convolution for callers that may not allocate device memory.
 //
 // The patch matrix and the padded weights, which hq_conv2d keeps in a buffer it allocates, live here

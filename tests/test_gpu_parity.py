@@ -140,6 +140,28 @@ def test_conv_tensor_core_clamp_variants(hq):
     run_conv_and_compare(hq, case, path=2)
 
 
+INT4_TC_CASES = [
+    # n, h, w, cin, cout, k, stride, pad, out_bits, residual
+    (2, 14, 14, 128, 128, 3, 1, 1, 4, False),      # uint4 in, uint4 out (conv inside a 4-bit block)
+    (2, 14, 14, 64, 256, 1, 1, 0, 8, True),        # uint4 in, uint8 stream out with residual (block's last conv)
+    (1, 14, 14, 256, 64, 1, 2, 0, 8, False),       # strided shortcut conv
+    (3, 7, 7, 32, 48, 3, 1, 1, 4, False),
+]
+
+
+@pytest.mark.parametrize("cfg", INT4_TC_CASES)
+def test_conv_int4_on_tensor_cores(hq, cfg):
+    n, h, w, cin, cout, k, stride, pad, out_bits, residual = cfg
+    case = inputs.conv_case(210, n, h, w, cin, cout, k, stride, pad, bits=4, out_bits=out_bits, residual=residual,
+                            c_range=(42, 46) if out_bits == 8 else (46, 50))
+    run_conv_and_compare(hq, case, path=2)          # 4-bit operands widened, contraction on tcgen05
+
+
+def test_conv_int4_signed_activations(hq):
+    case = inputs.conv_case(211, 2, 10, 10, 64, 64, 3, 1, 1, bits=4, in_signed=True, relu=False, c_range=(42, 46))
+    run_conv_and_compare(hq, case, path=2)
+
+
 LOWERED_CASES = [
     # n, h, w, cin, cout, k, stride, pad
     (2, 32, 32, 3, 64, 7, 2, 3),
