@@ -80,6 +80,12 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
     if (scratch && scratch_bytes >= need) return hq_launch_conv_widen4(h, a, scratch, s);
     if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_widen4(h, a, h->workspace, s);
   }
+  if (h->conv_path != 1 && hq_conv_s2d_applies(a)) {
+    // ImageNet-style first layer: space-to-depth copy of the image, then the tensor-core kernel
+    const size_t need = hq_conv_s2d_bytes(a);
+    if (scratch && scratch_bytes >= need) return hq_launch_conv_s2d(h, a, scratch, s);
+    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_s2d(h, a, h->workspace, s);
+  }
   if (h->conv_path != 1 && hq_conv_lowering_applies(a)) {
     // thin first layers: patch matrix in the handle's scratch buffer, then the tensor-core kernel
     const size_t need = hq_conv_lowering_bytes(a);
@@ -294,6 +300,10 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
             const size_t need = hq_conv_widen4_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
             net->launches += 2;                 // two widening kernels
+          } else if (hq_conv_s2d_applies(a)) {
+            const size_t need = hq_conv_s2d_bytes(a);
+            if (need > net->scratch_bytes) net->scratch_bytes = need;
+            net->launches += 2;                 // weight re-layout + space-to-depth kernels
           } else if (!hq_conv_tc_supported(a) && hq_conv_lowering_applies(a)) {
             const size_t need = hq_conv_lowering_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;

@@ -56,6 +56,9 @@ struct ConvArgs {
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   int32_t relu, qmin, qmax;
   void* out; int32_t ho, wo, out_bits, out_signed;
+  // internal lowerings only (zero for calls that come from the ABI):
+  int32_t pad_after_delta;   // padding after the last row/column minus `pad` (space-to-depth first layer: -1)
+  int32_t tap16;             // 1: cin == 16 and every filter tap is one 16-byte K chunk (un-swizzled X tiles)
 };
 
 struct EltArgs {
@@ -74,6 +77,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
 bool hq_conv_lowering_applies(const ConvArgs& a);
 size_t hq_conv_lowering_bytes(const ConvArgs& a);
 hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
+// 7x7 / stride 2 / 3-channel first layer as a 4x4 stride-1 conv over a space-to-depth copy of the image.
+bool hq_conv_s2d_applies(const ConvArgs& a);
+size_t hq_conv_s2d_bytes(const ConvArgs& a);
+hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
 // 4-bit operands: widen to bytes in scratch, then the tensor-core kernel.
 bool hq_conv_widen4_applies(const ConvArgs& a);
 size_t hq_conv_widen4_bytes(const ConvArgs& a);

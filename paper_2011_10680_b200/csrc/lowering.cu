@@ -113,6 +113,86 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
 }
 
 // ------------------------------------------------------------------------------------------------
+// First layer of ImageNet ResNets (7x7, stride 2, pad 3, 3 input channels) without a patch matrix.
+// A space-to-depth copy of the image, s2d[n][y][x][(dy*2+dx)*3 + c] = in[n][2y+dy][2x+dx][c] with the
+// 12 values padded to 16 channels, turns the layer into a 4x4 stride-1 convolution with 16-byte
+// pixels: output (oh, ow) reads s2d rows oh-2 .. oh+1 (two rows of padding before, one after), and
+// weight w2[oc][ty][tx][(dy*2+dx)*3 + c] = w[oc][2ty+dy-1][2tx+dx-1][c] (zero where the 7x7 index falls
+// outside 0..6 and in the padded channels).  Zeros add nothing, so the INT32 accumulator is unchanged.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+__global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned char* __restrict__ in, int n, int h, int w,
+                                                             uint4* __restrict__ out) {
+  const int h2 = h >> 1, w2 = w >> 1;
+  const long long total = (long long)n * h2 * w2;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int x = (int)(i % w2);
+    long long t = i / w2;
+    const int y = (int)(t % h2);
+    const int img = (int)(t / h2);
+    unsigned word[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int dy = 0; dy < 2; ++dy) {
+      const unsigned char* src = in + (((long long)img * h + 2 * y + dy) * w + 2 * x) * 3;   // 6 contiguous bytes
+#pragma unroll
+      for (int b = 0; b < 6; ++b) {
+        const int k = dy * 6 + b;
+        word[k >> 2] |= (unsigned)__ldg(src + b) << (8 * (k & 3));
+      }
+    }
+    out[i] = make_uint4(word[0], word[1], word[2], word[3]);
+  }
+}
+
+__global__ void s2d_weights_kernel(const signed char* __restrict__ w, int cout, signed char* __restrict__ out) {
+  const int total = cout * 256;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int ch16 = i & 15, tx = (i >> 4) & 3, ty = (i >> 6) & 3, oc = i >> 8;
+    signed char v = 0;
+    if (ch16 < 12) {
+      const int c = ch16 % 3, dx = (ch16 / 3) & 1, dy = ch16 / 6;
+      const int r = 2 * ty + dy - 1, sx = 2 * tx + dx - 1;
+      if (r >= 0 && r < 7 && sx >= 0 && sx < 7) v = w[((oc * 7 + r) * 7 + sx) * 3 + c];
+    }
+    out[i] = v;
+  }
+}
+
+}  // namespace
+
+bool hq_conv_s2d_applies(const ConvArgs& a) {
+  if (a.in_bits != 8 || a.cin != 3 || a.kh != 7 || a.kw != 7 || a.stride != 2 || a.pad != 3) return false;
+  if ((a.h & 1) || (a.w & 1) || a.tap16) return false;
+  ConvArgs t = a;
+  t.h = a.h / 2; t.w = a.w / 2; t.cin = 16; t.kh = t.kw = 4; t.stride = 1; t.pad = 2; t.pad_after_delta = -1; t.tap16 = 1;
+  return hq_conv_tc_supported(t);
+}
+
+size_t hq_conv_s2d_bytes(const ConvArgs& a) {
+  const long long img = (long long)a.n * (a.h / 2) * (a.w / 2) * 16, wts = (long long)a.cout * 256;
+  return (size_t)(((img + 255) / 256 + (wts + 255) / 256) * 256);
+}
+
+// `scratch` must hold hq_conv_s2d_bytes(a) bytes, 256-byte aligned.
+hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s) {
+  const long long px = (long long)a.n * (a.h / 2) * (a.w / 2);
+  if (px == 0) return HQ_OK;
+  unsigned char* img = (unsigned char*)scratch;
+  signed char* wts = (signed char*)(img + (px * 16 + 255) / 256 * 256);
+  s2d_weights_kernel<<<(a.cout * 256 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, wts);
+  if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+  long long blocks = (px + 255) / 256;
+  const long long cap = (long long)h->sm_count * 32;
+  space_to_depth_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, (uint4*)img);
+  if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+  ConvArgs t = a;
+  t.in = img; t.wgt = wts; t.h = a.h / 2; t.w = a.w / 2; t.cin = 16; t.kh = t.kw = 4; t.stride = 1; t.pad = 2;
+  t.pad_after_delta = -1; t.tap16 = 1;
+  return hq_launch_conv_tc(h, t, s);
+}
+
+// ------------------------------------------------------------------------------------------------
 // 4-bit operands on the tensor-core kernel.  sm_100 has no 4-bit integer MMA, so packed INT4
 // activations and weights (two per byte, even element in the low nibble) are widened to one byte
 // per value and the contraction of Eq. 3 runs on the 8-bit kernel; the integers, hence the results,
