@@ -156,6 +156,57 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Config 5: fused conv/GEMM sweep over the ResNet-50 layer shapes (INT8 and INT4, with and without the
+    residual add); per shape device time (CUDA events, L2 flushed between repetitions by writing 256 MB),
+    integer TOPS, achieved GB/s of the algorithmic bytes and the fraction of that shape's own roofline."""
+    import torch
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    hq = binding.Handle(0)
+    hbm_peak, bf16_peak, peak_kind = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    rows = []
+    shapes = inputs.SWEEP_LAYERS if args.sweep_only < 0 else [inputs.SWEEP_LAYERS[args.sweep_only]]
+    for (hw, cin, cout, k, stride, has_res) in shapes:
+        n = max(1, args.sweep_pixels // (hw * hw))
+        for bits in (8, 4):
+            for residual in ((False, True) if has_res else (False,)):
+                case = inputs.conv_case(5, n, hw, hw, cin, cout, k, stride, k // 2, bits=bits, residual=residual)
+                dev = binding.upload_case(case)
+                times = []
+                for rep in range(args.warmup + args.steps):
+                    flush.fill_(rep & 0xFF)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    st, out = hq.conv_case(case, dev)
+                    e1.record()
+                    assert st == binding.HQ_OK
+                    torch.cuda.synchronize()
+                    if rep >= args.warmup:
+                        times.append(e0.elapsed_time(e1) * 1e3)
+                hq.sync()
+                us = float(np.median(times))
+                m = n * case["ho"] * case["wo"]
+                kk = k * k * cin
+                ops = 2 * m * cout * kk
+                byt = n * hw * hw * cin * bits // 8 + cout * kk * bits // 8 + m * cout + (m * cout if residual else 0) + 13 * cout
+                t_roof = max(ops / (NOMINAL_I8_TOPS * 1e12), byt / (hbm_peak * 1e9)) * 1e6
+                rows.append(dict(hw=hw, cin=cin, cout=cout, k=k, batch=n, bits=bits, residual=residual, M=m, N=cout, K=kk,
+                                 us=us, best_us=float(min(times)), tops=ops / us / 1e6, gbs=byt / us / 1e3,
+                                 frac_of_i8_nominal=ops / us / 1e6 / NOMINAL_I8_TOPS, roofline_us=t_roof,
+                                 frac_of_own_roofline=t_roof / us, bound="tensor" if ops / (NOMINAL_I8_TOPS * 1e12) > byt / (hbm_peak * 1e9) else "hbm"))
+    if args.layers_out:
+        json.dump(rows, open(args.layers_out, "w"), indent=1)
+    best = max(rows, key=lambda r: r["tops"])
+    print(json.dumps({"metric": "fused conv INT TOPS vs tcgen05 i8 peak (sweep)", "shapes": len(rows),
+                      "best_tops": best["tops"], "best_shape": {k: best[k] for k in ("hw", "cin", "cout", "k", "batch", "bits")},
+                      "median_frac_of_own_roofline": float(np.median([r["frac_of_own_roofline"] for r in rows])),
+                      "hbm_peak": hbm_peak, "peak_kind": f"of {peak_kind}", "i8_nominal_tops": NOMINAL_I8_TOPS,
+                      "rows": [{k: (round(v, 3) if isinstance(v, float) else v) for k, v in r.items()} for r in rows]}), flush=True)
+    hq.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -166,6 +217,9 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (JSON) to this file")
+    ap.add_argument("--sweep", action="store_true", help="run the fused conv/GEMM sweep (config 5) instead of the network")
+    ap.add_argument("--sweep-pixels", type=int, default=200704, help="output pixels per sweep shape (batch is derived)")
+    ap.add_argument("--sweep-only", type=int, default=-1, help="run a single sweep shape (index), e.g. for profiling")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -174,6 +228,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
         return
 
     import torch

@@ -30,6 +30,7 @@
 // handle's status word, raises a CTA-wide abort flag and every role leaves its loop, drains what
 // it has in flight (again bounded), and the CTA frees its tensor memory and returns.
 #include <cuda.h>
+#include <climits>
 #include <cstdlib>
 
 #include "hq_internal.cuh"
@@ -246,7 +247,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t bkb) {
 
 // Per-thread (= per output channel) constants of the epilogue.
 struct ChanConst {
-  int b, sh;            // main branch multiplier; shift (c, or c - 32 on the fast path)
+  int b, sh;            // main branch multiplier; shift (c, or c - min(c,32) on the fast path)
+  int sh1;              // fast path: min(c, 32), the part of the shift taken by the funnel shift
+  int cmin31;           // fast path: min(c, 31)
   long long r0;         // bias*b + 2^(c-1)
   int rb, rh, rsh;      // residual multiplier; fast path: rh = 2^(rc-9), rsh = rc-8; else rsh = rc
   long long rr0;        // general path: 2^(rc-1)
@@ -258,10 +261,23 @@ struct ChanConst {
 //   residual  y += (hi32((r << 24) * rb) + 2^(rc-9)) >> (rc-8)                      (needs 9 <= rc)
 // The residual form is exact: (r<<24)*rb >> 32 = floor(r*rb / 2^8), the rounding constant 2^(rc-1) is
 // a multiple of 2^8, and the dropped low 8 bits of r*rb cannot carry across a multiple of 2^(rc-8).
-template <bool RES, bool RSIGNED>
+template <bool RES, bool RSIGNED, bool SMALL>
 __device__ __forceinline__ int requant_fast(int acc, unsigned rbyte, const ChanConst& k) {
   const long long t1 = (long long)acc * (long long)k.b + k.r0;
-  int s = (int)(t1 >> 32) >> k.sh;
+  int s;
+  if (!SMALL) {
+    s = (int)(t1 >> 32) >> k.sh;                       // c >= 32: |s| < 2^30
+  } else {
+    // some channel of this warp has c < 32: take bits [c, c+32) of the 64-bit value with a funnel shift
+    // and saturate to +-2^30 when the exact value does not fit (it is far outside every clamp range then,
+    // and |residual term| < 2^30 keeps the sum inside INT32)
+    const int hi = (int)(t1 >> 32);
+    const unsigned lo = (unsigned)t1;
+    const int s0 = (int)__funnelshift_rc(lo, (unsigned)hi, k.sh1);
+    const int above = hi >> k.cmin31;                  // the bits above the window (sign for c >= 32)
+    s = (above == (s0 >> 31)) ? (s0 >> k.sh) : (hi < 0 ? INT_MIN : INT_MAX);
+    s = max(min(s, 1 << 30), -(1 << 30));
+  }
   if (RES) {
     const unsigned top = rbyte << 24;
     if (RSIGNED) s += (__mulhi((int)top, k.rb) + k.rh) >> k.rsh;
@@ -269,7 +285,6 @@ __device__ __forceinline__ int requant_fast(int acc, unsigned rbyte, const ChanC
   }
   return s;
 }
-
 
 // Everything an epilogue warp needs, gathered once so the tile loops can live in their own functions.
 struct EpiCtx {
@@ -283,7 +298,7 @@ struct EpiCtx {
 // clamp by saturating convert or by min/max, optional 8-bit residual from the prefetched tile.  The
 // accumulator chunk of the next 32 pixels is requested from tensor memory before the current one is
 // processed, so the load's latency hides behind the arithmetic.
-template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED>
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL>
 __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e, const ChanConst& k) {
   const TcParams& p = *e.p;
   SharedCtl& ctl = *e.ctl;
@@ -323,7 +338,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e, const ChanC
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const unsigned rbyte = RES ? (unsigned)res_tile[(c * 32 + j) * kTileC] : 0u;
-          const int s = requant_fast<RES, RSIGNED>(va[j], rbyte, k);
+          const int s = requant_fast<RES, RSIGNED, SMALL>(va[j], rbyte, k);
           y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
         }
 #pragma unroll
@@ -338,7 +353,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e, const ChanC
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const unsigned rbyte = RES ? (unsigned)res_tile[((c + 1) * 32 + j) * kTileC] : 0u;
-            const int s = requant_fast<RES, RSIGNED>(vb[j], rbyte, k);
+            const int s = requant_fast<RES, RSIGNED, SMALL>(vb[j], rbyte, k);
             y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
           }
 #pragma unroll
@@ -430,13 +445,13 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
           const int variant = (p.res ? 2 : 0) | (p.res_signed ? 1 : 0);
           if (variant == 2) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, false>(v[j], rb8[j], k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, false, true>(v[j], rb8[j], k);
           } else if (variant == 3) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, true>(v[j], rb8[j], k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, true, true>(v[j], rb8[j], k);
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<false, false>(v[j], 0u, k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<false, false, true>(v[j], 0u, k);
           }
           if (p.sat_pack) {
             if (p.out_signed) {
@@ -683,7 +698,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (p.out_bits != 32) {
       k.b = ch_live ? p.b[ch] : 0;
       const int cc = ch_live ? p.c[ch] : 32;
-      if (cc < 32) fast = 0;
       k.sh = cc;
       k.r0 = (long long)k.bias * (long long)k.b + (1LL << (cc - 1));
       if (p.res) {
@@ -695,8 +709,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
     }
     fast = epi_bar_and(fast);                    // every live channel of the CTA allows 32-bit intermediates
+    const bool warp_small = __any_sync(0xffffffffu, k.sh < 32) != 0;     // some channel of this warp has c < 32
     if (fast) {
-      k.sh -= 32;
+      k.sh1 = k.sh < 32 ? k.sh : 32;
+      k.cmin31 = k.sh < 31 ? k.sh : 31;
+      k.sh -= k.sh1;
       if (p.res) {
         if (k.rsh >= 40) { k.rb = 0; k.rh = 0; k.rsh = 1; }            // |r*rb| < 2^39: rounds to 0
         else { k.rh = 1 << (k.rsh - 9); k.rsh -= 8; }
@@ -712,15 +729,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
-        case 0: epilogue_loop_fast8<false, false, false, false>(e, k); break;
-        case 1: if (p.out_signed) epilogue_loop_fast8<false, false, true, true>(e, k);
-                else epilogue_loop_fast8<false, false, true, false>(e, k); break;
-        case 4: epilogue_loop_fast8<true, false, false, false>(e, k); break;
-        case 5: if (p.out_signed) epilogue_loop_fast8<true, false, true, true>(e, k);
-                else epilogue_loop_fast8<true, false, true, false>(e, k); break;
-        case 6: epilogue_loop_fast8<true, true, false, false>(e, k); break;
-        default: if (p.out_signed) epilogue_loop_fast8<true, true, true, true>(e, k);
-                 else epilogue_loop_fast8<true, true, true, false>(e, k); break;
+#define HQ_FAST8(R, RS, S, OS) do { if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true>(e, k); \
+                                    else epilogue_loop_fast8<R, RS, S, OS, false>(e, k); } while (0)
+        case 0: HQ_FAST8(false, false, false, false); break;
+        case 1: if (p.out_signed) HQ_FAST8(false, false, true, true); else HQ_FAST8(false, false, true, false); break;
+        case 4: HQ_FAST8(true, false, false, false); break;
+        case 5: if (p.out_signed) HQ_FAST8(true, false, true, true); else HQ_FAST8(true, false, true, false); break;
+        case 6: HQ_FAST8(true, true, false, false); break;
+        default: if (p.out_signed) HQ_FAST8(true, true, true, true); else HQ_FAST8(true, true, true, false); break;
+#undef HQ_FAST8
       }
     } else {
       epilogue_loop_general(e, k, fast);
