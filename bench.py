@@ -36,6 +36,10 @@ WORKLOADS = {
 }
 METRIC = "int-only ResNet-50 images/s @bs256; fused conv INT TOPS vs tcgen05 i8 peak"
 NOMINAL_I8_TOPS = 4500.0
+# dram__bytes_read.sum + dram__bytes_write.sum of all conv_tc_kernel launches of one pass, captured with ncu at
+# batch 64 (profiles/resnet50_int8_b256_launch_list.md) and scaled per image; writes are under-counted there
+# (outputs stay dirty in L2), so this is a lower bound of the batch-256 traffic.
+NCU_CONV_DRAM_BYTES_PER_IMAGE = (998.4e6 + 136.7e6) / 64
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
@@ -361,7 +365,12 @@ def main():
             "gpu_launches": net.launch_count() * args.steps,
             "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                         "frac": achieved / hbm_peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                         "frac": achieved / hbm_peak,
+                         "traffic": (NCU_CONV_DRAM_BYTES_PER_IMAGE * batch / max(n_conv_tc, 1)
+                                     if args.workload == "resnet50_int8_b256" else None),
+                         "traffic_note": "avg DRAM bytes per conv launch from an ncu capture at batch 64, scaled by images",
+                         "algorithmic_bytes_per_launch": tc_bytes / max(n_conv_tc, 1),
+                         "peak_kind": f"of {peak_kind}",
                          "kernel": "conv_tc_kernel", "launches_per_step": n_conv_tc,
                          "avg_launch_us": tc_ns / 1e3 / max(n_conv_tc, 1),
                          "algorithmic_bytes_per_step": tc_bytes,
