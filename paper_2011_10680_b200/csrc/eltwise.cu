@@ -88,6 +88,87 @@ __global__ void __launch_bounds__(256) residual_add_vec_kernel(EltArgs a, int gr
   }
 }
 
+// ---- 8-bit operands: 32-bit fast path ----------------------------------------------------------
+// A thread owns four consecutive channels (one 32-bit word per pixel) for the whole launch, so its dyadic
+// pairs stay in registers and a warp reads / writes 128 contiguous bytes per pixel.  For an 8-bit value q
+// and 9 <= c:  (q*b + 2^(c-1)) >> c  ==  (hi32((q << 24) * b) + 2^(c-9)) >> (c-8)   exactly, because
+// (q<<24)*b >> 32 = floor(q*b / 2^8), 2^(c-1) is a multiple of 2^8 and the dropped low 8 bits cannot carry
+// across a multiple of 2^(c-8); for c >= 40 the term rounds to 0.  Channels with c < 9 take the 64-bit form.
+struct Dy8 { int b, h, sh, c; };     // multiplier, 2^(c-9), c-8, original c
+
+__device__ __forceinline__ Dy8 make_dy8(int b, int c) {
+  Dy8 d; d.c = c;
+  if (c >= 40) { d.b = 0; d.h = 0; d.sh = 1; }
+  else if (c >= 9) { d.b = b; d.h = 1 << (c - 9); d.sh = c - 8; }
+  else { d.b = b; d.h = 0; d.sh = 0; }                       // c < 9: the thread switches to the 64-bit form
+  return d;
+}
+template <bool SIGNED>
+__device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` = the byte in bits 31:24; needs d.c >= 9; |result| < 2^30
+  if (SIGNED) return (__mulhi((int)top, d.b) + d.h) >> d.sh;
+  return (int)((__umulhi(top, (unsigned)d.b) + (unsigned)d.h) >> d.sh);
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4>
+__global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int lo, int hi) {
+  const int wx = blockIdx.x * blockDim.x + threadIdx.x;     // word (4 channels) of the pixel
+  if (wx >= words) return;
+  Dy8 m[4], r[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m[i] = make_dy8(__ldg(a.mb + 4 * wx + i), __ldg(a.mc + 4 * wx + i));
+    if (RES) r[i] = make_dy8(__ldg(a.rb + 4 * wx + i), __ldg(a.rc + 4 * wx + i));
+  }
+  bool slow = false;                       // a shift below 9 on one of this thread's channels: 64-bit form for the thread
+#pragma unroll
+  for (int i = 0; i < 4; ++i) slow = slow || m[i].c < 9 || (RES && r[i].c < 9);
+  const unsigned* mp = (const unsigned*)a.main_t;
+  const unsigned* rp = (const unsigned*)a.res;
+  const long long step = (long long)gridDim.y * blockDim.y;
+  auto one = [&](unsigned mw, unsigned rw, long long idx) {
+    int y[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (!slow) {
+        int s = dn8<MSIGNED>(__byte_perm(mw, 0u, 0x0444u | ((unsigned)i << 12)), m[i]);
+        if (RES) s += dn8<RSIGNED>(__byte_perm(rw, 0u, 0x0444u | ((unsigned)i << 12)), r[i]);
+        y[i] = min(max(s, lo), hi);
+      } else {
+        const unsigned mbyte = (mw >> (8 * i)) & 0xFFu, rbyte = (rw >> (8 * i)) & 0xFFu;
+        long long s = hq_dn(MSIGNED ? (int)(signed char)mbyte : (int)mbyte, __ldg(a.mb + 4 * wx + i), m[i].c);
+        if (RES) s += hq_dn(RSIGNED ? (int)(signed char)rbyte : (int)rbyte, __ldg(a.rb + 4 * wx + i), r[i].c);
+        y[i] = (int)(s < (long long)lo ? (long long)lo : (s > (long long)hi ? (long long)hi : s));
+      }
+    }
+    if (OUT4) {
+      ((unsigned short*)a.out)[idx] = (unsigned short)((y[0] & 0xF) | ((y[1] & 0xF) << 4) | ((y[2] & 0xF) << 8) | ((y[3] & 0xF) << 12));
+    } else {
+      ((unsigned*)a.out)[idx] = (unsigned)(y[0] & 0xFF) | ((unsigned)(y[1] & 0xFF) << 8) | ((unsigned)(y[2] & 0xFF) << 16) |
+                                ((unsigned)(y[3] & 0xFF) << 24);
+    }
+  };
+  constexpr int U = 8;                     // pixels (independent 4-byte loads) in flight per thread
+  long long p = (long long)blockIdx.y * blockDim.y + threadIdx.y;
+  for (; p + (U - 1) * step < a.pixels; p += U * step) {
+    unsigned mw[U], rw[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) mw[u] = __ldg(mp + (p + u * step) * words + wx);
+#pragma unroll
+    for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rp + (p + u * step) * words + wx) : 0u;
+#pragma unroll
+    for (int u = 0; u < U; ++u) one(mw[u], rw[u], (p + u * step) * words + wx);
+  }
+  for (; p < a.pixels; p += step)
+    one(__ldg(mp + p * words + wx), RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx);
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED>
+cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, cudaStream_t s) {
+  if (a.out_bits == 4) requant8_kernel<RES, MSIGNED, RSIGNED, true><<<grid, block, 0, s>>>(a, words, lo, hi);
+  else requant8_kernel<RES, MSIGNED, RSIGNED, false><<<grid, block, 0, s>>>(a, words, lo, hi);
+  return cudaGetLastError();
+}
+
 // Any channel count: one thread per output byte (one element at 8 bit, two at 4 bit).
 __global__ void residual_add_scalar_kernel(EltArgs a) {
   const int per = (a.out_bits == 4) ? 2 : 1;
@@ -232,6 +313,26 @@ __global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int c
 
 cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s) {
   if (a.pixels == 0) return cudaSuccess;
+  // 8-bit operands with a channel count the word mapping covers: 32-bit fast kernel
+  const int words = a.ch / 4;
+  if (a.main_bits == 8 && (!a.res || a.res_bits == 8) && a.ch % 4 == 0 && (words <= 256 || words % 256 == 0)) {
+    const int bx = words <= 256 ? words : 256;
+    int by = 256 / bx; if (by < 1) by = 1;
+    dim3 block(bx, by), grid((words + bx - 1) / bx, 1);
+    long long gy = (a.pixels + by - 1) / by;
+    const long long cap = (long long)sm_count * 16 / grid.x + 1;
+    grid.y = (unsigned)(gy < cap ? gy : cap);
+    const int lo = a.relu ? (a.qmin > 0 ? a.qmin : 0) : a.qmin, hi = a.qmax;
+    const int v = (a.res ? 4 : 0) | (a.main_signed ? 2 : 0) | ((a.res && a.res_signed) ? 1 : 0);
+    switch (v) {
+      case 0: return launch_requant8<false, false, false>(a, grid, block, words, lo, hi, s);
+      case 2: return launch_requant8<false, true, false>(a, grid, block, words, lo, hi, s);
+      case 4: return launch_requant8<true, false, false>(a, grid, block, words, lo, hi, s);
+      case 5: return launch_requant8<true, false, true>(a, grid, block, words, lo, hi, s);
+      case 6: return launch_requant8<true, true, false>(a, grid, block, words, lo, hi, s);
+      default: return launch_requant8<true, true, true>(a, grid, block, words, lo, hi, s);
+    }
+  }
   const int groups = a.ch / 16;
   if (a.ch % 16 == 0 && groups <= 256) {
     const int ppb = 256 / groups;

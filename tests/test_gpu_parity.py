@@ -230,6 +230,31 @@ def test_residual_add(hq, main_bits, res_bits, out_bits, ch):
     assert np.array_equal(host(out, ref), ref)
 
 
+def test_residual_add_8bit_fast_kernel_every_shift(hq):
+    """8-bit operands take the 32-bit kernel; shifts from 1 to 62, signed and unsigned, both outputs."""
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(305)
+    ch, shape = 128, (2, 9, 7, 128)
+    for main_signed, res_signed, out_bits in ((0, 0, 8), (1, 1, 8), (0, 1, 4), (1, 0, 8)):
+        main = g.integers(-128, 128, size=shape, dtype=np.int64).astype(np.int8) if main_signed else \
+            g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8)
+        res = g.integers(-128, 128, size=shape, dtype=np.int64).astype(np.int8) if res_signed else \
+            g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8)
+        mb, rb = (g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32) for _ in range(2))
+        mc = (np.arange(ch) % 62 + 1).astype(np.int32)
+        rc = ((np.arange(ch) * 7) % 62 + 1).astype(np.int32)
+        qmin, qmax = (0, 15) if out_bits == 4 else (-128, 127)
+        out_signed = int(out_bits == 8)
+        ref = oracle().residual_add(main, 8, main_signed, mb, mc, res, 8, res_signed, rb, rc, ch, 0, qmin, qmax, out_bits, out_signed)
+        out = binding.alloc_out(*shape[:3], ch, out_bits, out_signed)
+        st = hq.residual_add(binding.to_device(main), 8, main_signed, binding.to_device(mb), binding.to_device(mc),
+                             binding.to_device(res), 8, res_signed, binding.to_device(rb), binding.to_device(rc),
+                             ch, 0, qmin, qmax, out, out_bits, out_signed)
+        assert st == binding.HQ_OK
+        hq.sync()
+        assert np.array_equal(host(out, ref), ref)
+
+
 @pytest.mark.parametrize("n,hw,ch,in_bits", [(4, 7, 64, 8), (2, 7, 2048, 8), (3, 5, 6, 8), (2, 4, 16, 32), (2, 3, 8, 4)])
 def test_avgpool_requant(hq, n, hw, ch, in_bits):
     from paper_2011_10680_b200 import binding
