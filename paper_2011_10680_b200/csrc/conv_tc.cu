@@ -19,12 +19,16 @@
 //               a plain tiled map when the conv is 1x1 / stride 1.  W tile = 128 output channels x BK
 //               bytes of the [cout][kh*kw*cin] weight matrix.  When a residual is fused, its
 //               [PT][128] tile of the stored 8-bit tensor is prefetched as well.
-//   warp 1      MMA issuer (one lane).  BK/32 instructions of shape 128 x PT x 32 per stage, two
-//               accumulator buffers in tensor memory so the epilogue of tile t overlaps tile t+1.
+//   warp 1      MMA issuer (one lane).  BK/32 instructions of shape 128 x PT x 32 per stage; two
+//               (PT = 256) or four (PT <= 128) accumulator buffers in tensor memory, so the MMAs of
+//               the next tiles run while the epilogue works on the current ones.
 //   warps 2-9   epilogue.  Warp (q, half) reads lanes 32q..32q+31 (tcgen05.ld 32x32b) of one half
 //               of the tile's pixel columns, applies the integer epilogue in registers and writes
 //               bytes to a private staging box that leaves through its own TMA store; no CTA-wide
-//               barrier per tile.
+//               barrier per tile.  The loop is software-pipelined: the accumulator buffer goes back
+//               to the MMA issuer as soon as its last chunk has been read, and the first chunk of
+//               the next tile is requested from tensor memory before the current tile's staging
+//               writes and store hand-over, whose latency it hides.
 // The CTA keeps one channel tile for its whole life (grid = multiple of the channel tiles).
 // Every wait on an mbarrier is bounded: after the budget the waiter records a code in the
 // handle's status word, raises a CTA-wide abort flag and every role leaves its loop, drains what
@@ -35,11 +39,16 @@
 
 #include "hq_internal.cuh"
 
+#ifndef HQ_EPI_WARPS
+#define HQ_EPI_WARPS 8
+#endif
+
 namespace {
 
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
-constexpr int kEpilogueWarps = 8;
+constexpr int kMaxAccBufs = 4;                                 // accumulator (and residual) buffers: 4 x 128 or 2 x 256 columns
+constexpr int kEpilogueWarps = HQ_EPI_WARPS;
 constexpr int kEpilogueThreads = kEpilogueWarps * 32;
 constexpr int kThreads = 64 + kEpilogueThreads;               // producer warp + MMA warp + epilogue warps
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;   // 2 s per wait
@@ -52,6 +61,8 @@ struct TcParams {
   int32_t k_blocks;      // kh * kw * cchunks
   int32_t pt;            // pixel tile = MMA N: 64, 128 or 256
   int32_t p_tiles, c_tiles, stages;
+  int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
+  int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
   int32_t x_tiled;       // 1: X is a dense [P][cin] matrix (1x1, stride 1, no padding) fetched by a tiled map
   int32_t x_tap16;       // 1: cin = 16: a K block is 8 filter taps, each an un-swizzled [pt][16 B] slab of the X tile
@@ -80,10 +91,10 @@ struct TcParams {
 struct SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
-  unsigned long long tfull[2];
-  unsigned long long tempty[2];
-  unsigned long long rfull[2];
-  unsigned long long rempty[2];
+  unsigned long long tfull[kMaxAccBufs];
+  unsigned long long tempty[kMaxAccBufs];
+  unsigned long long rfull[kMaxAccBufs];
+  unsigned long long rempty[kMaxAccBufs];
   unsigned long long drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -229,8 +240,14 @@ __device__ __forceinline__ unsigned ld_shared_u8(uint32_t addr) {
   asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ int sat_u8(int x) { int d; asm("cvt.sat.u8.s32 %0, %1;" : "=r"(d) : "r"(x)); return d; }
-__device__ __forceinline__ int sat_s8(int x) { int d; asm("cvt.sat.s8.s32 %0, %1;" : "=r"(d) : "r"(x)); return d; }
+// Saturating conversion to a byte.  The packing form of the convert (second source -> byte 0) is a single
+// integer-pipe instruction; the plain cvt.sat.u8.s32 measured at twice its issue cost.
+__device__ __forceinline__ int sat_u8(int x) {
+  int d; asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %1;" : "=r"(d) : "r"(0), "r"(x)); return d;
+}
+__device__ __forceinline__ int sat_s8(int x) {
+  int d; asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %1;" : "=r"(d) : "r"(0), "r"(x)); return d;
+}
 
 // Shared-memory matrix descriptor for a K-major operand tile whose rows are `bkb` bytes wide and
 // stored with the matching TMA swizzle (32/64/128 B): 8-row groups are bkb*8 bytes apart.
@@ -261,8 +278,10 @@ struct ChanConst {
 //   residual  y += (hi32((r << 24) * rb) + 2^(rc-9)) >> (rc-8)                      (needs 9 <= rc)
 // The residual form is exact: (r<<24)*rb >> 32 = floor(r*rb / 2^8), the rounding constant 2^(rc-1) is
 // a multiple of 2^8, and the dropped low 8 bits of r*rb cannot carry across a multiple of 2^(rc-8).
+// (A 64-bit multiply-add followed by a funnel shift measured no faster.)  `r` is the stored 8-bit
+// residual, already extended.  SMALL: some channel of the warp has c < 32.
 template <bool RES, bool RSIGNED, bool SMALL>
-__device__ __forceinline__ int requant_fast(int acc, unsigned rbyte, const ChanConst& k) {
+__device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) {
   const long long t1 = (long long)acc * (long long)k.b + k.r0;
   int s;
   if (!SMALL) {
@@ -279,7 +298,7 @@ __device__ __forceinline__ int requant_fast(int acc, unsigned rbyte, const ChanC
     s = max(min(s, 1 << 30), -(1 << 30));
   }
   if (RES) {
-    const unsigned top = rbyte << 24;
+    const unsigned top = (unsigned)r << 24;
     if (RSIGNED) s += (__mulhi((int)top, k.rb) + k.rh) >> k.rsh;
     else s += (int)((__umulhi(top, (unsigned)k.rb) + (unsigned)k.rh) >> k.rsh);
   }
@@ -295,85 +314,113 @@ struct EpiCtx {
 };
 
 // Lean tile loop for the common case: 8-bit output through the staging box, 32-bit fast arithmetic,
-// clamp by saturating convert or by min/max, optional 8-bit residual from the prefetched tile.  The
-// accumulator chunk of the next 32 pixels is requested from tensor memory before the current one is
-// processed, so the load's latency hides behind the arithmetic.
+// clamp by saturating convert or by min/max, optional 8-bit residual from the prefetched tile.
+// Software-pipelined across chunks and tiles: while one 32-pixel accumulator chunk is processed, the
+// next one (of this tile, or the first of the group's next tile) streams from tensor memory into the
+// other register set; the accumulator buffer is handed back as soon as its last chunk has been read,
+// the residual tile as soon as its last bytes have been used, both before the tile's store is issued.
 template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL>
-__device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e, const ChanConst& k) {
+__device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const ChanConst& k_in) {
+  // Private copies: the caller's objects live in local memory (their address is passed to the general
+  // loop), so every asm statement with a memory clobber would force their fields to be re-read.
+  const EpiCtx e = e_in;
+  const ChanConst k = k_in;
   const TcParams& p = *e.p;
   SharedCtl& ctl = *e.ctl;
   const int lane = e.lane, q = e.q, half = e.half, px_per_warp = e.px_per_warp;
-  const uint32_t my_stage = e.out_stage + (uint32_t)e.ew * (uint32_t)(kTileC * 32);
+  const uint32_t my_stage = e.out_stage + (uint32_t)e.ew * (uint32_t)(px_per_warp * 32);
   uint8_t* const my_stage_ptr = e.smem_raw + (my_stage - e.raw);
   const uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
-  const int nchunks = px_per_warp >> 5;
+  const int nchunks = px_per_warp >> 5;           // 2 or 4
+  const uint32_t bmask = (1u << p.lg_bufs) - 1u;
+  const int tile_step = e.p_step;
+  int p_tile = e.p_tile0;
+  if (p_tile >= p.p_tiles) return;
   uint32_t tcount = 0;
-  for (int p_tile = e.p_tile0; p_tile < p.p_tiles; p_tile += e.p_step, ++tcount) {
-    const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
+  uint32_t as = 0, aph = 0;
+  const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + half * px_per_warp;
+
+  auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
     uint32_t w = 1;
-    if (lane == 0) {
-      w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
-      if (RES && w) w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+    if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, w, 0) != 0;
+  };
+  auto chunk = [&](const int (&v)[32], const uint8_t* res_tile, int c) {
+    if (!e.warp_live) return;
+    int y[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int r = !RES ? 0 : RSIGNED ? (int)(signed char)res_tile[(c * 32 + j) * kTileC] : (int)res_tile[(c * 32 + j) * kTileC];
+      const int s = requant_fast<RES, RSIGNED, SMALL>(v[j], r, k);
+      y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
     }
-    w = __shfl_sync(0xffffffffu, w, 0);
-    if (!w) break;
-    tc_fence_after();                            // lane 0 observed the barriers; the shuffle ordered the warp
-    if (e.ew == 0 && lane == 0) HQ_TRACE(3, tcount);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)y[j];
+  };
+
+  int va[32], vb[32];
+  bool ok = wait_bar(&ctl.tfull[as], aph);
+  if (!ok) return;
+  tc_fence_after();
+  tmem_ld32_issue(t_warp + as * p.pt, va);
+  bool pending = true;                            // a tensor-memory load into va is in flight
+  while (true) {
+    if (lane == 0) HQ_TRACE(3, tcount * 8 + e.ew);
+    if (RES && !wait_bar(&ctl.rfull[as], aph)) break;
     const int p_base = p_tile * p.pt + half * px_per_warp;
     const uint8_t* const res_tile = res_stage_ptr + as * e.res_tile_bytes + (uint32_t)(half * px_per_warp) * kTileC + q * 32 + lane;
-    const uint32_t t_addr = e.tmem_base + ((uint32_t)(q * 32) << 16) + as * p.pt + half * px_per_warp;
+    const uint32_t t_addr = t_warp + as * p.pt;
+    const bool has_next = p_tile + tile_step < p.p_tiles;
+    const uint32_t nas = (tcount + 1u) & bmask, naph = ((tcount + 1u) >> p.lg_bufs) & 1u;
 
-    int va[32], vb[32];
-    tmem_ld32_issue(t_addr, va);
     for (int c = 0; c < nchunks; c += 2) {
       // ---- chunk c (registers va), while chunk c+1 streams into vb
       tmem_ld_wait();
-      if (c + 1 < nchunks) tmem_ld32_issue(t_addr + (c + 1) * 32, vb);
+      tmem_ld32_issue(t_addr + (c + 1) * 32, vb);
       if (c == 0) {                               // the previous tile's store must have read the staging box
         if (lane == 0) tma_store_wait_read0();
         __syncwarp();
       }
-      if (e.warp_live) {
-        int y[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const unsigned rbyte = RES ? (unsigned)res_tile[(c * 32 + j) * kTileC] : 0u;
-          const int s = requant_fast<RES, RSIGNED, SMALL>(va[j], rbyte, k);
-          y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)y[j];
+      chunk(va, res_tile, c);
+      // ---- chunk c+1 (registers vb), while the next chunk streams into va
+      tmem_ld_wait();
+      pending = false;
+      if (c + 2 < nchunks) {
+        tmem_ld32_issue(t_addr + (c + 2) * 32, va);
+        pending = true;
+      } else {
+        // every lane has read its last accumulator columns of this tile: hand the buffer back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[as]));
+        if (lane == 0) HQ_TRACE(6, tcount * 8 + e.ew);
       }
-      if (c + 1 < nchunks) {
-        // ---- chunk c+1 (registers vb), while chunk c+2 streams into va
-        tmem_ld_wait();
-        if (c + 2 < nchunks) tmem_ld32_issue(t_addr + (c + 2) * 32, va);
-        if (e.warp_live) {
-          int y[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const unsigned rbyte = RES ? (unsigned)res_tile[((c + 1) * 32 + j) * kTileC] : 0u;
-            const int s = requant_fast<RES, RSIGNED, SMALL>(vb[j], rbyte, k);
-            y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
-          }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) my_stage_ptr[((c + 1) * 32 + j) * 32 + lane] = (uint8_t)y[j];
-        }
-      }
+      chunk(vb, res_tile, c + 1);
+    }
+    if (RES) {                                    // every lane has used its last residual bytes of this tile
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl.rempty[as]));
+    }
+    // Only now wait for the group's next tile: its copies may be queued behind the buffers released above.
+    if (e.ew == 0 && lane == 0) HQ_TRACE(8, tcount);
+    if (has_next) {
+      ok = wait_bar(&ctl.tfull[nas], naph);
+      if (ok) { tc_fence_after(); tmem_ld32_issue(t_warp + nas * p.pt, va); pending = true; }
     }
     if (e.ew == 0 && lane == 0) HQ_TRACE(4, tcount);
-    tc_fence_before();
     fence_async_smem();                           // make this lane's box writes visible to the TMA engine
     __syncwarp();
     if (lane == 0) {
-      mbar_arrive(smem_u32(&ctl.tempty[as]));
-      if (RES) mbar_arrive(smem_u32(&ctl.rempty[as]));
       if (e.warp_live && p_base < p.P) {
         tma_store_2d(e.map_out, my_stage, e.c_tile * kTileC + q * 32, p_base);
         tma_store_commit();
       }
     }
+    if (e.ew == 0 && lane == 0) HQ_TRACE(7, tcount);
+    if (!has_next || !ok) break;
+    p_tile += tile_step; ++tcount; as = nas; aph = naph;
   }
+  if (pending) tmem_ld_wait();
   if (lane == 0) tma_store_wait_all();
 }
 
@@ -390,13 +437,14 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
   const bool ch_live = e.ch_live, warp_live = e.warp_live;
     // staging box of this warp: [px_per_warp pixels][32 channels] bytes (16 bytes per pixel at 4 bit)
     const int row_b = (p.out_bits == 4) ? 16 : 32;
-    const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(kTileC * 32);   // 128 rows x 32 bytes reserved per warp
+    const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(px_per_warp * 32);   // px_per_warp rows x 32 bytes reserved per warp
     // plain pointers to the same bytes: ordinary loads / stores that the compiler may schedule freely
     uint8_t* const my_stage_ptr = smem_raw + (my_stage - raw);
     const uint8_t* const res_stage_ptr = smem_raw + (res_stage - raw);
+    const uint32_t bmask = (1u << p.lg_bufs) - 1u;
     uint32_t tcount = 0;
     for (int p_tile = p_tile0; p_tile < p.p_tiles; p_tile += p_step, ++tcount) {
-      const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
+      const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
       uint32_t w = 1;
       if (lane == 0) {
         if (p.staged_out) tma_store_wait_read0();   // the previous store has read this warp's staging box
@@ -445,13 +493,13 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
           const int variant = (p.res ? 2 : 0) | (p.res_signed ? 1 : 0);
           if (variant == 2) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, false, true>(v[j], rb8[j], k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, false, true>(v[j], (int)rb8[j], k);
           } else if (variant == 3) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, true, true>(v[j], rb8[j], k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<true, true, true>(v[j], (int)(signed char)rb8[j], k);
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = requant_fast<false, false, true>(v[j], 0u, k);
+            for (int j = 0; j < 32; ++j) y[j] = requant_fast<false, false, true>(v[j], 0, k);
           }
           if (p.sat_pack) {
             if (p.out_signed) {
@@ -533,7 +581,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
-               const TcParams p) {
+               const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ SharedCtl ctl;
 
@@ -554,9 +602,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&ctl.full[s]), 1); mbar_init(smem_u32(&ctl.empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), kEpilogueWarps);
-      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), kEpilogueWarps);
+    for (int s = 0; s < (1 << p.lg_bufs); ++s) {
+      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), 4 * p.halves);
+      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), 4 * p.halves);
     }
     mbar_init(smem_u32(&ctl.drain), 1);
     ctl.abort_flag = 0;
@@ -574,6 +622,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       // No division or modulo in this loop: one thread runs it and every dependent instruction
       // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
+      const uint32_t bmask = (1u << p.lg_bufs) - 1u;
       bool ok = true;
       // (image, row, column) of the tile's first output pixel, advanced by a fixed step per tile
       const int ho = p.howo / p.wo;
@@ -585,7 +634,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
         const int p0 = p_tile * p.pt;
         if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
-          const uint32_t rbuf = tcount & 1u, rph = (tcount >> 1) & 1u;
+          const uint32_t rbuf = tcount & bmask, rph = (tcount >> p.lg_bufs) & 1u;
           if (!mbar_wait(smem_u32(&ctl.rempty[rbuf]), rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
           mbar_expect_tx(bar, res_tile_bytes);
@@ -629,11 +678,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
       if (p.staged_res) {
-        const uint32_t tiles_done = tcount < 2u ? tcount : 2u;
+        const uint32_t tiles_done = tcount < bmask + 1u ? tcount : bmask + 1u;
         for (uint32_t j = 0; j < tiles_done; ++j) {
           const uint32_t k = tcount - 1 - j;
           const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(smem_u32(&ctl.rfull[k & 1u]), (k >> 1) & 1u)) {
+          while (!mbar_try_wait(smem_u32(&ctl.rfull[k & bmask]), (k >> p.lg_bufs) & 1u)) {
             if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
           }
         }
@@ -646,6 +695,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const uint32_t idesc = (2u << 4) | (1u << 7) | ((uint32_t)(p.x_signed ? 1 : 0) << 10) |
                              ((uint32_t)(p.pt >> 3) << 17) | ((uint32_t)(kTileC >> 4) << 24);
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
+      const uint32_t bmask = (1u << p.lg_bufs) - 1u;
       bool ok = true;
       const uint64_t desc_hi = smem_desc(0, p.bkb);           // everything but the start address
       const int ksteps = p.bkb >> 5;
@@ -654,23 +704,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const uint64_t xdesc_hi = ((uint64_t)((p.pt * 16) >> 4) << 16) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
       const uint64_t bstep = p.x_tap16 ? (uint64_t)((2 * p.pt * 16) >> 4) : 2ull;   // two taps per instruction
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
-        const uint32_t as = tcount & 1u, aph = (tcount >> 1) & 1u;
+        const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
+        // The operands of the tile's first K block have usually landed long ago; looking at them first
+        // keeps that check off the path between the epilogue's hand-back and the first MMA.
+        if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         if (!mbar_wait(smem_u32(&ctl.tempty[as]), aph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         tc_fence_after();
+        HQ_TRACE(11, tcount);
         const uint32_t d_tmem = tmem_base + as * p.pt;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
-          tc_fence_after();
+          if (kb > 0 && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
           HQ_TRACE(1, it);
           const uint32_t w_addr = tiles + s * stage_bytes;
           uint64_t adesc = desc_hi | (uint64_t)((w_addr >> 4) & 0x3FFF);
           uint64_t bdesc = (p.x_tap16 ? xdesc_hi : desc_hi) | (uint64_t)(((w_addr + w_bytes) >> 4) & 0x3FFF);
           for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += bstep)     // 32 bytes of K per instruction
             mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+          HQ_TRACE(5, it);
+          // the accumulator's barrier first on the last K block: the epilogue is the one waiting
+          if (kb + 1 == p.k_blocks) mma_commit(smem_u32(&ctl.tfull[as]));
           mma_commit(smem_u32(&ctl.empty[s]));     // frees the stage when these MMAs have read it
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
-        if (ok) mma_commit(smem_u32(&ctl.tfull[as]));
         HQ_TRACE(2, tcount);
       }
       // Drain: all issued MMAs must have completed before tensor memory is freed.
@@ -685,7 +740,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read: channels 32q..32q+31
     const int ew = warp - 2;                      // 0..7
     const int half = ew >> 2;                     // which half of the tile's pixel columns this warp owns
-    const int px_per_warp = p.pt >> 1;
+    const int px_per_warp = p.pt / p.halves;      // 128 or 64 pixel columns
     const int ch = c_tile * kTileC + q * 32 + lane;          // this thread's output channel
     const bool ch_live = ch < p.C;
     const bool warp_live = (c_tile * kTileC + q * 32) < p.C; // warp-uniform
@@ -726,7 +781,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     e.warp = warp; e.lane = lane; e.q = q; e.ew = ew; e.half = half; e.px_per_warp = px_per_warp; e.ch = ch;
     e.c_tile = c_tile; e.p_tile0 = p_tile0; e.p_step = p_step; e.lo = lo; e.hi = hi;
     e.ch_live = ch_live; e.warp_live = warp_live;
-    if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
+    if (half >= p.halves) {
+      // the 64-pixel tile has one 64-column slice per lane quarter: this warp only took part in the vote above
+    } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
 #define HQ_FAST8(R, RS, S, OS) do { if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true>(e, k); \
@@ -857,19 +914,25 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.staged_out = (a.out_bits != 32 && out_row_bytes % 16 == 0) ? 1 : 0;
   p.staged_res = (p.staged_out && a.res && a.res_bits == 8 && a.cout % 16 == 0) ? 1 : 0;
   const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
-  // staging: 8 warps x 128 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 x [pt][128]
-  const int out_tile_bytes = p.staged_out ? kEpilogueWarps * kTileC * 32 : 0;
-  int stages = 0, stage_bytes = 0, res_tile_bytes = 0;
-  for (int cap = 256; cap >= 64; cap >>= 1) {          // largest pixel tile that leaves room for >= 3 stages
+  // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
+  int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
+  int cap0 = 256;
+#ifdef HQ_EXP_CAP
+  cap0 = HQ_EXP_CAP;
+#endif
+  for (int cap = cap0; cap >= 64; cap >>= 1) {         // largest pixel tile that leaves room for >= 3 stages
     p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
     stage_bytes = (kTileC + p.pt) * p.bkb;
+    p.halves = (kEpilogueWarps == 8 && p.pt >= 128) ? 2 : 1;
+    out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
+    p.lg_bufs = p.pt <= 128 ? 2 : 1;
     res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-    stages = (smem_budget - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
+    stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs)) / stage_bytes;
     if (stages >= 3 || p.pt == 64) break;
   }
   p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
   p.x_signed = a.in_signed;
-  p.tmem_cols = (uint32_t)(2 * p.pt);
+  p.tmem_cols = (uint32_t)(p.pt << p.lg_bufs);          // 512 columns, or 256 for the smallest tile
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return HQ_ERR_UNSUPPORTED;
   p.stages = stages;
@@ -922,12 +985,12 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   }
   if (!encode_rows_map(&map_w, a.wgt, a.cout, (long long)a.kh * a.kw * a.cin, p.bkb, kTileC, swz)) return HQ_ERR_CUDA;
   map_out = map_w; map_res = map_w;                    // valid placeholders when a path is not staged
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / 2,
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / p.halves,
                                        CU_TENSOR_MAP_SWIZZLE_NONE)) return HQ_ERR_CUDA;
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + 2 * res_tile_bytes + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_bufs) + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int grid = (int)(total_tiles <= h->sm_count ? total_tiles : (h->sm_count / p.c_tiles) * p.c_tiles);
