@@ -39,18 +39,18 @@
 
 #include "hq_internal.cuh"
 
-#ifndef HQ_EPI_WARPS
-#define HQ_EPI_WARPS 8
-#endif
-
 namespace {
 
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccBufs = 4;                                 // accumulator (and residual) buffers: 4 x 128 or 2 x 256 columns
-constexpr int kEpilogueWarps = HQ_EPI_WARPS;
-constexpr int kEpilogueThreads = kEpilogueWarps * 32;
-constexpr int kThreads = 64 + kEpilogueThreads;               // producer warp + MMA warp + epilogue warps
+// Two launch shapes of the same kernel:
+//   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 212 KiB of shared memory;
+//   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
+//         reduction are bound by the latency of the hand-over chain between the MMA issuer and the epilogue
+//         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
+constexpr int kSoloEpilogueWarps = 8;
+constexpr int kPairEpilogueWarps = 4;
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;   // 2 s per wait
 
 struct TcParams {
@@ -61,6 +61,7 @@ struct TcParams {
   int32_t k_blocks;      // kh * kw * cchunks
   int32_t pt;            // pixel tile = MMA N: 64, 128 or 256
   int32_t p_tiles, c_tiles, stages;
+  int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
@@ -166,6 +167,7 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void tma_store_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+template <int EPI_THREADS>
 __device__ __forceinline__ uint32_t epi_bar_and(uint32_t v) {
   uint32_t r;
   asm volatile(
@@ -173,7 +175,7 @@ __device__ __forceinline__ uint32_t epi_bar_and(uint32_t v) {
       "setp.ne.u32 q, %1, 0;\n\t"
       "bar.red.and.pred p, 1, %2, q;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r) : "r"(v), "n"(kEpilogueThreads) : "memory");
+      : "=r"(r) : "r"(v), "n"(EPI_THREADS) : "memory");
   return r;
 }
 
@@ -309,7 +311,7 @@ __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) 
 struct EpiCtx {
   const TcParams* p; SharedCtl* ctl; const CUtensorMap* map_out;
   uint8_t* smem_raw; uint32_t raw, out_stage, res_stage, res_tile_bytes, tmem_base;
-  int warp, lane, q, ew, half, px_per_warp, ch, c_tile, p_tile0, p_step, lo, hi;
+  int warp, lane, q, cq, ew, half, col0, px_per_warp, ch, c_tile, p_tile0, p_step, lo, hi;
   bool ch_live, warp_live;
 };
 
@@ -327,7 +329,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   const ChanConst k = k_in;
   const TcParams& p = *e.p;
   SharedCtl& ctl = *e.ctl;
-  const int lane = e.lane, q = e.q, half = e.half, px_per_warp = e.px_per_warp;
+  const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
   const uint32_t my_stage = e.out_stage + (uint32_t)e.ew * (uint32_t)(px_per_warp * 32);
   uint8_t* const my_stage_ptr = e.smem_raw + (my_stage - e.raw);
   const uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
@@ -338,7 +340,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   if (p_tile >= p.p_tiles) return;
   uint32_t tcount = 0;
   uint32_t as = 0, aph = 0;
-  const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + half * px_per_warp;
+  const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + col0;
 
   auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
     uint32_t w = 1;
@@ -367,8 +369,8 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   while (true) {
     if (lane == 0) HQ_TRACE(3, tcount * 8 + e.ew);
     if (RES && !wait_bar(&ctl.rfull[as], aph)) break;
-    const int p_base = p_tile * p.pt + half * px_per_warp;
-    const uint8_t* const res_tile = res_stage_ptr + as * e.res_tile_bytes + (uint32_t)(half * px_per_warp) * kTileC + q * 32 + lane;
+    const int p_base = p_tile * p.pt + col0;
+    const uint8_t* const res_tile = res_stage_ptr + as * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
     const uint32_t t_addr = t_warp + as * p.pt;
     const bool has_next = p_tile + tile_step < p.p_tiles;
     const uint32_t nas = (tcount + 1u) & bmask, naph = ((tcount + 1u) >> p.lg_bufs) & 1u;
@@ -412,7 +414,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     __syncwarp();
     if (lane == 0) {
       if (e.warp_live && p_base < p.P) {
-        tma_store_2d(e.map_out, my_stage, e.c_tile * kTileC + q * 32, p_base);
+        tma_store_2d(e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_base);
         tma_store_commit();
       }
     }
@@ -432,7 +434,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
   uint8_t* const smem_raw = e.smem_raw;
   const uint32_t raw = e.raw, out_stage = e.out_stage, res_stage = e.res_stage, res_tile_bytes = e.res_tile_bytes;
   const uint32_t tmem_base = e.tmem_base;
-  const int lane = e.lane, q = e.q, ew = e.ew, half = e.half, px_per_warp = e.px_per_warp, ch = e.ch;
+  const int lane = e.lane, q = e.q, cq = e.cq, ew = e.ew, col0 = e.col0, px_per_warp = e.px_per_warp, ch = e.ch;
   const int c_tile = e.c_tile, p_tile0 = e.p_tile0, p_step = e.p_step, lo = e.lo, hi = e.hi;
   const bool ch_live = e.ch_live, warp_live = e.warp_live;
     // staging box of this warp: [px_per_warp pixels][32 channels] bytes (16 bytes per pixel at 4 bit)
@@ -456,13 +458,13 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       if (!w) break;
       tc_fence_after();                            // lane 0 observed the barriers; the shuffle ordered the warp
       if (ew == 0 && lane == 0) HQ_TRACE(3, tcount);
-      const int p_base = p_tile * p.pt + half * px_per_warp;            // first pixel of this warp's columns
-      const uint8_t* const res_tile = res_stage_ptr + as * res_tile_bytes + (uint32_t)(half * px_per_warp) * kTileC + q * 32 + lane;
+      const int p_base = p_tile * p.pt + col0;                          // first pixel of this warp's columns
+      const uint8_t* const res_tile = res_stage_ptr + as * res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
 
       for (int cc0 = 0; cc0 < px_per_warp; cc0 += 32) {
         int v[32];
         if (ew == 0 && lane == 0) HQ_TRACE(8, tcount * 4 + (cc0 >> 5));
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * p.pt + half * px_per_warp + cc0, v);
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * p.pt + col0 + cc0, v);
         if (ew == 0 && lane == 0) HQ_TRACE(9, tcount * 4 + (cc0 >> 5));
         if (!warp_live) continue;
         const int px0 = p_base + cc0;                                     // global pixel of v[0]
@@ -568,7 +570,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
         mbar_arrive(smem_u32(&ctl.tempty[as]));
         if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
         if (p.staged_out && warp_live && p_base < p.P) {
-          tma_store_2d(&map_out, my_stage, ((c_tile * kTileC + q * 32) * p.out_bits) >> 3, p_base);
+          tma_store_2d(&map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_base);
           tma_store_commit();
         }
       }
@@ -578,7 +580,8 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 }
 
 // ---------------------------------------------------------------- the kernel -----------------
-__global__ void __launch_bounds__(kThreads, 1)
+template <int EPI_WARPS, int MIN_CTAS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
                const __grid_constant__ TcParams p) {
@@ -662,7 +665,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           } else {
             tma_load_im2col(w_dst + w_bytes, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
           }
-          tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
+          if (p.fold) {          // 64-row box, twice: accumulator lanes 64-127 repeat lanes 0-63
+            tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, 0);
+            tma_load_2d(w_dst + 64 * p.bkb, &map_w, bar, kb * p.bkb, 0);
+          } else {
+            tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
+          }
           if (!p.x_tap16 && ++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
@@ -739,11 +747,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // ------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read: channels 32q..32q+31
     const int ew = warp - 2;                      // 0..7
-    const int half = ew >> 2;                     // which half of the tile's pixel columns this warp owns
-    const int px_per_warp = p.pt / p.halves;      // 128 or 64 pixel columns
-    const int ch = c_tile * kTileC + q * 32 + lane;          // this thread's output channel
+    const int half = ew >> 2;                     // which half of its lane quarter's pixel columns this warp owns
+    // Channel tiles of at most 64 channels are folded: the weight rows are loaded twice, so accumulator
+    // lanes 64-127 repeat lanes 0-63, and lane quarters 2-3 take the second half of the pixel columns
+    // of channels 0-63 instead of idling on channels that do not exist.
+    const int cq = p.fold ? (q & 1) : q;          // which 32 channels of the tile
+    const int slices = p.halves << p.fold;        // pixel-column slices per channel quarter
+    const int px_per_warp = p.pt / slices;        // 128 or 64 pixel columns
+    const int col0 = ((p.fold ? (q >> 1) * p.halves : 0) + half) * px_per_warp;
+    const int ch = c_tile * kTileC + cq * 32 + lane;         // this thread's output channel
     const bool ch_live = ch < p.C;
-    const bool warp_live = (c_tile * kTileC + q * 32) < p.C; // warp-uniform
+    const bool warp_live = (c_tile * kTileC + cq * 32) < p.C; // warp-uniform
     const int lo = p.relu ? (p.qmin > 0 ? p.qmin : 0) : p.qmin, hi = p.qmax;
 
     // per-channel constants, once per kernel
@@ -763,7 +777,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         k.rr0 = 1LL << (rcc - 1);
       }
     }
-    fast = epi_bar_and(fast);                    // every live channel of the CTA allows 32-bit intermediates
+    fast = epi_bar_and<32 * EPI_WARPS>(fast);                    // every live channel of the CTA allows 32-bit intermediates
     const bool warp_small = __any_sync(0xffffffffu, k.sh < 32) != 0;     // some channel of this warp has c < 32
     if (fast) {
       k.sh1 = k.sh < 32 ? k.sh : 32;
@@ -778,7 +792,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     EpiCtx e;
     e.p = &p; e.ctl = &ctl; e.map_out = &map_out; e.smem_raw = smem_raw; e.raw = raw; e.out_stage = out_stage;
     e.res_stage = res_stage; e.res_tile_bytes = res_tile_bytes; e.tmem_base = tmem_base;
-    e.warp = warp; e.lane = lane; e.q = q; e.ew = ew; e.half = half; e.px_per_warp = px_per_warp; e.ch = ch;
+    e.warp = warp; e.lane = lane; e.q = q; e.cq = cq; e.ew = ew; e.half = half; e.col0 = col0; e.px_per_warp = px_per_warp; e.ch = ch;
     e.c_tile = c_tile; e.p_tile0 = p_tile0; e.p_step = p_step; e.lo = lo; e.hi = hi;
     e.ch_live = ch_live; e.warp_live = warp_live;
     if (half >= p.halves) {
@@ -879,7 +893,10 @@ int pick_pt(long long pixels, int c_tiles, int sm_count, int cap) {
 // tensor-map encoders and the kernel's dynamic shared-memory limit.
 bool hq_conv_tc_init() {
   if (!load_driver_entry_points()) return false;
-  return cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess;
+  return cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              214 * 1024) == cudaSuccess &&
+         cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              112 * 1024) == cudaSuccess;
 }
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
@@ -913,22 +930,45 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const long long out_row_bytes = (long long)a.cout * a.out_bits / 8;
   p.staged_out = (a.out_bits != 32 && out_row_bytes % 16 == 0) ? 1 : 0;
   p.staged_res = (p.staged_out && a.res && a.res_bits == 8 && a.cout % 16 == 0) ? 1 : 0;
-  const int smem_budget = 212 * 1024;                  // dynamic bytes after the 1024-byte alignment slack
-  // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
-  int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
-  int cap0 = 256;
-#ifdef HQ_EXP_CAP
-  cap0 = HQ_EXP_CAP;
+  // Launch shape: pair (two CTAs per SM) for short reductions when the tile pipeline fits half an SM.
+  const long long k_total = (long long)a.kh * a.kw * a.cin;
+  // (measured: the pair shape wins on the fused-residual expansions, whose epilogue is the longest per tile,
+  // and loses where a tile carries little epilogue work, e.g. 64 output channels)
+  bool pair = !a.tap16 && k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
+#ifdef HQ_EXP_PAIR
+  pair = !a.tap16 && (HQ_EXP_PAIR != 0);
 #endif
-  for (int cap = cap0; cap >= 64; cap >>= 1) {         // largest pixel tile that leaves room for >= 3 stages
-    p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
+  int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
+  if (pair) {
+    // 128-pixel tiles, two accumulator buffers (256 columns), K blocks of at most 64 bytes
+    if (p.bkb > 64) { p.bkb = 64; p.cchunks = a.cin / p.bkb; p.k_blocks = a.kh * a.kw * p.cchunks; }
+    p.pt = pick_pt(P, p.c_tiles, 2 * h->sm_count, 128);
     stage_bytes = (kTileC + p.pt) * p.bkb;
-    p.halves = (kEpilogueWarps == 8 && p.pt >= 128) ? 2 : 1;
-    out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
-    p.lg_bufs = p.pt <= 128 ? 2 : 1;
+    p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
+    p.halves = 1;
+    p.lg_bufs = 1;
+    out_tile_bytes = p.staged_out ? kPairEpilogueWarps * p.pt * 32 : 0;
     res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-    stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs)) / stage_bytes;
-    if (stages >= 3 || p.pt == 64) break;
+    stages = (110 * 1024 - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
+    if (stages < 3 || p.pt < 128) pair = false;
+  }
+  if (!pair) {
+    p.bkb = a.tap16 ? 128 : (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
+    p.cchunks = a.tap16 ? 1 : a.cin / p.bkb;
+    p.k_blocks = a.tap16 ? (a.kh * a.kw) / 8 : a.kh * a.kw * p.cchunks;
+    const int smem_budget = 212 * 1024;                // dynamic bytes after the 1024-byte alignment slack
+    // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
+    for (int cap = 256; cap >= 64; cap >>= 1) {        // largest pixel tile that leaves room for >= 3 stages
+      p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
+      stage_bytes = (kTileC + p.pt) * p.bkb;
+      p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
+      p.halves = p.pt >= (p.fold ? 256 : 128) ? 2 : 1;
+      out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
+      p.lg_bufs = p.pt <= 128 ? 2 : 1;
+      res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
+      stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs)) / stage_bytes;
+      if (stages >= 3 || p.pt == 64) break;
+    }
   }
   p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
   p.x_signed = a.in_signed;
@@ -983,9 +1023,9 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     if (g_driver_version <= 13010 && (long long)a.n * a.h * a.w * a.cin < 131072)
       reinterpret_cast<uint64_t*>(&map_x)[1] &= ~(1ull << 21);
   }
-  if (!encode_rows_map(&map_w, a.wgt, a.cout, (long long)a.kh * a.kw * a.cin, p.bkb, kTileC, swz)) return HQ_ERR_CUDA;
+  if (!encode_rows_map(&map_w, a.wgt, a.cout, (long long)a.kh * a.kw * a.cin, p.bkb, p.fold ? 64 : kTileC, swz)) return HQ_ERR_CUDA;
   map_out = map_w; map_res = map_w;                    // valid placeholders when a path is not staged
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / p.halves,
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / (p.halves << p.fold),
                                        CU_TENSOR_MAP_SWIZZLE_NONE)) return HQ_ERR_CUDA;
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;
@@ -993,10 +1033,15 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_bufs) + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
-  const int grid = (int)(total_tiles <= h->sm_count ? total_tiles : (h->sm_count / p.c_tiles) * p.c_tiles);
-  // keep one CTA per SM (tensor-memory allocation assumes it): never request less than 120 KiB
-  const size_t smem = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
-  conv_tc_kernel<<<grid, kThreads, smem, stream>>>(map_x, map_w, map_out, map_res, p);
+  const int slots = pair ? 2 * h->sm_count : h->sm_count;
+  const int grid = (int)(total_tiles <= slots ? total_tiles : (slots / p.c_tiles) * p.c_tiles);
+  if (pair) {
+    conv_tc_kernel<kPairEpilogueWarps, 2><<<grid, 64 + 32 * kPairEpilogueWarps, dyn_smem, stream>>>(map_x, map_w, map_out, map_res, p);
+  } else {
+    // one CTA per SM (it may allocate all 512 tensor-memory columns): never request less than 120 KiB
+    const size_t smem = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    conv_tc_kernel<kSoloEpilogueWarps, 1><<<grid, 64 + 32 * kSoloEpilogueWarps, smem, stream>>>(map_x, map_w, map_out, map_res, p);
+  }
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
