@@ -66,7 +66,6 @@ struct TcParams {
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
   int32_t x_tiled;       // 1: X is a dense [P][cin] matrix (1x1, stride 1, no padding) fetched by a tiled map
-  int32_t x_tap16;       // 1: cin = 16: a K block is 8 filter taps, each an un-swizzled [pt][16 B] slab of the X tile
   uint32_t tmem_cols;
   // epilogue
   int32_t staged_out;    // 1: bytes leave through per-warp staging boxes and TMA stores
@@ -234,14 +233,6 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, int (&v)[32]) {
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void st_shared_u8(uint32_t addr, int v) {
-  asm volatile("st.shared.u8 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned ld_shared_u8(uint32_t addr) {
-  unsigned v;
-  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
 // Saturating conversion to a byte.  The packing form of the convert (second source -> byte 0) is a single
 // integer-pipe instruction; the plain cvt.sat.u8.s32 measured at twice its issue cost.
 __device__ __forceinline__ int sat_u8(int x) {
@@ -654,13 +645,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const uint32_t bar = smem_u32(&ctl.full[s]);
           const uint32_t w_dst = tiles + s * stage_bytes;
           mbar_expect_tx(bar, stage_bytes);
-          if (p.x_tap16) {
-            // eight taps of 16 bytes: slab t of the X tile holds tap t for all pt pixels
-            for (int t = 0; t < 8; ++t) {
-              tma_load_im2col(w_dst + w_bytes + t * (p.pt * 16), &map_x, bar, 0, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
-              if (++tap_s == p.kw) { tap_s = 0; ++tap_r; }
-            }
-          } else if (p.x_tiled) {
+          if (p.x_tiled) {
             tma_load_2d(w_dst + w_bytes, &map_x, bar, chunk * p.bkb, p0);
           } else {
             tma_load_im2col(w_dst + w_bytes, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
@@ -671,7 +656,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           } else {
             tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
           }
-          if (!p.x_tap16 && ++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
+          if (++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
         }
       }
@@ -707,10 +692,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       const uint64_t desc_hi = smem_desc(0, p.bkb);           // everything but the start address
       const int ksteps = p.bkb >> 5;
-      // un-swizzled X tile (16-byte taps): 8 pixels x 16 B form a 128-byte core matrix; the next 8 pixels are 128 B
-      // further (stride offset), the next 16 bytes of K sit one slab = pt*16 B further (leading offset)
-      const uint64_t xdesc_hi = ((uint64_t)((p.pt * 16) >> 4) << 16) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
-      const uint64_t bstep = p.x_tap16 ? (uint64_t)((2 * p.pt * 16) >> 4) : 2ull;   // two taps per instruction
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
         const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
         // The operands of the tile's first K block have usually landed long ago; looking at them first
@@ -725,8 +706,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           HQ_TRACE(1, it);
           const uint32_t w_addr = tiles + s * stage_bytes;
           uint64_t adesc = desc_hi | (uint64_t)((w_addr >> 4) & 0x3FFF);
-          uint64_t bdesc = (p.x_tap16 ? xdesc_hi : desc_hi) | (uint64_t)(((w_addr + w_bytes) >> 4) & 0x3FFF);
-          for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += bstep)     // 32 bytes of K per instruction
+          uint64_t bdesc = desc_hi | (uint64_t)(((w_addr + w_bytes) >> 4) & 0x3FFF);
+          for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
             mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
           HQ_TRACE(5, it);
           // the accumulator's barrier first on the last K block: the epilogue is the one waiting
@@ -901,8 +882,7 @@ bool hq_conv_tc_init() {
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
   if (a.in_bits != 8) return false;
-  if (a.tap16) { if (a.cin != 16 || (a.kh * a.kw) % 8 != 0) return false; }
-  else if (a.cin % 32 != 0) return false;
+  if (a.cin % 32 != 0) return false;
   if (a.kh > 255 || a.kw > 255 || a.pad > 127 || a.stride > 8) return false;
   if ((long long)a.n * a.ho * a.wo >= (1ll << 31) - 256) return false;
   if ((long long)a.kh * a.kw * a.cin >= (1ll << 24)) return false;
@@ -920,10 +900,9 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   TcParams p{};
   p.P = (int32_t)P; p.C = a.cout; p.howo = a.ho * a.wo; p.wo = a.wo;
   p.stride = a.stride; p.pad = a.pad; p.kw = a.kw;
-  p.x_tap16 = a.tap16 ? 1 : 0;
-  p.bkb = a.tap16 ? 128 : (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
-  p.cchunks = a.tap16 ? 1 : a.cin / p.bkb;
-  p.k_blocks = a.tap16 ? (a.kh * a.kw) / 8 : a.kh * a.kw * p.cchunks;
+  p.bkb = (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
+  p.cchunks = a.cin / p.bkb;
+  p.k_blocks = a.kh * a.kw * p.cchunks;
   p.c_tiles = (a.cout + kTileC - 1) / kTileC;
   if (p.c_tiles > h->sm_count) return HQ_ERR_UNSUPPORTED;
   // outputs and 8-bit residuals whose rows are 16-byte multiples travel through TMA
@@ -934,9 +913,9 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const long long k_total = (long long)a.kh * a.kw * a.cin;
   // (measured: the pair shape wins on the fused-residual expansions, whose epilogue is the longest per tile,
   // and loses where a tile carries little epilogue work, e.g. 64 output channels)
-  bool pair = !a.tap16 && k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
+  bool pair = k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
 #ifdef HQ_EXP_PAIR
-  pair = !a.tap16 && (HQ_EXP_PAIR != 0);
+  pair = (HQ_EXP_PAIR != 0);
 #endif
   int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
   if (pair) {
@@ -953,9 +932,9 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     if (stages < 3 || p.pt < 128) pair = false;
   }
   if (!pair) {
-    p.bkb = a.tap16 ? 128 : (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
-    p.cchunks = a.tap16 ? 1 : a.cin / p.bkb;
-    p.k_blocks = a.tap16 ? (a.kh * a.kw) / 8 : a.kh * a.kw * p.cchunks;
+    p.bkb = (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
+    p.cchunks = a.cin / p.bkb;
+    p.k_blocks = a.kh * a.kw * p.cchunks;
     const int smem_budget = 212 * 1024;                // dynamic bytes after the 1024-byte alignment slack
     // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
     for (int cap = 256; cap >= 64; cap >>= 1) {        // largest pixel tile that leaves room for >= 3 stages
@@ -1000,21 +979,23 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
 
   const CUtensorMapSwizzle swz = swizzle_for(p.bkb);
   alignas(64) CUtensorMap map_x, map_w, map_out, map_res;
-  p.x_tiled = (!a.tap16 && a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0) ? 1 : 0;
+  p.x_tiled = (!a.pitch_w && a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0) ? 1 : 0;
   if (p.x_tiled) {
     if (!encode_rows_map(&map_x, a.in, P, a.cin, p.bkb, p.pt, swz)) return HQ_ERR_CUDA;
   } else {
     // activations: (C, W, H, N) with byte strides; base pixels range over
     // [-pad, W + pad - (kw-1)) so that the hardware's pixel walk equals the output raster
     const cuuint64_t dims[4] = {(cuuint64_t)a.cin, (cuuint64_t)a.w, (cuuint64_t)a.h, (cuuint64_t)a.n};
-    const cuuint64_t strides[3] = {(cuuint64_t)a.cin, (cuuint64_t)a.cin * a.w, (cuuint64_t)a.cin * a.w * a.h};
+    const cuuint64_t strides[3] = {(cuuint64_t)(a.pitch_w ? a.pitch_w : a.cin),
+                                   (cuuint64_t)(a.pitch_h ? a.pitch_h : (long long)a.cin * a.w),
+                                   (cuuint64_t)(a.pitch_n ? a.pitch_n : (long long)a.cin * a.w * a.h)};
     const int lower[2] = {-a.pad, -a.pad};
     const int pad_after = a.pad + a.pad_after_delta;
     const int upper[2] = {pad_after - (a.kw - 1), pad_after - (a.kh - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)a.stride, (cuuint32_t)a.stride, 1};
     const CUresult r = g_encode_im2col(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.in), dims, strides,
-                                       lower, upper, (cuuint32_t)(a.tap16 ? 16 : p.bkb), (cuuint32_t)p.pt, estr,
-                                       CU_TENSOR_MAP_INTERLEAVE_NONE, a.tap16 ? CU_TENSOR_MAP_SWIZZLE_NONE : swz,
+                                       lower, upper, (cuuint32_t)p.bkb, (cuuint32_t)p.pt, estr,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return HQ_ERR_CUDA;

@@ -57,8 +57,10 @@ struct ConvArgs {
   int32_t relu, qmin, qmax;
   void* out; int32_t ho, wo, out_bits, out_signed;
   // internal lowerings only (zero for calls that come from the ABI):
-  int32_t pad_after_delta;   // padding after the last row/column minus `pad` (space-to-depth first layer: -1)
-  int32_t tap16;             // 1: cin == 16 and every filter tap is one 16-byte K chunk (un-swizzled X tiles)
+  int32_t pad_after_delta;   // padding after the last row/column minus `pad`
+  // byte pitches of the activation tensor along W, H and N when it is not dense (0: dense NHWC).  A W pitch
+  // below cin bytes makes neighbouring "pixels" overlap: a pixel is then a window of adjacent stored pixels.
+  long long pitch_w, pitch_h, pitch_n;
 };
 
 struct EltArgs {

@@ -124,21 +124,24 @@ namespace {
 
 __global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned char* __restrict__ in, int n, int h, int w,
                                                              uint4* __restrict__ out) {
-  const int h2 = h >> 1, w2 = w >> 1;
-  const long long total = (long long)n * h2 * w2;
+  // output: [n][h/2 + 3][w/2 + 3] pixels of 16 bytes, the image surrounded by its zero padding (2 before, 1 after)
+  const int h2 = h >> 1, w2 = w >> 1, hp = h2 + 3, wp = w2 + 3;
+  const long long total = (long long)n * hp * wp;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    const int x = (int)(i % w2);
-    long long t = i / w2;
-    const int y = (int)(t % h2);
-    const int img = (int)(t / h2);
+    const int x = (int)(i % wp) - 2;
+    long long t = i / wp;
+    const int y = (int)(t % hp) - 2;
+    const int img = (int)(t / hp);
     unsigned word[4] = {0u, 0u, 0u, 0u};
+    if (x >= 0 && x < w2 && y >= 0 && y < h2) {
 #pragma unroll
-    for (int dy = 0; dy < 2; ++dy) {
-      const unsigned char* src = in + (((long long)img * h + 2 * y + dy) * w + 2 * x) * 3;   // 6 contiguous bytes
+      for (int dy = 0; dy < 2; ++dy) {
+        const unsigned char* src = in + (((long long)img * h + 2 * y + dy) * w + 2 * x) * 3;   // 6 contiguous bytes
 #pragma unroll
-      for (int b = 0; b < 6; ++b) {
-        const int k = dy * 6 + b;
-        word[k >> 2] |= (unsigned)__ldg(src + b) << (8 * (k & 3));
+        for (int b = 0; b < 6; ++b) {
+          const int k = dy * 6 + b;
+          word[k >> 2] |= (unsigned)__ldg(src + b) << (8 * (k & 3));
+        }
       }
     }
     out[i] = make_uint4(word[0], word[1], word[2], word[3]);
@@ -161,23 +164,35 @@ __global__ void s2d_weights_kernel(const signed char* __restrict__ w, int cout, 
 
 }  // namespace
 
+namespace {
+// The 4x4 / stride-1 convolution over the padded space-to-depth image, described to the tensor-core kernel as a
+// 4x1 convolution over 64-byte "pixels": the four taps of a filter row are 64 contiguous bytes of the image,
+// so a pixel is a window of four stored pixels and neighbouring windows overlap (W pitch 16 bytes < 64).
+ConvArgs s2d_conv_args(const ConvArgs& a, const void* img, const void* wts) {
+  ConvArgs t = a;
+  const int h2 = a.h / 2, w2 = a.w / 2, hp = h2 + 3, wp = w2 + 3;
+  t.in = img; t.wgt = wts;
+  t.h = hp; t.w = w2; t.cin = 64; t.kh = 4; t.kw = 1; t.stride = 1; t.pad = 0; t.pad_after_delta = 0;
+  t.pitch_w = 16; t.pitch_h = (long long)wp * 16; t.pitch_n = (long long)hp * wp * 16;
+  return t;
+}
+}  // namespace
+
 bool hq_conv_s2d_applies(const ConvArgs& a) {
   if (a.in_bits != 8 || a.cin != 3 || a.kh != 7 || a.kw != 7 || a.stride != 2 || a.pad != 3) return false;
-  if ((a.h & 1) || (a.w & 1) || a.tap16) return false;
-  ConvArgs t = a;
-  t.h = a.h / 2; t.w = a.w / 2; t.cin = 16; t.kh = t.kw = 4; t.stride = 1; t.pad = 2; t.pad_after_delta = -1; t.tap16 = 1;
-  return hq_conv_tc_supported(t);
+  if ((a.h & 1) || (a.w & 1) || a.pitch_w) return false;
+  return hq_conv_tc_supported(s2d_conv_args(a, a.in, a.wgt));
 }
 
 size_t hq_conv_s2d_bytes(const ConvArgs& a) {
-  const long long img = (long long)a.n * (a.h / 2) * (a.w / 2) * 16, wts = (long long)a.cout * 256;
+  const long long img = (long long)a.n * (a.h / 2 + 3) * (a.w / 2 + 3) * 16, wts = (long long)a.cout * 256;
   return (size_t)(((img + 255) / 256 + (wts + 255) / 256) * 256);
 }
 
 // `scratch` must hold hq_conv_s2d_bytes(a) bytes, 256-byte aligned.
 hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s) {
-  const long long px = (long long)a.n * (a.h / 2) * (a.w / 2);
-  if (px == 0) return HQ_OK;
+  const long long px = (long long)a.n * (a.h / 2 + 3) * (a.w / 2 + 3);
+  if (a.n == 0) return HQ_OK;
   unsigned char* img = (unsigned char*)scratch;
   signed char* wts = (signed char*)(img + (px * 16 + 255) / 256 * 256);
   s2d_weights_kernel<<<(a.cout * 256 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, wts);
@@ -186,10 +201,7 @@ hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cud
   const long long cap = (long long)h->sm_count * 32;
   space_to_depth_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, (uint4*)img);
   if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
-  ConvArgs t = a;
-  t.in = img; t.wgt = wts; t.h = a.h / 2; t.w = a.w / 2; t.cin = 16; t.kh = t.kw = 4; t.stride = 1; t.pad = 2;
-  t.pad_after_delta = -1; t.tap16 = 1;
-  return hq_launch_conv_tc(h, t, s);
+  return hq_launch_conv_tc(h, s2d_conv_args(a, img, wts), s);
 }
 
 // ------------------------------------------------------------------------------------------------
