@@ -34,7 +34,7 @@ inline long long tensor_bytes(int n, int h, int w, int c, int bits) {
 // `scratch` / `scratch_bytes`: buffer for the lowered first-layer path owned by the caller (a
 // network); NULL means use (and if needed grow) the handle's own buffer.
 hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream,
-                      void* scratch = nullptr, size_t scratch_bytes = 0) {
+                      void* scratch = nullptr, size_t scratch_bytes = 0, const void* res_narrow = nullptr) {
   if (!h || !d) return HQ_ERR_INVALID_ARG;
   hq_status st = check_tensor(in, true, true, false);
   if (st != HQ_OK) return st;
@@ -67,6 +67,7 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   if (d->residual && out->bits != 32) {
     a.res = d->residual->data; a.res_bits = d->residual->bits; a.res_signed = d->residual->is_signed;
     a.rb = d->res_rescale.b; a.rc = d->res_rescale.c;
+    a.res_narrow = res_narrow;
   }
   a.relu = d->relu; a.qmin = d->qmin; a.qmax = d->qmax;
   a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
@@ -117,6 +118,7 @@ struct hq_network {
   std::vector<long long> bytes;
   int32_t batch, image_h, image_w, image_c, image_signed;
   int32_t launches;
+  std::vector<void*> res_narrow;     // per conv layer with a fused 8-bit residual: its narrow residual pairs (owned)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
@@ -272,6 +274,7 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   net->layers.assign(table, table + n_layers);
   net->outs.resize(n_layers);
   net->bytes.resize(n_layers);
+  net->res_narrow.assign(n_layers, nullptr);
   net->launches = n_layers;
   hq_status st = HQ_OK;
   auto shape_of = [&](int id, hq_tensor* t) -> bool {
@@ -340,6 +343,18 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     if (cudaMalloc(&net->scratch, want) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; }
     else net->scratch_bytes = want;
   }
+  // narrow residual pairs of every conv with a fused 8-bit residual (a one-off search per channel)
+  for (int i = 0; st == HQ_OK && i < n_layers; ++i) {
+    const hq_layer& l = net->layers[i];
+    if (l.op != HQ_OP_CONV || l.in1 < 0 || net->outs[l.in1].bits != 8 || net->outs[i].bits == 32) continue;
+    if (!l.conv.res_rescale.b || !l.conv.res_rescale.c) continue;
+    void* buf = nullptr;
+    if (cudaMalloc(&buf, (size_t)l.conv.cout * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+    net->res_narrow[i] = buf;
+    if (hq_launch_residual_narrow(l.conv.res_rescale.b, l.conv.res_rescale.c, net->outs[l.in1].is_signed, l.conv.cout,
+                                  buf, nullptr) != cudaSuccess) st = HQ_ERR_CUDA;
+  }
+  if (st == HQ_OK && cudaDeviceSynchronize() != cudaSuccess) st = HQ_ERR_CUDA;
   if (st != HQ_OK) { hq_network_destroy(net); return st; }
   *out = net;
   return HQ_OK;
@@ -363,7 +378,7 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         d.residual = nullptr;
         if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
         if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
-        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes);
+        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i]);
         break;
       }
       case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
@@ -465,6 +480,7 @@ hq_status hq_network_destroy(hq_network* net) {
   if (!net) return HQ_ERR_INVALID_ARG;
   for (auto& g : net->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& t : net->outs) if (t.data) cudaFree(t.data);
+  for (void* q : net->res_narrow) if (q) cudaFree(q);
   if (net->scratch) cudaFree(net->scratch);
   delete net;
   return HQ_OK;

@@ -75,6 +75,7 @@ struct TcParams {
   uint32_t out_stage_off, res_stage_off;   // offsets from the 1024-aligned dynamic base
   const int32_t* bias; const int32_t* b; const int32_t* c;
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
+  const int4* res_narrow;   // optional per-channel {m, a, s, valid} from residual_narrow_kernel
   int32_t relu, qmin, qmax;
   void* out; int32_t out_bits;
   uint32_t* status;
@@ -273,7 +274,10 @@ struct ChanConst {
 // a multiple of 2^8, and the dropped low 8 bits of r*rb cannot carry across a multiple of 2^(rc-8).
 // (A 64-bit multiply-add followed by a funnel shift measured no faster.)  `r` is the stored 8-bit
 // residual, already extended.  SMALL: some channel of the warp has c < 32.
-template <bool RES, bool RSIGNED, bool SMALL>
+// RN: every channel of the warp has a narrow residual pair (m, a, s) with (r*m + a) >> s equal to the residual
+// term for all 256 values of r (found and checked exhaustively by residual_narrow_kernel); rb / rh / rsh hold
+// m / a / s then, and a 32-bit multiply-add replaces the shift, multiply-high and add.
+template <bool RES, bool RSIGNED, bool SMALL, bool RN = false>
 __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) {
   const long long t1 = (long long)acc * (long long)k.b + k.r0;
   int s;
@@ -290,7 +294,9 @@ __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) 
     s = (above == (s0 >> 31)) ? (s0 >> k.sh) : (hi < 0 ? INT_MIN : INT_MAX);
     s = max(min(s, 1 << 30), -(1 << 30));
   }
-  if (RES) {
+  if (RES && RN) {
+    s += (r * k.rb + k.rh) >> k.rsh;
+  } else if (RES) {
     const unsigned top = (unsigned)r << 24;
     if (RSIGNED) s += (__mulhi((int)top, k.rb) + k.rh) >> k.rsh;
     else s += (int)((__umulhi(top, (unsigned)k.rb) + (unsigned)k.rh) >> k.rsh);
@@ -312,7 +318,7 @@ struct EpiCtx {
 // next one (of this tile, or the first of the group's next tile) streams from tensor memory into the
 // other register set; the accumulator buffer is handed back as soon as its last chunk has been read,
 // the residual tile as soon as its last bytes have been used, both before the tile's store is issued.
-template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL>
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN>
 __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const ChanConst& k_in) {
   // Private copies: the caller's objects live in local memory (their address is passed to the general
   // loop), so every asm statement with a memory clobber would force their fields to be re-read.
@@ -344,7 +350,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
       const int r = !RES ? 0 : RSIGNED ? (int)(signed char)res_tile[(c * 32 + j) * kTileC] : (int)res_tile[(c * 32 + j) * kTileC];
-      const int s = requant_fast<RES, RSIGNED, SMALL>(v[j], r, k);
+      const int s = requant_fast<RES, RSIGNED, SMALL, RN>(v[j], r, k);
       y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
     }
 #pragma unroll
@@ -769,6 +775,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         else { k.rh = 1 << (k.rsh - 9); k.rsh -= 8; }
       }
     }
+    // narrow residual pairs, when the caller prepared them and every channel of this warp has one
+    bool warp_narrow = false;
+    if (fast && !warp_small && p.res && p.res_narrow) {
+      const int4 nr = ch_live ? p.res_narrow[ch] : make_int4(0, 0, 0, 1);
+      warp_narrow = __all_sync(0xffffffffu, nr.w != 0) != 0;
+      if (warp_narrow) { k.rb = nr.x; k.rh = nr.y; k.rsh = nr.z; }
+    }
 
     EpiCtx e;
     e.p = &p; e.ctl = &ctl; e.map_out = &map_out; e.smem_raw = smem_raw; e.raw = raw; e.out_stage = out_stage;
@@ -781,8 +794,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
-#define HQ_FAST8(R, RS, S, OS) do { if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true>(e, k); \
-                                    else epilogue_loop_fast8<R, RS, S, OS, false>(e, k); } while (0)
+#define HQ_FAST8(R, RS, S, OS) do { if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true, false>(e, k); \
+                                    else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, false, R>(e, k); \
+                                    else epilogue_loop_fast8<R, RS, S, OS, false, false>(e, k); } while (0)
         case 0: HQ_FAST8(false, false, false, false); break;
         case 1: if (p.out_signed) HQ_FAST8(false, false, true, true); else HQ_FAST8(false, false, true, false); break;
         case 4: HQ_FAST8(true, false, false, false); break;
@@ -804,6 +818,36 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
+}
+
+// ---------------------------------------------------------------- narrow residual pairs ------
+// The residual term dn(r, rb, rc) = (r*rb + 2^(rc-1)) >> rc (Section 3.3, Appendix G) has only 256 possible
+// inputs per channel.  For most (rb, rc) a 23-bit multiplier m ~ rb / 2^8 with s = rc - 8 and a = 2^(s-1)
+// gives (r*m + a) >> s == dn(r, rb, rc) for every one of them, and r*m + a fits 32 bits.  One thread per
+// channel tries the two neighbouring multipliers and checks all 256 inputs; channels without such a pair
+// are marked invalid and keep the wide form.  Run once per layer when a network is built.
+__global__ void residual_narrow_kernel(const int32_t* __restrict__ rb, const int32_t* __restrict__ rc, int is_signed,
+                                       int n, int4* __restrict__ out) {
+  const int ch = blockIdx.x * blockDim.x + threadIdx.x;
+  if (ch >= n) return;
+  const long long b = rb[ch];
+  const int c = rc[ch];
+  int4 res = make_int4(0, 0, 0, 0);
+  const int r_lo = is_signed ? -128 : 0, r_hi = is_signed ? 127 : 255;
+  if (c >= 41 && c <= 62) {
+    res = make_int4(0, 0, 0, 1);                       // |r*rb| < 2^39 <= 2^(rc-2): the term is 0 for every r
+  } else if (c >= 9 && c <= 38) {
+    const int s = c - 8, a = 1 << (s - 1);
+    for (int t = 0; t < 2 && !res.w; ++t) {
+      const long long m = (b >> 8) + t;
+      if (m > (1 << 23) || m < -(1 << 23)) continue;
+      bool same = true;
+      for (int r = r_lo; r <= r_hi && same; ++r)
+        same = (((long long)r * b + (1LL << (c - 1))) >> c) == (long long)((r * (int)m + a) >> s);
+      if (same) res = make_int4((int)m, a, s, 1);
+    }
+  }
+  out[ch] = res;
 }
 
 // ---------------------------------------------------------------- host side ------------------
@@ -959,6 +1003,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
+  p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
   p.relu = a.relu; p.qmin = a.qmin; p.qmax = a.qmax;
   p.out = a.out; p.out_bits = a.out_bits; p.out_signed = a.out_signed;
   {
@@ -1024,6 +1069,13 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     conv_tc_kernel<kSoloEpilogueWarps, 1><<<grid, 64 + 32 * kSoloEpilogueWarps, smem, stream>>>(map_x, map_w, map_out, map_res, p);
   }
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
+                                      cudaStream_t s) {
+  if (channels <= 0) return cudaSuccess;
+  residual_narrow_kernel<<<(channels + 127) / 128, 128, 0, s>>>(rb, rc, res_signed, channels, (int4*)out);
+  return cudaGetLastError();
 }
 
 #ifdef HQ_TC_TRACE

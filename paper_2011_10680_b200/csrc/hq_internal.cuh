@@ -56,7 +56,8 @@ struct ConvArgs {
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   int32_t relu, qmin, qmax;
   void* out; int32_t ho, wo, out_bits, out_signed;
-  // internal lowerings only (zero for calls that come from the ABI):
+  // internal (zero for calls that come straight from the ABI):
+  const void* res_narrow;    // per-channel narrow residual pairs prepared by hq_launch_residual_narrow, or NULL
   int32_t pad_after_delta;   // padding after the last row/column minus `pad`
   // byte pitches of the activation tensor along W, H and N when it is not dense (0: dense NHWC).  A W pitch
   // below cin bytes makes neighbouring "pixels" overlap: a pixel is then a window of adjacent stored pixels.
@@ -75,6 +76,9 @@ bool hq_conv_tc_init();
 bool hq_conv_tc_supported(const ConvArgs& a);
 // Tensor-core path; returns HQ_OK, HQ_ERR_UNSUPPORTED or HQ_ERR_CUDA.
 hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
+// Fills `out` (channels x 16 bytes) with the narrow residual pairs of an 8-bit residual branch.
+cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
+                                      cudaStream_t s);
 // Lowered path for thin first layers: patch matrix + padded weights in scratch, then the tensor-core kernel.
 bool hq_conv_lowering_applies(const ConvArgs& a);
 size_t hq_conv_lowering_bytes(const ConvArgs& a);

@@ -352,6 +352,25 @@ def test_reduced_resnet18_and_resnet50_every_layer(hq):
         run_network_and_compare(hq, t, batch=3, seed=depth)
 
 
+def test_network_residual_shifts_per_channel(hq):
+    """Fused residual adds inside a network with a different dyadic pair on every channel: shifts from 9 to
+    45 (terms that vanish, terms with and without a narrow 32-bit form), unsigned and signed residual
+    operands.  Every layer must still match the oracle bit for bit."""
+    t = inputs.resnet_table(50, seed=11, image_hw=64, classes=24, width=32)
+    g = inputs.rng(11, 3)
+    n_res = 0
+    for l in t["layers"]:
+        if l["op"] == "conv" and l["in1"] >= 0:
+            c = l["cout"]
+            l["rb"] = g.integers(1 << 30, 1 << 31, size=c, dtype=np.int64).astype(np.int32)
+            l["rc"] = g.integers(9, 46, size=c, dtype=np.int64).astype(np.int32)
+            if n_res % 2 == 0:          # a few layers with shifts in the common range only
+                l["rc"] = g.integers(28, 36, size=c, dtype=np.int64).astype(np.int32)
+            n_res += 1
+    assert n_res >= 8
+    run_network_and_compare(hq, t, batch=2, seed=12)
+
+
 def test_resnet18_imagenet_shape_batch8_every_layer(hq):
     """Benchmark config 2: ResNet-18, 224x224x3, 1000 classes, batch 8, all layers INT8."""
     t = inputs.resnet_table(18, seed=2)
