@@ -109,45 +109,56 @@ __device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` =
   return (int)((__umulhi(top, (unsigned)d.b) + (unsigned)d.h) >> d.sh);
 }
 
-template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4>
-__global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int lo, int hi) {
-  const int wx = blockIdx.x * blockDim.x + threadIdx.x;     // word (4 channels) of the pixel
-  if (wx >= words) return;
-  Dy8 m[4], r[4];
+// One pixel's word of four channels.  SLOW: one of the thread's channels has a shift below 9 (64-bit form).
+// SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing).
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP>
+__device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, unsigned mw,
+                                              unsigned rw, long long idx, int lo, int hi) {
+  int s[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    m[i] = make_dy8(__ldg(a.mb + 4 * wx + i), __ldg(a.mc + 4 * wx + i));
-    if (RES) r[i] = make_dy8(__ldg(a.rb + 4 * wx + i), __ldg(a.rc + 4 * wx + i));
+    if (!SLOW) {
+      s[i] = dn8<MSIGNED>(__byte_perm(mw, 0u, 0x0444u | ((unsigned)i << 12)), m[i]);
+      if (RES) s[i] += dn8<RSIGNED>(__byte_perm(rw, 0u, 0x0444u | ((unsigned)i << 12)), r[i]);
+    } else {
+      const unsigned mbyte = (mw >> (8 * i)) & 0xFFu, rbyte = (rw >> (8 * i)) & 0xFFu;
+      long long t = hq_dn(MSIGNED ? (int)(signed char)mbyte : (int)mbyte, __ldg(a.mb + 4 * wx + i), m[i].c);
+      if (RES) t += hq_dn(RSIGNED ? (int)(signed char)rbyte : (int)rbyte, __ldg(a.rb + 4 * wx + i), r[i].c);
+      s[i] = (int)(t < (long long)lo ? (long long)lo : (t > (long long)hi ? (long long)hi : t));
+    }
   }
-  bool slow = false;                       // a shift below 9 on one of this thread's channels: 64-bit form for the thread
-#pragma unroll
-  for (int i = 0; i < 4; ++i) slow = slow || m[i].c < 9 || (RES && r[i].c < 9);
-  const unsigned* mp = (const unsigned*)a.main_t;
-  const unsigned* rp = (const unsigned*)a.res;
-  const long long step = (long long)gridDim.y * blockDim.y;
-  auto one = [&](unsigned mw, unsigned rw, long long idx) {
+  if constexpr (!OUT4 && SATP != 0) {
+    unsigned w01, w;
+    if (SATP == 1) {
+      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w01) : "r"(s[3]), "r"(s[2]), "r"(0));
+      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(0));
+    } else {
+      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w01) : "r"(s[3]), "r"(s[2]), "r"(0));
+      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(0));
+    }
+    ((unsigned*)a.out)[idx] = __byte_perm(w, w01, 0x5410);        // bytes: s0 s1 s2 s3
+  } else {
     int y[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (!slow) {
-        int s = dn8<MSIGNED>(__byte_perm(mw, 0u, 0x0444u | ((unsigned)i << 12)), m[i]);
-        if (RES) s += dn8<RSIGNED>(__byte_perm(rw, 0u, 0x0444u | ((unsigned)i << 12)), r[i]);
-        y[i] = min(max(s, lo), hi);
-      } else {
-        const unsigned mbyte = (mw >> (8 * i)) & 0xFFu, rbyte = (rw >> (8 * i)) & 0xFFu;
-        long long s = hq_dn(MSIGNED ? (int)(signed char)mbyte : (int)mbyte, __ldg(a.mb + 4 * wx + i), m[i].c);
-        if (RES) s += hq_dn(RSIGNED ? (int)(signed char)rbyte : (int)rbyte, __ldg(a.rb + 4 * wx + i), r[i].c);
-        y[i] = (int)(s < (long long)lo ? (long long)lo : (s > (long long)hi ? (long long)hi : s));
-      }
-    }
+    for (int i = 0; i < 4; ++i) y[i] = SLOW ? s[i] : min(max(s[i], lo), hi);
     if (OUT4) {
-      ((unsigned short*)a.out)[idx] = (unsigned short)((y[0] & 0xF) | ((y[1] & 0xF) << 4) | ((y[2] & 0xF) << 8) | ((y[3] & 0xF) << 12));
+      // 0 <= y <= 15 after the clamp of an unsigned 4-bit output; signed nibbles keep their low four bits
+      const unsigned w = (unsigned)(y[0] & 0xF) + ((unsigned)(y[1] & 0xF) << 4) + ((unsigned)(y[2] & 0xF) << 8) + ((unsigned)(y[3] & 0xF) << 12);
+      ((unsigned short*)a.out)[idx] = (unsigned short)w;
     } else {
       ((unsigned*)a.out)[idx] = (unsigned)(y[0] & 0xFF) | ((unsigned)(y[1] & 0xFF) << 8) | ((unsigned)(y[2] & 0xFF) << 16) |
                                 ((unsigned)(y[3] & 0xFF) << 24);
     }
-  };
-  constexpr int U = 8;                     // pixels (independent 4-byte loads) in flight per thread
+  }
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP>
+__device__ __forceinline__ void requant8_pixels(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, int words,
+                                                int lo, int hi) {
+  const unsigned* mp = (const unsigned*)a.main_t;
+  const unsigned* rp = (const unsigned*)a.res;
+  const long long step = (long long)gridDim.y * blockDim.y;
+  constexpr int U = 4;                     // pixels (independent 4-byte loads) in flight per thread
   long long p = (long long)blockIdx.y * blockDim.y + threadIdx.y;
   for (; p + (U - 1) * step < a.pixels; p += U * step) {
     unsigned mw[U], rw[U];
@@ -156,16 +167,39 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
 #pragma unroll
     for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rp + (p + u * step) * words + wx) : 0u;
 #pragma unroll
-    for (int u = 0; u < U; ++u) one(mw[u], rw[u], (p + u * step) * words + wx);
+    for (int u = 0; u < U; ++u)
+      requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP>(a, m, r, wx, mw[u], rw[u], (p + u * step) * words + wx, lo, hi);
   }
   for (; p < a.pixels; p += step)
-    one(__ldg(mp + p * words + wx), RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx);
+    requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP>(a, m, r, wx, __ldg(mp + p * words + wx),
+                                                           RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx, lo, hi);
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
+__global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int lo, int hi) {
+  const int wx = blockIdx.x * blockDim.x + threadIdx.x;     // word (4 channels) of the pixel
+  if (wx >= words) return;
+  Dy8 m[4], r[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m[i] = make_dy8(__ldg(a.mb + 4 * wx + i), __ldg(a.mc + 4 * wx + i));
+    if (RES) r[i] = make_dy8(__ldg(a.rb + 4 * wx + i), __ldg(a.rc + 4 * wx + i));
+    else r[i] = m[i];
+  }
+  bool slow = false;                       // a shift below 9 on one of this thread's channels: 64-bit form for the thread
+#pragma unroll
+  for (int i = 0; i < 4; ++i) slow = slow || m[i].c < 9 || (RES && r[i].c < 9);
+  // two separate loops, so that the common one carries none of the 64-bit form's instructions
+  if (slow) requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, words, lo, hi);
+  else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, words, lo, hi);
 }
 
 template <bool RES, bool MSIGNED, bool RSIGNED>
 cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, cudaStream_t s) {
-  if (a.out_bits == 4) requant8_kernel<RES, MSIGNED, RSIGNED, true><<<grid, block, 0, s>>>(a, words, lo, hi);
-  else requant8_kernel<RES, MSIGNED, RSIGNED, false><<<grid, block, 0, s>>>(a, words, lo, hi);
+  if (a.out_bits == 4) requant8_kernel<RES, MSIGNED, RSIGNED, true, 0><<<grid, block, 0, s>>>(a, words, lo, hi);
+  else if (lo == 0 && hi == 255) requant8_kernel<RES, MSIGNED, RSIGNED, false, 1><<<grid, block, 0, s>>>(a, words, lo, hi);
+  else if (lo == -128 && hi == 127) requant8_kernel<RES, MSIGNED, RSIGNED, false, 2><<<grid, block, 0, s>>>(a, words, lo, hi);
+  else requant8_kernel<RES, MSIGNED, RSIGNED, false, 0><<<grid, block, 0, s>>>(a, words, lo, hi);
   return cudaGetLastError();
 }
 
@@ -235,6 +269,42 @@ __global__ void avgpool_vec4_kernel(const unsigned* __restrict__ in, int n, int 
   out[i] = w;
 }
 
+// Same result with more loads in flight: block (64 words, 4 pixel slices) per (image, 64 words); bytes are summed
+// as 16-bit lanes of two registers (h*w*255 <= 65535, i.e. up to 257 pixels; signed bytes are offset by 128 and
+// corrected at the end), the four slices meet in shared memory.
+__global__ void __launch_bounds__(256) avgpool_vec4_sliced_kernel(const unsigned* __restrict__ in, int hw, int ch, int is_signed,
+                                                                  const int32_t* __restrict__ b, const int32_t* __restrict__ c,
+                                                                  int qmin, int qmax, unsigned* __restrict__ out) {
+  __shared__ unsigned part[2][4][64];
+  const int cg = ch >> 2;
+  const int g = blockIdx.x * 64 + threadIdx.x, img = blockIdx.y;
+  unsigned lo = 0, hi = 0;
+  if (g < cg) {
+    const unsigned* p = in + (long long)img * hw * cg + g;
+    const unsigned flip = is_signed ? 0x80808080u : 0u;
+    for (int k = threadIdx.y; k < hw; k += 4) {
+      const unsigned v = __ldg(p + (long long)k * cg) ^ flip;
+      lo += v & 0x00FF00FFu;
+      hi += (v >> 8) & 0x00FF00FFu;
+    }
+  }
+  part[0][threadIdx.y][threadIdx.x] = lo;
+  part[1][threadIdx.y][threadIdx.x] = hi;
+  __syncthreads();
+  if (threadIdx.y != 0 || g >= cg) return;
+  lo = part[0][0][threadIdx.x] + part[0][1][threadIdx.x] + part[0][2][threadIdx.x] + part[0][3][threadIdx.x];
+  hi = part[1][0][threadIdx.x] + part[1][1][threadIdx.x] + part[1][2][threadIdx.x] + part[1][3][threadIdx.x];
+  const int off = is_signed ? 128 * hw : 0;
+  const int sums[4] = {(int)(lo & 0xFFFFu) - off, (int)(hi & 0xFFFFu) - off, (int)(lo >> 16) - off, (int)(hi >> 16) - off};
+  unsigned w = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int q = hq_clamp_ll(hq_dn(sums[j], b[4 * g + j], c[4 * g + j]), 0, qmin, qmax);
+    w |= (unsigned)(q & 0xFF) << (8 * j);
+  }
+  out[(long long)img * cg + g] = w;
+}
+
 __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int in_bits, int in_signed,
                                       const int32_t* b, const int32_t* c, int qmin, int qmax,
                                       void* out, int out_bits) {
@@ -256,31 +326,30 @@ __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int
 }
 
 // ---- max pooling ----------------------------------------------------------------------------
+// One block per (image, output row): no 64-bit index arithmetic per output (the division-heavy flat index
+// made an earlier version instruction-bound); a thread handles 16 channels of one output pixel at a time.
 template <bool SIGNED>
-__global__ void maxpool_vec16_kernel(const uint4* __restrict__ in, int n, int h, int w, int cg,
-                                     int k, int stride, int pad, uint4* __restrict__ out, int ho, int wo) {
-  const long long total = (long long)n * ho * wo * cg;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-       i += (long long)gridDim.x * blockDim.x) {
-    const int g = (int)(i % cg);
-    long long t = i / cg;
-    const int ow = (int)(t % wo); t /= wo;
-    const int oh = (int)(t % ho);
-    const int img = (int)(t / ho);
+__global__ void __launch_bounds__(256) maxpool_vec16_kernel(const uint4* __restrict__ in, int h, int w, int cg,
+                                                            int k, int stride, int pad, uint4* __restrict__ out, int ho, int wo) {
+  const int img = blockIdx.x / ho, oh = blockIdx.x - img * ho;
+  const uint4* in_img = in + (long long)img * h * w * cg;
+  uint4* out_row = out + ((long long)img * ho + oh) * wo * cg;
+  const int r_lo = max(0, pad - oh * stride), r_hi = min(k, h + pad - oh * stride);   // valid filter rows
+  const int row_items = wo * cg;
+  for (int idx = threadIdx.x; idx < row_items; idx += blockDim.x) {
+    const int ow = idx / cg, g = idx - ow * cg;
+    const int s_lo = max(0, pad - ow * stride), s_hi = min(k, w + pad - ow * stride);
     const unsigned init = SIGNED ? 0x80808080u : 0u;
     uint4 m = make_uint4(init, init, init, init);
-    for (int r = 0; r < k; ++r) {
-      const int ih = oh * stride + r - pad;
-      if (ih < 0 || ih >= h) continue;
-      for (int s = 0; s < k; ++s) {
-        const int iw = ow * stride + s - pad;
-        if (iw < 0 || iw >= w) continue;
-        const uint4 v = __ldg(in + (((long long)img * h + ih) * w + iw) * cg + g);
+    for (int r = r_lo; r < r_hi; ++r) {
+      const uint4* row = in_img + ((long long)(oh * stride + r - pad) * w + (ow * stride - pad)) * cg + g;
+      for (int s = s_lo; s < s_hi; ++s) {
+        const uint4 v = __ldg(row + s * cg);
         if (SIGNED) { m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y); m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w); }
         else        { m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w); }
       }
     }
-    out[i] = m;
+    out_row[idx] = m;
   }
 }
 
@@ -356,7 +425,10 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
                               const int32_t* b, const int32_t* c, int qmin, int qmax,
                               void* out, int out_bits, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  if (in_bits == 8 && out_bits == 8 && ch % 4 == 0) {
+  if (in_bits == 8 && out_bits == 8 && ch % 4 == 0 && h * w <= 257 && n <= 65535) {
+    const dim3 grid((ch / 4 + 63) / 64, n), block(64, 4);
+    avgpool_vec4_sliced_kernel<<<grid, block, 0, s>>>((const unsigned*)in, h * w, ch, in_signed, b, c, qmin, qmax, (unsigned*)out);
+  } else if (in_bits == 8 && out_bits == 8 && ch % 4 == 0) {
     const int total = n * (ch / 4);
     avgpool_vec4_kernel<<<(total + 127) / 128, 128, 0, s>>>((const unsigned*)in, n, h * w, ch, in_signed,
                                                              b, c, qmin, qmax, (unsigned*)out);
@@ -371,16 +443,11 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
 cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int is_signed,
                               int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  if (ch % 16 == 0) {
-    const long long total = (long long)n * ho * wo * (ch / 16);
-    long long blocks = (total + 255) / 256;
-    if (blocks > (1 << 20)) blocks = 1 << 20;
+  if (ch % 16 == 0 && (long long)n * ho < (1ll << 31) && (long long)wo * (ch / 16) < (1ll << 31)) {
     if (is_signed)
-      maxpool_vec16_kernel<true><<<(int)blocks, 256, 0, s>>>((const uint4*)in, n, h, w, ch / 16, k, stride, pad,
-                                                              (uint4*)out, ho, wo);
+      maxpool_vec16_kernel<true><<<n * ho, 256, 0, s>>>((const uint4*)in, h, w, ch / 16, k, stride, pad, (uint4*)out, ho, wo);
     else
-      maxpool_vec16_kernel<false><<<(int)blocks, 256, 0, s>>>((const uint4*)in, n, h, w, ch / 16, k, stride, pad,
-                                                               (uint4*)out, ho, wo);
+      maxpool_vec16_kernel<false><<<n * ho, 256, 0, s>>>((const uint4*)in, h, w, ch / 16, k, stride, pad, (uint4*)out, ho, wo);
   } else {
     const long long total = (long long)n * ho * wo * ch;
     long long blocks = (total + 255) / 256;
