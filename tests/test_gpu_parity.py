@@ -90,6 +90,12 @@ TC_CASES = [
     (1, 20, 20, 128, 256, 3, 1, 1, 8, True, 8, True),        # residual + 3x3 + two N tiles of 128
     (3, 8, 8, 64, 64, 1, 1, 0, 4, True, 8, True),            # uint4 output with residual
     (2, 16, 16, 32, 128, 1, 1, 0, 4, False, 8, True),        # uint4 output, 64-byte store boxes
+    # large enough for the benchmark's launch shapes (the pixel tile grows with the number of tiles per SM)
+    (33, 56, 56, 64, 64, 1, 1, 0, 8, False, 8, True),        # 256-pixel tiles, folded 64-channel tile, ragged last tile
+    (13, 56, 56, 64, 64, 3, 1, 1, 8, True, 8, True),         # 128-pixel tiles, four accumulator buffers, folded, residual
+    (17, 56, 56, 64, 256, 1, 1, 0, 8, True, 8, True),        # two CTAs per SM (fused residual, short K), ragged last tile
+    (21, 28, 28, 128, 512, 1, 1, 0, 8, True, 8, False),      # two CTAs per SM with 64-byte K blocks cut from cin = 128, signed out
+    (9, 28, 28, 128, 128, 3, 1, 1, 8, False, 8, True),       # 256-pixel tiles, long K, one CTA per SM
 ]
 
 
@@ -377,3 +383,38 @@ def test_resnet18_imagenet_shape_batch8_every_layer(hq):
     ref = run_network_and_compare(hq, t, batch=8, seed=2)
     sat = [float(np.mean((r == 0) | (r == 255))) for r, l in zip(ref, t["layers"]) if l["op"] == "conv" and l["out_bits"] == 8]
     assert min(sat) < 0.9, "every layer is saturated: the workload would not exercise the requantization"
+
+
+def test_resnet50_batch256_benchmark_configuration_sampled_images(hq):
+    """The benchmark workloads themselves (ResNet-50, 224x224, batch 256, INT8 and mixed INT4/8), in the launch
+    configuration bench.py times: tile sizes, folded channel tiles, the two-CTA shape and the number of
+    accumulator buffers all depend on the batch.  Images are independent, so the oracle runs the first two and
+    the last image of the batch and every layer's output for those images must match bit for bit."""
+    from oracle.network import run_network
+    from paper_2011_10680_b200 import binding
+    batch, pick = 256, [0, 1, 255]
+    for mixed, seed in ((False, 3), (True, 4)):
+        t = inputs.resnet_table(50, seed, mixed=mixed)
+        images = inputs.random_images(seed, batch, t["image_hw"])
+        ref = run_network(t, images[pick])
+        net = binding.Network(hq, t, batch)
+        try:
+            d_img = binding.to_device(images)
+            logits = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+            taps = net.alloc_taps()
+            assert net.run(d_img, logits, taps) == binding.HQ_OK
+            hq.sync()
+            for i, (tap, r) in enumerate(zip(taps, ref)):
+                per_image = tap.numel() // batch
+                got = tap.view(batch, per_image)[pick].cpu().numpy()
+                want = np.ascontiguousarray(r).view(np.uint8).reshape(len(pick), per_image)
+                assert np.array_equal(got, want), f"mixed={mixed} layer {i} ({t['layers'][i]['op']}) differs in {(got != want).sum()} bytes"
+            # the graph-replay path that the benchmark times
+            logits.zero_()
+            assert net.run(d_img, logits, None) == binding.HQ_OK
+            hq.sync()
+            assert np.array_equal(logits.cpu().numpy().reshape(batch, -1)[pick], ref[-1].reshape(len(pick), -1))
+            del taps
+        finally:
+            net.close()
+        torch.cuda.empty_cache()
