@@ -34,7 +34,8 @@ inline long long tensor_bytes(int n, int h, int w, int c, int bits) {
 // `scratch` / `scratch_bytes`: buffer for the lowered first-layer path owned by the caller (a
 // network); NULL means use (and if needed grow) the handle's own buffer.
 hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq_tensor* out, void* stream,
-                      void* scratch = nullptr, size_t scratch_bytes = 0, const void* res_narrow = nullptr) {
+                      void* scratch = nullptr, size_t scratch_bytes = 0, const void* res_narrow = nullptr,
+                      const void* wgt_widened = nullptr) {
   if (!h || !d) return HQ_ERR_INVALID_ARG;
   hq_status st = check_tensor(in, true, true, false);
   if (st != HQ_OK) return st;
@@ -62,7 +63,7 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   }
   ConvArgs a{};
   a.in = in->data; a.n = in->n; a.h = in->h; a.w = in->w; a.cin = in->c; a.in_bits = in->bits; a.in_signed = in->is_signed;
-  a.wgt = d->w; a.cout = d->cout; a.kh = d->kh; a.kw = d->kw; a.stride = d->stride; a.pad = d->pad;
+  a.wgt = d->w; a.wgt_widened = wgt_widened; a.cout = d->cout; a.kh = d->kh; a.kw = d->kw; a.stride = d->stride; a.pad = d->pad;
   a.bias = d->bias; a.b = d->requant.b; a.c = d->requant.c;
   if (d->residual && out->bits != 32) {
     a.res = d->residual->data; a.res_bits = d->residual->bits; a.res_signed = d->residual->is_signed;
@@ -119,6 +120,7 @@ struct hq_network {
   int32_t batch, image_h, image_w, image_c, image_signed;
   int32_t launches;
   std::vector<void*> res_narrow;     // per conv layer with a fused 8-bit residual: its narrow residual pairs (owned)
+  std::vector<void*> wgt_widened;    // per 4-bit conv layer on the tensor-core path: its weights, one byte per value (owned)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
@@ -275,6 +277,7 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   net->outs.resize(n_layers);
   net->bytes.resize(n_layers);
   net->res_narrow.assign(n_layers, nullptr);
+  net->wgt_widened.assign(n_layers, nullptr);
   net->launches = n_layers;
   hq_status st = HQ_OK;
   auto shape_of = [&](int id, hq_tensor* t) -> bool {
@@ -302,7 +305,12 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
           if (hq_conv_widen4_applies(a)) {
             const size_t need = hq_conv_widen4_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
-            net->launches += 2;                 // two widening kernels
+            net->launches += 1;                 // the activation-widening kernel (the weights are widened once, below)
+            const long long wvals = (long long)d.cout * d.kh * d.kw * in.c;
+            void* wbuf = nullptr;
+            if (cudaMalloc(&wbuf, (size_t)wvals + 256) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+            net->wgt_widened[i] = wbuf;
+            if (hq_launch_widen_weights(d.w, wvals, wbuf, h->sm_count, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
           } else if (hq_conv_s2d_applies(a)) {
             const size_t need = hq_conv_s2d_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
@@ -378,7 +386,7 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         d.residual = nullptr;
         if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
         if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
-        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i]);
+        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i], net->wgt_widened[i]);
         break;
       }
       case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
@@ -481,6 +489,7 @@ hq_status hq_network_destroy(hq_network* net) {
   for (auto& g : net->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& t : net->outs) if (t.data) cudaFree(t.data);
   for (void* q : net->res_narrow) if (q) cudaFree(q);
+  for (void* q : net->wgt_widened) if (q) cudaFree(q);
   if (net->scratch) cudaFree(net->scratch);
   delete net;
   return HQ_OK;

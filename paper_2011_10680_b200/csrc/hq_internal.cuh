@@ -58,6 +58,7 @@ struct ConvArgs {
   void* out; int32_t ho, wo, out_bits, out_signed;
   // internal (zero for calls that come straight from the ABI):
   const void* res_narrow;    // per-channel narrow residual pairs prepared by hq_launch_residual_narrow, or NULL
+  const void* wgt_widened;   // 4-bit weights already widened to one byte per value (a network does it once), or NULL
   int32_t pad_after_delta;   // padding after the last row/column minus `pad`
   // byte pitches of the activation tensor along W, H and N when it is not dense (0: dense NHWC).  A W pitch
   // below cin bytes makes neighbouring "pixels" overlap: a pixel is then a window of adjacent stored pixels.
@@ -91,6 +92,8 @@ hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cud
 bool hq_conv_widen4_applies(const ConvArgs& a);
 size_t hq_conv_widen4_bytes(const ConvArgs& a);
 hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
+// Widen packed 4-bit weights (cout*kh*kw*cin values, a multiple of 16) to bytes, once, for ConvArgs::wgt_widened.
+cudaError_t hq_launch_widen_weights(const void* wgt, long long values, void* out, int sm_count, cudaStream_t s);
 // Grow the handle's scratch buffer (not allowed while `s` is capturing).
 hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s);
 cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s);

@@ -213,22 +213,33 @@ hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cud
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-// 8 packed bytes -> 16 bytes; element 2j = low nibble of byte j.
+template <bool SIGNED>
+__device__ __forceinline__ uint4 widen4_vec(uint2 v) {
+  unsigned o[4];
+  const unsigned w[2] = {v.x, v.y};
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    unsigned lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
+    if (SIGNED) { lo |= (lo & 0x08080808u) * 0x1Eu; hi |= (hi & 0x08080808u) * 0x1Eu; }   // sign-extend each nibble
+    o[2 * k] = __byte_perm(lo, hi, 0x5140);          // n0 n1 n2 n3
+    o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);      // n4 n5 n6 n7
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// 8 packed bytes -> 16 bytes; element 2j = low nibble of byte j.  Four independent loads per thread and trip.
 template <bool SIGNED>
 __global__ void __launch_bounds__(256) widen4_kernel(const uint2* __restrict__ in, long long n_vec, uint4* __restrict__ out) {
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (long long)gridDim.x * blockDim.x) {
-    const uint2 v = __ldg(in + i);
-    unsigned o[4];
-    const unsigned w[2] = {v.x, v.y};
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < n_vec; i += 4 * stride) {
+    uint2 v[4];
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      unsigned lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
-      if (SIGNED) { lo |= (lo & 0x08080808u) * 0x1Eu; hi |= (hi & 0x08080808u) * 0x1Eu; }   // sign-extend each nibble
-      o[2 * k] = __byte_perm(lo, hi, 0x5140);          // n0 n1 n2 n3
-      o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);      // n4 n5 n6 n7
-    }
-    out[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    for (int u = 0; u < 4; ++u) v[u] = __ldg(in + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) out[i + u * stride] = widen4_vec<SIGNED>(v[u]);
   }
+  for (; i < n_vec; i += stride) out[i] = widen4_vec<SIGNED>(__ldg(in + i));
 }
 
 cudaError_t launch_widen4(const void* in, long long elems, int is_signed, void* out, int sm_count, cudaStream_t s) {
@@ -262,10 +273,14 @@ hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, 
   unsigned char* xw = (unsigned char*)scratch;
   unsigned char* ww = xw + (x + 255) / 256 * 256;
   if (launch_widen4(a.in, x, a.in_signed, xw, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
-  if (launch_widen4(a.wgt, w, 1, ww, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+  if (!a.wgt_widened && launch_widen4(a.wgt, w, 1, ww, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
   ConvArgs t = a;
-  t.in = xw; t.wgt = ww; t.in_bits = 8;
+  t.in = xw; t.wgt = a.wgt_widened ? a.wgt_widened : ww; t.in_bits = 8;
   return hq_launch_conv_tc(h, t, s);
+}
+
+cudaError_t hq_launch_widen_weights(const void* wgt, long long values, void* out, int sm_count, cudaStream_t s) {
+  return launch_widen4(wgt, values, 1, out, sm_count, s);
 }
 
 // ------------------------------------------------------------------------------------------------
