@@ -958,9 +958,6 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   // (measured: the pair shape wins on the fused-residual expansions, whose epilogue is the longest per tile,
   // and loses where a tile carries little epilogue work, e.g. 64 output channels)
   bool pair = k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
-#ifdef HQ_EXP_PAIR
-  pair = (HQ_EXP_PAIR != 0);
-#endif
   int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
   if (pair) {
     // 128-pixel tiles, two accumulator buffers (256 columns), K blocks of at most 64 bytes
