@@ -615,10 +615,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl.tmem_base;
+  // Programmatic dependent launch: this grid may have started while the previous kernel of the stream was
+  // still finishing (its CTAs leave the SMs one by one); everything above touched only this CTA's own
+  // resources.  The threads that read what the previous kernel wrote -- the producer lane (activations and
+  // residual tiles by TMA) and epilogue warps that load a residual directly -- wait for that grid to complete
+  // first; the other roles only consume what arrives behind the producer's barriers.  The next kernel's CTAs
+  // may start filling SMs as ours leave.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       // No division or modulo in this loop: one thread runs it and every dependent instruction
       // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
@@ -783,6 +791,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (warp_narrow) { k.rb = nr.x; k.rh = nr.y; k.rsh = nr.z; }
     }
 
+    if (p.res && !p.staged_res) asm volatile("griddepcontrol.wait;" ::: "memory");   // direct residual loads below
     EpiCtx e;
     e.p = &p; e.ctl = &ctl; e.map_out = &map_out; e.smem_raw = smem_raw; e.raw = raw; e.out_stage = out_stage;
     e.res_stage = res_stage; e.res_tile_bytes = res_tile_bytes; e.tmem_base = tmem_base;
@@ -1058,14 +1067,23 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int slots = pair ? 2 * h->sm_count : h->sm_count;
   const int grid = (int)(total_tiles <= slots ? total_tiles : (slots / p.c_tiles) * p.c_tiles);
+  // Launched with programmatic stream serialization: the grid may begin (barrier set-up, tensor-memory
+  // allocation) while the previous kernel drains; the kernel waits for it before reading any input.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+  cudaError_t err;
   if (pair) {
-    conv_tc_kernel<kPairEpilogueWarps, 2><<<grid, 64 + 32 * kPairEpilogueWarps, dyn_smem, stream>>>(map_x, map_w, map_out, map_res, p);
+    cfg.blockDim = dim3(64 + 32 * kPairEpilogueWarps); cfg.dynamicSmemBytes = dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kPairEpilogueWarps, 2>, map_x, map_w, map_out, map_res, p);
   } else {
     // one CTA per SM (it may allocate all 512 tensor-memory columns): never request less than 120 KiB
-    const size_t smem = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
-    conv_tc_kernel<kSoloEpilogueWarps, 1><<<grid, 64 + 32 * kSoloEpilogueWarps, smem, stream>>>(map_x, map_w, map_out, map_res, p);
+    cfg.blockDim = dim3(64 + 32 * kSoloEpilogueWarps); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kSoloEpilogueWarps, 1>, map_x, map_w, map_out, map_res, p);
   }
-  return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+  return err == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
