@@ -119,6 +119,15 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
 // pixels: output (oh, ow) reads s2d rows oh-2 .. oh+1 (two rows of padding before, one after), and
 // weight w2[oc][ty][tx][(dy*2+dx)*3 + c] = w[oc][2ty+dy-1][2tx+dx-1][c] (zero where the 7x7 index falls
 // outside 0..6 and in the padded channels).  Zeros add nothing, so the INT32 accumulator is unchanged.
+//
+// The copy is stored with its zero padding, so the taps of a filter row are contiguous bytes, and the
+// tensor-core kernel is handed a 4x1 convolution over "pixels" that are windows of the stored image:
+// one window of 8 stored pixels (128 bytes, W pitch 32 bytes: neighbouring windows overlap) feeds TWO
+// adjacent outputs, whose 2 x cout values are the window's "output channels": output 2q + o, channel ch is
+// virtual channel o*cout + ch of virtual pixel q, i.e. the same byte of the NHWC output tensor read as rows
+// of 2*cout bytes.  Virtual channel (o, ch) carries w2[ch][ty][i - o][.] at stored pixel i of the window
+// (zero outside 0 <= i - o <= 3).  That gives full 128-byte TMA rows and fills all 128 accumulator lanes
+// for cout = 64 (16-byte and 64-byte rows measured 4x and 1.4x slower), at the price of multiplying zeros.
 // ------------------------------------------------------------------------------------------------
 namespace {
 
@@ -148,60 +157,81 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned char
   }
 }
 
-__global__ void s2d_weights_kernel(const signed char* __restrict__ w, int cout, signed char* __restrict__ out) {
-  const int total = cout * 256;
+// Weights of the 2*cout virtual channels, [2*cout][4 filter rows][128 window bytes], and the per-channel
+// constants repeated for both outputs of a window.
+__global__ void s2d_weights_kernel(const signed char* __restrict__ w, int cout, signed char* __restrict__ out,
+                                   const int32_t* __restrict__ bias, const int32_t* __restrict__ b,
+                                   const int32_t* __restrict__ c, int32_t* __restrict__ consts) {
+  const int total = 2 * cout * 512;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-    const int ch16 = i & 15, tx = (i >> 4) & 3, ty = (i >> 6) & 3, oc = i >> 8;
-    signed char v = 0;
-    if (ch16 < 12) {
-      const int c = ch16 % 3, dx = (ch16 / 3) & 1, dy = ch16 / 6;
+    const int ch16 = i & 15, px = (i >> 4) & 7, ty = (i >> 7) & 3, v = i >> 9;
+    const int o = v / cout, oc = v - o * cout, tx = px - o;
+    signed char val = 0;
+    if (ch16 < 12 && tx >= 0 && tx < 4) {
+      const int cc = ch16 % 3, dx = (ch16 / 3) & 1, dy = ch16 / 6;
       const int r = 2 * ty + dy - 1, sx = 2 * tx + dx - 1;
-      if (r >= 0 && r < 7 && sx >= 0 && sx < 7) v = w[((oc * 7 + r) * 7 + sx) * 3 + c];
+      if (r >= 0 && r < 7 && sx >= 0 && sx < 7) val = w[((oc * 7 + r) * 7 + sx) * 3 + cc];
     }
-    out[i] = v;
+    out[i] = val;
+    if (i < 2 * cout) {
+      const int ch = i % cout;
+      consts[i] = bias ? bias[ch] : 0;
+      consts[2 * cout + i] = b ? b[ch] : 0;
+      consts[4 * cout + i] = c ? c[ch] : 1;
+    }
   }
 }
 
-}  // namespace
+// scratch layout: padded image | virtual weights | bias, b, c of the virtual channels
+struct S2dLayout { long long img_bytes, wts_off, wts_bytes, consts_off, total; };
+S2dLayout s2d_layout(const ConvArgs& a) {
+  S2dLayout l;
+  l.img_bytes = (long long)a.n * (a.h / 2 + 3) * (a.w / 2 + 3) * 16;
+  l.wts_off = (l.img_bytes + 255) / 256 * 256;          // the last window reads 48 bytes past the image: into the weights
+  l.wts_bytes = (long long)2 * a.cout * 512;
+  l.consts_off = l.wts_off + (l.wts_bytes + 255) / 256 * 256;
+  l.total = l.consts_off + ((long long)6 * a.cout * 4 + 255) / 256 * 256;
+  return l;
+}
 
-namespace {
-// The 4x4 / stride-1 convolution over the padded space-to-depth image, described to the tensor-core kernel as a
-// 4x1 convolution over 64-byte "pixels": the four taps of a filter row are 64 contiguous bytes of the image,
-// so a pixel is a window of four stored pixels and neighbouring windows overlap (W pitch 16 bytes < 64).
-ConvArgs s2d_conv_args(const ConvArgs& a, const void* img, const void* wts) {
+ConvArgs s2d_conv_args(const ConvArgs& a, const void* scratch) {
   ConvArgs t = a;
+  const S2dLayout l = s2d_layout(a);
   const int h2 = a.h / 2, w2 = a.w / 2, hp = h2 + 3, wp = w2 + 3;
-  t.in = img; t.wgt = wts;
-  t.h = hp; t.w = w2; t.cin = 64; t.kh = 4; t.kw = 1; t.stride = 1; t.pad = 0; t.pad_after_delta = 0;
-  t.pitch_w = 16; t.pitch_h = (long long)wp * 16; t.pitch_n = (long long)hp * wp * 16;
+  const unsigned char* base = (const unsigned char*)scratch;
+  const int32_t* consts = (const int32_t*)(base + l.consts_off);
+  t.in = base; t.wgt = base + l.wts_off;
+  t.h = hp; t.w = w2 / 2; t.cin = 128; t.kh = 4; t.kw = 1; t.stride = 1; t.pad = 0; t.pad_after_delta = 0;
+  t.pitch_w = 32; t.pitch_h = (long long)wp * 16; t.pitch_n = (long long)hp * wp * 16;
+  t.cout = 2 * a.cout; t.wo = a.wo / 2;
+  t.bias = consts; t.b = consts + 2 * a.cout; t.c = consts + 4 * a.cout;
   return t;
 }
 }  // namespace
 
 bool hq_conv_s2d_applies(const ConvArgs& a) {
   if (a.in_bits != 8 || a.cin != 3 || a.kh != 7 || a.kw != 7 || a.stride != 2 || a.pad != 3) return false;
-  if ((a.h & 1) || (a.w & 1) || a.pitch_w) return false;
-  return hq_conv_tc_supported(s2d_conv_args(a, a.in, a.wgt));
+  if ((a.h & 1) || (a.w & 3) || a.pitch_w || a.res || a.out_bits != 8) return false;       // pairs of outputs: w/2 even
+  if ((long long)a.cout * 1024 >= (1ll << 31)) return false;
+  return hq_conv_tc_supported(s2d_conv_args(a, a.in));
 }
 
-size_t hq_conv_s2d_bytes(const ConvArgs& a) {
-  const long long img = (long long)a.n * (a.h / 2 + 3) * (a.w / 2 + 3) * 16, wts = (long long)a.cout * 256;
-  return (size_t)(((img + 255) / 256 + (wts + 255) / 256) * 256);
-}
+size_t hq_conv_s2d_bytes(const ConvArgs& a) { return (size_t)s2d_layout(a).total; }
 
 // `scratch` must hold hq_conv_s2d_bytes(a) bytes, 256-byte aligned.
 hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s) {
-  const long long px = (long long)a.n * (a.h / 2 + 3) * (a.w / 2 + 3);
   if (a.n == 0) return HQ_OK;
-  unsigned char* img = (unsigned char*)scratch;
-  signed char* wts = (signed char*)(img + (px * 16 + 255) / 256 * 256);
-  s2d_weights_kernel<<<(a.cout * 256 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, wts);
+  const S2dLayout l = s2d_layout(a);
+  unsigned char* base = (unsigned char*)scratch;
+  s2d_weights_kernel<<<(2 * a.cout * 512 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, (signed char*)(base + l.wts_off),
+                                                                   a.bias, a.b, a.c, (int32_t*)(base + l.consts_off));
   if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+  const long long px = l.img_bytes / 16;
   long long blocks = (px + 255) / 256;
   const long long cap = (long long)h->sm_count * 32;
-  space_to_depth_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, (uint4*)img);
+  space_to_depth_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, (uint4*)base);
   if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
-  return hq_launch_conv_tc(h, s2d_conv_args(a, img, wts), s);
+  return hq_launch_conv_tc(h, s2d_conv_args(a, scratch), s);
 }
 
 // ------------------------------------------------------------------------------------------------
