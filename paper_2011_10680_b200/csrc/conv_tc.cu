@@ -61,6 +61,8 @@ struct TcParams {
   int32_t k_blocks;      // kh * kw * cchunks
   int32_t pt;            // pixel tile = MMA N: 64, 128 or 256
   int32_t p_tiles, c_tiles, stages;
+  int32_t wres;          // 1: the CTA's whole weight slab [k_blocks][128][bkb] is loaded once and stays in shared memory
+  uint32_t wres_off;     // its offset from the 1024-aligned dynamic base
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
@@ -97,6 +99,7 @@ struct SharedCtl {
   unsigned long long rfull[kMaxAccBufs];
   unsigned long long rempty[kMaxAccBufs];
   unsigned long long drain;
+  unsigned long long wfull;              // resident weight slab landed
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -589,7 +592,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // operand stages, 1024-byte aligned
   const uint32_t w_bytes = kTileC * p.bkb;
   const uint32_t x_bytes = p.pt * p.bkb;
-  const uint32_t stage_bytes = w_bytes + x_bytes;
+  const uint32_t x_off = p.wres ? 0u : w_bytes;          // offset of the X tile inside a stage
+  const uint32_t stage_bytes = x_off + x_bytes;
   const uint32_t out_stage = tiles + p.out_stage_off;
   const uint32_t res_stage = tiles + p.res_stage_off;
   const uint32_t res_tile_bytes = p.pt * kTileC;          // [pt pixels][128 channels] bytes
@@ -607,6 +611,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), 4 * p.halves);
     }
     mbar_init(smem_u32(&ctl.drain), 1);
+    mbar_init(smem_u32(&ctl.wfull), 1);
     ctl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -639,6 +644,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       int ow = (p_tile0 * p.pt) - img * p.howo - oh * p.wo;
       const int step = p_step * p.pt;
       const int d_img = step / p.howo, d_oh = (step - d_img * p.howo) / p.wo, d_ow = step - d_img * p.howo - d_oh * p.wo;
+      if (p.wres) {              // the channel tile's weights for every K block, once
+        const uint32_t bar = smem_u32(&ctl.wfull);
+        mbar_expect_tx(bar, (uint32_t)p.k_blocks * w_bytes);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          const uint32_t w_dst = tiles + p.wres_off + (uint32_t)kb * w_bytes;
+          if (p.fold) {
+            tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, 0);
+            tma_load_2d(w_dst + 64 * p.bkb, &map_w, bar, kb * p.bkb, 0);
+          } else {
+            tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
+          }
+        }
+      }
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
         const int p0 = p_tile * p.pt;
         if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
@@ -660,11 +678,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const uint32_t w_dst = tiles + s * stage_bytes;
           mbar_expect_tx(bar, stage_bytes);
           if (p.x_tiled) {
-            tma_load_2d(w_dst + w_bytes, &map_x, bar, chunk * p.bkb, p0);
+            tma_load_2d(w_dst + x_off, &map_x, bar, chunk * p.bkb, p0);
           } else {
-            tma_load_im2col(w_dst + w_bytes, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
+            tma_load_im2col(w_dst + x_off, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
           }
-          if (p.fold) {          // 64-row box, twice: accumulator lanes 64-127 repeat lanes 0-63
+          if (p.wres) {
+            // weights are resident
+          } else if (p.fold) {   // 64-row box, twice: accumulator lanes 64-127 repeat lanes 0-63
             tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, 0);
             tma_load_2d(w_dst + 64 * p.bkb, &map_w, bar, kb * p.bkb, 0);
           } else {
@@ -681,6 +701,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const uint32_t ds = k % p.stages, dph = (k / p.stages) & 1u;
         const unsigned long long t0 = global_ns();
         while (!mbar_try_wait(smem_u32(&ctl.full[ds]), dph)) {
+          if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
+        }
+      }
+      if (p.wres) {
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(smem_u32(&ctl.wfull), 0)) {
           if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
         }
       }
@@ -706,6 +732,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       const uint64_t desc_hi = smem_desc(0, p.bkb);           // everything but the start address
       const int ksteps = p.bkb >> 5;
+      if (p.wres && !mbar_wait(smem_u32(&ctl.wfull), 0, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) ok = false;
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
         const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
         // The operands of the tile's first K block have usually landed long ago; looking at them first
@@ -719,8 +746,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           if (kb > 0 && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
           HQ_TRACE(1, it);
           const uint32_t w_addr = tiles + s * stage_bytes;
-          uint64_t adesc = desc_hi | (uint64_t)((w_addr >> 4) & 0x3FFF);
-          uint64_t bdesc = desc_hi | (uint64_t)(((w_addr + w_bytes) >> 4) & 0x3FFF);
+          const uint32_t a_addr = p.wres ? tiles + p.wres_off + (uint32_t)kb * w_bytes : w_addr;
+          uint64_t adesc = desc_hi | (uint64_t)((a_addr >> 4) & 0x3FFF);
+          uint64_t bdesc = desc_hi | (uint64_t)(((w_addr + x_off) >> 4) & 0x3FFF);
           for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
             mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
           HQ_TRACE(5, it);
@@ -967,18 +995,21 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   // (measured: the pair shape wins on the fused-residual expansions, whose epilogue is the longest per tile,
   // and loses where a tile carries little epilogue work, e.g. 64 output channels)
   bool pair = k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
-  int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0;
+  int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0, wres_bytes = 0;
   if (pair) {
     // 128-pixel tiles, two accumulator buffers (256 columns), K blocks of at most 64 bytes
     if (p.bkb > 64) { p.bkb = 64; p.cchunks = a.cin / p.bkb; p.k_blocks = a.kh * a.kw * p.cchunks; }
     p.pt = pick_pt(P, p.c_tiles, 2 * h->sm_count, 128);
-    stage_bytes = (kTileC + p.pt) * p.bkb;
+    wres_bytes = p.k_blocks * kTileC * p.bkb;
+    p.wres = wres_bytes <= 16 * 1024 ? 1 : 0;              // short reductions: the weight slab stays resident
+    if (!p.wres) wres_bytes = 0;
+    stage_bytes = ((p.wres ? 0 : kTileC) + p.pt) * p.bkb;
     p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
     p.halves = 1;
     p.lg_bufs = 1;
     out_tile_bytes = p.staged_out ? kPairEpilogueWarps * p.pt * 32 : 0;
     res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-    stages = (110 * 1024 - out_tile_bytes - 2 * res_tile_bytes) / stage_bytes;
+    stages = (110 * 1024 - out_tile_bytes - 2 * res_tile_bytes - wres_bytes) / stage_bytes;
     if (stages < 3 || p.pt < 128) pair = false;
   }
   if (!pair) {
@@ -989,13 +1020,18 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
     for (int cap = 256; cap >= 64; cap >>= 1) {        // largest pixel tile that leaves room for >= 3 stages
       p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
-      stage_bytes = (kTileC + p.pt) * p.bkb;
+      // a weight slab of at most 72 KiB stays resident (the stages then hold activations only): a third less
+      // traffic into shared memory per K block
+      wres_bytes = p.k_blocks * kTileC * p.bkb;
+      p.wres = wres_bytes <= 72 * 1024 ? 1 : 0;
+      if (!p.wres) wres_bytes = 0;
+      stage_bytes = ((p.wres ? 0 : kTileC) + p.pt) * p.bkb;
       p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
       p.halves = p.pt >= (p.fold ? 256 : 128) ? 2 : 1;
       out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
       p.lg_bufs = p.pt <= 128 ? 2 : 1;
       res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-      stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs)) / stage_bytes;
+      stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs) - wres_bytes) / stage_bytes;
       if (stages >= 3 || p.pt == 64) break;
     }
   }
@@ -1007,6 +1043,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.stages = stages;
   p.out_stage_off = (uint32_t)(stages * stage_bytes);             // all pieces are multiples of 1024 bytes
   p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
+  p.wres_off = p.res_stage_off + ((uint32_t)res_tile_bytes << p.lg_bufs);
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
@@ -1062,7 +1099,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_bufs) + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_bufs) + wres_bytes + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int slots = pair ? 2 * h->sm_count : h->sm_count;
