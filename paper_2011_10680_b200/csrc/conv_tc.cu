@@ -992,9 +992,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.staged_res = (p.staged_out && a.res && a.res_bits == 8 && a.cout % 16 == 0) ? 1 : 0;
   // Launch shape: pair (two CTAs per SM) for short reductions when the tile pipeline fits half an SM.
   const long long k_total = (long long)a.kh * a.kw * a.cin;
-  // (measured: the pair shape wins on the fused-residual expansions, whose epilogue is the longest per tile,
-  // and loses where a tile carries little epilogue work, e.g. 64 output channels)
-  bool pair = k_total <= 256 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
+  // (measured: with the weight slab resident the one-CTA shape catches up for K >= 128; the pair shape still
+  // wins on the fused-residual expansions with the shortest reduction, and loses where a tile carries little
+  // epilogue work, e.g. 64 output channels)
+  bool pair = k_total <= 64 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
   int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0, wres_bytes = 0;
   if (pair) {
     // 128-pixel tiles, two accumulator buffers (256 columns), K blocks of at most 64 bytes
