@@ -120,6 +120,7 @@ struct hq_network {
   int32_t batch, image_h, image_w, image_c, image_signed;
   int32_t launches;
   std::vector<void*> res_narrow;     // per conv layer with a fused 8-bit residual: its narrow residual pairs (owned)
+  std::vector<void*> narrow0, narrow1; // per ADD / REQUANT layer with 8-bit operands: narrow pairs of the two branches (owned)
   std::vector<void*> wgt_widened;    // per 4-bit conv layer on the tensor-core path: its weights, one byte per value (owned)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
@@ -206,8 +207,9 @@ hq_status hq_linear(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, hq
   return conv_common(h, in, d, out, stream);
 }
 
-hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, const hq_tensor* res, hq_dyadic rr,
-                          int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream) {
+static hq_status residual_add_impl(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, const hq_tensor* res, hq_dyadic rr,
+                                   int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream,
+                                   const void* m_narrow, const void* r_narrow) {
   if (!h) return HQ_ERR_INVALID_ARG;
   hq_status st = check_tensor(main_t, true, true, true);
   if (st != HQ_OK) return st;
@@ -227,7 +229,13 @@ hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, c
   a.main_t = main_t->data; a.main_bits = main_t->bits; a.main_signed = main_t->is_signed; a.mb = mr.b; a.mc = mr.c;
   a.pixels = (long long)out->n * out->h * out->w; a.ch = out->c;
   a.relu = relu; a.qmin = qmin; a.qmax = qmax; a.out = out->data; a.out_bits = out->bits;
+  a.m_narrow = m_narrow; a.r_narrow = r_narrow;
   return hq_launch_residual_add(a, h->sm_count, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, const hq_tensor* res, hq_dyadic rr,
+                          int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream) {
+  return residual_add_impl(h, main_t, mr, res, rr, relu, qmin, qmax, out, stream, nullptr, nullptr);
 }
 
 hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic r, int32_t qmin, int32_t qmax,
@@ -278,6 +286,8 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   net->bytes.resize(n_layers);
   net->res_narrow.assign(n_layers, nullptr);
   net->wgt_widened.assign(n_layers, nullptr);
+  net->narrow0.assign(n_layers, nullptr);
+  net->narrow1.assign(n_layers, nullptr);
   net->launches = n_layers;
   hq_status st = HQ_OK;
   auto shape_of = [&](int id, hq_tensor* t) -> bool {
@@ -362,6 +372,26 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     if (hq_launch_residual_narrow(l.conv.res_rescale.b, l.conv.res_rescale.c, net->outs[l.in1].is_signed, l.conv.cout,
                                   buf, nullptr) != cudaSuccess) st = HQ_ERR_CUDA;
   }
+  // ... and of the 8-bit branches of ADD / REQUANT layers
+  for (int i = 0; st == HQ_OK && i < n_layers; ++i) {
+    const hq_layer& l = net->layers[i];
+    if (l.op != HQ_OP_ADD && l.op != HQ_OP_REQUANT) continue;
+    const hq_tensor& t0 = (l.in0 >= 0) ? net->outs[l.in0] : net->outs[i];
+    const int bits0 = l.in0 >= 0 ? t0.bits : 8, sgn0 = l.in0 >= 0 ? t0.is_signed : image_signed;
+    const int ch = net->outs[i].c;
+    if (bits0 != 8 || !l.rescale0.b || !l.rescale0.c) continue;
+    if (l.op == HQ_OP_ADD && (l.in1 < 0 || net->outs[l.in1].bits != 8 || !l.rescale1.b || !l.rescale1.c)) continue;
+    void* buf = nullptr;
+    if (cudaMalloc(&buf, (size_t)ch * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+    net->narrow0[i] = buf;
+    if (hq_launch_residual_narrow(l.rescale0.b, l.rescale0.c, sgn0, ch, buf, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
+    if (l.op == HQ_OP_ADD) {
+      void* buf1 = nullptr;
+      if (cudaMalloc(&buf1, (size_t)ch * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+      net->narrow1[i] = buf1;
+      if (hq_launch_residual_narrow(l.rescale1.b, l.rescale1.c, net->outs[l.in1].is_signed, ch, buf1, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
+    }
+  }
   if (st == HQ_OK && cudaDeviceSynchronize() != cudaSuccess) st = HQ_ERR_CUDA;
   if (st != HQ_OK) { hq_network_destroy(net); return st; }
   *out = net;
@@ -394,12 +424,12 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
       case HQ_OP_ADD: {
         if (l.in1 < 0) return HQ_ERR_INVALID_ARG;
         hq_tensor res = net->outs[l.in1];
-        st = hq_residual_add(h, &in, l.rescale0, &res, l.rescale1, l.relu, l.qmin, l.qmax, &o, s);
+        st = residual_add_impl(h, &in, l.rescale0, &res, l.rescale1, l.relu, l.qmin, l.qmax, &o, s, net->narrow0[i], net->narrow1[i]);
         break;
       }
       case HQ_OP_REQUANT: {
         hq_dyadic none{nullptr, nullptr};
-        st = hq_residual_add(h, &in, l.rescale0, nullptr, none, l.relu, l.qmin, l.qmax, &o, s);
+        st = residual_add_impl(h, &in, l.rescale0, nullptr, none, l.relu, l.qmin, l.qmax, &o, s, net->narrow0[i], nullptr);
         break;
       }
       default: return HQ_ERR_INVALID_ARG;
@@ -490,6 +520,8 @@ hq_status hq_network_destroy(hq_network* net) {
   for (auto& t : net->outs) if (t.data) cudaFree(t.data);
   for (void* q : net->res_narrow) if (q) cudaFree(q);
   for (void* q : net->wgt_widened) if (q) cudaFree(q);
+  for (void* q : net->narrow0) if (q) cudaFree(q);
+  for (void* q : net->narrow1) if (q) cudaFree(q);
   if (net->scratch) cudaFree(net->scratch);
   delete net;
   return HQ_OK;

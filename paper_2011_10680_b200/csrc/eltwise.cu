@@ -111,13 +111,26 @@ __device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` =
 
 // One pixel's word of four channels.  SLOW: one of the thread's channels has a shift below 9 (64-bit form).
 // SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing).
-template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP>
+// 8-bit value i of a word, zero- or sign-extended (one byte-permute either way: selector bit 3 replicates the
+// selected byte's sign bit).
+template <bool SIGNED>
+__device__ __forceinline__ int byte_of(unsigned w, int i) {
+  const unsigned sx = 8u | (unsigned)i;
+  return SIGNED ? (int)__byte_perm(w, 0u, (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)i)
+                : (int)__byte_perm(w, 0u, 0x4440u | (unsigned)i);
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW = false>
 __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, unsigned mw,
                                               unsigned rw, long long idx, int lo, int hi) {
   int s[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    if (!SLOW) {
+    if (NARROW) {
+      // Dy8 holds a narrow pair (b = m, h = a, sh = s): (q*m + a) >> s equals dn(q, b, c) for every 8-bit q
+      s[i] = (byte_of<MSIGNED>(mw, i) * m[i].b + m[i].h) >> m[i].sh;
+      if (RES) s[i] += (byte_of<RSIGNED>(rw, i) * r[i].b + r[i].h) >> r[i].sh;
+    } else if (!SLOW) {
       s[i] = dn8<MSIGNED>(__byte_perm(mw, 0u, 0x0444u | ((unsigned)i << 12)), m[i]);
       if (RES) s[i] += dn8<RSIGNED>(__byte_perm(rw, 0u, 0x0444u | ((unsigned)i << 12)), r[i]);
     } else {
@@ -152,27 +165,31 @@ __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4
   }
 }
 
-template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP>
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW = false>
 __device__ __forceinline__ void requant8_pixels(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, int words,
                                                 int lo, int hi) {
   const unsigned* mp = (const unsigned*)a.main_t;
   const unsigned* rp = (const unsigned*)a.res;
-  const long long step = (long long)gridDim.y * blockDim.y;
-  constexpr int U = 4;                     // pixels (independent 4-byte loads) in flight per thread
-  long long p = (long long)blockIdx.y * blockDim.y + threadIdx.y;
-  for (; p + (U - 1) * step < a.pixels; p += U * step) {
-    unsigned mw[U], rw[U];
+  constexpr int U = RES ? 4 : 8;            // pixels (independent 4-byte loads) in flight per thread
+  // A block walks runs of U * blockDim.y consecutive pixels: contiguous bytes per trip, friendly to DRAM pages.
+  const long long run = (long long)U * blockDim.y, trip = run * gridDim.y;
+  for (long long p0 = (long long)blockIdx.y * run + threadIdx.y; p0 < a.pixels; p0 += trip) {
+    if (p0 + (long long)(U - 1) * blockDim.y < a.pixels) {
+      unsigned mw[U], rw[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) mw[u] = __ldg(mp + (p + u * step) * words + wx);
+      for (int u = 0; u < U; ++u) mw[u] = __ldg(mp + (p0 + (long long)u * blockDim.y) * words + wx);
 #pragma unroll
-    for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rp + (p + u * step) * words + wx) : 0u;
+      for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rp + (p0 + (long long)u * blockDim.y) * words + wx) : 0u;
 #pragma unroll
-    for (int u = 0; u < U; ++u)
-      requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP>(a, m, r, wx, mw[u], rw[u], (p + u * step) * words + wx, lo, hi);
+      for (int u = 0; u < U; ++u)
+        requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, mw[u], rw[u],
+                                                                       (p0 + (long long)u * blockDim.y) * words + wx, lo, hi);
+    } else {
+      for (long long p = p0; p < a.pixels; p += blockDim.y)
+        requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, __ldg(mp + p * words + wx),
+                                                                       RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx, lo, hi);
+    }
   }
-  for (; p < a.pixels; p += step)
-    requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP>(a, m, r, wx, __ldg(mp + p * words + wx),
-                                                           RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx, lo, hi);
 }
 
 template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
@@ -189,6 +206,22 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
   bool slow = false;                       // a shift below 9 on one of this thread's channels: 64-bit form for the thread
 #pragma unroll
   for (int i = 0; i < 4; ++i) slow = slow || m[i].c < 9 || (RES && r[i].c < 9);
+  // narrow pairs prepared by the caller: usable when every channel of this thread has one
+  if (a.m_narrow && (!RES || a.r_narrow)) {
+    Dy8 nm[4], nr[4];
+    bool ok = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int4 pm = __ldg((const int4*)a.m_narrow + 4 * wx + i);
+      nm[i].b = pm.x; nm[i].h = pm.y; nm[i].sh = pm.z; nm[i].c = 0; ok = ok && pm.w != 0;
+      nr[i] = nm[i];
+      if (RES) {
+        const int4 pr = __ldg((const int4*)a.r_narrow + 4 * wx + i);
+        nr[i].b = pr.x; nr[i].h = pr.y; nr[i].sh = pr.z; ok = ok && pr.w != 0;
+      }
+    }
+    if (ok) { requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, words, lo, hi); return; }
+  }
   // two separate loops, so that the common one carries none of the 64-bit form's instructions
   if (slow) requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, words, lo, hi);
   else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, words, lo, hi);

@@ -70,6 +70,8 @@ struct EltArgs {
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   long long pixels; int32_t ch; int32_t relu, qmin, qmax;
   void* out; int32_t out_bits;
+  // optional narrow pairs {m, a, s, valid} per channel for 8-bit operands (see hq_launch_residual_narrow), or NULL
+  const void* m_narrow; const void* r_narrow;
 };
 
 cudaError_t hq_launch_conv_cuda_core(const ConvArgs& a, cudaStream_t s);
