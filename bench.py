@@ -211,6 +211,74 @@ def run_sweep(args):
     hq.close()
 
 
+def run_sweep_grid(args):
+    """Config 5 as a full grid: M in {3136, 12544, 50176, 200704} (= batch x H x W of a ResNet stage), N in
+    {64 .. 2048}, K in {64 (1x1, Cin 64), 576 / 1152 / 2304 / 4608 (3x3, Cin 64 / 128 / 256 / 512)}, INT8 and INT4
+    operands, epilogue with and without the residual add: 480 points.  Inputs are drawn on the device (timing only;
+    parity of these shapes is the tests' job).  Per point: device time, integer TOPS, GB/s of the algorithmic bytes,
+    fraction of the point's own roofline."""
+    import torch
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    hq = binding.Handle(0)
+    hbm_peak, bf16_peak, peak_kind = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    ri = lambda lo, hi, shape, dt: torch.randint(lo, hi, shape, generator=g, device="cuda", dtype=torch.int32).to(dt)
+    rows = []
+    for (kk, cin, k, hw) in ((64, 64, 1, 56), (576, 64, 3, 56), (1152, 128, 3, 28), (2304, 256, 3, 14), (4608, 512, 3, 7)):
+        for m in (3136, 12544, 50176, 200704):
+            n = m // (hw * hw)
+            for cout in (64, 128, 256, 512, 1024, 2048):
+                for bits in (8, 4):
+                    for residual in (False, True):
+                        per = 8 // bits
+                        x = ri(0, 256, (n, hw, hw, cin // per), torch.uint8)
+                        w = ri(-128, 128, (cout, k, k, cin // per), torch.int8)
+                        bias = ri(-(1 << 15), 1 << 15, (cout,), torch.int32)
+                        b = ri(1 << 30, (1 << 31) - 1, (cout,), torch.int32)
+                        lo_c = 36 + int(np.log2(kk)) // 2 - (8 if bits == 4 else 0)
+                        c = ri(lo_c, lo_c + 4, (cout,), torch.int32)
+                        res = ri(0, 256, (n, hw, hw, cout), torch.uint8) if residual else None
+                        rb = ri(1 << 30, (1 << 31) - 1, (cout,), torch.int32) if residual else None
+                        rc = ri(28, 35, (cout,), torch.int32) if residual else None
+                        out = torch.empty((n, hw, hw, cout), dtype=torch.uint8, device="cuda")
+                        times = []
+                        for rep in range(args.warmup + args.steps):
+                            flush.fill_(rep & 0xFF)
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record()
+                            st = hq.conv2d(x, bits, 0, cin, w, cout, k, k, 1, k // 2, bias, b, c, out, 8, 0,
+                                           res, 8 if residual else 0, 0, rb, rc, 1, 0, 255)
+                            e1.record()
+                            assert st == binding.HQ_OK, st
+                            torch.cuda.synchronize()
+                            if rep >= args.warmup:
+                                times.append(e0.elapsed_time(e1) * 1e3)
+                        us = float(np.median(times))
+                        ops = 2 * m * cout * kk
+                        byt = m * cin * bits // 8 + cout * kk * bits // 8 + m * cout + (m * cout if residual else 0) + 13 * cout
+                        t_ops, t_byt = ops / (NOMINAL_I8_TOPS * 1e12), byt / (hbm_peak * 1e9)
+                        rows.append(dict(M=m, N=cout, K=kk, bits=bits, residual=residual, us=round(us, 2), tops=round(ops / us / 1e6, 1),
+                                         gbs=round(byt / us / 1e3, 1), frac_of_own_roofline=round(max(t_ops, t_byt) * 1e6 / us, 3),
+                                         bound="tensor" if t_ops > t_byt else "hbm"))
+                        del x, w, res, out
+    hq.sync()
+    if args.layers_out:
+        json.dump(rows, open(args.layers_out, "w"), indent=1)
+    best = max(rows, key=lambda r: r["tops"])
+    med = lambda sel: float(np.median([r["frac_of_own_roofline"] for r in rows if sel(r)]))
+    big = lambda r: r["M"] == 200704 and r["bits"] == 8
+    print(json.dumps({"metric": "fused conv INT TOPS vs tcgen05 i8 peak (sweep grid)", "points": len(rows),
+                      "best_tops": best["tops"], "best_point": best,
+                      "median_frac_of_own_roofline": {"all": med(lambda r: True),
+                                                       "int8_M200704_tensor_bound": med(lambda r: big(r) and r["bound"] == "tensor"),
+                                                       "int8_M200704_hbm_bound": med(lambda r: big(r) and r["bound"] == "hbm")},
+                      "max_frac_of_i8_nominal": round(best["tops"] / NOMINAL_I8_TOPS, 3),
+                      "hbm_peak": hbm_peak, "peak_kind": f"of {peak_kind}", "i8_nominal_tops": NOMINAL_I8_TOPS}), flush=True)
+    hq.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -222,6 +290,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (JSON) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the fused conv/GEMM sweep (config 5) instead of the network")
+    ap.add_argument("--sweep-grid", action="store_true", help="run the full 480-point M x N x K x bits x residual grid of config 5")
     ap.add_argument("--sweep-pixels", type=int, default=200704, help="output pixels per sweep shape (batch is derived)")
     ap.add_argument("--sweep-only", type=int, default=-1, help="run a single sweep shape (index), e.g. for profiling")
     args = ap.parse_args()
@@ -232,6 +301,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.sweep_grid:
+        if rank == 0:
+            run_sweep_grid(args)
         return
     if args.sweep:
         if rank == 0:

@@ -65,6 +65,7 @@ struct TcParams {
   uint32_t wres_off;     // its offset from the 1024-aligned dynamic base
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
+  int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
   int32_t x_tiled;       // 1: X is a dense [P][cin] matrix (1x1, stride 1, no padding) fetched by a tiled map
@@ -334,7 +335,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   uint8_t* const my_stage_ptr = e.smem_raw + (my_stage - e.raw);
   const uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
   const int nchunks = px_per_warp >> 5;           // 2 or 4
-  const uint32_t bmask = (1u << p.lg_bufs) - 1u;
+  const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
   const int tile_step = e.p_step;
   int p_tile = e.p_tile0;
   if (p_tile >= p.p_tiles) return;
@@ -368,9 +369,10 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   bool pending = true;                            // a tensor-memory load into va is in flight
   while (true) {
     if (lane == 0) HQ_TRACE(3, tcount * 8 + e.ew);
-    if (RES && !wait_bar(&ctl.rfull[as], aph)) break;
+    const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;       // residual buffer and its phase
+    if (RES && !wait_bar(&ctl.rfull[rs], rph)) break;
     const int p_base = p_tile * p.pt + col0;
-    const uint8_t* const res_tile = res_stage_ptr + as * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
+    const uint8_t* const res_tile = res_stage_ptr + rs * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
     const uint32_t t_addr = t_warp + as * p.pt;
     const bool has_next = p_tile + tile_step < p.p_tiles;
     const uint32_t nas = (tcount + 1u) & bmask, naph = ((tcount + 1u) >> p.lg_bufs) & 1u;
@@ -401,7 +403,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     }
     if (RES) {                                    // every lane has used its last residual bytes of this tile
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctl.rempty[as]));
+      if (lane == 0) mbar_arrive(smem_u32(&ctl.rempty[rs]));
     }
     // Only now wait for the group's next tile: its copies may be queued behind the buffers released above.
     if (e.ew == 0 && lane == 0) HQ_TRACE(8, tcount);
@@ -447,19 +449,20 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
     uint32_t tcount = 0;
     for (int p_tile = p_tile0; p_tile < p.p_tiles; p_tile += p_step, ++tcount) {
       const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
+      const uint32_t rs = tcount & ((1u << p.lg_rbufs) - 1u), rph = (tcount >> p.lg_rbufs) & 1u;
       uint32_t w = 1;
       if (lane == 0) {
         if (p.staged_out) tma_store_wait_read0();   // the previous store has read this warp's staging box
         w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
         if (w && p.staged_res)
-          w = mbar_wait(smem_u32(&ctl.rfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+          w = mbar_wait(smem_u32(&ctl.rfull[rs]), rph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
       }
       w = __shfl_sync(0xffffffffu, w, 0);
       if (!w) break;
       tc_fence_after();                            // lane 0 observed the barriers; the shuffle ordered the warp
       if (ew == 0 && lane == 0) HQ_TRACE(3, tcount);
       const int p_base = p_tile * p.pt + col0;                          // first pixel of this warp's columns
-      const uint8_t* const res_tile = res_stage_ptr + as * res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
+      const uint8_t* const res_tile = res_stage_ptr + rs * res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
 
       for (int cc0 = 0; cc0 < px_per_warp; cc0 += 32) {
         int v[32];
@@ -568,7 +571,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(smem_u32(&ctl.tempty[as]));
-        if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[as]));
+        if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
         if (p.staged_out && warp_live && p_base < p.P) {
           tma_store_2d(&map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_base);
           tma_store_commit();
@@ -635,7 +638,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       // No division or modulo in this loop: one thread runs it and every dependent instruction
       // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
-      const uint32_t bmask = (1u << p.lg_bufs) - 1u;
+      const uint32_t rmask = (1u << p.lg_rbufs) - 1u;
+      // With as many residual buffers as accumulators the tile is fetched ahead of the operands; with fewer, beside
+      // the last operand block, when the epilogue of the tile before has long handed its buffer back.
+      const int res_kb = p.lg_rbufs < p.lg_bufs ? p.k_blocks - 1 : 0;
       bool ok = true;
       // (image, row, column) of the tile's first output pixel, advanced by a fixed step per tile
       const int ho = p.howo / p.wo;
@@ -659,19 +665,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
         const int p0 = p_tile * p.pt;
-        if (p.staged_res) {      // residual tile of this output tile, fetched ahead of the operands
-          const uint32_t rbuf = tcount & bmask, rph = (tcount >> p.lg_bufs) & 1u;
-          if (!mbar_wait(smem_u32(&ctl.rempty[rbuf]), rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-          const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
-          mbar_expect_tx(bar, res_tile_bytes);
-          tma_load_2d(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0);
-        }
         const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad, img_now = img;
         ow += d_ow; if (ow >= p.wo) { ow -= p.wo; ++oh; }
         oh += d_oh; if (oh >= ho) { oh -= ho; ++img; }
         img += d_img;
         int chunk = 0, tap_s = 0, tap_r = 0;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          if (p.staged_res && kb == res_kb) {   // residual tile of this output tile
+            const uint32_t rbuf = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
+            if (!mbar_wait(smem_u32(&ctl.rempty[rbuf]), rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+            const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
+            mbar_expect_tx(bar, res_tile_bytes);
+            tma_load_2d(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0);
+          }
           if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
           HQ_TRACE(0, it);
           const uint32_t bar = smem_u32(&ctl.full[s]);
@@ -711,11 +717,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
       if (p.staged_res) {
-        const uint32_t tiles_done = tcount < bmask + 1u ? tcount : bmask + 1u;
+        const uint32_t tiles_done = tcount < rmask + 1u ? tcount : rmask + 1u;
         for (uint32_t j = 0; j < tiles_done; ++j) {
           const uint32_t k = tcount - 1 - j;
           const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(smem_u32(&ctl.rfull[k & bmask]), (k >> p.lg_bufs) & 1u)) {
+          while (!mbar_try_wait(smem_u32(&ctl.rfull[k & rmask]), (k >> p.lg_rbufs) & 1u)) {
             if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
           }
         }
@@ -1008,6 +1014,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
     p.halves = 1;
     p.lg_bufs = 1;
+    p.lg_rbufs = 1;
     out_tile_bytes = p.staged_out ? kPairEpilogueWarps * p.pt * 32 : 0;
     res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
     stages = (110 * 1024 - out_tile_bytes - 2 * res_tile_bytes - wres_bytes) / stage_bytes;
@@ -1032,7 +1039,12 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
       out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
       p.lg_bufs = p.pt <= 128 ? 2 : 1;
       res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-      stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_bufs) - wres_bytes) / stage_bytes;
+      // residual tiles: as many buffers as accumulators, fewer when a long reduction needs the room for stages
+      // (its epilogue has slack: a single residual buffer only delays the next tile's prefetch)
+      for (p.lg_rbufs = p.lg_bufs; ; --p.lg_rbufs) {
+        stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_rbufs) - wres_bytes) / stage_bytes;
+        if (stages >= 3 || p.lg_rbufs == 0 || !res_tile_bytes || k_total < 1024) break;
+      }
       if (stages >= 3 || p.pt == 64) break;
     }
   }
@@ -1044,7 +1056,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.stages = stages;
   p.out_stage_off = (uint32_t)(stages * stage_bytes);             // all pieces are multiples of 1024 bytes
   p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
-  p.wres_off = p.res_stage_off + ((uint32_t)res_tile_bytes << p.lg_bufs);
+  p.wres_off = p.res_stage_off + ((uint32_t)res_tile_bytes << p.lg_rbufs);
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
@@ -1100,7 +1112,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_bufs) + wres_bytes + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_rbufs) + wres_bytes + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int slots = pair ? 2 * h->sm_count : h->sm_count;

@@ -96,6 +96,7 @@ TC_CASES = [
     (17, 56, 56, 64, 256, 1, 1, 0, 8, True, 8, True),        # two CTAs per SM (fused residual, short K), ragged last tile
     (21, 28, 28, 128, 512, 1, 1, 0, 8, True, 8, False),      # two CTAs per SM with 64-byte K blocks cut from cin = 128, signed out
     (9, 28, 28, 128, 128, 3, 1, 1, 8, False, 8, True),       # 256-pixel tiles, long K, one CTA per SM
+    (9, 28, 28, 128, 256, 3, 1, 1, 8, True, 8, True),        # 256-pixel tiles, long K, residual through a single staging tile
 ]
 
 
