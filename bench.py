@@ -211,6 +211,68 @@ def run_sweep(args):
     hq.close()
 
 
+def run_membound(args):
+    """The memory-bound kernels on their own, at ResNet-50 batch-256 tensor sizes (each operand larger than L2):
+    max pooling, dyadic requantization, the two-branch residual add and the average-pool requantization.  Device
+    time per call (CUDA events, 256 MB written between repetitions), achieved GB/s of the algorithmic bytes
+    (every operand read once, the result written once) and its fraction of the measured copy bandwidth."""
+    import torch
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    hq = binding.Handle(0)
+    hbm_peak, _, peak_kind = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    ri = lambda lo, hi, shape, dt: torch.randint(lo, hi, shape, generator=g, device="cuda", dtype=torch.int32).to(dt)
+    u8 = lambda *shape: ri(0, 256, shape, torch.uint8)
+    dy = lambda ch, lo, hi: (ri(1 << 30, (1 << 31) - 1, (ch,), torch.int32), ri(lo, hi, (ch,), torch.int32))
+    n = args.batch or 256
+    cases = []
+
+    x = u8(n, 112, 112, 64); o = torch.empty((n, 56, 56, 64), dtype=torch.uint8, device="cuda")
+    cases.append(("maxpool 3x3/2 u8 [%d,112,112,64]" % n, x.numel() + o.numel(),
+                  lambda x=x, o=o: hq.maxpool(x, 64, 0, 3, 2, 1, o)))
+    ch = 256
+    m = u8(n, 56, 56, ch); r = u8(n, 56, 56, ch); o = torch.empty_like(m)
+    mb, mc = dy(ch, 30, 33); rb, rc = dy(ch, 30, 33)
+    cases.append(("requant u8->u8 [%d,56,56,256]" % n, 2 * m.numel(),
+                  lambda m=m, o=o: hq.residual_add(m, 8, 0, mb, mc, None, 0, 0, None, None, ch, 1, 0, 255, o, 8, 0)))
+    cases.append(("add u8+u8->u8 [%d,56,56,256]" % n, 3 * m.numel(),
+                  lambda m=m, r=r, o=o: hq.residual_add(m, 8, 0, mb, mc, r, 8, 0, rb, rc, ch, 1, 0, 255, o, 8, 0)))
+    o4 = torch.empty((n, 56, 56, ch // 2), dtype=torch.uint8, device="cuda")
+    cases.append(("requant u8->u4 [%d,56,56,256]" % n, m.numel() + o4.numel(),
+                  lambda m=m, o4=o4: hq.residual_add(m, 8, 0, mb, mc, None, 0, 0, None, None, ch, 1, 0, 15, o4, 4, 0)))
+    a32 = ri(-(1 << 20), 1 << 20, (n, 56, 56, 64), torch.int32); o32 = torch.empty((n, 56, 56, 64), dtype=torch.uint8, device="cuda")
+    b32, c32 = dy(64, 44, 48)
+    cases.append(("requant s32->u8 [%d,56,56,64]" % n, 5 * a32.numel(),
+                  lambda: hq.residual_add(a32, 32, 1, b32, c32, None, 0, 0, None, None, 64, 1, 0, 255, o32, 8, 0)))
+    na = 8 * n
+    xa = u8(na, 7, 7, 2048); oa = torch.empty((na, 1, 1, 2048), dtype=torch.uint8, device="cuda")
+    ba, ca = dy(2048, 36, 38)
+    cases.append(("avgpool requant u8 [%d,7,7,2048]" % na, xa.numel() + oa.numel(),
+                  lambda: hq.avgpool_requant(xa, 2048, 8, 0, ba, ca, 0, 255, oa, 8, 0)))
+    rows = []
+    for name, byt, fn in cases:
+        times = []
+        for rep in range(args.warmup + args.steps):
+            flush.fill_(rep & 0xFF)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            st = fn()
+            e1.record()
+            assert st == binding.HQ_OK, (name, st)
+            torch.cuda.synchronize()
+            if rep >= args.warmup:
+                times.append(e0.elapsed_time(e1) * 1e3)
+        us = float(np.median(times))
+        rows.append(dict(kernel=name, bytes=int(byt), us=round(us, 2), gbs=round(byt / us / 1e3, 1),
+                         frac_of_hbm=round(byt / us / 1e3 / hbm_peak, 3)))
+    hq.sync()
+    print(json.dumps({"metric": "memory-bound kernels, achieved GB/s of algorithmic bytes", "hbm_peak": hbm_peak,
+                      "peak_kind": f"of {peak_kind}", "rows": rows}), flush=True)
+    hq.close()
+
+
 def run_sweep_grid(args):
     """Config 5 as a full grid: M in {3136, 12544, 50176, 200704} (= batch x H x W of a ResNet stage), N in
     {64 .. 2048}, K in {64 (1x1, Cin 64), 576 / 1152 / 2304 / 4608 (3x3, Cin 64 / 128 / 256 / 512)}, INT8 and INT4
@@ -291,6 +353,7 @@ def main():
     ap.add_argument("--layers-out", default=None, help="write the per-layer table (JSON) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the fused conv/GEMM sweep (config 5) instead of the network")
     ap.add_argument("--sweep-grid", action="store_true", help="run the full 480-point M x N x K x bits x residual grid of config 5")
+    ap.add_argument("--membound", action="store_true", help="time the memory-bound kernels (pooling, requantization, residual add) on their own")
     ap.add_argument("--sweep-pixels", type=int, default=200704, help="output pixels per sweep shape (batch is derived)")
     ap.add_argument("--sweep-only", type=int, default=-1, help="run a single sweep shape (index), e.g. for profiling")
     args = ap.parse_args()
@@ -305,6 +368,10 @@ def main():
     if args.sweep_grid:
         if rank == 0:
             run_sweep_grid(args)
+        return
+    if args.membound:
+        if rank == 0:
+            run_membound(args)
         return
     if args.sweep:
         if rank == 0:

@@ -359,30 +359,75 @@ __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int
 }
 
 // ---- max pooling ----------------------------------------------------------------------------
-// One block per (image, output row): no 64-bit index arithmetic per output (the division-heavy flat index
-// made an earlier version instruction-bound); a thread handles 16 channels of one output pixel at a time.
+// Byte-wise maxima run on the 16-bit pair instructions (a three-input max of two halfword pairs issues like
+// a plain integer instruction; the byte-wise intrinsics expand to long sequences): every loaded word is split
+// into its even and its odd bytes, widened to halfwords, and the pairs are merged again for the store.
 template <bool SIGNED>
+struct BytePairMax {
+  unsigned e, o;             // running maxima of bytes 0 / 2 and of bytes 1 / 3, one per halfword
+  __device__ __forceinline__ static unsigned even(unsigned w) { return __byte_perm(w, 0, SIGNED ? 0xA280 : 0x4240); }
+  __device__ __forceinline__ static unsigned odd(unsigned w) { return __byte_perm(w, 0, SIGNED ? 0xB391 : 0x4341); }
+  __device__ __forceinline__ void init(unsigned w) { e = even(w); o = odd(w); }
+  __device__ __forceinline__ void add(unsigned w) {
+    if (SIGNED) { e = __vmaxs2(e, even(w)); o = __vmaxs2(o, odd(w)); }
+    else        { e = __vmaxu2(e, even(w)); o = __vmaxu2(o, odd(w)); }
+  }
+  __device__ __forceinline__ void add2(unsigned w0, unsigned w1) {
+    if (SIGNED) { e = __vimax3_s16x2(e, even(w0), even(w1)); o = __vimax3_s16x2(o, odd(w0), odd(w1)); }
+    else        { e = __vimax3_u16x2(e, even(w0), even(w1)); o = __vimax3_u16x2(o, odd(w0), odd(w1)); }
+  }
+  __device__ __forceinline__ unsigned merged() const { return __byte_perm(e, o, 0x6240); }
+};
+
+// One block per (image, output row): no 64-bit index arithmetic per output (a division-heavy flat index is
+// instruction-bound); a thread handles 16 channels of one output pixel at a time.  K3: the 3x3 window, fully
+// unrolled; rows and columns that fall into the padding are replaced by their nearest valid neighbour, which
+// lies inside the same window (pad < k) and leaves the maximum unchanged.
+template <bool SIGNED, bool K3>
 __global__ void __launch_bounds__(256) maxpool_vec16_kernel(const uint4* __restrict__ in, int h, int w, int cg,
                                                             int k, int stride, int pad, uint4* __restrict__ out, int ho, int wo) {
   const int img = blockIdx.x / ho, oh = blockIdx.x - img * ho;
   const uint4* in_img = in + (long long)img * h * w * cg;
   uint4* out_row = out + ((long long)img * ho + oh) * wo * cg;
-  const int r_lo = max(0, pad - oh * stride), r_hi = min(k, h + pad - oh * stride);   // valid filter rows
   const int row_items = wo * cg;
-  for (int idx = threadIdx.x; idx < row_items; idx += blockDim.x) {
-    const int ow = idx / cg, g = idx - ow * cg;
-    const int s_lo = max(0, pad - ow * stride), s_hi = min(k, w + pad - ow * stride);
-    const unsigned init = SIGNED ? 0x80808080u : 0u;
-    uint4 m = make_uint4(init, init, init, init);
-    for (int r = r_lo; r < r_hi; ++r) {
-      const uint4* row = in_img + ((long long)(oh * stride + r - pad) * w + (ow * stride - pad)) * cg + g;
-      for (int s = s_lo; s < s_hi; ++s) {
-        const uint4 v = __ldg(row + s * cg);
-        if (SIGNED) { m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y); m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w); }
-        else        { m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w); }
-      }
+  if (K3) {
+    const int ih1 = oh * stride - pad + 1;                       // centre row of the window
+    const int r0 = min(max(ih1 - 1, 0), h - 1), r1 = min(max(ih1, 0), h - 1), r2 = min(max(ih1 + 1, 0), h - 1);
+    const uint4* row0 = in_img + (long long)r0 * w * cg;
+    const uint4* row1 = in_img + (long long)r1 * w * cg;
+    const uint4* row2 = in_img + (long long)r2 * w * cg;
+    for (int idx = threadIdx.x; idx < row_items; idx += blockDim.x) {
+      const int ow = idx / cg, g = idx - ow * cg;
+      const int iw1 = ow * stride - pad + 1;
+      const int c0 = min(max(iw1 - 1, 0), w - 1) * cg + g, c1 = min(max(iw1, 0), w - 1) * cg + g,
+                c2 = min(max(iw1 + 1, 0), w - 1) * cg + g;
+      const uint4 v0 = __ldg(row0 + c0), v1 = __ldg(row0 + c1), v2 = __ldg(row0 + c2);
+      const uint4 v3 = __ldg(row1 + c0), v4 = __ldg(row1 + c1), v5 = __ldg(row1 + c2);
+      const uint4 v6 = __ldg(row2 + c0), v7 = __ldg(row2 + c1), v8 = __ldg(row2 + c2);
+      uint4 m;
+#define HQ_MAX9(F) { BytePairMax<SIGNED> a; a.init(v0.F); a.add2(v1.F, v2.F); a.add2(v3.F, v4.F); \
+                     a.add2(v5.F, v6.F); a.add2(v7.F, v8.F); m.F = a.merged(); }
+      HQ_MAX9(x) HQ_MAX9(y) HQ_MAX9(z) HQ_MAX9(w)
+#undef HQ_MAX9
+      out_row[idx] = m;
     }
-    out_row[idx] = m;
+  } else {
+    const int r_lo = max(0, pad - oh * stride), r_hi = min(k, h + pad - oh * stride);   // valid filter rows
+    for (int idx = threadIdx.x; idx < row_items; idx += blockDim.x) {
+      const int ow = idx / cg, g = idx - ow * cg;
+      const int s_lo = max(0, pad - ow * stride), s_hi = min(k, w + pad - ow * stride);
+      const unsigned init = SIGNED ? 0x80808080u : 0u;
+      BytePairMax<SIGNED> mx, my, mz, mw;
+      mx.init(init); my.init(init); mz.init(init); mw.init(init);
+      for (int r = r_lo; r < r_hi; ++r) {
+        const uint4* row = in_img + ((long long)(oh * stride + r - pad) * w + (ow * stride - pad)) * cg + g;
+        for (int s = s_lo; s < s_hi; ++s) {
+          const uint4 v = __ldg(row + s * cg);
+          mx.add(v.x); my.add(v.y); mz.add(v.z); mw.add(v.w);
+        }
+      }
+      out_row[idx] = make_uint4(mx.merged(), my.merged(), mz.merged(), mw.merged());
+    }
   }
 }
 
@@ -477,10 +522,16 @@ cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int i
                               int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
   if (ch % 16 == 0 && (long long)n * ho < (1ll << 31) && (long long)wo * (ch / 16) < (1ll << 31)) {
-    if (is_signed)
-      maxpool_vec16_kernel<true><<<n * ho, 256, 0, s>>>((const uint4*)in, h, w, ch / 16, k, stride, pad, (uint4*)out, ho, wo);
-    else
-      maxpool_vec16_kernel<false><<<n * ho, 256, 0, s>>>((const uint4*)in, h, w, ch / 16, k, stride, pad, (uint4*)out, ho, wo);
+    const uint4* src = (const uint4*)in;
+    uint4* dst = (uint4*)out;
+    const int cg = ch / 16;
+    // the unrolled 3x3 form: with pad <= 1 at most one row / column of a window lies outside the image, next to
+    // a valid one of the same window
+    const bool k3 = k == 3 && pad <= 1;
+    if (is_signed && k3) maxpool_vec16_kernel<true, true><<<n * ho, 256, 0, s>>>(src, h, w, cg, k, stride, pad, dst, ho, wo);
+    else if (is_signed)  maxpool_vec16_kernel<true, false><<<n * ho, 256, 0, s>>>(src, h, w, cg, k, stride, pad, dst, ho, wo);
+    else if (k3)         maxpool_vec16_kernel<false, true><<<n * ho, 256, 0, s>>>(src, h, w, cg, k, stride, pad, dst, ho, wo);
+    else                 maxpool_vec16_kernel<false, false><<<n * ho, 256, 0, s>>>(src, h, w, cg, k, stride, pad, dst, ho, wo);
   } else {
     const long long total = (long long)n * ho * wo * ch;
     long long blocks = (total + 255) / 256;

@@ -295,6 +295,26 @@ def test_maxpool(hq, n, h, w, ch):
     assert np.array_equal(host(out, ref), ref)
 
 
+@pytest.mark.parametrize("k,stride,pad", [(3, 2, 1), (3, 1, 1), (3, 2, 0), (3, 3, 1), (2, 2, 0), (5, 2, 2), (3, 1, 2)])
+@pytest.mark.parametrize("signed", [0, 1])
+def test_maxpool_windows_and_signedness(hq, k, stride, pad, signed):
+    # every window form of the vector kernel (unrolled 3x3 with replaced border taps, general loop), on odd
+    # extents, with values that include both ends of the type's range
+    from paper_2011_10680_b200 import binding
+    n, h, w, ch = 2, 13, 10, 48
+    g = inputs.rng(304, k, stride, pad, signed)
+    x = g.integers(0, 256, size=(n, h, w, ch), dtype=np.int64).astype(np.uint8)
+    x[0, :3] = 0x80 if signed else 0            # whole windows at the type's minimum
+    x[1, -3:] = 0x7F if signed else 0xFF
+    xs = x.view(np.int8) if signed else x
+    ref = oracle().maxpool(xs, k, stride, pad, signed)
+    out = binding.alloc_out(n, ref.shape[1], ref.shape[2], ch, 8, signed)
+    st = hq.maxpool(binding.to_device(xs), ch, signed, k, stride, pad, out)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
 # ------------------------------------------------------------------ argument errors ------------
 def test_invalid_arguments_return_codes_not_crashes(hq):
     from paper_2011_10680_b200 import binding
