@@ -166,6 +166,9 @@ hq_status hq_create(int32_t device, hq_handle** out) {
   if (!hq_conv_tc_init()) { delete h; return HQ_ERR_CUDA; }
   if (cudaMalloc(&h->dev_status, sizeof(uint32_t)) != cudaSuccess) { delete h; return HQ_ERR_WORKSPACE; }
   if (cudaMemset(h->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) { cudaFree(h->dev_status); delete h; return HQ_ERR_CUDA; }
+  if (cudaMalloc(&h->narrow_pairs, (size_t)2 * kNarrowChannels * 16) != cudaSuccess) {
+    cudaFree(h->dev_status); delete h; return HQ_ERR_WORKSPACE;
+  }
   *out = h;
   return HQ_OK;
 }
@@ -173,6 +176,7 @@ hq_status hq_create(int32_t device, hq_handle** out) {
 hq_status hq_destroy(hq_handle* h) {
   if (!h) return HQ_ERR_INVALID_ARG;
   cudaFree(h->dev_status);
+  cudaFree(h->narrow_pairs);
   if (h->workspace) cudaFree(h->workspace);
   delete h;
   return HQ_OK;
@@ -230,7 +234,22 @@ static hq_status residual_add_impl(hq_handle* h, const hq_tensor* main_t, hq_dya
   a.pixels = (long long)out->n * out->h * out->w; a.ch = out->c;
   a.relu = relu; a.qmin = qmin; a.qmax = qmax; a.out = out->data; a.out_bits = out->bits;
   a.m_narrow = m_narrow; a.r_narrow = r_narrow;
-  return hq_launch_residual_add(a, h->sm_count, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+  a.status = h->dev_status;
+  // A single large call on 8-bit operands: the narrow pairs of both branches are worked out first, in the handle's
+  // buffer (a network prepares them once when it is built).  One small launch that the cheaper arithmetic repays.
+  cudaStream_t s = (cudaStream_t)stream;
+  if (!m_narrow && main_t->bits == 8 && (!res || res->bits == 8) && out->c <= kNarrowChannels &&
+      a.pixels * a.ch >= (1ll << 25)) {
+    char* base = (char*)h->narrow_pairs;
+    if (hq_launch_residual_narrow(a.mb, a.mc, a.main_signed, a.ch, base, s) != cudaSuccess) return HQ_ERR_CUDA;
+    a.m_narrow = base;
+    if (res) {
+      if (hq_launch_residual_narrow(a.rb, a.rc, a.res_signed, a.ch, base + (size_t)kNarrowChannels * 16, s) != cudaSuccess)
+        return HQ_ERR_CUDA;
+      a.r_narrow = base + (size_t)kNarrowChannels * 16;
+    }
+  }
+  return hq_launch_residual_add(a, h->sm_count, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic mr, const hq_tensor* res, hq_dyadic rr,

@@ -866,31 +866,37 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 // ---------------------------------------------------------------- narrow residual pairs ------
 // The residual term dn(r, rb, rc) = (r*rb + 2^(rc-1)) >> rc (Section 3.3, Appendix G) has only 256 possible
 // inputs per channel.  For most (rb, rc) a 23-bit multiplier m ~ rb / 2^8 with s = rc - 8 and a = 2^(s-1)
-// gives (r*m + a) >> s == dn(r, rb, rc) for every one of them, and r*m + a fits 32 bits.  One thread per
+// gives (r*m + a) >> s == dn(r, rb, rc) for every one of them, and r*m + a fits 32 bits.  One warp per
 // channel tries the two neighbouring multipliers and checks all 256 inputs; channels without such a pair
-// are marked invalid and keep the wide form.  Run once per layer when a network is built.
-__global__ void residual_narrow_kernel(const int32_t* __restrict__ rb, const int32_t* __restrict__ rc, int is_signed,
-                                       int n, int4* __restrict__ out) {
-  const int ch = blockIdx.x * blockDim.x + threadIdx.x;
+// are marked invalid and keep the wide form.  Run once per layer when a network is built, and ahead of a
+// single large element-wise call.
+__global__ void __launch_bounds__(128) residual_narrow_kernel(const int32_t* __restrict__ rb, const int32_t* __restrict__ rc,
+                                                              int is_signed, int n, int4* __restrict__ out) {
+  // one warp per channel: lane l checks the inputs l, l + 32, ... for both candidate multipliers
+  const int ch = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (ch >= n) return;
   const long long b = rb[ch];
   const int c = rc[ch];
   int4 res = make_int4(0, 0, 0, 0);
-  const int r_lo = is_signed ? -128 : 0, r_hi = is_signed ? 127 : 255;
+  const int r_lo = is_signed ? -128 : 0;
   if (c >= 41 && c <= 62) {
     res = make_int4(0, 0, 0, 1);                       // |r*rb| < 2^39 <= 2^(rc-2): the term is 0 for every r
   } else if (c >= 9 && c <= 38) {
     const int s = c - 8, a = 1 << (s - 1);
-    for (int t = 0; t < 2 && !res.w; ++t) {
-      const long long m = (b >> 8) + t;
-      if (m > (1 << 23) || m < -(1 << 23)) continue;
-      bool same = true;
-      for (int r = r_lo; r <= r_hi && same; ++r)
-        same = (((long long)r * b + (1LL << (c - 1))) >> c) == (long long)((r * (int)m + a) >> s);
-      if (same) res = make_int4((int)m, a, s, 1);
+    const long long m0 = b >> 8, m1 = m0 + 1;
+    bool same0 = m0 <= (1 << 23), same1 = m1 <= (1 << 23);
+    for (int j = 0; j < 8; ++j) {
+      const int r = r_lo + lane + 32 * j;
+      const long long exact = ((long long)r * b + (1LL << (c - 1))) >> c;
+      same0 = same0 && exact == (long long)((r * (int)m0 + a) >> s);
+      same1 = same1 && exact == (long long)((r * (int)m1 + a) >> s);
     }
+    same0 = __all_sync(0xffffffffu, same0);
+    same1 = __all_sync(0xffffffffu, same1);
+    if (same0) res = make_int4((int)m0, a, s, 1);
+    else if (same1) res = make_int4((int)m1, a, s, 1);
   }
-  out[ch] = res;
+  if (lane == 0) out[ch] = res;
 }
 
 // ---------------------------------------------------------------- host side ------------------
@@ -1139,7 +1145,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
 cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
                                       cudaStream_t s) {
   if (channels <= 0) return cudaSuccess;
-  residual_narrow_kernel<<<(channels + 127) / 128, 128, 0, s>>>(rb, rc, res_signed, channels, (int4*)out);
+  residual_narrow_kernel<<<(channels + 3) / 4, 128, 0, s>>>(rb, rc, res_signed, channels, (int4*)out);
   return cudaGetLastError();
 }
 

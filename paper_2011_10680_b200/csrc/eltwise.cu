@@ -122,7 +122,7 @@ __device__ __forceinline__ int byte_of(unsigned w, int i) {
 
 template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW = false>
 __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, unsigned mw,
-                                              unsigned rw, long long idx, int lo, int hi) {
+                                              unsigned rw, void* dst, int lo, int hi) {
   int s[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -141,15 +141,24 @@ __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4
     }
   }
   if constexpr (!OUT4 && SATP != 0) {
-    unsigned w01, w;
+    // two saturating packs; the second carries the first one's halfword in its upper half: bytes s0 s1 s2 s3
+    unsigned w23, w;
     if (SATP == 1) {
-      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w01) : "r"(s[3]), "r"(s[2]), "r"(0));
-      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(0));
+      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(s[3]), "r"(s[2]), "r"(0));
+      asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(w23));
     } else {
-      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w01) : "r"(s[3]), "r"(s[2]), "r"(0));
-      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(0));
+      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(s[3]), "r"(s[2]), "r"(0));
+      asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(w23));
     }
-    ((unsigned*)a.out)[idx] = __byte_perm(w, w01, 0x5410);        // bytes: s0 s1 s2 s3
+    *(unsigned*)dst = w;
+  } else if constexpr (OUT4 && SATP == 3) {
+    // clamp to [0, 15]: upper bound by a minimum, lower bound by the saturating pack; then the four bytes'
+    // low nibbles move next to each other
+    unsigned w23, w;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(min(s[3], 15)), "r"(min(s[2], 15)), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(min(s[1], 15)), "r"(min(s[0], 15)), "r"(w23));
+    const unsigned t = w | (w >> 4);                       // byte 0 = s0 | s1 << 4, byte 2 = s2 | s3 << 4
+    *(unsigned short*)dst = (unsigned short)__byte_perm(t, 0u, 0x4420);
   } else {
     int y[4];
 #pragma unroll
@@ -157,12 +166,18 @@ __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4
     if (OUT4) {
       // 0 <= y <= 15 after the clamp of an unsigned 4-bit output; signed nibbles keep their low four bits
       const unsigned w = (unsigned)(y[0] & 0xF) + ((unsigned)(y[1] & 0xF) << 4) + ((unsigned)(y[2] & 0xF) << 8) + ((unsigned)(y[3] & 0xF) << 12);
-      ((unsigned short*)a.out)[idx] = (unsigned short)w;
+      *(unsigned short*)dst = (unsigned short)w;
     } else {
-      ((unsigned*)a.out)[idx] = (unsigned)(y[0] & 0xFF) | ((unsigned)(y[1] & 0xFF) << 8) | ((unsigned)(y[2] & 0xFF) << 16) |
-                                ((unsigned)(y[3] & 0xFF) << 24);
+      *(unsigned*)dst = (unsigned)(y[0] & 0xFF) | ((unsigned)(y[1] & 0xFF) << 8) | ((unsigned)(y[2] & 0xFF) << 16) |
+                        ((unsigned)(y[3] & 0xFF) << 24);
     }
   }
+}
+
+// Destination of word `idx` of the output (four channels: a 32-bit word at 8 bit, a 16-bit word at 4 bit).
+template <bool OUT4>
+__device__ __forceinline__ void* out_word(const EltArgs& a, long long idx) {
+  return OUT4 ? (void*)((unsigned short*)a.out + idx) : (void*)((unsigned*)a.out + idx);
 }
 
 template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW = false>
@@ -183,19 +198,55 @@ __device__ __forceinline__ void requant8_pixels(const EltArgs& a, const Dy8 (&m)
 #pragma unroll
       for (int u = 0; u < U; ++u)
         requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, mw[u], rw[u],
-                                                                       (p0 + (long long)u * blockDim.y) * words + wx, lo, hi);
+                                                                       out_word<OUT4>(a, (p0 + (long long)u * blockDim.y) * words + wx), lo, hi);
     } else {
       for (long long p = p0; p < a.pixels; p += blockDim.y)
         requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, __ldg(mp + p * words + wx),
-                                                                       RES ? __ldg(rp + p * words + wx) : 0u, p * words + wx, lo, hi);
+                                                                       RES ? __ldg(rp + p * words + wx) : 0u, out_word<OUT4>(a, p * words + wx), lo, hi);
     }
   }
 }
 
-template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
+// Flat form for channel counts whose words divide the block (words a power of two, at most 256): the tensor is
+// one array of 32-bit words, a block of 256 threads takes 256 consecutive words per step, so a thread keeps its
+// four channels (word index mod words is fixed) and every address is a per-trip base plus a constant.
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW = false>
+__device__ __forceinline__ void requant8_flat(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, long long total,
+                                              int lo, int hi) {
+  constexpr int T = 256, U = RES ? 4 : 8;           // words in flight per thread
+  const unsigned* mp = (const unsigned*)a.main_t + threadIdx.x;
+  const unsigned* rp = RES ? (const unsigned*)a.res + threadIdx.x : nullptr;
+  const long long trip = (long long)gridDim.x * (U * T);
+  for (long long base = (long long)blockIdx.x * (U * T); base < total; base += trip) {
+    const unsigned* mq = mp + base;
+    const unsigned* rq = RES ? rp + base : nullptr;
+    void* dst0 = out_word<OUT4>(a, base + threadIdx.x);
+    auto dst = [&](int u) { return OUT4 ? (void*)((unsigned short*)dst0 + u * T) : (void*)((unsigned*)dst0 + u * T); };
+    if (base + U * T <= total) {
+      unsigned mw[U], rw[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) mw[u] = __ldg(mq + u * T);
+#pragma unroll
+      for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rq + u * T) : 0u;
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, mw[u], rw[u], dst(u), lo, hi);
+    } else {
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (base + u * T + threadIdx.x < total)
+          requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, __ldg(mq + u * T),
+                                                                         RES ? __ldg(rq + u * T) : 0u, dst(u), lo, hi);
+    }
+  }
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP, bool FLAT>
 __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int lo, int hi) {
-  const int wx = blockIdx.x * blockDim.x + threadIdx.x;     // word (4 channels) of the pixel
+  // word (4 channels) of the pixel
+  const int wx = FLAT ? (int)(threadIdx.x & (unsigned)(words - 1)) : (int)(blockIdx.x * blockDim.x + threadIdx.x);
   if (wx >= words) return;
+  const long long total = a.pixels * words;
   Dy8 m[4], r[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -220,20 +271,41 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
         nr[i].b = pr.x; nr[i].h = pr.y; nr[i].sh = pr.z; ok = ok && pr.w != 0;
       }
     }
-    if (ok) { requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, words, lo, hi); return; }
+    if (ok) {
+      if (FLAT) requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, total, lo, hi);
+      else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, words, lo, hi);
+      return;
+    }
   }
   // two separate loops, so that the common one carries none of the 64-bit form's instructions
-  if (slow) requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, words, lo, hi);
-  else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, words, lo, hi);
+  if (FLAT) {
+    if (slow) requant8_flat<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, total, lo, hi);
+    else requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, total, lo, hi);
+  } else {
+    if (slow) requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, words, lo, hi);
+    else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, words, lo, hi);
+  }
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
+cudaError_t launch_requant8_form(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, int sm_count, cudaStream_t s) {
+  if (words <= 256 && (words & (words - 1)) == 0) {
+    const long long total = a.pixels * words, per_block = 256 * (RES ? 4 : 8);
+    const long long blocks = (total + per_block - 1) / per_block, cap = (long long)sm_count * 16;
+    requant8_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP, true><<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(a, words, lo, hi);
+  } else {
+    requant8_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP, false><<<grid, block, 0, s>>>(a, words, lo, hi);
+  }
+  return cudaGetLastError();
 }
 
 template <bool RES, bool MSIGNED, bool RSIGNED>
-cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, cudaStream_t s) {
-  if (a.out_bits == 4) requant8_kernel<RES, MSIGNED, RSIGNED, true, 0><<<grid, block, 0, s>>>(a, words, lo, hi);
-  else if (lo == 0 && hi == 255) requant8_kernel<RES, MSIGNED, RSIGNED, false, 1><<<grid, block, 0, s>>>(a, words, lo, hi);
-  else if (lo == -128 && hi == 127) requant8_kernel<RES, MSIGNED, RSIGNED, false, 2><<<grid, block, 0, s>>>(a, words, lo, hi);
-  else requant8_kernel<RES, MSIGNED, RSIGNED, false, 0><<<grid, block, 0, s>>>(a, words, lo, hi);
-  return cudaGetLastError();
+cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, int sm_count, cudaStream_t s) {
+  if (a.out_bits == 4 && lo == 0 && hi == 15) return launch_requant8_form<RES, MSIGNED, RSIGNED, true, 3>(a, grid, block, words, lo, hi, sm_count, s);
+  if (a.out_bits == 4) return launch_requant8_form<RES, MSIGNED, RSIGNED, true, 0>(a, grid, block, words, lo, hi, sm_count, s);
+  if (lo == 0 && hi == 255) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 1>(a, grid, block, words, lo, hi, sm_count, s);
+  if (lo == -128 && hi == 127) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 2>(a, grid, block, words, lo, hi, sm_count, s);
+  return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 0>(a, grid, block, words, lo, hi, sm_count, s);
 }
 
 // Any channel count: one thread per output byte (one element at 8 bit, two at 4 bit).
@@ -336,6 +408,60 @@ __global__ void __launch_bounds__(256) avgpool_vec4_sliced_kernel(const unsigned
     w |= (unsigned)(q & 0xFF) << (8 * j);
   }
   out[(long long)img * cg + g] = w;
+}
+
+// 16 channels per thread (one 16-byte load per pixel), 8 pixel slices per block, four loads of a thread in flight
+// at a time; 512 channels per block.  Bytes are summed as 16-bit lanes (h*w*255 <= 65535, i.e. up to 257 pixels;
+// signed bytes are offset by 128 and corrected at the end).  The slices meet in shared memory and every thread
+// then finishes two channels.
+constexpr int kAvgSlices = 8;
+__global__ void __launch_bounds__(256) avgpool_vec16_kernel(const uint4* __restrict__ in, int hw, int ch, int is_signed,
+                                                            const int32_t* __restrict__ b, const int32_t* __restrict__ c,
+                                                            int qmin, int qmax, unsigned short* __restrict__ out) {
+  __shared__ unsigned part[kAvgSlices][8][32];        // [slice][even / odd byte sums of the four words][channel group]
+  const int cg = ch >> 4;
+  const int g = blockIdx.x * 32 + threadIdx.x, img = blockIdx.y;
+  // thread t finishes channels 2t and 2t+1 of the block's 512: group t / 8, word (t % 8) / 2, bytes 2 * (t % 2) + {0, 1}
+  const int t = threadIdx.y * 32 + threadIdx.x;
+  const int gl = t >> 3, word = (t & 7) >> 1, half = t & 1;
+  const int ch0 = (blockIdx.x * 32 + gl) * 16 + word * 4 + half * 2;
+  int2 bb = make_int2(0, 0), cc = make_int2(1, 1);
+  if (ch0 < ch) {                                    // fetched first: their latency hides behind the pixels'
+    bb = make_int2(__ldg(b + ch0), __ldg(b + ch0 + 1));
+    cc = make_int2(__ldg(c + ch0), __ldg(c + ch0 + 1));
+  }
+  unsigned acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (g < cg) {
+    const uint4* p = in + (long long)img * hw * cg + g;
+    const unsigned flip = is_signed ? 0x80808080u : 0u;
+    for (int k0 = threadIdx.y; k0 < hw; k0 += 4 * kAvgSlices) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int k = k0 + u * kAvgSlices;
+        v[u] = k < hw ? __ldg(p + (long long)k * cg) : make_uint4(flip, flip, flip, flip);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned w[4] = {v[u].x ^ flip, v[u].y ^ flip, v[u].z ^ flip, v[u].w ^ flip};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[2 * j] += w[j] & 0x00FF00FFu; acc[2 * j + 1] += (w[j] >> 8) & 0x00FF00FFu; }
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) part[threadIdx.y][j][threadIdx.x] = acc[j];
+  __syncthreads();
+  if (ch0 >= ch) return;
+  unsigned even = 0, odd = 0;
+#pragma unroll
+  for (int sl = 0; sl < kAvgSlices; ++sl) { even += part[sl][2 * word][gl]; odd += part[sl][2 * word + 1][gl]; }
+  const int off = is_signed ? 128 * hw : 0;
+  // byte 2*half of the word sits in halfword `half` of the even sums, byte 2*half+1 in halfword `half` of the odd sums
+  const int s0 = (int)((even >> (16 * half)) & 0xFFFFu) - off, s1 = (int)((odd >> (16 * half)) & 0xFFFFu) - off;
+  const int q0 = hq_clamp_ll(hq_dn(s0, bb.x, cc.x), 0, qmin, qmax);
+  const int q1 = hq_clamp_ll(hq_dn(s1, bb.y, cc.y), 0, qmin, qmax);
+  out[((long long)img * ch + ch0) >> 1] = (unsigned short)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
 }
 
 __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int in_bits, int in_signed,
@@ -472,12 +598,12 @@ cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t 
     const int lo = a.relu ? (a.qmin > 0 ? a.qmin : 0) : a.qmin, hi = a.qmax;
     const int v = (a.res ? 4 : 0) | (a.main_signed ? 2 : 0) | ((a.res && a.res_signed) ? 1 : 0);
     switch (v) {
-      case 0: return launch_requant8<false, false, false>(a, grid, block, words, lo, hi, s);
-      case 2: return launch_requant8<false, true, false>(a, grid, block, words, lo, hi, s);
-      case 4: return launch_requant8<true, false, false>(a, grid, block, words, lo, hi, s);
-      case 5: return launch_requant8<true, false, true>(a, grid, block, words, lo, hi, s);
-      case 6: return launch_requant8<true, true, false>(a, grid, block, words, lo, hi, s);
-      default: return launch_requant8<true, true, true>(a, grid, block, words, lo, hi, s);
+      case 0: return launch_requant8<false, false, false>(a, grid, block, words, lo, hi, sm_count, s);
+      case 2: return launch_requant8<false, true, false>(a, grid, block, words, lo, hi, sm_count, s);
+      case 4: return launch_requant8<true, false, false>(a, grid, block, words, lo, hi, sm_count, s);
+      case 5: return launch_requant8<true, false, true>(a, grid, block, words, lo, hi, sm_count, s);
+      case 6: return launch_requant8<true, true, false>(a, grid, block, words, lo, hi, sm_count, s);
+      default: return launch_requant8<true, true, true>(a, grid, block, words, lo, hi, sm_count, s);
     }
   }
   const int groups = a.ch / 16;
@@ -503,7 +629,10 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
                               const int32_t* b, const int32_t* c, int qmin, int qmax,
                               void* out, int out_bits, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  if (in_bits == 8 && out_bits == 8 && ch % 4 == 0 && h * w <= 257 && n <= 65535) {
+  if (in_bits == 8 && out_bits == 8 && ch % 16 == 0 && h * w <= 257 && n <= 65535) {
+    const dim3 grid((ch / 16 + 31) / 32, n), block(32, kAvgSlices);
+    avgpool_vec16_kernel<<<grid, block, 0, s>>>((const uint4*)in, h * w, ch, in_signed, b, c, qmin, qmax, (unsigned short*)out);
+  } else if (in_bits == 8 && out_bits == 8 && ch % 4 == 0 && h * w <= 257 && n <= 65535) {
     const dim3 grid((ch / 4 + 63) / 64, n), block(64, 4);
     avgpool_vec4_sliced_kernel<<<grid, block, 0, s>>>((const unsigned*)in, h * w, ch, in_signed, b, c, qmin, qmax, (unsigned*)out);
   } else if (in_bits == 8 && out_bits == 8 && ch % 4 == 0) {

@@ -12,7 +12,8 @@ enum : uint32_t {
   HQ_DEV_TIMEOUT_PRODUCER = 1,   // TMA producer waited too long for a free stage
   HQ_DEV_TIMEOUT_MMA = 2,        // MMA issuer waited too long for operands or a free accumulator
   HQ_DEV_TIMEOUT_EPILOGUE = 3,   // epilogue waited too long for a finished accumulator
-  HQ_DEV_TIMEOUT_DRAIN = 4       // teardown waited too long for work in flight
+  HQ_DEV_TIMEOUT_DRAIN = 4,      // teardown waited too long for work in flight
+  HQ_DEV_TIMEOUT_ELTWISE = 5     // a streaming kernel waited too long for a staged chunk or a free stage
 };
 
 struct hq_handle {
@@ -22,7 +23,9 @@ struct hq_handle {
   uint32_t* dev_status;       // one word in device memory, sticky until hq_sync
   void* workspace;            // scratch owned by the handle (grown on demand, never inside a capture)
   size_t workspace_bytes;
+  void* narrow_pairs;         // 2 x kNarrowChannels x 16 bytes: narrow pairs of a single element-wise call's two operands
 };
+constexpr int kNarrowChannels = 4096;
 
 // ------------------------------------------------------------------------------------------
 // Dyadic arithmetic (Eq. 4): dn(q, b, c) = (q*b + 2^(c-1)) >> c, 64-bit product, arithmetic shift.
@@ -72,6 +75,7 @@ struct EltArgs {
   void* out; int32_t out_bits;
   // optional narrow pairs {m, a, s, valid} per channel for 8-bit operands (see hq_launch_residual_narrow), or NULL
   const void* m_narrow; const void* r_narrow;
+  uint32_t* status;          // the handle's device status word (bounded waits report here), or NULL
 };
 
 cudaError_t hq_launch_conv_cuda_core(const ConvArgs& a, cudaStream_t s);

@@ -262,6 +262,56 @@ def test_residual_add_8bit_fast_kernel_every_shift(hq):
         assert np.array_equal(host(out, ref), ref)
 
 
+LARGE_ELT_CASES = [
+    # pixels (h x w of one image, n = 1), ch, main_signed, res (None / signed flag), out_bits, shifts
+    ((157, 131), 256, 0, 0, 8, "fast"),        # 20567 pixels of 64 words: a ragged last trip
+    ((157, 131), 256, 0, None, 8, "fast"),     # plain requantization (eight words in flight per thread)
+    ((211, 97), 64, 1, 1, 8, "fast"),          # signed operands and output
+    ((157, 131), 128, 0, 1, 4, "fast"),        # packed 4-bit output, clamp [0, 15]
+    ((95, 83), 1024, 0, 0, 8, "fast"),         # 256 words: one pixel per block step
+    ((157, 131), 256, 0, 0, 8, "every"),       # shifts 1..62: threads with a shift below 9 take the 64-bit form
+    ((301, 211), 32, 0, 0, 8, "fast"),         # 8 words per pixel
+    ((157, 131), 4, 0, 0, 8, "fast"),          # a single word per pixel
+    ((101, 67), 192, 0, 0, 8, "fast"),         # 48 words: not a power of two
+    ((157, 131), 128, 1, None, 4, "fast"),     # 4-bit output from signed input
+]
+
+
+@pytest.mark.parametrize("cfg", LARGE_ELT_CASES)
+def test_residual_add_large_tensors(hq, cfg):
+    """Tensors of many block trips with a ragged last trip: the flat word-array kernel (channel words a power of two),
+    every output form, and a channel count that keeps the pixel-row kernel (192 = 48 words)."""
+    from paper_2011_10680_b200 import binding
+    (h, w), ch, main_signed, res_signed, out_bits, shifts = cfg
+    g = inputs.rng(306, h, w, ch, main_signed, out_bits)
+    shape = (1, h, w, ch)
+    draw = lambda sg: (g.integers(-128, 128, size=shape, dtype=np.int64).astype(np.int8) if sg else
+                       g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8))
+    main = draw(main_signed)
+    res = draw(res_signed) if res_signed is not None else None
+    mb, rb = (g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32) for _ in range(2))
+    if shifts == "every":
+        mc = (np.arange(ch) % 62 + 1).astype(np.int32)
+        rc = ((np.arange(ch) * 7) % 62 + 1).astype(np.int32)
+    else:
+        mc = g.integers(29, 34, size=ch).astype(np.int32)
+        rc = g.integers(29, 34, size=ch).astype(np.int32)
+    out_signed = int(out_bits == 8 and main_signed == 1)
+    qmin, qmax = (0, 15) if out_bits == 4 else ((-128, 127) if out_signed else (0, 255))
+    relu = 0 if out_signed else 1
+    ref = oracle().residual_add(main, 8, main_signed, mb, mc, res, 8 if res is not None else 0, res_signed or 0,
+                                rb if res is not None else None, rc if res is not None else None, ch, relu, qmin, qmax,
+                                out_bits, out_signed)
+    out = binding.alloc_out(*shape[:3], ch, out_bits, out_signed)
+    st = hq.residual_add(binding.to_device(main), 8, main_signed, binding.to_device(mb), binding.to_device(mc),
+                         binding.to_device(res), 8 if res is not None else 0, res_signed or 0,
+                         binding.to_device(rb) if res is not None else None, binding.to_device(rc) if res is not None else None,
+                         ch, relu, qmin, qmax, out, out_bits, out_signed)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
 @pytest.mark.parametrize("n,hw,ch,in_bits", [(4, 7, 64, 8), (2, 7, 2048, 8), (3, 5, 6, 8), (2, 4, 16, 32), (2, 3, 8, 4)])
 def test_avgpool_requant(hq, n, hw, ch, in_bits):
     from paper_2011_10680_b200 import binding
@@ -310,6 +360,28 @@ def test_maxpool_windows_and_signedness(hq, k, stride, pad, signed):
     ref = oracle().maxpool(xs, k, stride, pad, signed)
     out = binding.alloc_out(n, ref.shape[1], ref.shape[2], ch, 8, signed)
     st = hq.maxpool(binding.to_device(xs), ch, signed, k, stride, pad, out)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
+@pytest.mark.parametrize("n,hw,ch,signed", [(3, 16, 48, 0), (2, 7, 528, 0), (2, 16, 64, 1), (5, 7, 2048, 1), (2, 9, 20, 1),
+                                            (2, 17, 32, 0)])
+def test_avgpool_requant_8bit_kernels(hq, n, hw, ch, signed):
+    # the 16-channel kernel with a partly filled block, two blocks per image, 256 pixels at the maximum value
+    # (16-bit lane sums at their limit), signed bytes; the 4-channel kernel (ch = 20); more than 257 pixels
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(305, n, hw, ch, signed)
+    x = g.integers(0, 256, size=(n, hw, hw, ch), dtype=np.int64).astype(np.uint8)
+    x[0] = 0x80 if signed else 0xFF
+    x[1, :, :, ::3] = 0x7F if signed else 0xFF
+    xs = x.view(np.int8) if signed else x
+    scale = np.exp(g.uniform(np.log(0.2), np.log(2.0), size=ch)) / (hw * hw)
+    b, c = inputs.dyadic_from_scale(scale)
+    lo, hi = (-128, 127) if signed else (0, 255)
+    ref = oracle().avgpool_requant(xs, ch, 8, signed, b, c, lo, hi, 8, signed)
+    out = binding.alloc_out(n, 1, 1, ch, 8, signed)
+    st = hq.avgpool_requant(binding.to_device(xs), ch, 8, signed, binding.to_device(b), binding.to_device(c), lo, hi, out, 8, signed)
     assert st == binding.HQ_OK
     hq.sync()
     assert np.array_equal(host(out, ref), ref)
