@@ -3,6 +3,7 @@
 // pooling.  Each streams its operands once with 16-byte accesses; the arithmetic is the dyadic
 // multiply-shift of Eq. 4 in 64-bit integers.  No floating point anywhere.
 #include "hq_internal.cuh"
+#include <cstdlib>
 
 namespace {
 
@@ -287,11 +288,195 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
   }
 }
 
+// ---- the flat form behind a bulk-copy pipeline -------------------------------------------------
+// For large tensors.  A persistent block walks chunks of U * 256 consecutive words.  One thread keeps
+// kEltStages - 1 chunks ahead with bulk asynchronous copies (global -> shared, completion counted on an
+// mbarrier), so the bytes in flight per SM depend neither on registers nor on occupancy; all threads read their
+// words from shared memory, requantize and store straight to global memory.  Every wait is bounded: after the
+// budget the block records HQ_DEV_TIMEOUT_ELTWISE, waits (bounded) for its copies in flight and returns.
+constexpr int kEltStages = 4;
+constexpr unsigned long long kEltWaitNs = 2000000000ull;
+
+struct EltPipe {
+  unsigned long long full[kEltStages];
+  unsigned long long empty[kEltStages];
+  volatile unsigned abort_flag;
+};
+
+__device__ __forceinline__ unsigned esmem(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ebar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void ebar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void ebar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool ebar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void ebulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ unsigned long long elt_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool ebar_wait(unsigned bar, unsigned parity, EltPipe* pipe, uint32_t* status) {
+  if (ebar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = elt_ns();
+  unsigned spins = 0;
+  while (!ebar_try_wait(bar, parity)) {
+    if ((++spins & 63u) == 0) {
+      if (pipe->abort_flag) return false;
+      if (elt_ns() - t0 > kEltWaitNs) {
+        pipe->abort_flag = 1u;
+        if (status) atomicCAS(status, 0u, (uint32_t)HQ_DEV_TIMEOUT_ELTWISE);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, bool SLOW, int SATP, bool NARROW>
+__device__ __forceinline__ void requant8_chunks(const EltArgs& a, const Dy8 (&m)[4], const Dy8 (&r)[4], int wx, long long total,
+                                                int lo, int hi, EltPipe* pipe, unsigned char* stage) {
+  constexpr int T = 256, U = RES ? 4 : 8;
+  constexpr unsigned chunk_bytes = U * T * 4, stage_bytes = RES ? 2u * chunk_bytes : chunk_bytes;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const long long n_chunks = total / (U * T);
+  const unsigned char* mg = (const unsigned char*)a.main_t;
+  const unsigned char* rg = (const unsigned char*)a.res;
+  auto issue = [&](long long chunk, unsigned slot) {
+    const unsigned bar = esmem(&pipe->full[slot]);
+    ebar_expect_tx(bar, stage_bytes);
+    ebulk_load(esmem(stage + slot * stage_bytes), mg + chunk * chunk_bytes, chunk_bytes, bar);
+    if (RES) ebulk_load(esmem(stage + slot * stage_bytes + chunk_bytes), rg + chunk * chunk_bytes, chunk_bytes, bar);
+  };
+  unsigned issued = 0;                                   // thread 0: chunks handed to the copy engine so far
+  if (tid == 0) {
+    for (int k = 0; k < kEltStages - 1; ++k) {
+      const long long chunk = blockIdx.x + (long long)k * gridDim.x;
+      if (chunk < n_chunks) { issue(chunk, (unsigned)k); ++issued; }
+    }
+  }
+  unsigned it = 0;
+  bool ok = true;
+  for (long long chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x, ++it) {
+    const unsigned s = it % kEltStages, ph = (it / kEltStages) & 1u;
+    if (tid == 0) {
+      const long long nxt = chunk + (long long)(kEltStages - 1) * gridDim.x;
+      if (nxt < n_chunks) {
+        const unsigned it2 = it + kEltStages - 1, s2 = it2 % kEltStages, use = it2 / kEltStages;
+        // the slot's previous use must have been read by every warp (a fresh barrier passes at once)
+        ok = ebar_wait(esmem(&pipe->empty[s2]), (use & 1u) ^ 1u, pipe, a.status);
+        if (ok) { issue(nxt, s2); ++issued; }
+      }
+    }
+    unsigned w = 1u;
+    if (lane == 0) w = (ok && ebar_wait(esmem(&pipe->full[s]), ph, pipe, a.status)) ? 1u : 0u;
+    w = __shfl_sync(0xffffffffu, w, 0);
+    if (!w) { ok = false; break; }
+    const unsigned* ms = (const unsigned*)(stage + s * stage_bytes) + tid;
+    const unsigned* rs = (const unsigned*)(stage + s * stage_bytes + chunk_bytes) + tid;
+    void* dst0 = out_word<OUT4>(a, chunk * (U * T) + tid);
+    unsigned mw[U], rw[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) { mw[u] = ms[u * T]; rw[u] = RES ? rs[u * T] : 0u; }
+    __syncwarp();
+    if (lane == 0) ebar_arrive(esmem(&pipe->empty[s]));     // the words are in registers: the slot may be refilled
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(
+          a, m, r, wx, mw[u], rw[u], OUT4 ? (void*)((unsigned short*)dst0 + u * T) : (void*)((unsigned*)dst0 + u * T), lo, hi);
+  }
+  if (ok) {
+    // words after the last full chunk: plain loads, spread over the blocks
+    const unsigned* mp = (const unsigned*)a.main_t;
+    const unsigned* rp = (const unsigned*)a.res;
+    for (long long i = n_chunks * (U * T) + (long long)blockIdx.x * T + tid; i < total; i += (long long)gridDim.x * T)
+      requant8_word<RES, MSIGNED, RSIGNED, OUT4, SLOW, SATP, NARROW>(a, m, r, wx, __ldg(mp + i), RES ? __ldg(rp + i) : 0u,
+                                                                     out_word<OUT4>(a, i), lo, hi);
+  } else if (tid == 0) {
+    // gave up: the copies already started must land before the block's shared memory is released
+    for (unsigned q = it; q < issued; ++q) {
+      const unsigned long long t0 = elt_ns();
+      while (!ebar_try_wait(esmem(&pipe->full[q % kEltStages]), (q / kEltStages) & 1u)) {
+        if (elt_ns() - t0 > kEltWaitNs) break;
+      }
+    }
+  }
+}
+
+template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
+__global__ void __launch_bounds__(256, RES ? 3 : 4) requant8_staged_kernel(EltArgs a, int words, int lo, int hi) {
+  extern __shared__ __align__(128) unsigned char stage[];
+  __shared__ EltPipe pipe;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    for (int k = 0; k < kEltStages; ++k) { ebar_init(esmem(&pipe.full[k]), 1u); ebar_init(esmem(&pipe.empty[k]), 256 / 32); }
+    pipe.abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const int wx = tid & (words - 1);           // word (4 channels) of the pixel; words is a power of two <= 256
+  const long long total = a.pixels * words;
+  Dy8 m[4], r[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m[i] = make_dy8(__ldg(a.mb + 4 * wx + i), __ldg(a.mc + 4 * wx + i));
+    if (RES) r[i] = make_dy8(__ldg(a.rb + 4 * wx + i), __ldg(a.rc + 4 * wx + i));
+    else r[i] = m[i];
+  }
+  bool slow = false;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) slow = slow || m[i].c < 9 || (RES && r[i].c < 9);
+  // the form is chosen per warp, so that a warp's lanes stay together through the pipeline's hand-shakes
+  slow = __any_sync(0xffffffffu, slow);
+  bool narrow = false;
+  Dy8 nm[4], nr[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { nm[i] = m[i]; nr[i] = r[i]; }
+  if (a.m_narrow && (!RES || a.r_narrow)) {
+    narrow = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int4 pm = __ldg((const int4*)a.m_narrow + 4 * wx + i);
+      nm[i].b = pm.x; nm[i].h = pm.y; nm[i].sh = pm.z; nm[i].c = 0; narrow = narrow && pm.w != 0;
+      nr[i] = nm[i];
+      if (RES) {
+        const int4 pr = __ldg((const int4*)a.r_narrow + 4 * wx + i);
+        nr[i].b = pr.x; nr[i].h = pr.y; nr[i].sh = pr.z; narrow = narrow && pr.w != 0;
+      }
+    }
+  }
+  narrow = __all_sync(0xffffffffu, narrow);
+  if (narrow) requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, total, lo, hi, &pipe, stage);
+  else if (slow) requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, true, 0, false>(a, m, r, wx, total, lo, hi, &pipe, stage);
+  else requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, SATP, false>(a, m, r, wx, total, lo, hi, &pipe, stage);
+}
+
 template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
 cudaError_t launch_requant8_form(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, int sm_count, cudaStream_t s) {
   if (words <= 256 && (words & (words - 1)) == 0) {
     const long long total = a.pixels * words, per_block = 256 * (RES ? 4 : 8);
     const long long blocks = (total + per_block - 1) / per_block, cap = (long long)sm_count * 16;
+    static const bool staged_on = getenv("HQ_ELT_STAGED") == nullptr || atoi(getenv("HQ_ELT_STAGED")) != 0;
+    if (staged_on && total / per_block >= 8ll * sm_count) {      // large: the bulk-copy pipeline, three or four persistent blocks per SM
+      const size_t smem = (size_t)kEltStages * per_block * 4 * (RES ? 2 : 1);
+      requant8_staged_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP><<<sm_count * (RES ? 3 : 4), 256, smem, s>>>(a, words, lo, hi);
+      return cudaGetLastError();
+    }
     requant8_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP, true><<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(a, words, lo, hi);
   } else {
     requant8_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP, false><<<grid, block, 0, s>>>(a, words, lo, hi);

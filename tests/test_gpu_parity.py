@@ -274,6 +274,11 @@ LARGE_ELT_CASES = [
     ((157, 131), 4, 0, 0, 8, "fast"),          # a single word per pixel
     ((101, 67), 192, 0, 0, 8, "fast"),         # 48 words: not a power of two
     ((157, 131), 128, 1, None, 4, "fast"),     # 4-bit output from signed input
+    # more than eight chunks per SM: the bulk-copy pipeline, with words left over after the last full chunk
+    ((331, 251), 128, 0, 0, 8, "fast"),
+    ((331, 251), 128, 0, None, 8, "fast"),
+    ((331, 251), 128, 1, 1, 4, "every"),
+    ((499, 333), 64, 0, 1, 8, "every"),
 ]
 
 
