@@ -3,7 +3,6 @@
 // pooling.  Each streams its operands once with 16-byte accesses; the arithmetic is the dyadic
 // multiply-shift of Eq. 4 in 64-bit integers.  No floating point anywhere.
 #include "hq_internal.cuh"
-#include <cstdlib>
 
 namespace {
 
@@ -111,7 +110,8 @@ __device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` =
 }
 
 // One pixel's word of four channels.  SLOW: one of the thread's channels has a shift below 9 (64-bit form).
-// SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing).
+// SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing);
+// 3 for a 4-bit output clamped to [0, 15]; 4 the same without a residual and with shifts reduced by four.
 // 8-bit value i of a word, zero- or sign-extended (one byte-permute either way: selector bit 3 replicates the
 // selected byte's sign bit).
 template <bool SIGNED>
@@ -152,6 +152,15 @@ __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4
       asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(w23));
     }
     *(unsigned*)dst = w;
+  } else if constexpr (OUT4 && SATP == 4) {
+    // No residual, clamp to [0, 15], and the shifts were reduced by four: s = floor(16 v).  The saturating pack
+    // clamps 16 v to [0, 255], whose high nibble is min(max(floor(v), 0), 15); the four high nibbles then move
+    // next to each other.
+    unsigned w23, w;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(s[3]), "r"(s[2]), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s[1]), "r"(s[0]), "r"(w23));
+    const unsigned p0 = __byte_perm(w, 0u, 0x4420), p1 = __byte_perm(w, 0u, 0x4431);    // bytes 0, 2 and bytes 1, 3
+    *(unsigned short*)dst = (unsigned short)(((p0 >> 4) & 0x0F0Fu) | (p1 & 0xF0F0u));
   } else if constexpr (OUT4 && SATP == 3) {
     // clamp to [0, 15]: upper bound by a minimum, lower bound by the saturating pack; then the four bytes'
     // low nibbles move next to each other
@@ -206,6 +215,15 @@ __device__ __forceinline__ void requant8_pixels(const EltArgs& a, const Dy8 (&m)
                                                                        RES ? __ldg(rp + p * words + wx) : 0u, out_word<OUT4>(a, p * words + wx), lo, hi);
     }
   }
+}
+
+// 4-bit output clamped to [0, 15] without a residual: when every channel of the thread shifts by at least four,
+// the shifts drop by four and the word is packed from the high nibbles (requant8_word, SATP == 4).
+__device__ __forceinline__ bool reduce_shifts_by_four(Dy8 (&d)[4], bool usable) {
+  bool ok = usable;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) ok = ok && d[i].sh >= 4;
+  return ok;
 }
 
 // Flat form for channel counts whose words divide the block (words a power of two, at most 256): the tensor is
@@ -273,6 +291,14 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
       }
     }
     if (ok) {
+      if constexpr (FLAT && OUT4 && SATP == 3 && !RES) {
+        if (reduce_shifts_by_four(nm, true)) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) nm[i].sh -= 4;
+          requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, 4, true>(a, nm, nr, wx, total, lo, hi);
+          return;
+        }
+      }
       if (FLAT) requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, total, lo, hi);
       else requant8_pixels<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, words, lo, hi);
       return;
@@ -280,6 +306,14 @@ __global__ void __launch_bounds__(256) requant8_kernel(EltArgs a, int words, int
   }
   // two separate loops, so that the common one carries none of the 64-bit form's instructions
   if (FLAT) {
+    if constexpr (OUT4 && SATP == 3 && !RES) {
+      if (!slow && reduce_shifts_by_four(m, true)) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i].sh -= 4;
+        requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, 4>(a, m, r, wx, total, lo, hi);
+        return;
+      }
+    }
     if (slow) requant8_flat<RES, MSIGNED, RSIGNED, OUT4, true, 0>(a, m, r, wx, total, lo, hi);
     else requant8_flat<RES, MSIGNED, RSIGNED, OUT4, false, SATP>(a, m, r, wx, total, lo, hi);
   } else {
@@ -419,7 +453,7 @@ __device__ __forceinline__ void requant8_chunks(const EltArgs& a, const Dy8 (&m)
 }
 
 template <bool RES, bool MSIGNED, bool RSIGNED, bool OUT4, int SATP>
-__global__ void __launch_bounds__(256, RES ? 3 : 4) requant8_staged_kernel(EltArgs a, int words, int lo, int hi) {
+__global__ void __launch_bounds__(256, RES ? 3 : 5) requant8_staged_kernel(EltArgs a, int words, int lo, int hi) {
   extern __shared__ __align__(128) unsigned char stage[];
   __shared__ EltPipe pipe;
   const int tid = threadIdx.x;
@@ -461,6 +495,17 @@ __global__ void __launch_bounds__(256, RES ? 3 : 4) requant8_staged_kernel(EltAr
     }
   }
   narrow = __all_sync(0xffffffffu, narrow);
+  if constexpr (OUT4 && SATP == 3 && !RES) {
+    // high-nibble packing, chosen per warp like the other forms
+    const bool nib = __all_sync(0xffffffffu, narrow ? reduce_shifts_by_four(nm, true) : reduce_shifts_by_four(m, !slow));
+    if (nib) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { nm[i].sh -= 4; m[i].sh -= 4; }
+      if (narrow) requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, 4, true>(a, nm, nr, wx, total, lo, hi, &pipe, stage);
+      else requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, 4, false>(a, m, r, wx, total, lo, hi, &pipe, stage);
+      return;
+    }
+  }
   if (narrow) requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, SATP, true>(a, nm, nr, wx, total, lo, hi, &pipe, stage);
   else if (slow) requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, true, 0, false>(a, m, r, wx, total, lo, hi, &pipe, stage);
   else requant8_chunks<RES, MSIGNED, RSIGNED, OUT4, false, SATP, false>(a, m, r, wx, total, lo, hi, &pipe, stage);
@@ -471,10 +516,9 @@ cudaError_t launch_requant8_form(const EltArgs& a, dim3 grid, dim3 block, int wo
   if (words <= 256 && (words & (words - 1)) == 0) {
     const long long total = a.pixels * words, per_block = 256 * (RES ? 4 : 8);
     const long long blocks = (total + per_block - 1) / per_block, cap = (long long)sm_count * 16;
-    static const bool staged_on = getenv("HQ_ELT_STAGED") == nullptr || atoi(getenv("HQ_ELT_STAGED")) != 0;
-    if (staged_on && total / per_block >= 8ll * sm_count) {      // large: the bulk-copy pipeline, three or four persistent blocks per SM
+    if (total / per_block >= 8ll * sm_count) {      // large: the bulk-copy pipeline, three or five persistent blocks per SM
       const size_t smem = (size_t)kEltStages * per_block * 4 * (RES ? 2 : 1);
-      requant8_staged_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP><<<sm_count * (RES ? 3 : 4), 256, smem, s>>>(a, words, lo, hi);
+      requant8_staged_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP><<<sm_count * (RES ? 3 : 5), 256, smem, s>>>(a, words, lo, hi);
       return cudaGetLastError();
     }
     requant8_kernel<RES, MSIGNED, RSIGNED, OUT4, SATP, true><<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(a, words, lo, hi);
@@ -491,6 +535,93 @@ cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, 
   if (lo == 0 && hi == 255) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 1>(a, grid, block, words, lo, hi, sm_count, s);
   if (lo == -128 && hi == 127) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 2>(a, grid, block, words, lo, hi, sm_count, s);
   return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 0>(a, grid, block, words, lo, hi, sm_count, s);
+}
+
+// ---- INT32 main operand, 8-bit output: flat form ------------------------------------------------
+// A thread owns four consecutive channels: one 16-byte load of accumulators per pixel (and one word of the 8-bit
+// residual), one word stored; quads-per-pixel a power of two up to 256, so the flat index keeps a thread on its
+// channels.  For 32 <= c the value is hi32(q*b + 2^(c-1)) >> (c-32) exactly (the low 32 bits cannot matter once
+// at least 32 bits are shifted out); a thread with a smaller shift on one of its channels takes the 64-bit form.
+struct Dy32 { int b; long long r0; int sh; };
+template <bool RES, bool RSIGNED, int SATP>
+__global__ void __launch_bounds__(256) requant32_flat_kernel(EltArgs a, int quads, int lo, int hi) {
+  constexpr int T = 256, U = 4;
+  const int wx = threadIdx.x & (quads - 1);
+  const long long total = a.pixels * quads;
+  Dy32 m[4];
+  Dy8 r[4];
+  bool slow = false;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = __ldg(a.mc + 4 * wx + i);
+    m[i].b = __ldg(a.mb + 4 * wx + i); m[i].r0 = 1LL << (c - 1); m[i].sh = c - 32;
+    slow = slow || c < 32;
+    if (RES) { r[i] = make_dy8(__ldg(a.rb + 4 * wx + i), __ldg(a.rc + 4 * wx + i)); slow = slow || r[i].c < 9; }
+    else r[i] = make_dy8(0, 40);
+  }
+  const int4* mp = (const int4*)a.main_t + threadIdx.x;
+  const unsigned* rp = RES ? (const unsigned*)a.res + threadIdx.x : nullptr;
+  unsigned* op = (unsigned*)a.out + threadIdx.x;
+  auto one = [&](const int4& q, unsigned rw, unsigned* dst) {
+    const int acc[4] = {q.x, q.y, q.z, q.w};
+    int sv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (!slow) {
+        sv[i] = (int)(((long long)acc[i] * (long long)m[i].b + m[i].r0) >> 32) >> m[i].sh;
+        if (RES) sv[i] += dn8<RSIGNED>(__byte_perm(rw, 0u, 0x0444u | ((unsigned)i << 12)), r[i]);
+      } else {
+        const unsigned rbyte = (rw >> (8 * i)) & 0xFFu;
+        long long t = hq_dn(acc[i], m[i].b, m[i].sh + 32);
+        if (RES) t += hq_dn(RSIGNED ? (int)(signed char)rbyte : (int)rbyte, __ldg(a.rb + 4 * wx + i), r[i].c);
+        sv[i] = (int)(t < (long long)lo ? (long long)lo : (t > (long long)hi ? (long long)hi : t));
+      }
+    }
+    if (SATP != 0) {
+      unsigned w23, w;
+      if (SATP == 1) {
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(sv[3]), "r"(sv[2]), "r"(0));
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(sv[1]), "r"(sv[0]), "r"(w23));
+      } else {
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(sv[3]), "r"(sv[2]), "r"(0));
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(sv[1]), "r"(sv[0]), "r"(w23));
+      }
+      *dst = w;
+    } else {
+      unsigned w = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w |= (unsigned)(min(max(sv[i], lo), hi) & 0xFF) << (8 * i);
+      *dst = w;
+    }
+  };
+  const long long trip = (long long)gridDim.x * (U * T);
+  for (long long base = (long long)blockIdx.x * (U * T); base < total; base += trip) {
+    if (base + U * T <= total) {
+      int4 q[U];
+      unsigned rw[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) q[u] = __ldg(mp + base + u * T);
+#pragma unroll
+      for (int u = 0; u < U; ++u) rw[u] = RES ? __ldg(rp + base + u * T) : 0u;
+#pragma unroll
+      for (int u = 0; u < U; ++u) one(q[u], rw[u], op + base + u * T);
+    } else {
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (base + u * T + threadIdx.x < total) one(__ldg(mp + base + u * T), RES ? __ldg(rp + base + u * T) : 0u, op + base + u * T);
+    }
+  }
+}
+
+template <bool RES, bool RSIGNED>
+cudaError_t launch_requant32(const EltArgs& a, int quads, int lo, int hi, int sm_count, cudaStream_t s) {
+  const long long total = a.pixels * quads, per_block = 256 * 4;
+  const long long blocks = (total + per_block - 1) / per_block, cap = (long long)sm_count * 16;
+  const unsigned grid = (unsigned)(blocks < cap ? blocks : cap);
+  if (lo == 0 && hi == 255) requant32_flat_kernel<RES, RSIGNED, 1><<<grid, 256, 0, s>>>(a, quads, lo, hi);
+  else if (lo == -128 && hi == 127) requant32_flat_kernel<RES, RSIGNED, 2><<<grid, 256, 0, s>>>(a, quads, lo, hi);
+  else requant32_flat_kernel<RES, RSIGNED, 0><<<grid, 256, 0, s>>>(a, quads, lo, hi);
+  return cudaGetLastError();
 }
 
 // Any channel count: one thread per output byte (one element at 8 bit, two at 4 bit).
@@ -595,58 +726,66 @@ __global__ void __launch_bounds__(256) avgpool_vec4_sliced_kernel(const unsigned
   out[(long long)img * cg + g] = w;
 }
 
-// 16 channels per thread (one 16-byte load per pixel), 8 pixel slices per block, four loads of a thread in flight
-// at a time; 512 channels per block.  Bytes are summed as 16-bit lanes (h*w*255 <= 65535, i.e. up to 257 pixels;
-// signed bytes are offset by 128 and corrected at the end).  The slices meet in shared memory and every thread
-// then finishes two channels.
-constexpr int kAvgSlices = 8;
-__global__ void __launch_bounds__(256) avgpool_vec16_kernel(const uint4* __restrict__ in, int hw, int ch, int is_signed,
-                                                            const int32_t* __restrict__ b, const int32_t* __restrict__ c,
-                                                            int qmin, int qmax, unsigned short* __restrict__ out) {
-  __shared__ unsigned part[kAvgSlices][8][32];        // [slice][even / odd byte sums of the four words][channel group]
+// 16 channels per thread (one 16-byte load per pixel), SLICES pixel slices per block (two for a 7x7 map, so that
+// a thread sums a dozen or more pixels and the block's closing steps weigh little), eight loads of a thread in
+// flight at a time; 512 channels per block.  Bytes are summed as 16-bit lanes (h*w*255 <= 65535, i.e. up to 257
+// pixels; signed bytes are offset by 128 and corrected at the end).  The slices meet in shared memory and every
+// thread then finishes its share of the block's channels, two at a time.
+template <int SLICES, bool SIGNED>
+__global__ void __launch_bounds__(32 * SLICES) avgpool_vec16_kernel(const uint4* __restrict__ in, int hw, int ch,
+                                                                    const int32_t* __restrict__ b, const int32_t* __restrict__ c,
+                                                                    int qmin, int qmax, unsigned short* __restrict__ out) {
+  __shared__ unsigned part[SLICES][8][32];            // [slice][even / odd byte sums of the four words][channel group]
   const int cg = ch >> 4;
   const int g = blockIdx.x * 32 + threadIdx.x, img = blockIdx.y;
-  // thread t finishes channels 2t and 2t+1 of the block's 512: group t / 8, word (t % 8) / 2, bytes 2 * (t % 2) + {0, 1}
-  const int t = threadIdx.y * 32 + threadIdx.x;
-  const int gl = t >> 3, word = (t & 7) >> 1, half = t & 1;
-  const int ch0 = (blockIdx.x * 32 + gl) * 16 + word * 4 + half * 2;
-  int2 bb = make_int2(0, 0), cc = make_int2(1, 1);
-  if (ch0 < ch) {                                    // fetched first: their latency hides behind the pixels'
-    bb = make_int2(__ldg(b + ch0), __ldg(b + ch0 + 1));
-    cc = make_int2(__ldg(c + ch0), __ldg(c + ch0 + 1));
-  }
   unsigned acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   if (g < cg) {
     const uint4* p = in + (long long)img * hw * cg + g;
-    const unsigned flip = is_signed ? 0x80808080u : 0u;
-    for (int k0 = threadIdx.y; k0 < hw; k0 += 4 * kAvgSlices) {
-      uint4 v[4];
+    constexpr unsigned flip = SIGNED ? 0x80808080u : 0u;
+    const int stride = SLICES * cg;
+    for (int k0 = threadIdx.y; k0 < hw; k0 += 8 * SLICES) {
+      const uint4* q = p + (long long)k0 * cg;
+      uint4 v[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int k = k0 + u * kAvgSlices;
-        v[u] = k < hw ? __ldg(p + (long long)k * cg) : make_uint4(flip, flip, flip, flip);
-      }
+      for (int u = 0; u < 8; ++u)
+        v[u] = k0 + u * SLICES < hw ? __ldg(q + u * stride) : make_uint4(flip, flip, flip, flip);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         const unsigned w[4] = {v[u].x ^ flip, v[u].y ^ flip, v[u].z ^ flip, v[u].w ^ flip};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { acc[2 * j] += w[j] & 0x00FF00FFu; acc[2 * j + 1] += (w[j] >> 8) & 0x00FF00FFu; }
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] += __byte_perm(w[j], 0u, 0x4240);          // bytes 0 and 2, one per halfword
+          acc[2 * j + 1] += __byte_perm(w[j], 0u, 0x4341);      // bytes 1 and 3
+        }
       }
     }
   }
 #pragma unroll
   for (int j = 0; j < 8; ++j) part[threadIdx.y][j][threadIdx.x] = acc[j];
   __syncthreads();
-  if (ch0 >= ch) return;
-  unsigned even = 0, odd = 0;
+  // pair index t covers channels 2t and 2t+1 of the block's 512: group t / 8, word (t % 8) / 2, bytes 2 * (t % 2) + {0, 1}
+  const int off = SIGNED ? 128 * hw : 0;
+  for (int t = threadIdx.y * 32 + threadIdx.x; t < 256; t += 32 * SLICES) {
+    const int gl = t >> 3, word = (t & 7) >> 1, half = t & 1;
+    const int ch0 = (blockIdx.x * 32 + gl) * 16 + word * 4 + half * 2;
+    if (ch0 >= ch) continue;
+    unsigned even = 0, odd = 0;
 #pragma unroll
-  for (int sl = 0; sl < kAvgSlices; ++sl) { even += part[sl][2 * word][gl]; odd += part[sl][2 * word + 1][gl]; }
-  const int off = is_signed ? 128 * hw : 0;
-  // byte 2*half of the word sits in halfword `half` of the even sums, byte 2*half+1 in halfword `half` of the odd sums
-  const int s0 = (int)((even >> (16 * half)) & 0xFFFFu) - off, s1 = (int)((odd >> (16 * half)) & 0xFFFFu) - off;
-  const int q0 = hq_clamp_ll(hq_dn(s0, bb.x, cc.x), 0, qmin, qmax);
-  const int q1 = hq_clamp_ll(hq_dn(s1, bb.y, cc.y), 0, qmin, qmax);
-  out[((long long)img * ch + ch0) >> 1] = (unsigned short)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
+    for (int sl = 0; sl < SLICES; ++sl) { even += part[sl][2 * word][gl]; odd += part[sl][2 * word + 1][gl]; }
+    // byte 2*half of the word sits in halfword `half` of the even sums, byte 2*half+1 in halfword `half` of the odd sums
+    const int s0 = (int)((even >> (16 * half)) & 0xFFFFu) - off, s1 = (int)((odd >> (16 * half)) & 0xFFFFu) - off;
+    const int q0 = hq_clamp_ll(hq_dn(s0, __ldg(b + ch0), __ldg(c + ch0)), 0, qmin, qmax);
+    const int q1 = hq_clamp_ll(hq_dn(s1, __ldg(b + ch0 + 1), __ldg(c + ch0 + 1)), 0, qmin, qmax);
+    out[((long long)img * ch + ch0) >> 1] = (unsigned short)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
+  }
+}
+
+template <int SLICES>
+void launch_avgpool_vec16(const void* in, int n, int hw, int ch, int in_signed, const int32_t* b, const int32_t* c,
+                          int qmin, int qmax, void* out, cudaStream_t s) {
+  const dim3 grid((ch / 16 + 31) / 32, n), block(32, SLICES);
+  if (in_signed) avgpool_vec16_kernel<SLICES, true><<<grid, block, 0, s>>>((const uint4*)in, hw, ch, b, c, qmin, qmax, (unsigned short*)out);
+  else avgpool_vec16_kernel<SLICES, false><<<grid, block, 0, s>>>((const uint4*)in, hw, ch, b, c, qmin, qmax, (unsigned short*)out);
 }
 
 __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int in_bits, int in_signed,
@@ -791,6 +930,14 @@ cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t 
       default: return launch_requant8<true, true, true>(a, grid, block, words, lo, hi, sm_count, s);
     }
   }
+  // INT32 main operand, 8-bit output (and residual, if any): flat kernel when the quads of a pixel divide the block
+  if (a.main_bits == 32 && a.out_bits == 8 && (!a.res || a.res_bits == 8) && a.ch % 4 == 0 && words <= 256 &&
+      (words & (words - 1)) == 0) {
+    const int lo = a.relu ? (a.qmin > 0 ? a.qmin : 0) : a.qmin, hi = a.qmax;
+    if (!a.res) return launch_requant32<false, false>(a, words, lo, hi, sm_count, s);
+    if (a.res_signed) return launch_requant32<true, true>(a, words, lo, hi, sm_count, s);
+    return launch_requant32<true, false>(a, words, lo, hi, sm_count, s);
+  }
   const int groups = a.ch / 16;
   if (a.ch % 16 == 0 && groups <= 256) {
     const int ppb = 256 / groups;
@@ -815,8 +962,10 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
                               void* out, int out_bits, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
   if (in_bits == 8 && out_bits == 8 && ch % 16 == 0 && h * w <= 257 && n <= 65535) {
-    const dim3 grid((ch / 16 + 31) / 32, n), block(32, kAvgSlices);
-    avgpool_vec16_kernel<<<grid, block, 0, s>>>((const uint4*)in, h * w, ch, in_signed, b, c, qmin, qmax, (unsigned short*)out);
+    const int hw = h * w;
+    if (hw >= 128) launch_avgpool_vec16<8>(in, n, hw, ch, in_signed, b, c, qmin, qmax, out, s);
+    else if (hw >= 64) launch_avgpool_vec16<4>(in, n, hw, ch, in_signed, b, c, qmin, qmax, out, s);
+    else launch_avgpool_vec16<2>(in, n, hw, ch, in_signed, b, c, qmin, qmax, out, s);
   } else if (in_bits == 8 && out_bits == 8 && ch % 4 == 0 && h * w <= 257 && n <= 65535) {
     const dim3 grid((ch / 4 + 63) / 64, n), block(64, 4);
     avgpool_vec4_sliced_kernel<<<grid, block, 0, s>>>((const unsigned*)in, h * w, ch, in_signed, b, c, qmin, qmax, (unsigned*)out);

@@ -237,6 +237,46 @@ def test_residual_add(hq, main_bits, res_bits, out_bits, ch):
     assert np.array_equal(host(out, ref), ref)
 
 
+@pytest.mark.parametrize("ch,res_signed,out_signed,shifts", [
+    (64, None, 0, "wide"), (256, 0, 0, "wide"), (128, 1, 1, "every"), (1024, 0, 0, "every"), (4, None, 1, "every"),
+    (64, 0, 0, "clamp"),
+])
+def test_residual_add_int32_main_flat_kernel(hq, ch, res_signed, out_signed, shifts):
+    """INT32 main operand -> 8-bit output on the flat kernel: full-range accumulators, shifts 1..62 (threads with a
+    shift below 32 take the 64-bit form), signed / unsigned residual and output, clamp bounds inside the range."""
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(307, ch, out_signed)
+    shape = (1, 83, 61, ch)                    # 5063 pixels: several block trips and a ragged last one
+    main = g.integers(-(1 << 31), 1 << 31, size=shape, dtype=np.int64).astype(np.int32)
+    main[0, :4] >>= 12                         # some rows of moderate size, so that not everything saturates
+    mb, rb = (g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32) for _ in range(2))
+    if shifts == "every":
+        mc = (np.arange(ch) % 62 + 1).astype(np.int32)
+        rc = ((np.arange(ch) * 7) % 62 + 1).astype(np.int32)
+    else:
+        mc = g.integers(50, 58, size=ch).astype(np.int32)
+        rc = g.integers(29, 34, size=ch).astype(np.int32)
+    res = None
+    if res_signed is not None:
+        res = (g.integers(-128, 128, size=shape, dtype=np.int64).astype(np.int8) if res_signed else
+               g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8))
+    qmin, qmax = (-128, 127) if out_signed else (0, 255)
+    if shifts == "clamp":
+        qmin, qmax = 7, 201
+    relu = 0 if out_signed else 1
+    ref = oracle().residual_add(main, 32, 1, mb, mc, res, 8 if res is not None else 0, res_signed or 0,
+                                rb if res is not None else None, rc if res is not None else None, ch, relu, qmin, qmax,
+                                8, out_signed)
+    out = binding.alloc_out(*shape[:3], ch, 8, out_signed)
+    st = hq.residual_add(binding.to_device(main), 32, 1, binding.to_device(mb), binding.to_device(mc),
+                         binding.to_device(res), 8 if res is not None else 0, res_signed or 0,
+                         binding.to_device(rb) if res is not None else None, binding.to_device(rc) if res is not None else None,
+                         ch, relu, qmin, qmax, out, 8, out_signed)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
 def test_residual_add_8bit_fast_kernel_every_shift(hq):
     """8-bit operands take the 32-bit kernel; shifts from 1 to 62, signed and unsigned, both outputs."""
     from paper_2011_10680_b200 import binding
@@ -279,6 +319,9 @@ LARGE_ELT_CASES = [
     ((331, 251), 128, 0, None, 8, "fast"),
     ((331, 251), 128, 1, 1, 4, "every"),
     ((499, 333), 64, 0, 1, 8, "every"),
+    ((331, 251), 128, 0, None, 4, "fast"),     # 4-bit output packed from high nibbles (shifts reduced by four)
+    ((331, 251), 128, 1, None, 4, "every"),    # the same with shifts below four in some warps (plain clamp there)
+    ((157, 131), 128, 0, None, 4, "every"),
 ]
 
 
