@@ -162,7 +162,7 @@ def run_reference(args, rank):
 
 def run_sweep(args):
     """Config 5: fused conv/GEMM sweep over the ResNet-50 layer shapes (INT8 and INT4, with and without the
-    residual add); per shape device time (CUDA events, L2 flushed between repetitions by writing 256 MB),
+    residual add); per shape device time (CUDA events, L2 flushed between repetitions by writing 256 MB and then reading another 256 MB),
     integer TOPS, achieved GB/s of the algorithmic bytes and the fraction of that shape's own roofline."""
     import torch
     from paper_2011_10680_b200 import binding, build
@@ -170,6 +170,7 @@ def run_sweep(args):
     hq = binding.Handle(0)
     hbm_peak, bf16_peak, peak_kind = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush_r = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")
     rows = []
     shapes = inputs.SWEEP_LAYERS if args.sweep_only < 0 else [inputs.SWEEP_LAYERS[args.sweep_only]]
     for (hw, cin, cout, k, stride, has_res) in shapes:
@@ -181,6 +182,7 @@ def run_sweep(args):
                 times = []
                 for rep in range(args.warmup + args.steps):
                     flush.fill_(rep & 0xFF)
+                    flush_r.view(torch.int32).sum()    # then 256 MB read: no backlog of dirty lines charged to the timed kernel
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
                     st, out = hq.conv_case(case, dev)
@@ -214,7 +216,7 @@ def run_sweep(args):
 def run_membound(args):
     """The memory-bound kernels on their own, at ResNet-50 batch-256 tensor sizes (each operand larger than L2):
     max pooling, dyadic requantization, the two-branch residual add and the average-pool requantization.  Device
-    time per call (CUDA events, 256 MB written between repetitions), achieved GB/s of the algorithmic bytes
+    time per call (CUDA events; 256 MB written, then 256 MB read between repetitions), achieved GB/s of the algorithmic bytes
     (every operand read once, the result written once) and its fraction of the measured copy bandwidth."""
     import torch
     from paper_2011_10680_b200 import binding, build
@@ -222,6 +224,7 @@ def run_membound(args):
     hq = binding.Handle(0)
     hbm_peak, _, peak_kind = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush_r = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")
     g = torch.Generator(device="cuda"); g.manual_seed(7)
     ri = lambda lo, hi, shape, dt: torch.randint(lo, hi, shape, generator=g, device="cuda", dtype=torch.int32).to(dt)
     u8 = lambda *shape: ri(0, 256, shape, torch.uint8)
@@ -252,14 +255,11 @@ def run_membound(args):
     cases.append(("avgpool requant u8 [%d,7,7,2048]" % na, xa.numel() + oa.numel(),
                   lambda: hq.avgpool_requant(xa, 2048, 8, 0, ba, ca, 0, 255, oa, 8, 0)))
     rows = []
-    flush_r = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for name, byt, fn in cases:
         times = []
         for rep in range(args.warmup + args.steps):
-            # 256 MB written, then 256 MB read: the L2 holds neither the operands nor a backlog of dirty lines
-            # whose write-back would be charged to the timed kernel
             flush.fill_(rep & 0xFF)
-            flush_r.view(torch.int32).sum()
+            flush_r.view(torch.int32).sum()    # then 256 MB read: no backlog of dirty lines charged to the timed kernel
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             st = fn()
@@ -300,6 +300,7 @@ def run_sweep_grid(args):
     hq = binding.Handle(0)
     hbm_peak, bf16_peak, peak_kind = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush_r = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")
     g = torch.Generator(device="cuda"); g.manual_seed(5)
     ri = lambda lo, hi, shape, dt: torch.randint(lo, hi, shape, generator=g, device="cuda", dtype=torch.int32).to(dt)
     rows = []
@@ -323,6 +324,7 @@ def run_sweep_grid(args):
                         times = []
                         for rep in range(args.warmup + args.steps):
                             flush.fill_(rep & 0xFF)
+                            flush_r.view(torch.int32).sum()    # then 256 MB read: no backlog of dirty lines charged to the timed kernel
                             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                             e0.record()
                             st = hq.conv2d(x, bits, 0, cin, w, cout, k, k, 1, k // 2, bias, b, c, out, 8, 0,

@@ -90,7 +90,10 @@ typedef struct {       /* one row of the per-layer table; layer i produces tenso
   int32_t relu, qmin, qmax;              /* AVGPOOL / ADD / REQUANT (CONV uses conv.*) */
 } hq_layer;
 
-/* Create / destroy the per-device context.  `device` is a CUDA ordinal.  Host call. */
+/* Create / destroy the per-device context.  `device` is a CUDA ordinal.  Host call.
+ * A handle owns small device buffers that its calls reuse (a status word, scratch for lowered or widened
+ * operands, the narrow multiply-add pairs of a large element-wise call): calls through ONE handle must be
+ * ordered on the device (one stream, or streams joined by events); use one handle per concurrent stream. */
 hq_status hq_create(int32_t device, hq_handle** out);
 hq_status hq_destroy(hq_handle* h);
 

@@ -241,13 +241,11 @@ static hq_status residual_add_impl(hq_handle* h, const hq_tensor* main_t, hq_dya
   if (!m_narrow && main_t->bits == 8 && (!res || res->bits == 8) && out->c <= kNarrowChannels &&
       a.pixels * a.ch >= (1ll << 25)) {
     char* base = (char*)h->narrow_pairs;
-    if (hq_launch_residual_narrow(a.mb, a.mc, a.main_signed, a.ch, base, s) != cudaSuccess) return HQ_ERR_CUDA;
+    char* base1 = res ? base + (size_t)kNarrowChannels * 16 : nullptr;
+    if (hq_launch_residual_narrow2(a.mb, a.mc, a.main_signed, base, a.rb, a.rc, a.res_signed, base1, a.ch, s) != cudaSuccess)
+      return HQ_ERR_CUDA;
     a.m_narrow = base;
-    if (res) {
-      if (hq_launch_residual_narrow(a.rb, a.rc, a.res_signed, a.ch, base + (size_t)kNarrowChannels * 16, s) != cudaSuccess)
-        return HQ_ERR_CUDA;
-      a.r_narrow = base + (size_t)kNarrowChannels * 16;
-    }
+    a.r_narrow = base1;
   }
   return hq_launch_residual_add(a, h->sm_count, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }

@@ -870,23 +870,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 // channel tries the two neighbouring multipliers and checks all 256 inputs; channels without such a pair
 // are marked invalid and keep the wide form.  Run once per layer when a network is built, and ahead of a
 // single large element-wise call.
-__global__ void __launch_bounds__(128) residual_narrow_kernel(const int32_t* __restrict__ rb, const int32_t* __restrict__ rc,
-                                                              int is_signed, int n, int4* __restrict__ out) {
-  // one warp per channel: lane l checks the inputs l, l + 32, ... for both candidate multipliers
-  const int ch = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (ch >= n) return;
-  const long long b = rb[ch];
-  const int c = rc[ch];
+struct NarrowJob { const int32_t* rb; const int32_t* rc; int is_signed; int4* out; };
+
+__global__ void __launch_bounds__(128) residual_narrow_kernel(NarrowJob j0, NarrowJob j1, int n) {
+  // one warp per channel: lane l checks the inputs l, l + 32, ... for both candidate multipliers; warps past the
+  // first n channels serve the second job (the other operand of an element-wise call), if there is one
+  int ch = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const bool second = ch >= n;
+  if (second) ch -= n;
+  const NarrowJob& j = second ? j1 : j0;
+  if (ch >= n || !j.out) return;
+  const long long b = j.rb[ch];
+  const int c = j.rc[ch];
   int4 res = make_int4(0, 0, 0, 0);
-  const int r_lo = is_signed ? -128 : 0;
+  const int r_lo = j.is_signed ? -128 : 0;
   if (c >= 41 && c <= 62) {
     res = make_int4(0, 0, 0, 1);                       // |r*rb| < 2^39 <= 2^(rc-2): the term is 0 for every r
   } else if (c >= 9 && c <= 38) {
     const int s = c - 8, a = 1 << (s - 1);
     const long long m0 = b >> 8, m1 = m0 + 1;
     bool same0 = m0 <= (1 << 23), same1 = m1 <= (1 << 23);
-    for (int j = 0; j < 8; ++j) {
-      const int r = r_lo + lane + 32 * j;
+    for (int k = 0; k < 8; ++k) {
+      const int r = r_lo + lane + 32 * k;
       const long long exact = ((long long)r * b + (1LL << (c - 1))) >> c;
       same0 = same0 && exact == (long long)((r * (int)m0 + a) >> s);
       same1 = same1 && exact == (long long)((r * (int)m1 + a) >> s);
@@ -896,7 +902,7 @@ __global__ void __launch_bounds__(128) residual_narrow_kernel(const int32_t* __r
     if (same0) res = make_int4((int)m0, a, s, 1);
     else if (same1) res = make_int4((int)m1, a, s, 1);
   }
-  if (lane == 0) out[ch] = res;
+  if (lane == 0) j.out[ch] = res;
 }
 
 // ---------------------------------------------------------------- host side ------------------
@@ -1144,8 +1150,16 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
 
 cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
                                       cudaStream_t s) {
+  return hq_launch_residual_narrow2(rb, rc, res_signed, out, nullptr, nullptr, 0, nullptr, channels, s);
+}
+
+cudaError_t hq_launch_residual_narrow2(const int32_t* b0, const int32_t* c0, int signed0, void* out0,
+                                       const int32_t* b1, const int32_t* c1, int signed1, void* out1, int channels,
+                                       cudaStream_t s) {
   if (channels <= 0) return cudaSuccess;
-  residual_narrow_kernel<<<(channels + 3) / 4, 128, 0, s>>>(rb, rc, res_signed, channels, (int4*)out);
+  const NarrowJob j0{b0, c0, signed0, (int4*)out0}, j1{b1, c1, signed1, (int4*)out1};
+  const int warps = out1 ? 2 * channels : channels;
+  residual_narrow_kernel<<<(warps + 3) / 4, 128, 0, s>>>(j0, j1, channels);
   return cudaGetLastError();
 }
 

@@ -86,6 +86,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
 // Fills `out` (channels x 16 bytes) with the narrow residual pairs of an 8-bit residual branch.
 cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,
                                       cudaStream_t s);
+// The same for the two operands of an element-wise call in one launch (`out1` NULL: first operand only).
+cudaError_t hq_launch_residual_narrow2(const int32_t* b0, const int32_t* c0, int signed0, void* out0,
+                                       const int32_t* b1, const int32_t* c1, int signed1, void* out1, int channels,
+                                       cudaStream_t s);
 // Lowered path for thin first layers: patch matrix + padded weights in scratch, then the tensor-core kernel.
 bool hq_conv_lowering_applies(const ConvArgs& a);
 size_t hq_conv_lowering_bytes(const ConvArgs& a);
