@@ -75,7 +75,17 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   cudaStream_t s = (cudaStream_t)stream;
   const bool tc_ok = hq_conv_tc_supported(a);
   if (h->conv_path == 2 && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
-  if (h->conv_path != 1 && tc_ok) return hq_launch_conv_tc(h, a, s);
+  if (h->conv_path != 1 && tc_ok) {
+    // A single large call with an 8-bit residual: its narrow residual pairs are worked out first, in the handle's
+    // buffer (a network prepares them once when it is built); one small launch that the cheaper epilogue repays.
+    if (a.res && a.res_bits == 8 && !a.res_narrow && a.cout <= kNarrowChannels &&
+        (long long)a.n * ho * wo * a.cout >= (1ll << 25) &&
+        hq_launch_residual_narrow(a.rb, a.rc, a.res_signed, a.cout, h->narrow_pairs, s) == cudaSuccess) {
+      a.res_narrow = h->narrow_pairs;
+      a.res_narrow_fresh = 1;
+    }
+    return hq_launch_conv_tc(h, a, s);
+  }
   if (h->conv_path != 1 && hq_conv_widen4_applies(a)) {
     // packed 4-bit operands: widened copies in scratch, then the tensor-core kernel
     const size_t need = hq_conv_widen4_bytes(a);

@@ -79,6 +79,7 @@ struct TcParams {
   const int32_t* bias; const int32_t* b; const int32_t* c;
   const void* res; int32_t res_bits, res_signed; const int32_t* rb; const int32_t* rc;
   const int4* res_narrow;   // optional per-channel {m, a, s, valid} from residual_narrow_kernel
+  int32_t narrow_fresh;     // 1: the pairs are written by the kernel launched just before this one
   int32_t relu, qmin, qmax;
   void* out; int32_t out_bits;
   uint32_t* status;
@@ -820,6 +821,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // narrow residual pairs, when the caller prepared them and every channel of this warp has one
     bool warp_narrow = false;
     if (fast && !warp_small && p.res && p.res_narrow) {
+      if (p.narrow_fresh) asm volatile("griddepcontrol.wait;" ::: "memory");
       const int4 nr = ch_live ? p.res_narrow[ch] : make_int4(0, 0, 0, 1);
       warp_narrow = __all_sync(0xffffffffu, nr.w != 0) != 0;
       if (warp_narrow) { k.rb = nr.x; k.rh = nr.y; k.rsh = nr.z; }
@@ -1038,26 +1040,30 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     p.k_blocks = a.kh * a.kw * p.cchunks;
     const int smem_budget = 212 * 1024;                // dynamic bytes after the 1024-byte alignment slack
     // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
-    for (int cap = 256; cap >= 64; cap >>= 1) {        // largest pixel tile that leaves room for >= 3 stages
+    bool chosen = false;
+    for (int cap = 256; cap >= 64 && !chosen; cap >>= 1) {   // largest pixel tile that leaves room for >= 3 stages
       p.pt = pick_pt(P, p.c_tiles, h->sm_count, cap);
-      // a weight slab of at most 72 KiB stays resident (the stages then hold activations only): a third less
-      // traffic into shared memory per K block
-      wres_bytes = p.k_blocks * kTileC * p.bkb;
-      p.wres = wres_bytes <= 72 * 1024 ? 1 : 0;
-      if (!p.wres) wres_bytes = 0;
-      stage_bytes = ((p.wres ? 0 : kTileC) + p.pt) * p.bkb;
-      p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
-      p.halves = p.pt >= (p.fold ? 256 : 128) ? 2 : 1;
-      out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
-      p.lg_bufs = p.pt <= 128 ? 2 : 1;
-      res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
-      // residual tiles: as many buffers as accumulators, fewer when a long reduction needs the room for stages
-      // (its epilogue has slack: a single residual buffer only delays the next tile's prefetch)
-      for (p.lg_rbufs = p.lg_bufs; ; --p.lg_rbufs) {
-        stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_rbufs) - wres_bytes) / stage_bytes;
-        if (stages >= 3 || p.lg_rbufs == 0 || !res_tile_bytes || k_total < 1024) break;
+      // A weight slab of at most 72 KiB stays resident (the stages then hold activations only): a third less
+      // traffic into shared memory per K block.  Where the slab would cost the larger pixel tile its stages, the
+      // tile wins and the weights travel with the stages.
+      for (int keep_w = 1; keep_w >= 0 && !chosen; --keep_w) {
+        wres_bytes = p.k_blocks * kTileC * p.bkb;
+        p.wres = (keep_w && wres_bytes <= 72 * 1024) ? 1 : 0;
+        if (!p.wres) { if (keep_w) continue; wres_bytes = 0; }
+        stage_bytes = ((p.wres ? 0 : kTileC) + p.pt) * p.bkb;
+        p.fold = (a.cout <= 64 && p.pt >= 128) ? 1 : 0;
+        p.halves = p.pt >= (p.fold ? 256 : 128) ? 2 : 1;
+        out_tile_bytes = p.staged_out ? 4 * p.pt * 32 : 0;
+        p.lg_bufs = p.pt <= 128 ? 2 : 1;
+        res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
+        // residual tiles: as many buffers as accumulators, fewer when a long reduction needs the room for stages
+        // (its epilogue has slack: a single residual buffer only delays the next tile's prefetch)
+        for (p.lg_rbufs = p.lg_bufs; ; --p.lg_rbufs) {
+          stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_rbufs) - wres_bytes) / stage_bytes;
+          if (stages >= 3 || p.lg_rbufs == 0 || !res_tile_bytes || k_total < 1024) break;
+        }
+        if (stages >= 3 || (p.pt == 64 && keep_w == 0)) chosen = true;
       }
-      if (stages >= 3 || p.pt == 64) break;
     }
   }
   p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
@@ -1072,6 +1078,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
+  p.narrow_fresh = a.res_narrow_fresh;
   p.relu = a.relu; p.qmin = a.qmin; p.qmax = a.qmax;
   p.out = a.out; p.out_bits = a.out_bits; p.out_signed = a.out_signed;
   {

@@ -61,6 +61,7 @@ struct ConvArgs {
   void* out; int32_t ho, wo, out_bits, out_signed;
   // internal (zero for calls that come straight from the ABI):
   const void* res_narrow;    // per-channel narrow residual pairs prepared by hq_launch_residual_narrow, or NULL
+  int32_t res_narrow_fresh;  // nonzero: the pairs come from the launch just before on the same stream (the kernel waits for it)
   const void* wgt_widened;   // 4-bit weights already widened to one byte per value (a network does it once), or NULL
   int32_t pad_after_delta;   // padding after the last row/column minus `pad`
   // byte pitches of the activation tensor along W, H and N when it is not dense (0: dense NHWC).  A W pitch
