@@ -199,7 +199,9 @@ hq_status hq_network_destroy(hq_network* net);
  */
 hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
 
-/* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail. */
+/* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail, 3 = like 2 and
+ * the tensor-core kernel's launch shapes are chosen by what the layer allows, not by its size (small test cases
+ * then reach the shapes of large layers). */
 hq_status hq_set_conv_path(hq_handle* h, int32_t path);
 
 const char* hq_status_string(hq_status s);

@@ -74,7 +74,7 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
   cudaStream_t s = (cudaStream_t)stream;
   const bool tc_ok = hq_conv_tc_supported(a);
-  if (h->conv_path == 2 && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
+  if (h->conv_path >= 2 && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
   if (h->conv_path != 1 && tc_ok) {
     // A single large call with an 8-bit residual: its narrow residual pairs are worked out first, in the handle's
     // buffer (a network prepares them once when it is built); one small launch that the cheaper epilogue repays.
@@ -193,7 +193,7 @@ hq_status hq_destroy(hq_handle* h) {
 }
 
 hq_status hq_set_conv_path(hq_handle* h, int32_t path) {
-  if (!h || path < 0 || path > 2) return HQ_ERR_INVALID_ARG;
+  if (!h || path < 0 || path > 3) return HQ_ERR_INVALID_ARG;
   h->conv_path = path;
   return HQ_OK;
 }

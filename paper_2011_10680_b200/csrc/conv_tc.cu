@@ -51,6 +51,8 @@ constexpr int kMaxAccBufs = 4;                                 // accumulator (a
 //         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
 constexpr int kSoloEpilogueWarps = 8;
 constexpr int kPairEpilogueWarps = 4;
+constexpr int kSoloIssuerWarps = 3;     // 1 + 3 + 8 warps = 384 threads: 168 registers per thread remain
+constexpr int kPairIssuerWarps = 1;
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;   // 2 s per wait
 
 struct TcParams {
@@ -66,9 +68,18 @@ struct TcParams {
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
+  int32_t ni;            // MMA issuer warps in use: min(issuer warps of the launch shape, k_blocks)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
   int32_t x_tiled;       // 1: X is a dense [P][cin] matrix (1x1, stride 1, no padding) fetched by a tiled map
+  // Strip mode (3x3, stride 1, pad 1): a tile is `rows` output rows of one image, laid out with a power-of-two
+  // pitch of 2^lg_wp positions (columns >= wo are scratch); one padded input patch per cin chunk feeds all nine taps.
+  int32_t strip;         // 1: strip mode
+  int32_t lg_wp, rows;   // log2 of the position pitch; output rows per tile (pt = rows << lg_wp)
+  int32_t tpi;           // tiles per image = ceil(ho / rows)
+  int32_t ho;            // output (= input) height
+  int32_t npatch;        // patch buffers (2 or 3)
+  uint32_t patch_bytes, patch_off;   // bytes of one patch [(rows+3) << lg_wp][bkb]; offset from the 1024-aligned base
   uint32_t tmem_cols;
   // epilogue
   int32_t staged_out;    // 1: bytes leave through per-warp staging boxes and TMA stores
@@ -98,10 +109,12 @@ struct SharedCtl {
   unsigned long long empty[kMaxStages];
   unsigned long long tfull[kMaxAccBufs];
   unsigned long long tempty[kMaxAccBufs];
+  unsigned long long tstart[kMaxAccBufs];   // the tile's first (overwriting) MMA has been issued
   unsigned long long rfull[kMaxAccBufs];
   unsigned long long rempty[kMaxAccBufs];
   unsigned long long drain;
   unsigned long long wfull;              // resident weight slab landed
+  unsigned long long pfull[3], pempty[3];  // strip mode: input patches
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -163,6 +176,15 @@ __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap*
       "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
       " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h, int n) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c, int w, int h, int n) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(map), "r"(src), "r"(c), "r"(w), "r"(h), "r"(n) : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
@@ -309,6 +331,27 @@ __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) 
   return s;
 }
 
+// The finished staging box of one warp leaves for global memory.  Dense tiles: one [columns][32 B] box at pixel
+// `p_tile * pt + col0`.  Strip tiles: one box per 32 positions (a row, half a row or two rows of the pitch-2^lg_wp
+// raster); columns at or beyond the image width and rows at or beyond its height fall outside the tensor map
+// and are clipped by the copy.
+__device__ __forceinline__ void store_warp_box(const TcParams& p, const CUtensorMap* map_out, uint32_t my_stage, int chx,
+                                               int p_tile, int col0, int px_per_warp) {
+  if (!p.strip) {
+    const int p_base = p_tile * p.pt + col0;
+    if (p_base < p.P) { tma_store_2d(map_out, my_stage, chx, p_base); tma_store_commit(); }
+    return;
+  }
+  const int img = p_tile / p.tpi, y0 = (p_tile - img * p.tpi) * p.rows;
+  bool any = false;
+  for (int c = 0; c < (px_per_warp >> 5); ++c) {
+    const int j0 = col0 + 32 * c;
+    const int y = y0 + (j0 >> p.lg_wp), x = j0 & ((1 << p.lg_wp) - 1);
+    if (y < p.ho && x < p.wo) { tma_store_4d(map_out, my_stage + (uint32_t)c * 1024u, chx, x, y, img); any = true; }
+  }
+  if (any) tma_store_commit();
+}
+
 // Everything an epilogue warp needs, gathered once so the tile loops can live in their own functions.
 struct EpiCtx {
   const TcParams* p; SharedCtl* ctl; const CUtensorMap* map_out;
@@ -372,7 +415,6 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     if (lane == 0) HQ_TRACE(3, tcount * 8 + e.ew);
     const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;       // residual buffer and its phase
     if (RES && !wait_bar(&ctl.rfull[rs], rph)) break;
-    const int p_base = p_tile * p.pt + col0;
     const uint8_t* const res_tile = res_stage_ptr + rs * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
     const uint32_t t_addr = t_warp + as * p.pt;
     const bool has_next = p_tile + tile_step < p.p_tiles;
@@ -415,12 +457,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     if (e.ew == 0 && lane == 0) HQ_TRACE(4, tcount);
     fence_async_smem();                           // make this lane's box writes visible to the TMA engine
     __syncwarp();
-    if (lane == 0) {
-      if (e.warp_live && p_base < p.P) {
-        tma_store_2d(e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_base);
-        tma_store_commit();
-      }
-    }
+    if (lane == 0 && e.warp_live) store_warp_box(p, e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_tile, col0, px_per_warp);
     if (e.ew == 0 && lane == 0) HQ_TRACE(7, tcount);
     if (!has_next || !ok) break;
     p_tile += tile_step; ++tcount; as = nas; aph = naph;
@@ -573,10 +610,8 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       if (lane == 0) {
         mbar_arrive(smem_u32(&ctl.tempty[as]));
         if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
-        if (p.staged_out && warp_live && p_base < p.P) {
-          tma_store_2d(&map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_base);
-          tma_store_commit();
-        }
+        if (p.staged_out && warp_live)
+          store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_tile, col0, px_per_warp);
       }
     }
 
@@ -584,8 +619,8 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 }
 
 // ---------------------------------------------------------------- the kernel -----------------
-template <int EPI_WARPS, int MIN_CTAS>
-__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
+template <int EPI_WARPS, int MIN_CTAS, int MMA_WARPS>
+__global__ void __launch_bounds__(32 * (1 + MMA_WARPS + EPI_WARPS), MIN_CTAS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
                const __grid_constant__ TcParams p) {
@@ -595,7 +630,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // operand stages, 1024-byte aligned
   const uint32_t w_bytes = kTileC * p.bkb;
-  const uint32_t x_bytes = p.pt * p.bkb;
+  const uint32_t x_bytes = p.strip ? 0u : (uint32_t)(p.pt * p.bkb);   // strip mode: the stages carry weights only
   const uint32_t x_off = p.wres ? 0u : w_bytes;          // offset of the X tile inside a stage
   const uint32_t stage_bytes = x_off + x_bytes;
   const uint32_t out_stage = tiles + p.out_stage_off;
@@ -611,11 +646,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&ctl.full[s]), 1); mbar_init(smem_u32(&ctl.empty[s]), 1); }
     for (int s = 0; s < (1 << p.lg_bufs); ++s) {
-      mbar_init(smem_u32(&ctl.tfull[s]), 1); mbar_init(smem_u32(&ctl.tempty[s]), 4 * p.halves);
+      mbar_init(smem_u32(&ctl.tfull[s]), p.ni); mbar_init(smem_u32(&ctl.tempty[s]), 4 * p.halves);
+      mbar_init(smem_u32(&ctl.tstart[s]), 1);
       mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), 4 * p.halves);
     }
-    mbar_init(smem_u32(&ctl.drain), 1);
+    mbar_init(smem_u32(&ctl.drain), p.ni);
     mbar_init(smem_u32(&ctl.wfull), 1);
+    for (int s = 0; s < 3; ++s) { mbar_init(smem_u32(&ctl.pfull[s]), 1); mbar_init(smem_u32(&ctl.pempty[s]), p.ni); }
     ctl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -664,7 +701,40 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           }
         }
       }
-      for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
+      uint32_t pit = 0;                                // strip mode: patches started
+      if (p.strip) {
+        uint32_t ps = 0, pph = 0;
+        for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
+          const int img_s = p_tile / p.tpi, y0 = (p_tile - img_s * p.tpi) * p.rows;
+          for (int chunk = 0; chunk < p.cchunks && ok; ++chunk) {
+            // the padded patch of this cin chunk: columns -1 .. 2^lg_wp - 2, rows y0-1 .. y0+rows+1 (zeros outside the image)
+            if (!mbar_wait(smem_u32(&ctl.pempty[ps]), pph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+            HQ_TRACE(9, pit);
+            const uint32_t pbar = smem_u32(&ctl.pfull[ps]);
+            mbar_expect_tx(pbar, p.patch_bytes);
+            tma_load_4d(tiles + p.patch_off + ps * p.patch_bytes, &map_x, pbar, chunk * p.bkb, -1, y0 - 1, img_s);
+            ++pit;
+            if (++ps == (uint32_t)p.npatch) { ps = 0; pph ^= 1u; }
+            if (p.wres) continue;
+            for (int tap = 0; tap < 9; ++tap, ++it) {      // the nine weight blocks that meet this patch
+              if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+              HQ_TRACE(0, it);
+              const uint32_t bar = smem_u32(&ctl.full[s]);
+              const uint32_t w_dst = tiles + s * stage_bytes;
+              const int kb = tap * p.cchunks + chunk;
+              mbar_expect_tx(bar, stage_bytes);
+              if (p.fold) {
+                tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, 0);
+                tma_load_2d(w_dst + 64 * p.bkb, &map_w, bar, kb * p.bkb, 0);
+              } else {
+                tma_load_2d(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
+              }
+              if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+            }
+          }
+        }
+      }
+      for (int p_tile = p_tile0; p_tile < p.p_tiles && ok && !p.strip; p_tile += p_step, ++tcount) {
         const int p0 = p_tile * p.pt;
         const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad, img_now = img;
         ow += d_ow; if (ow >= p.wo) { ow -= p.wo; ++oh; }
@@ -703,6 +773,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
       // Drain: every copy this thread started must have landed before the CTA may exit.
       const uint32_t issued = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
+      for (uint32_t j = 0; j < (p.npatch > 0 ? (pit < (uint32_t)p.npatch ? pit : (uint32_t)p.npatch) : 0u); ++j) {
+        const uint32_t k = pit - 1 - j;
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(smem_u32(&ctl.pfull[k % p.npatch]), (k / p.npatch) & 1u)) {
+          if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
+        }
+      }
       for (uint32_t j = 0; j < issued; ++j) {
         const uint32_t k = it - 1 - j;
         const uint32_t ds = k % p.stages, dph = (k / p.stages) & 1u;
@@ -728,19 +805,37 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (elect_one()) {
+  } else if (warp <= MMA_WARPS) {
+    // ------------------------------------------------------------ MMA issuers
+    // The K blocks of the CTA's tiles, numbered through (g = tile * k_blocks + b), are dealt round-robin to p.ni
+    // issuer warps (one lane each).  A single thread cannot keep the tensor pipe busy: every shared-memory
+    // operation it executes between two batches of MMAs (the wait for the next operands) holds it for a few hundred
+    // cycles while its own MMAs are in flight, and the pipe drains meanwhile; with the waits of one issuer falling
+    // into the MMAs of the others the pipe stays fed.  The stage count is a multiple of p.ni, so a stage is always
+    // read by the same issuer: its parity waits then follow one another like a single thread's (a thread that
+    // looked at a stage's barrier a whole fill early would take the fill before for its own).  Integer accumulation
+    // does not care about the order of the blocks; only the tile's first MMA, which overwrites the accumulator,
+    // must come first: whoever issues it signals `tstart` and the others wait for that.
+    const int iss = warp - 1;
+    if (iss < p.ni && elect_one()) {
       // instruction descriptor: D = S32, A = s8 weights, B = u8/s8 activations, both K-major, M = 128, N = pt
       const uint32_t idesc = (2u << 4) | (1u << 7) | ((uint32_t)(p.x_signed ? 1 : 0) << 10) |
                              ((uint32_t)(p.pt >> 3) << 17) | ((uint32_t)(kTileC >> 4) << 24);
-      uint32_t it = 0, tcount = 0, s = 0, ph = 0;
+      const uint32_t ni = (uint32_t)p.ni, nstages = (uint32_t)p.stages;
+      const bool ring = !(p.strip && p.wres);                 // do the blocks travel through the stage ring?
+      uint32_t tcount = 0, s = 0, ph = 0;
+      auto advance = [&](uint32_t d) { s += d; while (s >= nstages) { s -= nstages; ph ^= 1u; } };
+      if (ring) advance((uint32_t)iss);
+      int b = iss;                                           // my next block of the current tile
       const uint32_t bmask = (1u << p.lg_bufs) - 1u;
       bool ok = true;
       const uint64_t desc_hi = smem_desc(0, p.bkb);           // everything but the start address
       const int ksteps = p.bkb >> 5;
       if (p.wres && !mbar_wait(smem_u32(&ctl.wfull), 0, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) ok = false;
-      for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
+      // One issuer, plain form: the lean loop (the hand-over chain of short reductions is latency bound, every
+      // instruction on it counts).
+      const bool lean = ni == 1 && !p.strip;
+      for (int p_tile = p_tile0; p_tile < p.p_tiles && ok && lean; p_tile += p_step, ++tcount) {
         const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
         // The operands of the tile's first K block have usually landed long ago; looking at them first
         // keeps that check off the path between the epilogue's hand-back and the first MMA.
@@ -749,22 +844,85 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         tc_fence_after();
         HQ_TRACE(11, tcount);
         const uint32_t d_tmem = tmem_base + as * p.pt;
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (kb > 0 && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
-          HQ_TRACE(1, it);
+          HQ_TRACE(1, tcount * (uint32_t)p.k_blocks + (uint32_t)kb);
           const uint32_t w_addr = tiles + s * stage_bytes;
           const uint32_t a_addr = p.wres ? tiles + p.wres_off + (uint32_t)kb * w_bytes : w_addr;
           uint64_t adesc = desc_hi | (uint64_t)((a_addr >> 4) & 0x3FFF);
           uint64_t bdesc = desc_hi | (uint64_t)(((w_addr + x_off) >> 4) & 0x3FFF);
           for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
             mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
-          HQ_TRACE(5, it);
+          HQ_TRACE(5, tcount * (uint32_t)p.k_blocks + (uint32_t)kb);
           // the accumulator's barrier first on the last K block: the epilogue is the one waiting
           if (kb + 1 == p.k_blocks) mma_commit(smem_u32(&ctl.tfull[as]));
           mma_commit(smem_u32(&ctl.empty[s]));     // frees the stage when these MMAs have read it
-          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+          if (++s == nstages) { s = 0; ph ^= 1u; }
         }
         HQ_TRACE(2, tcount);
+      }
+      for (int p_tile = p_tile0; p_tile < p.p_tiles && ok && !lean; p_tile += p_step, ++tcount) {
+        const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
+        const uint32_t d_tmem = tmem_base + as * p.pt;
+        bool first = true;
+        int cur_chunk = -1;
+        uint32_t ps = 0;
+        for (; b < p.k_blocks; b += (int)ni) {
+          uint32_t a_addr, b_addr;
+          if (p.strip) {
+            // block b = (cin chunk, filter tap): the chunk's patch, read from (tr << lg_wp) + ts rows further on.
+            // The start is then not aligned to the swizzle pattern's eight rows, which needs nothing more: the
+            // pattern is a function of the shared-memory address, for the copy that wrote the patch and for the
+            // MMA that reads it alike (the descriptor's base-offset field stays 0; a phase there gives wrong sums).
+            const int chunk = b / 9, tap = b - 9 * chunk, tr = tap / 3, ts = tap - 3 * tr;
+            if (chunk != cur_chunk) {
+              if (cur_chunk >= 0) mma_commit(smem_u32(&ctl.pempty[ps]));    // my MMAs on the previous patch
+              cur_chunk = chunk;
+              const uint32_t pidx = tcount * (uint32_t)p.cchunks + (uint32_t)chunk;
+              ps = pidx % (uint32_t)p.npatch;
+              if (!mbar_wait(smem_u32(&ctl.pfull[ps]), (pidx / (uint32_t)p.npatch) & 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+              HQ_TRACE(10, pidx);
+            }
+            b_addr = tiles + p.patch_off + ps * p.patch_bytes + (uint32_t)(((tr << p.lg_wp) + ts) * p.bkb);
+            if (p.wres) {
+              a_addr = tiles + p.wres_off + (uint32_t)(tap * p.cchunks + chunk) * w_bytes;
+            } else {
+              if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+              a_addr = tiles + s * stage_bytes;
+            }
+          } else {
+            if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+            const uint32_t w_addr = tiles + s * stage_bytes;
+            a_addr = p.wres ? tiles + p.wres_off + (uint32_t)b * w_bytes : w_addr;
+            b_addr = w_addr + x_off;
+          }
+          if (first) {
+            // The operands of this issuer's first block have usually landed long ago; looking at them first keeps
+            // that check off the path between the epilogue's hand-back and the first MMA.
+            if (!mbar_wait(smem_u32(&ctl.tempty[as]), aph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+            if (b != 0 && !mbar_wait(smem_u32(&ctl.tstart[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+            tc_fence_after();
+            if (b == 0) HQ_TRACE(11, tcount);
+            first = false;
+          }
+          HQ_TRACE(1, tcount * (uint32_t)p.k_blocks + (uint32_t)b);
+          uint64_t adesc = desc_hi | (uint64_t)((a_addr >> 4) & 0x3FFF);
+          uint64_t bdesc = desc_hi | (uint64_t)((b_addr >> 4) & 0x3FFF);
+          for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
+            mma_i8(d_tmem, adesc, bdesc, idesc, (b | k) ? 1u : 0u);
+          HQ_TRACE(5, tcount * (uint32_t)p.k_blocks + (uint32_t)b);
+          if (b == 0 && ni > 1) mbar_arrive(smem_u32(&ctl.tstart[as]));   // the overwriting MMA is on its way
+          // the accumulator's barrier first on this issuer's last block: the epilogue is the one waiting
+          if (b + (int)ni >= p.k_blocks) mma_commit(smem_u32(&ctl.tfull[as]));
+          if (ring) {
+            mma_commit(smem_u32(&ctl.empty[s]));     // frees the stage when these MMAs have read it
+            advance(ni);                             // my next block, in this tile or the next
+          }
+        }
+        if (!ok) break;
+        if (p.strip && cur_chunk >= 0) mma_commit(smem_u32(&ctl.pempty[ps]));
+        b -= p.k_blocks;                             // the numbering runs on into the next tile
+        if (iss == 0) HQ_TRACE(2, tcount);
       }
       // Drain: all issued MMAs must have completed before tensor memory is freed.
       mma_commit(smem_u32(&ctl.drain));
@@ -774,9 +932,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..9)
+    // ------------------------------------------------------------ epilogue (the last EPI_WARPS warps)
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read: channels 32q..32q+31
-    const int ew = warp - 2;                      // 0..7
+    const int ew = warp - (1 + MMA_WARPS);        // 0..7
     const int half = ew >> 2;                     // which half of its lane quarter's pixel columns this warp owns
     // Channel tiles of at most 64 channels are folded: the weight rows are loaded twice, so accumulator
     // lanes 64-127 repeat lanes 0-63, and lane quarters 2-3 take the second half of the pixel columns
@@ -975,9 +1133,9 @@ int pick_pt(long long pixels, int c_tiles, int sm_count, int cap) {
 // tensor-map encoders and the kernel's dynamic shared-memory limit.
 bool hq_conv_tc_init() {
   if (!load_driver_entry_points()) return false;
-  return cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, kSoloIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               214 * 1024) == cudaSuccess &&
-         cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+         cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               112 * 1024) == cudaSuccess;
 }
 
@@ -1067,14 +1225,69 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     }
   }
   p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
+  // Strip mode for 3x3 / stride 1 / pad 1: one padded input patch per cin chunk serves all nine taps (a tap is a
+  // row offset into the patch), so the activations enter shared memory once instead of nine times.  The tile is
+  // 256 positions of a raster whose pitch is the next power of two above the padded width; worth it while at
+  // least three quarters of a pitch are real columns.
+  size_t patch_total = 0;
+  {
+    int lg_wp = 0;
+    if (a.w >= 11 && a.w <= 14) lg_wp = 4; else if (a.w >= 23 && a.w <= 30) lg_wp = 5; else if (a.w >= 47 && a.w <= 62) lg_wp = 6;
+    const bool shape_ok = !pair && lg_wp && a.kh == 3 && a.kw == 3 && a.stride == 1 && a.pad == 1 && !a.pitch_w && !a.res &&
+                          p.staged_out && a.out_bits == 8 && a.cin % 64 == 0 && a.n < 65536;
+    if (shape_ok) {
+      const int bkb = a.cin % 128 == 0 ? 128 : 64;
+      const int cchunks = a.cin / bkb, rows = 256 >> lg_wp, tpi = (a.h + rows - 1) / rows;
+      const long long tiles_all = (long long)a.n * tpi * p.c_tiles;
+      const size_t patch = (size_t)(rows + 3) * (1u << lg_wp) * bkb, wb = (size_t)kTileC * bkb;
+      const size_t slab = (size_t)9 * cchunks * wb;
+      const bool keep_w = slab <= 72 * 1024;
+      const size_t room = (size_t)212 * 1024 - 32 * 1024 - (keep_w ? slab : 0);
+      int npatch = 0, wstages = 0;
+      if (keep_w) { npatch = (int)(room / patch); if (npatch > 3) npatch = 3; }
+      else if (room >= 2 * patch + 3 * wb) { npatch = 2; wstages = (int)((room - 2 * patch) / wb); }
+      // measured: with the weights streaming through the stage ring the strip form is no faster than the plain
+      // one (both are bound by what the SM can take in per cycle), so it is used where the weights stay resident
+      if (((tiles_all >= 2LL * h->sm_count && keep_w) || h->conv_path == 3) && npatch >= 2) {
+        p.strip = 1; p.lg_wp = lg_wp; p.rows = rows; p.tpi = tpi; p.ho = a.h; p.npatch = npatch;
+        p.patch_bytes = (uint32_t)patch;
+        p.bkb = bkb; p.cchunks = cchunks; p.k_blocks = 9 * cchunks;
+        p.pt = 256; p.lg_bufs = 1; p.lg_rbufs = 1; p.halves = 2;
+        p.fold = a.cout <= 64 ? 1 : 0;
+        p.wres = keep_w ? 1 : 0;
+        wres_bytes = keep_w ? (int)slab : 0;
+        stage_bytes = keep_w ? 0 : (int)wb;
+        stages = keep_w ? 0 : (wstages > kMaxStages ? kMaxStages : wstages);
+        out_tile_bytes = 4 * 256 * 32;
+        res_tile_bytes = 0;
+        p.p_tiles = a.n * tpi;
+        patch_total = (size_t)npatch * patch;
+      }
+    }
+  }
   p.x_signed = a.in_signed;
+  {
+    // issuer warps in use: at most one per K block; where the blocks travel through the stage ring, the stage count
+    // becomes a multiple of it (every stage then belongs to one issuer)
+    // Measured: several issuers pay off where the operands are mostly in shared memory already (strip form,
+    // resident weights); where every block waits for 48 KiB from L2 the tile is bound by that stream and the extra
+    // issuers only cost a few percent.
+    const int issuers = pair ? kPairIssuerWarps : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
+    p.ni = p.k_blocks < issuers ? p.k_blocks : issuers;
+    if (!(p.strip && p.wres)) {
+      while (p.ni > 1 && stages < p.ni) --p.ni;
+      if (stages > kMaxStages) stages = kMaxStages;
+      stages -= stages % p.ni;
+    }
+  }
   p.tmem_cols = (uint32_t)(p.pt << p.lg_bufs);          // 512 columns, or 256 for the smallest tile
   if (stages > kMaxStages) stages = kMaxStages;
-  if (stages < 2) return HQ_ERR_UNSUPPORTED;
+  if (stages < 2 && !p.strip) return HQ_ERR_UNSUPPORTED;
   p.stages = stages;
   p.out_stage_off = (uint32_t)(stages * stage_bytes);             // all pieces are multiples of 1024 bytes
   p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
   p.wres_off = p.res_stage_off + ((uint32_t)res_tile_bytes << p.lg_rbufs);
+  p.patch_off = p.wres_off + (uint32_t)wres_bytes;
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
@@ -1100,7 +1313,17 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const CUtensorMapSwizzle swz = swizzle_for(p.bkb);
   alignas(64) CUtensorMap map_x, map_w, map_out, map_res;
   p.x_tiled = (!a.pitch_w && a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0) ? 1 : 0;
-  if (p.x_tiled) {
+  if (p.strip) {
+    // activations (C, W, H, N), box = one patch: bkb channels x pitch columns x (rows + 3) rows of one image
+    const cuuint64_t dims[4] = {(cuuint64_t)a.cin, (cuuint64_t)a.w, (cuuint64_t)a.h, (cuuint64_t)a.n};
+    const cuuint64_t strides[3] = {(cuuint64_t)a.cin, (cuuint64_t)a.cin * a.w, (cuuint64_t)a.cin * a.w * a.h};
+    const cuuint32_t box[4] = {(cuuint32_t)p.bkb, 1u << p.lg_wp, (cuuint32_t)(p.rows + 3), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (g_encode_tiled(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.in), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
+    p.x_tiled = 0;
+  } else if (p.x_tiled) {
     if (!encode_rows_map(&map_x, a.in, P, a.cin, p.bkb, p.pt, swz)) return HQ_ERR_CUDA;
   } else {
     // activations: (C, W, H, N) with byte strides; base pixels range over
@@ -1126,12 +1349,23 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   }
   if (!encode_rows_map(&map_w, a.wgt, a.cout, (long long)a.kh * a.kw * a.cin, p.bkb, p.fold ? 64 : kTileC, swz)) return HQ_ERR_CUDA;
   map_out = map_w; map_res = map_w;                    // valid placeholders when a path is not staged
+  if (p.strip) {
+    // output (C, W, H, N), box = 32 positions of the raster: 32 channels x min(pitch, 32) columns x the rows that makes
+    const cuuint32_t bw = p.lg_wp >= 5 ? 32u : (1u << p.lg_wp);
+    const cuuint64_t dims[4] = {(cuuint64_t)a.cout, (cuuint64_t)a.wo, (cuuint64_t)a.ho, (cuuint64_t)a.n};
+    const cuuint64_t strides[3] = {(cuuint64_t)a.cout, (cuuint64_t)a.cout * a.wo, (cuuint64_t)a.cout * a.wo * a.ho};
+    const cuuint32_t box[4] = {32, bw, 32u / bw, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (g_encode_tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, a.out, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
+  } else
   if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / (p.halves << p.fold),
                                        CU_TENSOR_MAP_SWIZZLE_NONE)) return HQ_ERR_CUDA;
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_rbufs) + wres_bytes + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_rbufs) + wres_bytes + patch_total + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int slots = pair ? 2 * h->sm_count : h->sm_count;
@@ -1145,12 +1379,12 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   cfg.gridDim = dim3((unsigned)grid); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
   cudaError_t err;
   if (pair) {
-    cfg.blockDim = dim3(64 + 32 * kPairEpilogueWarps); cfg.dynamicSmemBytes = dyn_smem;
-    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kPairEpilogueWarps, 2>, map_x, map_w, map_out, map_res, p);
+    cfg.blockDim = dim3(32 * (1 + kPairIssuerWarps + kPairEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, map_x, map_w, map_out, map_res, p);
   } else {
     // one CTA per SM (it may allocate all 512 tensor-memory columns): never request less than 120 KiB
-    cfg.blockDim = dim3(64 + 32 * kSoloEpilogueWarps); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
-    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kSoloEpilogueWarps, 1>, map_x, map_w, map_out, map_res, p);
+    cfg.blockDim = dim3(32 * (1 + kSoloIssuerWarps + kSoloEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kSoloEpilogueWarps, 1, kSoloIssuerWarps>, map_x, map_w, map_out, map_res, p);
   }
   return err == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }

@@ -110,6 +110,56 @@ def test_conv_tensor_core_path(hq, cfg):
     run_conv_and_compare(hq, case, path=2)
 
 
+STRIP_CASES = [
+    # n, h, w, cin, cout: 3x3 / stride 1 / pad 1 through the strip form (one input patch per cin chunk for all nine taps)
+    (2, 14, 14, 128, 128),     # pitch 16, a whole image per tile (two scratch rows), weights through the stage ring
+    (3, 14, 14, 256, 192),     # two cin chunks, ragged channel tile
+    (2, 28, 28, 128, 128),     # pitch 32, eight rows per tile, a partly filled last tile per image
+    (1, 56, 56, 64, 64),       # pitch 64, 64-byte K blocks, resident weights, folded channel tile
+    (2, 56, 56, 64, 128),      # the same with a full channel tile
+    (2, 12, 11, 64, 96),       # narrower and lower than the pitch / the tile
+    (1, 30, 25, 128, 64),      # width 25 on pitch 32, 30 rows (last tile of six rows), folded
+    (2, 50, 62, 64, 64),       # width 62: the padded row fills the pitch of 64 exactly
+]
+
+
+@pytest.mark.parametrize("cfg", STRIP_CASES)
+@pytest.mark.parametrize("signed_in", [0, 1])
+def test_conv_tensor_core_strip_form(hq, cfg, signed_in):
+    n, h, w, cin, cout = cfg
+    kk = 9 * cin
+    lo = 36 + int(np.log2(kk)) // 2
+    case = inputs.conv_case(209, n, h, w, cin, cout, 3, 1, 1, bits=8, relu=not signed_in, in_signed=bool(signed_in),
+                            c_range=(lo, lo + 4))
+    run_conv_and_compare(hq, case, path=3)
+
+
+@pytest.mark.parametrize("cin,cout,k,hw", [(512, 128, 1, 56), (640, 128, 1, 56), (1024, 256, 1, 28), (128, 128, 3, 28),
+                                           (64, 64, 3, 56), (256, 64, 1, 56)])
+def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw):
+    """Benchmark-sized launches (several tiles per CTA: every accumulator buffer, operand stage and issuer warp is
+    reused many times, with K block counts that do and do not divide among the issuers) at an oracle cost of two
+    images: the batch repeats two distinct images, and every copy must equal the oracle's result for its image."""
+    from paper_2011_10680_b200 import binding
+    n = 64
+    lo = 36 + int(np.log2(k * k * cin)) // 2
+    case = inputs.conv_case(210, 2, hw, hw, cin, cout, k, 1, k // 2, bits=8, c_range=(lo, lo + 4))
+    ref = oracle().conv_case(case)
+    big = dict(case)
+    big["x"] = np.ascontiguousarray(np.tile(case["x"], (n // 2, 1, 1, 1)))
+    big["n"] = n
+    hq.set_conv_path(2)
+    try:
+        st, out = hq.conv_case(big)
+        assert st == binding.HQ_OK
+        hq.sync()
+    finally:
+        hq.set_conv_path(0)
+    got = out.cpu().numpy().view(ref.dtype).reshape((n // 2, 2) + ref.shape[1:])
+    for i in range(n // 2):
+        assert np.array_equal(got[i], ref), f"copy {i} differs"
+
+
 def test_conv_tensor_core_config1_exact_distribution(hq):
     run_conv_and_compare(hq, inputs.config1_case(), path=2)
 
