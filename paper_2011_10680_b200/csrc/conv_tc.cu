@@ -11,7 +11,7 @@
 // constant fetch is needed, and the 32 lanes of a warp hold 32 consecutive channels of the same
 // pixel, which is a contiguous 32-byte run of the NHWC output.
 //
-// One persistent CTA per SM, ten warps:
+// One persistent CTA per SM, twelve warps (six in the two-CTAs-per-SM shape):
 //   warp 0      TMA producer.  X tile = PT consecutive output pixels x BK bytes of one filter tap,
 //               fetched by an im2col-mode tensor map straight from the NHWC activation tensor (the
 //               hardware walks pixels across rows and images, applies the stride and zero-fills the
@@ -19,10 +19,13 @@
 //               a plain tiled map when the conv is 1x1 / stride 1.  W tile = 128 output channels x BK
 //               bytes of the [cout][kh*kw*cin] weight matrix.  When a residual is fused, its
 //               [PT][128] tile of the stored 8-bit tensor is prefetched as well.
-//   warp 1      MMA issuer (one lane).  BK/32 instructions of shape 128 x PT x 32 per stage; two
-//               (PT = 256) or four (PT <= 128) accumulator buffers in tensor memory, so the MMAs of
-//               the next tiles run while the epilogue works on the current ones.
-//   warps 2-9   epilogue.  Warp (q, half) reads lanes 32q..32q+31 (tcgen05.ld 32x32b) of one half
+//   warps 1-3   MMA issuers (one lane each; a single issuer for layers whose weights stream from L2).
+//               BK/32 instructions of shape 128 x PT x 32 per stage; two (PT = 256) or four
+//               (PT <= 128) accumulator buffers in tensor memory, so the MMAs of the next tiles run
+//               while the epilogue works on the current ones.  3x3 / stride 1 layers with resident
+//               weights use the strip form: one padded input patch per cin chunk, read by all nine
+//               taps as row offsets (see the issuer loop).
+//   warps 4-11  epilogue.  Warp (q, half) reads lanes 32q..32q+31 (tcgen05.ld 32x32b) of one half
 //               of the tile's pixel columns, applies the integer epilogue in registers and writes
 //               bytes to a private staging box that leaves through its own TMA store; no CTA-wide
 //               barrier per tile.  The loop is software-pipelined: the accumulator buffer goes back
