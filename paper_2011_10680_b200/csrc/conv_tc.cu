@@ -369,7 +369,7 @@ struct EpiCtx {
 // next one (of this tile, or the first of the group's next tile) streams from tensor memory into the
 // other register set; the accumulator buffer is handed back as soon as its last chunk has been read,
 // the residual tile as soon as its last bytes have been used, both before the tile's store is issued.
-template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN>
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN, bool OUT4 = false>
 __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const ChanConst& k_in) {
   // Private copies: the caller's objects live in local memory (their address is passed to the general
   // loop), so every asm statement with a memory clobber would force their fields to be re-read.
@@ -404,8 +404,31 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
       const int s = requant_fast<RES, RSIGNED, SMALL, RN>(v[j], r, k);
       y[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
     }
+    if (!OUT4) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)y[j];
+      for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)y[j];
+    } else {
+      // Unsigned 4-bit output (0 <= y <= 15 after the clamp): a byte holds the channel pair of two neighbouring
+      // lanes.  Each lane packs its 32 pixels into four words of eight nibbles, the pair exchanges the words
+      // (4 shuffles instead of 32), both interleave them into bytes, and the even lane stores pixels 0-3 of every
+      // eight, the odd lane pixels 4-7: rows of 16 bytes per pixel in the staging box.
+      const bool odd = lane & 1;
+      const unsigned sel = odd ? 0x7362u : 0x5140u;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        unsigned mine = (unsigned)y[8 * w + 7];
+#pragma unroll
+        for (int i = 6; i >= 0; --i) mine = mine * 16u + (unsigned)y[8 * w + i];
+        const unsigned other = __shfl_xor_sync(0xffffffffu, mine, 1);
+        const unsigned a = odd ? other : mine, b = odd ? mine : other;        // even channel, odd channel
+        const unsigned t = (a & 0x0F0F0F0Fu) | ((b << 4) & 0xF0F0F0F0u);        // pixels 0, 2, 4, 6
+        const unsigned u = ((a >> 4) & 0x0F0F0F0Fu) | (b & 0xF0F0F0F0u);        // pixels 1, 3, 5, 7
+        const unsigned four = __byte_perm(t, u, sel);                          // pixels 0-3 (even lane) or 4-7 (odd lane)
+        const int px = c * 32 + 8 * w + (odd ? 4 : 0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) my_stage_ptr[(px + i) * 16 + (lane >> 1)] = (uint8_t)(four >> (8 * i));
+      }
+    }
   };
 
   int va[32], vb[32];
@@ -460,7 +483,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     if (e.ew == 0 && lane == 0) HQ_TRACE(4, tcount);
     fence_async_smem();                           // make this lane's box writes visible to the TMA engine
     __syncwarp();
-    if (lane == 0 && e.warp_live) store_warp_box(p, e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_tile, col0, px_per_warp);
+    if (lane == 0 && e.warp_live) store_warp_box(p, e.map_out, my_stage, (e.c_tile * kTileC + cq * 32) >> (OUT4 ? 1 : 0), p_tile, col0, px_per_warp);
     if (e.ew == 0 && lane == 0) HQ_TRACE(7, tcount);
     if (!has_next || !ok) break;
     p_tile += tile_step; ++tcount; as = nas; aph = naph;
@@ -997,6 +1020,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     e.ch_live = ch_live; e.warp_live = warp_live;
     if (half >= p.halves) {
       // the 64-pixel tile has one 64-column slice per lane quarter: this warp only took part in the vote above
+    } else if (fast && p.staged_out && p.out_bits == 4 && !p.res && !p.strip && lo >= 0 && hi <= 15) {
+      // unsigned 4-bit outputs without a residual (the convs inside a 4-bit block)
+      if (warp_small) epilogue_loop_fast8<false, false, false, false, true, false, true>(e, k);
+      else epilogue_loop_fast8<false, false, false, false, false, false, true>(e, k);
     } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {

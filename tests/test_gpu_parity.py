@@ -134,19 +134,29 @@ def test_conv_tensor_core_strip_form(hq, cfg, signed_in):
     run_conv_and_compare(hq, case, path=3)
 
 
-@pytest.mark.parametrize("cin,cout,k,hw", [(512, 128, 1, 56), (640, 128, 1, 56), (1024, 256, 1, 28), (128, 128, 3, 28),
-                                           (64, 64, 3, 56), (256, 64, 1, 56)])
-def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw):
+@pytest.mark.parametrize("cin,cout,k,hw,out_bits,residual", [
+    (512, 128, 1, 56, 8, False), (640, 128, 1, 56, 8, False), (1024, 256, 1, 28, 8, False), (128, 128, 3, 28, 8, False),
+    (64, 64, 3, 56, 8, False), (256, 64, 1, 56, 8, False),
+    (64, 256, 1, 56, 8, True),       # two CTAs per SM, residual pairs worked out ahead of the single large call
+    (256, 256, 3, 28, 4, False),     # 4-bit output through the pipelined epilogue
+    (1024, 256, 1, 28, 4, False),
+])
+def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw, out_bits, residual):
     """Benchmark-sized launches (several tiles per CTA: every accumulator buffer, operand stage and issuer warp is
     reused many times, with K block counts that do and do not divide among the issuers) at an oracle cost of two
     images: the batch repeats two distinct images, and every copy must equal the oracle's result for its image."""
     from paper_2011_10680_b200 import binding
     n = 64
     lo = 36 + int(np.log2(k * k * cin)) // 2
-    case = inputs.conv_case(210, 2, hw, hw, cin, cout, k, 1, k // 2, bits=8, c_range=(lo, lo + 4))
+    if out_bits == 4:
+        lo += 4
+    case = inputs.conv_case(210, 2, hw, hw, cin, cout, k, 1, k // 2, bits=8, out_bits=out_bits, residual=residual,
+                            c_range=(lo - 6, lo + 4) if out_bits == 4 else (lo, lo + 4))
     ref = oracle().conv_case(case)
     big = dict(case)
     big["x"] = np.ascontiguousarray(np.tile(case["x"], (n // 2, 1, 1, 1)))
+    if residual:
+        big["res"] = np.ascontiguousarray(np.tile(case["res"], (n // 2, 1, 1, 1)))
     big["n"] = n
     hq.set_conv_path(2)
     try:
