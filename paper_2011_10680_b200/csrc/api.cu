@@ -132,6 +132,7 @@ struct hq_network {
   std::vector<void*> res_narrow;     // per conv layer with a fused 8-bit residual: its narrow residual pairs (owned)
   std::vector<void*> narrow0, narrow1; // per ADD / REQUANT layer with 8-bit operands: narrow pairs of the two branches (owned)
   std::vector<void*> wgt_widened;    // per 4-bit conv layer on the tensor-core path: its weights, one byte per value (owned)
+  std::vector<char> stored_wide;     // per layer: its 4-bit output is kept one value per byte (all consumers are such convs)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
@@ -313,6 +314,7 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
   net->bytes.resize(n_layers);
   net->res_narrow.assign(n_layers, nullptr);
   net->wgt_widened.assign(n_layers, nullptr);
+  net->stored_wide.assign(n_layers, 0);
   net->narrow0.assign(n_layers, nullptr);
   net->narrow1.assign(n_layers, nullptr);
   net->launches = n_layers;
@@ -382,6 +384,33 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     o.data = buf;
     net->outs[i] = o;
   }
+  // A 4-bit tensor whose only readers are tensor-core convolutions (as their main input) is kept one value per
+  // byte: its producer writes bytes clamped to the 4-bit range, the readers are plain 8-bit convolutions over
+  // their widened weights, and no widening pass runs between them.  What leaves the network (layer taps, the
+  // last layer) is packed.
+  for (int i = 0; st == HQ_OK && i + 1 < n_layers; ++i) {
+    const hq_layer& l = net->layers[i];
+    if (net->outs[i].bits != 4) continue;
+    if (l.op != HQ_OP_CONV && l.op != HQ_OP_REQUANT && l.op != HQ_OP_ADD) continue;
+    if (((long long)net->outs[i].n * net->outs[i].h * net->outs[i].w * net->outs[i].c) % 8 != 0) continue;
+    bool ok = false;
+    for (int j = i + 1; j < n_layers; ++j) {
+      const hq_layer& c = net->layers[j];
+      if (c.in1 == i) { ok = false; break; }
+      if (c.in0 != i) continue;
+      if (c.op != HQ_OP_CONV || !net->wgt_widened[j]) { ok = false; break; }
+      ok = true;
+    }
+    if (!ok) continue;
+    net->stored_wide[i] = 1;
+    cudaFree(net->outs[i].data);
+    void* buf = nullptr;
+    const size_t wide = (size_t)net->outs[i].n * net->outs[i].h * net->outs[i].w * net->outs[i].c;
+    if (cudaMalloc(&buf, wide + 256) != cudaSuccess) { cudaGetLastError(); net->outs[i].data = nullptr; st = HQ_ERR_WORKSPACE; break; }
+    net->outs[i].data = buf;
+    for (int j = i + 1; j < n_layers; ++j)
+      if (net->layers[j].in0 == i) net->launches -= 1;        // no activation-widening kernel ahead of this conv
+  }
   if (st == HQ_OK && net->scratch_bytes) {
     const size_t want = net->scratch_bytes;
     net->scratch_bytes = 0;
@@ -435,6 +464,9 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
     hq_tensor in = (l.in0 == -1) ? *images : net->outs[l.in0];
     hq_tensor o = net->outs[i];
     if (i == n_layers - 1) o.data = logits->data;
+    const bool in_wide = l.in0 >= 0 && net->stored_wide[l.in0];
+    if (in_wide) in.bits = 8;                  // one value per byte
+    if (net->stored_wide[i]) o.bits = 8;       // written as bytes clamped to the 4-bit range
     hq_status st = HQ_OK;
     switch (l.op) {
       case HQ_OP_CONV: case HQ_OP_LINEAR: {
@@ -442,8 +474,9 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         hq_tensor res{};
         d.residual = nullptr;
         if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
+        if (in_wide) { d.w_bits = 8; d.w = net->wgt_widened[i]; }
         if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
-        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i], net->wgt_widened[i]);
+        else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i], in_wide ? nullptr : net->wgt_widened[i]);
         break;
       }
       case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
@@ -463,8 +496,11 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
     }
     if (st != HQ_OK) return st;
     if (taps && taps[i]) {
-      if (cudaMemcpyAsync(taps[i], o.data, (size_t)net->bytes[i], cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+      if (net->stored_wide[i]) {
+        if (hq_launch_pack4(o.data, (long long)o.n * o.h * o.w * o.c, taps[i], h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+      } else if (cudaMemcpyAsync(taps[i], o.data, (size_t)net->bytes[i], cudaMemcpyDeviceToDevice, s) != cudaSuccess) {
         return HQ_ERR_CUDA;
+      }
     }
   }
   if (marks && cudaEventRecord(marks[n_layers], s) != cudaSuccess) return HQ_ERR_CUDA;

@@ -272,6 +272,17 @@ __global__ void __launch_bounds__(256) widen4_kernel(const uint2* __restrict__ i
   for (; i < n_vec; i += stride) out[i] = widen4_vec<SIGNED>(__ldg(in + i));
 }
 
+// One byte per value -> two values per byte (low nibble first); 8 bytes in, 4 bytes out per thread and step.
+__global__ void __launch_bounds__(256) pack4_kernel(const uint2* __restrict__ in, long long n_vec, unsigned* __restrict__ out) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
+    const uint2 v = __ldg(in + i);
+    const unsigned lo = (v.x & 0x0F0F0F0Fu) | ((v.x >> 4) & 0x00F000F0u);      // bytes 0 and 2 hold the packed pairs
+    const unsigned hi = (v.y & 0x0F0F0F0Fu) | ((v.y >> 4) & 0x00F000F0u);
+    out[i] = __byte_perm(lo, hi, 0x6420);
+  }
+}
+
 cudaError_t launch_widen4(const void* in, long long elems, int is_signed, void* out, int sm_count, cudaStream_t s) {
   const long long n_vec = elems / 16;                  // callers guarantee a multiple of 16 elements
   if (n_vec == 0) return cudaSuccess;
@@ -307,6 +318,14 @@ hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, 
   ConvArgs t = a;
   t.in = xw; t.wgt = a.wgt_widened ? a.wgt_widened : ww; t.in_bits = 8;
   return hq_launch_conv_tc(h, t, s);
+}
+
+cudaError_t hq_launch_pack4(const void* in, long long values, void* out, int sm_count, cudaStream_t s) {
+  const long long n_vec = values / 8;                  // callers guarantee a multiple of 8 values
+  if (n_vec == 0) return cudaSuccess;
+  const long long blocks = (n_vec + 255) / 256, cap = (long long)sm_count * 16;
+  pack4_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const uint2*)in, n_vec, (unsigned*)out);
+  return cudaGetLastError();
 }
 
 cudaError_t hq_launch_widen_weights(const void* wgt, long long values, void* out, int sm_count, cudaStream_t s) {
