@@ -495,7 +495,10 @@ def main():
         work = layer_work(table, batch)
         rows, tc_bytes, tc_ops, tc_ns = [], 0, 0, 0.0
         for wk, ns, l in zip(work, layer_ns, table["layers"]):
-            on_tc = l["op"] in ("conv", "linear") and l["bits"] == 8 and l["cin"] % 32 == 0
+            # layers that run conv_tc_kernel: every conv / linear with a channel count the tensor maps take (4-bit
+            # operands included: widened, or kept one value per byte inside the network) and the 3-channel stem
+            # (space-to-depth form; its two helper kernels are part of the layer's time)
+            on_tc = l["op"] in ("conv", "linear") and (l["cin"] % 32 == 0 or (l["cin"] == 3 and l["kh"] == 7 and l["stride"] == 2))
             if on_tc:
                 tc_bytes += wk["bytes"]; tc_ops += wk["ops"]; tc_ns += ns
             rows.append({**wk, "us": ns / 1e3, "tensor_core": on_tc, "gbs": wk["bytes"] / max(ns, 1),
