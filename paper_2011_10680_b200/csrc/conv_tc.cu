@@ -47,11 +47,13 @@ namespace {
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccBufs = 4;                                 // accumulator (and residual) buffers: 4 x 128 or 2 x 256 columns
-// Two launch shapes of the same kernel:
+// Three launch shapes of the same kernel:
 //   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 212 KiB of shared memory;
 //   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
 //         reduction are bound by the latency of the hand-over chain between the MMA issuer and the epilogue
 //         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
+//   wide  16 epilogue warps and one issuer, one CTA per SM: fused-residual layers on 256-pixel tiles (the longest
+//         epilogue chain per value gains from four warps per scheduler; the loop keeps one chunk in registers).
 constexpr int kSoloEpilogueWarps = 8;
 constexpr int kPairEpilogueWarps = 4;
 constexpr int kSoloIssuerWarps = 3;     // 1 + 3 + 8 warps = 384 threads: 168 registers per thread remain
@@ -489,6 +491,62 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     p_tile += tile_step; ++tcount; as = nas; aph = naph;
   }
   if (pending) tmem_ld_wait();
+  if (lane == 0) tma_store_wait_all();
+}
+
+// The same arithmetic for the launch shape with sixteen epilogue warps (four per scheduler): no second register
+// set for the next chunk -- with four warps per scheduler the tensor-memory load of one warp hides behind the
+// arithmetic of the others -- which keeps the loop inside that shape's register budget.
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN>
+__device__ __forceinline__ void epilogue_loop_lean8(const EpiCtx& e_in, const ChanConst& k_in) {
+  const EpiCtx e = e_in;
+  const ChanConst k = k_in;
+  const TcParams& p = *e.p;
+  SharedCtl& ctl = *e.ctl;
+  const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
+  const uint32_t my_stage = e.out_stage + (uint32_t)e.ew * (uint32_t)(px_per_warp * 32);
+  uint8_t* const my_stage_ptr = e.smem_raw + (my_stage - e.raw);
+  const uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
+  const int nchunks = px_per_warp >> 5;
+  const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
+  const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + col0;
+  auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
+    uint32_t w = 1;
+    if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, w, 0) != 0;
+  };
+  uint32_t tcount = 0;
+  for (int p_tile = e.p_tile0; p_tile < p.p_tiles; p_tile += e.p_step, ++tcount) {
+    const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
+    const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
+    if (!wait_bar(&ctl.tfull[as], aph)) break;
+    if (RES && !wait_bar(&ctl.rfull[rs], rph)) break;
+    tc_fence_after();
+    if (lane == 0) tma_store_wait_read0();        // the previous tile's store has read the staging box
+    __syncwarp();
+    const uint8_t* const res_tile = res_stage_ptr + rs * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
+    for (int c = 0; c < nchunks; ++c) {
+      int v[32];
+      tmem_ld32(t_warp + as * p.pt + c * 32, v);
+      if (!e.warp_live) continue;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const int r = !RES ? 0 : RSIGNED ? (int)(signed char)res_tile[(c * 32 + j) * kTileC] : (int)res_tile[(c * 32 + j) * kTileC];
+        const int s = requant_fast<RES, RSIGNED, SMALL, RN>(v[j], r, k);
+        v[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)v[j];
+    }
+    tc_fence_before();
+    fence_async_smem();                           // make this lane's box writes visible to the TMA engine
+    __syncwarp();
+    if (lane == 0) {
+      mbar_arrive(smem_u32(&ctl.tempty[as]));
+      if (RES) mbar_arrive(smem_u32(&ctl.rempty[rs]));
+      if (e.warp_live) store_warp_box(p, e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_tile, col0, px_per_warp);
+    }
+  }
   if (lane == 0) tma_store_wait_all();
 }
 
@@ -1027,7 +1085,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
-#define HQ_FAST8(R, RS, S, OS) do { if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true, false>(e, k); \
+#define HQ_FAST8(R, RS, S, OS) do { if (EPI_WARPS == 16) { \
+                                      if (warp_small) epilogue_loop_lean8<R, RS, S, OS, true, false>(e, k); \
+                                      else if (R && warp_narrow) epilogue_loop_lean8<R, RS, S, OS, false, R>(e, k); \
+                                      else epilogue_loop_lean8<R, RS, S, OS, false, false>(e, k); \
+                                    } else if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true, false>(e, k); \
                                     else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, false, R>(e, k); \
                                     else epilogue_loop_fast8<R, RS, S, OS, false, false>(e, k); } while (0)
         case 0: HQ_FAST8(false, false, false, false); break;
@@ -1166,7 +1228,8 @@ bool hq_conv_tc_init() {
   return cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, kSoloIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               214 * 1024) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              112 * 1024) == cudaSuccess;
+                              112 * 1024) == cudaSuccess &&
+         cudaFuncSetAttribute(conv_tc_kernel<16, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess;
 }
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
@@ -1296,13 +1359,19 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     }
   }
   p.x_signed = a.in_signed;
+  bool wide = false;
   {
     // issuer warps in use: at most one per K block; where the blocks travel through the stage ring, the stage count
     // becomes a multiple of it (every stage then belongs to one issuer)
     // Measured: several issuers pay off where the operands are mostly in shared memory already (strip form,
     // resident weights); where every block waits for 48 KiB from L2 the tile is bound by that stream and the extra
     // issuers only cost a few percent.
-    const int issuers = pair ? kPairIssuerWarps : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
+    // Third launch shape, *wide*: sixteen epilogue warps (four per scheduler, 64 pixel columns each) with a loop that
+    // keeps one chunk in registers.  Measured per layer: it wins where the epilogue carries the residual add on
+    // 256-pixel tiles (1x1 128 -> 512 at 28x28: 81 -> 72 us) and loses a few percent everywhere else.
+    wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res;
+    if (wide) p.halves = 4;
+    const int issuers = pair ? kPairIssuerWarps : wide ? 1 : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
     p.ni = p.k_blocks < issuers ? p.k_blocks : issuers;
     if (!(p.strip && p.wres)) {
       while (p.ni > 1 && stages < p.ni) --p.ni;
@@ -1408,7 +1477,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
   cudaError_t err;
-  if (pair) {
+  if (wide) {
+    cfg.blockDim = dim3(32 * 18); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<16, 1, 1>, map_x, map_w, map_out, map_res, p);
+  } else if (pair) {
     cfg.blockDim = dim3(32 * (1 + kPairIssuerWarps + kPairEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem;
     err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, map_x, map_w, map_out, map_res, p);
   } else {
