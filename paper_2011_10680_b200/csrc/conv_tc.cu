@@ -1265,8 +1265,10 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const long long k_total = (long long)a.kh * a.kw * a.cin;
   // (measured: with the weight slab resident the one-CTA shape catches up for K >= 128; the pair shape still
   // wins on the fused-residual expansions with the shortest reduction, and loses where a tile carries little
-  // epilogue work, e.g. 64 output channels)
-  bool pair = k_total <= 64 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128;
+  // epilogue work, e.g. 64 output channels.  Where the layer is large enough for 256-pixel tiles and its residual
+  // travels by TMA, the wide shape below is faster still: 64 -> 256 at 56x56, batch 256: 129 -> 121 us.)
+  const bool wide_fits = p.staged_res && a.out_bits == 8 && a.cout > 64 && pick_pt(P, p.c_tiles, h->sm_count, 256) == 256;
+  bool pair = k_total <= 64 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128 && !wide_fits;
   int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0, wres_bytes = 0;
   if (pair) {
     // 128-pixel tiles, two accumulator buffers (256 columns), K blocks of at most 64 bytes
@@ -1368,8 +1370,9 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // issuers only cost a few percent.
     // Third launch shape, *wide*: sixteen epilogue warps (four per scheduler, 64 pixel columns each) with a loop that
     // keeps one chunk in registers.  Measured per layer: it wins where the epilogue carries the residual add on
-    // 256-pixel tiles (1x1 128 -> 512 at 28x28: 81 -> 72 us) and loses a few percent everywhere else.
-    wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res;
+    // 256-pixel tiles with a short reduction (1x1 128 -> 512 at 28x28: 81 -> 72 us) and loses a few percent
+    // everywhere else (long reductions are bound by the operand stream, not by the epilogue).
+    wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
     if (wide) p.halves = 4;
     const int issuers = pair ? kPairIssuerWarps : wide ? 1 : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
     p.ni = p.k_blocks < issuers ? p.k_blocks : issuers;
