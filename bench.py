@@ -39,7 +39,7 @@ NOMINAL_I8_TOPS = 4500.0
 # dram__bytes_read.sum + dram__bytes_write.sum of all conv_tc_kernel launches of one pass, captured with ncu at
 # batch 64 (profiles/resnet50_int8_b256_launch_list.md) and scaled per image; writes are under-counted there
 # (outputs stay dirty in L2), so this is a lower bound of the batch-256 traffic.
-NCU_CONV_DRAM_BYTES_PER_IMAGE = (902.5e6 + 53.1e6) / 64
+NCU_CONV_DRAM_BYTES_PER_IMAGE = (903.0e6 + 78.2e6) / 64
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
