@@ -204,6 +204,12 @@ hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* desc, hq_te
  * then reach the shapes of large layers). */
 hq_status hq_set_conv_path(hq_handle* h, int32_t path);
 
+/* Self-test of the bounded device-side waits: one thread waits on a barrier that nothing ever signals, for at
+ * most `budget_ms` milliseconds (1..2000), then records the expiry in the handle's status word and returns, as
+ * every wait inside the kernels does after its own budget.  The next hq_sync reports HQ_ERR_TIMEOUT; the
+ * context stays usable.  Asynchronous on `stream`. */
+hq_status hq_expire_wait_selftest(hq_handle* h, int32_t budget_ms, void* stream);
+
 const char* hq_status_string(hq_status s);
 
 #ifdef __cplusplus

@@ -21,7 +21,7 @@ HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant"
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
-    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc",
+    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
 ]
 
 
@@ -82,6 +82,8 @@ def lib():
         L.hq_network_launch_count.argtypes = [vp, C.POINTER(i32)]
         L.hq_network_destroy.argtypes = [vp]
         L.hq_set_conv_path.argtypes = [vp, i32]
+        L.hq_expire_wait_selftest.argtypes = [vp, i32, vp]
+        L.hq_expire_wait_selftest.restype = i32
         L.hq_status_string.argtypes = [i32]
         L.hq_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -152,6 +154,9 @@ class Handle:
 
     def set_conv_path(self, path: int):
         _check(lib().hq_set_conv_path(self._h, path), "hq_set_conv_path")
+
+    def expire_wait_selftest(self, budget_ms: int) -> int:
+        return lib().hq_expire_wait_selftest(self._h, budget_ms, _stream())
 
     def sync(self):
         _check(lib().hq_sync(self._h, _stream()), "hq_sync")

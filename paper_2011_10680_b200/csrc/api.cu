@@ -199,6 +199,11 @@ hq_status hq_set_conv_path(hq_handle* h, int32_t path) {
   return HQ_OK;
 }
 
+hq_status hq_expire_wait_selftest(hq_handle* h, int32_t budget_ms, void* stream) {
+  if (!h || budget_ms < 1 || budget_ms > 2000) return HQ_ERR_INVALID_ARG;
+  return hq_launch_expire_wait(h->dev_status, budget_ms, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
 hq_status hq_sync(hq_handle* h, void* stream) {
   if (!h) return HQ_ERR_INVALID_ARG;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HQ_ERR_CUDA;

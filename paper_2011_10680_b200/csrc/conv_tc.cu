@@ -1509,6 +1509,24 @@ cudaError_t hq_launch_residual_narrow2(const int32_t* b0, const int32_t* c0, int
   return cudaGetLastError();
 }
 
+namespace {
+// The wait of the kernels above in miniature: poll an mbarrier, give up after the budget, say so in the status word.
+__global__ void expire_wait_kernel(uint32_t* status, unsigned long long budget_ns) {
+  __shared__ unsigned long long bar;
+  mbar_init(smem_u32(&bar), 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait(smem_u32(&bar), 0)) {
+    if (global_ns() - t0 > budget_ns) { atomicCAS(status, 0u, (uint32_t)HQ_DEV_TIMEOUT_EPILOGUE); break; }
+  }
+}
+}  // namespace
+
+cudaError_t hq_launch_expire_wait(uint32_t* status, int budget_ms, cudaStream_t s) {
+  expire_wait_kernel<<<1, 1, 0, s>>>(status, (unsigned long long)budget_ms * 1000000ull);
+  return cudaGetLastError();
+}
+
 #ifdef HQ_TC_TRACE
 extern "C" int hq_debug_trace_read(long long* host) {
   if (!g_trace_buf) return 1;

@@ -106,6 +106,7 @@ hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, 
 // Widen packed 4-bit weights (cout*kh*kw*cin values, a multiple of 16) to bytes, once, for ConvArgs::wgt_widened.
 cudaError_t hq_launch_widen_weights(const void* wgt, long long values, void* out, int sm_count, cudaStream_t s);
 // Bytes holding 4-bit values (one per byte) -> packed 4-bit tensor; `values` a multiple of 8.
+cudaError_t hq_launch_expire_wait(uint32_t* status, int budget_ms, cudaStream_t s);
 cudaError_t hq_launch_pack4(const void* in, long long values, void* out, int sm_count, cudaStream_t s);
 // Grow the handle's scratch buffer (not allowed while `s` is capturing).
 hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s);

@@ -495,6 +495,23 @@ def test_avgpool_requant_8bit_kernels(hq, n, hw, ch, signed):
     assert np.array_equal(host(out, ref), ref)
 
 
+def test_bounded_wait_expires_and_context_stays_usable(hq):
+    """A device-side wait that nothing ever satisfies gives up after its budget, hq_sync reports it once, and the
+    same handle then runs a convolution bit-exactly (no trap, no hang, no lost context)."""
+    from paper_2011_10680_b200 import binding
+    import time
+    assert hq.expire_wait_selftest(0) == binding.HQ_ERR_INVALID_ARG
+    t0 = time.time()
+    assert hq.expire_wait_selftest(300) == binding.HQ_OK
+    with pytest.raises(binding.HqError) as err:
+        hq.sync()
+    assert err.value.code == binding.HQ_ERR_TIMEOUT
+    assert 0.25 < time.time() - t0 < 5.0
+    hq.sync()                                     # the status word was cleared by the report
+    case = inputs.conv_case(211, 2, 12, 12, 64, 64, 3, 1, 1)
+    run_conv_and_compare(hq, case, path=2)
+
+
 # ------------------------------------------------------------------ argument errors ------------
 def test_invalid_arguments_return_codes_not_crashes(hq):
     from paper_2011_10680_b200 import binding
