@@ -495,6 +495,30 @@ def test_avgpool_requant_8bit_kernels(hq, n, hw, ch, signed):
     assert np.array_equal(host(out, ref), ref)
 
 
+@pytest.mark.parametrize("path", [1, 2])
+def test_conv_degenerate_and_extreme_cases(hq, path):
+    """Extreme operands and degenerate geometry on both conv paths: every activation and weight at the end of its
+    range with the longest ResNet reduction (largest accumulators the workloads can produce, both signs, clamped at
+    both ends), all-zero operands (bias only), a filter as large as its input (one output pixel), a single pixel."""
+    def extreme(sign, relu):
+        case = inputs.conv_case(212, 1, 7, 7, 512, 64, 3, 1, 1, relu=relu, c_range=(44, 48))
+        case["x"][:] = 255
+        case["wgt"][:] = 127 * sign
+        case["bias"][:] = (1 << 15) * sign
+        return case
+    run_conv_and_compare(hq, extreme(+1, True), path)          # acc = 9 * 512 * 255 * 127 at the centre: saturates high
+    run_conv_and_compare(hq, extreme(-1, True), path)          # most negative accumulators: ReLU clamps to 0
+    neg = extreme(-1, False)
+    neg["qmin"], neg["qmax"], neg["out_signed"] = -128, 127, 1
+    run_conv_and_compare(hq, neg, path)                        # ... and to -128 without ReLU
+    zero = inputs.conv_case(213, 2, 9, 9, 64, 96, 3, 1, 1, c_range=(20, 24))
+    zero["x"][:] = 0
+    run_conv_and_compare(hq, zero, path)                       # bias * b >> c only; shifts below 32
+    run_conv_and_compare(hq, inputs.conv_case(214, 3, 7, 7, 64, 64, 7, 1, 0), path)    # one output pixel per image
+    run_conv_and_compare(hq, inputs.conv_case(215, 1, 1, 1, 64, 32, 1, 1, 0), path)    # a single pixel
+    run_conv_and_compare(hq, inputs.conv_case(216, 1, 1, 1, 32, 8, 3, 1, 1), path)     # all taps but the centre are padding
+
+
 def test_bounded_wait_expires_and_context_stays_usable(hq):
     """A device-side wait that nothing ever satisfies gives up after its budget, hq_sync reports it once, and the
     same handle then runs a convolution bit-exactly (no trap, no hang, no lost context)."""
