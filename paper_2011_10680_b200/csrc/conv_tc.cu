@@ -73,6 +73,7 @@ struct TcParams {
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
+  int32_t duo;           // 1: two CTAs of a cluster (adjacent SMs) share every MMA: 256 channels x 256 pixels per pair
   int32_t ni;            // MMA issuer warps in use: min(issuer warps of the launch shape, k_blocks)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
   int32_t x_signed;      // activations signed?
@@ -242,6 +243,50 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- two-CTA forms (cta_group::2).  `in_cta(addr, r)` names the same shared-memory offset in the cluster's CTA r.
+__device__ __forceinline__ uint32_t in_cta(uint32_t addr, uint32_t cta_rank) {
+  uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta_rank)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_i8_2cta(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// arrives on ONE barrier (of either CTA of the pair) when the pair's MMAs issued so far have completed
+__device__ __forceinline__ void mma_commit_2cta(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// loads of a CTA pair: the bytes land in the issuing CTA's shared memory and are counted on the leading CTA's barrier
+__device__ __forceinline__ void tma_load_2d_2cta(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(in_cta(bar, 0)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_2cta(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                     int c, int w, int h, int n, uint16_t off_w, uint16_t off_h) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+      ::"r"(dst), "l"(map), "r"(in_cta(bar, 0)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -357,6 +402,13 @@ __device__ __forceinline__ void store_warp_box(const TcParams& p, const CUtensor
   if (any) tma_store_commit();
 }
 
+// An epilogue warp hands its part of accumulator buffer `as` back.  The barrier that counts is the one the MMA issuer
+// waits on: this CTA's, or the leading CTA's when two CTAs share the MMAs.
+__device__ __forceinline__ void release_accumulator(const TcParams& p, SharedCtl& ctl, uint32_t as) {
+  const uint32_t bar = smem_u32(&ctl.tempty[as]);
+  if (p.duo) mbar_arrive_cluster(in_cta(bar, 0)); else mbar_arrive(bar);
+}
+
 // Everything an epilogue warp needs, gathered once so the tile loops can live in their own functions.
 struct EpiCtx {
   const TcParams* p; SharedCtl* ctl; const CUtensorMap* map_out;
@@ -467,7 +519,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
         // every lane has read its last accumulator columns of this tile: hand the buffer back
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[as]));
+        if (lane == 0) release_accumulator(p, ctl, as);
         if (lane == 0) HQ_TRACE(6, tcount * 8 + e.ew);
       }
       chunk(vb, res_tile, c + 1);
@@ -542,7 +594,7 @@ __device__ __forceinline__ void epilogue_loop_lean8(const EpiCtx& e_in, const Ch
     fence_async_smem();                           // make this lane's box writes visible to the TMA engine
     __syncwarp();
     if (lane == 0) {
-      mbar_arrive(smem_u32(&ctl.tempty[as]));
+      release_accumulator(p, ctl, as);
       if (RES) mbar_arrive(smem_u32(&ctl.rempty[rs]));
       if (e.warp_live) store_warp_box(p, e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_tile, col0, px_per_warp);
     }
@@ -692,7 +744,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       if (p.staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(smem_u32(&ctl.tempty[as]));
+        release_accumulator(p, ctl, as);
         if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
         if (p.staged_out && warp_live)
           store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_tile, col0, px_per_warp);
@@ -703,7 +755,9 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 }
 
 // ---------------------------------------------------------------- the kernel -----------------
-template <int EPI_WARPS, int MIN_CTAS, int MMA_WARPS>
+// DUO: the instantiation that may be launched as clusters of two CTAs sharing their MMAs; only it contains the
+// cta_group::2 instructions (a kernel that contains them cannot be launched without clusters).
+template <int EPI_WARPS, int MIN_CTAS, int MMA_WARPS, bool DUO = false>
 __global__ void __launch_bounds__(32 * (1 + MMA_WARPS + EPI_WARPS), MIN_CTAS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
@@ -714,7 +768,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // operand stages, 1024-byte aligned
   const uint32_t w_bytes = kTileC * p.bkb;
-  const uint32_t x_bytes = p.strip ? 0u : (uint32_t)(p.pt * p.bkb);   // strip mode: the stages carry weights only
+  // strip mode: the stages carry weights only; duo: each CTA of the pair holds half of the pixel rows
+  const uint32_t x_bytes = p.strip ? 0u : (uint32_t)((p.pt >> p.duo) * p.bkb);
+  uint32_t rank = 0u;                                      // 0 = the CTA that issues the pair's MMAs
+  if constexpr (DUO) rank = cluster_ctarank();
   const uint32_t x_off = p.wres ? 0u : w_bytes;          // offset of the X tile inside a stage
   const uint32_t stage_bytes = x_off + x_bytes;
   const uint32_t out_stage = tiles + p.out_stage_off;
@@ -730,7 +787,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&ctl.full[s]), 1); mbar_init(smem_u32(&ctl.empty[s]), 1); }
     for (int s = 0; s < (1 << p.lg_bufs); ++s) {
-      mbar_init(smem_u32(&ctl.tfull[s]), p.ni); mbar_init(smem_u32(&ctl.tempty[s]), 4 * p.halves);
+      mbar_init(smem_u32(&ctl.tfull[s]), p.ni); mbar_init(smem_u32(&ctl.tempty[s]), (4 * p.halves) << p.duo);
       mbar_init(smem_u32(&ctl.tstart[s]), 1);
       mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), 4 * p.halves);
     }
@@ -740,9 +797,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     ctl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(smem_u32(&ctl.tmem_base), p.tmem_cols);
+  if (warp == 1) { if constexpr (DUO) tmem_alloc2(smem_u32(&ctl.tmem_base), p.tmem_cols); else tmem_alloc(smem_u32(&ctl.tmem_base), p.tmem_cols); }
   tc_fence_before();
   __syncthreads();
+  if constexpr (DUO) cluster_sync_all();   // both CTAs' barriers exist before either touches the other's
   tc_fence_after();
   const uint32_t tmem_base = ctl.tmem_base;
   // Programmatic dependent launch: this grid may have started while the previous kernel of the stream was
@@ -767,9 +825,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       bool ok = true;
       // (image, row, column) of the tile's first output pixel, advanced by a fixed step per tile
       const int ho = p.howo / p.wo;
-      int img = (p_tile0 * p.pt) / p.howo;
-      int oh = ((p_tile0 * p.pt) - img * p.howo) / p.wo;
-      int ow = (p_tile0 * p.pt) - img * p.howo - oh * p.wo;
+      // (duo: this CTA fetches the half of the tile's pixel rows that starts at half_off)
+      const int half_off = p.duo ? (int)rank * (p.pt >> 1) : 0;
+      int img = (p_tile0 * p.pt + half_off) / p.howo;
+      int oh = ((p_tile0 * p.pt + half_off) - img * p.howo) / p.wo;
+      int ow = (p_tile0 * p.pt + half_off) - img * p.howo - oh * p.wo;
       const int step = p_step * p.pt;
       const int d_img = step / p.howo, d_oh = (step - d_img * p.howo) / p.wo, d_ow = step - d_img * p.howo - d_oh * p.wo;
       if (p.wres) {              // the channel tile's weights for every K block, once
@@ -837,6 +897,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           HQ_TRACE(0, it);
           const uint32_t bar = smem_u32(&ctl.full[s]);
           const uint32_t w_dst = tiles + s * stage_bytes;
+          if constexpr (DUO) {
+            // Both CTAs of the pair fetch their own weight rows and their half of the pixel rows into their own
+            // stage; all four copies are counted on the leading CTA's barrier, which alone expects the bytes.
+            if (rank == 0) mbar_expect_tx(bar, 2u * stage_bytes);
+            if (p.x_tiled) tma_load_2d_2cta(w_dst + x_off, &map_x, bar, chunk * p.bkb, p0 + half_off);
+            else tma_load_im2col_2cta(w_dst + x_off, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
+            tma_load_2d_2cta(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
+            if (++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
+            if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+            continue;
+          }
           mbar_expect_tx(bar, stage_bytes);
           if (p.x_tiled) {
             tma_load_2d(w_dst + x_off, &map_x, bar, chunk * p.bkb, p0);
@@ -856,7 +927,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
       // Drain: every copy this thread started must have landed before the CTA may exit.
-      const uint32_t issued = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
+      // (the odd CTA of a pair sees no completion of its own copies: they are counted on the leading CTA's barriers,
+      // whose MMAs consume them before the pair's closing cluster barrier)
+      const uint32_t issued = (p.duo && rank != 0) ? 0u : (it < (uint32_t)p.stages ? it : (uint32_t)p.stages);
       for (uint32_t j = 0; j < (p.npatch > 0 ? (pit < (uint32_t)p.npatch ? pit : (uint32_t)p.npatch) : 0u); ++j) {
         const uint32_t k = pit - 1 - j;
         const unsigned long long t0 = global_ns();
@@ -901,10 +974,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // does not care about the order of the blocks; only the tile's first MMA, which overwrites the accumulator,
     // must come first: whoever issues it signals `tstart` and the others wait for that.
     const int iss = warp - 1;
-    if (iss < p.ni && elect_one()) {
-      // instruction descriptor: D = S32, A = s8 weights, B = u8/s8 activations, both K-major, M = 128, N = pt
+    if (iss < p.ni && rank == 0 && elect_one()) {
+      // instruction descriptor: D = S32, A = s8 weights, B = u8/s8 activations, both K-major, N = pt,
+      // M = 128 (256 over the two CTAs of a pair)
       const uint32_t idesc = (2u << 4) | (1u << 7) | ((uint32_t)(p.x_signed ? 1 : 0) << 10) |
-                             ((uint32_t)(p.pt >> 3) << 17) | ((uint32_t)(kTileC >> 4) << 24);
+                             ((uint32_t)(p.pt >> 3) << 17) | ((uint32_t)((kTileC << p.duo) >> 4) << 24);
+      // completion of the MMAs issued so far, signalled on a barrier of this CTA -- and of its partner in a pair
+      auto commit = [&](uint32_t bar) {
+        if constexpr (DUO) { mma_commit_2cta(in_cta(bar, 0)); mma_commit_2cta(in_cta(bar, 1)); }
+        else mma_commit(bar);
+      };
       const uint32_t ni = (uint32_t)p.ni, nstages = (uint32_t)p.stages;
       const bool ring = !(p.strip && p.wres);                 // do the blocks travel through the stage ring?
       uint32_t tcount = 0, s = 0, ph = 0;
@@ -935,12 +1014,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const uint32_t a_addr = p.wres ? tiles + p.wres_off + (uint32_t)kb * w_bytes : w_addr;
           uint64_t adesc = desc_hi | (uint64_t)((a_addr >> 4) & 0x3FFF);
           uint64_t bdesc = desc_hi | (uint64_t)(((w_addr + x_off) >> 4) & 0x3FFF);
-          for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
-            mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+          if constexpr (DUO) {
+            for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)
+              mma_i8_2cta(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+          } else {
+            for (int k = 0; k < ksteps; ++k, adesc += 2, bdesc += 2)     // 32 bytes of K per instruction
+              mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+          }
           HQ_TRACE(5, tcount * (uint32_t)p.k_blocks + (uint32_t)kb);
           // the accumulator's barrier first on the last K block: the epilogue is the one waiting
-          if (kb + 1 == p.k_blocks) mma_commit(smem_u32(&ctl.tfull[as]));
-          mma_commit(smem_u32(&ctl.empty[s]));     // frees the stage when these MMAs have read it
+          if (kb + 1 == p.k_blocks) commit(smem_u32(&ctl.tfull[as]));
+          commit(smem_u32(&ctl.empty[s]));         // frees the stage when these MMAs have read it
           if (++s == nstages) { s = 0; ph ^= 1u; }
         }
         HQ_TRACE(2, tcount);
@@ -1009,7 +1093,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (iss == 0) HQ_TRACE(2, tcount);
       }
       // Drain: all issued MMAs must have completed before tensor memory is freed.
-      mma_commit(smem_u32(&ctl.drain));
+      if constexpr (DUO) mma_commit_2cta(in_cta(smem_u32(&ctl.drain), 0)); else mma_commit(smem_u32(&ctl.drain));
       const unsigned long long t0 = global_ns();
       while (!mbar_try_wait(smem_u32(&ctl.drain), 0)) {
         if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
@@ -1108,10 +1192,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
+  // A pair leaves together: the leading CTA has seen its MMAs complete (they read the partner's shared memory and
+  // signal its barriers), the partner has sent its last remote arrival.
+  if constexpr (DUO) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, p.tmem_cols);
+    if constexpr (DUO) tmem_dealloc2(tmem_base, p.tmem_cols); else tmem_dealloc(tmem_base, p.tmem_cols);
   }
 }
 
@@ -1229,7 +1316,9 @@ bool hq_conv_tc_init() {
                               214 * 1024) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               112 * 1024) == cudaSuccess &&
-         cudaFuncSetAttribute(conv_tc_kernel<16, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess;
+         cudaFuncSetAttribute(conv_tc_kernel<16, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess &&
+         cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              214 * 1024) == cudaSuccess;
 }
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
@@ -1374,6 +1463,15 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // everywhere else (long reductions are bound by the operand stream, not by the epilogue).
     wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
     if (wide) p.halves = 4;
+    // Fourth shape, *duo*: clusters of two CTAs on adjacent SMs share every MMA (cta_group::2, M = 256): each CTA
+    // fetches its own 128 weight rows and HALF of the tile's pixel rows, 32 KiB per K block and SM instead of
+    // 48 KiB for the same MMA time.  For the long reductions whose weights stream, which the operand fetch bounds.
+    p.duo = (!pair && !wide && !p.strip && !p.wres && !p.fold && p.pt >= 128 && p.bkb == 128 && a.cout % 256 == 0 &&
+             k_total >= 2048 && (long long)p.p_tiles * p.c_tiles >= 2LL * h->sm_count) ? 1 : 0;
+    if (p.duo) {
+      stage_bytes = (kTileC + p.pt / 2) * p.bkb;
+      stages = (212 * 1024 - out_tile_bytes - (res_tile_bytes << p.lg_rbufs)) / stage_bytes;
+    }
     const int issuers = pair ? kPairIssuerWarps : wide ? 1 : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
     p.ni = p.k_blocks < issuers ? p.k_blocks : issuers;
     if (!(p.strip && p.wres)) {
@@ -1426,7 +1524,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
     p.x_tiled = 0;
   } else if (p.x_tiled) {
-    if (!encode_rows_map(&map_x, a.in, P, a.cin, p.bkb, p.pt, swz)) return HQ_ERR_CUDA;
+    if (!encode_rows_map(&map_x, a.in, P, a.cin, p.bkb, p.pt >> p.duo, swz)) return HQ_ERR_CUDA;
   } else {
     // activations: (C, W, H, N) with byte strides; base pixels range over
     // [-pad, W + pad - (kw-1)) so that the hardware's pixel walk equals the output raster
@@ -1439,7 +1537,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     const int upper[2] = {pad_after - (a.kw - 1), pad_after - (a.kh - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)a.stride, (cuuint32_t)a.stride, 1};
     const CUresult r = g_encode_im2col(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.in), dims, strides,
-                                       lower, upper, (cuuint32_t)p.bkb, (cuuint32_t)p.pt, estr,
+                                       lower, upper, (cuuint32_t)p.bkb, (cuuint32_t)(p.pt >> p.duo), estr,
                                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1474,13 +1572,18 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   const int grid = (int)(total_tiles <= slots ? total_tiles : (slots / p.c_tiles) * p.c_tiles);
   // Launched with programmatic stream serialization: the grid may begin (barrier set-up, tensor-memory
   // allocation) while the previous kernel drains; the kernel waits for it before reading any input.
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;          // duo: consecutive CTAs (channel tiles 2j, 2j+1) pair up
+  attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)grid); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)grid); cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = p.duo ? 2 : 1;
   cudaError_t err;
-  if (wide) {
+  if (p.duo) {
+    cfg.blockDim = dim3(32 * (2 + kSoloEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kSoloEpilogueWarps, 1, 1, true>, map_x, map_w, map_out, map_res, p);
+  } else if (wide) {
     cfg.blockDim = dim3(32 * 18); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
     err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<16, 1, 1>, map_x, map_w, map_out, map_res, p);
   } else if (pair) {

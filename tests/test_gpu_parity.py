@@ -140,6 +140,9 @@ def test_conv_tensor_core_strip_form(hq, cfg, signed_in):
     (64, 256, 1, 56, 8, True),       # two CTAs per SM, residual pairs worked out ahead of the single large call
     (256, 256, 3, 28, 4, False),     # 4-bit output through the pipelined epilogue
     (1024, 256, 1, 28, 4, False),
+    (256, 256, 3, 28, 8, False),     # long reductions with 256 | cout: two CTAs share every MMA (cta_group::2)
+    (1024, 256, 1, 28, 8, True),
+    (512, 512, 3, 14, 8, False),
 ])
 def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw, out_bits, residual):
     """Benchmark-sized launches (several tiles per CTA: every accumulator buffer, operand stage and issuer warp is
