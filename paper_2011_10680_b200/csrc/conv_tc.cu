@@ -47,13 +47,15 @@ namespace {
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccBufs = 4;                                 // accumulator (and residual) buffers: 4 x 128 or 2 x 256 columns
-// Three launch shapes of the same kernel:
+// Four launch shapes of the same kernel:
 //   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 212 KiB of shared memory;
 //   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
 //         reduction are bound by the latency of the hand-over chain between the MMA issuer and the epilogue
 //         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
 //   wide  16 epilogue warps and one issuer, one CTA per SM: fused-residual layers on 256-pixel tiles (the longest
 //         epilogue chain per value gains from four warps per scheduler; the loop keeps one chunk in registers).
+//   duo   the solo roles in clusters of two CTAs that share every MMA (cta_group::2): long reductions whose weights
+//         stream; each CTA fetches its own weight rows and half of the pixel rows.
 constexpr int kSoloEpilogueWarps = 8;
 constexpr int kPairEpilogueWarps = 4;
 constexpr int kSoloIssuerWarps = 3;     // 1 + 3 + 8 warps = 384 threads: 168 registers per thread remain
