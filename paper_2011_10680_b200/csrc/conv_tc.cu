@@ -75,6 +75,7 @@ struct TcParams {
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
+  int32_t inplace;       // 1: the sixteen-warp shape: outputs overwrite the residual tile, which is stored as the box
   int32_t duo;           // 1: two CTAs of a cluster (adjacent SMs) share every MMA: 256 channels x 256 pixels per pair
   int32_t ni;            // MMA issuer warps in use: min(issuer warps of the launch shape, k_blocks)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
@@ -550,58 +551,80 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
 
 // The same arithmetic for the launch shape with sixteen epilogue warps (four per scheduler): no second register
 // set for the next chunk -- with four warps per scheduler the tensor-memory load of one warp hides behind the
-// arithmetic of the others -- which keeps the loop inside that shape's register budget.
+// arithmetic of the others -- which keeps the loop inside that shape's register budget.  This shape always carries
+// an 8-bit residual through the prefetched tile, and it works IN PLACE: a thread overwrites each residual byte
+// with the output value computed from it, so the [pixels][128 channels] residual tile doubles as the staging box
+// (no separate box: room for one more stage, and the store moves whole 128-byte rows).  The four warps that share
+// 64 pixel columns (one per channel quarter) meet at a named barrier, then one of them stores the columns' box and
+// hands the residual buffer back once the store has read it -- after the first chunk of the next tile, when that
+// read has long finished, unless there is only one buffer.
 template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN>
 __device__ __forceinline__ void epilogue_loop_lean8(const EpiCtx& e_in, const ChanConst& k_in) {
-  const EpiCtx e = e_in;
-  const ChanConst k = k_in;
-  const TcParams& p = *e.p;
-  SharedCtl& ctl = *e.ctl;
-  const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
-  const uint32_t my_stage = e.out_stage + (uint32_t)e.ew * (uint32_t)(px_per_warp * 32);
-  uint8_t* const my_stage_ptr = e.smem_raw + (my_stage - e.raw);
-  const uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
-  const int nchunks = px_per_warp >> 5;
-  const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
-  const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + col0;
-  auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
-    uint32_t w = 1;
-    if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
-    return __shfl_sync(0xffffffffu, w, 0) != 0;
-  };
-  uint32_t tcount = 0;
-  for (int p_tile = e.p_tile0; p_tile < p.p_tiles; p_tile += e.p_step, ++tcount) {
-    const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
-    const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
-    if (!wait_bar(&ctl.tfull[as], aph)) break;
-    if (RES && !wait_bar(&ctl.rfull[rs], rph)) break;
-    tc_fence_after();
-    if (lane == 0) tma_store_wait_read0();        // the previous tile's store has read the staging box
-    __syncwarp();
-    const uint8_t* const res_tile = res_stage_ptr + rs * e.res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
-    for (int c = 0; c < nchunks; ++c) {
-      int v[32];
-      tmem_ld32(t_warp + as * p.pt + c * 32, v);
-      if (!e.warp_live) continue;
+  if constexpr (RES) {
+    const EpiCtx e = e_in;
+    const ChanConst k = k_in;
+    const TcParams& p = *e.p;
+    SharedCtl& ctl = *e.ctl;
+    const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
+    uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
+    const int nchunks = px_per_warp >> 5;
+    const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
+    const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + col0;
+    const bool leader = q == 0;                     // the warp of its four that stores the box
+    auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
+      uint32_t w = 1;
+      if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+      return __shfl_sync(0xffffffffu, w, 0) != 0;
+    };
+    uint32_t tcount = 0, owed_rs = 0;
+    bool owe = false;                               // leader: the previous tile's residual buffer is still to be handed back
+    for (int p_tile = e.p_tile0; p_tile < p.p_tiles; p_tile += e.p_step, ++tcount) {
+      const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
+      const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
+      if (lane == 0) HQ_TRACE(7, tcount * 16 + e.ew);
+      if (!wait_bar(&ctl.tfull[as], aph)) break;
+      if (lane == 0) HQ_TRACE(8, tcount * 16 + e.ew);
+      if (!wait_bar(&ctl.rfull[rs], rph)) break;
+      if (lane == 0) HQ_TRACE(3, tcount * 16 + e.ew);
+      tc_fence_after();
+      const uint32_t box_off = rs * e.res_tile_bytes + (uint32_t)col0 * kTileC;      // the four warps' 64 rows of 128 bytes
+      uint8_t* const mine = res_stage_ptr + box_off + cq * 32 + lane;
+      for (int c = 0; c < nchunks; ++c) {
+        int v[32];
+        tmem_ld32(t_warp + as * p.pt + c * 32, v);
+        if (c == 0 && owe) {
+          if (lane == 0) { tma_store_wait_read0(); mbar_arrive(smem_u32(&ctl.rempty[owed_rs])); }
+          owe = false;
+        }
+        if (e.warp_live) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int r = !RES ? 0 : RSIGNED ? (int)(signed char)res_tile[(c * 32 + j) * kTileC] : (int)res_tile[(c * 32 + j) * kTileC];
-        const int s = requant_fast<RES, RSIGNED, SMALL, RN>(v[j], r, k);
-        v[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
+          for (int j = 0; j < 32; ++j) {
+            const int r = RSIGNED ? (int)(signed char)mine[(c * 32 + j) * kTileC] : (int)mine[(c * 32 + j) * kTileC];
+            const int s = requant_fast<true, RSIGNED, SMALL, RN>(v[j], r, k);
+            v[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mine[(c * 32 + j) * kTileC] = (uint8_t)v[j];
+        }
       }
-#pragma unroll
-      for (int j = 0; j < 32; ++j) my_stage_ptr[(c * 32 + j) * 32 + lane] = (uint8_t)v[j];
+      tc_fence_before();
+      fence_async_smem();                           // make this lane's box writes visible to the TMA engine
+      __syncwarp();
+      if (lane == 0) release_accumulator(p, ctl, as);
+      if (lane == 0) HQ_TRACE(9, tcount * 16 + e.ew);
+      asm volatile("bar.sync %0, 128;" :: "r"(2 + e.half) : "memory");
+      if (lane == 0) HQ_TRACE(6, tcount * 16 + e.ew);
+      if (leader) {
+        if (lane == 0) {
+          const int p_base = p_tile * p.pt + col0;
+          if (p_base < p.P) { tma_store_2d(e.map_out, e.res_stage + box_off, e.c_tile * kTileC, p_base); tma_store_commit(); }
+          if (rmask == 0) { tma_store_wait_read0(); mbar_arrive(smem_u32(&ctl.rempty[rs])); }
+        }
+        owe = rmask != 0; owed_rs = rs;
+      }
     }
-    tc_fence_before();
-    fence_async_smem();                           // make this lane's box writes visible to the TMA engine
-    __syncwarp();
-    if (lane == 0) {
-      release_accumulator(p, ctl, as);
-      if (RES) mbar_arrive(smem_u32(&ctl.rempty[rs]));
-      if (e.warp_live) store_warp_box(p, e.map_out, my_stage, e.c_tile * kTileC + cq * 32, p_tile, col0, px_per_warp);
-    }
+    if (leader && lane == 0) tma_store_wait_all();
   }
-  if (lane == 0) tma_store_wait_all();
 }
 
 // General tile loop: every output type, direct stores, 64-bit arithmetic, INT32 residuals.
@@ -615,6 +638,8 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
   const int lane = e.lane, q = e.q, cq = e.cq, ew = e.ew, col0 = e.col0, px_per_warp = e.px_per_warp, ch = e.ch;
   const int c_tile = e.c_tile, p_tile0 = e.p_tile0, p_step = e.p_step, lo = e.lo, hi = e.hi;
   const bool ch_live = e.ch_live, warp_live = e.warp_live;
+  // the in-place launch shape has no staging box: this loop then stores straight to global memory
+  const bool staged_out = p.staged_out && !p.inplace;
     // staging box of this warp: [px_per_warp pixels][32 channels] bytes (16 bytes per pixel at 4 bit)
     const int row_b = (p.out_bits == 4) ? 16 : 32;
     const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(px_per_warp * 32);   // px_per_warp rows x 32 bytes reserved per warp
@@ -628,7 +653,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       const uint32_t rs = tcount & ((1u << p.lg_rbufs) - 1u), rph = (tcount >> p.lg_rbufs) & 1u;
       uint32_t w = 1;
       if (lane == 0) {
-        if (p.staged_out) tma_store_wait_read0();   // the previous store has read this warp's staging box
+        if (staged_out) tma_store_wait_read0();   // the previous store has read this warp's staging box
         w = mbar_wait(smem_u32(&ctl.tfull[as]), aph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
         if (w && p.staged_res)
           w = mbar_wait(smem_u32(&ctl.rfull[rs]), rph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
@@ -721,7 +746,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
             const int other = __shfl_xor_sync(0xffffffffu, y[j], 1);
             y[j] = (y[j] & 0xF) | ((other & 0xF) << 4);
           }
-          if (p.staged_out) {
+          if (staged_out) {
             if (!(lane & 1)) {
 #pragma unroll
               for (int j = 0; j < 32; ++j) my_stage_ptr[(cc0 + j) * row_b + (lane >> 1)] = (uint8_t)y[j];
@@ -731,7 +756,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 #pragma unroll
             for (int j = 0; j < 32; ++j) if (px0 + j < p.P) dst[((long long)j * p.C) >> 1] = (unsigned char)y[j];
           }
-        } else if (p.staged_out) {
+        } else if (staged_out) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) my_stage_ptr[(cc0 + j) * 32 + lane] = (uint8_t)y[j];
         } else if (ch_live) {
@@ -743,17 +768,18 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       if (ew == 0 && lane == 0) HQ_TRACE(4, tcount);
       // accumulator columns (and the residual tile) are no longer needed by this warp: hand them back
       tc_fence_before();
-      if (p.staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
+      if (staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
       __syncwarp();
+      if (p.inplace) asm volatile("bar.sync %0, 128;" :: "r"(2 + e.half) : "memory");   // one arrival per four warps there
       if (lane == 0) {
         release_accumulator(p, ctl, as);
-        if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
-        if (p.staged_out && warp_live)
+        if (p.staged_res && (!p.inplace || q == 0)) mbar_arrive(smem_u32(&ctl.rempty[rs]));
+        if (staged_out && warp_live)
           store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_tile, col0, px_per_warp);
       }
     }
 
-    if (p.staged_out && lane == 0) tma_store_wait_all();
+    if (staged_out && lane == 0) tma_store_wait_all();
 }
 
 // ---------------------------------------------------------------- the kernel -----------------
@@ -791,7 +817,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     for (int s = 0; s < (1 << p.lg_bufs); ++s) {
       mbar_init(smem_u32(&ctl.tfull[s]), p.ni); mbar_init(smem_u32(&ctl.tempty[s]), (4 * p.halves) << p.duo);
       mbar_init(smem_u32(&ctl.tstart[s]), 1);
-      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), 4 * p.halves);
+      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), p.inplace ? p.halves : 4 * p.halves);
     }
     mbar_init(smem_u32(&ctl.drain), p.ni);
     mbar_init(smem_u32(&ctl.wfull), 1);
@@ -821,9 +847,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
       const uint32_t rmask = (1u << p.lg_rbufs) - 1u;
-      // With as many residual buffers as accumulators the tile is fetched ahead of the operands; with fewer, beside
-      // the last operand block, when the epilogue of the tile before has long handed its buffer back.
-      const int res_kb = p.lg_rbufs < p.lg_bufs ? p.k_blocks - 1 : 0;
       bool ok = true;
       // (image, row, column) of the tile's first output pixel, advanced by a fixed step per tile
       const int ho = p.howo / p.wo;
@@ -887,14 +910,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         oh += d_oh; if (oh >= ho) { oh -= ho; ++img; }
         img += d_img;
         int chunk = 0, tap_s = 0, tap_r = 0;
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          if (p.staged_res && kb == res_kb) {   // residual tile of this output tile
-            const uint32_t rbuf = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
-            if (!mbar_wait(smem_u32(&ctl.rempty[rbuf]), rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-            const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
-            mbar_expect_tx(bar, res_tile_bytes);
-            tma_load_2d(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0);
+        // The residual tile of this output tile is fetched as soon as its buffer is free, but this thread only
+        // blocks for the buffer after the tile's last operand block is on its way: the buffer comes back when the
+        // epilogue of an earlier tile ends, and the operand copies must not queue behind that.
+        bool res_due = p.staged_res != 0;
+        auto residual = [&](bool must) -> bool {
+          const uint32_t rbuf = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
+          const uint32_t rb = smem_u32(&ctl.rempty[rbuf]);
+          if (!mbar_try_wait(rb, rph ^ 1u)) {
+            if (!must) return true;
+            if (!mbar_wait(rb, rph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) return false;
           }
+          const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
+          mbar_expect_tx(bar, res_tile_bytes);
+          tma_load_2d(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0);
+          res_due = false;
+          return true;
+        };
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          if (res_due && !residual(false)) { ok = false; break; }
           if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
           HQ_TRACE(0, it);
           const uint32_t bar = smem_u32(&ctl.full[s]);
@@ -908,6 +942,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tma_load_2d_2cta(w_dst, &map_w, bar, kb * p.bkb, c_tile * kTileC);
             if (++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
             if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+            if (res_due && kb + 1 == p.k_blocks && !residual(true)) { ok = false; break; }
             continue;
           }
           mbar_expect_tx(bar, stage_bytes);
@@ -926,6 +961,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           }
           if (++chunk == p.cchunks) { chunk = 0; if (++tap_s == p.kw) { tap_s = 0; ++tap_r; } }
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+          if (res_due && kb + 1 == p.k_blocks && !residual(true)) { ok = false; break; }
         }
       }
       // Drain: every copy this thread started must have landed before the CTA may exit.
@@ -1402,11 +1438,16 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
         res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
         // residual tiles: as many buffers as accumulators, fewer when a long reduction needs the room for stages
         // (its epilogue has slack: a single residual buffer only delays the next tile's prefetch)
+        // The sixteen-warp shape (below) works in place in the residual tiles and needs no staging box; with the
+        // weights resident two stages are enough for its short reductions (the epilogue bounds the tile).
+        const bool wide_here = p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
+        if (wide_here) out_tile_bytes = 0;
+        const int min_stages = (wide_here && p.wres) ? 2 : 3;
         for (p.lg_rbufs = p.lg_bufs; ; --p.lg_rbufs) {
           stages = (smem_budget - out_tile_bytes - (res_tile_bytes << p.lg_rbufs) - wres_bytes) / stage_bytes;
-          if (stages >= 3 || p.lg_rbufs == 0 || !res_tile_bytes || k_total < 1024) break;
+          if (stages >= min_stages || p.lg_rbufs == 0 || !res_tile_bytes || k_total < 1024) break;
         }
-        if (stages >= 3 || (p.pt == 64 && keep_w == 0)) chosen = true;
+        if (stages >= min_stages || (p.pt == 64 && keep_w == 0)) chosen = true;
       }
     }
   }
@@ -1462,9 +1503,11 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // Third launch shape, *wide*: sixteen epilogue warps (four per scheduler, 64 pixel columns each) with a loop that
     // keeps one chunk in registers.  Measured per layer: it wins where the epilogue carries the residual add on
     // 256-pixel tiles with a short reduction (1x1 128 -> 512 at 28x28: 81 -> 72 us) and loses a few percent
-    // everywhere else (long reductions are bound by the operand stream, not by the epilogue).
+    // everywhere else (long reductions are bound by the operand stream, not by the epilogue).  Its outputs overwrite
+    // the residual tile they were computed from, which then leaves as the store's box: no staging box, so that
+    // 256-pixel tiles also fit beside a 32-64 KiB weight slab (1x1 256 -> 1024 at 14x14: 55 -> 44 us).
     wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
-    if (wide) p.halves = 4;
+    if (wide) { p.halves = 4; p.inplace = 1; }
     // Fourth shape, *duo*: clusters of two CTAs on adjacent SMs share every MMA (cta_group::2, M = 256): each CTA
     // fetches its own 128 weight rows and HALF of the tile's pixel rows, 32 KiB per K block and SM instead of
     // 48 KiB for the same MMA time.  For the long reductions whose weights stream, which the operand fetch bounds.
@@ -1562,7 +1605,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
   } else
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, a.out_bits == 4 ? 16 : 32, p.pt / (p.halves << p.fold),
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, p.inplace ? kTileC : a.out_bits == 4 ? 16 : 32, p.pt / (p.halves << p.fold),
                                        CU_TENSOR_MAP_SWIZZLE_NONE)) return HQ_ERR_CUDA;
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
     return HQ_ERR_CUDA;

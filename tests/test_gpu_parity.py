@@ -143,6 +143,9 @@ def test_conv_tensor_core_strip_form(hq, cfg, signed_in):
     (256, 256, 3, 28, 8, False),     # long reductions with 256 | cout: two CTAs share every MMA (cta_group::2)
     (1024, 256, 1, 28, 8, True),
     (512, 512, 3, 14, 8, False),
+    (128, 512, 1, 28, 8, True),      # sixteen epilogue warps working in place in the residual tiles
+    (256, 1024, 1, 28, 8, True),
+    (512, 2048, 1, 14, 8, True),     # the same with two operand stages beside a 64 KiB weight slab
 ])
 def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw, out_bits, residual):
     """Benchmark-sized launches (several tiles per CTA: every accumulator buffer, operand stage and issuer warp is
@@ -160,6 +163,47 @@ def test_conv_many_tiles_per_cta_repeated_images(hq, cin, cout, k, hw, out_bits,
     big["x"] = np.ascontiguousarray(np.tile(case["x"], (n // 2, 1, 1, 1)))
     if residual:
         big["res"] = np.ascontiguousarray(np.tile(case["res"], (n // 2, 1, 1, 1)))
+    big["n"] = n
+    hq.set_conv_path(2)
+    try:
+        st, out = hq.conv_case(big)
+        assert st == binding.HQ_OK
+        hq.sync()
+    finally:
+        hq.set_conv_path(0)
+    got = out.cpu().numpy().view(ref.dtype).reshape((n // 2, 2) + ref.shape[1:])
+    for i in range(n // 2):
+        assert np.array_equal(got[i], ref), f"copy {i} differs"
+
+
+@pytest.mark.parametrize("variant", ["small_residual_shift", "clamp_and_small_c", "signed_residual", "ragged_channels"])
+def test_conv_in_place_residual_shape_variants(hq, variant):
+    """The launch shape that overwrites the prefetched residual tile with its outputs (256-pixel tiles, 8-bit residual,
+    short reduction), in the cases that leave its common loop: residual shifts below 9 (64-bit tile loop, direct
+    stores), clamp bounds inside the type with main shifts below 32, a signed residual with every shift, and a
+    channel count that leaves the last channel tile ragged.  Two distinct images repeated over a batch of 16."""
+    from paper_2011_10680_b200 import binding
+    n, cout = 16, 256
+    kw = dict(residual=True, c_range=(39, 43))
+    if variant == "clamp_and_small_c":
+        kw["c_range"] = (28, 43)
+    if variant == "signed_residual":
+        kw["relu"] = False
+    if variant == "ragged_channels":
+        cout = 208
+    case = inputs.conv_case(212, 2, 56, 56, 64, cout, 1, 1, 0, **kw)
+    if variant == "small_residual_shift":
+        case["rc"][::3] = 5
+    if variant == "clamp_and_small_c":
+        case["qmin"], case["qmax"] = 3, 200
+    if variant == "signed_residual":
+        case["res"] = case["res"].view(np.int8)
+        case["res_signed"] = 1
+        case["rc"][:] = np.arange(cout) % 36 + 9
+    ref = oracle().conv_case(case)
+    big = dict(case)
+    big["x"] = np.ascontiguousarray(np.tile(case["x"], (n // 2, 1, 1, 1)))
+    big["res"] = np.ascontiguousarray(np.tile(case["res"], (n // 2, 1, 1, 1)))
     big["n"] = n
     hq.set_conv_path(2)
     try:
