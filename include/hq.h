@@ -43,7 +43,8 @@ typedef enum {
   HQ_ERR_RANGE = 4,        /* reserved: accumulator + bias left INT32 (the CPU oracle reports it) */
   HQ_ERR_WORKSPACE = 5,    /* device allocation failed */
   HQ_ERR_CUDA = 6,         /* a CUDA runtime or driver call failed */
-  HQ_ERR_TIMEOUT = 7       /* a bounded device-side wait expired; outputs are not valid */
+  HQ_ERR_TIMEOUT = 7,      /* a bounded device-side wait expired; outputs are not valid */
+  HQ_ERR_INFEASIBLE = 8    /* hq_ilp_solve: no assignment meets the limits */
 } hq_status;
 
 typedef struct {  /* activation tensor, dense NHWC */
@@ -209,6 +210,22 @@ hq_status hq_set_conv_path(hq_handle* h, int32_t path);
  * every wait inside the kernels does after its own budget.  The next hq_sync reports HQ_ERR_TIMEOUT; the
  * context stays usable.  Asynchronous on `stream`. */
 hq_status hq_expire_wait_selftest(hq_handle* h, int32_t budget_ms, void* stream);
+
+/* Bit-width selection by integer linear programming (Section 3.4, Eq. 5).  Every one of n_layers layers takes
+ * one of two precisions (choice 0 or 1, e.g. INT4 or INT8); the summed perturbation
+ *   sum_i omega[i][b_i]   is minimised subject to
+ *   sum_i size[i][b_i] <= size_limit,  sum_i bops[i][b_i] <= bops_limit,  sum_i latency[i][b_i] <= latency_limit
+ * (M_i, G_i = b_w b_a MAC_i and Q_i of the paper; latency is what was measured per layer on the target GPU).
+ * HOST pointers: four arrays of n_layers x 2 int64 values, [layer][choice], every value in [0, 2^40], in units of
+ * the caller's choice; a negative limit switches that constraint off.  choice_out[n_layers] receives an optimal
+ * assignment (any one of them when several are optimal) and objective_out, if not NULL, its perturbation.
+ * Exact (depth-first branch and bound with fractional-knapsack bounds); pure host code, no GPU work, no handle.
+ * Returns HQ_ERR_INFEASIBLE when no assignment meets the limits (choice_out untouched), HQ_ERR_INVALID_ARG for
+ * NULL arrays, n_layers outside [0, 4096] or values out of range, HQ_ERR_UNSUPPORTED if the search exceeds
+ * 2 * 10^8 nodes. */
+hq_status hq_ilp_solve(int32_t n_layers, const int64_t* omega, const int64_t* size, const int64_t* bops,
+                       const int64_t* latency, int64_t size_limit, int64_t bops_limit, int64_t latency_limit,
+                       int32_t* choice_out, int64_t* objective_out);
 
 const char* hq_status_string(hq_status s);
 

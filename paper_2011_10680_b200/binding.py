@@ -15,13 +15,14 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhq.so")
 
 HQ_OK, HQ_ERR_INVALID_ARG, HQ_ERR_UNSUPPORTED, HQ_ERR_ALIGNMENT = 0, 1, 2, 3
-HQ_ERR_RANGE, HQ_ERR_WORKSPACE, HQ_ERR_CUDA, HQ_ERR_TIMEOUT = 4, 5, 6, 7
+HQ_ERR_RANGE, HQ_ERR_WORKSPACE, HQ_ERR_CUDA, HQ_ERR_TIMEOUT, HQ_ERR_INFEASIBLE = 4, 5, 6, 7, 8
 HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant": 5}
 
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
     "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
+    "hq_ilp_solve",
 ]
 
 
@@ -84,6 +85,8 @@ def lib():
         L.hq_set_conv_path.argtypes = [vp, i32]
         L.hq_expire_wait_selftest.argtypes = [vp, i32, vp]
         L.hq_expire_wait_selftest.restype = i32
+        i64p = C.POINTER(C.c_int64)
+        L.hq_ilp_solve.argtypes = [i32, i64p, i64p, i64p, i64p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(i32), i64p]
         L.hq_status_string.argtypes = [i32]
         L.hq_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -91,6 +94,20 @@ def lib():
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
+
+
+def ilp_solve(omega, size, bops, latency, size_limit: int = -1, bops_limit: int = -1, latency_limit: int = -1):
+    """hq_ilp_solve on host arrays of shape [n_layers, 2] (int64).  Returns (status, choices, objective)."""
+    tabs = [np.ascontiguousarray(t, dtype=np.int64) for t in (omega, size, bops, latency)]
+    n = tabs[0].shape[0]
+    if any(t.shape != (n, 2) for t in tabs):
+        raise ValueError("every table must have shape [n_layers, 2]")
+    choice = np.zeros(max(n, 1), dtype=np.int32)
+    obj = C.c_int64(0)
+    i64p = C.POINTER(C.c_int64)
+    st = lib().hq_ilp_solve(n, *[t.ctypes.data_as(i64p) for t in tabs], int(size_limit), int(bops_limit),
+                            int(latency_limit), choice.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(obj))
+    return st, choice[:n].copy(), int(obj.value)
 
 
 def status_string(code: int) -> str:

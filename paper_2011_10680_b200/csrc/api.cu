@@ -153,6 +153,7 @@ const char* hq_status_string(hq_status s) {
     case HQ_ERR_WORKSPACE: return "HQ_ERR_WORKSPACE";
     case HQ_ERR_CUDA: return "HQ_ERR_CUDA";
     case HQ_ERR_TIMEOUT: return "HQ_ERR_TIMEOUT";
+    case HQ_ERR_INFEASIBLE: return "HQ_ERR_INFEASIBLE";
   }
   return "HQ_ERR_UNKNOWN";
 }

@@ -251,8 +251,15 @@ class _Builder:
         return self._emit(layer, s_out, (1, 1, c), 8)
 
 
+def resnet_choice_units(depth: int) -> int:
+    """Number of per-layer bit-width choices of a ResNet table: the convs of the residual blocks, a
+    down-sampling shortcut conv being tied to the block's first conv (they share one quantized input)."""
+    return {18: 16, 50: 48}[depth]
+
+
 def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: bool = False,
-                 image_hw: int = 224, classes: int = 1000, width: int = 64) -> dict:
+                 image_hw: int = 224, classes: int = 1000, width: int = 64,
+                 conv_bits: list[int] | None = None) -> dict:
     """Layer table of an ImageNet-shaped ResNet-18 or ResNet-50 with integer parameters.
 
     Tensor id -1 is the uint8 input image (n, image_hw, image_hw, 3); layer i produces tensor i.
@@ -264,6 +271,10 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
     convs inside the block write uint4 directly.  First conv and classifier stay 8-bit
     (Appendix H).  ResNet-50 puts the stride on the first 1x1 of a down-sampling bottleneck unless
     stride_on_3x3 is set; only that placement reproduces the paper's BOPS column (Table 1b).
+    conv_bits gives the bit-width (4 or 8) of every block conv in network order instead
+    (resnet_choice_units(depth) entries, e.g. the answer of the bit-width ILP of Section 3.4): a conv
+    writes its output at the bit-width of the conv that reads it, and a block whose first conv is
+    4-bit requantizes the stream tensor once for that conv and the shortcut conv.
     """
     if depth not in (18, 50):
         raise ValueError("depth must be 18 or 50")
@@ -273,29 +284,37 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
     x = bd.maxpool(x, 3, 2, 1)
     blocks = [2, 2, 2, 2] if depth == 18 else [3, 4, 6, 3]
     expansion = 1 if depth == 18 else 4
+    per_block = 2 if depth == 18 else 3
+    if conv_bits is None:
+        conv_bits = [4 if (mixed and stage >= 2) else 8 for stage, nblk in enumerate(blocks)
+                     for _ in range(nblk * per_block)]
+    if len(conv_bits) != sum(blocks) * per_block or any(b not in (4, 8) for b in conv_bits):
+        raise ValueError("conv_bits needs one entry (4 or 8) per block conv")
+    unit = 0
     for stage, nblk in enumerate(blocks):
         planes = width << stage
-        wb = 4 if (mixed and stage >= 2) else 8
         for blk in range(nblk):
             stride = 2 if (blk == 0 and stage > 0) else 1
             cin = bd.shape[x][2]
             need_ds = stride != 1 or cin != planes * expansion
-            xin = bd.requant(x, 4) if wb == 4 else x
+            wb = conv_bits[unit:unit + per_block]
+            unit += per_block
+            xin = bd.requant(x, 4) if wb[0] == 4 else x
             if depth == 18:
-                y = bd.conv(xin, planes, 3, stride, 1, wb, relu=True, out_bits=wb)
-                shortcut = bd.conv(xin, planes, 1, stride, 0, wb, relu=False, out_bits=8,
+                y = bd.conv(xin, planes, 3, stride, 1, wb[0], relu=True, out_bits=wb[1])
+                shortcut = bd.conv(xin, planes, 1, stride, 0, wb[0], relu=False, out_bits=8,
                                    out_signed=True) if need_ds else x
-                x = bd.conv(y, planes, 3, 1, 1, wb, relu=True, out_bits=8, res=shortcut)
+                x = bd.conv(y, planes, 3, 1, 1, wb[1], relu=True, out_bits=8, res=shortcut)
             else:
                 s1, s2 = (1, stride) if stride_on_3x3 else (stride, 1)
-                y = bd.conv(xin, planes, 1, s1, 0, wb, relu=True, out_bits=wb)
-                y = bd.conv(y, planes, 3, s2, 1, wb, relu=True, out_bits=wb)
-                shortcut = bd.conv(xin, planes * 4, 1, stride, 0, wb, relu=False, out_bits=8,
+                y = bd.conv(xin, planes, 1, s1, 0, wb[0], relu=True, out_bits=wb[1])
+                y = bd.conv(y, planes, 3, s2, 1, wb[1], relu=True, out_bits=wb[2])
+                shortcut = bd.conv(xin, planes * 4, 1, stride, 0, wb[0], relu=False, out_bits=8,
                                    out_signed=True) if need_ds else x
-                x = bd.conv(y, planes * 4, 1, 1, 0, wb, relu=True, out_bits=8, res=shortcut)
+                x = bd.conv(y, planes * 4, 1, 1, 0, wb[2], relu=True, out_bits=8, res=shortcut)
     x = bd.avgpool(x)
     x = bd.conv(x, classes, 1, 1, 0, 8, relu=False, out_bits=32, op="linear")
-    return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=depth,
+    return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=depth, conv_bits=list(conv_bits),
                 shapes=[bd.shape[i] for i in range(len(bd.layers))],
                 bits=[bd.bits[i] for i in range(len(bd.layers))])
 
