@@ -358,6 +358,99 @@ def run_sweep_grid(args):
     hq.close()
 
 
+def run_ilp(args):
+    """Hardware-aware bit-width selection (Section 3.4): per-layer latencies of the INT8 and INT4 forms measured
+    on this GPU feed the ILP, together with model size, BOPS and a synthetic sensitivity; every answer is then
+    built and timed as a network of its own."""
+    import torch
+    from paper_2011_10680_b200 import binding, build
+
+    build.build()
+    depth, seed = 50, 3
+    batch = args.batch or 256
+    units = inputs.resnet_choice_units(depth)
+    hq = binding.Handle(0)
+    images_d = torch.from_numpy(inputs.random_images(seed, batch)).cuda()
+    stream = torch.cuda.Stream()
+
+    def measure(conv_bits):
+        table = inputs.resnet_table(depth, seed, conv_bits=conv_bits)
+        net = binding.Network(hq, table, batch)
+        logits = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+        with torch.cuda.stream(stream):
+            for _ in range(max(args.warmup, 3)):
+                assert net.run(images_d, logits) == binding.HQ_OK
+            hq.sync()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                net.run(images_d, logits)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            ns = np.zeros(len(table["layers"]))
+            for _ in range(3):
+                ns += np.array(net.time_layers(images_d, logits), dtype=np.float64)
+            hq.sync()
+        net.close()
+        return table, ns / 3.0, ms
+
+    def per_unit(table, layer_ns):
+        q, m, g = np.zeros(units), np.zeros(units), np.zeros(units)
+        fixed = 0.0
+        for l, ns in zip(table["layers"], layer_ns):
+            u = l.get("unit", -1)
+            if u is None or u < 0:
+                fixed += ns
+                continue
+            q[u] += ns
+            if l["op"] == "conv":
+                m[u] += l["params"] * l["bits"] / 8.0
+                g[u] += float(l["bits"]) ** 2 * l["macs"]
+        return q, m, g, fixed
+
+    t8, ns8, ms8 = measure([8] * units)
+    t4, ns4, ms4 = measure([4] * units)
+    q8, m8, g8, fixed8 = per_unit(t8, ns8)
+    q4, m4, g4, _ = per_unit(t4, ns4)
+    lat = np.stack([q4, q8], axis=1).round().astype(np.int64)              # ns per batch, choice 0 = INT4, 1 = INT8
+    size = np.stack([m4, m8], axis=1).round().astype(np.int64)             # bytes
+    bops = (np.stack([g4, g8], axis=1) / 1e6).round().astype(np.int64)     # mega bit-operations per image
+    omega = inputs.synthetic_sensitivity(t8, seed)
+    rows = [{"case": "uniform INT8", "bits": "8" * units, "step_ms": ms8, "layer_sum_us": float(ns8.sum() / 1e3)},
+            {"case": "uniform INT4 (first and last layer INT8)", "bits": "4" * units, "step_ms": ms4,
+             "layer_sum_us": float(ns4.sum() / 1e3)}]
+
+    def span(t, frac):
+        lo, hi = int(t.min(axis=1).sum()), int(t.max(axis=1).sum())
+        return lo + int(frac * (hi - lo))
+
+    cases = [("size", 0, 0.5), ("size", 0, 0.25), ("bops", 1, 0.5), ("latency", 2, 0.5), ("latency", 2, 0.1),
+             ("size+latency", -1, 0.5)]
+    for name, which, frac in cases:
+        lims = [-1, -1, -1]
+        if which >= 0:
+            lims[which] = span((size, bops, lat)[which], frac)
+        else:
+            lims[0], lims[2] = span(size, frac), span(lat, frac)
+        t0 = time.time()
+        st, choice, obj = binding.ilp_solve(omega, size, bops, lat, *lims)
+        solve_s = time.time() - t0
+        if st != binding.HQ_OK:
+            rows.append({"case": name, "fraction_of_range": frac, "status": binding.status_string(st)})
+            continue
+        bits = [8 if c else 4 for c in choice]
+        table, ns, ms = measure(bits)
+        idx = np.arange(units)
+        rows.append({"case": f"{name} limit at {frac} of the INT4..INT8 range", "limits": lims, "solve_s": solve_s,
+                     "bits": "".join(str(b) for b in bits), "n_int4": int(sum(1 for b in bits if b == 4)), "omega": obj,
+                     "size_MB": float(size[idx, choice].sum() / 2 ** 20), "gbops_per_image": float(bops[idx, choice].sum() / 1e3),
+                     "predicted_us": float((lat[idx, choice].sum() + fixed8) / 1e3), "layer_sum_us": float(ns.sum() / 1e3),
+                     "step_ms": ms})
+    print(json.dumps({"metric": "bit-width ILP on measured B200 layer latencies (ResNet-50 block convs)", "batch": batch,
+                      "units": units, "latency_ns": lat.tolist(), "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -371,6 +464,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the fused conv/GEMM sweep (config 5) instead of the network")
     ap.add_argument("--sweep-grid", action="store_true", help="run the full 480-point M x N x K x bits x residual grid of config 5")
     ap.add_argument("--membound", action="store_true", help="time the memory-bound kernels (pooling, requantization, residual add) on their own")
+    ap.add_argument("--ilp", action="store_true", help="measure per-layer INT4/INT8 latencies and solve the bit-width ILP of Section 3.4 for several limits")
     ap.add_argument("--sweep-pixels", type=int, default=200704, help="output pixels per sweep shape (batch is derived)")
     ap.add_argument("--sweep-only", type=int, default=-1, help="run a single sweep shape (index), e.g. for profiling")
     args = ap.parse_args()
@@ -389,6 +483,10 @@ def main():
     if args.membound:
         if rank == 0:
             run_membound(args)
+        return
+    if args.ilp:
+        if rank == 0:
+            run_ilp(args)
         return
     if args.sweep:
         if rank == 0:

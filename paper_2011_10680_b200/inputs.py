@@ -196,7 +196,7 @@ class _Builder:
         return tid
 
     def conv(self, src: int, cout: int, k: int, stride: int, pad: int, bits: int, *, relu: bool,
-             out_bits: int, out_signed: bool = False, res: int = -1, op: str = "conv") -> int:
+             out_bits: int, out_signed: bool = False, res: int = -1, op: str = "conv", unit: int = -1) -> int:
         g = self.g
         h, w, cin = self.shape[src]
         assert self.bits[src] == bits, "conv input must already have the conv's bit-width"
@@ -208,7 +208,7 @@ class _Builder:
                      bits=bits, wgt=(pack4(q) if bits == 4 else q.astype(np.int8)), bias=bias,
                      relu=int(relu), out_bits=out_bits, out_signed=int(out_signed),
                      b=None, c=None, rb=None, rc=None, qmin=0, qmax=0,
-                     macs=ho * wo * cout * k * k * cin, params=cout * k * k * cin)
+                     macs=ho * wo * cout * k * k * cin, params=cout * k * k * cin, unit=unit)
         if out_bits == 32:                      # raw INT32 logits: bias added, no requantization
             layer.update(qmin=-(1 << 31), qmax=(1 << 31) - 1, out_signed=1)
             return self._emit(layer, s_in * float(s_w.mean()), (ho, wo, cout), 32)
@@ -224,14 +224,14 @@ class _Builder:
             layer.update(qmin=0, qmax=(1 << out_bits) - 1)
         return self._emit(layer, s_out, (ho, wo, cout), out_bits)
 
-    def requant(self, src: int, out_bits: int) -> int:
+    def requant(self, src: int, out_bits: int, unit: int = -1) -> int:
         """Unsigned stream tensor -> lower-bit unsigned copy (Fig. 2: quantize the input once)."""
         h, w, c = self.shape[src]
         s_out = _draw_scale(self.g) * (255.0 / 15.0 if out_bits == 4 else 1.0)
         b, cc = dyadic_from_scale(self.scale[src] / s_out)
         layer = dict(op="requant", in0=src, in1=-1, cout=c, b=np.full(c, b[0], np.int32),
                      c=np.full(c, cc[0], np.int32), rb=None, rc=None, relu=0, qmin=0,
-                     qmax=(1 << out_bits) - 1, out_bits=out_bits, out_signed=0, macs=0, params=0)
+                     qmax=(1 << out_bits) - 1, out_bits=out_bits, out_signed=0, macs=0, params=0, unit=unit)
         return self._emit(layer, s_out, (h, w, c), out_bits)
 
     def maxpool(self, src: int, k: int, stride: int, pad: int) -> int:
@@ -298,20 +298,21 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
             cin = bd.shape[x][2]
             need_ds = stride != 1 or cin != planes * expansion
             wb = conv_bits[unit:unit + per_block]
+            u0 = unit                             # layers carry the index of the choice they belong to
             unit += per_block
-            xin = bd.requant(x, 4) if wb[0] == 4 else x
+            xin = bd.requant(x, 4, unit=u0) if wb[0] == 4 else x
             if depth == 18:
-                y = bd.conv(xin, planes, 3, stride, 1, wb[0], relu=True, out_bits=wb[1])
+                y = bd.conv(xin, planes, 3, stride, 1, wb[0], relu=True, out_bits=wb[1], unit=u0)
                 shortcut = bd.conv(xin, planes, 1, stride, 0, wb[0], relu=False, out_bits=8,
-                                   out_signed=True) if need_ds else x
-                x = bd.conv(y, planes, 3, 1, 1, wb[1], relu=True, out_bits=8, res=shortcut)
+                                   out_signed=True, unit=u0) if need_ds else x
+                x = bd.conv(y, planes, 3, 1, 1, wb[1], relu=True, out_bits=8, res=shortcut, unit=u0 + 1)
             else:
                 s1, s2 = (1, stride) if stride_on_3x3 else (stride, 1)
-                y = bd.conv(xin, planes, 1, s1, 0, wb[0], relu=True, out_bits=wb[1])
-                y = bd.conv(y, planes, 3, s2, 1, wb[1], relu=True, out_bits=wb[2])
+                y = bd.conv(xin, planes, 1, s1, 0, wb[0], relu=True, out_bits=wb[1], unit=u0)
+                y = bd.conv(y, planes, 3, s2, 1, wb[1], relu=True, out_bits=wb[2], unit=u0 + 1)
                 shortcut = bd.conv(xin, planes * 4, 1, stride, 0, wb[0], relu=False, out_bits=8,
-                                   out_signed=True) if need_ds else x
-                x = bd.conv(y, planes * 4, 1, 1, 0, wb[2], relu=True, out_bits=8, res=shortcut)
+                                   out_signed=True, unit=u0) if need_ds else x
+                x = bd.conv(y, planes * 4, 1, 1, 0, wb[2], relu=True, out_bits=8, res=shortcut, unit=u0 + 2)
     x = bd.avgpool(x)
     x = bd.conv(x, classes, 1, 1, 0, 8, relu=False, out_bits=32, op="linear")
     return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=depth, conv_bits=list(conv_bits),
@@ -335,6 +336,24 @@ def table_cost(table: dict, force_bits: int | None = None) -> dict:
         bops += bits * bits * l["macs"]
         size_bits += bits * l["params"]
     return dict(macs=macs, params=params, bops=bops, weight_bytes=size_bits // 8)
+
+
+def synthetic_sensitivity(table: dict, seed: int) -> np.ndarray:
+    """Synthetic stand-in for the Hessian-based perturbation Omega_i^(b) of Section 3.4, [units, 2] int64 for
+    b = 4 and 8.  There are no trained weights here, so the average Hessian trace of a layer is drawn
+    log-normally around a value that falls by three decades from the first block to the last (early layers
+    are the sensitive ones in the paper's figures), and the squared quantization error of a layer is taken as
+    params * 4^-b (uniform quantization noise).  Only the ILP's input, never part of the integer pipeline.
+    """
+    units = len(table["conv_bits"])
+    g = rng(seed, 31, units)
+    params = np.zeros(units)
+    for l in table["layers"]:
+        if l["op"] == "conv" and l.get("unit", -1) >= 0:
+            params[l["unit"]] += l["params"]
+    trace = 10.0 ** (3.0 - 3.0 * np.arange(units) / max(units - 1, 1)) * np.exp(g.normal(0.0, 0.5, size=units))
+    om = np.stack([trace * params * 4.0 ** -4, trace * params * 4.0 ** -8], axis=1)
+    return np.maximum(np.rint(om / om.max() * 2.0 ** 36), 1).astype(np.int64)
 
 
 def random_images(seed: int, n: int, hw: int = 224) -> np.ndarray:

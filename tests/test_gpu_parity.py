@@ -647,6 +647,24 @@ def test_reduced_resnet18_and_resnet50_every_layer(hq):
         run_network_and_compare(hq, t, batch=3, seed=depth)
 
 
+@pytest.mark.parametrize("depth,pattern", [(18, "alternate"), (18, "random"), (50, "alternate"), (50, "random"),
+                                           (50, "all4")])
+def test_network_per_conv_bit_widths(hq, depth, pattern):
+    """Bit-width tables as the ILP of Section 3.4 emits them: 4 or 8 bit chosen per block conv, so that 8-bit convs
+    write 4-bit outputs for a 4-bit successor and the other way round, blocks requantize their input only when
+    their first conv is 4-bit, and a shortcut conv follows the block's first conv.  Every layer bit for bit."""
+    units = inputs.resnet_choice_units(depth)
+    g = inputs.rng(21, depth, len(pattern))
+    if pattern == "alternate":
+        bits = [8 if i % 2 == 0 else 4 for i in range(units)]
+    elif pattern == "random":
+        bits = [int(b) for b in g.choice([4, 8], size=units)]
+    else:
+        bits = [4] * units
+    t = inputs.resnet_table(depth, seed=6, image_hw=64, classes=24, width=32, conv_bits=bits)
+    run_network_and_compare(hq, t, batch=3, seed=depth + 1)
+
+
 def test_network_residual_shifts_per_channel(hq):
     """Fused residual adds inside a network with a different dyadic pair on every channel: shifts from 9 to
     45 (terms that vanish, terms with and without a narrow 32-bit form), unsigned and signed residual
