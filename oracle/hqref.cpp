@@ -295,6 +295,34 @@ int32_t hqref_maxpool(const void* in, int32_t n, int32_t h, int32_t w, int32_t c
   return HQREF_OK;
 }
 
+// One branch of an Inception-style concatenation (Appendix E, "Concatenation Layer"): every branch
+// is brought to the output scale by its own dyadic pairs, q_a[.., off + k] = DN(S_i / S_a) q_i[.., k],
+// and lands beside the others along the channel axis; the convolution branches arrive as stored
+// 8-bit (or 4-bit) tensors or as wide accumulators, the pooling branch as a wide (INT32) tensor.
+// `out` is the [pixels][out_ch] concatenated tensor, `ch_off` the branch's first channel in it.
+int32_t hqref_concat_branch(const void* in, int32_t in_bits, int32_t in_signed,
+                            const int32_t* b, const int32_t* c, int64_t pixels, int32_t ch,
+                            int32_t relu, int32_t qmin, int32_t qmax,
+                            void* out, int32_t out_bits, int32_t out_signed, int32_t out_ch, int32_t ch_off) {
+  if (!in || !out || pixels < 0 || ch < 1 || ch_off < 0 || out_ch < ch_off + ch) return HQREF_ERR_INVALID_ARG;
+  if (!bits_ok(in_bits, true) || !bits_ok(out_bits, false)) return HQREF_ERR_INVALID_ARG;
+  if (in_bits == 4 && (ch & 1)) return HQREF_ERR_INVALID_ARG;
+  if (out_bits == 4 && (out_ch & 1)) return HQREF_ERR_INVALID_ARG;
+  if (!dyadic_ok(b, c, ch)) return HQREF_ERR_INVALID_ARG;
+  if (!fits_type(qmin, qmax, out_bits, out_signed)) return HQREF_ERR_INVALID_ARG;
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < pixels; ++p) {
+    for (int32_t k = 0; k < ch; ++k) {
+      int64_t y = hqref_dn((int32_t)load_elem(in, p * ch + k, in_bits, in_signed), b[k], c[k]);
+      if (relu && y < 0) y = 0;
+      if (y < qmin) y = qmin;
+      if (y > qmax) y = qmax;
+      store_elem(out, p * out_ch + ch_off + k, out_bits, out_signed, y);
+    }
+  }
+  return HQREF_OK;
+}
+
 int32_t hqref_num_threads(void) {
   int32_t t = 1;
 #ifdef _OPENMP

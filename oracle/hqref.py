@@ -43,6 +43,8 @@ def lib():
         L.hqref_avgpool_requant.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, vp, i32, i32]
         L.hqref_maxpool.restype = i32
         L.hqref_maxpool.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+        L.hqref_concat_branch.restype = i32
+        L.hqref_concat_branch.argtypes = [vp, i32, i32, vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, i32, i32]
         L.hqref_num_threads.restype = i32
         _lib = L
     return _lib
@@ -144,6 +146,24 @@ def avgpool_requant(x, ch, in_bits, in_signed, b, c, qmin, qmax, out_bits=8, out
     b, c = _i32(b), _i32(c)
     _check(lib().hqref_avgpool_requant(_p(x), n, h, w, ch, in_bits, in_signed, _p(b), _p(c), qmin, qmax,
                                        _p(out), out_bits, out_signed))
+    return out
+
+
+def concat_requant(branches, relu, qmin, qmax, out_bits=8, out_signed=0):
+    """Inception concatenation (Appendix E): `branches` is a list of dicts {x, bits, signed, ch, b, c};
+    every branch is rescaled by its own dyadic pairs and written at its channel offset."""
+    first = np.ascontiguousarray(branches[0]["x"])
+    n, h, w = first.shape[:3]
+    pixels = n * h * w
+    out_ch = sum(int(br["ch"]) for br in branches)
+    out = _out_array((n, h, w, out_ch), out_bits, out_signed)
+    off = 0
+    for br in branches:
+        x = np.ascontiguousarray(br["x"])
+        b, c = _i32(br["b"]), _i32(br["c"])
+        _check(lib().hqref_concat_branch(_p(x), br["bits"], br["signed"], _p(b), _p(c), pixels, br["ch"],
+                                         relu, qmin, qmax, _p(out), out_bits, out_signed, out_ch, off))
+        off += int(br["ch"])
     return out
 
 

@@ -319,6 +319,59 @@ def test_residual_add_elementwise_vs_exact():
     assert np.array_equal(y.astype(np.int64), ref)
 
 
+# ---------------------------------------------------------------- concat (Appendix E) -----------
+def _concat_branches(g):
+    n, h, w = 2, 3, 5
+    specs = [(6, 8, 0), (4, 32, 1), (10, 8, 1), (2, 32, 1)]      # (channels, bits, signed)
+    branches = []
+    for ch, bits, signed in specs:
+        if bits == 32:
+            x = g.integers(-(1 << 20), 1 << 20, size=(n, h, w, ch)).astype(np.int32)
+            c = g.integers(40, 46, size=ch).astype(np.int32)
+        else:
+            x = g.integers(-128 if signed else 0, 128 if signed else 256, size=(n, h, w, ch)).astype(np.int8 if signed else np.uint8)
+            c = g.integers(29, 33, size=ch).astype(np.int32)
+        b = g.integers(1 << 30, 1 << 31, size=ch).astype(np.int32)
+        branches.append({"x": x, "bits": bits, "signed": signed, "ch": ch, "b": b, "c": c})
+    return branches
+
+
+def test_concat_places_every_branch_at_its_offset_with_exact_rounding():
+    """Each output channel range holds clamp(floor(q*b/2^c + 1/2)) of its own branch, in exact rationals."""
+    branches = _concat_branches(np.random.default_rng(21))
+    y = hqref.concat_requant(branches, 0, -128, 127, 8, 1).astype(np.int64)
+    off = 0
+    for br in branches:
+        x = br["x"].astype(np.int64)
+        for k in range(br["ch"]):
+            want = np.array([min(max(exact_round_half_up(int(q) * int(br["b"][k]), int(br["c"][k])), -128), 127)
+                             for q in x[..., k].ravel()]).reshape(x.shape[:3])
+            assert np.array_equal(y[..., off + k], want)
+        off += br["ch"]
+    assert off == y.shape[-1]
+
+
+def test_concat_with_unit_scales_is_numpy_concatenate_and_relu_clamps():
+    g = np.random.default_rng(22)
+    xs = [g.integers(-100, 100, size=(1, 4, 4, ch)).astype(np.int8) for ch in (2, 6, 4)]
+    branches = [{"x": x, "bits": 8, "signed": 1, "ch": x.shape[-1], "b": np.full(x.shape[-1], 1 << 30, np.int32),
+                 "c": np.full(x.shape[-1], 30, np.int32)} for x in xs]
+    cat = np.concatenate(xs, axis=-1)
+    assert np.array_equal(hqref.concat_requant(branches, 0, -128, 127, 8, 1), cat)
+    assert np.array_equal(hqref.concat_requant(branches, 1, 0, 15, 8, 0), np.clip(cat, 0, 15).astype(np.uint8))
+    packed = hqref.concat_requant(branches, 1, 0, 15, 4, 0)                  # 4-bit output: same values, two per byte
+    assert np.array_equal(inputs.unpack4(packed, False), np.clip(cat, 0, 15).astype(np.uint8))
+
+
+def test_concat_of_one_branch_is_the_plain_requantization():
+    g = np.random.default_rng(23)
+    x = g.integers(-(1 << 21), 1 << 21, size=(2, 2, 3, 8)).astype(np.int32)
+    b = g.integers(1 << 30, 1 << 31, size=8).astype(np.int32)
+    c = g.integers(42, 48, size=8).astype(np.int32)
+    one = hqref.concat_requant([{"x": x, "bits": 32, "signed": 1, "ch": 8, "b": b, "c": c}], 1, 0, 255, 8, 0)
+    assert np.array_equal(one, hqref.residual_add(x, 32, 1, b, c, None, 0, 0, None, None, 8, 1, 0, 255, 8, 0))
+
+
 # ---------------------------------------------------------------- P9: topology ------------------
 def test_table_cost_matches_the_papers_table1(golden_dir):
     want = {}
