@@ -254,6 +254,22 @@ def run_membound(args):
     ba, ca = dy(2048, 36, 38)
     cases.append(("avgpool requant u8 [%d,7,7,2048]" % na, xa.numel() + oa.numel(),
                   lambda: hq.avgpool_requant(xa, 2048, 8, 0, ba, ca, 0, 255, oa, 8, 0)))
+    # Inception concatenation (Appendix E) at the 35x35 module's sizes: three 8-bit convolution branches and the
+    # pooling branch in INT32, one dyadic pair per channel, 288 output channels
+    cat = [{"x": u8(n, 35, 35, c), "bits": 8, "signed": 0, "ch": c} for c in (64, 64, 96)]
+    cat.append({"x": ri(-(1 << 20), 1 << 20, (n, 35, 35, 64), torch.int32), "bits": 32, "signed": 1, "ch": 64})
+    for br in cat:
+        br["b"], br["c"] = dy(br["ch"], 44, 48) if br["bits"] == 32 else dy(br["ch"], 30, 33)
+    ocat = torch.empty((n, 35, 35, 288), dtype=torch.uint8, device="cuda")
+    cases.append(("concat 3x u8 + s32 -> u8 [%d,35,35,288]" % n,
+                  sum(br["x"].numel() * br["x"].element_size() for br in cat) + ocat.numel(),
+                  lambda: hq.concat_requant(cat, 1, 0, 255, ocat, 8, 0)))
+    cat17 = [{"x": u8(4 * n, 17, 17, 192), "bits": 8, "signed": 0, "ch": 192} for _ in range(4)]
+    for br in cat17:
+        br["b"], br["c"] = dy(192, 34, 37)
+    ocat17 = torch.empty((4 * n, 17, 17, 768), dtype=torch.uint8, device="cuda")
+    cases.append(("concat 4x u8 -> u8 [%d,17,17,768]" % (4 * n), 2 * ocat17.numel(),
+                  lambda: hq.concat_requant(cat17, 1, 0, 255, ocat17, 8, 0)))
     rows = []
     for name, byt, fn in cases:
         times = []

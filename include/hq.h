@@ -139,6 +139,22 @@ hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic main_
 hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic rescale,
                              int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
 
+/*
+ * Concatenation along the channel axis with a dyadic rescale per branch (Appendix E, "Concatenation
+ * Layer": the outputs of an Inception module's branches are "scaled and requantized before being
+ * concatenated", one DN operator per branch):
+ *   out[n,h,w, off_i + k] = clamp(relu?(dn(branch_i[n,h,w,k], b_i[k], c_i[k]))),  off_i = c_0 + ... + c_{i-1}.
+ * `branches` and `rescale` are HOST arrays of n_branches entries (1 <= n_branches <=
+ * HQ_CONCAT_MAX_BRANCHES); each tensor's data and each pair's b / c arrays (length = that branch's
+ * channel count) are DEVICE pointers, caller-owned.  Branch bits: 4, 8 or 32 (the paper keeps the
+ * pooling branch in INT32); all branches share out's n, h, w and their channel counts sum to out->c.
+ * out: bits 8, or 4 when every branch has an even channel count (else HQ_ERR_UNSUPPORTED).  One launch,
+ * asynchronous on `stream`; every operand is read once and the output written once.
+ */
+#define HQ_CONCAT_MAX_BRANCHES 8
+hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const hq_tensor* branches, const hq_dyadic* rescale,
+                            int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
+
 /* k x k max pooling of an 8-bit tensor; window taps outside the image are ignored (ResNet stem;
  * an integer max commutes with the monotone requantization of Eq. 4).  pad < k. */
 hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,

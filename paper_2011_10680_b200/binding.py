@@ -22,7 +22,7 @@ EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
     "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
-    "hq_ilp_solve",
+    "hq_ilp_solve", "hq_concat_requant",
 ]
 
 
@@ -75,6 +75,7 @@ def lib():
         L.hq_residual_add.argtypes = [vp, TP, hq_dyadic, TP, hq_dyadic, i32, i32, i32, TP, vp]
         L.hq_avgpool_requant.argtypes = [vp, TP, hq_dyadic, i32, i32, TP, vp]
         L.hq_maxpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
+        L.hq_concat_requant.argtypes = [vp, i32, TP, C.POINTER(hq_dyadic), i32, i32, i32, TP, vp]
         L.hq_network_create.argtypes = [vp, LP, i32, i32, i32, i32, i32, i32, C.POINTER(vp)]
         L.hq_run_network.argtypes = [vp, TP, TP, C.POINTER(vp), vp]
         L.hq_conv2d_noalloc.argtypes = [TP, DP, TP, vp]
@@ -202,6 +203,14 @@ class Handle:
         ti = tensor_of(x, ch, in_bits, in_signed)
         to = tensor_of(out, ch, out_bits, out_signed)
         return lib().hq_avgpool_requant(self._h, C.byref(ti), _dy(b, c), qmin, qmax, C.byref(to), _stream())
+
+    def concat_requant(self, branches, relu, qmin, qmax, out, out_bits, out_signed):
+        """`branches`: list of dicts {x, bits, signed, ch, b, c} of CUDA tensors; `out`: (n, h, w, sum ch)."""
+        n = len(branches)
+        ts = (hq_tensor * n)(*[tensor_of(br["x"], br["ch"], br["bits"], br["signed"]) for br in branches])
+        ds = (hq_dyadic * n)(*[_dy(br["b"], br["c"]) for br in branches])
+        to = tensor_of(out, out.shape[3] * (2 if out_bits == 4 else 1), out_bits, out_signed)
+        return lib().hq_concat_requant(self._h, n, ts, ds, relu, qmin, qmax, C.byref(to), _stream())
 
     def maxpool(self, x, ch, signed, k, stride, pad, out):
         ti = tensor_of(x, ch, 8, signed)

@@ -356,6 +356,33 @@ def synthetic_sensitivity(table: dict, seed: int) -> np.ndarray:
     return np.maximum(np.rint(om / om.max() * 2.0 ** 36), 1).astype(np.int64)
 
 
+def concat_case(seed: int, n: int, hw: int, branches, out_bits: int = 8, out_signed: int = 0, relu: int = 1) -> dict:
+    """Inputs of one Inception-style concatenation (Appendix E): `branches` lists (channels, bits, signed) per
+    branch, e.g. the 35x35 module of InceptionV3: three convolution branches (stored 8-bit tensors) and the pooling
+    branch kept in INT32.  Values: 8-/4-bit tensors uniform over their type's range, INT32 tensors uniform in
+    [-2^22, 2^22); per-channel pairs DN(S_i / S_a) with log-uniform scale ratios chosen so that outputs use the
+    output range (8-bit: ratio in [2^-1, 2); 32-bit: ratio in [2^-16, 2^-14))."""
+    g = rng(seed, 77, n, hw)
+    out = []
+    for ch, bits, signed in branches:
+        if bits == 32:
+            x = g.integers(-(1 << 22), 1 << 22, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+            ratio = np.exp2(g.uniform(-16.0, -14.0, size=ch))
+        elif bits == 8:
+            x = g.integers(-128 if signed else 0, 128 if signed else 256, size=(n, hw, hw, ch), dtype=np.int64)
+            x = x.astype(np.int8 if signed else np.uint8)
+            ratio = np.exp2(g.uniform(-1.0, 1.0, size=ch)) * (1.0 if out_bits == 8 else 1.0 / 16)
+        else:
+            x = pack4(g.integers(-8 if signed else 0, 8 if signed else 16, size=(n, hw, hw, ch), dtype=np.int64))
+            ratio = np.exp2(g.uniform(-1.0, 1.0, size=ch)) * (16.0 if out_bits == 8 else 1.0)
+        b, c = dyadic_from_scale(ratio)
+        out.append({"x": x, "bits": bits, "signed": signed, "ch": ch, "b": b, "c": c})
+    lo = -(1 << (out_bits - 1)) if out_signed else 0
+    hi = (1 << (out_bits - 1)) - 1 if out_signed else (1 << out_bits) - 1
+    return {"branches": out, "relu": relu, "qmin": lo, "qmax": hi, "out_bits": out_bits, "out_signed": out_signed,
+            "n": n, "hw": hw, "out_ch": sum(b[0] for b in branches)}
+
+
 def random_images(seed: int, n: int, hw: int = 224) -> np.ndarray:
     """uint8 images uniform in [0, 255], NHWC with 3 channels."""
     return rng(seed, 99, n, hw).integers(0, 256, size=(n, hw, hw, 3), dtype=np.int64).astype(np.uint8)

@@ -1,0 +1,120 @@
+"""Parity of hq_concat_requant (Inception concatenation, Appendix E) with the CPU oracle: bit-exact, through the C ABI."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_2011_10680_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hq():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    h = binding.Handle(0)
+    yield h
+    h.close()
+
+
+def run_and_compare(hq, case):
+    from oracle import hqref
+    from paper_2011_10680_b200 import binding
+    dev = [{**br, "x": binding.to_device(br["x"]), "b": binding.to_device(br["b"]), "c": binding.to_device(br["c"])}
+           for br in case["branches"]]
+    out = binding.alloc_out(case["n"], case["hw"], case["hw"], case["out_ch"], case["out_bits"], case["out_signed"])
+    out.fill_(0x5A)                                             # stale bytes must all be overwritten
+    st = hq.concat_requant(dev, case["relu"], case["qmin"], case["qmax"], out, case["out_bits"], case["out_signed"])
+    assert st == binding.HQ_OK, binding.status_string(st)
+    hq.sync()
+    ref = hqref.concat_requant(case["branches"], case["relu"], case["qmin"], case["qmax"], case["out_bits"], case["out_signed"])
+    got = out.cpu().numpy().view(ref.dtype).reshape(ref.shape)
+    if not np.array_equal(got, ref):
+        bad = np.argwhere(got != ref)
+        raise AssertionError(f"{len(bad)} of {ref.size} stored values differ; first at {bad[0]}: got {got[tuple(bad[0])]} want {ref[tuple(bad[0])]}")
+    return ref
+
+
+# (channels, bits, signed) per branch
+INCEPTION_A = [(64, 8, 0), (64, 8, 0), (96, 8, 0), (32, 32, 1)]            # 35x35 module: 1x1, 5x5, double 3x3, pool (INT32)
+INCEPTION_C = [(192, 8, 0), (192, 8, 0), (192, 8, 0), (192, 32, 1)]        # 17x17 module
+RAGGED = [(6, 8, 1), (20, 32, 1), (10, 4, 0), (48, 8, 0), (2, 32, 1), (16, 4, 1)]   # odd group sizes, unaligned offsets
+
+
+@pytest.mark.parametrize("branches,n,hw", [(INCEPTION_A, 3, 35), (INCEPTION_C, 2, 17), (RAGGED, 2, 9)])
+@pytest.mark.parametrize("out_bits,out_signed,relu", [(8, 0, 1), (8, 1, 0), (4, 0, 1)])
+def test_concat_matches_the_oracle(hq, branches, n, hw, out_bits, out_signed, relu):
+    case = inputs.concat_case(401, n, hw, branches, out_bits, out_signed, relu)
+    ref = run_and_compare(hq, case)
+    if branches is INCEPTION_A and out_bits == 8:
+        # the draw must exercise the arithmetic: not everything saturated
+        inner = np.count_nonzero((ref > case["qmin"]) & (ref < case["qmax"]))
+        assert inner > ref.size // 4
+
+
+def test_concat_every_shift_and_extreme_operands(hq):
+    """Shifts 1..62 across the channels (both forms of the arithmetic), full-range INT32 and 8-bit operands."""
+    g = inputs.rng(402)
+    n, hw = 1, 12
+    branches = []
+    for ch, bits, signed in [(64, 32, 1), (62, 8, 1), (64, 8, 0)]:
+        if bits == 32:
+            x = g.integers(-(1 << 31), 1 << 31, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+            x[0, 0, :4] = [[-(1 << 31)] * ch, [(1 << 31) - 1] * ch, [0] * ch, [-1] * ch]
+        else:
+            x = g.integers(-128 if signed else 0, 128 if signed else 256, size=(n, hw, hw, ch), dtype=np.int64)
+            x = x.astype(np.int8 if signed else np.uint8)
+        b = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+        b[:3] = [(1 << 31) - 1, 1 << 30, 0]
+        c = ((np.arange(ch) * 5) % 62 + 1).astype(np.int32)
+        branches.append({"x": x, "bits": bits, "signed": signed, "ch": ch, "b": b, "c": c})
+    for out_signed, relu in ((1, 0), (0, 1)):
+        lo, hi = (-128, 127) if out_signed else (0, 255)
+        case = {"branches": branches, "relu": relu, "qmin": lo, "qmax": hi, "out_bits": 8, "out_signed": out_signed,
+                "n": n, "hw": hw, "out_ch": 190}
+        run_and_compare(hq, case)
+
+
+def test_concat_single_branch_equals_residual_add_and_rejects_bad_arguments(hq):
+    from paper_2011_10680_b200 import binding
+    case = inputs.concat_case(403, 2, 8, [(32, 32, 1)])
+    ref = run_and_compare(hq, case)
+    br = case["branches"][0]
+    x, b, c = (binding.to_device(br[k]) for k in ("x", "b", "c"))
+    out = binding.alloc_out(2, 8, 8, 32, 8, 0)
+    st = hq.residual_add(x, 32, 1, b, c, None, 0, 0, None, None, 32, 1, 0, 255, out, 8, 0)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(out.cpu().numpy(), ref)
+    dev = [{**br, "x": x, "b": b, "c": c}]
+    # channel counts must sum to the output's; 4-bit outputs need even branches; at most eight branches
+    wrong = binding.alloc_out(2, 8, 8, 48, 8, 0)
+    assert hq.concat_requant(dev, 1, 0, 255, wrong, 8, 0) == binding.HQ_ERR_INVALID_ARG
+    assert hq.concat_requant(dev * 9, 1, 0, 255, out, 8, 0) == binding.HQ_ERR_INVALID_ARG
+    assert hq.concat_requant(dev, 1, 0, 300, out, 8, 0) == binding.HQ_ERR_INVALID_ARG
+    odd = inputs.concat_case(404, 1, 4, [(5, 8, 0), (3, 8, 0)])
+    odd_dev = [{**o, "x": binding.to_device(o["x"]), "b": binding.to_device(o["b"]), "c": binding.to_device(o["c"])}
+               for o in odd["branches"]]
+    out4 = binding.alloc_out(1, 4, 4, 8, 4, 0)
+    assert hq.concat_requant(odd_dev, 1, 0, 15, out4, 4, 0) == binding.HQ_ERR_UNSUPPORTED
+
+
+def test_concat_empty_batch_is_a_no_op(hq):
+    from paper_2011_10680_b200 import binding
+    x = torch.empty((0, 5, 5, 16), dtype=torch.uint8, device="cuda")
+    keep = torch.zeros(16, dtype=torch.uint8, device="cuda")        # a valid pointer for the empty tensors
+    b = binding.to_device(np.full(16, 1 << 30, np.int32))
+    c = binding.to_device(np.full(16, 30, np.int32))
+    tin = binding.hq_tensor(keep.data_ptr(), 0, 5, 5, 16, 8, 0)
+    tout = binding.hq_tensor(keep.data_ptr(), 0, 5, 5, 16, 8, 0)
+    import ctypes as C
+    ts = (binding.hq_tensor * 1)(tin)
+    ds = (binding.hq_dyadic * 1)(binding.hq_dyadic(b.data_ptr(), c.data_ptr()))
+    st = binding.lib().hq_concat_requant(hq._h, 1, ts, ds, 1, 0, 255, C.byref(tout), None)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert x.numel() == 0 and int(keep.sum()) == 0
