@@ -3,10 +3,12 @@
 // i.e. every branch (the convolution branches as stored 8- or 4-bit tensors or INT32 accumulators, the pooling
 // branch as an INT32 tensor) is brought to the output scale by its own DN pairs and lands beside the others along
 // the channel axis.  Memory bound: every operand is read once, the output written once, in ONE launch for all
-// branches.  A thread owns 16 consecutive channels of one branch at one pixel: a 16-byte (8-bit input), 64-byte
-// (INT32 input) or 8-byte (4-bit input) read, sixteen exact requantizations, one 16-byte (or 8-byte, 4-bit
-// output) write; neighbouring threads take neighbouring channel groups of the same output pixel, so the writes of
-// a warp cover contiguous bytes of the concatenated row.  Integer arithmetic only.
+// branches.  The blocks of the launch are dealt to the branches in proportion to their bytes, so a warp works on one
+// branch only (one operand type, one form of the arithmetic, no divergence).  A thread owns one 16-byte piece of a
+// branch's pixel row for the whole kernel -- 16 channels of an 8-bit branch (32 of a 4-bit one are two threads), 4
+// channels of an INT32 branch -- reads its dyadic pairs once, and keeps four pixels in flight; neighbouring lanes
+// read neighbouring 16-byte pieces of the dense branch tensor and write neighbouring pieces of the output row.
+// Integer arithmetic only.
 #include "hq_internal.cuh"
 
 namespace {
@@ -14,115 +16,235 @@ namespace {
 struct ConcatBranch {
   const void* in; const int32_t* b; const int32_t* c;
   int32_t bits, is_signed, ch, ch_off;
-  int32_t unit0;      // index of this branch's first 16-channel group among a pixel's groups
-  int32_t vec;        // 1: rows and dyadic arrays allow 16-byte accesses (ch % 16 == 0, aligned arrays)
+  int32_t width;      // channels a thread owns: 16, or 4 for an INT32 branch read in 16-byte pieces
+  int32_t upp;        // threads (units) per pixel of this branch = ceil(ch / width)
+  int32_t block0, nblocks;   // this branch's blocks of the launch
+  int32_t vec;        // 1: rows and dyadic arrays allow 16-byte reads (ch % 16 == 0 resp. ch % 4 == 0, aligned arrays)
 };
 
 struct ConcatArgs {
   ConcatBranch br[HQ_CONCAT_MAX_BRANCHES];
-  int32_t n_br, units_per_px, out_ch, out_bits, relu, qmin, qmax;
+  int32_t n_br, out_ch, out_bits, relu, qmin, qmax;
   long long pixels;
   void* out;
+  const int4* narrow;   // per OUTPUT channel {m, a, s, valid} from concat_narrow_kernel (8-/4-bit branches), or NULL
+  int32_t sat;          // 1: relu and the clamp bounds equal a saturating conversion to the 8-bit output type
 };
 
-// One value: the 64-bit definition, or for c >= 33 its high-word form (the rounding constant 2^(c-1) is then a
-// multiple of 2^32, so it adds to the high word of q*b without a carry from the low word).
-__device__ __forceinline__ int concat_dn(int q, int b, int c, int relu, int qmin, int qmax) {
-  if (c >= 33) {
-    int y = (__mulhi(q, b) + (1 << (c - 33))) >> (c - 32);      // |q*b| < 2^62: the sum stays inside INT32
-    if (relu) y = max(y, 0);
-    return min(max(y, qmin), qmax);
+// Narrow multiply-add pairs for the 8- and 4-bit branches.  A stored 8-bit value r has 256 possible values, so
+// dn(r, b, c) can often be written (r*m + a) >> s in 32-bit arithmetic, m ~ b / 2^8: one warp per output channel
+// tries the two neighbouring multipliers against the 64-bit definition for every r and records the one that agrees
+// everywhere (valid = 1), else valid = 0 and the channel keeps the wide form.  c >= 41 makes the term 0 for every r.
+__global__ void __launch_bounds__(128) concat_narrow_kernel(const __grid_constant__ ConcatArgs a, int4* out) {
+  const int oc = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (oc >= a.out_ch) return;
+  int i = 0;
+#pragma unroll
+  for (int j = 1; j < HQ_CONCAT_MAX_BRANCHES; ++j)
+    if (j < a.n_br && oc >= a.br[j].ch_off) i = j;
+  int4 res = make_int4(0, 0, 0, 0);
+  if (a.br[i].bits != 32) {
+    const int k = oc - a.br[i].ch_off;
+    const long long b = a.br[i].b[k];
+    const int c = a.br[i].c[k];
+    const int r_lo = a.br[i].is_signed ? -128 : 0;
+    if (c >= 41) {
+      res = make_int4(0, 0, 0, 1);                     // |r*b| < 2^39 <= 2^(c-2)
+    } else if (c >= 9 && c <= 38) {
+      const int s = c - 8, add = 1 << (s - 1);
+      const long long m0 = b >> 8, m1 = m0 + 1;
+      bool ok0 = m0 <= (1 << 23), ok1 = m1 <= (1 << 23);
+      for (int t = 0; t < 8; ++t) {
+        const int r = r_lo + lane + 32 * t;
+        const long long exact = hq_dn(r, (int)b, c);
+        ok0 = ok0 && exact == (long long)((r * (int)m0 + add) >> s);
+        ok1 = ok1 && exact == (long long)((r * (int)m1 + add) >> s);
+      }
+      ok0 = __all_sync(0xffffffffu, ok0);
+      ok1 = __all_sync(0xffffffffu, ok1);
+      if (ok0) res = make_int4((int)m0, add, s, 1);
+      else if (ok1) res = make_int4((int)m1, add, s, 1);
+    }
   }
-  return hq_clamp_ll(hq_dn(q, b, c), relu, qmin, qmax);
+  if (lane == 0) out[oc] = res;
 }
 
-__global__ void __launch_bounds__(256) concat_requant_kernel(const __grid_constant__ ConcatArgs a) {
-  const long long total = a.pixels * (long long)a.units_per_px;
-  for (long long t = (long long)blockIdx.x * 256 + threadIdx.x; t < total; t += (long long)gridDim.x * 256) {
-    const long long px = t / a.units_per_px;
-    const int u = (int)(t - px * a.units_per_px);
-    int i = 0;
+// Four values clamped to the unsigned / signed 8-bit range and packed, first value in the low byte.
+__device__ __forceinline__ unsigned pack4_sat(int v0, int v1, int v2, int v3, bool is_signed) {
+  unsigned hi2, w;
+  if (is_signed) {
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi2) : "r"(v3), "r"(v2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v1), "r"(v0), "r"(hi2));
+  } else {
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(hi2) : "r"(v3), "r"(v2), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v1), "r"(v0), "r"(hi2));
+  }
+  return w;
+}
+
+// One value by the 64-bit definition.
+__device__ __forceinline__ int concat_dn64(int q, int b, int c, int lo, int hi) {
+  long long y = hq_dn(q, b, c);
+  if (y < (long long)lo) y = lo;
+  if (y > (long long)hi) y = hi;
+  return (int)y;
+}
+
+constexpr int kPix = 4;      // pixels (16-byte reads) a thread keeps in flight
+
+// Store `n` (<= 16) clamped values of one thread: 8-bit bytes or 4-bit nibbles (low nibble first), widest aligned form.
+template <int N>
+__device__ __forceinline__ void concat_store(const ConcatArgs& a, int (&o)[N], int n, long long o0, int lo, int hi) {
+  if (a.out_bits == 8) {
+    unsigned char* op = (unsigned char*)a.out + o0;
+    const bool whole = n == N && (o0 & (N - 1)) == 0;
+    if (whole) {
+      unsigned w[N / 4];
+      if (a.sat) {
 #pragma unroll
-    for (int j = 1; j < HQ_CONCAT_MAX_BRANCHES; ++j)
-      if (j < a.n_br && u >= a.br[j].unit0) i = j;
-    const ConcatBranch& B = a.br[i];
-    const int k0 = (u - B.unit0) * 16;
-    const int nk = min(16, B.ch - k0);
-    const long long e0 = px * (long long)B.ch + k0;              // first input element of this thread
-    int q[16], bb[16], cc[16];
-    if (B.vec) {
-      const int4* bp = (const int4*)(B.b + k0);
-      const int4* cp = (const int4*)(B.c + k0);
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const int4 x = __ldg(bp + v), y = __ldg(cp + v);
-        bb[4 * v] = x.x; bb[4 * v + 1] = x.y; bb[4 * v + 2] = x.z; bb[4 * v + 3] = x.w;
-        cc[4 * v] = y.x; cc[4 * v + 1] = y.y; cc[4 * v + 2] = y.z; cc[4 * v + 3] = y.w;
-      }
-      if (B.bits == 8) {
-        const uint4 x = *(const uint4*)((const unsigned char*)B.in + e0);
-        const unsigned w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const unsigned byte = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-          q[j] = B.is_signed ? (int)(signed char)byte : (int)byte;
-        }
-      } else if (B.bits == 32) {
-        const int4* ip = (const int4*)((const int*)B.in + e0);
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const int4 x = ip[v];
-          q[4 * v] = x.x; q[4 * v + 1] = x.y; q[4 * v + 2] = x.z; q[4 * v + 3] = x.w;
-        }
+        for (int v = 0; v < N / 4; ++v) w[v] = pack4_sat(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3], lo < 0);
       } else {
-        const uint2 x = *(const uint2*)((const unsigned char*)B.in + (e0 >> 1));
-        const unsigned w[2] = {x.x, x.y};
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          int v = (int)((w[j >> 3] >> (4 * (j & 7))) & 0xFu);
-          if (B.is_signed && (v & 8)) v -= 16;
-          q[j] = v;
-        }
-      }
-    } else {
+        for (int j = 0; j < N; ++j) o[j] = min(max(o[j], lo), hi);
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        if (j < nk) { q[j] = hq_load_elem(B.in, e0 + j, B.bits, B.is_signed); bb[j] = B.b[k0 + j]; cc[j] = B.c[k0 + j]; }
-        else { q[j] = 0; bb[j] = 0; cc[j] = 33; }
-      }
-    }
-    int o[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) o[j] = concat_dn(q[j], bb[j], cc[j], a.relu, a.qmin, a.qmax);
-    const long long o0 = px * (long long)a.out_ch + B.ch_off + k0;   // first output element
-    if (a.out_bits == 8) {
-      unsigned char* op = (unsigned char*)a.out + o0;
-      if (nk == 16 && (o0 & 15) == 0) {
-        unsigned w[4];
-#pragma unroll
-        for (int v = 0; v < 4; ++v)
+        for (int v = 0; v < N / 4; ++v)
           w[v] = (unsigned)(o[4 * v] & 0xFF) | ((unsigned)(o[4 * v + 1] & 0xFF) << 8) |
                  ((unsigned)(o[4 * v + 2] & 0xFF) << 16) | ((unsigned)(o[4 * v + 3] & 0xFF) << 24);
-        *(uint4*)op = make_uint4(w[0], w[1], w[2], w[3]);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) if (j < nk) op[j] = (unsigned char)o[j];
       }
+      if (N == 16) *(uint4*)op = make_uint4(w[0], w[N / 4 > 1 ? 1 : 0], w[N / 4 > 2 ? 2 : 0], w[N / 4 > 3 ? 3 : 0]);
+      else *(unsigned*)op = w[0];
     } else {
-      // 4-bit output: channel counts and offsets are even, so a byte's two nibbles belong to this thread
-      unsigned char* op = (unsigned char*)a.out + (o0 >> 1);
-      if (nk == 16 && ((o0 >> 1) & 7) == 0) {
-        unsigned w[2] = {0u, 0u};
 #pragma unroll
-        for (int j = 0; j < 16; ++j) w[j >> 3] |= (unsigned)(o[j] & 0xF) << (4 * (j & 7));
-        *(uint2*)op = make_uint2(w[0], w[1]);
-      } else {
+      for (int j = 0; j < N; ++j) if (j < n) op[j] = (unsigned char)min(max(o[j], lo), hi);
+    }
+  } else {
+    // 4-bit output: channel counts and offsets are even, so a byte's two nibbles belong to this thread
+    unsigned char* op = (unsigned char*)a.out + (o0 >> 1);
 #pragma unroll
-        for (int j = 0; j < 16; j += 2)
-          if (j < nk) op[j >> 1] = (unsigned char)((o[j] & 0xF) | ((o[j + 1] & 0xF) << 4));
-      }
+    for (int j = 0; j < N; ++j) o[j] = min(max(o[j], lo), hi) & 0xF;
+    const bool whole = n == N && (o0 & (N - 1)) == 0;
+    if (whole) {
+      unsigned w[N / 8 > 0 ? N / 8 : 1] = {};
+#pragma unroll
+      for (int j = 0; j < N; ++j) w[j >> 3] |= (unsigned)o[j] << (4 * (j & 7));
+      if (N == 16) *(uint2*)op = make_uint2(w[0], w[N / 8 > 1 ? 1 : 0]);
+      else *(unsigned short*)op = (unsigned short)w[0];
+    } else {
+#pragma unroll
+      for (int j = 0; j < N; j += 2)
+        if (j < n) op[j >> 1] = (unsigned char)(o[j] | (o[j + 1] << 4));
     }
   }
+}
+
+// One branch's share of the blocks.  N = channels per thread (16: 8-/4-bit branches and ragged INT32 ones; 4: INT32
+// branches read in 16-byte pieces).  Thread t of the block's first upp * ppb threads owns unit t % upp of pixel
+// t / upp of every block step, i.e. consecutive lanes walk consecutive 16-byte pieces of the dense branch tensor.
+template <int N>
+__device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) {
+  const void* const in = a.br[i].in;
+  const int bits = a.br[i].bits, is_signed = a.br[i].is_signed, ch = a.br[i].ch, vec = a.br[i].vec;
+  const int upp = a.br[i].upp, ppb = 256 / upp;
+  const int tid = threadIdx.x;
+  if (tid >= upp * ppb) return;
+  const int u = tid % upp, y = tid / upp;
+  const int k0 = u * N;
+  const int nk = min(N, ch - k0);
+  const int off = a.br[i].ch_off + k0;
+  const int lo = a.relu ? max(a.qmin, 0) : a.qmin, hi = a.qmax;
+  // Per-channel constants, three forms of y = dn(q, b, c):
+  //   narrow (8-/4-bit operands with a checked pair)   (q*m + a) >> s
+  //   fast   (every c of the thread >= 33)             (mulhi(q, b) + 2^(c-33)) >> (c-32): the rounding constant is
+  //          then a multiple of 2^32 and adds to the high word of q*b without a carry; |q*b| < 2^62 keeps it in INT32
+  //   else   the 64-bit definition
+  int bb[N], hh[N], ss[N];
+  bool fast = true;
+#pragma unroll
+  for (int j = 0; j < N; ++j) {
+    const int b = j < nk ? __ldg(a.br[i].b + k0 + j) : 0;
+    const int c = j < nk ? __ldg(a.br[i].c + k0 + j) : 33;
+    bb[j] = b; ss[j] = c; hh[j] = 0;
+    fast = fast && c >= 33;
+  }
+  bool narrow = a.narrow != nullptr && bits != 32 && nk == N;
+  if (narrow) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) narrow = narrow && __ldg(&a.narrow[off + j].w) != 0;
+    if (narrow) {
+#pragma unroll
+      for (int j = 0; j < N; ++j) { const int4 t = __ldg(a.narrow + off + j); bb[j] = t.x; hh[j] = t.y; ss[j] = t.z; }
+    }
+  }
+  if (fast && !narrow) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) { hh[j] = 1 << (ss[j] - 33); ss[j] -= 32; }
+  }
+  const long long step = (long long)a.br[i].nblocks * ppb;
+  const long long first = (long long)(blockIdx.x - a.br[i].block0) * ppb + y;
+  for (long long px0 = first; px0 < a.pixels; px0 += step * kPix) {
+    uint4 raw[kPix];
+    if (vec) {
+#pragma unroll
+      for (int p = 0; p < kPix; ++p) {
+        const long long px = px0 + p * step;
+        if (px < a.pixels) {
+          const long long e0 = px * (long long)ch + k0;
+          if (bits == 4) { const uint2 t = *(const uint2*)((const unsigned char*)in + (e0 >> 1)); raw[p].x = t.x; raw[p].y = t.y; }
+          else raw[p] = *(const uint4*)((const unsigned char*)in + e0 * (bits >> 3));
+        }
+      }
+    }
+#pragma unroll
+    for (int p = 0; p < kPix; ++p) {
+      const long long px = px0 + p * step;
+      if (px >= a.pixels) break;
+      int q[N];
+      if (vec) {
+        const unsigned w[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
+        if (N == 4) {
+#pragma unroll
+          for (int j = 0; j < N; ++j) q[j] = (int)w[j & 3];
+        } else if (bits == 8) {
+#pragma unroll
+          for (int j = 0; j < N; ++j) {
+            const unsigned sh = w[(j >> 2) & 3] >> (8 * (j & 3));
+            q[j] = is_signed ? (int)(signed char)sh : (int)(sh & 0xFFu);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < N; ++j) {
+            const unsigned sh = w[(j >> 3) & 1] >> (4 * (j & 7));
+            q[j] = is_signed ? ((int)(sh << 28) >> 28) : (int)(sh & 0xFu);
+          }
+        }
+      } else {
+        const long long e0 = px * (long long)ch + k0;
+#pragma unroll
+        for (int j = 0; j < N; ++j) q[j] = j < nk ? hq_load_elem(in, e0 + j, bits, is_signed) : 0;
+      }
+      int o[N];
+      if (narrow) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) o[j] = (q[j] * bb[j] + hh[j]) >> ss[j];
+      } else if (fast) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) o[j] = (__mulhi(q[j], bb[j]) + hh[j]) >> ss[j];
+      } else {
+#pragma unroll
+        for (int j = 0; j < N; ++j) o[j] = concat_dn64(q[j], bb[j], ss[j], lo, hi);
+      }
+      concat_store<N>(a, o, nk, px * (long long)a.out_ch + off, lo, hi);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256, 2) concat_requant_kernel(const __grid_constant__ ConcatArgs a) {
+  int i = 0;
+#pragma unroll
+  for (int j = 1; j < HQ_CONCAT_MAX_BRANCHES; ++j)
+    if (j < a.n_br && (int)blockIdx.x >= a.br[j].block0) i = j;
+  if (a.br[i].width == 4) concat_branch<4>(a, i);
+  else concat_branch<16>(a, i);
 }
 
 inline bool al16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
@@ -143,7 +265,8 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     if (qmin > qmax || qmin < lo || qmax > hi) return HQ_ERR_INVALID_ARG;
   }
   ConcatArgs a{};
-  int off = 0, units = 0;
+  int off = 0;
+  long long weight[HQ_CONCAT_MAX_BRANCHES], weight_sum = 0;
   for (int i = 0; i < n_branches; ++i) {
     const hq_tensor& t = branches[i];
     if (!t.data || !rescale[i].b || !rescale[i].c) return HQ_ERR_INVALID_ARG;
@@ -154,21 +277,50 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     if (!al16(t.data)) return HQ_ERR_ALIGNMENT;
     ConcatBranch& B = a.br[i];
     B.in = t.data; B.b = rescale[i].b; B.c = rescale[i].c;
-    B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = t.c; B.ch_off = off; B.unit0 = units;
-    B.vec = (t.c % 16 == 0 && al16(B.b) && al16(B.c)) ? 1 : 0;
+    B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = t.c; B.ch_off = off;
+    if (t.bits == 32 && t.c % 4 == 0 && t.c <= 4 * 256) { B.width = 4; B.vec = 1; }
+    else { B.width = 16; B.vec = (t.bits != 32 && t.c % 16 == 0) ? 1 : 0; }
+    B.upp = (t.c + B.width - 1) / B.width;
+    if (B.upp > 256) return HQ_ERR_UNSUPPORTED;                   // more than 4096 channels in one branch
+    weight[i] = (long long)t.c * (t.bits + out->bits);
+    weight_sum += weight[i];
     off += t.c;
-    units += (t.c + 15) / 16;
   }
   if (off != out->c) return HQ_ERR_INVALID_ARG;
-  a.n_br = n_branches; a.units_per_px = units; a.out_ch = out->c; a.out_bits = out->bits;
+  a.n_br = n_branches; a.out_ch = out->c; a.out_bits = out->bits;
   a.relu = relu; a.qmin = qmin; a.qmax = qmax;
   a.pixels = (long long)out->n * out->h * out->w;
   a.out = out->data;
-  const long long total = a.pixels * units;
-  if (total == 0) return HQ_OK;
-  long long blocks = (total + 255) / 256;
-  const long long cap = (long long)h->sm_count * 16;                // grid-stride beyond eight blocks per SM twice over
-  if (blocks > cap) blocks = cap;
+  if (a.pixels == 0) return HQ_OK;
+  // blocks of the one launch, dealt to the branches in proportion to the bytes they move
+  const long long cap = (long long)h->sm_count * 8;
+  long long blocks = 0;
+  for (int i = 0; i < n_branches; ++i) {
+    ConcatBranch& B = a.br[i];
+    const long long per_block = (long long)(256 / B.upp) * kPix;
+    const long long need = (a.pixels + per_block - 1) / per_block;
+    long long share = (cap * weight[i] + weight_sum - 1) / weight_sum;
+    if (share > need) share = need;
+    if (share < 1) share = 1;
+    B.block0 = (int32_t)blocks; B.nblocks = (int32_t)share;
+    blocks += share;
+  }
+  {
+    const int lo = relu ? (qmin > 0 ? qmin : 0) : qmin;
+    a.sat = (out->bits == 8 && ((!out->is_signed && lo == 0 && qmax == 255) ||
+                                (out->is_signed && lo == -128 && qmax == 127))) ? 1 : 0;
+  }
+  // A large call first works out the narrow pairs of its 8- and 4-bit branches in the handle's buffer (one small
+  // launch on the same stream, repaid by the cheaper arithmetic).
+  a.narrow = nullptr;
+  bool any_narrow = false;
+  for (int i = 0; i < n_branches; ++i) any_narrow = any_narrow || branches[i].bits != 32;
+  if (any_narrow && h->narrow_pairs && out->c <= 2 * kNarrowChannels && a.pixels * out->c >= (1ll << 22)) {
+    int4* tab = (int4*)h->narrow_pairs;
+    concat_narrow_kernel<<<(out->c + 3) / 4, 128, 0, (cudaStream_t)stream>>>(a, tab);
+    if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+    a.narrow = tab;
+  }
   concat_requant_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a);
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }

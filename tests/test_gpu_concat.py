@@ -56,6 +56,30 @@ def test_concat_matches_the_oracle(hq, branches, n, hw, out_bits, out_signed, re
         assert inner > ref.size // 4
 
 
+def test_concat_large_call_with_narrow_pairs(hq):
+    """Above 2^22 outputs the 8- and 4-bit branches run on narrow multiply-add pairs worked out by a first launch;
+    shifts from 9 to 45 across the channels so that channels with and without a pair (and with a zero term) mix."""
+    g = inputs.rng(405)
+    n, hw = 12, 35
+    branches = []
+    for ch, bits, signed in [(64, 8, 0), (64, 8, 1), (96, 4, 0), (64, 32, 1)]:
+        if bits == 32:
+            x = g.integers(-(1 << 22), 1 << 22, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+            c = g.integers(44, 48, size=ch).astype(np.int32)
+        else:
+            lo, hi = ((-128, 128) if signed else (0, 256)) if bits == 8 else ((-8, 8) if signed else (0, 16))
+            x = g.integers(lo, hi, size=(n, hw, hw, ch), dtype=np.int64)
+            x = inputs.pack4(x) if bits == 4 else x.astype(np.int8 if signed else np.uint8)
+            c = (9 + (np.arange(ch) * 3) % 37).astype(np.int32)
+            c[:16] = g.integers(29, 33, size=16)                 # one group of sixteen that surely has pairs
+        b = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+        branches.append({"x": x, "bits": bits, "signed": signed, "ch": ch, "b": b, "c": c})
+    for out_bits, out_signed, relu, lo, hi in ((8, 0, 1, 0, 255), (8, 1, 0, -128, 127), (8, 0, 0, 3, 200), (4, 0, 1, 0, 15)):
+        case = {"branches": branches, "relu": relu, "qmin": lo, "qmax": hi, "out_bits": out_bits, "out_signed": out_signed,
+                "n": n, "hw": hw, "out_ch": 288}
+        run_and_compare(hq, case)
+
+
 def test_concat_every_shift_and_extreme_operands(hq):
     """Shifts 1..62 across the channels (both forms of the arithmetic), full-range INT32 and 8-bit operands."""
     g = inputs.rng(402)
