@@ -194,13 +194,17 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
         }
       }
     }
-#pragma unroll
-    for (int p = 0; p < kPix; ++p) {
+#pragma unroll 1
+    for (int p = 0; p < kPix; ++p) {                 // one copy of the arithmetic: the instruction stream stays small
       const long long px = px0 + p * step;
       if (px >= a.pixels) break;
       int q[N];
       if (vec) {
-        const unsigned w[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
+        uint4 r = raw[0];
+        if (p == 1) r = raw[1];
+        if (p == 2) r = raw[2];
+        if (p == 3) r = raw[3];
+        const unsigned w[4] = {r.x, r.y, r.z, r.w};
         if (N == 4) {
 #pragma unroll
           for (int j = 0; j < N; ++j) q[j] = (int)w[j & 3];
