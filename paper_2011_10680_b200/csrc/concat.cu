@@ -32,7 +32,7 @@ struct ConcatArgs {
 };
 
 // Narrow multiply-add pairs for the 8- and 4-bit branches.  A stored 8-bit value r has 256 possible values, so
-// dn(r, b, c) can often be written (r*m + a) >> s in 32-bit arithmetic, m ~ b / 2^8: one warp per output channel
+// dn(r, b, c) can often be written (r*m + a) >> s in 32-bit arithmetic (on unsigned words for unsigned operands), m ~ b / 2^8: one warp per output channel
 // tries the two neighbouring multipliers against the 64-bit definition for every r and records the one that agrees
 // everywhere (valid = 1), else valid = 0 and the channel keeps the wide form.  c >= 41 makes the term 0 for every r.
 __global__ void __launch_bounds__(128) concat_narrow_kernel(const __grid_constant__ ConcatArgs a, int4* out) {
@@ -54,11 +54,15 @@ __global__ void __launch_bounds__(128) concat_narrow_kernel(const __grid_constan
       const int s = c - 8, add = 1 << (s - 1);
       const long long m0 = b >> 8, m1 = m0 + 1;
       bool ok0 = m0 <= (1 << 23), ok1 = m1 <= (1 << 23);
+      // signed operands: |r*m| <= 2^30 and a <= 2^29 fit INT32; unsigned ones (r*m + a < 2^32) take the same
+      // multiply-add on unsigned words with a logical shift, which the pixel loops mirror
+      const bool uns = r_lo == 0;
       for (int t = 0; t < 8; ++t) {
         const int r = r_lo + lane + 32 * t;
         const long long exact = hq_dn(r, (int)b, c);
-        ok0 = ok0 && exact == (long long)((r * (int)m0 + add) >> s);
-        ok1 = ok1 && exact == (long long)((r * (int)m1 + add) >> s);
+        const unsigned t0 = (unsigned)r * (unsigned)m0 + (unsigned)add, t1 = (unsigned)r * (unsigned)m1 + (unsigned)add;
+        ok0 = ok0 && exact == (uns ? (long long)(t0 >> s) : (long long)((int)t0 >> s));
+        ok1 = ok1 && exact == (uns ? (long long)(t1 >> s) : (long long)((int)t1 >> s));
       }
       ok0 = __all_sync(0xffffffffu, ok0);
       ok1 = __all_sync(0xffffffffu, ok1);
@@ -229,7 +233,10 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
       int o[N];
       if (narrow) {
 #pragma unroll
-        for (int j = 0; j < N; ++j) o[j] = (q[j] * bb[j] + hh[j]) >> ss[j];
+        for (int j = 0; j < N; ++j) {
+          const unsigned t = (unsigned)q[j] * (unsigned)bb[j] + (unsigned)hh[j];
+          o[j] = is_signed ? (int)t >> ss[j] : (int)(t >> ss[j]);
+        }
       } else if (fast) {
 #pragma unroll
         for (int j = 0; j < N; ++j) o[j] = (__mulhi(q[j], bb[j]) + hh[j]) >> ss[j];
@@ -242,13 +249,153 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
   }
 }
 
-__global__ void __launch_bounds__(256, 2) concat_requant_kernel(const __grid_constant__ ConcatArgs a) {
-  int i = 0;
+struct W4State {
+  const unsigned char* ip; unsigned char* op;
+  long long px, step, in_row, out_row, pixels;
+  int lo, hi; bool word_out;
+};
+
+// Pixel loop of the four-channel form.  SIGNED: operand signedness; MODE: 2 narrow pair, 1 high-word form, 0 the
+// 64-bit definition; OUT: 0 8-bit output by saturating packs, 1 8-bit output with explicit bounds, 2 4-bit output.
+template <int BITS, bool SIGNED, int MODE, int OUT>
+__device__ __forceinline__ void concat_w4_loop(W4State t, const int (&bb)[4], const int (&hh)[4], const int (&ss)[4]) {
+  constexpr int KP = BITS == 32 ? 4 : 8;
+  const long long istep = t.step * t.in_row, ostep = t.step * t.out_row;
+  auto one = [&](const uint4 r, unsigned char* o_ptr) {
+    int q[4];
+    if (BITS == 32) { q[0] = (int)r.x; q[1] = (int)r.y; q[2] = (int)r.z; q[3] = (int)r.w; }
+    else if (BITS == 8) {
 #pragma unroll
-  for (int j = 1; j < HQ_CONCAT_MAX_BRANCHES; ++j)
-    if (j < a.n_br && (int)blockIdx.x >= a.br[j].block0) i = j;
-  if (a.br[i].width == 4) concat_branch<4>(a, i);
-  else concat_branch<16>(a, i);
+      for (int j = 0; j < 4; ++j) {
+        const unsigned sh = r.x >> (8 * j);
+        q[j] = SIGNED ? (int)(signed char)sh : (int)(sh & 0xFFu);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned sh = r.x >> (4 * j);
+        q[j] = SIGNED ? ((int)(sh << 28) >> 28) : (int)(sh & 0xFu);
+      }
+    }
+    int o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      o[j] = MODE == 2 ? (SIGNED ? (int)((unsigned)q[j] * (unsigned)bb[j] + (unsigned)hh[j]) >> ss[j]
+                                 : (int)(((unsigned)q[j] * (unsigned)bb[j] + (unsigned)hh[j]) >> ss[j]))
+           : MODE == 1 ? (__mulhi(q[j], bb[j]) + hh[j]) >> ss[j]
+                       : concat_dn64(q[j], bb[j], ss[j], t.lo, t.hi);
+    if (OUT != 2) {
+      unsigned w;
+      if (OUT == 0) w = pack4_sat(o[0], o[1], o[2], o[3], t.lo < 0);
+      else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = min(max(o[j], t.lo), t.hi) & 0xFF;
+        w = (unsigned)o[0] | ((unsigned)o[1] << 8) | ((unsigned)o[2] << 16) | ((unsigned)o[3] << 24);
+      }
+      if (t.word_out) *(unsigned*)o_ptr = w;
+      else { o_ptr[0] = (unsigned char)w; o_ptr[1] = (unsigned char)(w >> 8); o_ptr[2] = (unsigned char)(w >> 16); o_ptr[3] = (unsigned char)(w >> 24); }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[j] = min(max(o[j], t.lo), t.hi) & 0xF;
+      const unsigned w = (unsigned)o[0] | ((unsigned)o[1] << 4) | ((unsigned)o[2] << 8) | ((unsigned)o[3] << 12);
+      if (t.word_out) *(unsigned short*)o_ptr = (unsigned short)w;
+      else { o_ptr[0] = (unsigned char)w; o_ptr[1] = (unsigned char)(w >> 8); }
+    }
+  };
+  auto fetch = [&](const unsigned char* p) -> uint4 {
+    uint4 r = make_uint4(0u, 0u, 0u, 0u);
+    if (BITS == 32) r = *(const uint4*)p;
+    else if (BITS == 8) r.x = *(const unsigned*)p;
+    else r.x = *(const unsigned short*)p;
+    return r;
+  };
+  // whole groups of KP pixels: all reads first, then the arithmetic and the stores
+  while (t.px + (KP - 1) * t.step < t.pixels) {
+    uint4 raw[KP];
+#pragma unroll
+    for (int p = 0; p < KP; ++p) raw[p] = fetch(t.ip + p * istep);
+#pragma unroll
+    for (int p = 0; p < KP; ++p) one(raw[p], t.op + p * ostep);
+    t.px += KP * t.step; t.ip += KP * istep; t.op += KP * ostep;
+  }
+  for (; t.px < t.pixels; t.px += t.step, t.ip += istep, t.op += ostep) one(fetch(t.ip), t.op);
+}
+
+// Four channels per thread: the form for every branch whose channel count is a multiple of 4 (up to 1024 channels).
+// A thread reads 16 bytes (INT32), one word (8 bit) or two bytes (4 bit) per pixel through a running pointer, keeps
+// KP pixels in flight and twelve constants in registers, so many warps fit an SM; consecutive lanes read consecutive
+// pieces of the dense branch tensor and write consecutive words of the output row.
+template <int BITS>
+__device__ __forceinline__ void concat_w4(const ConcatArgs& a, const int i) {
+  const int is_signed = a.br[i].is_signed, ch = a.br[i].ch;
+  const int upp = a.br[i].upp, ppb = 256 / upp;
+  const int tid = threadIdx.x;
+  if (tid >= upp * ppb) return;
+  const int u = tid % upp, y = tid / upp;
+  const int k0 = u * 4, off = a.br[i].ch_off + k0;
+  const int lo = a.relu ? max(a.qmin, 0) : a.qmin, hi = a.qmax;
+  int bb[4], hh[4], ss[4];
+  bool fast = true;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    bb[j] = __ldg(a.br[i].b + k0 + j); ss[j] = __ldg(a.br[i].c + k0 + j); hh[j] = 0;
+    fast = fast && ss[j] >= 33;
+  }
+  bool narrow = a.narrow != nullptr && BITS != 32;
+  if (narrow) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) narrow = narrow && __ldg(&a.narrow[off + j].w) != 0;
+    if (narrow) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { const int4 t = __ldg(a.narrow + off + j); bb[j] = t.x; hh[j] = t.y; ss[j] = t.z; }
+    }
+  }
+  if (fast && !narrow) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { hh[j] = 1 << (ss[j] - 33); ss[j] -= 32; }
+  }
+  const int mode = narrow ? 2 : fast ? 1 : 0;
+  W4State t;
+  t.step = (long long)a.br[i].nblocks * ppb;
+  t.px = (long long)(blockIdx.x - a.br[i].block0) * ppb + y;
+  t.in_row = (long long)ch * BITS / 8; t.out_row = (long long)a.out_ch * a.out_bits / 8;
+  t.ip = (const unsigned char*)a.br[i].in + t.px * t.in_row + (long long)k0 * BITS / 8;
+  t.op = (unsigned char*)a.out + t.px * t.out_row + (long long)off * a.out_bits / 8;
+  t.lo = lo; t.hi = hi; t.pixels = a.pixels;
+  t.word_out = (off & 3) == 0 && (a.out_ch & 3) == 0;      // the thread's outputs are one aligned word / halfword
+  // one straight-line loop per signedness, form of the arithmetic and output type, chosen once
+  const int outk = a.out_bits == 4 ? 2 : a.sat ? 0 : 1;
+#define HQ_W4_OUT(S, M) \
+  do { if (outk == 0) concat_w4_loop<BITS, S, M, 0>(t, bb, hh, ss); \
+       else if (outk == 1) concat_w4_loop<BITS, S, M, 1>(t, bb, hh, ss); \
+       else concat_w4_loop<BITS, S, M, 2>(t, bb, hh, ss); } while (0)
+#define HQ_W4_MODE(S) \
+  do { if (mode == 2) HQ_W4_OUT(S, 2); else if (mode == 1) HQ_W4_OUT(S, 1); else HQ_W4_OUT(S, 0); } while (0)
+  if (BITS == 32 || is_signed) HQ_W4_MODE(true); else HQ_W4_MODE(false);
+#undef HQ_W4_MODE
+#undef HQ_W4_OUT
+}
+
+// The branch a block works for: the last branch of the wanted width whose first block is not beyond this one.
+__device__ __forceinline__ int concat_my_branch(const ConcatArgs& a, int width) {
+  int i = -1;
+#pragma unroll
+  for (int j = 0; j < HQ_CONCAT_MAX_BRANCHES; ++j)
+    if (j < a.n_br && a.br[j].width == width && (i < 0 || (int)blockIdx.x >= a.br[j].block0)) i = j;
+  return i;
+}
+
+// Branches in the four-channel form (few registers, many warps per SM) ...
+__global__ void __launch_bounds__(256, 4) concat_requant_kernel(const __grid_constant__ ConcatArgs a) {
+  const int i = concat_my_branch(a, 4);
+  if (a.br[i].bits == 32) concat_w4<32>(a, i);
+  else if (a.br[i].bits == 8) concat_w4<8>(a, i);
+  else concat_w4<4>(a, i);
+}
+
+// ... and the others (ragged or very wide branches) in the sixteen-channel form, in a launch of their own.
+__global__ void __launch_bounds__(256, 2) concat_requant_wide_kernel(const __grid_constant__ ConcatArgs a) {
+  concat_branch<16>(a, concat_my_branch(a, 16));
 }
 
 inline bool al16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
@@ -282,7 +429,7 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     ConcatBranch& B = a.br[i];
     B.in = t.data; B.b = rescale[i].b; B.c = rescale[i].c;
     B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = t.c; B.ch_off = off;
-    if (t.bits == 32 && t.c % 4 == 0 && t.c <= 4 * 256) { B.width = 4; B.vec = 1; }
+    if (t.c % 4 == 0 && t.c <= 4 * 256 && out->c % 2 == 0) { B.width = 4; B.vec = 1; }
     else { B.width = 16; B.vec = (t.bits != 32 && t.c % 16 == 0) ? 1 : 0; }
     B.upp = (t.c + B.width - 1) / B.width;
     if (B.upp > 256) return HQ_ERR_UNSUPPORTED;                   // more than 4096 channels in one branch
@@ -298,14 +445,15 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
   if (a.pixels == 0) return HQ_OK;
   // blocks of the one launch, dealt to the branches in proportion to the bytes they move
   const long long cap = (long long)h->sm_count * 8;
-  long long blocks = 0;
+  long long blocks4 = 0, blocks16 = 0;
   for (int i = 0; i < n_branches; ++i) {
     ConcatBranch& B = a.br[i];
-    const long long per_block = (long long)(256 / B.upp) * kPix;
+    const long long per_block = (long long)(256 / B.upp) * (B.width == 4 && B.bits != 32 ? 8 : kPix);
     const long long need = (a.pixels + per_block - 1) / per_block;
     long long share = (cap * weight[i] + weight_sum - 1) / weight_sum;
     if (share > need) share = need;
     if (share < 1) share = 1;
+    long long& blocks = B.width == 4 ? blocks4 : blocks16;          // each form numbers its own launch's blocks
     B.block0 = (int32_t)blocks; B.nblocks = (int32_t)share;
     blocks += share;
   }
@@ -325,6 +473,7 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
     a.narrow = tab;
   }
-  concat_requant_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a);
+  if (blocks4) concat_requant_kernel<<<(unsigned)blocks4, 256, 0, (cudaStream_t)stream>>>(a);
+  if (blocks16) concat_requant_wide_kernel<<<(unsigned)blocks16, 256, 0, (cudaStream_t)stream>>>(a);
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
