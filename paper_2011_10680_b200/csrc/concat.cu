@@ -3,12 +3,13 @@
 // i.e. every branch (the convolution branches as stored 8- or 4-bit tensors or INT32 accumulators, the pooling
 // branch as an INT32 tensor) is brought to the output scale by its own DN pairs and lands beside the others along
 // the channel axis.  Memory bound: every operand is read once, the output written once, in ONE launch for all
-// branches.  The blocks of the launch are dealt to the branches in proportion to their bytes, so a warp works on one
-// branch only (one operand type, one form of the arithmetic, no divergence).  A thread owns one 16-byte piece of a
-// branch's pixel row for the whole kernel -- 16 channels of an 8-bit branch (32 of a 4-bit one are two threads), 4
-// channels of an INT32 branch -- reads its dyadic pairs once, and keeps four pixels in flight; neighbouring lanes
-// read neighbouring 16-byte pieces of the dense branch tensor and write neighbouring pieces of the output row.
-// Integer arithmetic only.
+// branches whose channel count is a multiple of 4 (ragged ones take a second launch in a sixteen-channel form).
+// The blocks of the launch are dealt to the branches in proportion to their bytes, so a warp works on one branch
+// only.  A thread owns four channels of a branch for the whole kernel -- 16 bytes per pixel of an INT32 branch, one
+// word of an 8-bit branch, two bytes of a 4-bit one -- reads its dyadic pairs once, walks the pixels through running
+// pointers and keeps several pixels in flight; neighbouring lanes read neighbouring pieces of the dense branch
+// tensor and write neighbouring words of the output row.  The pixel loop is compiled per operand signedness, form
+// of the arithmetic and output type and chosen once per thread.  Integer arithmetic only.
 #include "hq_internal.cuh"
 
 namespace {

@@ -80,6 +80,12 @@ def test_concat_large_call_with_narrow_pairs(hq):
         run_and_compare(hq, case)
 
 
+def test_concat_at_the_benchmark_size(hq):
+    """The 35x35 module at batch 256, as `bench.py --membound` times it (90 M outputs): every stored value."""
+    case = inputs.concat_case(406, 256, 35, [(64, 8, 0), (64, 8, 0), (96, 8, 0), (64, 32, 1)])
+    run_and_compare(hq, case)
+
+
 def test_concat_every_shift_and_extreme_operands(hq):
     """Shifts 1..62 across the channels (both forms of the arithmetic), full-range INT32 and 8-bit operands."""
     g = inputs.rng(402)
