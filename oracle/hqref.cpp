@@ -323,6 +323,48 @@ int32_t hqref_concat_branch(const void* in, int32_t in_bits, int32_t in_signed,
   return HQREF_OK;
 }
 
+// Windowed sum pooling on wide integers (Appendix E: the pooling branch of an Inception module stays in
+// INT32): out[n,oh,ow,c] = sum over the k x k window of in[n, oh*stride+r-pad, ow*stride+s-pad, c], taps
+// outside the image counting as 0; the reciprocal of the window size of an average pool belongs to the dyadic pair of the
+// consumer (no division, Section 1).  in: bits 4/8/32; out: INT32 [n, oh, ow, c].
+int32_t hqref_sumpool(const void* in, int32_t n, int32_t h, int32_t w, int32_t ch, int32_t bits, int32_t is_signed,
+                      int32_t k, int32_t stride, int32_t pad, int32_t* out) {
+  if (!in || !out || n < 0 || h < 1 || w < 1 || ch < 1 || k < 1 || stride < 1 || pad < 0 || pad >= k)
+    return HQREF_ERR_INVALID_ARG;
+  if (!bits_ok(bits, true) || (bits == 4 && (ch & 1))) return HQREF_ERR_INVALID_ARG;
+  if (h + 2 * pad < k || w + 2 * pad < k) return HQREF_ERR_INVALID_ARG;
+  int32_t oh_n = 0, ow_n = 0;                      // window positions, counted (no division anywhere in this file)
+  for (int32_t y = 0; y + k <= h + 2 * pad; y += stride) ++oh_n;
+  for (int32_t x = 0; x + k <= w + 2 * pad; x += stride) ++ow_n;
+  int32_t status = HQREF_OK;
+#pragma omp parallel for schedule(static)
+  for (int32_t in_n = 0; in_n < n; ++in_n) {
+    for (int32_t oh = 0; oh < oh_n; ++oh) {
+      for (int32_t ow = 0; ow < ow_n; ++ow) {
+        for (int32_t cc = 0; cc < ch; ++cc) {
+          int64_t sum = 0;
+          for (int32_t r = 0; r < k; ++r) {
+            const int32_t ih = oh * stride + r - pad;
+            if (ih < 0 || ih >= h) continue;
+            for (int32_t s = 0; s < k; ++s) {
+              const int32_t iw = ow * stride + s - pad;
+              if (iw < 0 || iw >= w) continue;
+              sum += load_elem(in, (((int64_t)in_n * h + ih) * w + iw) * ch + cc, bits, is_signed);
+            }
+          }
+          if (sum < INT32_MIN || sum > INT32_MAX) {
+#pragma omp atomic write
+            status = HQREF_ERR_RANGE;
+            sum = 0;
+          }
+          out[(((int64_t)in_n * oh_n + oh) * ow_n + ow) * ch + cc] = (int32_t)sum;
+        }
+      }
+    }
+  }
+  return status;
+}
+
 int32_t hqref_num_threads(void) {
   int32_t t = 1;
 #ifdef _OPENMP

@@ -45,6 +45,8 @@ def lib():
         L.hqref_maxpool.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.hqref_concat_branch.restype = i32
         L.hqref_concat_branch.argtypes = [vp, i32, i32, vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, i32, i32]
+        L.hqref_sumpool.restype = i32
+        L.hqref_sumpool.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.hqref_num_threads.restype = i32
         _lib = L
     return _lib
@@ -164,6 +166,17 @@ def concat_requant(branches, relu, qmin, qmax, out_bits=8, out_signed=0):
         _check(lib().hqref_concat_branch(_p(x), br["bits"], br["signed"], _p(b), _p(c), pixels, br["ch"],
                                          relu, qmin, qmax, _p(out), out_bits, out_signed, out_ch, off))
         off += int(br["ch"])
+    return out
+
+
+def sumpool(x, ch, bits, signed, k, stride, pad):
+    """k x k window sums in INT32 (taps outside the image count as 0): the Inception pooling branch, Appendix E."""
+    x = np.ascontiguousarray(x)
+    n, h, w = x.shape[:3]
+    ho = (h + 2 * pad - k) // stride + 1
+    wo = (w + 2 * pad - k) // stride + 1
+    out = np.zeros((n, ho, wo, ch), np.int32)
+    _check(lib().hqref_sumpool(_p(x), n, h, w, ch, bits, signed, k, stride, pad, _p(out)))
     return out
 
 

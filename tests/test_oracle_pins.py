@@ -372,6 +372,29 @@ def test_concat_of_one_branch_is_the_plain_requantization():
     assert np.array_equal(one, hqref.residual_add(x, 32, 1, b, c, None, 0, 0, None, None, 8, 1, 0, 255, 8, 0))
 
 
+def test_sumpool_counts_taps_and_matches_padded_window_sums():
+    """Constant input: 9v inside, 6v on edges, 4v in corners (zero padding); random input: numpy window sums."""
+    v = np.full((1, 5, 6, 2), 7, np.int32)
+    y = hqref.sumpool(v, 2, 32, 1, 3, 1, 1)
+    assert y[0, 2, 3, 0] == 63 and y[0, 0, 2, 1] == 42 and y[0, 4, 5, 0] == 28 and y.shape == (1, 5, 6, 2)
+    g = np.random.default_rng(31)
+    for bits, k, stride, pad in ((32, 3, 1, 1), (8, 3, 2, 1), (32, 2, 2, 0), (8, 5, 1, 2)):
+        x = (g.integers(-(1 << 20), 1 << 20, size=(2, 7, 9, 4)).astype(np.int32) if bits == 32
+             else g.integers(-128, 128, size=(2, 7, 9, 4)).astype(np.int8))
+        y = hqref.sumpool(x, 4, bits, 1, k, stride, pad)
+        xp = np.pad(x.astype(np.int64), ((0, 0), (pad, pad), (pad, pad), (0, 0)))
+        ref = np.zeros(y.shape, np.int64)
+        for oh in range(y.shape[1]):
+            for ow in range(y.shape[2]):
+                ref[:, oh, ow] = xp[:, oh * stride:oh * stride + k, ow * stride:ow * stride + k].sum(axis=(1, 2))
+        assert np.array_equal(y.astype(np.int64), ref)
+    # an average pool without division: window sum, then DN(1/9): a constant v comes back in the interior
+    b, c = inputs.dyadic_from_scale(1.0 / 9)
+    s9 = hqref.sumpool(np.full((1, 5, 5, 1), 100, np.int32), 1, 32, 1, 3, 1, 1)
+    avg = hqref.residual_add(s9, 32, 1, b, c, None, 0, 0, None, None, 1, 0, -128, 127, 8, 1)
+    assert avg[0, 2, 2, 0] == 100 and avg[0, 0, 0, 0] == 44          # corner: round(400 / 9)
+
+
 # ---------------------------------------------------------------- P9: topology ------------------
 def test_table_cost_matches_the_papers_table1(golden_dir):
     want = {}
