@@ -155,6 +155,17 @@ hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic rescal
 hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const hq_tensor* branches, const hq_dyadic* rescale,
                             int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
 
+/*
+ * k x k window SUMS on wide integers (Appendix E: "we use INT32 for the pooling layer"; the pooling
+ * branch of an Inception module works on the INT32 feature map):
+ *   out[n,oh,ow,c] = sum_{r,s < k} in[n, oh*stride+r-pad, ow*stride+s-pad, c], taps outside the image = 0.
+ * An average pool is this sum followed by a dyadic pair that carries 1/k^2 (hq_concat_requant,
+ * hq_residual_add): no division (Section 1).  in: bits 4, 8 or 32; out: bits 32, extents
+ * (h + 2 pad - k) / stride + 1.  pad < k.  Sums beyond INT32 are undefined (the oracle reports them).
+ */
+hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,
+                     hq_tensor* out, void* stream);
+
 /* k x k max pooling of an 8-bit tensor; window taps outside the image are ignored (ResNet stem;
  * an integer max commutes with the monotone requantization of Eq. 4).  pad < k. */
 hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,

@@ -22,7 +22,7 @@ EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
     "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
-    "hq_ilp_solve", "hq_concat_requant",
+    "hq_ilp_solve", "hq_concat_requant", "hq_sumpool",
 ]
 
 
@@ -75,6 +75,7 @@ def lib():
         L.hq_residual_add.argtypes = [vp, TP, hq_dyadic, TP, hq_dyadic, i32, i32, i32, TP, vp]
         L.hq_avgpool_requant.argtypes = [vp, TP, hq_dyadic, i32, i32, TP, vp]
         L.hq_maxpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
+        L.hq_sumpool.argtypes = [vp, TP, i32, i32, i32, TP, vp]
         L.hq_concat_requant.argtypes = [vp, i32, TP, C.POINTER(hq_dyadic), i32, i32, i32, TP, vp]
         L.hq_network_create.argtypes = [vp, LP, i32, i32, i32, i32, i32, i32, C.POINTER(vp)]
         L.hq_run_network.argtypes = [vp, TP, TP, C.POINTER(vp), vp]
@@ -211,6 +212,11 @@ class Handle:
         ds = (hq_dyadic * n)(*[_dy(br["b"], br["c"]) for br in branches])
         to = tensor_of(out, out.shape[3] * (2 if out_bits == 4 else 1), out_bits, out_signed)
         return lib().hq_concat_requant(self._h, n, ts, ds, relu, qmin, qmax, C.byref(to), _stream())
+
+    def sumpool(self, x, ch, bits, signed, k, stride, pad, out):
+        ti = tensor_of(x, ch, bits, signed)
+        to = tensor_of(out, ch, 32, 1)
+        return lib().hq_sumpool(self._h, C.byref(ti), k, stride, pad, C.byref(to), _stream())
 
     def maxpool(self, x, ch, signed, k, stride, pad, out):
         ti = tensor_of(x, ch, 8, signed)

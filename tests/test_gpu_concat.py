@@ -148,3 +148,55 @@ def test_concat_empty_batch_is_a_no_op(hq):
     assert st == binding.HQ_OK
     hq.sync()
     assert x.numel() == 0 and int(keep.sum()) == 0
+
+
+# ------------------------------------------------------------------ INT32 window sums (pooling branch) ----
+@pytest.mark.parametrize("n,h,w,ch,bits,signed,k,stride,pad", [
+    (2, 35, 35, 64, 32, 1, 3, 1, 1),        # the 35x35 module's pooling branch
+    (3, 17, 17, 192, 32, 1, 3, 1, 1),
+    (2, 9, 7, 6, 32, 1, 3, 2, 1),           # channel count not a multiple of 4, stride 2, H != W
+    (2, 8, 8, 10, 8, 0, 3, 1, 1),
+    (1, 6, 5, 8, 4, 1, 2, 2, 0),
+    (1, 7, 7, 4, 8, 1, 5, 1, 2),
+])
+def test_sumpool_matches_the_oracle(hq, n, h, w, ch, bits, signed, k, stride, pad):
+    from oracle import hqref
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(407, n, h, ch, bits)
+    if bits == 32:
+        x = g.integers(-(1 << 26), 1 << 26, size=(n, h, w, ch), dtype=np.int64).astype(np.int32)
+    elif bits == 8:
+        x = g.integers(-128 if signed else 0, 128 if signed else 256, size=(n, h, w, ch), dtype=np.int64).astype(np.int8 if signed else np.uint8)
+    else:
+        x = inputs.pack4(g.integers(-8 if signed else 0, 8 if signed else 16, size=(n, h, w, ch), dtype=np.int64))
+    ref = hqref.sumpool(x, ch, bits, signed, k, stride, pad)
+    out = torch.full(ref.shape, 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    st = hq.sumpool(binding.to_device(x), ch, bits, signed, k, stride, pad, out)
+    assert st == binding.HQ_OK, binding.status_string(st)
+    hq.sync()
+    assert np.array_equal(out.cpu().numpy(), ref)
+
+
+def test_pooling_branch_then_concat_is_an_inception_module_tail(hq):
+    """INT32 feature map -> 3x3 window sums (INT32) -> concatenated with 8-bit branches, 1/9 inside the pooling
+    branch's dyadic pairs: both calls chained on the device against the oracle's chain."""
+    from oracle import hqref
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(408)
+    n, hw = 2, 35
+    fmap = g.integers(-(1 << 18), 1 << 18, size=(n, hw, hw, 32), dtype=np.int64).astype(np.int32)
+    pb, pc = inputs.dyadic_from_scale(np.exp2(g.uniform(-12.0, -10.0, size=32)) / 9.0)
+    case = inputs.concat_case(409, n, hw, [(64, 8, 0), (96, 8, 0)])
+    pooled_ref = hqref.sumpool(fmap, 32, 32, 1, 3, 1, 1)
+    branches_ref = case["branches"] + [{"x": pooled_ref, "bits": 32, "signed": 1, "ch": 32, "b": pb, "c": pc}]
+    ref = hqref.concat_requant(branches_ref, 1, 0, 255, 8, 0)
+    pooled = torch.empty((n, hw, hw, 32), dtype=torch.int32, device="cuda")
+    assert hq.sumpool(binding.to_device(fmap), 32, 32, 1, 3, 1, 1, pooled) == binding.HQ_OK
+    dev = [{**br, "x": binding.to_device(br["x"]), "b": binding.to_device(br["b"]), "c": binding.to_device(br["c"])}
+           for br in case["branches"]]
+    dev.append({"x": pooled, "bits": 32, "signed": 1, "ch": 32, "b": binding.to_device(pb), "c": binding.to_device(pc)})
+    out = binding.alloc_out(n, hw, hw, 192, 8, 0)
+    assert hq.concat_requant(dev, 1, 0, 255, out, 8, 0) == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(out.cpu().numpy(), ref)
+    assert np.count_nonzero((ref[..., 160:] > 0) & (ref[..., 160:] < 255)) > ref[..., 160:].size // 4
