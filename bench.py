@@ -215,7 +215,8 @@ def run_sweep(args):
 
 def run_membound(args):
     """The memory-bound kernels on their own, at ResNet-50 batch-256 tensor sizes (each operand larger than L2):
-    max pooling, dyadic requantization, the two-branch residual add and the average-pool requantization.  Device
+    max pooling, dyadic requantization, the two-branch residual add, the average-pool requantization, and at
+    InceptionV3 module sizes the concatenation with per-branch rescale and the INT32 window sums.  Device
     time per call (CUDA events; 256 MB written, then 256 MB read between repetitions), achieved GB/s of the algorithmic bytes
     (every operand read once, the result written once) and its fraction of the measured copy bandwidth."""
     import torch
@@ -270,6 +271,10 @@ def run_membound(args):
     ocat17 = torch.empty((4 * n, 17, 17, 768), dtype=torch.uint8, device="cuda")
     cases.append(("concat 4x u8 -> u8 [%d,17,17,768]" % (4 * n), 2 * ocat17.numel(),
                   lambda: hq.concat_requant(cat17, 1, 0, 255, ocat17, 8, 0)))
+    # the pooling branch of that module: 3x3 / stride 1 window sums over the INT32 feature map
+    xp = ri(-(1 << 20), 1 << 20, (n, 35, 35, 192), torch.int32); op_ = torch.empty_like(xp)
+    cases.append(("sumpool 3x3/1 s32 -> s32 [%d,35,35,192]" % n, 2 * xp.numel() * 4,
+                  lambda: hq.sumpool(xp, 192, 32, 1, 3, 1, 1, op_)))
     rows = []
     for name, byt, fn in cases:
         times = []

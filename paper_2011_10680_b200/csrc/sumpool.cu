@@ -15,42 +15,47 @@ struct SumPoolArgs {
   int32_t vec;     // 1: INT32 input with ch % 4 == 0: 16-byte accesses
 };
 
+// Block x = one output row (image, oh); block y, thread = a piece of that row: (ow, group of four channels), or
+// (ow, channel) for element-wise reads.  K = 3 unrolls the window so that its nine reads are in flight together;
+// K = 0 takes the window size from the arguments.
+template <int K>
 __global__ void __launch_bounds__(256) sumpool_kernel(const __grid_constant__ SumPoolArgs a) {
+  const int k = K ? K : a.k;
   const int cg = a.vec ? a.ch >> 2 : a.ch;                       // channel groups per pixel
-  const long long total = (long long)a.n * a.oh_n * a.ow_n * cg;
-  for (long long t = (long long)blockIdx.x * 256 + threadIdx.x; t < total; t += (long long)gridDim.x * 256) {
-    const int g = (int)(t % cg);
-    long long pix = t / cg;
-    const int ow = (int)(pix % a.ow_n); pix /= a.ow_n;
-    const int oh = (int)(pix % a.oh_n);
-    const long long img = pix / a.oh_n;
-    const int ih0 = oh * a.stride - a.pad, iw0 = ow * a.stride - a.pad;
-    if (a.vec) {
-      int4 sum = make_int4(0, 0, 0, 0);
-      for (int r = 0; r < a.k; ++r) {
-        const int ih = ih0 + r;
-        if (ih < 0 || ih >= a.h) continue;
-        for (int s = 0; s < a.k; ++s) {
-          const int iw = iw0 + s;
-          if (iw < 0 || iw >= a.w) continue;
-          const int4 v = *((const int4*)((const int*)a.in + ((img * a.h + ih) * a.w + iw) * a.ch) + g);
+  const int col = blockIdx.y * 256 + threadIdx.x;
+  if (col >= a.ow_n * cg) return;
+  const int ow = col / cg, g = col - ow * cg;
+  const int img = blockIdx.x / a.oh_n, oh = blockIdx.x - img * a.oh_n;
+  const int ih0 = oh * a.stride - a.pad, iw0 = ow * a.stride - a.pad;
+  const long long o_idx = ((long long)blockIdx.x * a.ow_n + ow) * cg + g;   // in units of the thread's piece
+  const long long img_base = (long long)img * a.h * a.w;
+  if (a.vec) {
+    int4 sum = make_int4(0, 0, 0, 0);
+#pragma unroll
+    for (int r = 0; r < k; ++r) {
+      const int ih = ih0 + r;
+#pragma unroll
+      for (int s = 0; s < k; ++s) {
+        const int iw = iw0 + s;
+        if (ih >= 0 && ih < a.h && iw >= 0 && iw < a.w) {
+          const int4 v = *((const int4*)((const int*)a.in + (img_base + (long long)ih * a.w + iw) * a.ch) + g);
           sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
       }
-      *((int4*)(a.out + t * 4)) = sum;                             // t enumerates the output's 16-byte pieces in order
-    } else {
-      int sum = 0;
-      for (int r = 0; r < a.k; ++r) {
-        const int ih = ih0 + r;
-        if (ih < 0 || ih >= a.h) continue;
-        for (int s = 0; s < a.k; ++s) {
-          const int iw = iw0 + s;
-          if (iw < 0 || iw >= a.w) continue;
-          sum += hq_load_elem(a.in, ((img * a.h + ih) * a.w + iw) * a.ch + g, a.bits, a.is_signed);
-        }
-      }
-      a.out[t] = sum;
     }
+    *((int4*)a.out + o_idx) = sum;
+  } else {
+    int sum = 0;
+    for (int r = 0; r < k; ++r) {
+      const int ih = ih0 + r;
+      if (ih < 0 || ih >= a.h) continue;
+      for (int s = 0; s < k; ++s) {
+        const int iw = iw0 + s;
+        if (iw < 0 || iw >= a.w) continue;
+        sum += hq_load_elem(a.in, (img_base + (long long)ih * a.w + iw) * a.ch + g, a.bits, a.is_signed);
+      }
+    }
+    a.out[o_idx] = sum;
   }
 }
 
@@ -72,11 +77,11 @@ extern "C" hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, in
   a.n = in->n; a.h = in->h; a.w = in->w; a.ch = in->c; a.bits = in->bits; a.is_signed = in->bits == 32 ? 1 : in->is_signed;
   a.k = k; a.stride = stride; a.pad = pad; a.oh_n = ho; a.ow_n = wo;
   a.vec = (in->bits == 32 && in->c % 4 == 0) ? 1 : 0;
-  const long long total = (long long)a.n * ho * wo * (a.vec ? a.ch / 4 : a.ch);
-  if (total == 0) return HQ_OK;
-  long long blocks = (total + 255) / 256;
-  const long long cap = (long long)h->sm_count * 32;
-  if (blocks > cap) blocks = cap;
-  sumpool_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a);
+  if (a.n == 0) return HQ_OK;
+  const long long rows = (long long)a.n * ho, cols = (long long)wo * (a.vec ? a.ch / 4 : a.ch);
+  if (rows > 0x7fffffffLL || (cols + 255) / 256 > 65535) return HQ_ERR_UNSUPPORTED;
+  const dim3 grid((unsigned)rows, (unsigned)((cols + 255) / 256));
+  if (k == 3) sumpool_kernel<3><<<grid, 256, 0, (cudaStream_t)stream>>>(a);
+  else sumpool_kernel<0><<<grid, 256, 0, (cudaStream_t)stream>>>(a);
   return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
