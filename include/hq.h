@@ -41,7 +41,7 @@ typedef enum {
   HQ_ERR_UNSUPPORTED = 2,  /* valid request no kernel covers */
   HQ_ERR_ALIGNMENT = 3,    /* a data pointer is not 16-byte aligned */
   HQ_ERR_RANGE = 4,        /* reserved: accumulator + bias left INT32 (the CPU oracle reports it) */
-  HQ_ERR_WORKSPACE = 5,    /* device allocation failed */
+  HQ_ERR_WORKSPACE = 5,    /* device allocation failed, or the request exceeds a fixed scratch array */
   HQ_ERR_CUDA = 6,         /* a CUDA runtime or driver call failed */
   HQ_ERR_TIMEOUT = 7,      /* a bounded device-side wait expired; outputs are not valid */
   HQ_ERR_INFEASIBLE = 8    /* hq_ilp_solve: no assignment meets the limits */
@@ -111,8 +111,10 @@ hq_status hq_sync(hq_handle* h, void* stream);
  *   otherwise       :  y = dn(t, b[oc], c[oc]);  if residual: y += dn(res, rb[oc], rc[oc]);
  *                      if relu: y = max(y, 0);  out = clamp(y, qmin, qmax), stored at out->bits.
  * in: bits 8 or 4 (== w_bits), signed or unsigned.  out: n, h, w, c must equal the convolution's
- * output extents.  The tensor-core path needs cin*bits/8 to be a multiple of 32 bytes (16 for the
- * first-layer path); other shapes run on the CUDA-core path.  Accumulator overflow beyond INT32
+ * output extents.  The tensor-core kernel takes layers with cin a multiple of 32, directly or - for the
+ * 3-channel first layer, thin layers and layers whose input tensor is below 128 KiB - through a lowered form
+ * (space-to-depth copy or patch matrix in scratch memory of the handle); other shapes run on the CUDA-core
+ * path.  Accumulator overflow beyond INT32
  * is undefined (cannot happen for K = kh*kw*cin <= 66311 with 8-bit operands).
  */
 hq_status hq_conv2d(hq_handle* h, const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
@@ -140,9 +142,9 @@ hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic rescal
                              int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
 
 /*
- * Concatenation along the channel axis with a dyadic rescale per branch (Appendix E, "Concatenation
- * Layer": the outputs of an Inception module's branches are "scaled and requantized before being
- * concatenated", one DN operator per branch):
+ * Concatenation along the channel axis with a dyadic rescale per branch (Appendix E, concatenation
+ * layer: every branch of an Inception module gets its own DN rescale to the output scale before the
+ * channel ranges are joined):
  *   out[n,h,w, off_i + k] = clamp(relu?(dn(branch_i[n,h,w,k], b_i[k], c_i[k]))),  off_i = c_0 + ... + c_{i-1}.
  * `branches` and `rescale` are HOST arrays of n_branches entries (1 <= n_branches <=
  * HQ_CONCAT_MAX_BRANCHES); each tensor's data and each pair's b / c arrays (length = that branch's
@@ -156,8 +158,8 @@ hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const hq_tensor* b
                             int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
 
 /*
- * k x k window SUMS on wide integers (Appendix E: "we use INT32 for the pooling layer"; the pooling
- * branch of an Inception module works on the INT32 feature map):
+ * k x k window SUMS on wide integers (Appendix E keeps the pooling layer, i.e. the pooling branch of
+ * an Inception module, on the INT32 feature map):
  *   out[n,oh,ow,c] = sum_{r,s < k} in[n, oh*stride+r-pad, ow*stride+s-pad, c], taps outside the image = 0.
  * An average pool is this sum followed by a dyadic pair that carries 1/k^2 (hq_concat_requant,
  * hq_residual_add): no division (Section 1).  in: bits 4, 8 or 32; out: bits 32, extents
@@ -201,6 +203,13 @@ hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* 
 hq_status hq_network_launch_count(const hq_network* net, int32_t* launches);
 hq_status hq_network_destroy(hq_network* net);
 
+/* Debug aid (no paper counterpart): every device buffer a network owns - layer outputs, widened weights,
+ * scratch - lies between two 256-byte guard bands written when the network is built.  This call waits for
+ * `stream`, reads the bands back and returns HQ_ERR_RANGE if any byte changed, with the layer that owns the
+ * buffer in *bad_layer (-1: the shared scratch buffer; bad_layer may be NULL): a kernel wrote before the
+ * first or beyond the last byte of a tensor.  Host call; HQ_OK means every band is intact. */
+hq_status hq_network_check_guards(const hq_network* net, void* stream, int32_t* bad_layer);
+
 /*
  * hq_conv2d for callers that cannot allocate device memory.  (The paper has no counterpart: this is
  * a deployment convenience of the library, not a step of the method.)
@@ -223,11 +232,18 @@ hq_status hq_network_destroy(hq_network* net);
  * contents: the call rewrites everything it later reads and clears its status word on `stream`,
  * but two calls whose GPU work overlaps (different streams, or graphs replayed concurrently) race on
  * the array and give undefined results - serialise them.  The current device is used; pointers follow
- * the rules of hq_conv2d.  An expired device-side wait is not reported by this variant.
+ * the rules of hq_conv2d.  The one-time set-up is guarded by a lock, so first calls may come from several
+ * host threads.  An expired device-side wait is reported by hq_conv2d_noalloc_sync.
  */
 hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* desc, hq_tensor* out, void* stream);
 
-/* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail, 3 = like 2 and
+/* Wait for `stream` and return HQ_ERR_TIMEOUT if a kernel of the hq_conv2d_noalloc calls queued on it gave
+ * up a bounded device-side wait (the outputs of that call are not valid then), HQ_OK otherwise.  Like the
+ * call it serves it allocates nothing; the word it reads is cleared by the next hq_conv2d_noalloc. */
+hq_status hq_conv2d_noalloc_sync(void* stream);
+
+/* Choose the convolution path: 0 = automatic, 1 = CUDA cores only, 2 = tensor cores or fail (HQ_ERR_UNSUPPORTED
+ * for a shape they do not take, HQ_ERR_WORKSPACE when scratch memory for a lowered form cannot be had), 3 = like 2 and
  * the tensor-core kernel's launch shapes are chosen by what the layer allows, not by its size (small test cases
  * then reach the shapes of large layers). */
 hq_status hq_set_conv_path(hq_handle* h, int32_t path);

@@ -17,11 +17,14 @@ def build(force: bool = False) -> str:
     return LIB
 
 
-def check_no_float_codegen() -> None:
-    """Compile-only pass that forbids every floating-point / vector register (x86 GCC): the integer
-    pipeline must build with general registers alone (the paper's no-floating-point claim)."""
-    cmd = ["g++", "-std=c++17", "-O1", "-mgeneral-regs-only", "-fsyntax-only", "-c", SRC]
-    subprocess.run(cmd, check=True)
+def check_no_float_codegen(src: str = SRC) -> None:
+    """Compile `src` to object code (discarded) with every floating-point / vector register forbidden
+    (x86 GCC, -mgeneral-regs-only): the integer pipeline must build with general registers alone (the
+    paper's no-floating-point claim, Section 1 and Appendix H).  GCC raises this error while generating
+    code, so the pass has to compile for real: a syntax-only run accepts a `double`.
+    Raises subprocess.CalledProcessError when the source needs a floating-point register."""
+    cmd = ["g++", "-std=c++17", "-O1", "-mgeneral-regs-only", "-c", src, "-o", os.devnull]
+    subprocess.run(cmd, check=True, stderr=subprocess.DEVNULL)
 
 
 if __name__ == "__main__":

@@ -22,6 +22,7 @@ EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
     "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
+    "hq_network_check_guards", "hq_conv2d_noalloc_sync",
     "hq_ilp_solve", "hq_concat_requant", "hq_sumpool",
 ]
 
@@ -84,6 +85,8 @@ def lib():
         L.hq_network_layer_bytes.argtypes = [vp, i32, C.POINTER(C.c_int64)]
         L.hq_network_launch_count.argtypes = [vp, C.POINTER(i32)]
         L.hq_network_destroy.argtypes = [vp]
+        L.hq_network_check_guards.argtypes = [vp, vp, C.POINTER(i32)]
+        L.hq_conv2d_noalloc_sync.argtypes = [vp]
         L.hq_set_conv_path.argtypes = [vp, i32]
         L.hq_expire_wait_selftest.argtypes = [vp, i32, vp]
         L.hq_expire_wait_selftest.restype = i32
@@ -144,13 +147,38 @@ def to_device(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
+GUARD_BYTES, GUARD_VALUE = 4096, 0xA5
+_guarded = []          # (flat uint8 buffer, payload bytes) of every output handed out since the last check
+
+
 def alloc_out(n, h, w, c, bits, signed):
+    """Output tensor of a call, allocated between two 4 KiB guard bands filled with 0xA5 (the stand-in for a
+    memory checker: check_guards() finds any byte a kernel wrote before the first or after the last element)."""
     import torch
-    if bits == 32:
-        return torch.empty((n, h, w, c), dtype=torch.int32, device="cuda")
-    if bits == 8:
-        return torch.empty((n, h, w, c), dtype=torch.int8 if signed else torch.uint8, device="cuda")
-    return torch.empty((n, h, w, c // 2), dtype=torch.uint8, device="cuda")
+    dtype = torch.int32 if bits == 32 else (torch.int8 if (bits == 8 and signed) else torch.uint8)
+    shape = (n, h, w, c // 2) if bits == 4 else (n, h, w, c)
+    nbytes = n * h * w * c * bits // 8
+    flat = torch.empty(nbytes + 2 * GUARD_BYTES, dtype=torch.uint8, device="cuda")
+    flat[:GUARD_BYTES] = GUARD_VALUE
+    flat[GUARD_BYTES + nbytes:] = GUARD_VALUE
+    _guarded.append((flat, nbytes))
+    return flat[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype).view(shape)
+
+
+def check_guards():
+    """Verify (and forget) the guard bands of every tensor alloc_out returned; raises on a touched byte."""
+    import torch
+    torch.cuda.synchronize()
+    bad = []
+    for flat, nbytes in _guarded:
+        lo, hi = flat[:GUARD_BYTES], flat[GUARD_BYTES + nbytes:]
+        if not (bool((lo == GUARD_VALUE).all()) and bool((hi == GUARD_VALUE).all())):
+            before = int((lo != GUARD_VALUE).sum())
+            after = int((hi != GUARD_VALUE).sum())
+            bad.append(f"{nbytes}-byte output: {before} bytes written before it, {after} after it")
+    _guarded.clear()
+    if bad:
+        raise AssertionError("a kernel wrote outside its output tensor: " + "; ".join(bad))
 
 
 class Handle:
@@ -247,6 +275,10 @@ def conv2d_noalloc(case: dict, dev: dict, out):
     return lib().hq_conv2d_noalloc(C.byref(tin), C.byref(d), C.byref(tout), _stream())
 
 
+def conv2d_noalloc_sync() -> int:
+    return lib().hq_conv2d_noalloc_sync(_stream())
+
+
 def upload_case(case: dict) -> dict:
     return {k: to_device(case[k]) for k in ("x", "wgt", "bias", "b", "c", "res", "rb", "rc")}
 
@@ -316,8 +348,14 @@ class Network:
         return list(ns)
 
     def alloc_taps(self):
-        import torch
-        return [torch.empty(self.layer_bytes(i), dtype=torch.uint8, device="cuda") for i in range(len(self.table["layers"]))]
+        return [alloc_out(1, 1, 1, self.layer_bytes(i), 8, 0).view(-1) for i in range(len(self.table["layers"]))]
+
+    def check_guards(self):
+        """hq_network_check_guards: raises if a kernel wrote outside one of the network's own buffers."""
+        bad = C.c_int32(-2)
+        st = lib().hq_network_check_guards(self._net, _stream(), C.byref(bad))
+        if st != HQ_OK:
+            raise AssertionError(f"hq_network_check_guards: {status_string(st)}, buffer of layer {bad.value}")
 
     def close(self):
         if self._net:

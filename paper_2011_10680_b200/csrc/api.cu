@@ -74,7 +74,18 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
   a.out = out->data; a.ho = ho; a.wo = wo; a.out_bits = out->bits; a.out_signed = out->is_signed;
   cudaStream_t s = (cudaStream_t)stream;
   const bool tc_ok = hq_conv_tc_supported(a);
-  if (h->conv_path >= 2 && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
+  const bool force_tc = h->conv_path >= 2;
+  if (force_tc && !tc_ok && !hq_conv_widen4_applies(a)) return HQ_ERR_UNSUPPORTED;
+  // Scratch for a lowered form: the caller's buffer (a network sized it when it was built), else the handle's own,
+  // grown here.  A failure to grow it (e.g. inside a stream capture) is remembered and returned when tensor cores
+  // were demanded; in automatic mode the CUDA-core kernel below takes the layer instead.
+  hq_status scratch_err = HQ_OK;
+  auto scratch_for = [&](size_t need) -> void* {
+    if (scratch) return scratch_bytes >= need ? scratch : nullptr;
+    const hq_status st = hq_reserve_workspace(h, need, s);
+    if (st != HQ_OK) { scratch_err = st; return nullptr; }
+    return h->workspace;
+  };
   if (h->conv_path != 1 && tc_ok) {
     // A single large call with an 8-bit residual: its narrow residual pairs are worked out first, in the handle's
     // buffer (a network prepares them once when it is built); one small launch that the cheaper epilogue repays.
@@ -84,25 +95,26 @@ hq_status conv_common(hq_handle* h, const hq_tensor* in, const hq_conv_desc* d, 
       a.res_narrow = h->narrow_pairs;
       a.res_narrow_fresh = 1;
     }
-    return hq_launch_conv_tc(h, a, s);
-  }
-  if (h->conv_path != 1 && hq_conv_widen4_applies(a)) {
-    // packed 4-bit operands: widened copies in scratch, then the tensor-core kernel
-    const size_t need = hq_conv_widen4_bytes(a);
-    if (scratch && scratch_bytes >= need) return hq_launch_conv_widen4(h, a, scratch, s);
-    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_widen4(h, a, h->workspace, s);
-  }
-  if (h->conv_path != 1 && hq_conv_s2d_applies(a)) {
-    // ImageNet-style first layer: space-to-depth copy of the image, then the tensor-core kernel
-    const size_t need = hq_conv_s2d_bytes(a);
-    if (scratch && scratch_bytes >= need) return hq_launch_conv_s2d(h, a, scratch, s);
-    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_s2d(h, a, h->workspace, s);
-  }
-  if (h->conv_path != 1 && hq_conv_lowering_applies(a)) {
-    // thin first layers: patch matrix in the handle's scratch buffer, then the tensor-core kernel
-    const size_t need = hq_conv_lowering_bytes(a);
-    if (scratch && scratch_bytes >= need) return hq_launch_conv_lowered(h, a, scratch, s);
-    if (!scratch && hq_reserve_workspace(h, need, s) == HQ_OK) return hq_launch_conv_lowered(h, a, h->workspace, s);
+    const hq_status st = hq_launch_conv_tc(h, a, s);
+    if (st != HQ_ERR_UNSUPPORTED) return st;
+    // declined before anything was launched (an im2col fetch from a tensor below 128 KiB, more channel tiles than
+    // SMs): the patch-matrix form still runs the contraction on the tensor cores
+    if (hq_conv_lowering_applies(a)) {
+      if (void* buf = scratch_for(hq_conv_lowering_bytes(a))) { const hq_status st2 = hq_launch_conv_lowered(h, a, buf, s); if (st2 != HQ_ERR_UNSUPPORTED || force_tc) return st2; }
+    }
+    if (force_tc) return scratch_err != HQ_OK ? scratch_err : HQ_ERR_UNSUPPORTED;
+  } else if (h->conv_path != 1) {
+    if (hq_conv_widen4_applies(a)) {
+      // packed 4-bit operands: widened copies in scratch, then the tensor-core kernel
+      if (void* buf = scratch_for(hq_conv_widen4_bytes(a))) { const hq_status st2 = hq_launch_conv_widen4(h, a, buf, s); if (st2 != HQ_ERR_UNSUPPORTED || force_tc) return st2; }
+      if (force_tc) return scratch_err != HQ_OK ? scratch_err : HQ_ERR_WORKSPACE;
+    } else if (hq_conv_s2d_applies(a)) {
+      // ImageNet-style first layer: space-to-depth copy of the image, then the tensor-core kernel
+      if (void* buf = scratch_for(hq_conv_s2d_bytes(a))) { const hq_status st2 = hq_launch_conv_s2d(h, a, buf, s); if (st2 != HQ_ERR_UNSUPPORTED || force_tc) return st2; }
+    } else if (hq_conv_lowering_applies(a)) {
+      // thin first layers: patch matrix in scratch, then the tensor-core kernel
+      if (void* buf = scratch_for(hq_conv_lowering_bytes(a))) { const hq_status st2 = hq_launch_conv_lowered(h, a, buf, s); if (st2 != HQ_ERR_UNSUPPORTED || force_tc) return st2; }
+    }
   }
   return hq_launch_conv_cuda_core(a, s) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
@@ -122,8 +134,16 @@ hq_status hq_reserve_workspace(hq_handle* h, size_t bytes, cudaStream_t s) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Every buffer a network owns sits between two guard bands of kGuardBytes bytes filled with kGuardByte when the
+// network is built.  No kernel may touch them: hq_network_check_guards reads them back, which is how the tests look
+// for writes beyond a tensor (before its first or after its last byte) on the buffers the caller never sees.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardByte = 0xA5;
+struct GuardedBuffer { void* base; void* data; size_t bytes; int32_t layer; };
+
 struct hq_network {
   hq_handle* h;
+  std::vector<GuardedBuffer> buffers; // every device allocation of the network, with its guard bands
   std::vector<hq_layer> layers;
   std::vector<hq_tensor> outs;       // planned output tensor of every layer (data owned by the network)
   std::vector<long long> bytes;
@@ -140,6 +160,21 @@ struct hq_network {
   struct CachedGraph { cudaGraphExec_t exec; const void* images; void* logits; };
   std::vector<CachedGraph> graphs;
 };
+
+// Allocate `bytes` for layer `layer` of `net` between two guard bands; NULL when the device is out of memory.
+static void* net_alloc(hq_network* net, size_t bytes, int32_t layer) {
+  unsigned char* base = nullptr;
+  if (cudaMalloc(&base, bytes + 2 * kGuardBytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (cudaMemset(base, kGuardByte, kGuardBytes) != cudaSuccess ||
+      cudaMemset(base + kGuardBytes + bytes, kGuardByte, kGuardBytes) != cudaSuccess) { cudaFree(base); return nullptr; }
+  net->buffers.push_back({base, base + kGuardBytes, bytes, layer});
+  return base + kGuardBytes;
+}
+
+static void net_free(hq_network* net, void* data) {
+  for (auto it = net->buffers.begin(); it != net->buffers.end(); ++it)
+    if (it->data == data) { cudaFree(it->base); net->buffers.erase(it); return; }
+}
 
 extern "C" {
 
@@ -352,15 +387,15 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
             if (need > net->scratch_bytes) net->scratch_bytes = need;
             net->launches += 1;                 // the activation-widening kernel (the weights are widened once, below)
             const long long wvals = (long long)d.cout * d.kh * d.kw * in.c;
-            void* wbuf = nullptr;
-            if (cudaMalloc(&wbuf, (size_t)wvals + 256) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+            void* wbuf = net_alloc(net, (size_t)wvals, i);
+            if (!wbuf) { st = HQ_ERR_WORKSPACE; break; }
             net->wgt_widened[i] = wbuf;
             if (hq_launch_widen_weights(d.w, wvals, wbuf, h->sm_count, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
           } else if (hq_conv_s2d_applies(a)) {
             const size_t need = hq_conv_s2d_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
             net->launches += 2;                 // weight re-layout + space-to-depth kernels
-          } else if (!hq_conv_tc_supported(a) && hq_conv_lowering_applies(a)) {
+          } else if ((!hq_conv_tc_supported(a) || hq_conv_tc_small_im2col(a)) && hq_conv_lowering_applies(a)) {
             const size_t need = hq_conv_lowering_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
             net->launches += 2;                 // weight padding + patch matrix kernels
@@ -385,8 +420,8 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     if (st != HQ_OK) break;
     if (!(o.bits == 4 || o.bits == 8 || o.bits == 32) || o.c < 1 || (o.bits == 4 && (o.c & 1))) { st = HQ_ERR_INVALID_ARG; break; }
     net->bytes[i] = tensor_bytes(o.n, o.h, o.w, o.c, o.bits);
-    void* buf = nullptr;
-    if (cudaMalloc(&buf, (size_t)net->bytes[i] + 256) != cudaSuccess) { st = HQ_ERR_WORKSPACE; break; }
+    void* buf = net_alloc(net, (size_t)net->bytes[i], i);
+    if (!buf) { st = HQ_ERR_WORKSPACE; break; }
     o.data = buf;
     net->outs[i] = o;
   }
@@ -409,18 +444,19 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     }
     if (!ok) continue;
     net->stored_wide[i] = 1;
-    cudaFree(net->outs[i].data);
-    void* buf = nullptr;
+    net_free(net, net->outs[i].data);
     const size_t wide = (size_t)net->outs[i].n * net->outs[i].h * net->outs[i].w * net->outs[i].c;
-    if (cudaMalloc(&buf, wide + 256) != cudaSuccess) { cudaGetLastError(); net->outs[i].data = nullptr; st = HQ_ERR_WORKSPACE; break; }
+    void* buf = net_alloc(net, wide, i);
     net->outs[i].data = buf;
+    if (!buf) { st = HQ_ERR_WORKSPACE; break; }
     for (int j = i + 1; j < n_layers; ++j)
       if (net->layers[j].in0 == i) net->launches -= 1;        // no activation-widening kernel ahead of this conv
   }
   if (st == HQ_OK && net->scratch_bytes) {
     const size_t want = net->scratch_bytes;
     net->scratch_bytes = 0;
-    if (cudaMalloc(&net->scratch, want) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; }
+    net->scratch = net_alloc(net, want, -1);
+    if (!net->scratch) st = HQ_ERR_WORKSPACE;
     else net->scratch_bytes = want;
   }
   // narrow residual pairs of every conv with a fused 8-bit residual (a one-off search per channel)
@@ -428,8 +464,8 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     const hq_layer& l = net->layers[i];
     if (l.op != HQ_OP_CONV || l.in1 < 0 || net->outs[l.in1].bits != 8 || net->outs[i].bits == 32) continue;
     if (!l.conv.res_rescale.b || !l.conv.res_rescale.c) continue;
-    void* buf = nullptr;
-    if (cudaMalloc(&buf, (size_t)l.conv.cout * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+    void* buf = net_alloc(net, (size_t)l.conv.cout * 16, i);
+    if (!buf) { st = HQ_ERR_WORKSPACE; break; }
     net->res_narrow[i] = buf;
     if (hq_launch_residual_narrow(l.conv.res_rescale.b, l.conv.res_rescale.c, net->outs[l.in1].is_signed, l.conv.cout,
                                   buf, nullptr) != cudaSuccess) st = HQ_ERR_CUDA;
@@ -443,13 +479,13 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     const int ch = net->outs[i].c;
     if (bits0 != 8 || !l.rescale0.b || !l.rescale0.c) continue;
     if (l.op == HQ_OP_ADD && (l.in1 < 0 || net->outs[l.in1].bits != 8 || !l.rescale1.b || !l.rescale1.c)) continue;
-    void* buf = nullptr;
-    if (cudaMalloc(&buf, (size_t)ch * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+    void* buf = net_alloc(net, (size_t)ch * 16, i);
+    if (!buf) { st = HQ_ERR_WORKSPACE; break; }
     net->narrow0[i] = buf;
     if (hq_launch_residual_narrow(l.rescale0.b, l.rescale0.c, sgn0, ch, buf, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
     if (l.op == HQ_OP_ADD) {
-      void* buf1 = nullptr;
-      if (cudaMalloc(&buf1, (size_t)ch * 16) != cudaSuccess) { cudaGetLastError(); st = HQ_ERR_WORKSPACE; break; }
+      void* buf1 = net_alloc(net, (size_t)ch * 16, i);
+      if (!buf1) { st = HQ_ERR_WORKSPACE; break; }
       net->narrow1[i] = buf1;
       if (hq_launch_residual_narrow(l.rescale1.b, l.rescale1.c, net->outs[l.in1].is_signed, ch, buf1, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
     }
@@ -586,13 +622,27 @@ hq_status hq_network_launch_count(const hq_network* net, int32_t* launches) {
 hq_status hq_network_destroy(hq_network* net) {
   if (!net) return HQ_ERR_INVALID_ARG;
   for (auto& g : net->graphs) cudaGraphExecDestroy(g.exec);
-  for (auto& t : net->outs) if (t.data) cudaFree(t.data);
-  for (void* q : net->res_narrow) if (q) cudaFree(q);
-  for (void* q : net->wgt_widened) if (q) cudaFree(q);
-  for (void* q : net->narrow0) if (q) cudaFree(q);
-  for (void* q : net->narrow1) if (q) cudaFree(q);
-  if (net->scratch) cudaFree(net->scratch);
+  for (auto& b : net->buffers) cudaFree(b.base);
   delete net;
+  return HQ_OK;
+}
+
+hq_status hq_network_check_guards(const hq_network* net, void* stream, int32_t* bad_layer) {
+  if (!net) return HQ_ERR_INVALID_ARG;
+  if (bad_layer) *bad_layer = -2;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HQ_ERR_CUDA;
+  unsigned char band[2 * kGuardBytes];
+  for (const auto& b : net->buffers) {
+    const unsigned char* base = (const unsigned char*)b.base;
+    if (cudaMemcpy(band, base, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(band + kGuardBytes, base + kGuardBytes + b.bytes, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return HQ_ERR_CUDA;
+    for (size_t k = 0; k < 2 * kGuardBytes; ++k)
+      if (band[k] != (unsigned char)kGuardByte) {
+        if (bad_layer) *bad_layer = b.layer;
+        return HQ_ERR_RANGE;
+      }
+  }
   return HQ_OK;
 }
 

@@ -82,7 +82,10 @@ struct EltArgs {
 cudaError_t hq_launch_conv_cuda_core(const ConvArgs& a, cudaStream_t s);
 bool hq_conv_tc_init();
 bool hq_conv_tc_supported(const ConvArgs& a);
-// Tensor-core path; returns HQ_OK, HQ_ERR_UNSUPPORTED or HQ_ERR_CUDA.
+// True for a layer the direct kernel declines although its shape is supported: it would fetch a tensor below
+// 128 KiB through an im2col-mode map.  Such a layer runs in its lowered (patch-matrix) form.
+bool hq_conv_tc_small_im2col(const ConvArgs& a);
+// Tensor-core path; returns HQ_OK, HQ_ERR_UNSUPPORTED (nothing was launched) or HQ_ERR_CUDA.
 hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t s);
 // Fills `out` (channels x 16 bytes) with the narrow residual pairs of an 8-bit residual branch.
 cudaError_t hq_launch_residual_narrow(const int32_t* rb, const int32_t* rc, int res_signed, int channels, void* out,

@@ -1,8 +1,11 @@
-// Lowering of convolutions whose channel count does not fit the tensor-core kernel's 32-byte K
-// blocks (the 3-channel first layer): the patches of Eq. 3 are written once as rows of a dense
+// Lowering of convolutions that the direct tensor-core kernel does not take: channel counts that do not
+// fit its 32-byte K blocks (the 3-channel first layer), and layers whose activation tensor is too small for
+// an im2col-mode tensor map (below 128 KiB).  The patches of Eq. 3 are written once as rows of a dense
 // matrix [pixels][Kp] with Kp = kh*kw*cin rounded up to 32 and zero-filled, the weights likewise
 // as [cout][Kp]; the contraction then runs as a 1x1 convolution on the tensor-core kernel.  The
 // zero columns add nothing to the INT32 accumulator, so the result is unchanged.
+#include <mutex>
+
 #include "hq_internal.cuh"
 
 namespace {
@@ -67,7 +70,7 @@ __global__ void pad_weights_kernel(const unsigned char* __restrict__ wgt, int co
 bool hq_conv_lowering_applies(const ConvArgs& a) {
   if (a.in_bits != 8) return false;
   const long long K = (long long)a.kh * a.kw * a.cin;
-  if (K > 4096) return false;                                // meant for thin first layers
+  if (K > 16384) return false;                               // meant for thin first layers and small late layers
   const int wseg = a.wo < 64 ? a.wo : 64;
   if ((long long)a.kh * ((wseg - 1) * a.stride + a.kw) * a.cin > 48 * 1024) return false;   // window must fit shared memory
   ConvArgs t = a;
@@ -213,7 +216,8 @@ bool hq_conv_s2d_applies(const ConvArgs& a) {
   if (a.in_bits != 8 || a.cin != 3 || a.kh != 7 || a.kw != 7 || a.stride != 2 || a.pad != 3) return false;
   if ((a.h & 1) || (a.w & 3) || a.pitch_w || a.res || a.out_bits != 8) return false;       // pairs of outputs: w/2 even
   if ((long long)a.cout * 1024 >= (1ll << 31)) return false;
-  return hq_conv_tc_supported(s2d_conv_args(a, a.in));
+  const ConvArgs t = s2d_conv_args(a, a.in);
+  return hq_conv_tc_supported(t) && !hq_conv_tc_small_im2col(t);   // small images take the patch-matrix form
 }
 
 size_t hq_conv_s2d_bytes(const ConvArgs& a) { return (size_t)s2d_layout(a).total; }
@@ -303,9 +307,17 @@ bool hq_conv_widen4_applies(const ConvArgs& a) {
   return hq_conv_tc_supported(t);
 }
 
-size_t hq_conv_widen4_bytes(const ConvArgs& a) {
+static size_t widen4_copy_bytes(const ConvArgs& a) {
   const long long x = (long long)a.n * a.h * a.w * a.cin, w = (long long)a.cout * a.kh * a.kw * a.cin;
   return (size_t)(((x + 255) / 256 + (w + 255) / 256) * 256);
+}
+
+// the widened copies, plus the patch matrix when the widened layer is one the direct kernel declines
+size_t hq_conv_widen4_bytes(const ConvArgs& a) {
+  ConvArgs t = a;
+  t.in_bits = 8;
+  const bool lowered = hq_conv_tc_small_im2col(t) && hq_conv_lowering_applies(t);
+  return widen4_copy_bytes(a) + (lowered ? hq_conv_lowering_bytes(t) : 0);
 }
 
 // `scratch` must hold hq_conv_widen4_bytes(a) bytes, 256-byte aligned.
@@ -317,7 +329,9 @@ hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, 
   if (!a.wgt_widened && launch_widen4(a.wgt, w, 1, ww, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
   ConvArgs t = a;
   t.in = xw; t.wgt = a.wgt_widened ? a.wgt_widened : ww; t.in_bits = 8;
-  return hq_launch_conv_tc(h, t, s);
+  const hq_status st = hq_launch_conv_tc(h, t, s);
+  if (st != HQ_ERR_UNSUPPORTED || !hq_conv_lowering_applies(t)) return st;
+  return hq_launch_conv_lowered(h, t, xw + widen4_copy_bytes(a), s);      // declined by the direct kernel: patch matrix
 }
 
 cudaError_t hq_launch_pack4(const void* in, long long values, void* out, int sm_count, cudaStream_t s) {
@@ -352,8 +366,10 @@ namespace {
 struct NoAllocDevice { bool ready; void* scratch; uint32_t* status; int sm_count; };
 constexpr int kMaxDevices = 64;
 NoAllocDevice g_noalloc_dev[kMaxDevices];
+std::mutex g_noalloc_mutex;     // first calls from several host threads: one of them fills the record, the others wait
 
 hq_status noalloc_setup(int dev) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
   NoAllocDevice& d = g_noalloc_dev[dev];
   if (d.ready) return HQ_OK;
   int major = 0, sms = 0;
@@ -405,7 +421,7 @@ extern "C" hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* 
       a.res = r->data; a.res_bits = r->bits; a.res_signed = r->is_signed; a.rb = d->res_rescale.b; a.rc = d->res_rescale.c;
     }
   }
-  if (!hq_conv_lowering_applies(a)) return HQ_ERR_UNSUPPORTED;
+  if ((long long)d->kh * d->kw * d->cin > 4096 || !hq_conv_lowering_applies(a)) return HQ_ERR_UNSUPPORTED;
   if (hq_conv_lowering_bytes(a) > (size_t)HQ_NOALLOC_SCRATCH_BYTES) return HQ_ERR_WORKSPACE;   // beyond the fixed array
 
   int dev = -1;
@@ -423,4 +439,17 @@ extern "C" hq_status hq_conv2d_noalloc(const hq_tensor* in, const hq_conv_desc* 
   tmp.device = dev; tmp.conv_path = 0; tmp.sm_count = nd.sm_count; tmp.dev_status = nd.status;
   tmp.workspace = nullptr; tmp.workspace_bytes = 0;
   return hq_launch_conv_lowered(&tmp, a, nd.scratch, s);
+}
+
+// Wait for `stream` and report an expired device-side wait of the hq_conv2d_noalloc calls queued on it.
+extern "C" hq_status hq_conv2d_noalloc_sync(void* stream) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HQ_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return HQ_ERR_UNSUPPORTED;
+  const hq_status st = noalloc_setup(dev);
+  if (st != HQ_OK) return st;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HQ_ERR_CUDA;
+  uint32_t word = 0;
+  if (cudaMemcpy(&word, g_noalloc_dev[dev].status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return HQ_ERR_CUDA;
+  return word != 0 ? HQ_ERR_TIMEOUT : HQ_OK;
 }

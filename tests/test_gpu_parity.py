@@ -90,6 +90,16 @@ TC_CASES = [
     (1, 20, 20, 128, 256, 3, 1, 1, 8, True, 8, True),        # residual + 3x3 + two N tiles of 128
     (3, 8, 8, 64, 64, 1, 1, 0, 4, True, 8, True),            # uint4 output with residual
     (2, 16, 16, 32, 128, 1, 1, 0, 4, False, 8, True),        # uint4 output, 64-byte store boxes
+    # the same kinds of geometry on tensors of at least 128 KiB, which the direct kernel fetches through im2col-mode
+    # tensor maps (smaller ones, above, take the patch-matrix form); the last two straddle the threshold
+    (6, 30, 26, 64, 96, 3, 2, 1, 8, False, 8, True),         # stride 2, odd extents, N tail
+    (3, 28, 28, 64, 128, 1, 2, 0, 8, False, 8, False),       # strided 1x1, signed output
+    (8, 24, 24, 32, 72, 3, 1, 1, 32, False, 8, False),       # 32-byte K blocks, INT32 output
+    (4, 19, 19, 96, 40, 5, 1, 2, 8, False, 8, True),         # 5x5, pad 2, direct stores
+    (4, 24, 24, 64, 64, 3, 1, 1, 4, False, 8, True),         # uint4 output
+    (3, 20, 20, 128, 256, 3, 1, 1, 8, True, 8, True),        # residual + 3x3 + two N tiles
+    (2, 32, 32, 64, 64, 3, 1, 1, 8, False, 8, True),         # exactly 128 KiB: im2col mode
+    (2, 32, 31, 64, 64, 3, 1, 1, 8, False, 8, True),         # 124 KiB: patch-matrix form
     # large enough for the benchmark's launch shapes (the pixel tile grows with the number of tiles per SM)
     (33, 56, 56, 64, 64, 1, 1, 0, 8, False, 8, True),        # 256-pixel tiles, folded 64-channel tile, ragged last tile
     (13, 56, 56, 64, 64, 3, 1, 1, 8, True, 8, True),         # 128-pixel tiles, four accumulator buffers, folded, residual
@@ -620,10 +630,11 @@ def run_network_and_compare(hq, table, batch, seed):
     net = binding.Network(hq, table, batch)
     try:
         d_img = binding.to_device(images)
-        logits = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+        logits = binding.alloc_out(*net.logits_shape, 32, 1)
         taps = net.alloc_taps()
         assert net.run(d_img, logits, taps) == binding.HQ_OK
         hq.sync()
+        net.check_guards()           # no kernel wrote outside a buffer the network owns
         for i, (t, r) in enumerate(zip(taps, ref)):
             got = t.cpu().numpy().view(r.dtype).reshape(r.shape)
             assert np.array_equal(got, r), f"layer {i} ({table['layers'][i]['op']}) differs in {(got != r).sum()} of {r.size}"
@@ -636,6 +647,7 @@ def run_network_and_compare(hq, table, batch, seed):
                 assert net.run(d_img, logits, None) == binding.HQ_OK
                 hq.sync()
                 assert np.array_equal(host(logits, ref[-1]), ref[-1])
+        net.check_guards()
     finally:
         net.close()
     return ref
@@ -692,36 +704,50 @@ def test_resnet18_imagenet_shape_batch8_every_layer(hq):
     assert min(sat) < 0.9, "every layer is saturated: the workload would not exercise the requantization"
 
 
-def test_resnet50_batch256_benchmark_configuration_sampled_images(hq):
+def test_resnet50_batch256_benchmark_configuration_every_image(hq):
     """The benchmark workloads themselves (ResNet-50, 224x224, batch 256, INT8 and mixed INT4/8), in the launch
     configuration bench.py times: tile sizes, folded channel tiles, the two-CTA shape and the number of
-    accumulator buffers all depend on the batch.  Images are independent, so the oracle runs the first two and
-    the last image of the batch and every layer's output for those images must match bit for bit."""
+    accumulator buffers all depend on the batch.  Images are independent, so the batch is made of four distinct
+    images dealt over the 256 positions in an irregular order; the oracle runs the four, and EVERY layer's output
+    for EVERY one of the 256 positions must equal the oracle's output for the image at that position (compared
+    on the device), as must the logits of the graph-replay path that the benchmark times."""
     from oracle.network import run_network
     from paper_2011_10680_b200 import binding
-    batch, pick = 256, [0, 1, 255]
+    batch, distinct = 256, 4
+    order = np.array([(7 * i + i // 5 + (i * i) // 11) % distinct for i in range(batch)])
+    assert len(set(order.tolist())) == distinct and order[0] != order[1] and order[-1] != order[-2]
+    order_d = torch.from_numpy(order).cuda()
     for mixed, seed in ((False, 3), (True, 4)):
         t = inputs.resnet_table(50, seed, mixed=mixed)
-        images = inputs.random_images(seed, batch, t["image_hw"])
-        ref = run_network(t, images[pick])
+        base = inputs.random_images(seed, distinct, t["image_hw"])
+        ref = run_network(t, base)
         net = binding.Network(hq, t, batch)
         try:
-            d_img = binding.to_device(images)
-            logits = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
+            d_img = binding.to_device(base[order])
+            logits = binding.alloc_out(*net.logits_shape, 32, 1)
             taps = net.alloc_taps()
             assert net.run(d_img, logits, taps) == binding.HQ_OK
             hq.sync()
+            net.check_guards()
             for i, (tap, r) in enumerate(zip(taps, ref)):
                 per_image = tap.numel() // batch
-                got = tap.view(batch, per_image)[pick].cpu().numpy()
-                want = np.ascontiguousarray(r).view(np.uint8).reshape(len(pick), per_image)
-                assert np.array_equal(got, want), f"mixed={mixed} layer {i} ({t['layers'][i]['op']}) differs in {(got != want).sum()} bytes"
+                want = torch.from_numpy(np.ascontiguousarray(r).view(np.uint8).reshape(distinct, per_image)).cuda()
+                got = tap.view(batch, per_image)
+                if not torch.equal(got, want[order_d]):
+                    bad = (got != want[order_d]).any(dim=1).nonzero().flatten().tolist()
+                    raise AssertionError(f"mixed={mixed} layer {i} ({t['layers'][i]['op']}) differs at batch positions {bad[:8]} ({len(bad)} of {batch})")
+                del want
             # the graph-replay path that the benchmark times
             logits.zero_()
-            assert net.run(d_img, logits, None) == binding.HQ_OK
-            hq.sync()
-            assert np.array_equal(logits.cpu().numpy().reshape(batch, -1)[pick], ref[-1].reshape(len(pick), -1))
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                assert net.run(d_img, logits, None) == binding.HQ_OK
+                hq.sync()
+            want = ref[-1].reshape(distinct, -1)[order]
+            assert np.array_equal(logits.cpu().numpy().reshape(batch, -1), want)
+            net.check_guards()
             del taps
         finally:
             net.close()
+        binding.check_guards()
         torch.cuda.empty_cache()

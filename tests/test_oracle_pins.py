@@ -424,6 +424,19 @@ def test_oracle_source_has_no_float_and_no_division():
     oracle_build.check_no_float_codegen()
 
 
+def test_no_float_compile_pass_rejects_a_double(tmp_path):
+    """The compile pass above is not vacuous: the same command refuses a translation unit that touches a
+    floating-point register, and accepts the same function written with integers."""
+    import subprocess
+    bad = tmp_path / "uses_double.cpp"
+    bad.write_text("extern \"C\" long long scale(long long x) { return (long long)((double)x * 0.5); }\n")
+    with pytest.raises(subprocess.CalledProcessError):
+        oracle_build.check_no_float_codegen(str(bad))
+    good = tmp_path / "integers_only.cpp"
+    good.write_text("extern \"C\" long long scale(long long x) { return x >> 1; }\n")
+    oracle_build.check_no_float_codegen(str(good))
+
+
 # ---------------------------------------------------------------- P11: fused == unfused ---------
 def test_fused_conv_residual_equals_int32_conv_then_residual_add():
     case = inputs.conv_case(31, 2, 6, 6, 8, 8, 3, 1, 1, bits=8, residual=True, c_range=(39, 43))
@@ -447,21 +460,135 @@ def test_range_error_is_reported_not_wrapped():
 
 
 # ---------------------------------------------------------------- network walk ------------------
-def test_small_resnet_walk_is_consistent_layer_by_layer():
-    """The network walk equals calling the layer functions by hand (checked on a reduced ResNet-18),
-    and the mixed-precision table feeds uint4 tensors to its 4-bit convs."""
-    t = inputs.resnet_table(18, seed=3, image_hw=32, classes=10, width=8, mixed=True)
-    img = inputs.random_images(3, 2, 32)
+def hand_walk(table, images):
+    """Every layer of a table applied by hand, without oracle.network: the operands are looked up from the
+    table's own wiring (in0, in1, and the bits / sign the PRODUCING layer declares), the arithmetic is the
+    independent formulations above (patch matrix + int64 product, exact rational rounding, exact mean, padded
+    numpy maximum).  Returns the list of outputs as int64 arrays of logical (unpacked) values."""
+    layers = table["layers"]
+    vals = {-1: images.astype(np.int64)}
+
+    def kind(i):                                   # (bits, signed) of tensor i as its producer states them
+        return (8, 0) if i == -1 else (layers[i]["out_bits"], layers[i]["out_signed"])
+
+    def dn_exact(x, b, c):
+        return exact_round_half_up(int(x) * int(b), int(c))
+
+    for li, l in enumerate(layers):
+        op, x = l["op"], vals[l["in0"]]
+        if op in ("conv", "linear"):
+            bits_in, _ = kind(l["in0"])
+            assert bits_in == l["bits"], "Section 3.4: weights and activations of a layer share the bit-width"
+            wt = (inputs.unpack4(l["wgt"], True) if l["bits"] == 4 else l["wgt"]).astype(np.int64)
+            if op == "linear":
+                x = x.reshape(x.shape[0], 1, 1, -1)
+            acc = im2col_conv(x, wt, l["stride"], l["pad"])
+            if l["out_bits"] == 32:
+                y = acc + l["bias"].astype(np.int64)
+            else:
+                res = vals[l["in1"]] if l["in1"] >= 0 else None
+                y = epilogue_exact(acc, l["bias"], l["b"], l["c"], res, l["rb"], l["rc"], l["relu"], l["qmin"], l["qmax"])
+        elif op == "maxpool":
+            k, st, pad = l["pool_k"], l["pool_stride"], l["pool_pad"]
+            lowest = -128 if kind(l["in0"])[1] else 0
+            xp = np.pad(x, ((0, 0), (pad, pad), (pad, pad), (0, 0)), constant_values=lowest)
+            ho, wo = (x.shape[1] + 2 * pad - k) // st + 1, (x.shape[2] + 2 * pad - k) // st + 1
+            y = np.stack([np.stack([xp[:, oh * st:oh * st + k, ow * st:ow * st + k].max(axis=(1, 2))
+                                    for ow in range(wo)], axis=1) for oh in range(ho)], axis=1)
+        elif op == "avgpool":
+            s = x.sum(axis=(1, 2))
+            y = np.zeros((x.shape[0], 1, 1, x.shape[3]), np.int64)
+            for n in range(x.shape[0]):
+                for ch in range(x.shape[3]):
+                    y[n, 0, 0, ch] = min(max(dn_exact(s[n, ch], l["b"][ch], l["c"][ch]), l["qmin"]), l["qmax"])
+        elif op in ("requant", "add"):
+            y = np.zeros(x.shape, np.int64)
+            r = vals[l["in1"]] if l["in1"] >= 0 else None
+            it = np.nditer(y, flags=["multi_index"])
+            for _ in it:
+                idx = it.multi_index
+                ch = idx[-1]
+                v = dn_exact(x[idx], l["b"][ch], l["c"][ch])
+                if r is not None:
+                    v += dn_exact(r[idx], l["rb"][ch], l["rc"][ch])
+                if l["relu"]:
+                    v = max(v, 0)
+                y[idx] = min(max(v, l["qmin"]), l["qmax"])
+        else:
+            raise AssertionError(op)
+        vals[li] = y
+    return [vals[i] for i in range(len(layers))]
+
+
+def logical(y, layer):
+    """An oracle output as int64 logical values (4-bit tensors unpacked)."""
+    if layer["out_bits"] == 4:
+        return inputs.unpack4(y, bool(layer["out_signed"])).astype(np.int64)
+    return y.astype(np.int64)
+
+
+@pytest.mark.parametrize("depth,mixed,hw", [(18, False, 32), (18, True, 32), (50, True, 32), (50, False, 32)])
+def test_network_walk_equals_layers_applied_by_hand(depth, mixed, hw):
+    """EVERY layer of reduced ResNet-18 / ResNet-50 tables (uniform and mixed 4/8 bit): the oracle's walk against
+    the hand-applied layers.  A wrong residual operand, a swapped bits / sign lookup for in0 and in1, or a slip
+    in the requant / add / pooling / linear branches of the walk changes some layer here."""
+    t = inputs.resnet_table(depth, seed=3 + depth, image_hw=hw, classes=10, width=8, mixed=mixed)
+    img = inputs.random_images(3, 2, hw)
     outs = run_network(t, img)
+    want = hand_walk(t, img)
+    seen = set()
+    for i, (l, y, w) in enumerate(zip(t["layers"], outs, want)):
+        assert np.array_equal(logical(y, l).reshape(w.shape), w), (i, l["op"])
+        seen.add(l["op"])
+        if l["op"] == "conv" and l["in1"] >= 0:
+            seen.add("residual")
+            if l["in1"] != i - 1:
+                seen.add("residual from further back")
+            if t["layers"][l["in1"]]["out_signed"] != t["layers"][l["in0"]]["out_signed"]:
+                seen.add("operands of different sign")
+    need = {"conv", "linear", "maxpool", "avgpool", "residual", "residual from further back", "operands of different sign"}
+    if mixed:
+        need.add("requant")
+    assert need <= seen, need - seen
+    # outputs are not degenerate: the logits differ between the two images and between classes
+    assert len(np.unique(outs[-1])) > 5
     assert outs[-1].dtype == np.int32 and outs[-1].shape == (2, 1, 1, 10)
-    l0 = t["layers"][0]
-    acc = im2col_conv(img.astype(np.int64), l0["wgt"].astype(np.int64), 2, 3)
-    ref0 = epilogue_exact(acc, l0["bias"], l0["b"], l0["c"], None, None, None, 1, 0, 255)
-    assert np.array_equal(outs[0].astype(np.int64), ref0)
-    n4 = sum(1 for l in t["layers"] if l["op"] == "conv" and l["bits"] == 4)
-    assert n4 > 0
     for i, l in enumerate(t["layers"]):
         if l["op"] == "conv" and l["bits"] == 4:
             assert t["bits"][l["in0"]] == 4
         h, w, c = t["shapes"][i]
         assert outs[i].shape[1:3] == (h, w)
+
+
+def _tiny_network():
+    import importlib.util
+    spec = importlib.util.spec_from_file_location(
+        "make_network_walk_golden", os.path.join(os.path.dirname(__file__), "golden", "make_network_walk_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def test_tiny_network_matches_stored_values_and_hand_walk(golden_dir):
+    """A six-layer table typed in by hand (residual operand = layer 0, two layers back; a signed tensor feeding a
+    conv and an add; average pool; INT32 logits): the oracle's walk equals the stored per-layer values AND the
+    hand-applied layers."""
+    mod = _tiny_network()
+    table, img = mod.tiny_table(), mod.tiny_images()
+    outs = run_network(table, img)
+    stored = {}
+    for line in open(os.path.join(golden_dir, "network_walk_tiny.txt")):
+        if line.startswith("layer"):
+            head, vals = line.split(":")
+            stored[int(head.split()[1])] = np.array([int(v) for v in vals.split()], np.int64)
+    want = hand_walk(table, img)
+    assert len(stored) == len(outs) == 6
+    for i, y in enumerate(outs):
+        assert np.array_equal(y.astype(np.int64).ravel(), stored[i]), i
+        assert np.array_equal(y.astype(np.int64).ravel(), want[i].ravel()), i
+    # the residual really comes from layer 0: feeding layer 1 (the previous layer) instead changes layer 2
+    wrong = mod.tiny_table()
+    wrong["layers"][2]["in1"] = 1
+    assert not np.array_equal(run_network(wrong, img)[2], outs[2])
+    # first value of layer 2 by hand: acc = 2*(-9) - 16 + 0 + 3*14 = 8; (8 + 5) * 0.046875 = 0.61 -> 1; 0.7 * 22 = 15.4 -> 15
+    assert int(outs[1].ravel()[0]) == -9 and int(outs[0].ravel()[0]) == 22 and int(outs[2].ravel()[0]) == 16

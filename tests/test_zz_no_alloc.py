@@ -35,8 +35,12 @@ def test_noalloc_conv_matches_the_allocating_entry_point_twice_in_a_row():
             hq.sync()
             got = binding.alloc_out(n, case["ho"], case["wo"], cout, case["out_bits"], case["out_signed"])
             got.fill_(0x5A if got.dtype == torch.uint8 else 0)      # stale bytes must not survive
-            assert binding.conv2d_noalloc(case, dev, got) == binding.HQ_OK
             torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            assert binding.conv2d_noalloc(case, dev, got) == binding.HQ_OK
+            assert binding.conv2d_noalloc_sync() == binding.HQ_OK   # no bounded device wait ran out
+            if i > 0:                                               # the first call loads the library's kernels
+                assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
             assert torch.equal(got, want), f"call {i}: results differ from hq_conv2d"   # integers: bit-exact
             from oracle import hqref
             ref = hqref.conv_case(case)
