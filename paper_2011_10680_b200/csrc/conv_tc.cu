@@ -52,8 +52,9 @@ constexpr int kMaxAccBufs = 4;                                 // accumulator (a
 //   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
 //         reduction are bound by the latency of the hand-over chain between the MMA issuer and the epilogue
 //         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
-//   wide  16 epilogue warps and one issuer, one CTA per SM: fused-residual layers on 256-pixel tiles (the longest
-//         epilogue chain per value gains from four warps per scheduler; the loop keeps one chunk in registers).
+//   rtm   ("residual through tensor memory") 8 epilogue warps, one issuer and a store warp, one CTA per SM, 128-pixel
+//         tiles: fused 8-bit residuals with a short reduction.  The residual tile is transposed and widened by an MMA
+//         with the identity matrix, the epilogue works on 16 x 8 fragments and writes with transposing matrix stores.
 //   duo   the solo roles in clusters of two CTAs that share every MMA (cta_group::2): long reductions whose weights
 //         stream; each CTA fetches its own weight rows and half of the pixel rows.
 constexpr int kSoloEpilogueWarps = 8;
@@ -77,6 +78,11 @@ struct TcParams {
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
   int32_t inplace;       // 1: the sixteen-warp shape: outputs overwrite the residual tile, which is stored as the box
+  int32_t rtm;           // 1: the 8-bit residual tile reaches the epilogue through tensor memory: an MMA with the identity
+                         //    matrix as its A operand turns the [pixels][128 channels] byte tile into INT32 columns beside
+                         //    the accumulator, in the accumulator's own layout (see epilogue_loop_frag)
+  int32_t acc_stride;    // tensor-memory columns between accumulator buffers: pt, or 2 * pt with rtm
+  uint32_t ident_off;    // rtm: offset of the 128 x 128 identity matrix (16 KiB, 128-byte swizzle) from the 1024-aligned base
   int32_t duo;           // 1: two CTAs of a cluster (adjacent SMs) share every MMA: 256 channels x 256 pixels per pair
   int32_t ni;            // MMA issuer warps in use: min(issuer warps of the launch shape, k_blocks)
   int32_t lg_bufs;       // log2 of the accumulator / residual buffer count: tile t of a CTA uses buffer t mod 2^lg_bufs
@@ -114,6 +120,7 @@ struct SharedCtl {
   unsigned long long tstart[kMaxAccBufs];   // the tile's first (overwriting) MMA has been issued
   unsigned long long rfull[kMaxAccBufs];
   unsigned long long rempty[kMaxAccBufs];
+  unsigned long long ofull[kMaxAccBufs];    // rtm: every epilogue warp has written its pieces of the output tile
   unsigned long long drain;
   unsigned long long wfull;              // resident weight slab landed
   unsigned long long pfull[3], pempty[3];  // strip mode: input patches
@@ -307,6 +314,36 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, int (&v)[32]) {
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 lanes x 32 columns in the layout of an MMA accumulator fragment: thread T (t4 = T / 4, q2 = T % 4) receives, for
+// every group g of eight columns, v[4g + 0/1] = lane t4, columns 8g + 2 q2 + 0/1 and v[4g + 2/3] = lane t4 + 8, same columns.
+__device__ __forceinline__ void tmem_ld_frag16(uint32_t taddr, int (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+// Four 16 x 8 byte matrices, stored transposed: register g of thread T holds, in byte order, the elements
+// (m, n) = (t4, 2 q2), (t4, 2 q2 + 1), (t4 + 8, 2 q2), (t4 + 8, 2 q2 + 1) of matrix g -- the byte-packed form of the
+// fragment above -- and matrix g's column n becomes the 16 contiguous bytes at the address thread 8 g + n supplies.
+__device__ __forceinline__ void stmatrix_t_x4(uint32_t row_addr, unsigned r0, unsigned r1, unsigned r2, unsigned r3) {
+  asm volatile("stmatrix.sync.aligned.m16n8.x4.trans.shared.b8 [%0], {%1, %2, %3, %4};"
+               ::"r"(row_addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
+// four values -> four bytes (s0 lowest), clamped to the unsigned / signed 8-bit range by two chained saturating packs
+template <bool OSIGNED>
+__device__ __forceinline__ unsigned sat_pack4(int s0, int s1, int s2, int s3) {
+  unsigned w23, w;
+  if (OSIGNED) {
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(s3), "r"(s2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s1), "r"(s0), "r"(w23));
+  } else {
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(s3), "r"(s2), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(s1), "r"(s0), "r"(w23));
+  }
+  return w;
+}
 // Saturating conversion to a byte.  The packing form of the convert (second source -> byte 0) is a single
 // integer-pipe instruction; the plain cvt.sat.u8.s32 measured at twice its issue cost.
 __device__ __forceinline__ int sat_u8(int x) {
@@ -350,9 +387,14 @@ struct ChanConst {
 // RN: every channel of the warp has a narrow residual pair (m, a, s) with (r*m + a) >> s equal to the residual
 // term for all 256 values of r (found and checked exhaustively by residual_narrow_kernel); rb / rh / rsh hold
 // m / a / s then, and a 32-bit multiply-add replaces the shift, multiply-high and add.
-template <bool RES, bool RSIGNED, bool SMALL, bool RN = false>
+// SPELLED: the product is written as the 32 x 32 -> 64 multiply-add instruction it is.  In the fragment loop, left
+// to the compiler, the sign extension of k.b is hoisted out of the loop and the product becomes a full 64 x 64
+// multiply (three to four multiply instructions per value); the other loops compile to the short form by themselves.
+template <bool RES, bool RSIGNED, bool SMALL, bool RN = false, bool SPELLED = false>
 __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) {
-  const long long t1 = (long long)acc * (long long)k.b + k.r0;
+  long long t1;
+  if (SPELLED) asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(t1) : "r"(acc), "r"(k.b), "l"(k.r0));
+  else t1 = (long long)acc * (long long)k.b + k.r0;
   int s;
   if (!SMALL) {
     s = (int)(t1 >> 32) >> k.sh;                       // c >= 32: |s| < 2^30
@@ -537,77 +579,153 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
   if (lane == 0) tma_store_wait_all();
 }
 
-// The same arithmetic for the launch shape with sixteen epilogue warps (four per scheduler): no second register
-// set for the next chunk -- with four warps per scheduler the tensor-memory load of one warp hides behind the
-// arithmetic of the others -- which keeps the loop inside that shape's register budget.  This shape always carries
-// an 8-bit residual through the prefetched tile, and it works IN PLACE: a thread overwrites each residual byte
-// with the output value computed from it, so the [pixels][128 channels] residual tile doubles as the staging box
-// (no separate box: room for one more stage, and the store moves whole 128-byte rows).  The four warps that share
-// 64 pixel columns (one per channel quarter) meet at a named barrier, then one of them stores the columns' box and
-// hands the residual buffer back once the store has read it -- after the first chunk of the next tile, when that
-// read has long finished, unless there is only one buffer.
-template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN>
-__device__ __forceinline__ void epilogue_loop_lean8(const EpiCtx& e_in, const ChanConst& k_in) {
-  if constexpr (RES) {
-    const EpiCtx e = e_in;
-    const ChanConst k = k_in;
-    const TcParams& p = *e.p;
-    SharedCtl& ctl = *e.ctl;
-    const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
-    uint8_t* const res_stage_ptr = e.smem_raw + (e.res_stage - e.raw);
-    const int nchunks = px_per_warp >> 5;
-    const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
-    const uint32_t t_warp = e.tmem_base + ((uint32_t)(q * 32) << 16) + col0;
-    const bool leader = q == 0;                     // the warp of its four that stores the box
-    auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
-      uint32_t w = 1;
-      if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
-      return __shfl_sync(0xffffffffu, w, 0) != 0;
-    };
-    uint32_t tcount = 0, owed_rs = 0;
-    bool owe = false;                               // leader: the previous tile's residual buffer is still to be handed back
-    for (int p_tile = e.p_tile0; p_tile < p.p_tiles; p_tile += e.p_step, ++tcount) {
-      const uint32_t as = tcount & bmask, aph = (tcount >> p.lg_bufs) & 1u;
-      const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
-      if (!wait_bar(&ctl.tfull[as], aph)) break;
-      if (!wait_bar(&ctl.rfull[rs], rph)) break;
-      tc_fence_after();
-      const uint32_t box_off = rs * e.res_tile_bytes + (uint32_t)col0 * kTileC;      // the four warps' 64 rows of 128 bytes
-      uint8_t* const mine = res_stage_ptr + box_off + cq * 32 + lane;
-      for (int c = 0; c < nchunks; ++c) {
-        int v[32];
-        tmem_ld32(t_warp + as * p.pt + c * 32, v);
-        if (c == 0 && owe) {
-          if (lane == 0) { tma_store_wait_read0(); mbar_arrive(smem_u32(&ctl.rempty[owed_rs])); }
-          owe = false;
-        }
-        if (e.warp_live) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int r = RSIGNED ? (int)(signed char)mine[(c * 32 + j) * kTileC] : (int)mine[(c * 32 + j) * kTileC];
-            const int s = requant_fast<true, RSIGNED, SMALL, RN>(v[j], r, k);
-            v[j] = SAT ? (OSIGNED ? sat_s8(s) : sat_u8(s)) : min(max(s, e.lo), e.hi);
-          }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) mine[(c * 32 + j) * kTileC] = (uint8_t)v[j];
-        }
-      }
-      tc_fence_before();
-      fence_async_smem();                           // make this lane's box writes visible to the TMA engine
-      __syncwarp();
-      if (lane == 0) release_accumulator(p, ctl, as);
-      asm volatile("bar.sync %0, 128;" :: "r"(2 + e.half) : "memory");
-      if (leader) {
-        if (lane == 0) {
-          const int p_base = p_tile * p.pt + col0;
-          if (p_base < p.P) { tma_store_2d(e.map_out, e.res_stage + box_off, e.c_tile * kTileC, p_base); tma_store_commit(); }
-          if (rmask == 0) { tma_store_wait_read0(); mbar_arrive(smem_u32(&ctl.rempty[rs])); }
-        }
-        owe = rmask != 0; owed_rs = rs;
-      }
-    }
-    if (leader && lane == 0) tma_store_wait_all();
+// Per-channel constants of one output channel (Eq. 4 and the residual rescale of Section 3.3), as the loops below want
+// them: `fast` selects the 32-bit forms (see requant_fast), `narrow` the checked narrow residual pair of the channel.
+__device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, bool fast, bool narrow) {
+  ChanConst k{};
+  const bool live = ch < p.C;
+  k.bias = (live && p.bias) ? p.bias[ch] : 0;
+  k.b = live ? p.b[ch] : 0;
+  const int cc = live ? p.c[ch] : 32;
+  k.sh = cc;
+  k.r0 = (long long)k.bias * (long long)k.b + (1LL << (cc - 1));
+  if (p.res) {
+    const int rcc = live ? p.rc[ch] : 32;
+    k.rb = live ? p.rb[ch] : 0;
+    k.rsh = rcc;
+    k.rr0 = 1LL << (rcc - 1);
   }
+  if (fast) {
+    k.sh1 = k.sh < 32 ? k.sh : 32;
+    k.cmin31 = k.sh < 31 ? k.sh : 31;
+    k.sh -= k.sh1;
+    if (p.res) {
+      if (k.rsh >= 40) { k.rb = 0; k.rh = 0; k.rsh = 1; }            // |r*rb| < 2^39: rounds to 0
+      else { k.rh = 1 << (k.rsh - 9); k.rsh -= 8; }
+    }
+  }
+  if (narrow) {
+    const int4 nr = live ? p.res_narrow[ch] : make_int4(0, 0, 0, 1);
+    k.rb = nr.x; k.rh = nr.y; k.rsh = nr.z;
+  }
+  return k;
+}
+
+// Tile loop of the launch shape for fused 8-bit residuals (eight epilogue warps and a store warp, 128-pixel tiles).
+//
+// Nothing moves byte by byte here.  The residual tile [128 pixels][128 channels] lands in shared memory by TMA in the
+// 128-byte-swizzled K-major form of an MMA operand, and the MMA issuer multiplies it by the 128 x 128 identity matrix:
+// D2[ch][px] = sum_k I[ch][k] * R[px][k] = R[px][ch], i.e. the tensor core transposes the tile and widens it to INT32
+// in tensor-memory columns next to the accumulator.  An epilogue warp owns 16 accumulator lanes (channels) and reads
+// accumulator and residual with the same 16x256b loads, which hand thread T the values of channels t4, t4 + 8 for
+// pixel pairs -- the fragment of a 16 x 8 matrix.  It applies Eq. 4 and the residual add of Section 3.3 with the
+// constants of its two channels in registers, packs four results into a word with two saturating converts, and one
+// stmatrix (transposing, b8) writes 32 pixels x 16 channels as 16-byte row pieces into the tile the residual came
+// from (the MMA has finished reading it: the accumulator barrier is committed after the identity MMAs).  The loads of
+// the next 32 columns (or of the next tile's first) are in flight while a unit is processed.  Warps do not wait for
+// each other: each arrives on the tile's `ofull` barrier when its pieces are written, and the store warp alone waits
+// there, stores the [128][128] box (128-byte swizzle, as it was loaded) and hands the buffer back.
+// GEN: 64-bit arithmetic for every shift 1..62 (some channel has c < 32 or a residual shift below 9).
+template <bool GEN, bool RSIGNED, bool SAT, bool OSIGNED, bool RN>
+__device__ __forceinline__ void epilogue_loop_frag(const EpiCtx& e_in) {
+  const EpiCtx e = e_in;
+  const TcParams& p = *e.p;
+  SharedCtl& ctl = *e.ctl;
+  const int lane = e.lane, q = e.q, hh = e.half;
+  const int t4 = lane >> 2;
+  ChanConst k[2];                                   // channels 32 q + 16 hh + 8 r + t4, r = 0, 1
+#pragma unroll
+  for (int r = 0; r < 2; ++r) k[r] = chan_const_for(p, e.c_tile * kTileC + 32 * q + 16 * hh + 8 * r + t4, !GEN, RN);
+  const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
+  constexpr int units = 4;                          // 32 pixel columns per unit, 128-pixel tiles
+  const uint32_t t_lane = e.tmem_base + ((uint32_t)(q * 32 + 16 * hh) << 16);
+  // byte offset of this thread's 16-byte piece in a unit's 32 rows: row `lane`, chunk (2 q + hh) ^ (row % 8)
+  const uint32_t row_off = (uint32_t)lane * 128u + ((uint32_t)((2 * q + hh) ^ (lane & 7)) << 4);
+  if (e.p_tile0 >= p.p_tiles) return;
+  auto wait_bar = [&](unsigned long long* bar, uint32_t ph) -> bool {
+    uint32_t w = 1;
+    if (lane == 0) w = mbar_wait(smem_u32(bar), ph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, w, 0) != 0;
+  };
+  auto one = [&](int acc, int r, const ChanConst& c) -> int {
+    if (GEN) {
+      const long long y = (((long long)acc * (long long)c.b + c.r0) >> c.sh) + (((long long)r * (long long)c.rb + c.rr0) >> c.rsh);
+      return hq_clamp_ll(y, p.relu, p.qmin, p.qmax);
+    }
+    const int y = requant_fast<true, RSIGNED, false, RN, true>(acc, r, c);
+    return SAT ? y : min(max(y, e.lo), e.hi);
+  };
+  // one unit: 16 values per thread -> four words -> one transposing store of 32 pixel rows x 16 channel bytes
+  auto unit = [&](const int (&va)[16], const int (&vr)[16], uint32_t tile, int u) {
+    unsigned w[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const int y0 = one(va[4 * g + 0], vr[4 * g + 0], k[0]), y1 = one(va[4 * g + 1], vr[4 * g + 1], k[0]);
+      const int y2 = one(va[4 * g + 2], vr[4 * g + 2], k[1]), y3 = one(va[4 * g + 3], vr[4 * g + 3], k[1]);
+      w[g] = sat_pack4<OSIGNED>(y0, y1, y2, y3);
+    }
+    // this thread names the row of pixel 32 u + lane: 16 bytes at channel offset 32 q + 16 hh of the row (row_off)
+    if (e.warp_live) stmatrix_t_x4(tile + row_off + (uint32_t)u * 4096u, w[0], w[1], w[2], w[3]);
+  };
+  auto issue = [&](uint32_t as, int u, int (&va)[16], int (&vr)[16]) {
+    const uint32_t t_addr = t_lane + as * p.acc_stride + 32 * u;
+    tmem_ld_frag16(t_addr, va);
+    tmem_ld_frag16(t_addr + p.pt, vr);
+  };
+
+  int a0[16], r0[16], a1[16], r1[16];
+  uint32_t tcount = 0, as = 0;
+  int p_tile = e.p_tile0;
+  if (!wait_bar(&ctl.tfull[0], 0)) return;          // accumulator AND transposed residual are in tensor memory
+  tc_fence_after();
+  issue(0, 0, a0, r0);
+  bool pending = true;
+  while (true) {
+    const uint32_t rs = tcount & rmask;
+    const uint32_t tile = e.res_stage + rs * e.res_tile_bytes;          // [128 pixels][128 bytes], 128-byte swizzle
+    const bool has_next = p_tile + e.p_step < p.p_tiles;
+    const uint32_t nas = (tcount + 1u) & bmask, naph = ((tcount + 1u) >> p.lg_bufs) & 1u;
+    bool ok = true, next_issued = false;
+#pragma unroll
+    for (int u = 0; u < units; u += 2) {
+      // ---- unit u (registers a0 / r0), while unit u + 1 streams into a1 / r1
+      tmem_ld_wait();
+      issue(as, u + 1, a1, r1);
+      unit(a0, r0, tile, u);
+      // ---- unit u + 1, while the next unit streams into a0 / r0
+      tmem_ld_wait();
+      pending = false;
+      if (u + 2 < units) {
+        issue(as, u + 2, a0, r0);
+        pending = true;
+      } else {
+        // every lane has read its last columns of this tile: hand the accumulator buffer back, and start on the next
+        // tile's first unit if that tile is already there (else after this unit's arithmetic)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) release_accumulator(p, ctl, as);
+        if (has_next) {
+          uint32_t there = 0;
+          if (lane == 0) there = mbar_try_wait(smem_u32(&ctl.tfull[nas]), naph) ? 1u : 0u;
+          if (__shfl_sync(0xffffffffu, there, 0)) { tc_fence_after(); issue(nas, 0, a0, r0); pending = true; next_issued = true; }
+        }
+      }
+      unit(a1, r1, tile, u + 1);
+    }
+    fence_async_smem();                             // make this lane's pieces visible to the TMA engine
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl.ofull[rs]));
+    if (!has_next) break;
+    if (!next_issued) {
+      ok = wait_bar(&ctl.tfull[nas], naph);
+      if (!ok) break;
+      tc_fence_after();
+      issue(nas, 0, a0, r0);
+      pending = true;
+    }
+    p_tile += e.p_step; ++tcount; as = nas;
+  }
+  if (pending) tmem_ld_wait();
 }
 
 // General tile loop: every output type, direct stores, 64-bit arithmetic, INT32 residuals.
@@ -763,8 +881,10 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
 // ---------------------------------------------------------------- the kernel -----------------
 // DUO: the instantiation that may be launched as clusters of two CTAs sharing their MMAs; only it contains the
 // cta_group::2 instructions (a kernel that contains them cannot be launched without clusters).
-template <int EPI_WARPS, int MIN_CTAS, int MMA_WARPS, bool DUO = false>
-__global__ void __launch_bounds__(32 * (1 + MMA_WARPS + EPI_WARPS), MIN_CTAS)
+// RTM: the instantiation for fused 8-bit residuals that travel through tensor memory; it has one more warp, which
+// stores the finished output tiles.
+template <int EPI_WARPS, int MIN_CTAS, int MMA_WARPS, bool DUO = false, bool RTM = false>
+__global__ void __launch_bounds__(32 * (1 + MMA_WARPS + EPI_WARPS + (RTM ? 1 : 0)), MIN_CTAS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
                const __grid_constant__ TcParams p) {
@@ -795,7 +915,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     for (int s = 0; s < (1 << p.lg_bufs); ++s) {
       mbar_init(smem_u32(&ctl.tfull[s]), p.ni); mbar_init(smem_u32(&ctl.tempty[s]), (4 * p.halves) << p.duo);
       mbar_init(smem_u32(&ctl.tstart[s]), 1);
-      mbar_init(smem_u32(&ctl.rfull[s]), 1); mbar_init(smem_u32(&ctl.rempty[s]), p.inplace ? p.halves : 4 * p.halves);
+    }
+    for (int s = 0; s < (1 << p.lg_rbufs); ++s) {
+      mbar_init(smem_u32(&ctl.rfull[s]), 1);
+      mbar_init(smem_u32(&ctl.rempty[s]), RTM ? 1 : p.inplace ? p.halves : 4 * p.halves);
+      mbar_init(smem_u32(&ctl.ofull[s]), EPI_WARPS);
     }
     mbar_init(smem_u32(&ctl.drain), p.ni);
     mbar_init(smem_u32(&ctl.wfull), 1);
@@ -804,6 +928,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) { if constexpr (DUO) tmem_alloc2(smem_u32(&ctl.tmem_base), p.tmem_cols); else tmem_alloc(smem_u32(&ctl.tmem_base), p.tmem_cols); }
+  if (p.rtm) {
+    // the identity matrix as a K-major MMA operand, [128 rows][128 bytes] with the 128-byte swizzle: 16-byte chunk
+    // c of row r sits at chunk position c ^ (r % 8); row r holds a single 1 at byte r
+    uint4* ident = (uint4*)(smem_raw + (tiles - raw) + p.ident_off);
+    for (int i = threadIdx.x; i < 1024; i += blockDim.x) {
+      const int r = i >> 3, c = (i & 7) ^ (r & 7);
+      uint32_t word[4] = {0u, 0u, 0u, 0u};
+      if (c == (r >> 4)) word[(r & 15) >> 2] = 1u << (8 * (r & 3));
+      ident[i] = make_uint4(word[0], word[1], word[2], word[3]);
+    }
+    fence_async_smem();
+  }
   tc_fence_before();
   __syncthreads();
   if constexpr (DUO) cluster_sync_all();   // both CTAs' barriers exist before either touches the other's
@@ -1018,7 +1154,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         if (!mbar_wait(smem_u32(&ctl.tempty[as]), aph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + as * p.pt;
+        const uint32_t d_tmem = tmem_base + as * p.acc_stride;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (kb > 0 && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
           const uint32_t w_addr = tiles + s * stage_bytes;
@@ -1033,9 +1169,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
               mma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
           }
           // the accumulator's barrier first on the last K block: the epilogue is the one waiting
-          if (kb + 1 == p.k_blocks) commit(smem_u32(&ctl.tfull[as]));
+          if (kb + 1 == p.k_blocks && !p.rtm) commit(smem_u32(&ctl.tfull[as]));
           commit(smem_u32(&ctl.empty[s]));         // frees the stage when these MMAs have read it
           if (++s == nstages) { s = 0; ph ^= 1u; }
+        }
+        if (p.rtm && ok) {
+          // The residual tile through the tensor core: D2[ch][px] = sum_k I[ch][k] * R[px][k] = R[px][ch], INT32, in the
+          // pt columns after the accumulator.  Four MMAs of 32 channels of K each; the accumulator barrier then stands
+          // for both results, and for the tile in shared memory being free to be overwritten by the outputs.
+          const uint32_t rs = tcount & ((1u << p.lg_rbufs) - 1u), rph = (tcount >> p.lg_rbufs) & 1u;
+          if (!mbar_wait(smem_u32(&ctl.rfull[rs]), rph, &ctl, p.status, HQ_DEV_TIMEOUT_MMA)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t hi128 = smem_desc(0, 128);
+          uint64_t adesc = hi128 | (uint64_t)(((tiles + p.ident_off) >> 4) & 0x3FFF);
+          uint64_t bdesc = hi128 | (uint64_t)(((res_stage + rs * res_tile_bytes) >> 4) & 0x3FFF);
+          const uint32_t idesc_r = (2u << 4) | (1u << 7) | ((uint32_t)(p.res_signed ? 1 : 0) << 10) |
+                                   ((uint32_t)(p.pt >> 3) << 17) | ((uint32_t)(kTileC >> 4) << 24);
+          for (int k = 0; k < 4; ++k, adesc += 2, bdesc += 2) mma_i8(d_tmem + p.pt, adesc, bdesc, idesc_r, k ? 1u : 0u);
+          commit(smem_u32(&ctl.tfull[as]));
         }
       }
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok && !lean; p_tile += p_step, ++tcount) {
@@ -1103,6 +1254,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (global_ns() - t0 > kWaitBudgetNs) { atomicCAS(p.status, 0u, (uint32_t)HQ_DEV_TIMEOUT_DRAIN); break; }
       }
     }
+  } else if (RTM && warp == 1 + MMA_WARPS + EPI_WARPS) {
+    // ------------------------------------------------------------ store warp (rtm): finished tiles leave by TMA
+    if (elect_one()) {
+      const uint32_t rmask = (1u << p.lg_rbufs) - 1u;
+      uint32_t tcount = 0;
+      for (int p_tile = p_tile0; p_tile < p.p_tiles; p_tile += p_step, ++tcount) {
+        const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
+        if (!mbar_wait(smem_u32(&ctl.ofull[rs]), rph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE)) break;
+        tma_store_2d(&map_out, res_stage + rs * res_tile_bytes, c_tile * kTileC, p_tile * p.pt);
+        tma_store_commit();
+        if (rmask < 3u) {
+          // only two tile buffers: hand this one back as soon as the store has read it
+          tma_store_wait_read0();
+          mbar_arrive(smem_u32(&ctl.rempty[rs]));
+        } else if (tcount > 0) {
+          // the store before this one has read its tile by now: that buffer may be loaded again
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          mbar_arrive(smem_u32(&ctl.rempty[(tcount - 1u) & rmask]));
+        }
+      }
+      tma_store_wait_all();
+    }
   } else {
     // ------------------------------------------------------------ epilogue (the last EPI_WARPS warps)
     const int q = warp & 3;                       // the TMEM lane quarter this warp may read: channels 32q..32q+31
@@ -1164,7 +1337,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     e.warp = warp; e.lane = lane; e.q = q; e.cq = cq; e.ew = ew; e.half = half; e.col0 = col0; e.px_per_warp = px_per_warp; e.ch = ch;
     e.c_tile = c_tile; e.p_tile0 = p_tile0; e.p_step = p_step; e.lo = lo; e.hi = hi;
     e.ch_live = ch_live; e.warp_live = warp_live;
-    if (half >= p.halves) {
+    if (p.rtm) {
+      if constexpr (RTM) {
+        // residual through tensor memory: the fragment loop, in its general form when some channel needs 64-bit steps
+        const bool rn = warp_narrow;
+        if (!fast || epi_bar_and<32 * EPI_WARPS>(warp_small ? 0u : 1u) == 0u) {
+          if (p.out_signed) epilogue_loop_frag<true, false, false, true, false>(e); else epilogue_loop_frag<true, false, false, false, false>(e);
+        } else if (p.sat_pack) {
+          if (p.out_signed) { if (rn) epilogue_loop_frag<false, false, true, true, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, true, false>(e); else epilogue_loop_frag<false, false, true, true, false>(e); }
+          else { if (rn) epilogue_loop_frag<false, false, true, false, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, false, false>(e); else epilogue_loop_frag<false, false, true, false, false>(e); }
+        } else {
+          if (p.out_signed) { if (rn) epilogue_loop_frag<false, false, false, true, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, false, true, false>(e); else epilogue_loop_frag<false, false, false, true, false>(e); }
+          else { if (rn) epilogue_loop_frag<false, false, false, false, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, false, false, false>(e); else epilogue_loop_frag<false, false, false, false, false>(e); }
+        }
+      }
+    } else if (half >= p.halves) {
       // the 64-pixel tile has one 64-column slice per lane quarter: this warp only took part in the vote above
     } else if (fast && p.staged_out && p.out_bits == 4 && !p.res && !p.strip && lo >= 0 && hi <= 15) {
       // unsigned 4-bit outputs without a residual (the convs inside a 4-bit block)
@@ -1173,10 +1360,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
-#define HQ_FAST8(R, RS, S, OS) do { if (EPI_WARPS == 16) { \
-                                      if (warp_small) epilogue_loop_lean8<R, RS, S, OS, true, false>(e, k); \
-                                      else if (R && warp_narrow) epilogue_loop_lean8<R, RS, S, OS, false, R>(e, k); \
-                                      else epilogue_loop_lean8<R, RS, S, OS, false, false>(e, k); \
+#define HQ_FAST8(R, RS, S, OS) do { if (RTM) { \
                                     } else if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true, false>(e, k); \
                                     else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, false, R>(e, k); \
                                     else epilogue_loop_fast8<R, RS, S, OS, false, false>(e, k); } while (0)
@@ -1315,7 +1499,7 @@ bool hq_conv_tc_init() {
                               214 * 1024) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               112 * 1024) == cudaSuccess &&
-         cudaFuncSetAttribute(conv_tc_kernel<16, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess &&
+         cudaFuncSetAttribute(conv_tc_kernel<8, 1, 1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               214 * 1024) == cudaSuccess;
 }
@@ -1366,7 +1550,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   // (measured: with the weight slab resident the one-CTA shape catches up for K >= 128; the pair shape still
   // wins on the fused-residual expansions with the shortest reduction, and loses where a tile carries little
   // epilogue work, e.g. 64 output channels.  Where the layer is large enough for 256-pixel tiles and its residual
-  // travels by TMA, the wide shape below is faster still: 64 -> 256 at 56x56, batch 256: 129 -> 121 us.)
+  // travels by TMA, the rtm shape below is faster still: 64 -> 256 at 56x56, batch 256: 129 -> 122 us.)
   const bool wide_fits = p.staged_res && a.out_bits == 8 && a.cout > 64 && pick_pt(P, p.c_tiles, h->sm_count, 256) == 256;
   bool pair = k_total <= 64 && a.res != nullptr && a.res_bits == 8 && a.cout >= 128 && !wide_fits;
   int stages = 0, stage_bytes = 0, res_tile_bytes = 0, out_tile_bytes = 0, wres_bytes = 0;
@@ -1477,14 +1661,32 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     // Measured: several issuers pay off where the operands are mostly in shared memory already (strip form,
     // resident weights); where every block waits for 48 KiB from L2 the tile is bound by that stream and the extra
     // issuers only cost a few percent.
-    // Third launch shape, *wide*: sixteen epilogue warps (four per scheduler, 64 pixel columns each) with a loop that
-    // keeps one chunk in registers.  Measured per layer: it wins where the epilogue carries the residual add on
-    // 256-pixel tiles with a short reduction (1x1 128 -> 512 at 28x28: 81 -> 72 us) and loses a few percent
-    // everywhere else (long reductions are bound by the operand stream, not by the epilogue).  Its outputs overwrite
-    // the residual tile they were computed from, which then leaves as the store's box: no staging box, so that
-    // 256-pixel tiles also fit beside a 32-64 KiB weight slab (1x1 256 -> 1024 at 14x14: 55 -> 44 us).
+    // Third launch shape, *rtm*, for the fused 8-bit residual with a short reduction on layers large enough for
+    // 256-pixel tiles (here called `wide` for the condition it shares with the tile choice above): the residual tile
+    // goes through the tensor core into tensor memory, see epilogue_loop_frag.  Measured against the shape it replaced
+    // (sixteen warps, one channel per thread, one byte load and one byte store per value, in place in the residual tile):
+    // 1x1 64 -> 256 at 56x56, batch 256, 125 -> 122 us; 128 -> 512 at 28x28 72 -> 70 us; no byte-wise shared-memory
+    // traffic is left, the epilogue is bound by the integer instructions of Eq. 4 and the residual term themselves.
     wide = !pair && !p.strip && p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
-    if (wide) { p.halves = 4; p.inplace = 1; }
+    if (wide) {
+      // 128-pixel tiles, two buffers of (accumulator + transposed residual) = 512 tensor-memory columns; the two
+      // residual tiles double as the output boxes; the identity matrix takes 16 KiB
+      p.rtm = 1; p.inplace = 1; p.halves = 2;
+      p.pt = 128; p.lg_bufs = 1; p.lg_rbufs = 1;
+      p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
+      out_tile_bytes = 0;
+      res_tile_bytes = p.pt * kTileC;
+      wres_bytes = p.k_blocks * kTileC * p.bkb;
+      p.wres = wres_bytes <= 72 * 1024 ? 1 : 0;
+      if (!p.wres) wres_bytes = 0;
+      stage_bytes = ((p.wres ? 0 : kTileC) + p.pt) * p.bkb;
+      // four residual / output tiles when they leave room for three operand stages: a tile is held from its load to
+      // the end of its store, and the loads of the next tiles must be in flight meanwhile to cover the memory latency
+      for (p.lg_rbufs = 2; ; --p.lg_rbufs) {
+        stages = (212 * 1024 - (res_tile_bytes << p.lg_rbufs) - wres_bytes - 16 * 1024) / stage_bytes;
+        if (stages >= 3 || p.lg_rbufs == 1) break;
+      }
+    }
     // Fourth shape, *duo*: clusters of two CTAs on adjacent SMs share every MMA (cta_group::2, M = 256): each CTA
     // fetches its own 128 weight rows and HALF of the tile's pixel rows, 32 KiB per K block and SM instead of
     // 48 KiB for the same MMA time.  For the long reductions whose weights stream, which the operand fetch bounds.
@@ -1502,7 +1704,8 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
       stages -= stages % p.ni;
     }
   }
-  p.tmem_cols = (uint32_t)(p.pt << p.lg_bufs);          // 512 columns, or 256 for the smallest tile
+  p.acc_stride = p.rtm ? 2 * p.pt : p.pt;
+  p.tmem_cols = (uint32_t)(p.acc_stride << p.lg_bufs);  // 512 columns, or 256 for the smallest tile
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2 && !p.strip) return HQ_ERR_UNSUPPORTED;
   p.stages = stages;
@@ -1510,6 +1713,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   p.res_stage_off = p.out_stage_off + (uint32_t)out_tile_bytes;
   p.wres_off = p.res_stage_off + ((uint32_t)res_tile_bytes << p.lg_rbufs);
   p.patch_off = p.wres_off + (uint32_t)wres_bytes;
+  p.ident_off = p.patch_off + (uint32_t)patch_total;
   p.bias = a.bias; p.b = a.b; p.c = a.c;
   p.res = a.res; p.res_bits = a.res_bits; p.res_signed = a.res_signed; p.rb = a.rb; p.rc = a.rc;
   p.res_narrow = (a.res && a.res_bits == 8) ? (const int4*)a.res_narrow : nullptr;
@@ -1558,6 +1762,8 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   }
   if (!encode_rows_map(&map_w, a.wgt, a.cout, (long long)a.kh * a.kw * a.cin, p.bkb, p.fold ? 64 : kTileC, swz)) return HQ_ERR_CUDA;
   map_out = map_w; map_res = map_w;                    // valid placeholders when a path is not staged
+  // (with rtm the residual tile is an MMA operand and, later, the output box: 128-byte swizzle both ways)
+  const CUtensorMapSwizzle box_swz = p.rtm ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
   if (p.strip) {
     // output (C, W, H, N), box = 32 positions of the raster: 32 channels x min(pitch, 32) columns x the rows that makes
     const cuuint32_t bw = p.lg_wp >= 5 ? 32u : (1u << p.lg_wp);
@@ -1569,12 +1775,13 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
   } else
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, p.inplace ? kTileC : a.out_bits == 4 ? 16 : 32, p.pt / (p.halves << p.fold),
-                                       CU_TENSOR_MAP_SWIZZLE_NONE)) return HQ_ERR_CUDA;
-  if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, CU_TENSOR_MAP_SWIZZLE_NONE))
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, p.inplace ? kTileC : a.out_bits == 4 ? 16 : 32, p.rtm ? p.pt : p.pt / (p.halves << p.fold),
+                                       box_swz)) return HQ_ERR_CUDA;
+  if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, box_swz))
     return HQ_ERR_CUDA;
 
-  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_rbufs) + wres_bytes + patch_total + 1024;
+  const size_t dyn_smem = (size_t)stages * stage_bytes + out_tile_bytes + ((size_t)res_tile_bytes << p.lg_rbufs) + wres_bytes + patch_total +
+                          (p.rtm ? 16 * 1024 : 0) + 1024;
   const long long total_tiles = (long long)p.p_tiles * p.c_tiles;
   // a multiple of c_tiles, so that every CTA keeps one channel tile
   const int slots = pair ? 2 * h->sm_count : h->sm_count;
@@ -1593,8 +1800,8 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     cfg.blockDim = dim3(32 * (2 + kSoloEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
     err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kSoloEpilogueWarps, 1, 1, true>, map_x, map_w, map_out, map_res, p);
   } else if (wide) {
-    cfg.blockDim = dim3(32 * 18); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
-    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<16, 1, 1>, map_x, map_w, map_out, map_res, p);
+    cfg.blockDim = dim3(32 * 11); cfg.dynamicSmemBytes = dyn_smem < 120 * 1024 ? 120 * 1024 : dyn_smem;
+    err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<8, 1, 1, false, true>, map_x, map_w, map_out, map_res, p);
   } else if (pair) {
     cfg.blockDim = dim3(32 * (1 + kPairIssuerWarps + kPairEpilogueWarps)); cfg.dynamicSmemBytes = dyn_smem;
     err = cudaLaunchKernelEx(&cfg, conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, map_x, map_w, map_out, map_res, p);
