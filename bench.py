@@ -36,11 +36,19 @@ WORKLOADS = {
 }
 METRIC = "int-only ResNet-50 images/s @bs256; fused conv INT TOPS vs tcgen05 i8 peak"
 NOMINAL_I8_TOPS = 4500.0
-# dram__bytes_read.sum + dram__bytes_write.sum of all conv_tc_kernel launches of one pass, captured with ncu at
-# batch 64 (profiles/resnet50_int8_b256_launch_list.md) and scaled per image; writes are under-counted there
-# (outputs stay dirty in L2), so this is a lower bound of the batch-256 traffic.
-NCU_CONV_DRAM_BYTES_PER_IMAGE = (903.0e6 + 78.2e6) / 64
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+# Figures taken from profiler / measurement runs, kept beside their summaries under profiles/ (small tracked JSON):
+# DRAM bytes of the conv launches of one pass (ncu capture at a reduced batch, scaled by images), and the
+# MMA-only tcgen05 kind::i8 ceiling measured by `bench.py --mma-peak`.
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "resnet50_int8_conv_dram_traffic.json")
+I8_PEAK_JSON = os.path.join(ROOT, "profiles", "mma_peak_kind_i8.json")
+
+
+def tracked_json(path):
+    try:
+        return json.load(open(path))
+    except (OSError, ValueError):
+        return None
 
 
 def measured_peaks():
@@ -379,6 +387,53 @@ def run_sweep_grid(args):
     hq.close()
 
 
+def run_mma_peak(args):
+    """The MMA-only ceiling of tcgen05 kind::i8 on this GPU (hq_mma_peak_launch): every SM issues 128 x 256 x 32
+    instructions back to back from pseudo-random operands resident in shared memory, for at least --min-seconds
+    (default 2 s) of device time, with the SM clock sampled meanwhile.  Prints integer POPS (2 per MAC) for the
+    whole run and for the best launch."""
+    import torch
+    from paper_2011_10680_b200 import binding, build
+    build.build()
+    hq = binding.Handle(0)
+    stream = torch.cuda.Stream()
+    want_s = args.min_seconds if args.min_seconds > 0 else 2.0
+    rounds, blocks = 8, 4096                       # 8 x 4096 blocks of 128 x 256 x 128 B: about 10 ms per launch
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            hq.mma_peak_launch(rounds, blocks)
+        hq.sync()
+        sampler = ClockSampler(0)
+        sampler.start()
+        time.sleep(0.25)
+        times, ops_total, total_ms = [], 0, 0.0
+        while total_ms < want_s * 1e3:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ops = 0
+            for _ in range(10):
+                ops += hq.mma_peak_launch(rounds, blocks)
+            e1.record(stream)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1)
+            times.append((ms, ops)); total_ms += ms; ops_total += ops
+        clocks = sampler.stop()
+        hq.sync()
+    best_pops = max(o / m for m, o in times) / 1e12          # ops per ms / 1e12 = peta-ops per second
+    pops = ops_total / total_ms / 1e12
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    mhz = clocks.get("sm_mhz") or 1965.0
+    line = {"metric": "tcgen05.mma kind::i8 MMA-only ceiling", "pops": pops, "best_launch_group_pops": best_pops,
+            "seconds": total_ms / 1e3, "launches": 10 * len(times), "nominal_pops": NOMINAL_I8_TOPS / 1e3,
+            "frac_of_nominal": pops / (NOMINAL_I8_TOPS / 1e3), "clocks": clocks,
+            "mac_per_clk_per_sm_at_median_clock": (ops_total / 2) / (total_ms * 1e-3) / sms / (mhz * 1e6),
+            "operands": "pseudo-random bytes resident in shared memory, s8 x u8 -> s32, 128 x 256 x 32 per instruction"}
+    if args.layers_out:
+        json.dump(line, open(args.layers_out, "w"), indent=1)
+    print(json.dumps(line), flush=True)
+    hq.close()
+
+
 def run_ilp(args):
     """Hardware-aware bit-width selection (Section 3.4): per-layer latencies of the INT8 and INT4 forms measured
     on this GPU feed the ILP, together with model size, BOPS and a synthetic sensitivity; every answer is then
@@ -488,6 +543,10 @@ def main():
     ap.add_argument("--ilp", action="store_true", help="measure per-layer INT4/INT8 latencies and solve the bit-width ILP of Section 3.4 for several limits")
     ap.add_argument("--sweep-pixels", type=int, default=200704, help="output pixels per sweep shape (batch is derived)")
     ap.add_argument("--sweep-only", type=int, default=-1, help="run a single sweep shape (index), e.g. for profiling")
+    ap.add_argument("--mma-peak", action="store_true", help="measure the MMA-only tcgen05 kind::i8 ceiling (>= --min-seconds, default 2 s)")
+    ap.add_argument("--min-seconds", type=float, default=-1.0,
+                    help="after the K timed steps, keep repeating K-step blocks until this much device time has passed and report "
+                         "the sustained figure beside the K-step one (default 3 s; 0 switches it off)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -497,6 +556,12 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank)
         return
+    if args.mma_peak:
+        if rank == 0:
+            run_mma_peak(args)
+        return
+    if args.min_seconds < 0:
+        args.min_seconds = 3.0
     if args.sweep_grid:
         if rank == 0:
             run_sweep_grid(args)
@@ -565,6 +630,35 @@ def main():
         clocks = sampler.stop() if rank == 0 else None
         hq.sync()
 
+        # ---------------- sustained: K-step blocks back to back for at least --min-seconds -----
+        sustained = None
+        if args.min_seconds > 0:
+            sampler2 = ClockSampler(local_rank)
+            barrier()
+            if rank == 0:
+                sampler2.start()
+            blocks_ms, n_blocks = 0.0, 0
+            g0 = torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            while True:
+                g1 = torch.cuda.Event(enable_timing=True)
+                for _ in range(args.steps):
+                    net.run(images_d, logits_d)
+                g1.record(stream)
+                g1.synchronize()
+                n_blocks += 1
+                blocks_ms = g0.elapsed_time(g1)
+                go = torch.tensor([1.0 if blocks_ms < args.min_seconds * 1e3 else 0.0], device="cuda")
+                if world > 1:
+                    dist.all_reduce(go, op=dist.ReduceOp.MAX)      # every rank runs the same number of blocks
+                if float(go[0]) == 0.0:
+                    break
+            barrier()
+            c2 = sampler2.stop() if rank == 0 else None
+            sustained = {"seconds": blocks_ms / 1e3, "steps": n_blocks * args.steps,
+                         "ms_per_step": blocks_ms / (n_blocks * args.steps), "clocks": c2}
+            hq.sync()
+
         # ---------------- end to end: pinned host images in, logits out, double-buffered ----
         copy_stream = torch.cuda.Stream()
         img_bufs = [torch.empty_like(images_d) for _ in range(2)]
@@ -605,9 +699,11 @@ def main():
         layer_ns /= reps
 
     if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        t = torch.tensor([ms, ms_e2e, sustained["ms_per_step"] if sustained else 0.0], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms, ms_e2e = float(t[0]), float(t[1])
+        if sustained:
+            sustained["ms_per_step"] = float(t[2])
 
     if rank == 0:
         hbm_peak, bf16_peak, peak_kind = measured_peaks()
@@ -625,12 +721,31 @@ def main():
         if args.layers_out:
             json.dump(rows, open(args.layers_out, "w"), indent=1)
         n_conv_tc = sum(1 for r in rows if r["tensor_core"])
-        achieved = tc_bytes / max(tc_ns, 1)                      # bytes per ns = GB/s
         total_ops = sum(r["ops"] for r in rows)
         value = world * batch * args.steps / (ms / 1e3)
+        step_ms = ms / args.steps
+        # The dominant kernel is conv_tc_kernel (all its launch shapes).  Its time per step is the graph-replay step
+        # time times its share of the summed per-layer event times (plain launches with an event pair per layer run
+        # slower than the graph, so only their RATIO is used); achieved = its algorithmic bytes per step / that time.
+        share = tc_ns / max(layer_ns.sum(), 1)
+        conv_ms = step_ms * share
+        achieved = tc_bytes / (conv_ms * 1e-3) / 1e9                  # GB/s
+        # layer by layer: the time each layer would take at its own roofline (tensor peak or HBM bandwidth)
+        i8_meas = tracked_json(I8_PEAK_JSON)
+        i8_meas_tops = i8_meas["pops"] * 1e3 if i8_meas else None
+        def layerwise_ms(tops):
+            return sum(max(r["ops"] / (tops * 1e12), r["bytes"] / (hbm_peak * 1e9)) for r in rows) * 1e3
+        lw_nominal = layerwise_ms(NOMINAL_I8_TOPS)
+        lw_measured = layerwise_ms(i8_meas_tops) if i8_meas_tops else None
+        traffic = tracked_json(TRAFFIC_JSON)
+        traffic_per_launch = None
+        if traffic and args.workload == "resnet50_int8_b256":
+            per_image = (traffic["conv_tc_kernel"]["dram_read_bytes"] + traffic["conv_tc_kernel"]["dram_write_bytes"]) / traffic["batch"]
+            traffic_per_launch = per_image * batch / max(n_conv_tc, 1)
+        tensor_tops = tc_ops / (conv_ms * 1e-3) / 1e12
         line = {
             "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8" if not mixed else "int4/int8", "data": "synthetic",
             "config": {"workload": args.workload + (f" (batch overridden to {batch})" if args.batch else ""),
                        "global_batch": world * batch, "image": "224x224x3 uint8",
@@ -645,19 +760,32 @@ def main():
             "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                          "frac": achieved / hbm_peak,
-                         "traffic": (NCU_CONV_DRAM_BYTES_PER_IMAGE * batch / max(n_conv_tc, 1)
-                                     if args.workload == "resnet50_int8_b256" else None),
-                         "traffic_note": "avg DRAM bytes per conv launch from an ncu capture at batch 64, scaled by images",
+                         "traffic": traffic_per_launch,
+                         "traffic_note": (f"avg DRAM bytes per conv launch: ncu capture at batch {traffic['batch']} "
+                                          f"({os.path.basename(TRAFFIC_JSON)}), scaled by images") if traffic_per_launch else None,
                          "algorithmic_bytes_per_launch": tc_bytes / max(n_conv_tc, 1),
                          "peak_kind": f"of {peak_kind}",
                          "kernel": "conv_tc_kernel", "launches_per_step": n_conv_tc,
-                         "avg_launch_us": tc_ns / 1e3 / max(n_conv_tc, 1),
+                         "avg_launch_us": conv_ms * 1e3 / max(n_conv_tc, 1),
+                         "kernel_ms_per_step": conv_ms, "share_of_step": share,
+                         "how": "algorithmic bytes of the conv launches / (ms_per_step x their share of the per-layer event times)",
                          "algorithmic_bytes_per_step": tc_bytes,
-                         "tensor_tops": tc_ops / max(tc_ns, 1) / 1e3,
-                         "tensor_frac_of_nominal_4500": tc_ops / max(tc_ns, 1) / 1e3 / NOMINAL_I8_TOPS,
-                         "tensor_frac_of_2x_measured_bf16": tc_ops / max(tc_ns, 1) / 1e3 / (2 * bf16_peak),
-                         "share_of_step": tc_ns / max(layer_ns.sum(), 1)},
+                         "layerwise_frac": lw_nominal / step_ms,
+                         "layerwise_roofline_ms": lw_nominal,
+                         "layerwise_note": "sum over layers of max(ops / 4.5 POPS nominal, algorithmic bytes / measured HBM) / ms_per_step",
+                         "layerwise_frac_measured_i8_peak": (lw_measured / step_ms) if lw_measured else None,
+                         "tensor_tops": tensor_tops,
+                         "tensor_frac_of_nominal_4500": tensor_tops / NOMINAL_I8_TOPS,
+                         "tensor_frac_of_measured_i8_peak": (tensor_tops / i8_meas_tops) if i8_meas_tops else None,
+                         "measured_i8_peak_tops": i8_meas_tops,
+                         "tensor_frac_of_2x_measured_bf16": tensor_tops / (2 * bf16_peak)},
         }
+        if sustained:
+            sustained["value"] = world * batch / (sustained["ms_per_step"] / 1e3)
+            sustained["unit"] = "images/s"
+            mhz = (sustained.get("clocks") or {}).get("sm_mhz")
+            sustained["ms_per_step_x_sm_ghz"] = sustained["ms_per_step"] * mhz / 1e3 if mhz else None
+            line["sustained"] = sustained
         if world == 1 and not args.no_cpu_baseline:
             from oracle import hqref
             from oracle.network import run_network

@@ -198,6 +198,13 @@ hq_status hq_run_network(hq_network* net, const hq_tensor* images, hq_tensor* lo
 hq_status hq_network_time_layers(hq_network* net, const hq_tensor* images, hq_tensor* logits, int64_t* ns,
                                  void* stream);
 
+/* Measurement aid: the contraction of Eq. 3 alone.  Launches one kernel (asynchronous on `stream`) in which every
+ * SM issues `rounds` x `blocks_per_round` blocks of four tcgen05.mma kind::i8 instructions (128 x 256 x 32, s8 x u8 ->
+ * s32) back to back from pseudo-random operands resident in shared memory, with no loads and no epilogue, and
+ * writes the integer operations of the launch (2 per multiply-accumulate) to *ops (HOST, may be NULL).  Timed by the
+ * caller (events on `stream`); hq_sync reports an expired wait.  rounds in [1, 2^20], blocks_per_round in [1, 2^16]. */
+hq_status hq_mma_peak_launch(hq_handle* h, int32_t rounds, int32_t blocks_per_round, int64_t* ops, void* stream);
+
 /* Bytes of layer i's stored output and the number of kernels one hq_run_network launches. */
 hq_status hq_network_layer_bytes(const hq_network* net, int32_t layer, int64_t* bytes);
 hq_status hq_network_launch_count(const hq_network* net, int32_t* launches);

@@ -22,7 +22,7 @@ EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
     "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
-    "hq_network_check_guards", "hq_conv2d_noalloc_sync",
+    "hq_network_check_guards", "hq_conv2d_noalloc_sync", "hq_mma_peak_launch",
     "hq_ilp_solve", "hq_concat_requant", "hq_sumpool",
 ]
 
@@ -87,6 +87,7 @@ def lib():
         L.hq_network_destroy.argtypes = [vp]
         L.hq_network_check_guards.argtypes = [vp, vp, C.POINTER(i32)]
         L.hq_conv2d_noalloc_sync.argtypes = [vp]
+        L.hq_mma_peak_launch.argtypes = [vp, i32, i32, C.POINTER(C.c_int64), vp]
         L.hq_set_conv_path.argtypes = [vp, i32]
         L.hq_expire_wait_selftest.argtypes = [vp, i32, vp]
         L.hq_expire_wait_selftest.restype = i32
@@ -207,6 +208,12 @@ class Handle:
 
     def sync(self):
         _check(lib().hq_sync(self._h, _stream()), "hq_sync")
+
+    def mma_peak_launch(self, rounds: int, blocks_per_round: int) -> int:
+        """hq_mma_peak_launch on the current stream; returns the integer operations the launch performs."""
+        ops = C.c_int64()
+        _check(lib().hq_mma_peak_launch(self._h, rounds, blocks_per_round, C.byref(ops), _stream()), "hq_mma_peak_launch")
+        return ops.value
 
     # ---- one call per C entry point --------------------------------------------------------
     def conv2d(self, x, in_bits, in_signed, cin, wgt, cout, kh, kw, stride, pad, bias, b, c, out, out_bits, out_signed,
