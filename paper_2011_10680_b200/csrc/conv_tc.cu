@@ -956,7 +956,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
-      asm volatile("griddepcontrol.wait;" ::: "memory");
       // No division or modulo in this loop: one thread runs it and every dependent instruction
       // costs its full latency, so stage / phase / filter-tap indices are carried incrementally.
       uint32_t it = 0, tcount = 0, s = 0, ph = 0;
@@ -984,6 +983,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           }
         }
       }
+      // The resident weights above do not wait for the previous kernel: weights are never written by the launch
+      // immediately before this one (the helper kernels that prepare weights are always followed by another launch).
+      // Everything below reads activations, which the previous kernel may still be writing.
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       uint32_t pit = 0;                                // strip mode: patches started
       if (p.strip) {
         uint32_t ps = 0, pph = 0;

@@ -325,8 +325,9 @@ hq_status hq_launch_conv_widen4(hq_handle* h, const ConvArgs& a, void* scratch, 
   const long long x = (long long)a.n * a.h * a.w * a.cin, w = (long long)a.cout * a.kh * a.kw * a.cin;
   unsigned char* xw = (unsigned char*)scratch;
   unsigned char* ww = xw + (x + 255) / 256 * 256;
-  if (launch_widen4(a.in, x, a.in_signed, xw, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+  // (weights first: the convolution fetches resident weights without waiting for the launch just before it)
   if (!a.wgt_widened && launch_widen4(a.wgt, w, 1, ww, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
+  if (launch_widen4(a.in, x, a.in_signed, xw, h->sm_count, s) != cudaSuccess) return HQ_ERR_CUDA;
   ConvArgs t = a;
   t.in = xw; t.wgt = a.wgt_widened ? a.wgt_widened : ww; t.in_bits = 8;
   const hq_status st = hq_launch_conv_tc(h, t, s);

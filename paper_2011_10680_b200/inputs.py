@@ -16,6 +16,8 @@ from __future__ import annotations
 
 import numpy as np
 
+from .offline import dyadic_from_scale, quantize_weights   # DN(.) and the weight quantizer belong to the offline tool
+
 __all__ = [
     "rng", "dyadic_from_scale", "pack4", "unpack4", "conv_case", "config1_case",
     "resnet_table", "table_cost", "out_hw", "SWEEP_LAYERS",
@@ -25,36 +27,6 @@ __all__ = [
 def rng(seed: int, *stream: int) -> np.random.Generator:
     """Counter-based generator keyed by (seed, stream ids): the same key gives the same numbers."""
     return np.random.Generator(np.random.Philox(key=np.random.SeedSequence([seed, *stream]).generate_state(2, np.uint64)))
-
-
-# --------------------------------------------------------------------------------------------
-# DN(.): real scale -> dyadic pair (offline; Section 3.1, equation after Eq. 4)
-# --------------------------------------------------------------------------------------------
-def dyadic_from_scale(s):
-    """Return int32 arrays (b, c) with b / 2^c ~= s, 2^30 <= b < 2^31 and 1 <= c <= 62.
-
-    The paper defines DN only by its result.  Reading used here: normalise s = m * 2^e with
-    m in [0.5, 1), take b = round_half_up(m * 2^31), c = 31 - e (and renormalise if b hits 2^31).
-    The error is at most 2^-(c+1).  Scales so small that c would pass 62 keep c = 62 and a
-    smaller b; scales of 2^30 and above are rejected.
-    """
-    s = np.atleast_1d(np.asarray(s, dtype=np.float64))
-    if np.any(~np.isfinite(s)) or np.any(s <= 0):
-        raise ValueError("scale must be finite and positive")
-    m, e = np.frexp(s)
-    b = np.floor(m * float(2 ** 31) + 0.5).astype(np.int64)
-    c = 31 - e.astype(np.int64)
-    carry = b == 2 ** 31
-    b[carry] = 2 ** 30
-    c[carry] -= 1
-    if np.any(c < 1):
-        raise ValueError("scale too large for a dyadic pair with c >= 1")
-    deep = c > 62
-    if np.any(deep):
-        sh = c[deep] - 62
-        b[deep] = (b[deep] + (1 << (sh - 1))) >> sh
-        c[deep] = 62
-    return b.astype(np.int32), c.astype(np.int32)
 
 
 # --------------------------------------------------------------------------------------------
@@ -174,11 +146,7 @@ def _draw_weights(g: np.random.Generator, cout: int, k: int, cin: int, bits: int
     """Real weights N(0, sqrt(2/fan_in)) quantized symmetrically per output channel (Appendix A)."""
     fan_in = k * k * cin
     wr = g.standard_normal(size=(cout, k, k, cin)) * np.sqrt(2.0 / fan_in)
-    wmax = (1 << (bits - 1)) - 1
-    s_w = np.abs(wr).reshape(cout, -1).max(axis=1) / wmax
-    q = np.floor(wr / s_w[:, None, None, None] + 0.5)
-    q = np.clip(q, -wmax, wmax).astype(np.int64)
-    return q, s_w
+    return quantize_weights(wr, bits)
 
 
 class _Builder:

@@ -696,6 +696,36 @@ def test_network_residual_shifts_per_channel(hq):
     run_network_and_compare(hq, t, batch=2, seed=12)
 
 
+def test_table_from_the_offline_tool_runs_bit_exact(hq):
+    """Float network (batch norm, a residual block, pooling, classifier) -> the offline tool (BN fold, channel-wise
+    weight quantizer, INT32 bias, DN pairs, static calibration) -> hq_run_network: every layer equals the oracle."""
+    from paper_2011_10680_b200 import offline
+    g = np.random.default_rng(17)
+    n, hw, c1, classes = 3, 16, 32, 12
+    images = g.integers(0, 256, size=(n, hw, hw, 3)).astype(np.uint8)
+
+    def bn(ch):
+        return (g.uniform(0.8, 1.2, ch), g.normal(0, 0.1, ch), g.normal(0, 0.1, ch), g.uniform(0.8, 1.2, ch))
+
+    layers = [
+        dict(op="conv", in0=-1, in1=-1, w=g.normal(size=(c1, 3, 3, 3)) * 0.4, bn=bn(c1), stride=1, pad=1, bits=8, relu=True),
+        dict(op="maxpool", in0=0, k=3, stride=2, pad=1),
+        dict(op="conv", in0=1, in1=-1, w=g.normal(size=(c1, 3, 3, c1)) * 0.08, bn=bn(c1), stride=1, pad=1, bits=8, relu=True),
+        dict(op="conv", in0=2, in1=1, w=g.normal(size=(c1, 1, 1, c1)) * 0.2, bn=bn(c1), stride=1, pad=0, bits=8, relu=True),
+        dict(op="avgpool", in0=3, hw=(hw // 2) ** 2, channels=c1),
+        dict(op="linear", in0=4, in1=-1, w=g.normal(size=(classes, 1, 1, c1)) * 0.3, bn=None, bias=np.full(classes, -0.1),
+             bits=8, relu=False, s_out=None),
+    ]
+    s_img = 1.0 / 255.0
+    table = offline.quantize_network(offline.calibrate(layers, images * s_img), s_img, image_hw=hw)
+    for l in table["layers"]:
+        if l["op"] == "maxpool":
+            l["cout"] = c1
+    # run_network_and_compare draws its own images from the table's image size; same shapes as the calibration batch
+    ref = run_network_and_compare(hq, table, batch=n, seed=3)
+    assert ref[-1].dtype == np.int32 and len(np.unique(ref[-1])) > classes
+
+
 def test_resnet18_imagenet_shape_batch8_every_layer(hq):
     """Benchmark config 2: ResNet-18, 224x224x3, 1000 classes, batch 8, all layers INT8."""
     t = inputs.resnet_table(18, seed=2)
