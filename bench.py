@@ -33,7 +33,14 @@ WORKLOADS = {
     "resnet50_int8_b256": (50, False, 256, 3),
     "resnet50_int4_8_mixed_b256": (50, True, 256, 4),
     "resnet18_int8_b8": (18, False, 8, 2),
+    # the same ResNet-50 with the residual stream kept in INT32 between blocks, as Fig. 2 draws it (element-wise adds)
+    "resnet50_int8_int32stream_b256": (50, False, 256, 3),
 }
+
+
+def workload_table(name):
+    depth, mixed, batch, seed = WORKLOADS[name]
+    return inputs.resnet_table(depth, seed, mixed=mixed, int32_stream="int32stream" in name)
 METRIC = "int-only ResNet-50 images/s @bs256; fused conv INT TOPS vs tcgen05 i8 peak"
 NOMINAL_I8_TOPS = 4500.0
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
@@ -139,7 +146,7 @@ def run_reference(args, rank):
     from oracle import hqref
     from oracle.network import run_network
     depth, mixed, batch, seed = WORKLOADS[args.workload]
-    table = inputs.resnet_table(depth, seed, mixed=mixed)
+    table = workload_table(args.workload)
     t0 = time.perf_counter()
     run_network(table, inputs.random_images(seed, 1))
     t1 = time.perf_counter() - t0
@@ -596,7 +603,7 @@ def main():
 
     depth, mixed, batch, seed = WORKLOADS[args.workload]
     batch = args.batch or batch
-    table = inputs.resnet_table(depth, seed, mixed=mixed)
+    table = workload_table(args.workload)
     hq = binding.Handle(local_rank)
     net = binding.Network(hq, table, batch)
     images_h = torch.from_numpy(inputs.random_images(seed + 1000 * rank, batch)).pin_memory()

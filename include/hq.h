@@ -127,7 +127,8 @@ hq_status hq_linear(hq_handle* h, const hq_tensor* in, const hq_conv_desc* desc,
  * Integer residual add on stored tensors (Section 3.3): per element of channel ch
  *   y = dn(main, mb[ch], mc[ch]) + (res ? dn(res, rb[ch], rc[ch]) : 0); ReLU; clamp; store.
  * Each branch is rounded on its own and then added (Appendix G).  main/res: bits 4, 8 or 32;
- * out: bits 4 or 8.  res == NULL gives a plain dyadic requantization.
+ * out: bits 4, 8 or 32 (32: the sum stays INT32, the wide residual stream of Fig. 2, clamped to [qmin, qmax]).
+ * res == NULL gives a plain dyadic requantization.
  */
 hq_status hq_residual_add(hq_handle* h, const hq_tensor* main_t, hq_dyadic main_rescale,
                           const hq_tensor* res, hq_dyadic res_rescale,

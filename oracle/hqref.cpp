@@ -209,7 +209,8 @@ int32_t hqref_residual_add(const void* main_t, int32_t main_bits, int32_t main_s
                            int32_t relu, int32_t qmin, int32_t qmax,
                            void* out, int32_t out_bits, int32_t out_signed) {
   if (!main_t || !out || pixels < 0 || ch < 1) return HQREF_ERR_INVALID_ARG;
-  if (!bits_ok(main_bits, true) || !bits_ok(out_bits, false)) return HQREF_ERR_INVALID_ARG;
+  // out_bits == 32: the sum stays a wide integer (the INT32 residual stream of Fig. 2), clamped to [qmin, qmax]
+  if (!bits_ok(main_bits, true) || !bits_ok(out_bits, true)) return HQREF_ERR_INVALID_ARG;
   if ((main_bits == 4 || out_bits == 4) && (ch & 1)) return HQREF_ERR_INVALID_ARG;
   if (!dyadic_ok(mb, mc, ch)) return HQREF_ERR_INVALID_ARG;
   if (res && (!bits_ok(res_bits, true) || !dyadic_ok(rb, rc, ch))) return HQREF_ERR_INVALID_ARG;

@@ -269,7 +269,7 @@ static hq_status residual_add_impl(hq_handle* h, const hq_tensor* main_t, hq_dya
   if (!h) return HQ_ERR_INVALID_ARG;
   hq_status st = check_tensor(main_t, true, true, true);
   if (st != HQ_OK) return st;
-  st = check_tensor(out, true, true, false);
+  st = check_tensor(out, true, true, true);
   if (st != HQ_OK) return st;
   if (out->n != main_t->n || out->h != main_t->h || out->w != main_t->w || out->c != main_t->c) return HQ_ERR_INVALID_ARG;
   if (!mr.b || !mr.c) return HQ_ERR_INVALID_ARG;

@@ -624,6 +624,61 @@ cudaError_t launch_requant32(const EltArgs& a, int quads, int lo, int hi, int sm
   return cudaGetLastError();
 }
 
+// INT32 output (the wide residual stream of Fig. 2: the add of Section 3.3 with its result kept in INT32):
+// one thread per element, 64-bit dyadic arithmetic, consecutive threads on consecutive channels.
+__global__ void __launch_bounds__(256) residual_add_out32_kernel(EltArgs a) {
+  const long long total = a.pixels * a.ch;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const int ch = (int)(e % a.ch);
+    long long y = hq_dn(hq_load_elem(a.main_t, e, a.main_bits, a.main_signed), __ldg(a.mb + ch), __ldg(a.mc + ch));
+    if (a.res) y += hq_dn(hq_load_elem(a.res, e, a.res_bits, a.res_signed), __ldg(a.rb + ch), __ldg(a.rc + ch));
+    ((int*)a.out)[e] = hq_clamp_ll(y, a.relu, a.qmin, a.qmax);
+  }
+}
+
+// The same for channel counts that are a multiple of four, operands of 8 or 32 bits: a thread owns four channels
+// (their pairs stay in registers: the launch makes the thread count a multiple of the quads per pixel), reads
+// 16 bytes of an INT32 operand (4 of an 8-bit one) and writes 16 bytes per step, two steps in flight.
+template <int MB, int RB>   // operand bits: 8 or 32; RB = 0: no second operand
+__global__ void __launch_bounds__(256) residual_add_out32_vec_kernel(EltArgs a) {
+  const long long quads = a.pixels * (a.ch >> 2);
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= quads) return;
+  const int ch = (int)(i % (a.ch >> 2)) << 2;
+  int mb[4], mc[4], rb[4], rc[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    mb[j] = a.mb[ch + j]; mc[j] = a.mc[ch + j];
+    rb[j] = RB ? a.rb[ch + j] : 0; rc[j] = RB ? a.rc[ch + j] : 1;
+  }
+  auto load = [&](const void* base, int bits, int is_signed, long long q, int (&v)[4]) {
+    if (bits == 32) {
+      const int4 t = __ldg((const int4*)base + q);
+      v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else {
+      const unsigned t = __ldg((const unsigned*)base + q);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = is_signed ? (int)(signed char)(t >> (8 * j)) : (int)((t >> (8 * j)) & 0xFFu);
+    }
+  };
+  auto one = [&](long long q) {
+    int m[4], r[4] = {0, 0, 0, 0};
+    load(a.main_t, MB, a.main_signed, q, m);
+    if (RB) load(a.res, RB, a.res_signed, q, r);
+    int y[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      long long s = hq_dn(m[j], mb[j], mc[j]);
+      if (RB) s += hq_dn(r[j], rb[j], rc[j]);
+      y[j] = hq_clamp_ll(s, a.relu, a.qmin, a.qmax);
+    }
+    ((int4*)a.out)[q] = make_int4(y[0], y[1], y[2], y[3]);
+  };
+  for (; i + stride < quads; i += 2 * stride) { one(i); one(i + stride); }
+  if (i < quads) one(i);
+}
+
 // Any channel count: one thread per output byte (one element at 8 bit, two at 4 bit).
 __global__ void residual_add_scalar_kernel(EltArgs a) {
   const int per = (a.out_bits == 4) ? 2 : 1;
@@ -910,6 +965,34 @@ __global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int c
 
 cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t s) {
   if (a.pixels == 0) return cudaSuccess;
+  if (a.out_bits == 32) {
+    const int quads = a.ch >> 2;
+    const bool vec = a.ch % 4 == 0 && (a.main_bits == 8 || a.main_bits == 32) && (!a.res || a.res_bits == 8 || a.res_bits == 32);
+    if (vec) {
+      // thread count a multiple of the quads per pixel, so that a thread keeps its four channels
+      long long blocks = (a.pixels * quads + 255) / 256;
+      const long long cap = (long long)sm_count * 16;
+      if (blocks > cap) blocks = cap;
+      int unit = quads, t = 256;                       // blocks must be a multiple of quads / gcd(quads, 256)
+      while (t) { const int r = unit % t; unit = t; t = r; }      // unit = gcd(quads, 256)
+      const long long mult = quads / unit;
+      blocks = blocks / mult * mult;
+      if (blocks >= mult) {
+        const int g = (int)blocks;
+        const int rbits = a.res ? a.res_bits : 0;
+        if (a.main_bits == 32 && rbits == 32) residual_add_out32_vec_kernel<32, 32><<<g, 256, 0, s>>>(a);
+        else if (a.main_bits == 32 && rbits == 8) residual_add_out32_vec_kernel<32, 8><<<g, 256, 0, s>>>(a);
+        else if (a.main_bits == 32) residual_add_out32_vec_kernel<32, 0><<<g, 256, 0, s>>>(a);
+        else if (rbits == 32) residual_add_out32_vec_kernel<8, 32><<<g, 256, 0, s>>>(a);
+        else if (rbits == 8) residual_add_out32_vec_kernel<8, 8><<<g, 256, 0, s>>>(a);
+        else residual_add_out32_vec_kernel<8, 0><<<g, 256, 0, s>>>(a);
+        return cudaGetLastError();
+      }
+    }
+    const long long blocks = (a.pixels * a.ch + 255) / 256, cap = (long long)sm_count * 32;
+    residual_add_out32_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>(a);
+    return cudaGetLastError();
+  }
   // 8-bit operands with a channel count the word mapping covers: 32-bit fast kernel
   const int words = a.ch / 4;
   if (a.main_bits == 8 && (!a.res || a.res_bits == 8) && a.ch % 4 == 0 && (words <= 256 || words % 256 == 0)) {

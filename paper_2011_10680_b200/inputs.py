@@ -154,6 +154,7 @@ class _Builder:
         self.g = rng(seed, 7)
         self.layers: list[dict] = []
         self.scale: dict[int, float] = {}
+        self.chscale: dict[int, np.ndarray] = {}           # raw INT32 conv outputs: scale per channel, S_h * S_w[oc]
         self.shape: dict[int, tuple[int, int, int]] = {}   # h, w, c of each tensor id
         self.bits: dict[int, int] = {}
 
@@ -177,9 +178,11 @@ class _Builder:
                      relu=int(relu), out_bits=out_bits, out_signed=int(out_signed),
                      b=None, c=None, rb=None, rc=None, qmin=0, qmax=0,
                      macs=ho * wo * cout * k * k * cin, params=cout * k * k * cin, unit=unit)
-        if out_bits == 32:                      # raw INT32 logits: bias added, no requantization
+        if out_bits == 32:                      # raw INT32 accumulator + bias (logits; main branch of an INT32 add)
             layer.update(qmin=-(1 << 31), qmax=(1 << 31) - 1, out_signed=1)
-            return self._emit(layer, s_in * float(s_w.mean()), (ho, wo, cout), 32)
+            tid = self._emit(layer, s_in * float(s_w.mean()), (ho, wo, cout), 32)
+            self.chscale[tid] = s_in * s_w
+            return tid
         s_out = _draw_scale(g)
         layer["b"], layer["c"] = dyadic_from_scale(s_w * s_in / s_out)
         if res >= 0:
@@ -191,6 +194,18 @@ class _Builder:
         else:
             layer.update(qmin=0, qmax=(1 << out_bits) - 1)
         return self._emit(layer, s_out, (ho, wo, cout), out_bits)
+
+    def add32(self, main: int, res: int, s_out: float, unit: int = -1) -> int:
+        """The residual add of Section 3.3 / Fig. 2 on stored tensors with an INT32 result: both branches rescaled by
+        their own dyadic pairs to s_out (per channel where a branch is a raw accumulator), rounded, added, ReLU."""
+        h, w, c = self.shape[main]
+        sm = self.chscale.get(main, np.full(c, self.scale[main]))
+        sr = self.chscale.get(res, np.full(c, self.scale[res]))
+        b, cc = dyadic_from_scale(sm / s_out)
+        rb, rc = dyadic_from_scale(sr / s_out)
+        layer = dict(op="add", in0=main, in1=res, cout=c, b=b, c=cc, rb=rb, rc=rc, relu=1, qmin=0, qmax=(1 << 31) - 1,
+                     out_bits=32, out_signed=1, macs=0, params=0, unit=unit)
+        return self._emit(layer, s_out, (h, w, c), 32)
 
     def requant(self, src: int, out_bits: int, unit: int = -1) -> int:
         """Unsigned stream tensor -> lower-bit unsigned copy (Fig. 2: quantize the input once)."""
@@ -227,7 +242,7 @@ def resnet_choice_units(depth: int) -> int:
 
 def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: bool = False,
                  image_hw: int = 224, classes: int = 1000, width: int = 64,
-                 conv_bits: list[int] | None = None) -> dict:
+                 conv_bits: list[int] | None = None, int32_stream: bool = False) -> dict:
     """Layer table of an ImageNet-shaped ResNet-18 or ResNet-50 with integer parameters.
 
     Tensor id -1 is the uint8 input image (n, image_hw, image_hw, 3); layer i produces tensor i.
@@ -243,6 +258,10 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
     (resnet_choice_units(depth) entries, e.g. the answer of the bit-width ILP of Section 3.4): a conv
     writes its output at the bit-width of the conv that reads it, and a block whose first conv is
     4-bit requantizes the stream tensor once for that conv and the shortcut conv.
+    int32_stream=True lays the table out as the paper draws Fig. 2: the residual stream between blocks is an INT32
+    tensor (at 1/256 of an 8-bit activation scale), every block requantizes it once to the bit-width of its first
+    conv, the block's last conv and a down-sampling shortcut conv return their raw INT32 accumulators, and an
+    element-wise add rescales both branches with their own dyadic pairs, adds them in INT32 and applies the ReLU.
     """
     if depth not in (18, 50):
         raise ValueError("depth must be 18 or 50")
@@ -268,6 +287,21 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
             wb = conv_bits[unit:unit + per_block]
             u0 = unit                             # layers carry the index of the choice they belong to
             unit += per_block
+            if int32_stream:
+                # Fig. 2 as drawn: wide stream, one requantization per block input, raw accumulators into an INT32 add
+                xin = bd.requant(x, wb[0], unit=u0) if (bd.bits[x] == 32 or wb[0] == 4) else x
+                if depth == 18:
+                    y = bd.conv(xin, planes, 3, stride, 1, wb[0], relu=True, out_bits=wb[1], unit=u0)
+                    main = bd.conv(y, planes, 3, 1, 1, wb[1], relu=False, out_bits=32, unit=u0 + 1)
+                    shortcut = bd.conv(xin, planes, 1, stride, 0, wb[0], relu=False, out_bits=32, unit=u0) if need_ds else x
+                else:
+                    s1, s2 = (1, stride) if stride_on_3x3 else (stride, 1)
+                    y = bd.conv(xin, planes, 1, s1, 0, wb[0], relu=True, out_bits=wb[1], unit=u0)
+                    y = bd.conv(y, planes, 3, s2, 1, wb[1], relu=True, out_bits=wb[2], unit=u0 + 1)
+                    main = bd.conv(y, planes * 4, 1, 1, 0, wb[2], relu=False, out_bits=32, unit=u0 + 2)
+                    shortcut = bd.conv(xin, planes * 4, 1, stride, 0, wb[0], relu=False, out_bits=32, unit=u0) if need_ds else x
+                x = bd.add32(main, shortcut, _draw_scale(bd.g) / 256.0, unit=u0 + per_block - 1)
+                continue
             xin = bd.requant(x, 4, unit=u0) if wb[0] == 4 else x
             if depth == 18:
                 y = bd.conv(xin, planes, 3, stride, 1, wb[0], relu=True, out_bits=wb[1], unit=u0)

@@ -696,6 +696,40 @@ def test_network_residual_shifts_per_channel(hq):
     run_network_and_compare(hq, t, batch=2, seed=12)
 
 
+@pytest.mark.parametrize("depth,mixed", [(18, False), (50, False), (50, True)])
+def test_network_with_int32_residual_stream_every_layer(hq, depth, mixed):
+    """The dataflow of Fig. 2 as the paper draws it: INT32 residual stream between blocks, one requantization per
+    block input, raw INT32 accumulators of the block's last conv and of the shortcut conv into an element-wise add
+    with an INT32 result.  Every layer equals the oracle."""
+    t = inputs.resnet_table(depth, seed=8, image_hw=64, classes=24, width=32, mixed=mixed, int32_stream=True)
+    assert sum(1 for l in t["layers"] if l["op"] == "add" and l["out_bits"] == 32) == {18: 8, 50: 16}[depth]
+    run_network_and_compare(hq, t, batch=3, seed=depth + 2)
+
+
+def test_residual_add_int32_result(hq):
+    """hq_residual_add with out bits 32 on its own: INT32 + INT32 and INT32 + 8-bit operands, every shift."""
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(43, 1)
+    n, hw, ch = 2, 9, 40
+    main = g.integers(-(1 << 24), 1 << 24, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+    mb = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+    mc = (np.arange(ch) % 62 + 1).astype(np.int32)
+    for res_bits in (32, 8):
+        res = (g.integers(-(1 << 20), 1 << 20, size=main.shape, dtype=np.int64).astype(np.int32) if res_bits == 32
+               else g.integers(0, 256, size=main.shape, dtype=np.int64).astype(np.uint8))
+        rb = g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32)
+        rc = ((np.arange(ch) * 7) % 62 + 1).astype(np.int32)
+        ref = oracle().residual_add(main, 32, 1, mb, mc, res, res_bits, int(res_bits == 32), rb, rc, ch, 0,
+                                    -(1 << 31), (1 << 31) - 1, 32, 1)
+        out = binding.alloc_out(n, hw, hw, ch, 32, 1)
+        st = hq.residual_add(binding.to_device(main), 32, 1, binding.to_device(mb), binding.to_device(mc),
+                             binding.to_device(res), res_bits, int(res_bits == 32), binding.to_device(rb), binding.to_device(rc),
+                             ch, 0, -(1 << 31), (1 << 31) - 1, out, 32, 1)
+        assert st == binding.HQ_OK
+        hq.sync()
+        assert np.array_equal(host(out, ref), ref)
+
+
 def test_table_from_the_offline_tool_runs_bit_exact(hq):
     """Float network (batch norm, a residual block, pooling, classifier) -> the offline tool (BN fold, channel-wise
     weight quantizer, INT32 bias, DN pairs, static calibration) -> hq_run_network: every layer equals the oracle."""

@@ -527,12 +527,35 @@ def logical(y, layer):
     return y.astype(np.int64)
 
 
-@pytest.mark.parametrize("depth,mixed,hw", [(18, False, 32), (18, True, 32), (50, True, 32), (50, False, 32)])
-def test_network_walk_equals_layers_applied_by_hand(depth, mixed, hw):
+def test_residual_add_with_int32_result_matches_exact_rational():
+    """The add of Section 3.3 with its sum kept in INT32 (the wide residual stream of Fig. 2): a raw INT32 main branch
+    with a pair per channel plus an INT32 or 8-bit second branch, every value against exact rational rounding."""
+    g = np.random.default_rng(41)
+    ch = 6
+    main = g.integers(-(1 << 22), 1 << 22, size=(2, 3, 4, ch)).astype(np.int32)
+    b, c = inputs.dyadic_from_scale(np.exp(g.uniform(np.log(2.0 ** -9), np.log(2.0 ** -5), ch)))
+    for res_bits in (32, 8):
+        res = (g.integers(0, 1 << 17, size=main.shape).astype(np.int32) if res_bits == 32
+               else g.integers(0, 256, size=main.shape).astype(np.uint8))
+        rb, rc = inputs.dyadic_from_scale(np.full(ch, 0.37 if res_bits == 32 else 181.0))
+        y = hqref.residual_add(main, 32, 1, b, c, res, res_bits, int(res_bits == 32), rb, rc, ch, 1, 0, (1 << 31) - 1, 32, 1)
+        assert y.dtype == np.int32
+        for idx in np.ndindex(main.shape):
+            k = idx[-1]
+            want = exact_round_half_up(int(main[idx]) * int(b[k]), int(c[k])) + exact_round_half_up(int(res[idx]) * int(rb[k]), int(rc[k]))
+            assert int(y[idx]) == max(want, 0), idx
+    # the clamp applies to the wide result too
+    y = hqref.residual_add(main, 32, 1, b, c, None, 0, 0, None, None, ch, 0, -100, 100, 32, 1)
+    assert y.min() == -100 and y.max() == 100
+
+
+@pytest.mark.parametrize("depth,mixed,hw,wide", [(18, False, 32, False), (18, True, 32, False), (50, True, 32, False),
+                                                  (50, False, 32, False), (50, False, 32, True), (18, True, 32, True)])
+def test_network_walk_equals_layers_applied_by_hand(depth, mixed, hw, wide):
     """EVERY layer of reduced ResNet-18 / ResNet-50 tables (uniform and mixed 4/8 bit): the oracle's walk against
     the hand-applied layers.  A wrong residual operand, a swapped bits / sign lookup for in0 and in1, or a slip
     in the requant / add / pooling / linear branches of the walk changes some layer here."""
-    t = inputs.resnet_table(depth, seed=3 + depth, image_hw=hw, classes=10, width=8, mixed=mixed)
+    t = inputs.resnet_table(depth, seed=3 + depth, image_hw=hw, classes=10, width=8, mixed=mixed, int32_stream=wide)
     img = inputs.random_images(3, 2, hw)
     outs = run_network(t, img)
     want = hand_walk(t, img)
@@ -547,6 +570,9 @@ def test_network_walk_equals_layers_applied_by_hand(depth, mixed, hw):
             if t["layers"][l["in1"]]["out_signed"] != t["layers"][l["in0"]]["out_signed"]:
                 seen.add("operands of different sign")
     need = {"conv", "linear", "maxpool", "avgpool", "residual", "residual from further back", "operands of different sign"}
+    if wide:              # Fig. 2 as drawn: INT32 stream, element-wise adds, one requantization per block input
+        need = {"conv", "linear", "maxpool", "avgpool", "add", "requant"}
+        assert sum(1 for l, y in zip(t["layers"], outs) if l["op"] == "add" and y.dtype == np.int32) == {18: 8, 50: 16}[depth]
     if mixed:
         need.add("requant")
     assert need <= seen, need - seen
