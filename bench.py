@@ -35,11 +35,16 @@ WORKLOADS = {
     "resnet18_int8_b8": (18, False, 8, 2),
     # the same ResNet-50 with the residual stream kept in INT32 between blocks, as Fig. 2 draws it (element-wise adds)
     "resnet50_int8_int32stream_b256": (50, False, 256, 3),
+    # Inception modules as Appendix E draws them (35x35 and 17x17 module shapes, 4-bit convolution inputs, INT32
+    # pooling branch, per-branch DN and concatenation); image 299 / 4 -> 71x71 so that the stem lands on 35x35
+    "inception_modules_int4_b256": (0, True, 256, 6),
 }
 
 
 def workload_table(name):
     depth, mixed, batch, seed = WORKLOADS[name]
+    if depth == 0:
+        return inputs.inception_table(seed, conv_bits=4 if mixed else 8, image_hw=71, width=64, modules35=2, modules17=2)
     return inputs.resnet_table(depth, seed, mixed=mixed, int32_stream="int32stream" in name)
 METRIC = "int-only ResNet-50 images/s @bs256; fused conv INT TOPS vs tcgen05 i8 peak"
 NOMINAL_I8_TOPS = 4500.0
@@ -148,11 +153,11 @@ def run_reference(args, rank):
     depth, mixed, batch, seed = WORKLOADS[args.workload]
     table = workload_table(args.workload)
     t0 = time.perf_counter()
-    run_network(table, inputs.random_images(seed, 1))
+    run_network(table, inputs.random_images(seed, 1, table["image_hw"]))
     t1 = time.perf_counter() - t0
     total_steps = args.steps + args.warmup
     sample = int(max(1, min(batch, 90.0 / max(t1, 1e-3) / total_steps)))
-    images = inputs.random_images(seed, sample)
+    images = inputs.random_images(seed, sample, table["image_hw"])
     for _ in range(args.warmup):
         run_network(table, images)
     t0 = time.perf_counter()
@@ -606,7 +611,7 @@ def main():
     table = workload_table(args.workload)
     hq = binding.Handle(local_rank)
     net = binding.Network(hq, table, batch)
-    images_h = torch.from_numpy(inputs.random_images(seed + 1000 * rank, batch)).pin_memory()
+    images_h = torch.from_numpy(inputs.random_images(seed + 1000 * rank, batch, table["image_hw"])).pin_memory()
     images_d = images_h.cuda()
     logits_d = torch.empty(net.logits_shape, dtype=torch.int32, device="cuda")
     stream = torch.cuda.Stream()
@@ -755,7 +760,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8" if not mixed else "int4/int8", "data": "synthetic",
             "config": {"workload": args.workload + (f" (batch overridden to {batch})" if args.batch else ""),
-                       "global_batch": world * batch, "image": "224x224x3 uint8",
+                       "global_batch": world * batch, "image": f"{table['image_hw']}x{table['image_hw']}x3 uint8",
                        "parallelism": f"dp{world}" if world > 1 else "single",
                        "l2": "activations per step (GBs) exceed the 126 MB L2; no explicit flush",
                        "launch": "CUDA graph replay of the whole layer table"},
@@ -796,10 +801,10 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             from oracle import hqref
             from oracle.network import run_network
-            one = inputs.random_images(seed, 1)
+            one = inputs.random_images(seed, 1, table["image_hw"])
             t0 = time.perf_counter(); run_network(table, one); t1 = time.perf_counter() - t0
             sample = int(max(1, min(batch, 15.0 / max(t1, 1e-3))))
-            imgs = inputs.random_images(seed, sample)
+            imgs = inputs.random_images(seed, sample, table["image_hw"])
             t0 = time.perf_counter(); ref = run_network(table, imgs); dt = time.perf_counter() - t0
             line["cpu_baseline"] = {"value": sample / dt, "unit": "images/s", "cores": hqref.num_threads(),
                                     "kind": "oracle", "sample": f"first {sample} of {batch} images, one pass"}

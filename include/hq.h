@@ -71,13 +71,17 @@ typedef struct {
   int32_t qmin, qmax;        /* clamp bounds, inside the output type's range */
 } hq_conv_desc;
 
+#define HQ_CONCAT_MAX_BRANCHES 8
+
 typedef enum {
   HQ_OP_CONV = 0,    /* hq_conv2d; in1 = residual tensor id or -1 */
   HQ_OP_LINEAR = 1,  /* hq_linear on the flattened input */
   HQ_OP_MAXPOOL = 2, /* hq_maxpool */
   HQ_OP_AVGPOOL = 3, /* hq_avgpool_requant with `rescale0` */
   HQ_OP_ADD = 4,     /* hq_residual_add(in0 by rescale0, in1 by rescale1) */
-  HQ_OP_REQUANT = 5  /* hq_residual_add with no second operand */
+  HQ_OP_REQUANT = 5, /* hq_residual_add with no second operand */
+  HQ_OP_CONCAT = 6,  /* hq_concat_requant over the tensors ins[0 .. n_in) with the pairs rescales[] (Appendix E) */
+  HQ_OP_SUMPOOL = 7  /* hq_sumpool of in0 with pool_k / pool_stride / pool_pad: INT32 window sums (Appendix E) */
 } hq_op;
 
 typedef struct {       /* one row of the per-layer table; layer i produces tensor id i */
@@ -88,7 +92,10 @@ typedef struct {       /* one row of the per-layer table; layer i produces tenso
   hq_dyadic rescale1;  /* ADD: pair applied to in1 */
   int32_t pool_k, pool_stride, pool_pad; /* MAXPOOL */
   int32_t out_bits, out_signed;          /* type of the produced tensor */
-  int32_t relu, qmin, qmax;              /* AVGPOOL / ADD / REQUANT (CONV uses conv.*) */
+  int32_t relu, qmin, qmax;              /* AVGPOOL / ADD / REQUANT / CONCAT (CONV uses conv.*) */
+  int32_t n_in;                          /* CONCAT: number of branches, 1 .. HQ_CONCAT_MAX_BRANCHES */
+  int32_t ins[8];                        /* CONCAT: tensor ids of the branches, in channel order */
+  hq_dyadic rescales[8];                 /* CONCAT: DN(S_i / S_a) of branch i, arrays of that branch's channel count */
 } hq_layer;
 
 /* Create / destroy the per-device context.  `device` is a CUDA ordinal.  Host call.
@@ -154,7 +161,6 @@ hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic rescal
  * out: bits 8, or 4 when every branch has an even channel count (else HQ_ERR_UNSUPPORTED).  One launch,
  * asynchronous on `stream`; every operand is read once and the output written once.
  */
-#define HQ_CONCAT_MAX_BRANCHES 8
 hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const hq_tensor* branches, const hq_dyadic* rescale,
                             int32_t relu, int32_t qmin, int32_t qmax, hq_tensor* out, void* stream);
 
@@ -169,8 +175,8 @@ hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const hq_tensor* b
 hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,
                      hq_tensor* out, void* stream);
 
-/* k x k max pooling of an 8-bit tensor; window taps outside the image are ignored (ResNet stem;
- * an integer max commutes with the monotone requantization of Eq. 4).  pad < k. */
+/* k x k max pooling of an 8-bit or INT32 tensor (Appendix E pools on the wide feature map); window taps outside
+ * the image are ignored (ResNet stem; an integer max commutes with the monotone requantization of Eq. 4).  pad < k. */
 hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,
                      hq_tensor* out, void* stream);
 

@@ -266,7 +266,7 @@ int32_t hqref_maxpool(const void* in, int32_t n, int32_t h, int32_t w, int32_t c
                       int32_t k, int32_t stride, int32_t pad, void* out) {
   if (!in || !out || n < 0 || h < 1 || w < 1 || ch < 1 || k < 1 || stride < 1 || pad < 0)
     return HQREF_ERR_INVALID_ARG;
-  if (bits != 8) return HQREF_ERR_INVALID_ARG;
+  if (bits != 8 && bits != 32) return HQREF_ERR_INVALID_ARG;   // 32: pooling on the wide feature map (Appendix E)
   if (pad >= k) return HQREF_ERR_INVALID_ARG;   // every window must touch the image
   int32_t oh_n = 0, ow_n = 0;
   for (int32_t y = 0; y + k <= h + 2 * pad; y += stride) ++oh_n;

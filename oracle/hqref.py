@@ -186,5 +186,6 @@ def maxpool(x, k, stride, pad, signed=0):
     ho = (h + 2 * pad - k) // stride + 1
     wo = (w + 2 * pad - k) // stride + 1
     out = np.zeros((n, ho, wo, ch), x.dtype)
-    _check(lib().hqref_maxpool(_p(x), n, h, w, ch, 8, signed, k, stride, pad, _p(out)))
+    bits = 32 if x.dtype == np.int32 else 8
+    _check(lib().hqref_maxpool(_p(x), n, h, w, ch, bits, 1 if bits == 32 else signed, k, stride, pad, _p(out)))
     return out

@@ -1,7 +1,9 @@
 """Oracle network walk: apply the layer functions over a table, in table order, keeping every output.
 
 Follows the dataflow of the paper's Fig. 2 in its fused form: a conv layer may carry the residual
-operand (tensor id in1); 'requant' quantizes a stream tensor once for all its consumers.
+operand (tensor id in1); 'requant' quantizes a stream tensor once for all its consumers; 'add' is the
+element-wise add of Section 3.3 on stored tensors; 'sumpool' and 'concat' are the pooling branch and
+the concatenation of an Inception module (Appendix E).
 """
 from __future__ import annotations
 
@@ -54,6 +56,15 @@ def run_network(table: dict, images: np.ndarray) -> list[np.ndarray]:
             y = hqref.residual_add(t(l["in0"]), in_bits, in_signed, l["b"], l["c"], res, res_bits, res_signed,
                                    rb, rc, l["cout"], l["relu"], l["qmin"], l["qmax"],
                                    l["out_bits"], l["out_signed"])
+        elif op == "sumpool":
+            # the pooling branch of an Inception module works on the wide feature map: INT32 window sums (Appendix E)
+            in_bits, in_signed = meta[l["in0"]]
+            y = hqref.sumpool(t(l["in0"]), l["cout"], in_bits, in_signed, l["pool_k"], l["pool_stride"], l["pool_pad"])
+        elif op == "concat":
+            # every branch rescaled by its own dyadic pairs, then joined along the channels (Appendix E)
+            branches = [{"x": t(i), "bits": meta[i][0], "signed": meta[i][1], "ch": int(len(b)), "b": b, "c": c}
+                        for i, b, c in zip(l["ins"], l["bs"], l["cs"])]
+            y = hqref.concat_requant(branches, l["relu"], l["qmin"], l["qmax"], l["out_bits"], l["out_signed"])
         else:
             raise ValueError(f"unknown op {op!r} in layer {li}")
         outs.append(y)

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libhq.so")
 
 HQ_OK, HQ_ERR_INVALID_ARG, HQ_ERR_UNSUPPORTED, HQ_ERR_ALIGNMENT = 0, 1, 2, 3
 HQ_ERR_RANGE, HQ_ERR_WORKSPACE, HQ_ERR_CUDA, HQ_ERR_TIMEOUT, HQ_ERR_INFEASIBLE = 4, 5, 6, 7, 8
-HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant": 5}
+HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant": 5, "concat": 6, "sumpool": 7}
 
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
@@ -53,7 +53,8 @@ class hq_layer(C.Structure):
     _fields_ = [("op", C.c_int32), ("in0", C.c_int32), ("in1", C.c_int32), ("conv", hq_conv_desc),
                 ("rescale0", hq_dyadic), ("rescale1", hq_dyadic), ("pool_k", C.c_int32),
                 ("pool_stride", C.c_int32), ("pool_pad", C.c_int32), ("out_bits", C.c_int32),
-                ("out_signed", C.c_int32), ("relu", C.c_int32), ("qmin", C.c_int32), ("qmax", C.c_int32)]
+                ("out_signed", C.c_int32), ("relu", C.c_int32), ("qmin", C.c_int32), ("qmax", C.c_int32),
+                ("n_in", C.c_int32), ("ins", C.c_int32 * 8), ("rescales", hq_dyadic * 8)]
 
 
 _lib = None
@@ -253,9 +254,9 @@ class Handle:
         to = tensor_of(out, ch, 32, 1)
         return lib().hq_sumpool(self._h, C.byref(ti), k, stride, pad, C.byref(to), _stream())
 
-    def maxpool(self, x, ch, signed, k, stride, pad, out):
-        ti = tensor_of(x, ch, 8, signed)
-        to = tensor_of(out, ch, 8, signed)
+    def maxpool(self, x, ch, signed, k, stride, pad, out, bits: int = 8):
+        ti = tensor_of(x, ch, bits, signed)
+        to = tensor_of(out, ch, bits, signed)
         return lib().hq_maxpool(self._h, C.byref(ti), k, stride, pad, C.byref(to), _stream())
 
     # ---- convenience for the dict-shaped single-layer cases of the workload generator -------
@@ -310,8 +311,15 @@ class Network:
                                       dv["wgt"].data_ptr(),
                                       dv["bias"].data_ptr() if dv["bias"] is not None else None, _dy(dv["b"], dv["c"]), None,
                                       _dy(dv["rb"], dv["rc"]), l["relu"], l["qmin"], l["qmax"])
-            elif l["op"] == "maxpool":
+            elif l["op"] in ("maxpool", "sumpool"):
                 e.pool_k, e.pool_stride, e.pool_pad = l["pool_k"], l["pool_stride"], l["pool_pad"]
+            elif l["op"] == "concat":
+                e.n_in, e.in0 = len(l["ins"]), l["ins"][0]
+                for k, (tid, b, c) in enumerate(zip(l["ins"], l["bs"], l["cs"])):
+                    dv = {"b": to_device(b), "c": to_device(c)}
+                    self._keep.append(dv)
+                    e.ins[k] = tid
+                    e.rescales[k] = _dy(dv["b"], dv["c"])
             else:
                 dv = {k: to_device(l.get(k)) for k in ("b", "c", "rb", "rc")}
                 self._keep.append(dv)

@@ -325,17 +325,18 @@ hq_status hq_avgpool_requant(hq_handle* h, const hq_tensor* in, hq_dyadic r, int
 hq_status hq_maxpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad, hq_tensor* out,
                      void* stream) {
   if (!h) return HQ_ERR_INVALID_ARG;
-  hq_status st = check_tensor(in, false, true, false);
+  hq_status st = check_tensor(in, false, true, true);
   if (st != HQ_OK) return st;
-  st = check_tensor(out, false, true, false);
+  st = check_tensor(out, false, true, true);
   if (st != HQ_OK) return st;
+  if (in->bits != out->bits) return HQ_ERR_INVALID_ARG;
   if (k < 1 || stride < 1 || pad < 0 || pad >= k) return HQ_ERR_INVALID_ARG;
   if (in->h + 2 * pad < k || in->w + 2 * pad < k) return HQ_ERR_INVALID_ARG;
   const int ho = (in->h + 2 * pad - k) / stride + 1, wo = (in->w + 2 * pad - k) / stride + 1;
   if (out->n != in->n || out->h != ho || out->w != wo || out->c != in->c || out->is_signed != in->is_signed)
     return HQ_ERR_INVALID_ARG;
-  return hq_launch_maxpool(in->data, in->n, in->h, in->w, in->c, in->is_signed, k, stride, pad, out->data, ho, wo,
-                           (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+  return hq_launch_maxpool(in->data, in->n, in->h, in->w, in->c, in->bits == 32 ? 32 : 8, in->is_signed, k, stride, pad,
+                           out->data, ho, wo, (cudaStream_t)stream) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -415,6 +416,22 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
         break;
       case HQ_OP_AVGPOOL: o.h = 1; o.w = 1; o.c = in.c; break;
       case HQ_OP_ADD: case HQ_OP_REQUANT: o.h = in.h; o.w = in.w; o.c = in.c; break;
+      case HQ_OP_SUMPOOL:
+        if (l.pool_k < 1 || l.pool_stride < 1 || l.pool_pad < 0 || l.pool_pad >= l.pool_k || in.h + 2 * l.pool_pad < l.pool_k ||
+            in.w + 2 * l.pool_pad < l.pool_k || l.out_bits != 32) { st = HQ_ERR_INVALID_ARG; break; }
+        o.h = (in.h + 2 * l.pool_pad - l.pool_k) / l.pool_stride + 1;
+        o.w = (in.w + 2 * l.pool_pad - l.pool_k) / l.pool_stride + 1; o.c = in.c;
+        break;
+      case HQ_OP_CONCAT: {
+        if (l.n_in < 1 || l.n_in > HQ_CONCAT_MAX_BRANCHES || l.in0 != l.ins[0]) { st = HQ_ERR_INVALID_ARG; break; }
+        o.h = in.h; o.w = in.w; o.c = 0;
+        for (int k = 0; k < l.n_in; ++k) {
+          const int id = l.ins[k];
+          if (id < 0 || id >= i || net->outs[id].h != in.h || net->outs[id].w != in.w) { st = HQ_ERR_INVALID_ARG; break; }
+          o.c += net->outs[id].c;
+        }
+        break;
+      }
       default: st = HQ_ERR_INVALID_ARG; break;
     }
     if (st != HQ_OK) break;
@@ -438,6 +455,12 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
     for (int j = i + 1; j < n_layers; ++j) {
       const hq_layer& c = net->layers[j];
       if (c.in1 == i) { ok = false; break; }
+      if (c.op == HQ_OP_CONCAT) {
+        bool used = false;
+        for (int k = 0; k < c.n_in; ++k) used = used || c.ins[k] == i;
+        if (used) { ok = false; break; }
+        continue;
+      }
       if (c.in0 != i) continue;
       if (c.op != HQ_OP_CONV || !net->wgt_widened[j]) { ok = false; break; }
       ok = true;
@@ -532,6 +555,13 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
       case HQ_OP_REQUANT: {
         hq_dyadic none{nullptr, nullptr};
         st = residual_add_impl(h, &in, l.rescale0, nullptr, none, l.relu, l.qmin, l.qmax, &o, s, net->narrow0[i], nullptr);
+        break;
+      }
+      case HQ_OP_SUMPOOL: st = hq_sumpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;
+      case HQ_OP_CONCAT: {
+        hq_tensor br[HQ_CONCAT_MAX_BRANCHES];
+        for (int k = 0; k < l.n_in; ++k) br[k] = net->outs[l.ins[k]];
+        st = hq_concat_requant(h, l.n_in, br, l.rescales, l.relu, l.qmin, l.qmax, &o, s);
         break;
       }
       default: return HQ_ERR_INVALID_ARG;

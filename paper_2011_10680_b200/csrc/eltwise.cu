@@ -2,6 +2,8 @@
 // tensors (Section 3.3), global average pooling on wide integers (Appendix E) and the stem's max
 // pooling.  Each streams its operands once with 16-byte accesses; the arithmetic is the dyadic
 // multiply-shift of Eq. 4 in 64-bit integers.  No floating point anywhere.
+#include <climits>
+
 #include "hq_internal.cuh"
 
 namespace {
@@ -936,7 +938,7 @@ __global__ void __launch_bounds__(256) maxpool_vec16_kernel(const uint4* __restr
   }
 }
 
-__global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int ch, int is_signed,
+__global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int ch, int bits, int is_signed,
                                       int k, int stride, int pad, void* out, int ho, int wo) {
   const long long total = (long long)n * ho * wo * ch;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -946,18 +948,19 @@ __global__ void maxpool_scalar_kernel(const void* in, int n, int h, int w, int c
     const int ow = (int)(t % wo); t /= wo;
     const int oh = (int)(t % ho);
     const int img = (int)(t / ho);
-    int best = is_signed ? -128 : 0;
+    int best = bits == 32 ? INT_MIN : is_signed ? -128 : 0;
     for (int r = 0; r < k; ++r) {
       const int ih = oh * stride + r - pad;
       if (ih < 0 || ih >= h) continue;
       for (int s = 0; s < k; ++s) {
         const int iw = ow * stride + s - pad;
         if (iw < 0 || iw >= w) continue;
-        const int v = hq_load_elem(in, (((long long)img * h + ih) * w + iw) * ch + cc, 8, is_signed);
+        const int v = hq_load_elem(in, (((long long)img * h + ih) * w + iw) * ch + cc, bits, is_signed);
         best = v > best ? v : best;
       }
     }
-    ((unsigned char*)out)[i] = (unsigned char)(best & 0xFF);
+    if (bits == 32) ((int*)out)[i] = best;
+    else ((unsigned char*)out)[i] = (unsigned char)(best & 0xFF);
   }
 }
 
@@ -1064,10 +1067,10 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
   return cudaGetLastError();
 }
 
-cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int is_signed,
+cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int bits, int is_signed,
                               int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  if (ch % 16 == 0 && (long long)n * ho < (1ll << 31) && (long long)wo * (ch / 16) < (1ll << 31)) {
+  if (bits == 8 && ch % 16 == 0 && (long long)n * ho < (1ll << 31) && (long long)wo * (ch / 16) < (1ll << 31)) {
     const uint4* src = (const uint4*)in;
     uint4* dst = (uint4*)out;
     const int cg = ch / 16;
@@ -1082,7 +1085,7 @@ cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int i
     const long long total = (long long)n * ho * wo * ch;
     long long blocks = (total + 255) / 256;
     if (blocks > (1 << 20)) blocks = 1 << 20;
-    maxpool_scalar_kernel<<<(int)blocks, 256, 0, s>>>(in, n, h, w, ch, is_signed, k, stride, pad, out, ho, wo);
+    maxpool_scalar_kernel<<<(int)blocks, 256, 0, s>>>(in, n, h, w, ch, bits, is_signed, k, stride, pad, out, ho, wo);
   }
   return cudaGetLastError();
 }

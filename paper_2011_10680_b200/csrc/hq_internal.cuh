@@ -117,5 +117,5 @@ cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t 
 cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int in_bits, int in_signed,
                               const int32_t* b, const int32_t* c, int qmin, int qmax,
                               void* out, int out_bits, cudaStream_t s);
-cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int is_signed,
+cudaError_t hq_launch_maxpool(const void* in, int n, int h, int w, int ch, int bits, int is_signed,
                               int k, int stride, int pad, void* out, int ho, int wo, cudaStream_t s);

@@ -301,10 +301,13 @@ cudaError_t launch_widen4(const void* in, long long elems, int is_signed, void* 
 }  // namespace
 
 bool hq_conv_widen4_applies(const ConvArgs& a) {
-  if (a.in_bits != 4 || a.cin % 32 != 0) return false;
+  // (16 values per step of the widening kernels; channel counts the direct kernel does not take go on to the
+  // patch-matrix form after widening, e.g. the 48-channel 5x5 branch of an Inception module)
+  if (a.in_bits != 4) return false;
+  if (((long long)a.n * a.h * a.w * a.cin) % 16 != 0 || ((long long)a.cout * a.kh * a.kw * a.cin) % 16 != 0) return false;
   ConvArgs t = a;
   t.in_bits = 8;
-  return hq_conv_tc_supported(t);
+  return hq_conv_tc_supported(t) || hq_conv_lowering_applies(t);
 }
 
 static size_t widen4_copy_bytes(const ConvArgs& a) {
@@ -316,7 +319,7 @@ static size_t widen4_copy_bytes(const ConvArgs& a) {
 size_t hq_conv_widen4_bytes(const ConvArgs& a) {
   ConvArgs t = a;
   t.in_bits = 8;
-  const bool lowered = hq_conv_tc_small_im2col(t) && hq_conv_lowering_applies(t);
+  const bool lowered = (!hq_conv_tc_supported(t) || hq_conv_tc_small_im2col(t)) && hq_conv_lowering_applies(t);
   return widen4_copy_bytes(a) + (lowered ? hq_conv_lowering_bytes(t) : 0);
 }
 

@@ -3,8 +3,8 @@
 // taps outside the image count as 0 and the reciprocal of the window size of an average pool is left to the dyadic
 // pair of the consumer (hq_concat_requant, hq_residual_add), so no division touches the data.  Memory bound: a
 // thread owns four channels of one output pixel (one 16-byte read per tap of an INT32 tensor, served by L1 / L2 for
-// the overlapping windows) and writes one 16-byte piece of the INT32 output; other channel counts and 8-/4-bit
-// inputs read element-wise.
+// the overlapping windows, one word of an 8-bit tensor) and writes one 16-byte piece of the INT32 output; other
+// channel counts and 4-bit inputs read element-wise.
 #include "hq_internal.cuh"
 
 namespace {
@@ -12,7 +12,7 @@ namespace {
 struct SumPoolArgs {
   const void* in; int32_t* out;
   int32_t n, h, w, ch, bits, is_signed, k, stride, pad, oh_n, ow_n;
-  int32_t vec;     // 1: INT32 input with ch % 4 == 0: 16-byte accesses
+  int32_t vec;     // 1: INT32 input with ch % 4 == 0: 16-byte accesses; 2: 8-bit input with ch % 4 == 0: one word per tap
 };
 
 // Block x = one output row (image, oh); block y, thread = a piece of that row: (ow, group of four channels), or
@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(256) sumpool_kernel(const __grid_constant__ Su
   const int ih0 = oh * a.stride - a.pad, iw0 = ow * a.stride - a.pad;
   const long long o_idx = ((long long)blockIdx.x * a.ow_n + ow) * cg + g;   // in units of the thread's piece
   const long long img_base = (long long)img * a.h * a.w;
-  if (a.vec) {
+  if (a.vec == 1) {
     int4 sum = make_int4(0, 0, 0, 0);
 #pragma unroll
     for (int r = 0; r < k; ++r) {
@@ -40,6 +40,27 @@ __global__ void __launch_bounds__(256) sumpool_kernel(const __grid_constant__ Su
         if (ih >= 0 && ih < a.h && iw >= 0 && iw < a.w) {
           const int4 v = *((const int4*)((const int*)a.in + (img_base + (long long)ih * a.w + iw) * a.ch) + g);
           sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+        }
+      }
+    }
+    *((int4*)a.out + o_idx) = sum;
+  } else if (a.vec == 2) {
+    // 8-bit input: four channels in one 32-bit word per tap, widened as they are added; 16-byte INT32 output
+    int4 sum = make_int4(0, 0, 0, 0);
+#pragma unroll
+    for (int r = 0; r < k; ++r) {
+      const int ih = ih0 + r;
+#pragma unroll
+      for (int s = 0; s < k; ++s) {
+        const int iw = iw0 + s;
+        if (ih >= 0 && ih < a.h && iw >= 0 && iw < a.w) {
+          const unsigned v = __ldg((const unsigned*)a.in + (((img_base + (long long)ih * a.w + iw) * a.ch) >> 2) + g);
+          if (a.is_signed) {
+            sum.x += (int)(signed char)v; sum.y += (int)(signed char)(v >> 8);
+            sum.z += (int)(signed char)(v >> 16); sum.w += (int)v >> 24;
+          } else {
+            sum.x += (int)(v & 0xFFu); sum.y += (int)((v >> 8) & 0xFFu); sum.z += (int)((v >> 16) & 0xFFu); sum.w += (int)(v >> 24);
+          }
         }
       }
     }
@@ -76,7 +97,7 @@ extern "C" hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, in
   a.in = in->data; a.out = (int32_t*)out->data;
   a.n = in->n; a.h = in->h; a.w = in->w; a.ch = in->c; a.bits = in->bits; a.is_signed = in->bits == 32 ? 1 : in->is_signed;
   a.k = k; a.stride = stride; a.pad = pad; a.oh_n = ho; a.ow_n = wo;
-  a.vec = (in->bits == 32 && in->c % 4 == 0) ? 1 : 0;
+  a.vec = in->c % 4 != 0 ? 0 : in->bits == 32 ? 1 : in->bits == 8 ? 2 : 0;
   if (a.n == 0) return HQ_OK;
   const long long rows = (long long)a.n * ho, cols = (long long)wo * (a.vec ? a.ch / 4 : a.ch);
   if (rows > 0x7fffffffLL || (cols + 255) / 256 > 65535) return HQ_ERR_UNSUPPORTED;

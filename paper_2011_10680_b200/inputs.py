@@ -20,7 +20,7 @@ from .offline import dyadic_from_scale, quantize_weights   # DN(.) and the weigh
 
 __all__ = [
     "rng", "dyadic_from_scale", "pack4", "unpack4", "conv_case", "config1_case",
-    "resnet_table", "table_cost", "out_hw", "SWEEP_LAYERS",
+    "resnet_table", "inception_table", "table_cost", "out_hw", "SWEEP_LAYERS",
 ]
 
 
@@ -224,6 +224,29 @@ class _Builder:
                      out_bits=8, out_signed=0, relu=0, qmin=0, qmax=255, macs=0, params=0)
         return self._emit(layer, self.scale[src], (ho, wo, c), 8)
 
+    def sumpool(self, src: int, k: int, stride: int, pad: int) -> int:
+        """k x k window sums in INT32 (Appendix E pools on the wide feature map); the tensor's scale carries the 1 / k^2 of
+        the average, so that the consumer's dyadic pair turns the sum into the mean without a division."""
+        h, w, c = self.shape[src]
+        ho, wo = out_hw(h, w, k, stride, pad)
+        layer = dict(op="sumpool", in0=src, in1=-1, pool_k=k, pool_stride=stride, pool_pad=pad, cout=c, out_bits=32,
+                     out_signed=1, relu=0, qmin=-(1 << 31), qmax=(1 << 31) - 1, macs=0, params=0)
+        return self._emit(layer, self.scale[src] / (k * k), (ho, wo, c), 32)
+
+    def concat(self, srcs: list[int], out_bits: int = 8) -> int:
+        """Concatenation along the channels with one dyadic pair per branch channel, DN(S_i / S_a) (Appendix E)."""
+        h, w, _ = self.shape[srcs[0]]
+        s_out = _draw_scale(self.g) * (255.0 / 15.0 if out_bits == 4 else 1.0)
+        bs, cs = [], []
+        for t in srcs:
+            c = self.shape[t][2]
+            b, cc = dyadic_from_scale(self.chscale.get(t, np.full(c, self.scale[t])) / s_out)
+            bs.append(b); cs.append(cc)
+        total = sum(self.shape[t][2] for t in srcs)
+        layer = dict(op="concat", in0=srcs[0], in1=-1, ins=list(srcs), bs=bs, cs=cs, cout=total, relu=1, qmin=0,
+                     qmax=(1 << out_bits) - 1, out_bits=out_bits, out_signed=0, macs=0, params=0)
+        return self._emit(layer, s_out, (h, w, total), out_bits)
+
     def avgpool(self, src: int) -> int:
         h, w, c = self.shape[src]
         s_out = _draw_scale(self.g)
@@ -320,6 +343,45 @@ def resnet_table(depth: int, seed: int, *, mixed: bool = False, stride_on_3x3: b
     return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=depth, conv_bits=list(conv_bits),
                 shapes=[bd.shape[i] for i in range(len(bd.layers))],
                 bits=[bd.bits[i] for i in range(len(bd.layers))])
+
+
+def inception_table(seed: int, *, conv_bits: int = 4, image_hw: int = 71, classes: int = 1000, width: int = 64,
+                    modules35: int = 2, modules17: int = 2) -> dict:
+    """Layer table shaped like InceptionV3's 35x35 and 17x17 modules, wired as the paper's Appendix E draws an
+    Inception module: the module input is requantized once (to conv_bits, 4 in the figure) for the three convolution
+    branches -- 1x1; 1x1 -> 5x5 (3x3 in the 17x17 modules); 1x1 -> 3x3 -> 3x3 -- while the pooling branch works on the
+    module input itself in INT32 (3x3 window sums, the 1/9 of the average inside its dyadic pair); every branch is
+    rescaled by its own DN(S_i / S_a) and the four are joined along the channels.  Channel counts per module (width 64):
+    64 + 64 + 96 + the input's channels at 35x35 (InceptionV3: 64, 64, 96), 192 + 192 + 192 + the input's at 17x17.
+    A 3x3 / stride 2 stem takes the image to 35x35 (image_hw 71), a 3x3 / stride 2 max pool takes 35x35 to 17x17;
+    global average pool and an 8-bit classifier close the table.  First and last layer stay 8-bit (Appendix H)."""
+    if conv_bits not in (4, 8):
+        raise ValueError("conv_bits must be 4 or 8")
+    bd = _Builder(seed)
+    bd.scale[-1], bd.shape[-1], bd.bits[-1] = _draw_scale(bd.g), (image_hw, image_hw, 3), 8
+    x = bd.conv(-1, width, 3, 2, 0, 8, relu=True, out_bits=8)
+
+    def module(x, c1, c2a, c2b, k2, c3a, c3b):
+        xin = bd.requant(x, conv_bits) if conv_bits == 4 else x
+        cb = conv_bits
+        m = bd.conv(xin, c1, 1, 1, 0, cb, relu=True, out_bits=8)
+        n = bd.conv(xin, c2a, 1, 1, 0, cb, relu=True, out_bits=cb)
+        n = bd.conv(n, c2b, k2, 1, k2 // 2, cb, relu=True, out_bits=8)
+        l = bd.conv(xin, c3a, 1, 1, 0, cb, relu=True, out_bits=cb)
+        l = bd.conv(l, c3b, 3, 1, 1, cb, relu=True, out_bits=cb)
+        l = bd.conv(l, c3b, 3, 1, 1, cb, relu=True, out_bits=8)
+        p = bd.sumpool(x, 3, 1, 1)
+        return bd.concat([m, n, l, p])
+
+    for _ in range(modules35):
+        x = module(x, width, (width * 3) // 4, width, 5, width, (width * 3) // 2)
+    x = bd.maxpool(x, 3, 2, 0)
+    for _ in range(modules17):
+        x = module(x, 3 * width, 2 * width, 3 * width, 3, 2 * width, 3 * width)
+    x = bd.avgpool(x)
+    x = bd.conv(x, classes, 1, 1, 0, 8, relu=False, out_bits=32, op="linear")
+    return dict(layers=bd.layers, image_hw=image_hw, classes=classes, depth=0, conv_bits=[conv_bits],
+                shapes=[bd.shape[i] for i in range(len(bd.layers))], bits=[bd.bits[i] for i in range(len(bd.layers))])
 
 
 def table_cost(table: dict, force_bits: int | None = None) -> dict:

@@ -52,7 +52,7 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding.hq_tensor) == 32
     assert ctypes.sizeof(binding.hq_dyadic) == 16
     assert ctypes.sizeof(binding.hq_conv_desc) == 104
-    assert ctypes.sizeof(binding.hq_layer) == 184
+    assert ctypes.sizeof(binding.hq_layer) == 352
 
 
 def test_cuda_sources_have_no_floating_point():

@@ -730,6 +730,28 @@ def test_residual_add_int32_result(hq):
         assert np.array_equal(host(out, ref), ref)
 
 
+@pytest.mark.parametrize("conv_bits", [4, 8])
+def test_inception_modules_every_layer(hq, conv_bits):
+    """Inception modules as Appendix E draws them, through hq_run_network: requantized input for the convolution
+    branches, INT32 window sums of the module input as the pooling branch, per-branch DN, concatenation; 35x35 and
+    17x17 module shapes at reduced width.  Every layer equals the oracle."""
+    t = inputs.inception_table(7, conv_bits=conv_bits, image_hw=71, classes=24, width=32, modules35=2, modules17=1)
+    ops = [l["op"] for l in t["layers"]]
+    assert ops.count("concat") == 3 and ops.count("sumpool") == 3
+    run_network_and_compare(hq, t, batch=2, seed=31)
+
+
+def test_maxpool_int32(hq):
+    from paper_2011_10680_b200 import binding
+    g = inputs.rng(44, 2)
+    x = g.integers(-(1 << 30), 1 << 30, size=(2, 11, 9, 20), dtype=np.int64).astype(np.int32)
+    ref = oracle().maxpool(x, 3, 2, 1)
+    out = binding.alloc_out(2, ref.shape[1], ref.shape[2], 20, 32, 1)
+    assert hq.maxpool(binding.to_device(x), 20, 1, 3, 2, 1, out, bits=32) == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
 def test_table_from_the_offline_tool_runs_bit_exact(hq):
     """Float network (batch norm, a residual block, pooling, classifier) -> the offline tool (BN fold, channel-wise
     weight quantizer, INT32 bias, DN pairs, static calibration) -> hq_run_network: every layer equals the oracle."""

@@ -514,6 +514,26 @@ def hand_walk(table, images):
                 if l["relu"]:
                     v = max(v, 0)
                 y[idx] = min(max(v, l["qmin"]), l["qmax"])
+        elif op == "sumpool":
+            k, st, pad = l["pool_k"], l["pool_stride"], l["pool_pad"]
+            xp = np.pad(x, ((0, 0), (pad, pad), (pad, pad), (0, 0)))
+            ho, wo = (x.shape[1] + 2 * pad - k) // st + 1, (x.shape[2] + 2 * pad - k) // st + 1
+            y = np.stack([np.stack([xp[:, oh * st:oh * st + k, ow * st:ow * st + k].sum(axis=(1, 2))
+                                    for ow in range(wo)], axis=1) for oh in range(ho)], axis=1)
+        elif op == "concat":
+            parts = []
+            for tid, b, c in zip(l["ins"], l["bs"], l["cs"]):
+                src = vals[tid]
+                part = np.zeros(src.shape, np.int64)
+                it = np.nditer(part, flags=["multi_index"])
+                for _ in it:
+                    idx = it.multi_index
+                    v = dn_exact(src[idx], b[idx[-1]], c[idx[-1]])
+                    if l["relu"]:
+                        v = max(v, 0)
+                    part[idx] = min(max(v, l["qmin"]), l["qmax"])
+                parts.append(part)
+            y = np.concatenate(parts, axis=-1)
         else:
             raise AssertionError(op)
         vals[li] = y
@@ -584,6 +604,41 @@ def test_network_walk_equals_layers_applied_by_hand(depth, mixed, hw, wide):
             assert t["bits"][l["in0"]] == 4
         h, w, c = t["shapes"][i]
         assert outs[i].shape[1:3] == (h, w)
+
+
+@pytest.mark.parametrize("conv_bits", [4, 8])
+def test_inception_walk_equals_layers_applied_by_hand(conv_bits):
+    """A reduced table of Inception modules wired as Appendix E draws them (one requantization of the module input
+    for the three convolution branches, INT32 window sums of the module input itself as the pooling branch, one DN per
+    branch channel, concatenation): every layer of the oracle's walk against the hand-applied layers."""
+    t = inputs.inception_table(9, conv_bits=conv_bits, image_hw=23, classes=7, width=8, modules35=1, modules17=1)
+    img = inputs.random_images(5, 2, 23)
+    outs = run_network(t, img)
+    want = hand_walk(t, img)
+    ops = [l["op"] for l in t["layers"]]
+    assert ops.count("concat") == 2 and ops.count("sumpool") == 2 and ("requant" in ops) == (conv_bits == 4)
+    for i, (l, y, w) in enumerate(zip(t["layers"], outs, want)):
+        assert np.array_equal(logical(y, l).reshape(w.shape), w), (i, l["op"])
+    for i, l in enumerate(t["layers"]):
+        if l["op"] == "sumpool":
+            assert outs[i].dtype == np.int32
+        if l["op"] == "concat":
+            pool = l["ins"][-1]
+            assert t["layers"][pool]["op"] == "sumpool"                       # the pooling branch enters as INT32 sums
+            src = t["layers"][pool]["in0"]
+            assert t["layers"][src]["out_bits"] == 8                          # ... of the module input, not of the 4-bit copy
+            mid = (outs[i] > 0) & (outs[i] < 255)
+            assert mid.mean() > 0.05, "concatenation degenerate: everything saturates"
+
+
+def test_maxpool_on_int32_matches_padded_numpy_max():
+    g = np.random.default_rng(12)
+    x = g.integers(-(1 << 30), 1 << 30, size=(2, 9, 10, 3)).astype(np.int32)
+    y = hqref.maxpool(x, 3, 2, 1)
+    xp = np.pad(x.astype(np.int64), ((0, 0), (1, 1), (1, 1), (0, 0)), constant_values=-(1 << 40))
+    for oh in range(y.shape[1]):
+        for ow in range(y.shape[2]):
+            assert np.array_equal(y[:, oh, ow], xp[:, 2 * oh:2 * oh + 3, 2 * ow:2 * ow + 3].max(axis=(1, 2)))
 
 
 def _tiny_network():
