@@ -46,7 +46,8 @@ namespace {
 
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
-constexpr int kMaxAccBufs = 4;                                 // accumulator (and residual) buffers: 4 x 128 or 2 x 256 columns
+constexpr int kMaxAccBufs = 4;                                 // accumulator buffers: 4 x 128 or 2 x 256 columns
+constexpr int kMaxResBufs = 8;                                 // residual / output tiles in shared memory
 // Four launch shapes of the same kernel:
 //   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 212 KiB of shared memory;
 //   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
@@ -118,9 +119,9 @@ struct SharedCtl {
   unsigned long long tfull[kMaxAccBufs];
   unsigned long long tempty[kMaxAccBufs];
   unsigned long long tstart[kMaxAccBufs];   // the tile's first (overwriting) MMA has been issued
-  unsigned long long rfull[kMaxAccBufs];
-  unsigned long long rempty[kMaxAccBufs];
-  unsigned long long ofull[kMaxAccBufs];    // rtm: every epilogue warp has written its pieces of the output tile
+  unsigned long long rfull[kMaxResBufs];
+  unsigned long long rempty[kMaxResBufs];
+  unsigned long long ofull[kMaxResBufs];    // rtm: every epilogue warp has written its pieces of the output tile
   unsigned long long drain;
   unsigned long long wfull;              // resident weight slab landed
   unsigned long long pfull[3], pempty[3];  // strip mode: input patches
@@ -625,8 +626,9 @@ __device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, b
 // the next 32 columns (or of the next tile's first) are in flight while a unit is processed.  Warps do not wait for
 // each other: each arrives on the tile's `ofull` barrier when its pieces are written, and the store warp alone waits
 // there, stores the [128][128] box (128-byte swizzle, as it was loaded) and hands the buffer back.
-// GEN: 64-bit arithmetic for every shift 1..62 (some channel has c < 32 or a residual shift below 9).
-template <bool GEN, bool RSIGNED, bool SAT, bool OSIGNED, bool RN>
+// GEN: 64-bit arithmetic for every shift 1..62 (a residual shift below 9, or an INT32 residual).  SMALL: some channel
+// of the warp has c < 32 (common with 4-bit operands, whose accumulators are small): funnel-shift form of Eq. 4.
+template <bool GEN, bool RSIGNED, bool SAT, bool OSIGNED, bool RN, bool SMALL = false>
 __device__ __forceinline__ void epilogue_loop_frag(const EpiCtx& e_in) {
   const EpiCtx e = e_in;
   const TcParams& p = *e.p;
@@ -652,7 +654,7 @@ __device__ __forceinline__ void epilogue_loop_frag(const EpiCtx& e_in) {
       const long long y = (((long long)acc * (long long)c.b + c.r0) >> c.sh) + (((long long)r * (long long)c.rb + c.rr0) >> c.rsh);
       return hq_clamp_ll(y, p.relu, p.qmin, p.qmax);
     }
-    const int y = requant_fast<true, RSIGNED, false, RN, true>(acc, r, c);
+    const int y = requant_fast<true, RSIGNED, SMALL, RN, true>(acc, r, c);
     return SAT ? y : min(max(y, e.lo), e.hi);
   };
   // one unit: 16 values per thread -> four words -> one transposing store of 32 pixel rows x 16 channel bytes
@@ -1344,8 +1346,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if constexpr (RTM) {
         // residual through tensor memory: the fragment loop, in its general form when some channel needs 64-bit steps
         const bool rn = warp_narrow;
-        if (!fast || epi_bar_and<32 * EPI_WARPS>(warp_small ? 0u : 1u) == 0u) {
+        if (!fast) {
           if (p.out_signed) epilogue_loop_frag<true, false, false, true, false>(e); else epilogue_loop_frag<true, false, false, false, false>(e);
+        } else if (warp_small) {
+          // (no narrow residual pairs here: the plain multiply-high form of the residual term)
+          if (p.sat_pack) {
+            if (p.out_signed) { if (p.res_signed) epilogue_loop_frag<false, true, true, true, false, true>(e); else epilogue_loop_frag<false, false, true, true, false, true>(e); }
+            else { if (p.res_signed) epilogue_loop_frag<false, true, true, false, false, true>(e); else epilogue_loop_frag<false, false, true, false, false, true>(e); }
+          } else {
+            if (p.out_signed) { if (p.res_signed) epilogue_loop_frag<false, true, false, true, false, true>(e); else epilogue_loop_frag<false, false, false, true, false, true>(e); }
+            else { if (p.res_signed) epilogue_loop_frag<false, true, false, false, false, true>(e); else epilogue_loop_frag<false, false, false, false, false, true>(e); }
+          }
         } else if (p.sat_pack) {
           if (p.out_signed) { if (rn) epilogue_loop_frag<false, false, true, true, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, true, false>(e); else epilogue_loop_frag<false, false, true, true, false>(e); }
           else { if (rn) epilogue_loop_frag<false, false, true, false, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, false, false>(e); else epilogue_loop_frag<false, false, true, false, false>(e); }
