@@ -17,6 +17,7 @@ namespace {
 struct ConcatBranch {
   const void* in; const int32_t* b; const int32_t* c;
   int32_t bits, is_signed, ch, ch_off;
+  int32_t row_ch;     // channels per pixel of the tensor this entry reads (> ch for a piece of a very wide branch)
   int32_t width;      // channels a thread owns: 16, or 4 for an INT32 branch read in 16-byte pieces
   int32_t upp;        // threads (units) per pixel of this branch = ceil(ch / width)
   int32_t block0, nblocks;   // this branch's blocks of the launch
@@ -328,7 +329,7 @@ __device__ __forceinline__ void concat_w4_loop(W4State t, const int (&bb)[4], co
 // pieces of the dense branch tensor and write consecutive words of the output row.
 template <int BITS>
 __device__ __forceinline__ void concat_w4(const ConcatArgs& a, const int i) {
-  const int is_signed = a.br[i].is_signed, ch = a.br[i].ch;
+  const int is_signed = a.br[i].is_signed;
   const int upp = a.br[i].upp, ppb = 256 / upp;
   const int tid = threadIdx.x;
   if (tid >= upp * ppb) return;
@@ -359,7 +360,7 @@ __device__ __forceinline__ void concat_w4(const ConcatArgs& a, const int i) {
   W4State t;
   t.step = (long long)a.br[i].nblocks * ppb;
   t.px = (long long)(blockIdx.x - a.br[i].block0) * ppb + y;
-  t.in_row = (long long)ch * BITS / 8; t.out_row = (long long)a.out_ch * a.out_bits / 8;
+  t.in_row = (long long)a.br[i].row_ch * BITS / 8; t.out_row = (long long)a.out_ch * a.out_bits / 8;
   t.ip = (const unsigned char*)a.br[i].in + t.px * t.in_row + (long long)k0 * BITS / 8;
   t.op = (unsigned char*)a.out + t.px * t.out_row + (long long)off * a.out_bits / 8;
   t.lo = lo; t.hi = hi; t.pixels = a.pixels;
@@ -417,8 +418,11 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     if (qmin > qmax || qmin < lo || qmax > hi) return HQ_ERR_INVALID_ARG;
   }
   ConcatArgs a{};
-  int off = 0;
+  int off = 0, nb = 0;
   long long weight[HQ_CONCAT_MAX_BRANCHES], weight_sum = 0;
+  // A branch of more than 1024 channels (a multiple of 4) is entered as several pieces of at most 1024, each read
+  // with the whole tensor's row pitch, while entries are left; otherwise it takes the sixteen-channel form.
+  int spare = HQ_CONCAT_MAX_BRANCHES - n_branches;
   for (int i = 0; i < n_branches; ++i) {
     const hq_tensor& t = branches[i];
     if (!t.data || !rescale[i].b || !rescale[i].c) return HQ_ERR_INVALID_ARG;
@@ -427,19 +431,28 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
     if (t.bits == 4 && (t.c & 1)) return HQ_ERR_INVALID_ARG;
     if (out->bits == 4 && (t.c & 1)) return HQ_ERR_UNSUPPORTED;   // a byte of the output would span two branches
     if (!al16(t.data)) return HQ_ERR_ALIGNMENT;
-    ConcatBranch& B = a.br[i];
-    B.in = t.data; B.b = rescale[i].b; B.c = rescale[i].c;
-    B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = t.c; B.ch_off = off;
-    if (t.c % 4 == 0 && t.c <= 4 * 256 && out->c % 2 == 0) { B.width = 4; B.vec = 1; }
-    else { B.width = 16; B.vec = (t.bits != 32 && t.c % 16 == 0) ? 1 : 0; }
-    B.upp = (t.c + B.width - 1) / B.width;
-    if (B.upp > 256) return HQ_ERR_UNSUPPORTED;                   // more than 4096 channels in one branch
-    weight[i] = (long long)t.c * (t.bits + out->bits);
-    weight_sum += weight[i];
-    off += t.c;
+    const bool four = t.c % 4 == 0 && out->c % 2 == 0;
+    int pieces = 1;
+    if (four && t.c > 1024) {
+      pieces = (t.c + 1023) / 1024;
+      if (pieces - 1 > spare) pieces = 1; else spare -= pieces - 1;
+    }
+    for (int pc = 0, k0 = 0; pc < pieces; ++pc) {
+      const int chp = pieces == 1 ? t.c : (t.c - k0 < 1024 ? t.c - k0 : 1024);
+      ConcatBranch& B = a.br[nb];
+      B.in = (const unsigned char*)t.data + (long long)k0 * t.bits / 8; B.b = rescale[i].b + k0; B.c = rescale[i].c + k0;
+      B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = chp; B.ch_off = off; B.row_ch = t.c;
+      if (four && chp <= 4 * 256) { B.width = 4; B.vec = 1; }
+      else { B.width = 16; B.vec = (t.bits != 32 && t.c % 16 == 0) ? 1 : 0; }
+      B.upp = (chp + B.width - 1) / B.width;
+      if (B.upp > 256) return HQ_ERR_UNSUPPORTED;                 // more than 4096 channels in one branch
+      weight[nb] = (long long)chp * (t.bits + out->bits);
+      weight_sum += weight[nb];
+      off += chp; k0 += chp; ++nb;
+    }
   }
   if (off != out->c) return HQ_ERR_INVALID_ARG;
-  a.n_br = n_branches; a.out_ch = out->c; a.out_bits = out->bits;
+  a.n_br = nb; a.out_ch = out->c; a.out_bits = out->bits;
   a.relu = relu; a.qmin = qmin; a.qmax = qmax;
   a.pixels = (long long)out->n * out->h * out->w;
   a.out = out->data;
@@ -447,7 +460,7 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
   // blocks of the one launch, dealt to the branches in proportion to the bytes they move
   const long long cap = (long long)h->sm_count * 8;
   long long blocks4 = 0, blocks16 = 0;
-  for (int i = 0; i < n_branches; ++i) {
+  for (int i = 0; i < nb; ++i) {
     ConcatBranch& B = a.br[i];
     const long long per_block = (long long)(256 / B.upp) * (B.width == 4 && B.bits != 32 ? 8 : kPix);
     const long long need = (a.pixels + per_block - 1) / per_block;

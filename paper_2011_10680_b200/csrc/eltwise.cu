@@ -998,8 +998,10 @@ cudaError_t hq_launch_residual_add(const EltArgs& a, int sm_count, cudaStream_t 
   }
   // 8-bit operands with a channel count the word mapping covers: 32-bit fast kernel
   const int words = a.ch / 4;
-  if (a.main_bits == 8 && (!a.res || a.res_bits == 8) && a.ch % 4 == 0 && (words <= 256 || words % 256 == 0)) {
-    const int bx = words <= 256 ? words : 256;
+  if (a.main_bits == 8 && (!a.res || a.res_bits == 8) && a.ch % 4 == 0) {
+    // more than 256 words per pixel: the fewest blocks along the words, each a whole number of warps wide
+    const int xblocks = (words + 255) / 256;
+    const int bx = words <= 256 ? words : ((words + xblocks - 1) / xblocks + 31) / 32 * 32;
     int by = 256 / bx; if (by < 1) by = 1;
     dim3 block(bx, by), grid((words + bx - 1) / bx, 1);
     long long gy = (a.pixels + by - 1) / by;

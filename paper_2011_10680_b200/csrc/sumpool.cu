@@ -4,7 +4,8 @@
 // pair of the consumer (hq_concat_requant, hq_residual_add), so no division touches the data.  Memory bound: a
 // thread owns four channels of one output pixel (one 16-byte read per tap of an INT32 tensor, served by L1 / L2 for
 // the overlapping windows, one word of an 8-bit tensor) and writes one 16-byte piece of the INT32 output; other
-// channel counts and 4-bit inputs read element-wise.
+// channel counts and 4-bit inputs read element-wise.  The 3 x 3 / stride 1 / pad 1 window of the Inception modules has
+// its own kernel, which forms every row's three-pixel sum once (sumpool3_rows_kernel).
 #include "hq_internal.cuh"
 
 namespace {
@@ -80,6 +81,75 @@ __global__ void __launch_bounds__(256) sumpool_kernel(const __grid_constant__ Su
   }
 }
 
+// 3 x 3 / stride 1 / pad 1 (the pooling branch of an Inception module) with four channels per thread.  A thread walks
+// down one output column of a strip of rows: the sum over the three pixels (ow - 1, ow, ow + 1) of an input row is
+// formed once and serves the three output rows it belongs to, so an output costs three reads instead of nine; the
+// sums of the last two rows stay in registers.  Consecutive threads hold consecutive channel groups of a pixel, then
+// the next pixel: reads and the 16-byte stores are consecutive across a warp.  8-bit inputs are summed as two pairs
+// of 16-bit lanes per word (nine bytes add up to at most 2295); signed bytes are biased by 128 first (a tap outside
+// the image counts as the biased zero), and 9 * 128 comes off at the end.
+template <int IN8, int SIGNED>
+__global__ void __launch_bounds__(256) sumpool3_rows_kernel(const __grid_constant__ SumPoolArgs a, int strip_rows, int strips) {
+  const int cg = a.ch >> 2;
+  const int col = blockIdx.x * 256 + threadIdx.x;
+  if (col >= a.w * cg) return;
+  const int ow = col / cg, g = col - ow * cg;
+  const int img = blockIdx.y / strips, strip = blockIdx.y - img * strips;
+  const int r0 = strip * strip_rows, r1 = min(r0 + strip_rows, a.h);
+  const bool left = ow > 0, right = ow + 1 < a.w;
+  const long long img_row0 = (long long)img * a.h;
+  int4* __restrict__ outp = (int4*)a.out + ((img_row0 + r0) * a.w + ow) * cg + g;
+  const long long out_step = (long long)a.w * cg;
+  if constexpr (IN8) {
+    const unsigned* __restrict__ in = (const unsigned*)a.in;
+    constexpr unsigned kBias = SIGNED ? 0x80808080u : 0u;
+    // the row's three-pixel sum as (bytes 0, 2) and (bytes 1, 3) in 16-bit lanes
+    auto hsum = [&](int ih, unsigned& lo, unsigned& hi) {
+      unsigned v0 = 0, v1 = 0, v2 = 0;
+      if (ih >= 0 && ih < a.h) {
+        const unsigned* row = in + ((img_row0 + ih) * a.w + ow) * cg + g;
+        v1 = __ldg(row);
+        if (left) v0 = __ldg(row - cg);
+        if (right) v2 = __ldg(row + cg);
+      }
+      v0 ^= kBias; v1 ^= kBias; v2 ^= kBias;
+      lo = (v0 & 0x00FF00FFu) + (v1 & 0x00FF00FFu) + (v2 & 0x00FF00FFu);
+      hi = ((v0 >> 8) & 0x00FF00FFu) + ((v1 >> 8) & 0x00FF00FFu) + ((v2 >> 8) & 0x00FF00FFu);
+    };
+    unsigned l0, h0, l1, h1;
+    hsum(r0 - 1, l0, h0);
+    hsum(r0, l1, h1);
+#pragma unroll 4
+    for (int oh = r0; oh < r1; ++oh, outp += out_step) {
+      unsigned l2, h2;
+      hsum(oh + 1, l2, h2);
+      const unsigned lo = l0 + l1 + l2, hi = h0 + h1 + h2;
+      constexpr int kOff = SIGNED ? 9 * 128 : 0;
+      *outp = make_int4((int)(lo & 0xFFFFu) - kOff, (int)(hi & 0xFFFFu) - kOff, (int)(lo >> 16) - kOff, (int)(hi >> 16) - kOff);
+      l0 = l1; h0 = h1; l1 = l2; h1 = h2;
+    }
+  } else {
+    const int4* __restrict__ in = (const int4*)a.in;
+    auto hsum = [&](int ih) -> int4 {
+      int4 s = make_int4(0, 0, 0, 0);
+      if (ih >= 0 && ih < a.h) {
+        const int4* row = in + ((img_row0 + ih) * a.w + ow) * cg + g;
+        s = __ldg(row);
+        if (left) { const int4 v = __ldg(row - cg); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+        if (right) { const int4 v = __ldg(row + cg); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+      }
+      return s;
+    };
+    int4 s0 = hsum(r0 - 1), s1 = hsum(r0);
+#pragma unroll 4
+    for (int oh = r0; oh < r1; ++oh, outp += out_step) {
+      const int4 s2 = hsum(oh + 1);
+      *outp = make_int4(s0.x + s1.x + s2.x, s0.y + s1.y + s2.y, s0.z + s1.z + s2.z, s0.w + s1.w + s2.w);
+      s0 = s1; s1 = s2;
+    }
+  }
+}
+
 }  // namespace
 
 extern "C" hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, int32_t stride, int32_t pad,
@@ -99,6 +169,21 @@ extern "C" hq_status hq_sumpool(hq_handle* h, const hq_tensor* in, int32_t k, in
   a.k = k; a.stride = stride; a.pad = pad; a.oh_n = ho; a.ow_n = wo;
   a.vec = in->c % 4 != 0 ? 0 : in->bits == 32 ? 1 : in->bits == 8 ? 2 : 0;
   if (a.n == 0) return HQ_OK;
+  if (a.vec && k == 3 && stride == 1 && pad == 1) {
+    // strips of rows: long enough that the two extra input rows per strip matter little, short enough to fill the GPU
+    const long long cols3 = (long long)a.w * (a.ch / 4);
+    int strip_rows = 8;
+    while (strip_rows > 2 && (cols3 + 255) / 256 * a.n * ((a.h + strip_rows - 1) / strip_rows) < 16LL * h->sm_count) strip_rows >>= 1;
+    const int strips = (a.h + strip_rows - 1) / strip_rows;
+    if ((cols3 + 255) / 256 <= 0x7fffffffLL && (long long)a.n * strips <= 65535) {
+      const dim3 grid3((unsigned)((cols3 + 255) / 256), (unsigned)(a.n * strips));
+      cudaStream_t st = (cudaStream_t)stream;
+      if (a.vec == 1) sumpool3_rows_kernel<0, 0><<<grid3, 256, 0, st>>>(a, strip_rows, strips);
+      else if (a.is_signed) sumpool3_rows_kernel<1, 1><<<grid3, 256, 0, st>>>(a, strip_rows, strips);
+      else sumpool3_rows_kernel<1, 0><<<grid3, 256, 0, st>>>(a, strip_rows, strips);
+      return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+    }
+  }
   const long long rows = (long long)a.n * ho, cols = (long long)wo * (a.vec ? a.ch / 4 : a.ch);
   if (rows > 0x7fffffffLL || (cols + 255) / 256 > 65535) return HQ_ERR_UNSUPPORTED;
   const dim3 grid((unsigned)rows, (unsigned)((cols + 255) / 256));

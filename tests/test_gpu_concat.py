@@ -43,9 +43,12 @@ def run_and_compare(hq, case):
 INCEPTION_A = [(64, 8, 0), (64, 8, 0), (96, 8, 0), (32, 32, 1)]            # 35x35 module: 1x1, 5x5, double 3x3, pool (INT32)
 INCEPTION_C = [(192, 8, 0), (192, 8, 0), (192, 8, 0), (192, 32, 1)]        # 17x17 module
 RAGGED = [(6, 8, 1), (20, 32, 1), (10, 4, 0), (48, 8, 0), (2, 32, 1), (16, 4, 1)]   # odd group sizes, unaligned offsets
+VERY_WIDE = [(192, 8, 0), (1088, 32, 1), (2120, 8, 1), (64, 8, 0)]         # branches of more than 1024 channels: entered in pieces
+TOO_MANY_PIECES = [(8, 8, 0)] * 6 + [(3080, 8, 0), (16, 32, 1)]            # no entries left for pieces: sixteen-channel form
 
 
-@pytest.mark.parametrize("branches,n,hw", [(INCEPTION_A, 3, 35), (INCEPTION_C, 2, 17), (RAGGED, 2, 9)])
+@pytest.mark.parametrize("branches,n,hw", [(INCEPTION_A, 3, 35), (INCEPTION_C, 2, 17), (RAGGED, 2, 9), (VERY_WIDE, 2, 9),
+                                          (TOO_MANY_PIECES, 1, 7)])
 @pytest.mark.parametrize("out_bits,out_signed,relu", [(8, 0, 1), (8, 1, 0), (4, 0, 1)])
 def test_concat_matches_the_oracle(hq, branches, n, hw, out_bits, out_signed, relu):
     case = inputs.concat_case(401, n, hw, branches, out_bits, out_signed, relu)
@@ -158,6 +161,10 @@ def test_concat_empty_batch_is_a_no_op(hq):
     (2, 8, 8, 10, 8, 0, 3, 1, 1),
     (1, 6, 5, 8, 4, 1, 2, 2, 0),
     (1, 7, 7, 4, 8, 1, 5, 1, 2),
+    (3, 35, 35, 288, 8, 0, 3, 1, 1),        # the layer-table form: 8-bit module input, four channels per thread
+    (2, 17, 19, 64, 8, 1, 3, 1, 1),         # signed bytes, H != W, several strips of rows
+    (1, 1, 1, 8, 8, 1, 3, 1, 1),            # a single pixel: every neighbour is padding
+    (2, 3, 40, 12, 32, 1, 3, 1, 1),         # fewer rows than a strip
 ])
 def test_sumpool_matches_the_oracle(hq, n, h, w, ch, bits, signed, k, stride, pad):
     from oracle import hqref

@@ -439,6 +439,10 @@ LARGE_ELT_CASES = [
     ((331, 251), 128, 0, None, 4, "fast"),     # 4-bit output packed from high nibbles (shifts reduced by four)
     ((331, 251), 128, 1, None, 4, "every"),    # the same with shifts below four in some warps (plain clamp there)
     ((157, 131), 128, 0, None, 4, "every"),
+    # more than 256 words per pixel that do not divide into blocks of 256 (the 17x17 Inception module's 1088 channels)
+    ((53, 41), 1088, 0, None, 4, "fast"),
+    ((53, 41), 1088, 0, 1, 8, "every"),
+    ((37, 29), 2052, 1, None, 8, "fast"),
 ]
 
 
