@@ -54,6 +54,42 @@ __global__ void __launch_bounds__(256) patch_matrix_kernel(const unsigned char* 
   }
 }
 
+// The same for channel counts that are a multiple of 16 (e.g. the 48-channel branches of an Inception module): the
+// window rows, the taps of a filter row and the patch rows are then whole 16-byte pieces, so both passes move
+// 16 bytes per access and a patch piece is one shared-memory read.
+__global__ void __launch_bounds__(256) patch_matrix_vec16_kernel(const uint4* __restrict__ in, int n, int h, int w,
+                                                                 int cin, int kh, int kw, int stride, int pad, int ho, int wo,
+                                                                 int K, int Kp, int wseg, int segs, int win_bytes,
+                                                                 uint4* __restrict__ out) {
+  extern __shared__ uint4 win16[];                           // [kh][win_bytes / 16]
+  const int seg = blockIdx.x % segs;
+  const int oh = (blockIdx.x / segs) % ho;
+  const int img = blockIdx.x / (segs * ho);
+  const int ow0 = seg * wseg;
+  const int npix = (wo - ow0) < wseg ? (wo - ow0) : wseg;
+  const int c16 = cin >> 4, wq = win_bytes >> 4, rowq = w * c16;
+  const int col0 = (ow0 * stride - pad) * c16;                // first 16-byte piece of the window inside an input row
+  for (int i = threadIdx.x; i < kh * wq; i += blockDim.x) {
+    const int r = i / wq, b = i - r * wq;
+    const int ih = oh * stride + r - pad, col = col0 + b;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (ih >= 0 && ih < h && col >= 0 && col < rowq) v = __ldg(in + ((long long)img * h + ih) * rowq + col);
+    win16[i] = v;
+  }
+  __syncthreads();
+  const int cpr = Kp >> 4, kq = K >> 4, kwq = kw * c16;
+  uint4* dst = out + (((long long)img * ho + oh) * wo + ow0) * cpr;
+  for (int i = threadIdx.x; i < npix * cpr; i += blockDim.x) {
+    const int px = i / cpr, j = i - px * cpr;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (j < kq) {
+      const int r = j / kwq, t = j - r * kwq;
+      v = win16[r * wq + px * stride * c16 + t];
+    }
+    dst[i] = v;
+  }
+}
+
 __global__ void pad_weights_kernel(const unsigned char* __restrict__ wgt, int cout, int K, int Kp,
                                    unsigned char* __restrict__ out) {
   const long long total = (long long)cout * Kp;
@@ -105,6 +141,11 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
     if (smem > 48 * 1024) return HQ_ERR_UNSUPPORTED;
     const long long blocks = (long long)a.n * a.ho * segs;
     if (blocks >= (1ll << 31)) return HQ_ERR_UNSUPPORTED;
+    if (a.cin % 16 == 0 && ((uintptr_t)a.in & 15u) == 0 && !a.pitch_w)
+      patch_matrix_vec16_kernel<<<(int)blocks, 256, smem, s>>>((const uint4*)a.in, a.n, a.h, a.w, a.cin, a.kh, a.kw,
+                                                               a.stride, a.pad, a.ho, a.wo, K, Kp, wseg, segs, win_bytes,
+                                                               (uint4*)patches);
+    else
     patch_matrix_kernel<<<(int)blocks, 256, smem, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, a.cin, a.kh, a.kw,
                                                        a.stride, a.pad, a.ho, a.wo, K, Kp, wseg, segs, win_bytes,
                                                        (uint4*)patches);
