@@ -199,13 +199,14 @@ def run_sweep(args):
             for residual in ((False, True) if has_res else (False,)):
                 case = inputs.conv_case(5, n, hw, hw, cin, cout, k, stride, k // 2, bits=bits, residual=residual)
                 dev = binding.upload_case(case)
+                out = binding.alloc_out(case["n"], case["ho"], case["wo"], case["cout"], case["out_bits"], case["out_signed"])
                 times = []
                 for rep in range(args.warmup + args.steps):
                     flush.fill_(rep & 0xFF)
                     flush_r.view(torch.int32).sum()    # then 256 MB read: no backlog of dirty lines charged to the timed kernel
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
-                    st, out = hq.conv_case(case, dev)
+                    st, _ = hq.conv_case(case, dev, out)
                     e1.record()
                     assert st == binding.HQ_OK
                     torch.cuda.synchronize()

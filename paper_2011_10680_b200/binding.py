@@ -260,10 +260,12 @@ class Handle:
         return lib().hq_maxpool(self._h, C.byref(ti), k, stride, pad, C.byref(to), _stream())
 
     # ---- convenience for the dict-shaped single-layer cases of the workload generator -------
-    def conv_case(self, case: dict, dev: dict | None = None):
-        """Upload (or reuse `dev`) a generated conv case, run hq_conv2d, return (status, out tensor)."""
+    def conv_case(self, case: dict, dev: dict | None = None, out=None):
+        """Upload (or reuse `dev`) a generated conv case, run hq_conv2d, return (status, out tensor).  `out`: an output
+        tensor allocated by the caller (a timing loop keeps the allocation and its guard-band fills out of the timed region)."""
         dev = dev if dev is not None else upload_case(case)
-        out = alloc_out(case["n"], case["ho"], case["wo"], case["cout"], case["out_bits"], case["out_signed"])
+        if out is None:
+            out = alloc_out(case["n"], case["ho"], case["wo"], case["cout"], case["out_bits"], case["out_signed"])
         st = self.conv2d(dev["x"], case["bits"], case["in_signed"], case["cin"], dev["wgt"], case["cout"], case["kh"],
                          case["kw"], case["stride"], case["pad"], dev["bias"], dev["b"], dev["c"], out,
                          case["out_bits"], case["out_signed"], dev["res"], case["res_bits"], case["res_signed"],
