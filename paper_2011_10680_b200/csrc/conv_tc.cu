@@ -1526,6 +1526,10 @@ bool hq_conv_tc_supported(const ConvArgs& a) {
   if ((long long)a.kh * a.kw * a.cin >= (1ll << 24)) return false;
   if (a.out_bits == 4 && (a.cout & 1)) return false;
   if (a.res && !(a.res_bits == 8 || a.res_bits == 32)) return false;
+  // the corners of an im2col-mode tensor map are 8-bit signed offsets: wider filters are declined here, before any
+  // map is encoded (more channel tiles than the GPU has SMs are declined by the launcher, which knows the count)
+  const int pad_after = a.pad + a.pad_after_delta;
+  if (pad_after - (a.kw - 1) < -128 || pad_after - (a.kh - 1) < -128 || pad_after > 127) return false;
   return true;
 }
 

@@ -46,6 +46,18 @@ def run_conv_and_compare(hq, case, path):
         raise AssertionError(f"{len(bad)} of {ref.size} outputs differ; first at {bad[0]}: got {got[tuple(bad[0])]} want {ref[tuple(bad[0])]}")
 
 
+@pytest.mark.parametrize("shape", [
+    (1, 136, 136, 32, 8, 131, 1, 0),      # a filter wider than an im2col tensor map's corner range (kw > pad + 129)
+    (1, 8, 8, 32, 19072, 1, 1, 0),        # more channel tiles than a persistent grid has CTAs
+])
+def test_automatic_path_falls_back_when_the_tensor_core_launcher_declines(hq, shape):
+    """Shapes that pass the tensor-core path's argument checks but that its launcher declines before launching anything:
+    the automatic path must still return the right integers (CUDA-core kernel), not the launcher's status."""
+    n, h, w, cin, cout, k, stride, pad = shape
+    case = inputs.conv_case(311, n, h, w, cin, cout, k, stride, pad, c_range=(40, 46))
+    run_conv_and_compare(hq, case, 0)
+
+
 # ------------------------------------------------------------------ CUDA-core conv path --------
 CORE_CASES = [
     # n, h, w, cin, cout, k, stride, pad, bits, out_bits, residual, res_bits, relu

@@ -14,9 +14,12 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 CASES = [
-    # n, h, w, cin, cout, k, stride, pad, residual: two calls in a row on the shared fixed array
-    (2, 32, 32, 3, 16, 7, 2, 3, False),
-    (1, 20, 20, 5, 32, 3, 1, 1, True),
+    # n, h, w, cin, cout, k, stride, pad, residual, out_bits: calls in a row on the shared fixed array
+    (2, 32, 32, 3, 16, 7, 2, 3, False, 8),
+    (1, 20, 20, 5, 32, 3, 1, 1, True, 8),
+    (2, 24, 24, 3, 16, 3, 1, 1, False, 4),       # packed 4-bit outputs
+    (1, 18, 22, 6, 24, 3, 2, 1, False, 32),      # raw INT32 accumulators
+    (4, 228, 228, 3, 64, 7, 2, 3, False, 8),     # patch matrix + weights = 8327680 bytes: just inside the 8 MiB array
 ]
 
 
@@ -27,8 +30,9 @@ def test_noalloc_conv_matches_the_allocating_entry_point_twice_in_a_row():
     build.build()
     hq = binding.Handle(0)                      # only for the entry point being compared against
     try:
-        for i, (n, h, w, cin, cout, k, stride, pad, residual) in enumerate(CASES):
-            case = inputs.conv_case(900 + i, n, h, w, cin, cout, k, stride, pad, residual=residual, c_range=(38, 42))
+        for i, (n, h, w, cin, cout, k, stride, pad, residual, out_bits) in enumerate(CASES):
+            case = inputs.conv_case(900 + i, n, h, w, cin, cout, k, stride, pad, residual=residual, c_range=(38, 42),
+                                    out_bits=out_bits, relu=out_bits != 32)
             dev = binding.upload_case(case)
             st, want = hq.conv_case(case, dev)                     # existing entry point (scratch from cudaMalloc)
             assert st == binding.HQ_OK
@@ -46,9 +50,9 @@ def test_noalloc_conv_matches_the_allocating_entry_point_twice_in_a_row():
             ref = hqref.conv_case(case)
             assert np.array_equal(got.cpu().numpy().view(ref.dtype).reshape(ref.shape), ref)
         # a request beyond the fixed 8 MiB array is refused with a clear status, nothing is launched
-        big = inputs.conv_case(990, 8, 224, 224, 3, 64, 7, 2, 3)
+        big = inputs.conv_case(990, 4, 230, 230, 3, 64, 7, 2, 3)       # 8474240 bytes: just outside
         dev = binding.upload_case(big)
-        out = binding.alloc_out(8, big["ho"], big["wo"], 64, 8, 0)
+        out = binding.alloc_out(4, big["ho"], big["wo"], 64, 8, 0)
         assert binding.conv2d_noalloc(big, dev, out) == binding.HQ_ERR_WORKSPACE
         assert binding.status_string(binding.HQ_ERR_WORKSPACE) == "HQ_ERR_WORKSPACE"
     finally:
