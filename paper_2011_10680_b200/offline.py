@@ -13,13 +13,15 @@ Nothing in this module is called while a layer runs.
     quantize_network   a list of float layers with static activation scales -> a layer table for hq_run_network
     float_forward      the float network evaluated in numpy (what the scales are calibrated on)
     calibrate          static activation scales from float activations (Appendix B: static quantization)
+    fold_input_zero_point   an input tensor with a non-zero zero point Z (Eq. 2): Z leaves the tensor, its effect
+                            goes into the first layer's INT32 bias
 """
 from __future__ import annotations
 
 import numpy as np
 
 __all__ = ["dyadic_from_scale", "fold_bn", "quantize_weights", "quantize_bias", "conv_params", "quantize_network",
-           "float_forward", "calibrate"]
+           "float_forward", "calibrate", "fold_input_zero_point"]
 
 
 # --------------------------------------------------------------------------------------------
@@ -228,3 +230,25 @@ def quantize_network(layers: list[dict], s_image: float, image_hw: int | None = 
             raise ValueError(f"unknown op {op!r}")
     classes = table[-1]["cout"] if table and table[-1]["op"] == "linear" else None
     return {"layers": table, "scales": [scale[i] for i in range(len(layers))], "image_hw": image_hw, "classes": classes}
+
+
+
+# --------------------------------------------------------------------------------------------
+# Non-zero zero point of the network input (Eq. 2 carries a zero point, Eq. 3-4 do not)
+# --------------------------------------------------------------------------------------------
+def fold_input_zero_point(q_bias: np.ndarray, q_w: np.ndarray, z: int, pad: int = 0) -> np.ndarray:
+    """The kernels compute sum_k q_x[k] q_w[k] on stored values with zero point 0.  For an input whose
+    real value is S (q_x - Z), sum_k (q_x[k] - Z) q_w[oc, k] = sum_k q_x[k] q_w[oc, k] - Z sum_k q_w[oc, k]:
+    the correction is a per-channel constant and moves into the INT32 bias, exactly.  That holds where every
+    tap of the window reads a stored value, i.e. for an unpadded layer (padding writes the integer 0, which
+    stands for the real value -S Z, not 0); a padded first layer needs the input re-centred instead, which for
+    Z = 128 on 8-bit data is the signed image the kernels accept as it is.
+
+    q_bias: INT32 bias at S_h S_w (quantize_bias); q_w: integer weights [cout, kh, kw, cin]."""
+    if pad != 0:
+        raise ValueError("the fold is exact for unpadded layers only: re-centre the input (Z = 128: signed image) instead")
+    corr = np.asarray(q_w, np.int64).reshape(q_w.shape[0], -1).sum(axis=1) * int(z)
+    out = np.asarray(q_bias, np.int64) - corr
+    if np.any(out < -(1 << 31)) or np.any(out >= (1 << 31)):
+        raise ValueError("the folded bias leaves the INT32 range")
+    return out.astype(np.int32)

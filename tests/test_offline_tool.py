@@ -118,3 +118,28 @@ def test_quantized_network_tracks_its_float_evaluation():
     assert np.array_equal(np.argmax(logits, axis=1), np.argmax(f4, axis=1))
     # the residual operand of layer 2 is the block input (layer 0), with its own DN(S_r / S_a)
     assert net["layers"][2]["in1"] == 0 and net["layers"][2]["rb"] is not None
+
+
+def test_input_zero_point_folds_into_the_bias_exactly():
+    """Eq. 2's zero point on the network input: conv(q_x - Z) with bias equals conv(q_x) with the folded bias,
+    integer for integer (unpadded layer), checked through the oracle's convolution; a padded layer is refused."""
+    import pytest
+    from oracle import hqref
+    g = np.random.default_rng(7)
+    n, hw, cin, cout, k, z = 2, 9, 3, 6, 3, 117
+    qx = g.integers(0, 256, size=(n, hw, hw, cin)).astype(np.uint8)
+    qw = g.integers(-127, 128, size=(cout, k, k, cin)).astype(np.int8)
+    qb = g.integers(-(1 << 15), 1 << 15, size=cout).astype(np.int32)
+    folded = offline.fold_input_zero_point(qb, qw, z)
+    got = hqref.conv2d(qx, cin, 8, 0, qw, cout, k, k, 1, 0, folded, None, None, out_bits=32, out_signed=1,
+                       qmin=-(1 << 31), qmax=(1 << 31) - 1)
+    want = float_conv(qx.astype(np.float64) - z, qw.astype(np.float64), 1, 0) + qb         # exact in doubles at these sizes
+    assert np.array_equal(got.astype(np.int64), want.astype(np.int64))
+    with pytest.raises(ValueError):
+        offline.fold_input_zero_point(qb, qw, z, pad=1)
+    # Z = 128 on 8-bit data is the signed image: same real values, no fold needed
+    signed = (qx.astype(np.int16) - 128).astype(np.int8)
+    a = hqref.conv2d(signed, cin, 8, 1, qw, cout, k, k, 1, 1, qb, None, None, out_bits=32, out_signed=1,
+                     qmin=-(1 << 31), qmax=(1 << 31) - 1)
+    b = float_conv(qx.astype(np.float64) - 128, qw.astype(np.float64), 1, 1) + qb
+    assert np.array_equal(a.astype(np.int64), b.astype(np.int64))
