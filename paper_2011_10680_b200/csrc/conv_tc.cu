@@ -82,6 +82,7 @@ struct TcParams {
   int32_t rtm;           // 1: the 8-bit residual tile reaches the epilogue through tensor memory: an MMA with the identity
                          //    matrix as its A operand turns the [pixels][128 channels] byte tile into INT32 columns beside
                          //    the accumulator, in the accumulator's own layout (see epilogue_loop_frag)
+  int32_t acc_bits;      // |accumulator| < 2^acc_bits for every 8-bit operand pair: ceil(log2(K * 255 * 128 + 1))
   int32_t acc_stride;    // tensor-memory columns between accumulator buffers: pt, or 2 * pt with rtm
   uint32_t ident_off;    // rtm: offset of the 128 x 128 identity matrix (16 KiB, 128-byte swizzle) from the 1024-aligned base
   int32_t duo;           // 1: two CTAs of a cluster (adjacent SMs) share every MMA: 256 channels x 256 pixels per pair
@@ -372,6 +373,7 @@ struct ChanConst {
   int b, sh;            // main branch multiplier; shift (c, or c - min(c,32) on the fast path)
   int sh1;              // fast path: min(c, 32), the part of the shift taken by the funnel shift
   int cmin31;           // fast path: min(c, 31)
+  int pre;              // pre-shift form (SMALL == 2): 32 - min(c, 32), the accumulator is shifted left by it first
   long long r0;         // bias*b + 2^(c-1)
   int rb, rh, rsh;      // residual multiplier; fast path: rh = 2^(rc-9), rsh = rc-8; else rsh = rc
   long long rr0;        // general path: 2^(rc-1)
@@ -384,21 +386,26 @@ struct ChanConst {
 // The residual form is exact: (r<<24)*rb >> 32 = floor(r*rb / 2^8), the rounding constant 2^(rc-1) is
 // a multiple of 2^8, and the dropped low 8 bits of r*rb cannot carry across a multiple of 2^(rc-8).
 // (A 64-bit multiply-add followed by a funnel shift measured no faster.)  `r` is the stored 8-bit
-// residual, already extended.  SMALL: some channel of the warp has c < 32.
+// residual, already extended.  SMALL: 1 when some channel of the warp has c < 32 (exact funnel-shift form with a
+// saturation guard); 2 when, besides, every such channel's accumulator and bias are known to stay below 2^(c-2)
+// (TcParams::acc_bits, checked per channel when the constants are set up): the accumulator is then shifted left by
+// 32 - c first and r0 was shifted with it, (acc << pre) * b + (r0 << pre) = (acc * b + r0) << pre exactly and without
+// overflow, and the plain form applies again at the cost of one shift.
 // RN: every channel of the warp has a narrow residual pair (m, a, s) with (r*m + a) >> s equal to the residual
 // term for all 256 values of r (found and checked exhaustively by residual_narrow_kernel); rb / rh / rsh hold
 // m / a / s then, and a 32-bit multiply-add replaces the shift, multiply-high and add.
 // SPELLED: the product is written as the 32 x 32 -> 64 multiply-add instruction it is.  In the fragment loop, left
 // to the compiler, the sign extension of k.b is hoisted out of the loop and the product becomes a full 64 x 64
 // multiply (three to four multiply instructions per value); the other loops compile to the short form by themselves.
-template <bool RES, bool RSIGNED, bool SMALL, bool RN = false, bool SPELLED = false>
+template <bool RES, bool RSIGNED, int SMALL, bool RN = false, bool SPELLED = false>
 __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) {
+  if (SMALL == 2) acc <<= k.pre;
   long long t1;
   if (SPELLED) asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(t1) : "r"(acc), "r"(k.b), "l"(k.r0));
   else t1 = (long long)acc * (long long)k.b + k.r0;
   int s;
-  if (!SMALL) {
-    s = (int)(t1 >> 32) >> k.sh;                       // c >= 32: |s| < 2^30
+  if (SMALL != 1) {
+    s = (int)(t1 >> 32) >> k.sh;                       // c >= 32 (or pre-shifted): |s| < 2^30
   } else {
     // some channel of this warp has c < 32: take bits [c, c+32) of the 64-bit value with a funnel shift
     // and saturate to +-2^30 when the exact value does not fit (it is far outside every clamp range then,
@@ -462,12 +469,14 @@ struct EpiCtx {
 // next one (of this tile, or the first of the group's next tile) streams from tensor memory into the
 // other register set; the accumulator buffer is handed back as soon as its last chunk has been read,
 // the residual tile as soon as its last bytes have been used, both before the tile's store is issued.
-template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, bool SMALL, bool RN, bool OUT4 = false>
+template <bool RES, bool RSIGNED, bool SAT, bool OSIGNED, int SMALL, bool RN, bool OUT4 = false>
 __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const ChanConst& k_in) {
   // Private copies: the caller's objects live in local memory (their address is passed to the general
   // loop), so every asm statement with a memory clobber would force their fields to be re-read.
   const EpiCtx e = e_in;
-  const ChanConst k = k_in;
+  ChanConst k_own = k_in;
+  if (SMALL == 2) k_own.r0 <<= k_own.pre;          // the pre-shift form of requant_fast
+  const ChanConst k = k_own;
   const TcParams& p = *e.p;
   SharedCtl& ctl = *e.ctl;
   const int lane = e.lane, q = e.q, cq = e.cq, col0 = e.col0, px_per_warp = e.px_per_warp;
@@ -582,7 +591,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
 
 // Per-channel constants of one output channel (Eq. 4 and the residual rescale of Section 3.3), as the loops below want
 // them: `fast` selects the 32-bit forms (see requant_fast), `narrow` the checked narrow residual pair of the channel.
-__device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, bool fast, bool narrow) {
+__device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, bool fast, bool narrow, bool pre = false) {
   ChanConst k{};
   const bool live = ch < p.C;
   k.bias = (live && p.bias) ? p.bias[ch] : 0;
@@ -600,6 +609,8 @@ __device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, b
     k.sh1 = k.sh < 32 ? k.sh : 32;
     k.cmin31 = k.sh < 31 ? k.sh : 31;
     k.sh -= k.sh1;
+    k.pre = 32 - k.sh1;
+    if (pre) k.r0 <<= k.pre;                                         // the pre-shift form (the caller checked its bounds)
     if (p.res) {
       if (k.rsh >= 40) { k.rb = 0; k.rh = 0; k.rsh = 1; }            // |r*rb| < 2^39: rounds to 0
       else { k.rh = 1 << (k.rsh - 9); k.rsh -= 8; }
@@ -628,7 +639,7 @@ __device__ __forceinline__ ChanConst chan_const_for(const TcParams& p, int ch, b
 // there, stores the [128][128] box (128-byte swizzle, as it was loaded) and hands the buffer back.
 // GEN: 64-bit arithmetic for every shift 1..62 (a residual shift below 9, or an INT32 residual).  SMALL: some channel
 // of the warp has c < 32 (common with 4-bit operands, whose accumulators are small): funnel-shift form of Eq. 4.
-template <bool GEN, bool RSIGNED, bool SAT, bool OSIGNED, bool RN, bool SMALL = false>
+template <bool GEN, bool RSIGNED, bool SAT, bool OSIGNED, bool RN, int SMALL = 0>
 __device__ __forceinline__ void epilogue_loop_frag(const EpiCtx& e_in) {
   const EpiCtx e = e_in;
   const TcParams& p = *e.p;
@@ -637,7 +648,7 @@ __device__ __forceinline__ void epilogue_loop_frag(const EpiCtx& e_in) {
   const int t4 = lane >> 2;
   ChanConst k[2];                                   // channels 32 q + 16 hh + 8 r + t4, r = 0, 1
 #pragma unroll
-  for (int r = 0; r < 2; ++r) k[r] = chan_const_for(p, e.c_tile * kTileC + 32 * q + 16 * hh + 8 * r + t4, !GEN, RN);
+  for (int r = 0; r < 2; ++r) k[r] = chan_const_for(p, e.c_tile * kTileC + 32 * q + 16 * hh + 8 * r + t4, !GEN, RN, SMALL == 2);
   const uint32_t bmask = (1u << p.lg_bufs) - 1u, rmask = (1u << p.lg_rbufs) - 1u;
   constexpr int units = 4;                          // 32 pixel columns per unit, 128-pixel tiles
   const uint32_t t_lane = e.tmem_base + ((uint32_t)(q * 32 + 16 * hh) << 16);
@@ -1317,10 +1328,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     fast = epi_bar_and<32 * EPI_WARPS>(fast);                    // every live channel of the CTA allows 32-bit intermediates
     const bool warp_small = __any_sync(0xffffffffu, k.sh < 32) != 0;     // some channel of this warp has c < 32
+    // ... and for each of them accumulator and bias stay below 2^(c-2): the pre-shift form of requant_fast is exact
+    // and its result below 2^30 in magnitude, so that the residual term still adds without overflow
+    const int babs = k.bias < 0 ? ~k.bias : k.bias;
+    const bool warp_pre = warp_small &&
+        __all_sync(0xffffffffu, k.sh >= 32 || (k.sh - 2 >= p.acc_bits && k.sh >= 3 && babs < (1 << (k.sh - 2)))) != 0;
     if (fast) {
       k.sh1 = k.sh < 32 ? k.sh : 32;
       k.cmin31 = k.sh < 31 ? k.sh : 31;
       k.sh -= k.sh1;
+      k.pre = 32 - k.sh1;                        // (r0 is shifted by the loops that use the pre-shift form)
       if (p.res) {
         if (k.rsh >= 40) { k.rb = 0; k.rh = 0; k.rsh = 1; }            // |r*rb| < 2^39: rounds to 0
         else { k.rh = 1 << (k.rsh - 9); k.rsh -= 8; }
@@ -1350,13 +1367,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           if (p.out_signed) epilogue_loop_frag<true, false, false, true, false>(e); else epilogue_loop_frag<true, false, false, false, false>(e);
         } else if (warp_small) {
           // (no narrow residual pairs here: the plain multiply-high form of the residual term)
+#define HQ_FRAG_SMALL(RS, S, OS) do { if (warp_pre) epilogue_loop_frag<false, RS, S, OS, false, 2>(e); else epilogue_loop_frag<false, RS, S, OS, false, 1>(e); } while (0)
           if (p.sat_pack) {
-            if (p.out_signed) { if (p.res_signed) epilogue_loop_frag<false, true, true, true, false, true>(e); else epilogue_loop_frag<false, false, true, true, false, true>(e); }
-            else { if (p.res_signed) epilogue_loop_frag<false, true, true, false, false, true>(e); else epilogue_loop_frag<false, false, true, false, false, true>(e); }
+            if (p.out_signed) { if (p.res_signed) HQ_FRAG_SMALL(true, true, true); else HQ_FRAG_SMALL(false, true, true); }
+            else { if (p.res_signed) HQ_FRAG_SMALL(true, true, false); else HQ_FRAG_SMALL(false, true, false); }
           } else {
-            if (p.out_signed) { if (p.res_signed) epilogue_loop_frag<false, true, false, true, false, true>(e); else epilogue_loop_frag<false, false, false, true, false, true>(e); }
-            else { if (p.res_signed) epilogue_loop_frag<false, true, false, false, false, true>(e); else epilogue_loop_frag<false, false, false, false, false, true>(e); }
+            if (p.out_signed) { if (p.res_signed) HQ_FRAG_SMALL(true, false, true); else HQ_FRAG_SMALL(false, false, true); }
+            else { if (p.res_signed) HQ_FRAG_SMALL(true, false, false); else HQ_FRAG_SMALL(false, false, false); }
           }
+#undef HQ_FRAG_SMALL
         } else if (p.sat_pack) {
           if (p.out_signed) { if (rn) epilogue_loop_frag<false, false, true, true, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, true, false>(e); else epilogue_loop_frag<false, false, true, true, false>(e); }
           else { if (rn) epilogue_loop_frag<false, false, true, false, true>(e); else if (p.res_signed) epilogue_loop_frag<false, true, true, false, false>(e); else epilogue_loop_frag<false, false, true, false, false>(e); }
@@ -1369,15 +1388,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       // the 64-pixel tile has one 64-column slice per lane quarter: this warp only took part in the vote above
     } else if (fast && p.staged_out && p.out_bits == 4 && !p.res && !p.strip && lo >= 0 && hi <= 15) {
       // unsigned 4-bit outputs without a residual (the convs inside a 4-bit block)
-      if (warp_small) epilogue_loop_fast8<false, false, false, false, true, false, true>(e, k);
-      else epilogue_loop_fast8<false, false, false, false, false, false, true>(e, k);
+      if (warp_pre) epilogue_loop_fast8<false, false, false, false, 2, false, true>(e, k);
+      else if (warp_small) epilogue_loop_fast8<false, false, false, false, 1, false, true>(e, k);
+      else epilogue_loop_fast8<false, false, false, false, 0, false, true>(e, k);
     } else if (fast && p.staged_out && p.out_bits == 8 && (!p.res || p.staged_res)) {
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
 #define HQ_FAST8(R, RS, S, OS) do { if (RTM) { \
-                                    } else if (warp_small) epilogue_loop_fast8<R, RS, S, OS, true, false>(e, k); \
-                                    else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, false, R>(e, k); \
-                                    else epilogue_loop_fast8<R, RS, S, OS, false, false>(e, k); } while (0)
+                                    } else if (warp_pre) epilogue_loop_fast8<R, RS, S, OS, 2, false>(e, k); \
+                                    else if (warp_small) epilogue_loop_fast8<R, RS, S, OS, 1, false>(e, k); \
+                                    else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, 0, R>(e, k); \
+                                    else epilogue_loop_fast8<R, RS, S, OS, 0, false>(e, k); } while (0)
         case 0: HQ_FAST8(false, false, false, false); break;
         case 1: if (p.out_signed) HQ_FAST8(false, false, true, true); else HQ_FAST8(false, false, true, false); break;
         case 4: HQ_FAST8(true, false, false, false); break;
@@ -1723,6 +1744,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     }
   }
   p.acc_stride = p.rtm ? 2 * p.pt : p.pt;
+  { const long long bound = k_total * 255 * 128; int bits = 0; while ((1LL << bits) <= bound) ++bits; p.acc_bits = bits; }
   p.tmem_cols = (uint32_t)(p.acc_stride << p.lg_bufs);  // 512 columns, or 256 for the smallest tile
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2 && !p.strip) return HQ_ERR_UNSUPPORTED;

@@ -251,6 +251,27 @@ def test_conv_tensor_core_signed_input_and_small_c(hq):
     run_conv_and_compare(hq, case, path=2)
 
 
+@pytest.mark.parametrize("residual,big", [(False, False), (True, False), (True, True), (False, True)])
+def test_conv_small_shifts_pre_shift_form_and_its_bounds(hq, residual, big):
+    """Shifts below 32 (common with 4-bit operands): where accumulator and bias are known to stay below 2^(c-2) the
+    epilogue shifts the accumulator left first and uses the plain form; elsewhere the exact funnel-shift form.  K = 64
+    bounds |acc| by 64 * 255 * 128 < 2^21, so c >= 23 qualifies; activations and weights at their extremes, biases
+    just inside the bound for channels 0-127 and just outside it for channels 128-255 (whole warps fall back).
+    The large case reaches the 256-pixel tiles and, with a residual, the fragment epilogue."""
+    n, hw = (40, 56) if big else (2, 12)
+    case = inputs.conv_case(312, n, hw, hw, 64, 256, 1, 1, 0, residual=residual, c_range=(23, 35))
+    case["x"][0, :2] = 255
+    case["x"][-1, -1] = 0
+    case["wgt"][0:32] = 127
+    case["wgt"][32:64] = -128
+    case["wgt"][128:160] = 127
+    sign = np.where(np.arange(256) % 2 == 0, 1, -1)
+    edge = (1 << (np.minimum(case["c"].astype(np.int64), 31) - 2))
+    bias = np.where(np.arange(256) < 128, edge - 1, edge + 5) * sign
+    case["bias"] = bias.astype(np.int32)
+    run_conv_and_compare(hq, case, 2)
+
+
 def test_conv_tensor_core_general_tiles_with_residual(hq):
     # residual shifts below 9 and main shifts below 32 force the 64-bit tile path, staged and direct
     for cout in (64, 40):
