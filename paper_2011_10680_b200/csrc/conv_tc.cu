@@ -1345,7 +1345,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     // narrow residual pairs, when the caller prepared them and every channel of this warp has one
     bool warp_narrow = false;
-    if (fast && !warp_small && p.res && p.res_narrow) {
+    if (fast && (!warp_small || warp_pre) && p.res && p.res_narrow) {
       if (p.narrow_fresh) asm volatile("griddepcontrol.wait;" ::: "memory");
       const int4 nr = ch_live ? p.res_narrow[ch] : make_int4(0, 0, 0, 1);
       warp_narrow = __all_sync(0xffffffffu, nr.w != 0) != 0;
@@ -1366,8 +1366,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (!fast) {
           if (p.out_signed) epilogue_loop_frag<true, false, false, true, false>(e); else epilogue_loop_frag<true, false, false, false, false>(e);
         } else if (warp_small) {
-          // (no narrow residual pairs here: the plain multiply-high form of the residual term)
-#define HQ_FRAG_SMALL(RS, S, OS) do { if (warp_pre) epilogue_loop_frag<false, RS, S, OS, false, 2>(e); else epilogue_loop_frag<false, RS, S, OS, false, 1>(e); } while (0)
+          // (narrow residual pairs only with the pre-shift form; the funnel-shift form keeps the plain multiply-high term)
+#define HQ_FRAG_SMALL(RS, S, OS) do { if (warp_pre && rn) epilogue_loop_frag<false, false, S, OS, true, 2>(e); \
+                                      else if (warp_pre) epilogue_loop_frag<false, RS, S, OS, false, 2>(e); \
+                                      else epilogue_loop_frag<false, RS, S, OS, false, 1>(e); } while (0)
           if (p.sat_pack) {
             if (p.out_signed) { if (p.res_signed) HQ_FRAG_SMALL(true, true, true); else HQ_FRAG_SMALL(false, true, true); }
             else { if (p.res_signed) HQ_FRAG_SMALL(true, true, false); else HQ_FRAG_SMALL(false, true, false); }
@@ -1395,7 +1397,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const int variant = (p.res ? 4 : 0) | ((p.res && p.res_signed) ? 2 : 0) | (p.sat_pack ? 1 : 0);
       switch (variant) {
 #define HQ_FAST8(R, RS, S, OS) do { if (RTM) { \
-                                    } else if (warp_pre) epilogue_loop_fast8<R, RS, S, OS, 2, false>(e, k); \
+                                    } else if (warp_pre && R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, 2, R>(e, k); \
+                                    else if (warp_pre) epilogue_loop_fast8<R, RS, S, OS, 2, false>(e, k); \
                                     else if (warp_small) epilogue_loop_fast8<R, RS, S, OS, 1, false>(e, k); \
                                     else if (R && warp_narrow) epilogue_loop_fast8<R, RS, S, OS, 0, R>(e, k); \
                                     else epilogue_loop_fast8<R, RS, S, OS, 0, false>(e, k); } while (0)
