@@ -46,10 +46,14 @@ namespace {
 
 constexpr int kTileC = 128;                   // output channels per tile = MMA M = TMEM lanes
 constexpr int kMaxStages = 8;
+// Dynamic shared memory of a one-CTA-per-SM launch: 224 KiB for the pipeline's pieces + 1 KiB of alignment slack, inside
+// the 226 KiB the kernels ask for (227 KiB per block is the limit, the control block is static).
+constexpr int kSmemBudget = 224 * 1024;
+constexpr int kSmemAttr = 226 * 1024;
 constexpr int kMaxAccBufs = 4;                                 // accumulator buffers: 4 x 128 or 2 x 256 columns
 constexpr int kMaxResBufs = 8;                                 // residual / output tiles in shared memory
 // Four launch shapes of the same kernel:
-//   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 212 KiB of shared memory;
+//   solo  8 epilogue warps, one CTA per SM, up to 512 tensor-memory columns, up to 224 KiB of shared memory;
 //   pair  4 epilogue warps, two CTAs per SM with 256 columns and at most 110 KiB each.  Layers with a short
 //         reduction are bound by the latency of the hand-over chain between the MMA issuer and the epilogue
 //         (barrier, fences, MMA, commit), not by any throughput; two independent CTAs hide each other's chain.
@@ -1534,12 +1538,12 @@ int pick_pt(long long pixels, int c_tiles, int sm_count, int cap) {
 bool hq_conv_tc_init() {
   if (!load_driver_entry_points()) return false;
   return cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, kSoloIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              214 * 1024) == cudaSuccess &&
+                              kSmemAttr) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kPairEpilogueWarps, 2, kPairIssuerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               112 * 1024) == cudaSuccess &&
-         cudaFuncSetAttribute(conv_tc_kernel<8, 1, 1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 214 * 1024) == cudaSuccess &&
+         cudaFuncSetAttribute(conv_tc_kernel<8, 1, 1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemAttr) == cudaSuccess &&
          cudaFuncSetAttribute(conv_tc_kernel<kSoloEpilogueWarps, 1, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              214 * 1024) == cudaSuccess;
+                              kSmemAttr) == cudaSuccess;
 }
 
 bool hq_conv_tc_supported(const ConvArgs& a) {
@@ -1617,7 +1621,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     p.bkb = (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;
     p.cchunks = a.cin / p.bkb;
     p.k_blocks = a.kh * a.kw * p.cchunks;
-    const int smem_budget = 212 * 1024;                // dynamic bytes after the 1024-byte alignment slack
+    const int smem_budget = kSmemBudget;                // dynamic bytes after the 1024-byte alignment slack
     // staging: 8 warps x pt/2 pixel rows x 32 bytes (reserved at the 8-bit size), residual 2 or 4 x [pt][128]
     bool chosen = false;
     for (int cap = 256; cap >= 64 && !chosen; cap >>= 1) {   // largest pixel tile that leaves room for >= 3 stages
@@ -1668,7 +1672,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
       const size_t patch = (size_t)(rows + 3) * (1u << lg_wp) * bkb, wb = (size_t)kTileC * bkb;
       const size_t slab = (size_t)9 * cchunks * wb;
       const bool keep_w = slab <= 72 * 1024;
-      const size_t room = (size_t)212 * 1024 - 32 * 1024 - (keep_w ? slab : 0);
+      const size_t room = (size_t)kSmemBudget - 32 * 1024 - (keep_w ? slab : 0);
       int npatch = 0, wstages = 0;
       if (keep_w) { npatch = (int)(room / patch); if (npatch > 3) npatch = 3; }
       else if (room >= 2 * patch + 3 * wb) { npatch = 2; wstages = (int)((room - 2 * patch) / wb); }
@@ -1725,7 +1729,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
       // four residual / output tiles when they leave room for three operand stages: a tile is held from its load to
       // the end of its store, and the loads of the next tiles must be in flight meanwhile to cover the memory latency
       for (p.lg_rbufs = 2; ; --p.lg_rbufs) {
-        stages = (212 * 1024 - (res_tile_bytes << p.lg_rbufs) - wres_bytes - 16 * 1024) / stage_bytes;
+        stages = (kSmemBudget - (res_tile_bytes << p.lg_rbufs) - wres_bytes - 16 * 1024) / stage_bytes;
         if (stages >= 3 || p.lg_rbufs == 1) break;
       }
     }
@@ -1736,13 +1740,16 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
              k_total >= 2048 && (long long)p.p_tiles * p.c_tiles >= 2LL * h->sm_count) ? 1 : 0;
     if (p.duo) {
       stage_bytes = (kTileC + p.pt / 2) * p.bkb;
-      stages = (212 * 1024 - out_tile_bytes - (res_tile_bytes << p.lg_rbufs)) / stage_bytes;
+      stages = (kSmemBudget - out_tile_bytes - (res_tile_bytes << p.lg_rbufs)) / stage_bytes;
     }
     const int issuers = pair ? kPairIssuerWarps : wide ? 1 : (p.strip || p.wres) ? kSoloIssuerWarps : 1;
     p.ni = p.k_blocks < issuers ? p.k_blocks : issuers;
     if (!(p.strip && p.wres)) {
       while (p.ni > 1 && stages < p.ni) --p.ni;
       if (stages > kMaxStages) stages = kMaxStages;
+      // every stage counts more than the third issuer: the bytes in flight set the tile rate of the layers that wait
+      // on memory latency (first layer: three 32 KiB stages 163 us, four with two issuers 143 us)
+      while (p.ni > 1 && stages % p.ni) --p.ni;
       stages -= stages % p.ni;
     }
   }
