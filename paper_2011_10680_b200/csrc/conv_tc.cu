@@ -82,7 +82,6 @@ struct TcParams {
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
   int32_t halves;        // 2: two warps share a lane quarter's pixel columns; 1 for the 64-pixel tile (warps 6-9 idle)
   int32_t lg_rbufs;      // log2 of the residual-tile buffer count (<= lg_bufs; 0 when a long reduction leaves no room)
-  int32_t inplace;       // 1: the sixteen-warp shape: outputs overwrite the residual tile, which is stored as the box
   int32_t rtm;           // 1: the 8-bit residual tile reaches the epilogue through tensor memory: an MMA with the identity
                          //    matrix as its A operand turns the [pixels][128 channels] byte tile into INT32 columns beside
                          //    the accumulator, in the accumulator's own layout (see epilogue_loop_frag)
@@ -756,8 +755,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
   const int lane = e.lane, q = e.q, cq = e.cq, ew = e.ew, col0 = e.col0, px_per_warp = e.px_per_warp, ch = e.ch;
   const int c_tile = e.c_tile, p_tile0 = e.p_tile0, p_step = e.p_step, lo = e.lo, hi = e.hi;
   const bool ch_live = e.ch_live, warp_live = e.warp_live;
-  // the in-place launch shape has no staging box: this loop then stores straight to global memory
-  const bool staged_out = p.staged_out && !p.inplace;
+  const bool staged_out = p.staged_out != 0;
     // staging box of this warp: [px_per_warp pixels][32 channels] bytes (16 bytes per pixel at 4 bit)
     const int row_b = (p.out_bits == 4) ? 16 : 32;
     const uint32_t my_stage = out_stage + (uint32_t)ew * (uint32_t)(px_per_warp * 32);   // px_per_warp rows x 32 bytes reserved per warp
@@ -883,10 +881,9 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       tc_fence_before();
       if (staged_out) fence_async_smem();        // make this lane's box writes visible to the TMA engine
       __syncwarp();
-      if (p.inplace) asm volatile("bar.sync %0, 128;" :: "r"(2 + e.half) : "memory");   // one arrival per four warps there
       if (lane == 0) {
         release_accumulator(p, ctl, as);
-        if (p.staged_res && (!p.inplace || q == 0)) mbar_arrive(smem_u32(&ctl.rempty[rs]));
+        if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
         if (staged_out && warp_live)
           store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_tile, col0, px_per_warp);
       }
@@ -935,7 +932,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     for (int s = 0; s < (1 << p.lg_rbufs); ++s) {
       mbar_init(smem_u32(&ctl.rfull[s]), 1);
-      mbar_init(smem_u32(&ctl.rempty[s]), RTM ? 1 : p.inplace ? p.halves : 4 * p.halves);
+      mbar_init(smem_u32(&ctl.rempty[s]), RTM ? 1 : 4 * p.halves);
       mbar_init(smem_u32(&ctl.ofull[s]), EPI_WARPS);
     }
     mbar_init(smem_u32(&ctl.drain), p.ni);
@@ -1641,7 +1638,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
         res_tile_bytes = p.staged_res ? p.pt * kTileC : 0;
         // residual tiles: as many buffers as accumulators, fewer when a long reduction needs the room for stages
         // (its epilogue has slack: a single residual buffer only delays the next tile's prefetch)
-        // The sixteen-warp shape (below) works in place in the residual tiles and needs no staging box; with the
+        // The rtm shape (below) works in place in the residual tiles and needs no staging box; with the
         // weights resident two stages are enough for its short reductions (the epilogue bounds the tile).
         const bool wide_here = p.pt == 256 && !p.fold && p.staged_out && a.out_bits == 8 && p.staged_res && k_total < 1024;
         if (wide_here) out_tile_bytes = 0;
@@ -1717,7 +1714,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
     if (wide) {
       // 128-pixel tiles, two buffers of (accumulator + transposed residual) = 512 tensor-memory columns; the two
       // residual tiles double as the output boxes; the identity matrix takes 16 KiB
-      p.rtm = 1; p.inplace = 1; p.halves = 2;
+      p.rtm = 1; p.halves = 2;
       p.pt = 128; p.lg_bufs = 1; p.lg_rbufs = 1;
       p.p_tiles = (int32_t)((P + p.pt - 1) / p.pt);
       out_tile_bytes = 0;
@@ -1825,7 +1822,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return HQ_ERR_CUDA;
   } else
-  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, p.inplace ? kTileC : a.out_bits == 4 ? 16 : 32, p.rtm ? p.pt : p.pt / (p.halves << p.fold),
+  if (p.staged_out && !encode_rows_map(&map_out, a.out, P, out_row_bytes, p.rtm ? kTileC : a.out_bits == 4 ? 16 : 32, p.rtm ? p.pt : p.pt / (p.halves << p.fold),
                                        box_swz)) return HQ_ERR_CUDA;
   if (p.staged_res && !encode_rows_map(&map_res, a.res, P, a.cout, kTileC, p.pt, box_swz))
     return HQ_ERR_CUDA;
