@@ -58,6 +58,93 @@ def test_automatic_path_falls_back_when_the_tensor_core_launcher_declines(hq, sh
     run_conv_and_compare(hq, case, 0)
 
 
+def _random_conv_configs(count, seed):
+    """Seeded random single-layer configurations over everything the dispatch looks at: channel counts the direct
+    kernel takes or not, filter sizes, strides, padding, operand and output widths, residual kinds, signs, shift
+    ranges on both sides of 32."""
+    g = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        bits = int(g.choice([8, 8, 4]))
+        cin = int(g.choice([3, 8, 16, 32, 48, 64, 96, 128]))
+        if bits == 4 and cin % 2:
+            continue
+        cout = int(g.choice([8, 16, 24, 64, 100, 128, 192]))
+        k = int(g.choice([1, 1, 3, 3, 5]))
+        stride = int(g.choice([1, 1, 2]))
+        pad = int(g.choice([0, k // 2]))
+        h, w = int(g.integers(5, 21)), int(g.integers(5, 21))
+        if h + 2 * pad < k or w + 2 * pad < k:
+            continue
+        out_bits = int(g.choice([8, 8, 4, 32]))
+        if out_bits == 4 and cout % 2:
+            continue
+        res = None if out_bits == 32 else g.choice([None, None, 8, 32])
+        lo = int(g.integers(24, 41))
+        out.append(dict(n=int(g.integers(1, 4)), h=h, w=w, cin=cin, cout=cout, k=k, stride=stride, pad=pad, bits=bits,
+                        out_bits=out_bits, residual=res is not None, res_bits=int(res) if res is not None else 8,
+                        relu=bool(g.integers(0, 2)), in_signed=bool(g.integers(0, 2)), c_range=(lo, lo + int(g.integers(0, 9)))))
+    return out
+
+
+@pytest.mark.parametrize("path", [0, 3])
+def test_conv_random_configurations(hq, path):
+    """48 seeded random layers through hq_conv2d on the automatic path and with the tensor-core launch shapes chosen by
+    what a layer allows rather than by its size: every dispatch branch (direct, lowered, widened, first-layer form,
+    CUDA cores) must return the oracle's integers."""
+    from paper_2011_10680_b200 import binding
+    for i, cfg in enumerate(_random_conv_configs(48, 20260 + path)):
+        case = inputs.conv_case(7000 + i, cfg["n"], cfg["h"], cfg["w"], cfg["cin"], cfg["cout"], cfg["k"], cfg["stride"],
+                                cfg["pad"], bits=cfg["bits"], out_bits=cfg["out_bits"], residual=cfg["residual"],
+                                res_bits=cfg["res_bits"], relu=cfg["relu"], in_signed=cfg["in_signed"], c_range=cfg["c_range"])
+        hq.set_conv_path(path)
+        try:
+            st, out = hq.conv_case(case)
+            if path == 3 and st == binding.HQ_ERR_UNSUPPORTED:
+                continue                                   # tensor cores demanded for a shape they do not take
+            assert st == binding.HQ_OK, (cfg, binding.status_string(st))
+            hq.sync()
+        finally:
+            hq.set_conv_path(0)
+        ref = oracle().conv_case(case)
+        got = host(out, ref)
+        assert np.array_equal(got, ref), (i, cfg, int((got != ref).sum()))
+
+
+def test_conv_random_midsize_layers_reach_every_launch_shape(hq):
+    """16 seeded random layers of 20-60 thousand output pixels with the channel counts of ResNet stages: large enough for
+    im2col maps, 256-pixel tiles, resident weights, the strip form, the fragment epilogue and the two-CTA shape, small
+    enough for the oracle; shift ranges on both sides of 32, with and without an 8-bit residual, 8- and 4-bit operands."""
+    from paper_2011_10680_b200 import binding
+    g = np.random.default_rng(20261)
+    for i in range(16):
+        hw = int(g.choice([14, 28, 56]))
+        n = max(1, int(g.integers(20000, 60000)) // (hw * hw))
+        cin, cout = int(g.choice([64, 128, 256, 512])), int(g.choice([64, 128, 256, 512]))
+        k = int(g.choice([1, 1, 3]))
+        if k == 3 and cin * cout > 256 * 256:
+            cin = 128
+        bits = int(g.choice([8, 8, 4]))
+        lo = int(g.integers(26, 41))
+        residual = bool(g.integers(0, 2))
+        case = inputs.conv_case(7100 + i, n, hw, hw, cin, cout, k, 1, k // 2, bits=bits, residual=residual,
+                                in_signed=bool(g.integers(0, 2)), c_range=(lo, lo + 6))
+        for path in (0, 3):
+            hq.set_conv_path(path)
+            try:
+                st, out = hq.conv_case(case)
+                assert st == binding.HQ_OK, (i, path, binding.status_string(st))
+                hq.sync()
+            finally:
+                hq.set_conv_path(0)
+            if path == 0:
+                ref = oracle().conv_case(case)
+            got = host(out, ref)
+            assert np.array_equal(got, ref), (i, path, hw, n, cin, cout, k, bits, residual, int((got != ref).sum()))
+            del out
+        binding.check_guards()
+
+
 # ------------------------------------------------------------------ CUDA-core conv path --------
 CORE_CASES = [
     # n, h, w, cin, cout, k, stride, pad, bits, out_bits, residual, res_bits, relu
