@@ -395,7 +395,12 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
           } else if (hq_conv_s2d_applies(a)) {
             const size_t need = hq_conv_s2d_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;
-            net->launches += 2;                 // weight re-layout + space-to-depth kernels
+            net->launches += 1;                 // the space-to-depth kernel (the weights are re-laid out once, here)
+            a.wgt = d.w; a.bias = d.bias; a.b = d.requant.b; a.c = d.requant.c;
+            void* wbuf = net_alloc(net, hq_conv_s2d_prepared_bytes(a), i);
+            if (!wbuf) { st = HQ_ERR_WORKSPACE; break; }
+            net->wgt_widened[i] = wbuf;
+            if (hq_prepare_conv_s2d(a, wbuf, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
           } else if ((!hq_conv_tc_supported(a) || hq_conv_tc_small_im2col(a)) && hq_conv_lowering_applies(a)) {
             const size_t need = hq_conv_lowering_bytes(a);
             if (need > net->scratch_bytes) net->scratch_bytes = need;

@@ -62,7 +62,8 @@ struct ConvArgs {
   // internal (zero for calls that come straight from the ABI):
   const void* res_narrow;    // per-channel narrow residual pairs prepared by hq_launch_residual_narrow, or NULL
   int32_t res_narrow_fresh;  // nonzero: the pairs come from the launch just before on the same stream (the kernel waits for it)
-  const void* wgt_widened;   // 4-bit weights already widened to one byte per value (a network does it once), or NULL
+  const void* wgt_widened;   // weights as the lowered form wants them, prepared once by a network, or NULL: 4-bit weights widened
+                             // to one byte per value; for the first-layer form the virtual-channel weights and constants
   int32_t pad_after_delta;   // padding after the last row/column minus `pad`
   // byte pitches of the activation tensor along W, H and N when it is not dense (0: dense NHWC).  A W pitch
   // below cin bytes makes neighbouring "pixels" overlap: a pixel is then a window of adjacent stored pixels.
@@ -102,6 +103,8 @@ hq_status hq_launch_conv_lowered(hq_handle* h, const ConvArgs& a, void* scratch,
 bool hq_conv_s2d_applies(const ConvArgs& a);
 size_t hq_conv_s2d_bytes(const ConvArgs& a);
 hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s);
+size_t hq_conv_s2d_prepared_bytes(const ConvArgs& a);
+cudaError_t hq_prepare_conv_s2d(const ConvArgs& a, void* buf, cudaStream_t s);
 // 4-bit operands: widen to bytes in scratch, then the tensor-core kernel.
 bool hq_conv_widen4_applies(const ConvArgs& a);
 size_t hq_conv_widen4_bytes(const ConvArgs& a);

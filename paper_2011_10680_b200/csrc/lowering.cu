@@ -177,27 +177,36 @@ namespace {
 
 __global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned char* __restrict__ in, int n, int h, int w,
                                                              uint4* __restrict__ out) {
-  // output: [n][h/2 + 3][w/2 + 3] pixels of 16 bytes, the image surrounded by its zero padding (2 before, 1 after)
-  const int h2 = h >> 1, w2 = w >> 1, hp = h2 + 3, wp = w2 + 3;
-  const long long total = (long long)n * hp * wp;
+  // output: [n][h/2 + 3][w/2 + 3] pixels of 16 bytes, the image surrounded by its zero padding (2 before, 1 after).
+  // A thread builds two neighbouring output pixels x0 = 2p - 2, x0 + 1: their 2 x 12 source bytes are three aligned
+  // words in each of the two image rows (w % 4 == 0 and a 16-byte aligned image make (2 x0) * 3 a multiple of 4).
+  const int h2 = h >> 1, w2 = w >> 1, hp = h2 + 3, wp = w2 + 3, pairs = (wp + 1) >> 1;
+  const long long total = (long long)n * hp * pairs;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    const int x = (int)(i % wp) - 2;
-    long long t = i / wp;
+    const int pr = (int)(i % pairs);
+    long long t = i / pairs;
     const int y = (int)(t % hp) - 2;
     const int img = (int)(t / hp);
-    unsigned word[4] = {0u, 0u, 0u, 0u};
-    if (x >= 0 && x < w2 && y >= 0 && y < h2) {
+    const int x0 = 2 * pr - 2;
+    unsigned a[4] = {0u, 0u, 0u, 0u}, b[4] = {0u, 0u, 0u, 0u};          // pixels x0 and x0 + 1
+    if (y >= 0 && y < h2 && x0 >= 0 && x0 < w2) {                       // w2 is even: x0 + 1 is inside with x0
 #pragma unroll
       for (int dy = 0; dy < 2; ++dy) {
-        const unsigned char* src = in + (((long long)img * h + 2 * y + dy) * w + 2 * x) * 3;   // 6 contiguous bytes
-#pragma unroll
-        for (int b = 0; b < 6; ++b) {
-          const int k = dy * 6 + b;
-          word[k >> 2] |= (unsigned)__ldg(src + b) << (8 * (k & 3));
+        const unsigned* src = (const unsigned*)(in + (((long long)img * h + 2 * y + dy) * w + 2 * x0) * 3);
+        const unsigned s0 = __ldg(src), s1 = __ldg(src + 1), s2 = __ldg(src + 2);   // 12 bytes: 6 of pixel x0, 6 of x0 + 1
+        // byte k = dy * 6 + j of a 16-byte output pixel
+        const unsigned long long pa = (unsigned long long)s0 | ((unsigned long long)(s1 & 0xFFFFu) << 32);       // 6 bytes
+        const unsigned long long pb = (unsigned long long)(s1 >> 16) | ((unsigned long long)s2 << 16);           // 6 bytes
+        if (dy == 0) { a[0] = (unsigned)pa; a[1] = (unsigned)(pa >> 32); b[0] = (unsigned)pb; b[1] = (unsigned)(pb >> 32); }
+        else {
+          a[1] |= (unsigned)(pa << 16); a[2] = (unsigned)(pa >> 16);
+          b[1] |= (unsigned)(pb << 16); b[2] = (unsigned)(pb >> 16);
         }
       }
     }
-    out[i] = make_uint4(word[0], word[1], word[2], word[3]);
+    uint4* dst = out + ((long long)img * hp + (y + 2)) * wp + (x0 + 2);
+    dst[0] = make_uint4(a[0], a[1], a[2], a[3]);
+    if (x0 + 3 < wp) dst[1] = make_uint4(b[0], b[1], b[2], b[3]);
   }
 }
 
@@ -243,8 +252,11 @@ ConvArgs s2d_conv_args(const ConvArgs& a, const void* scratch) {
   const S2dLayout l = s2d_layout(a);
   const int h2 = a.h / 2, w2 = a.w / 2, hp = h2 + 3, wp = w2 + 3;
   const unsigned char* base = (const unsigned char*)scratch;
-  const int32_t* consts = (const int32_t*)(base + l.consts_off);
-  t.in = base; t.wgt = base + l.wts_off;
+  // weights and constants of the virtual channels: prepared once by the caller (a network), else in the scratch block
+  const unsigned char* prep = a.wgt_widened ? (const unsigned char*)a.wgt_widened : base + l.wts_off;
+  const int32_t* consts = (const int32_t*)(prep + (l.consts_off - l.wts_off));
+  t.wgt_widened = nullptr;
+  t.in = base; t.wgt = prep;
   t.h = hp; t.w = w2 / 2; t.cin = 128; t.kh = 4; t.kw = 1; t.stride = 1; t.pad = 0; t.pad_after_delta = 0;
   t.pitch_w = 32; t.pitch_h = (long long)wp * 16; t.pitch_n = (long long)hp * wp * 16;
   t.cout = 2 * a.cout; t.wo = a.wo / 2;
@@ -263,15 +275,23 @@ bool hq_conv_s2d_applies(const ConvArgs& a) {
 
 size_t hq_conv_s2d_bytes(const ConvArgs& a) { return (size_t)s2d_layout(a).total; }
 
+// The layer's weights in the form of the virtual channels, with their constants: a network prepares them once when it
+// is built and hands the block over as ConvArgs::wgt_widened; `buf` holds hq_conv_s2d_prepared_bytes(a) bytes.
+size_t hq_conv_s2d_prepared_bytes(const ConvArgs& a) { const S2dLayout l = s2d_layout(a); return (size_t)(l.total - l.wts_off); }
+cudaError_t hq_prepare_conv_s2d(const ConvArgs& a, void* buf, cudaStream_t s) {
+  const S2dLayout l = s2d_layout(a);
+  s2d_weights_kernel<<<(2 * a.cout * 512 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, (signed char*)buf, a.bias, a.b, a.c,
+                                                                   (int32_t*)((unsigned char*)buf + (l.consts_off - l.wts_off)));
+  return cudaGetLastError();
+}
+
 // `scratch` must hold hq_conv_s2d_bytes(a) bytes, 256-byte aligned.
 hq_status hq_launch_conv_s2d(hq_handle* h, const ConvArgs& a, void* scratch, cudaStream_t s) {
   if (a.n == 0) return HQ_OK;
   const S2dLayout l = s2d_layout(a);
   unsigned char* base = (unsigned char*)scratch;
-  s2d_weights_kernel<<<(2 * a.cout * 512 + 255) / 256, 256, 0, s>>>((const signed char*)a.wgt, a.cout, (signed char*)(base + l.wts_off),
-                                                                   a.bias, a.b, a.c, (int32_t*)(base + l.consts_off));
-  if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
-  const long long px = l.img_bytes / 16;
+  if (!a.wgt_widened && hq_prepare_conv_s2d(a, base + l.wts_off, s) != cudaSuccess) return HQ_ERR_CUDA;
+  const long long px = l.img_bytes / 16 / 2;          // a thread builds two pixels
   long long blocks = (px + 255) / 256;
   const long long cap = (long long)h->sm_count * 32;
   space_to_depth_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, s>>>((const unsigned char*)a.in, a.n, a.h, a.w, (uint4*)base);
