@@ -785,8 +785,8 @@ __global__ void __launch_bounds__(256) avgpool_vec4_sliced_kernel(const unsigned
 
 // 16 channels per thread (one 16-byte load per pixel), SLICES pixel slices per block (two for a 7x7 map, so that
 // a thread sums a dozen or more pixels and the block's closing steps weigh little), eight loads of a thread in
-// flight at a time; 512 channels per block.  Bytes are summed as 16-bit lanes (h*w*255 <= 65535, i.e. up to 257
-// pixels; signed bytes are offset by 128 and corrected at the end).  The slices meet in shared memory and every
+// flight at a time; 512 channels per block.  Bytes are summed as 16-bit lanes inside a slice (255 * pixels <= 65535, i.e. up
+// to 257 pixels per slice: maps of up to 2056 pixels with eight slices; signed bytes are offset by 128 and corrected at the end).  The slices meet in shared memory and every
 // thread then finishes its share of the block's channels, two at a time.
 template <int SLICES, bool SIGNED>
 __global__ void __launch_bounds__(32 * SLICES) avgpool_vec16_kernel(const uint4* __restrict__ in, int hw, int ch,
@@ -826,11 +826,15 @@ __global__ void __launch_bounds__(32 * SLICES) avgpool_vec16_kernel(const uint4*
     const int gl = t >> 3, word = (t & 7) >> 1, half = t & 1;
     const int ch0 = (blockIdx.x * 32 + gl) * 16 + word * 4 + half * 2;
     if (ch0 >= ch) continue;
+    // byte 2*half of the word sits in halfword `half` of the even sums, byte 2*half+1 in halfword `half` of the odd sums;
+    // a slice's halfword holds at most 257 pixels, the slices are added at full width
     unsigned even = 0, odd = 0;
 #pragma unroll
-    for (int sl = 0; sl < SLICES; ++sl) { even += part[sl][2 * word][gl]; odd += part[sl][2 * word + 1][gl]; }
-    // byte 2*half of the word sits in halfword `half` of the even sums, byte 2*half+1 in halfword `half` of the odd sums
-    const int s0 = (int)((even >> (16 * half)) & 0xFFFFu) - off, s1 = (int)((odd >> (16 * half)) & 0xFFFFu) - off;
+    for (int sl = 0; sl < SLICES; ++sl) {
+      even += (part[sl][2 * word][gl] >> (16 * half)) & 0xFFFFu;
+      odd += (part[sl][2 * word + 1][gl] >> (16 * half)) & 0xFFFFu;
+    }
+    const int s0 = (int)even - off, s1 = (int)odd - off;
     const int q0 = hq_clamp_ll(hq_dn(s0, __ldg(b + ch0), __ldg(c + ch0)), 0, qmin, qmax);
     const int q1 = hq_clamp_ll(hq_dn(s1, __ldg(b + ch0 + 1), __ldg(c + ch0 + 1)), 0, qmin, qmax);
     out[((long long)img * ch + ch0) >> 1] = (unsigned short)((q0 & 0xFF) | ((q1 & 0xFF) << 8));
@@ -1049,7 +1053,7 @@ cudaError_t hq_launch_avgpool(const void* in, int n, int h, int w, int ch, int i
                               const int32_t* b, const int32_t* c, int qmin, int qmax,
                               void* out, int out_bits, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  if (in_bits == 8 && out_bits == 8 && ch % 16 == 0 && h * w <= 257 && n <= 65535) {
+  if (in_bits == 8 && out_bits == 8 && ch % 16 == 0 && h * w <= 8 * 257 && n <= 65535) {
     const int hw = h * w;
     if (hw >= 128) launch_avgpool_vec16<8>(in, n, hw, ch, in_signed, b, c, qmin, qmax, out, s);
     else if (hw >= 64) launch_avgpool_vec16<4>(in, n, hw, ch, in_signed, b, c, qmin, qmax, out, s);

@@ -655,10 +655,12 @@ def test_maxpool_windows_and_signedness(hq, k, stride, pad, signed):
 
 
 @pytest.mark.parametrize("n,hw,ch,signed", [(3, 16, 48, 0), (2, 7, 528, 0), (2, 16, 64, 1), (5, 7, 2048, 1), (2, 9, 20, 1),
-                                            (2, 17, 32, 0)])
+                                            (2, 17, 32, 0), (2, 17, 1664, 1), (2, 35, 288, 0), (2, 45, 48, 1), (2, 46, 32, 0)])
 def test_avgpool_requant_8bit_kernels(hq, n, hw, ch, signed):
     # the 16-channel kernel with a partly filled block, two blocks per image, 256 pixels at the maximum value
-    # (16-bit lane sums at their limit), signed bytes; the 4-channel kernel (ch = 20); more than 257 pixels
+    # (16-bit lane sums at their limit), signed bytes; the 4-channel kernel (ch = 20); more than 257 pixels: slices of the
+    # 16-channel kernel added at full width (Inception's 17x17 and 35x35 maps, 45x45 = 2025 pixels with every slice at
+    # its limit), and beyond 2056 pixels the 4-channel kernel again
     from paper_2011_10680_b200 import binding
     g = inputs.rng(305, n, hw, ch, signed)
     x = g.integers(0, 256, size=(n, hw, hw, ch), dtype=np.int64).astype(np.uint8)
