@@ -94,10 +94,12 @@ def layer_work(table, batch):
             byt = in_bytes + co * k * l["bits"] // 8 + out_bytes + 13 * co
             if l["in1"] >= 0:
                 byt += batch * ho * wo * co * hw_in[l["in1"]][3] // 8
+        elif l["op"] == "concat":
+            byt = out_bytes + sum(batch * hw_in[t][0] * hw_in[t][1] * hw_in[t][2] * hw_in[t][3] // 8 for t in l["ins"])
         else:
             byt = batch * h * w * c * b_in // 8 + out_bytes
             if l["in1"] >= 0:
-                byt += out_bytes
+                byt += batch * ho * wo * co * hw_in[l["in1"]][3] // 8
         rows.append(dict(layer=i, op=l["op"], ops=ops, bytes=byt))
     return rows
 
