@@ -113,7 +113,8 @@ __device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` =
 
 // One pixel's word of four channels.  SLOW: one of the thread's channels has a shift below 9 (64-bit form).
 // SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing);
-// 3 for a 4-bit output clamped to [0, 15]; 4 the same without a residual and with shifts reduced by four.
+// 3 for a 4-bit output clamped to [0, 15]; 4 the same without a residual and with shifts reduced by four;
+// 5 for a byte-wide output clamped to [0, 15].
 // 8-bit value i of a word, zero- or sign-extended (one byte-permute either way: selector bit 3 replicates the
 // selected byte's sign bit).
 template <bool SIGNED>
@@ -143,7 +144,14 @@ __device__ __forceinline__ void requant8_word(const EltArgs& a, const Dy8 (&m)[4
       s[i] = (int)(t < (long long)lo ? (long long)lo : (t > (long long)hi ? (long long)hi : t));
     }
   }
-  if constexpr (!OUT4 && SATP != 0) {
+  if constexpr (!OUT4 && SATP == 5) {
+    // byte-wide output clamped to [0, 15] (a 4-bit tensor kept one value per byte inside a network): upper bound by a
+    // minimum, lower bound and packing by the saturating packs
+    unsigned w23, w;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w23) : "r"(min(s[3], 15)), "r"(min(s[2], 15)), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(min(s[1], 15)), "r"(min(s[0], 15)), "r"(w23));
+    *(unsigned*)dst = w;
+  } else if constexpr (!OUT4 && SATP != 0) {
     // two saturating packs; the second carries the first one's halfword in its upper half: bytes s0 s1 s2 s3
     unsigned w23, w;
     if (SATP == 1) {
@@ -534,6 +542,7 @@ template <bool RES, bool MSIGNED, bool RSIGNED>
 cudaError_t launch_requant8(const EltArgs& a, dim3 grid, dim3 block, int words, int lo, int hi, int sm_count, cudaStream_t s) {
   if (a.out_bits == 4 && lo == 0 && hi == 15) return launch_requant8_form<RES, MSIGNED, RSIGNED, true, 3>(a, grid, block, words, lo, hi, sm_count, s);
   if (a.out_bits == 4) return launch_requant8_form<RES, MSIGNED, RSIGNED, true, 0>(a, grid, block, words, lo, hi, sm_count, s);
+  if (lo == 0 && hi == 15) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 5>(a, grid, block, words, lo, hi, sm_count, s);
   if (lo == 0 && hi == 255) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 1>(a, grid, block, words, lo, hi, sm_count, s);
   if (lo == -128 && hi == 127) return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 2>(a, grid, block, words, lo, hi, sm_count, s);
   return launch_requant8_form<RES, MSIGNED, RSIGNED, false, 0>(a, grid, block, words, lo, hi, sm_count, s);
