@@ -675,32 +675,37 @@ def main():
             hq.sync()
 
         # ---------------- end to end: pinned host images in, logits out, double-buffered ----
-        copy_stream = torch.cuda.Stream()
+        copy_stream, back_stream = torch.cuda.Stream(), torch.cuda.Stream()     # images in, logits out
         img_bufs = [torch.empty_like(images_d) for _ in range(2)]
         log_bufs = [torch.empty_like(logits_d) for _ in range(2)]
         logits_h = [torch.empty(net.logits_shape, dtype=torch.int32).pin_memory() for _ in range(2)]
         ready = [torch.cuda.Event() for _ in range(2)]
+        ran = [torch.cuda.Event() for _ in range(2)]
         done = [torch.cuda.Event() for _ in range(2)]
 
         def e2e_steps(k):
             for i in range(k):
                 j = i & 1
                 with torch.cuda.stream(copy_stream):
-                    copy_stream.wait_event(done[j])              # buffer j free again
+                    copy_stream.wait_event(done[j])              # buffer pair j free again: its logits have left
                     img_bufs[j].copy_(images_h, non_blocking=True)
                     ready[j].record(copy_stream)
                 stream.wait_event(ready[j])
                 net.run(img_bufs[j], log_bufs[j])
-                logits_h[j].copy_(log_bufs[j], non_blocking=True)
-                done[j].record(stream)
+                ran[j].record(stream)
+                with torch.cuda.stream(back_stream):             # the read-back does not hold the next step up
+                    back_stream.wait_event(ran[j])
+                    logits_h[j].copy_(log_bufs[j], non_blocking=True)
+                    done[j].record(back_stream)
 
         e2e_steps(max(args.warmup, 4))
         barrier()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
         e2e_steps(args.steps)
+        stream.wait_event(done[0]); stream.wait_event(done[1])      # the timed region ends when the last logits are on the host
         f1.record(stream)
-        copy_stream.synchronize()
+        copy_stream.synchronize(); back_stream.synchronize()
         barrier()
         ms_e2e = f0.elapsed_time(f1)
         hq.sync()
