@@ -115,12 +115,12 @@ __device__ __forceinline__ int dn8(unsigned top, const Dy8& d) {      // `top` =
 // SATP: 1 / 2 when the clamp bounds equal the range of u8 / s8 (a saturating pack does clamp and packing);
 // 3 for a 4-bit output clamped to [0, 15]; 4 the same without a residual and with shifts reduced by four;
 // 5 for a byte-wide output clamped to [0, 15].
-// 8-bit value i of a word, zero- or sign-extended (one byte-permute either way: selector bit 3 replicates the
-// selected byte's sign bit).
+// 8-bit value i of a word, zero- or sign-extended (one byte permute either way; the signed form needs the full
+// selector of hq_prmt: bit 3 of a nibble replicates the selected byte's sign bit).
 template <bool SIGNED>
 __device__ __forceinline__ int byte_of(unsigned w, int i) {
   const unsigned sx = 8u | (unsigned)i;
-  return SIGNED ? (int)__byte_perm(w, 0u, (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)i)
+  return SIGNED ? (int)hq_prmt(w, 0u, (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)i)
                 : (int)__byte_perm(w, 0u, 0x4440u | (unsigned)i);
 }
 
@@ -885,8 +885,8 @@ __global__ void avgpool_scalar_kernel(const void* in, int n, int hw, int ch, int
 template <bool SIGNED>
 struct BytePairMax {
   unsigned e, o;             // running maxima of bytes 0 / 2 and of bytes 1 / 3, one per halfword
-  __device__ __forceinline__ static unsigned even(unsigned w) { return __byte_perm(w, 0, SIGNED ? 0xA280 : 0x4240); }
-  __device__ __forceinline__ static unsigned odd(unsigned w) { return __byte_perm(w, 0, SIGNED ? 0xB391 : 0x4341); }
+  __device__ __forceinline__ static unsigned even(unsigned w) { return hq_prmt(w, 0u, SIGNED ? 0xA280u : 0x4240u); }
+  __device__ __forceinline__ static unsigned odd(unsigned w) { return hq_prmt(w, 0u, SIGNED ? 0xB391u : 0x4341u); }
   __device__ __forceinline__ void init(unsigned w) { e = even(w); o = odd(w); }
   __device__ __forceinline__ void add(unsigned w) {
     if (SIGNED) { e = __vmaxs2(e, even(w)); o = __vmaxs2(o, odd(w)); }

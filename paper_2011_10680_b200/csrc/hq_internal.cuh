@@ -35,6 +35,14 @@ __device__ __forceinline__ long long hq_dn(int q, int b, int c) {
 }
 
 // Element access for dense tensors with 4, 8 or 32 bits per element (even element = low nibble).
+// Byte permute with the full PTX selector: bit 3 of a selector nibble replicates the selected byte's sign bit over the
+// target byte.  (The __byte_perm intrinsic keeps three bits per nibble and cannot sign-extend.)
+__device__ __forceinline__ unsigned hq_prmt(unsigned a, unsigned b, unsigned sel) {
+  unsigned d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
 __device__ __forceinline__ int hq_load_elem(const void* base, long long idx, int bits, int is_signed) {
   if (bits == 32) return ((const int*)base)[idx];
   if (bits == 8) return is_signed ? (int)((const signed char*)base)[idx] : (int)((const unsigned char*)base)[idx];

@@ -566,6 +566,40 @@ LARGE_ELT_CASES = [
 ]
 
 
+@pytest.mark.parametrize("main_signed,res_signed,out_bits", [(1, 1, 8), (1, None, 8), (0, 1, 8), (1, 0, 8), (1, None, 4)])
+def test_residual_add_narrow_pairs_with_signed_operands(hq, main_signed, res_signed, out_bits):
+    """A single call on at least 2^25 values works out narrow multiply-add pairs first and then reads every byte
+    through the one-instruction extraction; signed bytes must come out sign-extended.  Negative operands on both
+    branches, every stored value compared."""
+    from paper_2011_10680_b200 import binding
+    h, w, ch = 727, 723, 64
+    assert h * w * ch >= 1 << 25
+    g = inputs.rng(307, main_signed, 2 if res_signed is None else res_signed, out_bits)
+    shape = (1, h, w, ch)
+    draw = lambda sg: (g.integers(-128, 128, size=shape, dtype=np.int64).astype(np.int8) if sg else
+                       g.integers(0, 256, size=shape, dtype=np.int64).astype(np.uint8))
+    main = draw(main_signed)
+    res = draw(res_signed) if res_signed is not None else None
+    mb, rb = (g.integers(1 << 30, 1 << 31, size=ch, dtype=np.int64).astype(np.int32) for _ in range(2))
+    mc = g.integers(31, 34, size=ch).astype(np.int32)
+    rc = g.integers(31, 34, size=ch).astype(np.int32)
+    out_signed = int(out_bits == 8)
+    qmin, qmax = (0, 15) if out_bits == 4 else (-128, 127)
+    ref = oracle().residual_add(main, 8, main_signed, mb, mc, res, 8 if res is not None else 0, res_signed or 0,
+                                rb if res is not None else None, rc if res is not None else None, ch, 0, qmin, qmax,
+                                out_bits, out_signed)
+    if out_bits == 8:
+        assert np.count_nonzero((ref > qmin) & (ref < 0)) > ref.size // 8        # negative results that are not clamped
+    out = binding.alloc_out(*shape[:3], ch, out_bits, out_signed)
+    st = hq.residual_add(binding.to_device(main), 8, main_signed, binding.to_device(mb), binding.to_device(mc),
+                         binding.to_device(res), 8 if res is not None else 0, res_signed or 0,
+                         binding.to_device(rb) if res is not None else None, binding.to_device(rc) if res is not None else None,
+                         ch, 0, qmin, qmax, out, out_bits, out_signed)
+    assert st == binding.HQ_OK
+    hq.sync()
+    assert np.array_equal(host(out, ref), ref)
+
+
 @pytest.mark.parametrize("cfg", LARGE_ELT_CASES)
 def test_residual_add_large_tensors(hq, cfg):
     """Tensors of many block trips with a ragged last trip: the flat word-array kernel (channel words a power of two),
