@@ -294,6 +294,20 @@ def run_membound(args):
     ocat17 = torch.empty((4 * n, 17, 17, 768), dtype=torch.uint8, device="cuda")
     cases.append(("concat 4x u8 -> u8 [%d,17,17,768]" % (4 * n), 2 * ocat17.numel(),
                   lambda: hq.concat_requant(cat17, 1, 0, 255, ocat17, 8, 0)))
+    # the same two calls with ONE pair per branch, DN(S_i / S_a) of per-tensor activation scales (the form Appendix E
+    # writes down; the rows above draw a pair per channel)
+    def one_pair(brs):
+        res = []
+        for br in brs:
+            b, c = br["b"], br["c"]
+            res.append({**br, "b": b[:1].repeat(br["ch"]).contiguous(), "c": c[:1].repeat(br["ch"]).contiguous()})
+        return res
+    cat_u, cat17_u = one_pair(cat), one_pair(cat17)
+    cases.append(("concat 3x u8 + s32 -> u8 [%d,35,35,288], one pair per branch" % n,
+                  sum(br["x"].numel() * br["x"].element_size() for br in cat) + ocat.numel(),
+                  lambda: hq.concat_requant(cat_u, 1, 0, 255, ocat, 8, 0)))
+    cases.append(("concat 4x u8 -> u8 [%d,17,17,768], one pair per branch" % (4 * n), 2 * ocat17.numel(),
+                  lambda: hq.concat_requant(cat17_u, 1, 0, 255, ocat17, 8, 0)))
     # the pooling branch of that module: 3x3 / stride 1 window sums over the INT32 feature map
     xp = ri(-(1 << 20), 1 << 20, (n, 35, 35, 192), torch.int32); op_ = torch.empty_like(xp)
     cases.append(("sumpool 3x3/1 s32 -> s32 [%d,35,35,192]" % n, 2 * xp.numel() * 4,

@@ -22,6 +22,7 @@ struct ConcatBranch {
   int32_t upp;        // threads (units) per pixel of this branch = ceil(ch / width)
   int32_t block0, nblocks;   // this branch's blocks of the launch
   int32_t vec;        // 1: rows and dyadic arrays allow 16-byte reads (ch % 16 == 0 resp. ch % 4 == 0, aligned arrays)
+  int32_t piece16;    // 1: an 8-bit branch whose rows, offset and output rows are whole 16-byte pieces (see concat_uniform8)
 };
 
 struct ConcatArgs {
@@ -251,6 +252,70 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
   }
 }
 
+// An 8-bit branch whose channels all share ONE dyadic pair -- the case Appendix E writes down, DN(S_i / S_a) with
+// per-tensor activation scales -- needs no thread-to-channel binding: the branch is walked as 16-byte pieces (sixteen
+// channels) dealt round-robin to all threads of the branch's blocks, four pieces in flight per thread, three
+// constants in registers, one 16-byte store per piece.  (m, a, s) is the checked narrow pair of the shared (b, c).
+template <bool SIGNED, int OUT>
+__device__ __forceinline__ void concat_uniform8(const ConcatArgs& a, const int i, const unsigned m, const unsigned add,
+                                                const int s, const int lo, const int hi) {
+  const ConcatBranch& B = a.br[i];
+  const int P = B.ch >> 4;                                        // pieces per pixel
+  const long long total = a.pixels * P;
+  const int S = B.nblocks * 256;                                  // pieces per round of the branch's threads
+  long long idx = (long long)((int)blockIdx.x - B.block0) * 256 + threadIdx.x;
+  if (idx >= total) return;
+  const int dpx = S / P, du = S % P;
+  const long long px = idx / P;
+  int u = (int)(idx - px * P);
+  const long long in_row = B.row_ch, out_row = a.out_ch;
+  const unsigned char* ip = (const unsigned char*)B.in + px * in_row + u * 16;
+  unsigned char* op = (unsigned char*)a.out + px * out_row + B.ch_off + u * 16;
+  // one round moves a thread dpx pixels and du pieces on; past the row's last piece it wraps into the next pixel
+  const long long istep = dpx * in_row + du * 16, ostep = dpx * out_row + du * 16;
+  const long long iwrap = in_row - 16 * P, owrap = out_row - 16 * P;
+  constexpr int KP = 4;
+  while (idx < total) {
+    uint4 raw[KP];
+    unsigned char* dst[KP];
+#pragma unroll
+    for (int k = 0; k < KP; ++k) {
+      dst[k] = idx < total ? op : nullptr;
+      if (idx < total) raw[k] = __ldg((const uint4*)ip);
+      idx += S; u += du;
+      const bool wrap = u >= P;
+      if (wrap) u -= P;
+      ip += istep + (wrap ? iwrap : 0ll);
+      op += ostep + (wrap ? owrap : 0ll);
+    }
+#pragma unroll
+    for (int k = 0; k < KP; ++k) {
+      if (!dst[k]) break;
+      const unsigned w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+      unsigned o[4];
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        int y[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          // byte j zero- or sign-extended by one byte permute
+          const unsigned sx = 8u | (unsigned)j;
+          const unsigned q = hq_prmt(w[v], 0u, SIGNED ? (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)j : 0x4440u | (unsigned)j);
+          const unsigned t = q * m + add;
+          y[j] = SIGNED ? (int)t >> s : (int)(t >> s);
+        }
+        if (OUT == 0) o[v] = pack4_sat(y[0], y[1], y[2], y[3], lo < 0);
+        else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) y[j] = min(max(y[j], lo), hi) & 0xFF;
+          o[v] = (unsigned)y[0] | ((unsigned)y[1] << 8) | ((unsigned)y[2] << 16) | ((unsigned)y[3] << 24);
+        }
+      }
+      *(uint4*)dst[k] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
 struct W4State {
   const unsigned char* ip; unsigned char* op;
   long long px, step, in_row, out_row, pixels;
@@ -332,10 +397,25 @@ __device__ __forceinline__ void concat_w4(const ConcatArgs& a, const int i) {
   const int is_signed = a.br[i].is_signed;
   const int upp = a.br[i].upp, ppb = 256 / upp;
   const int tid = threadIdx.x;
+  const int lo = a.relu ? max(a.qmin, 0) : a.qmin, hi = a.qmax;
+  if (BITS == 8 && a.br[i].piece16 && a.narrow != nullptr) {
+    // Do all channels of the branch share one pair with a checked narrow form?  The block's threads look at four
+    // channels each (together all of them) and vote; the branch and the flag are the same for the whole block.
+    const int kc = (tid % upp) * 4;
+    const int b0 = __ldg(a.br[i].b), c0 = __ldg(a.br[i].c);
+    bool same = true;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) same = same && __ldg(a.br[i].b + kc + j) == b0 && __ldg(a.br[i].c + kc + j) == c0;
+    const int4 n0 = __ldg(a.narrow + a.br[i].ch_off);
+    if (__syncthreads_and(same && n0.w != 0)) {
+      if (is_signed) { if (a.sat) concat_uniform8<true, 0>(a, i, n0.x, n0.y, n0.z, lo, hi); else concat_uniform8<true, 1>(a, i, n0.x, n0.y, n0.z, lo, hi); }
+      else { if (a.sat) concat_uniform8<false, 0>(a, i, n0.x, n0.y, n0.z, lo, hi); else concat_uniform8<false, 1>(a, i, n0.x, n0.y, n0.z, lo, hi); }
+      return;
+    }
+  }
   if (tid >= upp * ppb) return;
   const int u = tid % upp, y = tid / upp;
   const int k0 = u * 4, off = a.br[i].ch_off + k0;
-  const int lo = a.relu ? max(a.qmin, 0) : a.qmin, hi = a.qmax;
   int bb[4], hh[4], ss[4];
   bool fast = true;
 #pragma unroll
@@ -444,6 +524,8 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
       B.bits = t.bits; B.is_signed = t.bits == 32 ? 1 : t.is_signed; B.ch = chp; B.ch_off = off; B.row_ch = t.c;
       if (four && chp <= 4 * 256) { B.width = 4; B.vec = 1; }
       else { B.width = 16; B.vec = (t.bits != 32 && t.c % 16 == 0) ? 1 : 0; }
+      B.piece16 = (B.width == 4 && t.bits == 8 && out->bits == 8 && chp % 16 == 0 && t.c % 16 == 0 && off % 16 == 0 &&
+                   out->c % 16 == 0) ? 1 : 0;
       B.upp = (chp + B.width - 1) / B.width;
       if (B.upp > 256) return HQ_ERR_UNSUPPORTED;                 // more than 4096 channels in one branch
       weight[nb] = (long long)chp * (t.bits + out->bits);

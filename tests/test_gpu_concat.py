@@ -83,6 +83,64 @@ def test_concat_large_call_with_narrow_pairs(hq):
         run_and_compare(hq, case)
 
 
+def _uniform_branch(g, n, hw, ch, bits, signed, b, c, uniform=True):
+    """One branch whose channels all share the pair (b, c) (or, with uniform=False, all but the last channel)."""
+    if bits == 32:
+        x = g.integers(-(1 << 22), 1 << 22, size=(n, hw, hw, ch), dtype=np.int64).astype(np.int32)
+    else:
+        x = g.integers(-128 if signed else 0, 128 if signed else 256, size=(n, hw, hw, ch), dtype=np.int64)
+        x = x.astype(np.int8 if signed else np.uint8)
+    bb = np.full(ch, b, np.int32)
+    cc = np.full(ch, c, np.int32)
+    if not uniform:
+        bb[-1] = b - 12345
+    return {"x": x, "bits": bits, "signed": signed, "ch": ch, "b": bb, "c": cc}
+
+
+@pytest.mark.parametrize("layout", ["module_35", "module_17", "signed_mix", "pieces", "unaligned_offset"])
+def test_concat_branches_with_one_pair_per_branch(hq, layout):
+    """Per-tensor activation scales give ONE pair DN(S_i / S_a) per branch (Appendix E); such 8-bit branches are walked
+    in 16-byte pieces.  Cases: the two module shapes, signed operands beside unsigned ones, a branch that is uniform
+    except for its last channel (must stay on the per-channel form), a branch wider than 1024 channels entered in
+    pieces, an output offset that is not a multiple of sixteen (per-channel form), and pixel counts that leave a
+    ragged last round; each with the saturating and the explicit clamp and a signed output."""
+    g = inputs.rng(411)
+    pair = lambda lo_c, hi_c: (int(g.integers(1 << 30, 1 << 31)), int(g.integers(lo_c, hi_c)))
+    if layout == "module_35":
+        n, hw = 15, 35
+        spec = [(64, 8, 0, True), (64, 8, 0, True), (96, 8, 0, True), (64, 32, 1, True)]
+    elif layout == "module_17":
+        n, hw = 25, 17
+        spec = [(192, 8, 0, True)] * 3 + [(192, 8, 0, False)]
+    elif layout == "signed_mix":
+        n, hw = 31, 19
+        spec = [(48, 8, 1, True), (80, 8, 0, True), (16, 8, 1, True), (112, 8, 1, False), (128, 8, 0, True)]
+    elif layout == "pieces":
+        n, hw = 5, 23
+        spec = [(64, 8, 0, True), (2064, 8, 0, True), (32, 32, 1, True)]
+    else:
+        n, hw = 40, 21
+        spec = [(8, 8, 0, True), (64, 8, 0, True), (120, 8, 1, True), (64, 8, 0, True)]
+    branches = []
+    for ch, bits, signed, uniform in spec:
+        b, c = pair(44, 48) if bits == 32 else pair(29, 33)
+        branches.append(_uniform_branch(g, n, hw, ch, bits, signed, b, c, uniform))
+    out_ch = sum(s[0] for s in spec)
+    assert n * hw * hw * out_ch >= 1 << 22                          # large enough for the narrow pairs
+    for out_signed, relu, lo, hi in ((0, 1, 0, 255), (1, 0, -128, 127), (0, 0, 3, 200)):
+        case = {"branches": branches, "relu": relu, "qmin": lo, "qmax": hi, "out_bits": 8, "out_signed": out_signed,
+                "n": n, "hw": hw, "out_ch": out_ch}
+        ref = run_and_compare(hq, case)
+        inner = np.count_nonzero((ref > lo) & (ref < hi))
+        assert inner > ref.size // 8
+    # a pair whose shift has no narrow form (c = 40) and one whose term is always zero (c = 45)
+    for c in (40, 45):
+        odd = [_uniform_branch(g, n, hw, ch, bits, signed, (1 << 31) - 7, c if bits == 8 else 46, True)
+               for ch, bits, signed, _ in spec]
+        run_and_compare(hq, {"branches": odd, "relu": 1, "qmin": 0, "qmax": 255, "out_bits": 8, "out_signed": 0,
+                             "n": n, "hw": hw, "out_ch": out_ch})
+
+
 def test_concat_at_the_benchmark_size(hq):
     """The 35x35 module at batch 256, as `bench.py --membound` times it (90 M outputs): every stored value."""
     case = inputs.concat_case(406, 256, 35, [(64, 8, 0), (64, 8, 0), (96, 8, 0), (64, 32, 1)])
