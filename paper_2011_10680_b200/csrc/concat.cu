@@ -253,67 +253,58 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
 }
 
 // An 8-bit branch whose channels all share ONE dyadic pair -- the case Appendix E writes down, DN(S_i / S_a) with
-// per-tensor activation scales -- needs no thread-to-channel binding: the branch is walked as 16-byte pieces (sixteen
-// channels) dealt round-robin to all threads of the branch's blocks, four pieces in flight per thread, three
-// constants in registers, one 16-byte store per piece.  (m, a, s) is the checked narrow pair of the shared (b, c).
+// per-tensor activation scales -- needs no per-channel constants: a thread owns one 16-byte piece (sixteen channels)
+// of the pixel row, walks the pixels through running pointers with four pieces in flight, three constants in
+// registers, one 16-byte store per piece.  (m, a, s) is the checked narrow pair of the shared (b, c).
 template <bool SIGNED, int OUT>
 __device__ __forceinline__ void concat_uniform8(const ConcatArgs& a, const int i, const unsigned m, const unsigned add,
                                                 const int s, const int lo, const int hi) {
   const ConcatBranch& B = a.br[i];
-  const int P = B.ch >> 4;                                        // pieces per pixel
-  const long long total = a.pixels * P;
-  const int S = B.nblocks * 256;                                  // pieces per round of the branch's threads
-  long long idx = (long long)((int)blockIdx.x - B.block0) * 256 + threadIdx.x;
-  if (idx >= total) return;
-  const int dpx = S / P, du = S % P;
-  const long long px = idx / P;
-  int u = (int)(idx - px * P);
-  const long long in_row = B.row_ch, out_row = a.out_ch;
-  const unsigned char* ip = (const unsigned char*)B.in + px * in_row + u * 16;
-  unsigned char* op = (unsigned char*)a.out + px * out_row + B.ch_off + u * 16;
-  // one round moves a thread dpx pixels and du pieces on; past the row's last piece it wraps into the next pixel
-  const long long istep = dpx * in_row + du * 16, ostep = dpx * out_row + du * 16;
-  const long long iwrap = in_row - 16 * P, owrap = out_row - 16 * P;
-  constexpr int KP = 4;
-  while (idx < total) {
-    uint4 raw[KP];
-    unsigned char* dst[KP];
+  const int P = B.ch >> 4;                                        // pieces per pixel (at most 64)
+  const int ppb = 256 / P;                                        // pixels per block step
+  const int tid = threadIdx.x;
+  if (tid >= P * ppb) return;
+  const int u = tid % P, y = tid / P;
+  const long long step = (long long)B.nblocks * ppb;
+  long long px = (long long)((int)blockIdx.x - B.block0) * ppb + y;
+  const long long istep = step * B.row_ch, ostep = step * a.out_ch;
+  const unsigned char* ip = (const unsigned char*)B.in + px * B.row_ch + u * 16;
+  unsigned char* op = (unsigned char*)a.out + px * a.out_ch + B.ch_off + u * 16;
+  auto one = [&](const uint4 r, unsigned char* dst) {
+    const unsigned w[4] = {r.x, r.y, r.z, r.w};
+    unsigned o[4];
 #pragma unroll
-    for (int k = 0; k < KP; ++k) {
-      dst[k] = idx < total ? op : nullptr;
-      if (idx < total) raw[k] = __ldg((const uint4*)ip);
-      idx += S; u += du;
-      const bool wrap = u >= P;
-      if (wrap) u -= P;
-      ip += istep + (wrap ? iwrap : 0ll);
-      op += ostep + (wrap ? owrap : 0ll);
-    }
+    for (int v = 0; v < 4; ++v) {
+      int yv[4];
 #pragma unroll
-    for (int k = 0; k < KP; ++k) {
-      if (!dst[k]) break;
-      const unsigned w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
-      unsigned o[4];
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        int y[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          // byte j zero- or sign-extended by one byte permute
-          const unsigned sx = 8u | (unsigned)j;
-          const unsigned q = hq_prmt(w[v], 0u, SIGNED ? (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)j : 0x4440u | (unsigned)j);
-          const unsigned t = q * m + add;
-          y[j] = SIGNED ? (int)t >> s : (int)(t >> s);
-        }
-        if (OUT == 0) o[v] = pack4_sat(y[0], y[1], y[2], y[3], lo < 0);
-        else {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) y[j] = min(max(y[j], lo), hi) & 0xFF;
-          o[v] = (unsigned)y[0] | ((unsigned)y[1] << 8) | ((unsigned)y[2] << 16) | ((unsigned)y[3] << 24);
-        }
+      for (int j = 0; j < 4; ++j) {
+        // byte j zero- or sign-extended by one byte permute
+        const unsigned sx = 8u | (unsigned)j;
+        const unsigned q = hq_prmt(w[v], 0u, SIGNED ? (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)j : 0x4440u | (unsigned)j);
+        const unsigned t = q * m + add;
+        yv[j] = SIGNED ? (int)t >> s : (int)(t >> s);
       }
-      *(uint4*)dst[k] = make_uint4(o[0], o[1], o[2], o[3]);
+      if (OUT == 0) o[v] = pack4_sat(yv[0], yv[1], yv[2], yv[3], lo < 0);
+      else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) yv[j] = min(max(yv[j], lo), hi) & 0xFF;
+        o[v] = (unsigned)yv[0] | ((unsigned)yv[1] << 8) | ((unsigned)yv[2] << 16) | ((unsigned)yv[3] << 24);
+      }
     }
+    *(uint4*)dst = make_uint4(o[0], o[1], o[2], o[3]);
+  };
+  constexpr int KP = 4;                                           // eight in flight measured the same
+  while (px + (KP - 1) * step < a.pixels) {                      // whole groups: all reads first
+    uint4 r[KP];
+    const unsigned char* q = ip;
+#pragma unroll
+    for (int k = 0; k < KP; ++k) { r[k] = __ldg((const uint4*)q); q += istep; }
+    unsigned char* d = op;
+#pragma unroll
+    for (int k = 0; k < KP; ++k) { one(r[k], d); d += ostep; }
+    px += KP * step; ip = q; op = d;
   }
+  for (; px < a.pixels; px += step, ip += istep, op += ostep) one(__ldg((const uint4*)ip), op);
 }
 
 struct W4State {
