@@ -325,8 +325,8 @@ __device__ __forceinline__ void concat_w4_loop(W4State t, const int (&bb)[4], co
     else if (BITS == 8) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const unsigned sh = r.x >> (8 * j);
-        q[j] = SIGNED ? (int)(signed char)sh : (int)(sh & 0xFFu);
+        const unsigned sx = 8u | (unsigned)j;          // one byte permute, zero- or sign-extending
+        q[j] = (int)hq_prmt(r.x, 0u, SIGNED ? (sx << 12) | (sx << 8) | (sx << 4) | (unsigned)j : 0x4440u | (unsigned)j);
       }
     } else {
 #pragma unroll
@@ -370,11 +370,13 @@ __device__ __forceinline__ void concat_w4_loop(W4State t, const int (&bb)[4], co
   // whole groups of KP pixels: all reads first, then the arithmetic and the stores
   while (t.px + (KP - 1) * t.step < t.pixels) {
     uint4 raw[KP];
+    const unsigned char* q = t.ip;
 #pragma unroll
-    for (int p = 0; p < KP; ++p) raw[p] = fetch(t.ip + p * istep);
+    for (int p = 0; p < KP; ++p) { raw[p] = fetch(q); q += istep; }
+    unsigned char* d = t.op;
 #pragma unroll
-    for (int p = 0; p < KP; ++p) one(raw[p], t.op + p * ostep);
-    t.px += KP * t.step; t.ip += KP * istep; t.op += KP * ostep;
+    for (int p = 0; p < KP; ++p) { one(raw[p], d); d += ostep; }
+    t.px += KP * t.step; t.ip = q; t.op = d;
   }
   for (; t.px < t.pixels; t.px += t.step, t.ip += istep, t.op += ostep) one(fetch(t.ip), t.op);
 }
