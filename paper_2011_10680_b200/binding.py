@@ -21,7 +21,7 @@ HQ_OP = {"conv": 0, "linear": 1, "maxpool": 2, "avgpool": 3, "add": 4, "requant"
 EXPORTS = [
     "hq_create", "hq_destroy", "hq_sync", "hq_conv2d", "hq_linear", "hq_residual_add", "hq_avgpool_requant",
     "hq_maxpool", "hq_network_create", "hq_run_network", "hq_network_layer_bytes", "hq_network_launch_count",
-    "hq_network_destroy", "hq_set_conv_path", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
+    "hq_network_destroy", "hq_set_conv_path", "hq_set_tile_order", "hq_status_string", "hq_network_time_layers", "hq_conv2d_noalloc", "hq_expire_wait_selftest",
     "hq_network_check_guards", "hq_conv2d_noalloc_sync", "hq_mma_peak_launch",
     "hq_ilp_solve", "hq_concat_requant", "hq_sumpool",
 ]
@@ -90,6 +90,7 @@ def lib():
         L.hq_conv2d_noalloc_sync.argtypes = [vp]
         L.hq_mma_peak_launch.argtypes = [vp, i32, i32, C.POINTER(C.c_int64), vp]
         L.hq_set_conv_path.argtypes = [vp, i32]
+        L.hq_set_tile_order.argtypes = [vp, i32]
         L.hq_expire_wait_selftest.argtypes = [vp, i32, vp]
         L.hq_expire_wait_selftest.restype = i32
         i64p = C.POINTER(C.c_int64)
@@ -203,6 +204,9 @@ class Handle:
 
     def set_conv_path(self, path: int):
         _check(lib().hq_set_conv_path(self._h, path), "hq_set_conv_path")
+
+    def set_tile_order(self, order: int):
+        _check(lib().hq_set_tile_order(self._h, order), "hq_set_tile_order")
 
     def expire_wait_selftest(self, budget_ms: int) -> int:
         return lib().hq_expire_wait_selftest(self._h, budget_ms, _stream())

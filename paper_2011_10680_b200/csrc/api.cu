@@ -153,6 +153,7 @@ struct hq_network {
   std::vector<void*> narrow0, narrow1; // per ADD / REQUANT layer with 8-bit operands: narrow pairs of the two branches (owned)
   std::vector<void*> wgt_widened;    // per 4-bit conv layer on the tensor-core path: its weights, one byte per value (owned)
   std::vector<char> stored_wide;     // per layer: its 4-bit output is kept one value per byte (all consumers are such convs)
+  std::vector<char> tile_order;      // per conv / linear layer: pixel tiles walked from the last to the first (see plan_tile_orders)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
@@ -160,6 +161,24 @@ struct hq_network {
   struct CachedGraph { cudaGraphExec_t exec; const void* images; void* logits; };
   std::vector<CachedGraph> graphs;
 };
+
+// Order in which every convolution walks its pixel tiles.  At large batch a layer's tensors exceed the L2, which still
+// holds what the launch before wrote LAST; a consumer that starts at the same end reads that part without going to
+// HBM.  So a convolution runs opposite to the layer that produced its main input, except when the layer right after
+// it is an element-wise or pooling kernel reading its output (those always run first to last): then it runs last to
+// first for that kernel's sake.  The arithmetic does not depend on the order.
+static void plan_tile_orders(hq_network* net) {
+  const int n = (int)net->layers.size();
+  net->tile_order.assign(n, 0);
+  auto is_conv = [&](int i) { return net->layers[i].op == HQ_OP_CONV || net->layers[i].op == HQ_OP_LINEAR; };
+  for (int i = 0; i < n; ++i) {
+    if (!is_conv(i)) continue;
+    const int src = net->layers[i].in0;
+    char order = src < 0 ? 0 : is_conv(src) ? !net->tile_order[src] : 1;
+    if (i + 1 < n && !is_conv(i + 1) && net->layers[i + 1].in0 == i) order = 1;
+    net->tile_order[i] = order;
+  }
+}
 
 // Allocate `bytes` for layer `layer` of `net` between two guard bands; NULL when the device is out of memory.
 static void* net_alloc(hq_network* net, size_t bytes, int32_t layer) {
@@ -207,6 +226,7 @@ hq_status hq_create(int32_t device, hq_handle** out) {
   if (!h) return HQ_ERR_WORKSPACE;
   h->device = device;
   h->conv_path = 0;
+  h->tile_order = 0;
   h->sm_count = prop.multiProcessorCount;
   h->workspace = nullptr;
   h->workspace_bytes = 0;
@@ -232,6 +252,12 @@ hq_status hq_destroy(hq_handle* h) {
 hq_status hq_set_conv_path(hq_handle* h, int32_t path) {
   if (!h || path < 0 || path > 3) return HQ_ERR_INVALID_ARG;
   h->conv_path = path;
+  return HQ_OK;
+}
+
+hq_status hq_set_tile_order(hq_handle* h, int32_t order) {
+  if (!h || order < 0 || order > 1) return HQ_ERR_INVALID_ARG;
+  h->tile_order = order;
   return HQ_OK;
 }
 
@@ -518,6 +544,7 @@ hq_status hq_network_create(hq_handle* h, const hq_layer* table, int32_t n_layer
       if (hq_launch_residual_narrow(l.rescale1.b, l.rescale1.c, net->outs[l.in1].is_signed, ch, buf1, nullptr) != cudaSuccess) { st = HQ_ERR_CUDA; break; }
     }
   }
+  if (st == HQ_OK) plan_tile_orders(net);
   if (st == HQ_OK && cudaDeviceSynchronize() != cudaSuccess) st = HQ_ERR_CUDA;
   if (st != HQ_OK) { hq_network_destroy(net); return st; }
   *out = net;
@@ -545,8 +572,11 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
         d.residual = nullptr;
         if (l.op == HQ_OP_CONV && l.in1 >= 0) { res = net->outs[l.in1]; d.residual = &res; }
         if (in_wide) { d.w_bits = 8; d.w = net->wgt_widened[i]; }
+        const int32_t callers_order = h->tile_order;
+        h->tile_order = net->tile_order[i];
         if (l.op == HQ_OP_LINEAR) { in.c = in.h * in.w * in.c; in.h = 1; in.w = 1; st = hq_linear(h, &in, &d, &o, s); }
         else st = conv_common(h, &in, &d, &o, s, net->scratch, net->scratch_bytes, net->res_narrow[i], in_wide ? nullptr : net->wgt_widened[i]);
+        h->tile_order = callers_order;
         break;
       }
       case HQ_OP_MAXPOOL: st = hq_maxpool(h, &in, l.pool_k, l.pool_stride, l.pool_pad, &o, s); break;

@@ -77,6 +77,8 @@ struct TcParams {
   int32_t k_blocks;      // kh * kw * cchunks
   int32_t pt;            // pixel tile = MMA N: 64, 128 or 256
   int32_t p_tiles, c_tiles, stages;
+  int32_t rev;           // 1: a CTA's t-th pixel tile is tile p_tiles - 1 - t: the layer walks its tensors from the end, so
+                         //    that it reads first what the kernel before it wrote last (still in the L2)
   int32_t wres;          // 1: the CTA's whole weight slab [k_blocks][128][bkb] is loaded once and stays in shared memory
   uint32_t wres_off;     // its offset from the 1024-aligned dynamic base
   int32_t fold;          // 1: at most 64 output channels: W rows loaded twice, lane quarters 2-3 share the pixel columns
@@ -430,6 +432,9 @@ __device__ __forceinline__ int requant_fast(int acc, int r, const ChanConst& k) 
   return s;
 }
 
+// Pixel tile behind position `t` of the tile order (see TcParams::rev).
+__device__ __forceinline__ int tile_at(const TcParams& p, int t) { return p.rev ? p.p_tiles - 1 - t : t; }
+
 // The finished staging box of one warp leaves for global memory.  Dense tiles: one [columns][32 B] box at pixel
 // `p_tile * pt + col0`.  Strip tiles: one box per 32 positions (a row, half a row or two rows of the pitch-2^lg_wp
 // raster); columns at or beyond the image width and rows at or beyond its height fall outside the tensor map
@@ -584,7 +589,7 @@ __device__ __forceinline__ void epilogue_loop_fast8(const EpiCtx& e_in, const Ch
     }
     fence_async_smem();                           // make this lane's box writes visible to the TMA engine
     __syncwarp();
-    if (lane == 0 && e.warp_live) store_warp_box(p, e.map_out, my_stage, (e.c_tile * kTileC + cq * 32) >> (OUT4 ? 1 : 0), p_tile, col0, px_per_warp);
+    if (lane == 0 && e.warp_live) store_warp_box(p, e.map_out, my_stage, (e.c_tile * kTileC + cq * 32) >> (OUT4 ? 1 : 0), tile_at(p, p_tile), col0, px_per_warp);
     if (!has_next || !ok) break;
     p_tile += tile_step; ++tcount; as = nas; aph = naph;
   }
@@ -777,7 +782,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
       w = __shfl_sync(0xffffffffu, w, 0);
       if (!w) break;
       tc_fence_after();                            // lane 0 observed the barriers; the shuffle ordered the warp
-      const int p_base = p_tile * p.pt + col0;                          // first pixel of this warp's columns
+      const int p_base = tile_at(p, p_tile) * p.pt + col0;              // first pixel of this warp's columns
       const uint8_t* const res_tile = res_stage_ptr + rs * res_tile_bytes + (uint32_t)col0 * kTileC + cq * 32 + lane;
 
       for (int cc0 = 0; cc0 < px_per_warp; cc0 += 32) {
@@ -885,7 +890,7 @@ __device__ __noinline__ void epilogue_loop_general(const EpiCtx& e, const ChanCo
         release_accumulator(p, ctl, as);
         if (p.staged_res) mbar_arrive(smem_u32(&ctl.rempty[rs]));
         if (staged_out && warp_live)
-          store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, p_tile, col0, px_per_warp);
+          store_warp_box(p, &map_out, my_stage, ((c_tile * kTileC + cq * 32) * p.out_bits) >> 3, tile_at(p, p_tile), col0, px_per_warp);
       }
     }
 
@@ -979,9 +984,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const int ho = p.howo / p.wo;
       // (duo: this CTA fetches the half of the tile's pixel rows that starts at half_off)
       const int half_off = p.duo ? (int)rank * (p.pt >> 1) : 0;
-      int img = (p_tile0 * p.pt + half_off) / p.howo;
-      int oh = ((p_tile0 * p.pt + half_off) - img * p.howo) / p.wo;
-      int ow = (p_tile0 * p.pt + half_off) - img * p.howo - oh * p.wo;
+      const int px_first = tile_at(p, p_tile0) * p.pt + half_off;
+      int img = px_first / p.howo;
+      int oh = (px_first - img * p.howo) / p.wo;
+      int ow = px_first - img * p.howo - oh * p.wo;
       const int step = p_step * p.pt;
       const int d_img = step / p.howo, d_oh = (step - d_img * p.howo) / p.wo, d_ow = step - d_img * p.howo - d_oh * p.wo;
       if (p.wres) {              // the channel tile's weights for every K block, once
@@ -1005,7 +1011,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (p.strip) {
         uint32_t ps = 0, pph = 0;
         for (int p_tile = p_tile0; p_tile < p.p_tiles && ok; p_tile += p_step, ++tcount) {
-          const int img_s = p_tile / p.tpi, y0 = (p_tile - img_s * p.tpi) * p.rows;
+          const int t_act = tile_at(p, p_tile);
+          const int img_s = t_act / p.tpi, y0 = (t_act - img_s * p.tpi) * p.rows;
           for (int chunk = 0; chunk < p.cchunks && ok; ++chunk) {
             // the padded patch of this cin chunk: columns -1 .. 2^lg_wp - 2, rows y0-1 .. y0+rows+1 (zeros outside the image)
             if (!mbar_wait(smem_u32(&ctl.pempty[ps]), pph ^ 1u, &ctl, p.status, HQ_DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
@@ -1033,11 +1040,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
       }
       for (int p_tile = p_tile0; p_tile < p.p_tiles && ok && !p.strip; p_tile += p_step, ++tcount) {
-        const int p0 = p_tile * p.pt;
+        const int p0 = tile_at(p, p_tile) * p.pt;
         const int cw = ow * p.stride - p.pad, chh = oh * p.stride - p.pad, img_now = img;
-        ow += d_ow; if (ow >= p.wo) { ow -= p.wo; ++oh; }
-        oh += d_oh; if (oh >= ho) { oh -= ho; ++img; }
-        img += d_img;
+        if (!p.rev) {
+          ow += d_ow; if (ow >= p.wo) { ow -= p.wo; ++oh; }
+          oh += d_oh; if (oh >= ho) { oh -= ho; ++img; }
+          img += d_img;
+        } else {                                     // the same step backwards, with borrows (unused after the last tile)
+          ow -= d_ow; if (ow < 0) { ow += p.wo; --oh; }
+          oh -= d_oh; if (oh < 0) { oh += ho; --img; }
+          img -= d_img;
+        }
         int chunk = 0, tap_s = 0, tap_r = 0;
         // The residual tile of this output tile is fetched as soon as its buffer is free, but this thread only
         // blocks for the buffer after the tile's last operand block is on its way: the buffer comes back when the
@@ -1279,7 +1292,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       for (int p_tile = p_tile0; p_tile < p.p_tiles; p_tile += p_step, ++tcount) {
         const uint32_t rs = tcount & rmask, rph = (tcount >> p.lg_rbufs) & 1u;
         if (!mbar_wait(smem_u32(&ctl.ofull[rs]), rph, &ctl, p.status, HQ_DEV_TIMEOUT_EPILOGUE)) break;
-        tma_store_2d(&map_out, res_stage + rs * res_tile_bytes, c_tile * kTileC, p_tile * p.pt);
+        tma_store_2d(&map_out, res_stage + rs * res_tile_bytes, c_tile * kTileC, tile_at(p, p_tile) * p.pt);
         tma_store_commit();
         if (rmask < 3u) {
           // only two tile buffers: hand this one back as soon as the store has read it
@@ -1577,6 +1590,7 @@ hq_status hq_launch_conv_tc(hq_handle* h, const ConvArgs& a, cudaStream_t stream
   if (P == 0) return HQ_OK;
 
   TcParams p{};
+  p.rev = h->tile_order ? 1 : 0;
   p.P = (int32_t)P; p.C = a.cout; p.howo = a.ho * a.wo; p.wo = a.wo;
   p.stride = a.stride; p.pad = a.pad; p.kw = a.kw;
   p.bkb = (a.cin % 128 == 0) ? 128 : (a.cin % 64 == 0) ? 64 : 32;

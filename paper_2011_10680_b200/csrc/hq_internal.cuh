@@ -24,6 +24,7 @@ struct hq_handle {
   void* workspace;            // scratch owned by the handle (grown on demand, never inside a capture)
   size_t workspace_bytes;
   void* narrow_pairs;         // 2 x kNarrowChannels x 16 bytes: narrow pairs of a single element-wise call's two operands
+  int32_t tile_order;         // tensor-core convolutions walk their pixel tiles 0: first to last, 1: last to first
 };
 constexpr int kNarrowChannels = 4096;
 
@@ -34,7 +35,6 @@ __device__ __forceinline__ long long hq_dn(int q, int b, int c) {
   return ((long long)q * (long long)b + (1LL << (c - 1))) >> c;
 }
 
-// Element access for dense tensors with 4, 8 or 32 bits per element (even element = low nibble).
 // Byte permute with the full PTX selector: bit 3 of a selector nibble replicates the selected byte's sign bit over the
 // target byte.  (The __byte_perm intrinsic keeps three bits per nibble and cannot sign-extend.)
 __device__ __forceinline__ unsigned hq_prmt(unsigned a, unsigned b, unsigned sel) {
@@ -43,6 +43,7 @@ __device__ __forceinline__ unsigned hq_prmt(unsigned a, unsigned b, unsigned sel
   return d;
 }
 
+// Element access for dense tensors with 4, 8 or 32 bits per element (even element = low nibble).
 __device__ __forceinline__ int hq_load_elem(const void* base, long long idx, int bits, int is_signed) {
   if (bits == 32) return ((const int*)base)[idx];
   if (bits == 8) return is_signed ? (int)((const signed char*)base)[idx] : (int)((const unsigned char*)base)[idx];

@@ -87,11 +87,21 @@ def _random_conv_configs(count, seed):
     return out
 
 
+@pytest.mark.parametrize("order", [0, 1])
 @pytest.mark.parametrize("path", [0, 3])
-def test_conv_random_configurations(hq, path):
+def test_conv_random_configurations(hq, path, order):
     """48 seeded random layers through hq_conv2d on the automatic path and with the tensor-core launch shapes chosen by
     what a layer allows rather than by its size: every dispatch branch (direct, lowered, widened, first-layer form,
-    CUDA cores) must return the oracle's integers."""
+    CUDA cores) must return the oracle's integers, whichever end of the tensor the pixel tiles start from."""
+    from paper_2011_10680_b200 import binding
+    hq.set_tile_order(order)
+    try:
+        _random_configurations_body(hq, path)
+    finally:
+        hq.set_tile_order(0)
+
+
+def _random_configurations_body(hq, path):
     from paper_2011_10680_b200 import binding
     for i, cfg in enumerate(_random_conv_configs(48, 20260 + path)):
         case = inputs.conv_case(7000 + i, cfg["n"], cfg["h"], cfg["w"], cfg["cin"], cfg["cout"], cfg["k"], cfg["stride"],
@@ -129,18 +139,20 @@ def test_conv_random_midsize_layers_reach_every_launch_shape(hq):
         residual = bool(g.integers(0, 2))
         case = inputs.conv_case(7100 + i, n, hw, hw, cin, cout, k, 1, k // 2, bits=bits, residual=residual,
                                 in_signed=bool(g.integers(0, 2)), c_range=(lo, lo + 6))
-        for path in (0, 3):
+        for path, order in ((0, 0), (3, 0), (0, 1), (3, 1)):         # order 1: pixel tiles from the last to the first
             hq.set_conv_path(path)
+            hq.set_tile_order(order)
             try:
                 st, out = hq.conv_case(case)
                 assert st == binding.HQ_OK, (i, path, binding.status_string(st))
                 hq.sync()
             finally:
                 hq.set_conv_path(0)
-            if path == 0:
+                hq.set_tile_order(0)
+            if path == 0 and order == 0:
                 ref = oracle().conv_case(case)
             got = host(out, ref)
-            assert np.array_equal(got, ref), (i, path, hw, n, cin, cout, k, bits, residual, int((got != ref).sum()))
+            assert np.array_equal(got, ref), (i, path, order, hw, n, cin, cout, k, bits, residual, int((got != ref).sum()))
             del out
         binding.check_guards()
 
