@@ -186,6 +186,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+// The same copy with an L2 eviction priority.  Activations and residual tiles that a layer reads exactly once per
+// channel tile are fetched "evict first": they then make room before the output lines the layer is writing, and the
+// next layer (which starts at the end this one wrote last, see TcParams::rev) finds more of its input in the L2.
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 unsigned long long pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                                 int c, int w, int h, int n, uint16_t off_w, uint16_t off_h) {
   asm volatile(
@@ -1007,6 +1021,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       // immediately before this one (the helper kernels that prepare weights are always followed by another launch).
       // Everything below reads activations, which the previous kernel may still be writing.
       asm volatile("griddepcontrol.wait;" ::: "memory");
+      const unsigned long long pol_first = policy_evict_first();
       uint32_t pit = 0;                                // strip mode: patches started
       if (p.strip) {
         uint32_t ps = 0, pph = 0;
@@ -1065,7 +1080,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           }
           const uint32_t bar = smem_u32(&ctl.rfull[rbuf]);
           mbar_expect_tx(bar, res_tile_bytes);
-          tma_load_2d(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0);
+          tma_load_2d_hint(res_stage + rbuf * res_tile_bytes, &map_res, bar, c_tile * kTileC, p0, pol_first);
           res_due = false;
           return true;
         };
@@ -1088,7 +1103,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           }
           mbar_expect_tx(bar, stage_bytes);
           if (p.x_tiled) {
-            tma_load_2d(w_dst + x_off, &map_x, bar, chunk * p.bkb, p0);
+            tma_load_2d_hint(w_dst + x_off, &map_x, bar, chunk * p.bkb, p0, pol_first);
           } else {
             tma_load_im2col(w_dst + x_off, &map_x, bar, chunk * p.bkb, cw, chh, img_now, (uint16_t)tap_s, (uint16_t)tap_r);
           }
