@@ -262,8 +262,8 @@ hq_status hq_conv2d_noalloc_sync(void* stream);
  * then reach the shapes of large layers). */
 hq_status hq_set_conv_path(hq_handle* h, int32_t path);
 
-/* Order in which the tensor-core convolutions of this handle walk their pixel tiles: 0 = from the first output pixel
- * to the last (default), 1 = from the last to the first.  The results are identical; the order only decides which
+/* Order in which the tensor-core convolutions (pixel tiles) and hq_concat_requant (pixels) of this handle walk their
+ * tensors: 0 = from the first output pixel to the last (default), 1 = from the last to the first.  The results are identical; the order only decides which
  * end of a large tensor is touched first, and with it what a layer finds in the L2 of what the call before it wrote
  * (a network chooses the order layer by layer itself and ignores this setting).  (No counterpart in the paper.) */
 hq_status hq_set_tile_order(hq_handle* h, int32_t order);

@@ -153,7 +153,7 @@ struct hq_network {
   std::vector<void*> narrow0, narrow1; // per ADD / REQUANT layer with 8-bit operands: narrow pairs of the two branches (owned)
   std::vector<void*> wgt_widened;    // per 4-bit conv layer on the tensor-core path: its weights, one byte per value (owned)
   std::vector<char> stored_wide;     // per layer: its 4-bit output is kept one value per byte (all consumers are such convs)
-  std::vector<char> tile_order;      // per conv / linear layer: pixel tiles walked from the last to the first (see plan_tile_orders)
+  std::vector<char> tile_order;      // per conv / linear / concat layer: tensors walked from the last pixel to the first (see plan_tile_orders)
   void* scratch;                     // patch matrix of the lowered first layer (owned)
   size_t scratch_bytes;
   // graph cache: one instantiated graph per (images, logits) pointer pair, a few pairs kept so
@@ -162,20 +162,27 @@ struct hq_network {
   std::vector<CachedGraph> graphs;
 };
 
-// Order in which every convolution walks its pixel tiles.  At large batch a layer's tensors exceed the L2, which still
-// holds what the launch before wrote LAST; a consumer that starts at the same end reads that part without going to
-// HBM.  So a convolution runs opposite to the layer that produced its main input, except when the layer right after
-// it is an element-wise or pooling kernel reading its output (those always run first to last): then it runs last to
-// first for that kernel's sake.  The arithmetic does not depend on the order.
+// Order in which every convolution (and concatenation) walks its tensors.  At large batch a layer's tensors exceed the
+// L2, which still holds what the launch before wrote LAST; a consumer that starts at the same end reads that part
+// without going to HBM.  So a convolution runs opposite to the layer that produced its main input, except when the
+// layer right after it is an element-wise or pooling kernel reading its output (those always run first to last): then
+// it runs last to first for that kernel's sake.  A concatenation runs opposite to the launch right before it (the
+// pooling branch's window sums in an Inception module).  The arithmetic does not depend on the order.
 static void plan_tile_orders(hq_network* net) {
   const int n = (int)net->layers.size();
   net->tile_order.assign(n, 0);
   auto is_conv = [&](int i) { return net->layers[i].op == HQ_OP_CONV || net->layers[i].op == HQ_OP_LINEAR; };
+  auto either_way = [&](int i) { return is_conv(i) || net->layers[i].op == HQ_OP_CONCAT; };
   for (int i = 0; i < n; ++i) {
-    if (!is_conv(i)) continue;
-    const int src = net->layers[i].in0;
-    char order = src < 0 ? 0 : is_conv(src) ? !net->tile_order[src] : 1;
-    if (i + 1 < n && !is_conv(i + 1) && net->layers[i + 1].in0 == i) order = 1;
+    if (!either_way(i)) continue;
+    char order;
+    if (!is_conv(i)) {
+      order = i > 0 ? !net->tile_order[i - 1] : 0;
+    } else {
+      const int src = net->layers[i].in0;
+      order = src < 0 ? 0 : !net->tile_order[src];
+    }
+    if (i + 1 < n && !either_way(i + 1) && net->layers[i + 1].in0 == i) order = 1;
     net->tile_order[i] = order;
   }
 }
@@ -596,7 +603,10 @@ static hq_status run_layers(hq_network* net, const hq_tensor* images, hq_tensor*
       case HQ_OP_CONCAT: {
         hq_tensor br[HQ_CONCAT_MAX_BRANCHES];
         for (int k = 0; k < l.n_in; ++k) br[k] = net->outs[l.ins[k]];
+        const int32_t callers_order = h->tile_order;
+        h->tile_order = net->tile_order[i];
         st = hq_concat_requant(h, l.n_in, br, l.rescales, l.relu, l.qmin, l.qmax, &o, s);
+        h->tile_order = callers_order;
         break;
       }
       default: return HQ_ERR_INVALID_ARG;

@@ -32,6 +32,7 @@ struct ConcatArgs {
   void* out;
   const int4* narrow;   // per OUTPUT channel {m, a, s, valid} from concat_narrow_kernel (8-/4-bit branches), or NULL
   int32_t sat;          // 1: relu and the clamp bounds equal a saturating conversion to the 8-bit output type
+  int32_t rev;          // 1: pixels are walked from the last to the first (the handle's tile order): same results
 };
 
 // Narrow multiply-add pairs for the 8- and 4-bit branches.  A stored 8-bit value r has 256 possible values, so
@@ -195,7 +196,7 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
       for (int p = 0; p < kPix; ++p) {
         const long long px = px0 + p * step;
         if (px < a.pixels) {
-          const long long e0 = px * (long long)ch + k0;
+          const long long e0 = (a.rev ? a.pixels - 1 - px : px) * (long long)ch + k0;
           if (bits == 4) { const uint2 t = *(const uint2*)((const unsigned char*)in + (e0 >> 1)); raw[p].x = t.x; raw[p].y = t.y; }
           else raw[p] = *(const uint4*)((const unsigned char*)in + e0 * (bits >> 3));
         }
@@ -203,8 +204,9 @@ __device__ __forceinline__ void concat_branch(const ConcatArgs& a, const int i) 
     }
 #pragma unroll 1
     for (int p = 0; p < kPix; ++p) {                 // one copy of the arithmetic: the instruction stream stays small
-      const long long px = px0 + p * step;
-      if (px >= a.pixels) break;
+      const long long pxl = px0 + p * step;
+      if (pxl >= a.pixels) break;
+      const long long px = a.rev ? a.pixels - 1 - pxl : pxl;
       int q[N];
       if (vec) {
         uint4 r = raw[0];
@@ -267,9 +269,11 @@ __device__ __forceinline__ void concat_uniform8(const ConcatArgs& a, const int i
   const int u = tid % P, y = tid / P;
   const long long step = (long long)B.nblocks * ppb;
   long long px = (long long)((int)blockIdx.x - B.block0) * ppb + y;
-  const long long istep = step * B.row_ch, ostep = step * a.out_ch;
-  const unsigned char* ip = (const unsigned char*)B.in + px * B.row_ch + u * 16;
-  unsigned char* op = (unsigned char*)a.out + px * a.out_ch + B.ch_off + u * 16;
+  // (px counts positions of the walk; position t is pixel t, or pixel pixels - 1 - t when walking backwards)
+  const long long px_at = a.rev ? a.pixels - 1 - px : px, dir = a.rev ? -1 : 1;
+  const long long istep = dir * step * B.row_ch, ostep = dir * step * a.out_ch;
+  const unsigned char* ip = (const unsigned char*)B.in + px_at * B.row_ch + u * 16;
+  unsigned char* op = (unsigned char*)a.out + px_at * a.out_ch + B.ch_off + u * 16;
   auto one = [&](const uint4 r, unsigned char* dst) {
     const unsigned w[4] = {r.x, r.y, r.z, r.w};
     unsigned o[4];
@@ -309,7 +313,7 @@ __device__ __forceinline__ void concat_uniform8(const ConcatArgs& a, const int i
 
 struct W4State {
   const unsigned char* ip; unsigned char* op;
-  long long px, step, in_row, out_row, pixels;
+  long long px, step, in_row, out_row, pixels, dir;
   int lo, hi; bool word_out;
 };
 
@@ -318,7 +322,7 @@ struct W4State {
 template <int BITS, bool SIGNED, int MODE, int OUT>
 __device__ __forceinline__ void concat_w4_loop(W4State t, const int (&bb)[4], const int (&hh)[4], const int (&ss)[4]) {
   constexpr int KP = BITS == 32 ? 4 : 8;
-  const long long istep = t.step * t.in_row, ostep = t.step * t.out_row;
+  const long long istep = t.dir * t.step * t.in_row, ostep = t.dir * t.step * t.out_row;
   auto one = [&](const uint4 r, unsigned char* o_ptr) {
     int q[4];
     if (BITS == 32) { q[0] = (int)r.x; q[1] = (int)r.y; q[2] = (int)r.z; q[3] = (int)r.w; }
@@ -434,8 +438,10 @@ __device__ __forceinline__ void concat_w4(const ConcatArgs& a, const int i) {
   t.step = (long long)a.br[i].nblocks * ppb;
   t.px = (long long)(blockIdx.x - a.br[i].block0) * ppb + y;
   t.in_row = (long long)a.br[i].row_ch * BITS / 8; t.out_row = (long long)a.out_ch * a.out_bits / 8;
-  t.ip = (const unsigned char*)a.br[i].in + t.px * t.in_row + (long long)k0 * BITS / 8;
-  t.op = (unsigned char*)a.out + t.px * t.out_row + (long long)off * a.out_bits / 8;
+  const long long px_at = a.rev ? a.pixels - 1 - t.px : t.px;      // t.px counts positions of the walk
+  t.ip = (const unsigned char*)a.br[i].in + px_at * t.in_row + (long long)k0 * BITS / 8;
+  t.op = (unsigned char*)a.out + px_at * t.out_row + (long long)off * a.out_bits / 8;
+  t.dir = a.rev ? -1 : 1;
   t.lo = lo; t.hi = hi; t.pixels = a.pixels;
   t.word_out = (off & 3) == 0 && (a.out_ch & 3) == 0;      // the thread's outputs are one aligned word / halfword
   // one straight-line loop per signedness, form of the arithmetic and output type, chosen once
@@ -529,6 +535,7 @@ extern "C" hq_status hq_concat_requant(hq_handle* h, int32_t n_branches, const h
   if (off != out->c) return HQ_ERR_INVALID_ARG;
   a.n_br = nb; a.out_ch = out->c; a.out_bits = out->bits;
   a.relu = relu; a.qmin = qmin; a.qmax = qmax;
+  a.rev = h->tile_order ? 1 : 0;
   a.pixels = (long long)out->n * out->h * out->w;
   a.out = out->data;
   if (a.pixels == 0) return HQ_OK;

@@ -53,6 +53,11 @@ TOO_MANY_PIECES = [(8, 8, 0)] * 6 + [(3080, 8, 0), (16, 32, 1)]            # no 
 def test_concat_matches_the_oracle(hq, branches, n, hw, out_bits, out_signed, relu):
     case = inputs.concat_case(401, n, hw, branches, out_bits, out_signed, relu)
     ref = run_and_compare(hq, case)
+    hq.set_tile_order(1)                     # the same pixels walked from the last to the first
+    try:
+        run_and_compare(hq, case)
+    finally:
+        hq.set_tile_order(0)
     if branches is INCEPTION_A and out_bits == 8:
         # the draw must exercise the arithmetic: not everything saturated
         inner = np.count_nonzero((ref > case["qmin"]) & (ref < case["qmax"]))
@@ -81,6 +86,11 @@ def test_concat_large_call_with_narrow_pairs(hq):
         case = {"branches": branches, "relu": relu, "qmin": lo, "qmax": hi, "out_bits": out_bits, "out_signed": out_signed,
                 "n": n, "hw": hw, "out_ch": 288}
         run_and_compare(hq, case)
+        hq.set_tile_order(1)
+        try:
+            run_and_compare(hq, case)
+        finally:
+            hq.set_tile_order(0)
 
 
 def _uniform_branch(g, n, hw, ch, bits, signed, b, c, uniform=True):
@@ -133,6 +143,11 @@ def test_concat_branches_with_one_pair_per_branch(hq, layout):
         ref = run_and_compare(hq, case)
         inner = np.count_nonzero((ref > lo) & (ref < hi))
         assert inner > ref.size // 8
+        hq.set_tile_order(1)
+        try:
+            run_and_compare(hq, case)
+        finally:
+            hq.set_tile_order(0)
     # a pair whose shift has no narrow form (c = 40) and one whose term is always zero (c = 45)
     for c in (40, 45):
         odd = [_uniform_branch(g, n, hw, ch, bits, signed, (1 << 31) - 7, c if bits == 8 else 46, True)
