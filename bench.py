@@ -795,7 +795,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                          "frac": achieved / hbm_peak,
                          "traffic": traffic_per_launch,
-                         "traffic_note": (f"avg DRAM bytes per conv launch: ncu capture at batch {traffic['batch']} "
+                         "traffic_note": (f"avg DRAM bytes per conv launch: ncu capture at batch {traffic['batch']}, caches left alone "
                                           f"({os.path.basename(TRAFFIC_JSON)}), scaled by images") if traffic_per_launch else None,
                          "algorithmic_bytes_per_launch": tc_bytes / max(n_conv_tc, 1),
                          "peak_kind": f"of {peak_kind}",
