@@ -113,7 +113,7 @@ def test_concat_branches_with_one_pair_per_branch(hq, layout):
     in 16-byte pieces.  Cases: the two module shapes, signed operands beside unsigned ones, a branch that is uniform
     except for its last channel (must stay on the per-channel form), a branch wider than 1024 channels entered in
     pieces, an output offset that is not a multiple of sixteen (per-channel form), and pixel counts that leave a
-    ragged last round; each with the saturating and the explicit clamp and a signed output."""
+    ragged last group of pixels; each with the saturating and the explicit clamp and a signed output."""
     g = inputs.rng(411)
     pair = lambda lo_c, hi_c: (int(g.integers(1 << 30, 1 << 31)), int(g.integers(lo_c, hi_c)))
     if layout == "module_35":
